@@ -1,0 +1,167 @@
+/*
+ * qmm.h -- C ABI of libqmm: fused dequantise-and-multiply of block-quantised
+ * weights (Q4 / Q8, 32-element blocks along K, one fp16 scale per block) by
+ * fp16 activations, for NVIDIA B200 (sm_100a) only.
+ *
+ * The operations follow the paper's statement of the problem: weights stay in
+ * their quantised storage format and are dequantised inside the inner loop of
+ * the product instead of being materialised (Sec. 3.3); decode is the M = 1
+ * matrix-vector product, prefill the same product on [seq_len x dim]
+ * activations (Sec. 3.3, Sec. 3.4); the runtime is reached through a C API,
+ * allocates nothing on the hot path and reports errors through a static
+ * thread-local buffer (Sec. 3, Sec. 3.2).  The paper gives no block layout, no
+ * quantisation formula and no mixture-of-experts algorithm; those conventions
+ * are stated here.
+ *
+ * Conventions for every call
+ *   - W is [N, K]: N output features, K input features.  y = W x, Y = X W^T.
+ *   - "device" pointers are CUDA device allocations owned by the caller on the
+ *     current device; "host" pointers are ordinary host memory.  The library
+ *     never allocates or frees device memory and never keeps a pointer after
+ *     the call's work has run.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     Calls only enqueue work on it and return; they do not synchronise
+ *     (qmm_status_check is the exception).
+ *   - Arguments are checked on the host before anything is launched.  On
+ *     failure nothing is enqueued, a qmm_status other than QMM_OK is returned
+ *     and qmm_last_error() describes the problem.
+ *   - Supported shapes: K a multiple of 256, N a multiple of 128, M >= 1
+ *     (M = 0 / T = 0 is accepted and does nothing).  Other shapes return
+ *     QMM_ERR_UNSUPPORTED.  There is no CPU fallback and no other GPU target.
+ *   - Device pointers must be 16-byte aligned.
+ *
+ * Canonical block format (what qmm_pack reads)
+ *   Q4 block, 18 bytes: uint16 d (fp16 bits, little endian), uint8 qs[16];
+ *     element i of the block has code q_i in [-8, 7] stored as u_i = q_i + 8,
+ *     qs[j] = u_{2j} | (u_{2j+1} << 4).
+ *   Q8 block, 34 bytes: uint16 d, int8 qs[32] (two's complement).
+ *   Row n of W holds K/32 consecutive blocks; rows are consecutive; block b of
+ *   row n covers k in [32 b, 32 b + 32).  Weight value: float(d) * q (exact in
+ *   fp32).  Scales must be finite.
+ */
+#ifndef QMM_H
+#define QMM_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    QMM_OK = 0,
+    QMM_ERR_INVALID_ARG = 1,   /* null pointer, unknown format, negative size           */
+    QMM_ERR_SHAPE = 2,         /* K % 32 != 0, ld < row length, topk > E, ...           */
+    QMM_ERR_ALIGNMENT = 3,     /* a device pointer or leading dimension is misaligned   */
+    QMM_ERR_WORKSPACE = 4,     /* workspace missing or smaller than *_workspace_bytes   */
+    QMM_ERR_UNSUPPORTED = 5,   /* valid problem outside what the kernels cover          */
+    QMM_ERR_CUDA = 6,          /* a CUDA runtime/driver call failed (message has it)    */
+    QMM_ERR_DEVICE_TIMEOUT = 7 /* a bounded wait inside a kernel gave up                */
+} qmm_status;
+
+typedef enum { QMM_Q4 = 4, QMM_Q8 = 8 } qmm_format;
+
+/* Description of the last failure on the calling thread.  Points into a static
+ * thread-local buffer (Sec. 3.2: error handling without allocation); never
+ * NULL; valid until the next failing call on the same thread.               */
+const char* qmm_last_error(void);
+
+/* Library version, major * 10000 + minor * 100 + patch.                     */
+int qmm_version(void);
+
+/* Bytes of the canonical block stream for W[N,K]: N * (K/32) * 18 (Q4) or
+ * * 34 (Q8).  0 if the arguments are invalid.                               */
+size_t qmm_canonical_bytes(qmm_format fmt, int64_t N, int64_t K);
+
+/* Bytes of the device layout produced by qmm_pack (opaque, position
+ * independent, copyable with cudaMemcpy; packed buffers of matrices with the
+ * same K may be concatenated to form the packed buffer of the row-wise
+ * concatenated matrix).  0 if the arguments are invalid or unsupported.     */
+size_t qmm_packed_bytes(qmm_format fmt, int64_t N, int64_t K);
+
+/* Repack canonical blocks into the device layout (the analogue of the paper's
+ * offline conversion into its native weight format, Sec. 3 / Sec. 4.1).  Off
+ * the hot path; integer and bit moves only.
+ *   canonical  device, qmm_canonical_bytes(fmt,N,K) bytes, read only
+ *   packed     device, qmm_packed_bytes(fmt,N,K) bytes, written            */
+qmm_status qmm_pack(qmm_format fmt, const void* canonical, int64_t N, int64_t K,
+                    void* packed, void* stream);
+
+/* Validation aid: device layout -> fp32 W[N,K] row-major, w = float(d) * q.
+ *   packed  device, read only;  w_out  device, N*K floats, written.        */
+qmm_status qmm_dequant(qmm_format fmt, const void* packed, int64_t N, int64_t K,
+                       float* w_out, void* stream);
+
+/* Decode matrix-vector product (Sec. 3.3, "GEMV (decode, M=1)"):
+ *   y[n] = fp16( sum_b float(d[n,b]) * sum_{i<32} q[n,b,i] * x[32 b + i] ),
+ * accumulated in fp32.  When N is too small to occupy the GPU the K range is
+ * split across thread blocks, fp32 partial sums go to the workspace and a
+ * second stage adds them in a fixed order.
+ *   packed    device, from qmm_pack, read only
+ *   x_fp16    device, K fp16 values (bit patterns), read only
+ *   y_fp16    device, N fp16 values, written
+ *   ws        device, at least qmm_gemv_workspace_bytes(fmt,N,K) bytes; may be
+ *             NULL when that size is 0.  Contents are scratch.              */
+size_t qmm_gemv_workspace_bytes(qmm_format fmt, int64_t N, int64_t K);
+qmm_status qmm_gemv(qmm_format fmt, const void* packed, int64_t N, int64_t K,
+                    const uint16_t* x_fp16, uint16_t* y_fp16,
+                    void* ws, size_t ws_bytes, void* stream);
+
+/* Prefill matrix-matrix product (Sec. 3.3 "GEMM (prefill, M>1)", Sec. 3.4):
+ *   Y[m,n] = fp16( sum_k w[n,k] * X[m,k] ), fp32 accumulation on the tensor
+ * cores; weights enter the contraction as fp16(float(d) * q).
+ *   X_fp16  device, [M, ldx] fp16 row-major, ldx >= K, ldx % 8 == 0
+ *   Y_fp16  device, [M, ldy] fp16 row-major, ldy >= N, ldy % 8 == 0, written
+ *   ws      device, at least qmm_gemm_workspace_bytes(...) bytes            */
+size_t qmm_gemm_workspace_bytes(qmm_format fmt, int64_t M, int64_t N, int64_t K);
+qmm_status qmm_gemm(qmm_format fmt, const void* packed, int64_t N, int64_t K,
+                    const uint16_t* X_fp16, int64_t ldx,
+                    uint16_t* Y_fp16, int64_t ldy, int64_t M,
+                    void* ws, size_t ws_bytes, void* stream);
+
+/* Top-k mixture-of-experts feed-forward layer.  The paper names
+ * mixture-of-experts models as the case with its largest prefill gains
+ * (Sec. 4.3) but gives no algorithm; this library defines it as
+ *   1. routing: per token the topk largest router logits, larger first, equal
+ *      logits -> lower expert index first; weights = softmax over the selected
+ *      logits (fp32);
+ *   2. permutation: the T*topk (token, slot) pairs sorted by (expert, token);
+ *      perm[r] = t*topk + j, expert_offsets[e] = first sorted row of expert e;
+ *   3. per expert e on its rows: G = X Wgate_e^T, U = X Wup_e^T,
+ *      Hm = fp16(silu(G) * U) with silu(g) = g / (1 + exp(-g));
+ *   4. D = fp16(Hm Wdown_e^T);
+ *   5. out[t,:] = fp16( sum_{j<topk} p[t,j] * D[row(t,j),:] ), fp32, j ascending.
+ * All pointers are device pointers.                                          */
+typedef struct {
+    int32_t T, H, I, E, topk;      /* tokens, hidden, expert intermediate, experts, k   */
+    int32_t fmt;                   /* qmm_format of all expert matrices                 */
+    const float* logits;           /* [T,E] fp32, finite, read only                     */
+    const uint16_t* X;             /* [T,H] fp16, read only                             */
+    const void* w_gate;            /* E packed [I,H] matrices, stride packed_bytes(I,H) */
+    const void* w_up;              /* same                                              */
+    const void* w_down;            /* E packed [H,I] matrices, stride packed_bytes(H,I) */
+    uint16_t* out;                 /* [T,H] fp16, written                               */
+    int32_t* topk_idx;             /* [T,topk]  optional (NULL = not exported)          */
+    float* topk_w;                 /* [T,topk]  optional                                */
+    int32_t* perm;                 /* [T*topk]  optional                                */
+    int32_t* expert_offsets;       /* [E+1]     optional                                */
+    uint16_t* dbg_H;               /* [T*topk, I] fp16 in permuted row order, optional  */
+    uint16_t* dbg_D;               /* [T*topk, H] fp16 in permuted row order, optional  */
+} qmm_moe_args;
+
+size_t qmm_moe_workspace_bytes(const qmm_moe_args* args);   /* host pointer to args */
+/* Steps 1-5.  ws: device, >= qmm_moe_workspace_bytes(args).                  */
+qmm_status qmm_moe(const qmm_moe_args* args, void* ws, size_t ws_bytes, void* stream);
+/* Steps 1-2 only; fills the optional routing outputs that are non-NULL.      */
+qmm_status qmm_moe_route(const qmm_moe_args* args, void* ws, size_t ws_bytes, void* stream);
+
+/* Waits for `stream`, then reports whether any kernel that used `ws` gave up
+ * on a bounded wait (QMM_ERR_DEVICE_TIMEOUT) since the workspace was last
+ * cleared by this call.  ws: device workspace of qmm_gemm or qmm_moe.        */
+qmm_status qmm_status_check(void* ws, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QMM_H */

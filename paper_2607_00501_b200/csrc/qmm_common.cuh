@@ -1,0 +1,161 @@
+// qmm_common.cuh -- device layout of packed weights and small device helpers
+// shared by the kernels of libqmm (sm_100a only).
+//
+// Device layout ("row-group tiles").  Rows are taken in groups of 32 (one row
+// per lane of a warp, and one row per lane of tensor memory in the GEMM).
+// For each row group the K axis is cut into tiles; the tiles of one row group
+// are consecutive in memory, row groups follow each other.
+//
+//   Q4 tile = 64 weights per row (two quantisation blocks), 1152 bytes:
+//     [32 rows][32 B codes]  row r at byte 32 r: eight 32-bit words; word j
+//                            holds elements k = 8j .. 8j+7 of the tile as
+//                            nibbles u = q + 8 in the order 0,2,4,6,1,3,5,7
+//                            (low nibble first), so (word >> 4p) & 0x000F000F
+//                            is the pair (k = 8j+2p, 8j+2p+1) in the low/high
+//                            half-word;
+//     [32 rows][2 x fp16]    scales of the tile's two blocks, row r at 1024 + 4 r.
+//   Q8 tile = 32 weights per row (one block), 1088 bytes:
+//     [32 rows][32 B codes]  byte i = q_i ^ 0x80 (offset binary), k ascending;
+//     [32 rows][fp16]        scale, row r at 1024 + 2 r.
+//
+// Every lane's code load is one 32-byte access and a warp's 32 loads cover
+// 1024 consecutive bytes.  packed_bytes == canonical_bytes.
+#pragma once
+
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/qmm.h"
+
+namespace qmm {
+
+constexpr int kRowsPerGroup = 32;
+constexpr int kQ4TileK = 64;
+constexpr int kQ8TileK = 32;
+constexpr int kQ4TileBytes = 1152;
+constexpr int kQ8TileBytes = 1088;
+constexpr int kTileCodeBytes = 1024;
+constexpr int kNumSMs = 148;
+
+template <int FMT> struct Fmt;
+template <> struct Fmt<QMM_Q4> {
+    static constexpr int tile_k = kQ4TileK;
+    static constexpr int tile_bytes = kQ4TileBytes;
+    static constexpr int canon_block = 18;
+};
+template <> struct Fmt<QMM_Q8> {
+    static constexpr int tile_k = kQ8TileK;
+    static constexpr int tile_bytes = kQ8TileBytes;
+    static constexpr int canon_block = 34;
+};
+
+__host__ __device__ inline int tile_k_of(int fmt) { return fmt == QMM_Q4 ? kQ4TileK : kQ8TileK; }
+__host__ __device__ inline int tile_bytes_of(int fmt) { return fmt == QMM_Q4 ? kQ4TileBytes : kQ8TileBytes; }
+
+// Host-side error reporting (thread-local buffer; see qmm_api.cu).
+qmm_status fail(qmm_status code, const char* fmt, ...);
+qmm_status check_cuda(cudaError_t e, const char* what);
+
+// ---------------------------------------------------------------- loads
+
+struct __align__(32) u32x8 {
+    uint32_t v[8];
+};
+
+// 32-byte streaming load of weight codes: read-only path, no L1 allocation,
+// first in line for L2 eviction (each byte is used once per product).
+__device__ __forceinline__ u32x8 ld_stream_256(const void* p)
+{
+    u32x8 r;
+    asm volatile("ld.global.nc.L1::no_allocate.L2::evict_first.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r.v[0]), "=r"(r.v[1]), "=r"(r.v[2]), "=r"(r.v[3]),
+                   "=r"(r.v[4]), "=r"(r.v[5]), "=r"(r.v[6]), "=r"(r.v[7])
+                 : "l"(p));
+    return r;
+}
+
+// Same bytes, but kept in L2 (weights that are re-read by other thread blocks).
+__device__ __forceinline__ u32x8 ld_keep_256(const void* p)
+{
+    u32x8 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r.v[0]), "=r"(r.v[1]), "=r"(r.v[2]), "=r"(r.v[3]),
+                   "=r"(r.v[4]), "=r"(r.v[5]), "=r"(r.v[6]), "=r"(r.v[7])
+                 : "l"(p));
+    return r;
+}
+
+__device__ __forceinline__ uint32_t ld_nc_u32(const void* p)
+{
+    uint32_t r;
+    asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(r) : "l"(p));
+    return r;
+}
+
+__device__ __forceinline__ uint16_t ld_nc_u16(const void* p)
+{
+    uint16_t r;
+    asm volatile("ld.global.nc.u16 %0, [%1];" : "=h"(r) : "l"(p));
+    return r;
+}
+
+// ------------------------------------------------ integer codes -> fp16
+
+__device__ __forceinline__ __half2 as_h2(uint32_t u)
+{
+    return *reinterpret_cast<__half2*>(&u);
+}
+__device__ __forceinline__ uint32_t as_u32(__half2 h)
+{
+    return *reinterpret_cast<uint32_t*>(&h);
+}
+
+// Q4: the four element pairs of one packed word as exact integers q in fp16.
+// 0x6400 | u is the fp16 value 1024 + u; 0x6400 | (u << 4) is 1024 + 16 u.
+// (1024 + u) - 1032 = q and (1024 + 16 u) / 16 - 72 = q are both exact.
+__device__ __forceinline__ void q4_word_to_h2(uint32_t w, __half2 (&q)[4])
+{
+    const __half2 c1032 = as_h2(0x64086408u);
+    const __half2 c16th = as_h2(0x2C002C00u);
+    const __half2 cm72 = as_h2(0xD480D480u);
+    const uint32_t w8 = w >> 8;
+    q[0] = __hsub2(as_h2((w & 0x000F000Fu) | 0x64006400u), c1032);
+    q[1] = __hfma2(as_h2((w & 0x00F000F0u) | 0x64006400u), c16th, cm72);
+    q[2] = __hsub2(as_h2((w8 & 0x000F000Fu) | 0x64006400u), c1032);
+    q[3] = __hfma2(as_h2((w8 & 0x00F000F0u) | 0x64006400u), c16th, cm72);
+}
+
+// Q8: the two element pairs of one packed word (4 offset-binary bytes) as
+// exact integers in fp16.  0x6400 | (q + 128) is 1024 + 128 + q.
+__device__ __forceinline__ void q8_word_to_h2(uint32_t w, __half2 (&q)[2])
+{
+    const __half2 c1152 = as_h2(0x64806480u);
+    q[0] = __hsub2(as_h2(__byte_perm(w, 0x64646464u, 0x4140)), c1152);
+    q[1] = __hsub2(as_h2(__byte_perm(w, 0x64646464u, 0x4342)), c1152);
+}
+
+// acc += q * x with fp16 inputs widened exactly and one fp32 rounding.
+__device__ __forceinline__ void fma_f16_f32(float& acc, __half a, __half b)
+{
+    asm("fma.rn.f32.f16 %0, %1, %2, %0;" : "+f"(acc) : "h"(__half_as_ushort(a)), "h"(__half_as_ushort(b)));
+}
+
+__device__ __forceinline__ void dot2_f32(float& acc0, float& acc1, __half2 q, __half2 x)
+{
+    fma_f16_f32(acc0, __low2half(q), __low2half(x));
+    fma_f16_f32(acc1, __high2half(q), __high2half(x));
+}
+
+// Programmatic dependent launch: let the next kernel in the stream start its
+// prologue now / wait until the previous kernel's writes are visible.
+__device__ __forceinline__ void pdl_launch_dependents()
+{
+    asm volatile("griddepcontrol.launch_dependents;");
+}
+__device__ __forceinline__ void pdl_wait()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
+}  // namespace qmm

@@ -1,0 +1,348 @@
+// qmm_gemv.cu -- decode matrix-vector product y = W x on packed Q4/Q8 weights.
+//
+// The paper's decode kernels dequantise inside the inner loop so that only the
+// quantised bytes cross the memory bus (Sec. 3.3); this is the same idea laid
+// out for B200: the kernel is bound by HBM bandwidth on the packed bytes, so
+// each lane streams 32-byte code chunks with many loads in flight, expands
+// them to exact fp16 integers in registers and accumulates in fp32.
+//
+// Work decomposition.  A row group is 32 rows, one per lane, so no cross-lane
+// reduction is ever needed: every lane owns one output.  A thread block takes
+// one (row group, K split) item; its warps share the item's tiles round-robin,
+// then add their per-lane partial sums through shared memory in warp order.
+// With splits > 1 the block writes fp32 partials [split][N] to the workspace
+// and a second kernel adds the splits in ascending order (fixed order, so the
+// result does not depend on scheduling).
+#include "qmm_common.cuh"
+
+#include <stdio.h>
+#include <stdlib.h>
+
+namespace qmm {
+
+constexpr int kUnroll = 2;   // tile pairs in flight per warp (4 x 1 KiB of codes per warp)
+
+// D(16x8, fp32) += A(16x16, fp16, row) * B(16x8, fp16, col) on the warp-level tensor path.
+__device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// How a warp multiplies with one row per lane and no shuffles.
+//
+// Lane l = 4g + t holds codes of matrix row l of two row groups (P and Q) for
+// the same k range.  Its pairs go into the A fragment of m16n8k16 as
+//   a0/a2 -> MMA row g,   k slots {2t,2t+1} / {2t+8,2t+9}   (row group P)
+//   a1/a3 -> MMA row g+8, same slots                         (row group Q)
+// so MMA row g carries, in the four slot groups t = 0..3, the same four k of
+// the four matrix rows 4g..4g+3.  B column j is the activation quadruple in
+// slot group j and zero elsewhere, hence D[g][j] = (row 4g+j of P) . x and
+// D[g+8][j] = (row 4g+j of Q) . x for j < 4.  Lanes with t < 2 receive them:
+// c0,c1 = rows 4g+2t, 4g+2t+1 of P;  c2,c3 = the same rows of Q.
+// Products (small integer x fp16) are exact; accumulation is fp32.
+
+// Activations for B come from shared memory: lanes 0,5,10,15 (g == t) read x,
+// every other lane reads an all-zero region of the same size, so that one
+// per-lane base pointer and immediate offsets serve all loads.
+
+// Q4: tile = 64 k.  acc[0..1] rows of P, acc[2..3] rows of Q (see above).
+__device__ __forceinline__ void tile_pair_mma_q4(const u32x8& cp, const u32x8& cq, uint2 sp, uint2 sq,
+                                                 const uint4* xt, float (&acc)[4])
+{
+#pragma unroll
+    for (int b = 0; b < 2; ++b) {
+        float c[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint4 xv = xt[b * 4 + i];                      // activations k = 8(4b+i) .. +7
+            __half2 p[4], q[4];
+            q4_word_to_h2(cp.v[b * 4 + i], p);
+            q4_word_to_h2(cq.v[b * 4 + i], q);
+            mma16816(c, as_u32(p[0]), as_u32(q[0]), as_u32(p[1]), as_u32(q[1]), xv.x, xv.y);
+            mma16816(c, as_u32(p[2]), as_u32(q[2]), as_u32(p[3]), as_u32(q[3]), xv.z, xv.w);
+        }
+        // scales: sp.x / sp.y = rows 4g+2t / 4g+2t+1 of P as (block 0, block 1) fp16 pairs
+        const float dp0 = __half2float(b ? __high2half(as_h2(sp.x)) : __low2half(as_h2(sp.x)));
+        const float dp1 = __half2float(b ? __high2half(as_h2(sp.y)) : __low2half(as_h2(sp.y)));
+        const float dq0 = __half2float(b ? __high2half(as_h2(sq.x)) : __low2half(as_h2(sq.x)));
+        const float dq1 = __half2float(b ? __high2half(as_h2(sq.y)) : __low2half(as_h2(sq.y)));
+        acc[0] = fmaf(dp0, c[0], acc[0]);
+        acc[1] = fmaf(dp1, c[1], acc[1]);
+        acc[2] = fmaf(dq0, c[2], acc[2]);
+        acc[3] = fmaf(dq1, c[3], acc[3]);
+    }
+}
+
+// Q8: tile = 32 k (one block); scales are one fp16 per row: s.x low/high = rows 4g+2t, 4g+2t+1.
+__device__ __forceinline__ void tile_pair_mma_q8(const u32x8& cp, const u32x8& cq, uint32_t sp, uint32_t sq,
+                                                 const uint4* xt, float (&acc)[4])
+{
+    float c[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint4 xv = xt[i];                                  // activations k = 8i .. 8i+7
+        __half2 p[2], q[2];
+        q8_word_to_h2(cp.v[2 * i], p);
+        q8_word_to_h2(cq.v[2 * i], q);
+        mma16816(c, as_u32(p[0]), as_u32(q[0]), as_u32(p[1]), as_u32(q[1]), xv.x, xv.y);
+        q8_word_to_h2(cp.v[2 * i + 1], p);
+        q8_word_to_h2(cq.v[2 * i + 1], q);
+        mma16816(c, as_u32(p[0]), as_u32(q[0]), as_u32(p[1]), as_u32(q[1]), xv.z, xv.w);
+    }
+    acc[0] = fmaf(__half2float(__low2half(as_h2(sp))), c[0], acc[0]);
+    acc[1] = fmaf(__half2float(__high2half(as_h2(sp))), c[1], acc[1]);
+    acc[2] = fmaf(__half2float(__low2half(as_h2(sq))), c[2], acc[2]);
+    acc[3] = fmaf(__half2float(__high2half(as_h2(sq))), c[3], acc[3]);
+}
+
+template <int FMT> struct ScaleRegs;
+template <> struct ScaleRegs<QMM_Q4> { using type = uint2; };
+template <> struct ScaleRegs<QMM_Q8> { using type = uint32_t; };
+
+// Scales of rows 4g+2(t&1) and the next row of one tile (the rows whose sums this lane receives).
+template <int FMT>
+__device__ __forceinline__ typename ScaleRegs<FMT>::type load_scales(const uint8_t* tile, int lane);
+template <>
+__device__ __forceinline__ uint2 load_scales<QMM_Q4>(const uint8_t* tile, int lane)
+{
+    const int row = (lane & ~3) + 2 * (lane & 1);
+    uint2 r;
+    asm volatile("ld.global.nc.v2.u32 {%0,%1}, [%2];" : "=r"(r.x), "=r"(r.y) : "l"(tile + kTileCodeBytes + 4 * row));
+    return r;
+}
+template <>
+__device__ __forceinline__ uint32_t load_scales<QMM_Q8>(const uint8_t* tile, int lane)
+{
+    const int row = (lane & ~3) + 2 * (lane & 1);
+    return ld_nc_u32(tile + kTileCodeBytes + 2 * row);
+}
+
+// Codes and scales of kUnroll tile pairs held in registers.
+template <int FMT>
+struct TileRegs {
+    u32x8 cp[kUnroll], cq[kUnroll];
+    typename ScaleRegs<FMT>::type sp[kUnroll], sq[kUnroll];
+};
+
+// grid.x blocks loop over items = (row-group pairs) * splits; block = WARPS warps.
+// Dynamic shared memory: K fp16 activations, K fp16 zeros, then WARPS*64 floats.
+//
+// Weights never depend on the previous kernel in the stream, activations do.
+// So each warp issues the loads of its first group *before* waiting for the
+// previous kernel (programmatic dependent launch): the HBM latency of one
+// product hides behind the tail of the one before it.
+template <int FMT, int WARPS>
+__global__ void __launch_bounds__(WARPS * 32, 768 / (WARPS * 32))
+gemv_kernel(const uint8_t* __restrict__ packed, const uint16_t* __restrict__ x,
+            uint16_t* __restrict__ y, float* __restrict__ partial,
+            int N, int K, int tiles_per_row, int splits, int items)
+{
+    extern __shared__ uint4 smem[];
+    uint4* xs = smem;
+    uint4* zs = smem + K / 8;
+    float* red = reinterpret_cast<float*>(smem + K / 4);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr int TB = Fmt<FMT>::tile_bytes;
+    constexpr int XV = Fmt<FMT>::tile_k / 8;                    // uint4 of activations per tile
+    constexpr int STEP = kUnroll * WARPS;
+
+    const int tps = tiles_per_row / splits;                     // tiles per item
+    const size_t group_bytes = (size_t)tiles_per_row * TB;
+    const uint8_t* lane_base = packed + 32 * lane;
+
+    int item = blockIdx.x;
+    int pair = item / splits, s = item - pair * splits;
+    int t = s * tps + warp, t_end = (s + 1) * tps;
+    const uint8_t* tiles_p = lane_base + (size_t)(2 * pair) * group_bytes;
+
+    TileRegs<FMT> r;
+    auto load_group = [&]() {
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            const int tt = t + u * WARPS;
+            if (tt < t_end) {
+                const uint8_t* tp = tiles_p + (size_t)tt * TB;
+                const uint8_t* tq = tp + group_bytes;
+                r.cp[u] = ld_stream_256(tp);
+                r.cq[u] = ld_stream_256(tq);
+                r.sp[u] = load_scales<FMT>(tp - 32 * lane, lane);
+                r.sq[u] = load_scales<FMT>(tq - 32 * lane, lane);
+            }
+        }
+    };
+    if (item < items) load_group();
+
+    pdl_launch_dependents();
+    pdl_wait();                                                 // x may come from the previous kernel
+    for (int i = threadIdx.x; i < K / 8; i += WARPS * 32) {
+        xs[i] = reinterpret_cast<const uint4*>(x)[i];
+        zs[i] = make_uint4(0u, 0u, 0u, 0u);
+    }
+    __syncthreads();
+    const uint4* xb = ((lane >> 2) == (lane & 3)) ? xs : zs;
+
+    while (item < items) {
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        while (t < t_end) {
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) {
+                const int tt = t + u * WARPS;
+                if (tt < t_end) {
+                    if constexpr (FMT == QMM_Q4)
+                        tile_pair_mma_q4(r.cp[u], r.cq[u], r.sp[u], r.sq[u], xb + tt * XV, acc);
+                    else
+                        tile_pair_mma_q8(r.cp[u], r.cq[u], r.sp[u], r.sq[u], xb + tt * XV, acc);
+                }
+            }
+            t += STEP;
+            if (t < t_end) load_group();
+        }
+        const int done_pair = pair, done_s = s;
+        item += gridDim.x;
+        if (item < items) {                                     // next item's loads fly during the reduction
+            pair = item / splits;
+            s = item - pair * splits;
+            t = s * tps + warp;
+            t_end = (s + 1) * tps;
+            tiles_p = lane_base + (size_t)(2 * pair) * group_bytes;
+            load_group();
+        }
+        // add the warps' partial sums in warp order
+        if ((lane & 3) < 2) {                                   // lanes that received sums (see above)
+            const int row = (lane & ~3) + 2 * (lane & 1);
+            float* w = red + warp * 64;
+            w[row] = acc[0];
+            w[row + 1] = acc[1];
+            w[32 + row] = acc[2];
+            w[32 + row + 1] = acc[3];
+        }
+        __syncthreads();
+        if (threadIdx.x < 64) {
+            float sum = red[threadIdx.x];
+#pragma unroll
+            for (int w = 1; w < WARPS; ++w) sum += red[w * 64 + threadIdx.x];
+            const int n = done_pair * 64 + threadIdx.x;
+            if (splits == 1)
+                y[n] = __half_as_ushort(__float2half_rn(sum));
+            else
+                partial[(size_t)done_s * N + n] = sum;
+        }
+        __syncthreads();
+    }
+}
+
+// Second stage of split-K: y[n] = fp16(sum_s partial[s][n]), s ascending.
+__global__ void gemv_reduce_kernel(const float* __restrict__ partial, uint16_t* __restrict__ y, int N, int splits)
+{
+    pdl_launch_dependents();
+    pdl_wait();
+    const int n = blockIdx.x * blockDim.x + threadIdx.x;
+    if (n >= N) return;
+    float sum = partial[n];
+    for (int s = 1; s < splits; ++s) sum += partial[(size_t)s * N + n];
+    y[n] = __half_as_ushort(__float2half_rn(sum));
+}
+
+// ------------------------------------------------------------------ host
+
+struct GemvPlan {
+    int warps;    // 8 or 16
+    int splits;   // K splits across thread blocks
+    int grid;
+};
+
+// Shape -> launch geometry.  The aim is >= ~2 resident blocks' worth of loads
+// on every SM: prefer more warps per block, and split K across blocks only
+// when the row groups alone cannot cover the SMs.
+GemvPlan gemv_plan(int fmt, int64_t N, int64_t K)
+{
+    GemvPlan p;
+    const int tpr = (int)(K / tile_k_of(fmt));
+    const int groups = (int)(N / (2 * kRowsPerGroup));       // items are pairs of row groups
+    int warps = 16;                                           // <= 512 threads: two generations of blocks fit on an SM
+    while (warps > 8 && warps > tpr) warps >>= 1;
+    // large problems: fewer warps per block so that several blocks share an SM
+    if ((int64_t)groups * tpr >= (int64_t)kNumSMs * 64 * 4 && warps > 8) warps = 8;
+    else if ((int64_t)groups * tpr >= (int64_t)kNumSMs * 64 && warps > 16) warps = 16;
+    int splits = 1;
+    while (groups * splits < kNumSMs && tpr / (splits * 2) >= warps && (tpr % (splits * 2)) == 0 && splits < 16)
+        splits *= 2;
+    if (const char* f = getenv("QMM_GEMV_FORCE")) {           // "warps,splits" for sweeps
+        int w = 0, s = 0;
+        if (sscanf(f, "%d,%d", &w, &s) == 2 && (w == 8 || w == 16) && s >= 1 && tpr % s == 0) {
+            warps = w;
+            splits = s;
+        }
+    }
+    p.warps = warps;
+    p.splits = splits;
+    const int items = groups * splits;
+    const int per_sm = 768 / (warps * 32);
+    p.grid = items < kNumSMs * per_sm ? items : kNumSMs * per_sm;
+    return p;
+}
+
+size_t gemv_workspace_bytes(int fmt, int64_t N, int64_t K)
+{
+    const GemvPlan p = gemv_plan(fmt, N, K);
+    return p.splits > 1 ? (size_t)p.splits * (size_t)N * sizeof(float) : 0;
+}
+
+template <typename... Args>
+static cudaError_t launch_pdl(void (*kernel)(Args...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
+template <int FMT, int WARPS>
+static qmm_status launch_gemv_t(const GemvPlan& p, const void* packed, int64_t N, int64_t K,
+                                const uint16_t* x, uint16_t* y, float* partial, cudaStream_t st)
+{
+    const size_t smem = (size_t)K * 4 + (size_t)WARPS * 64 * sizeof(float);
+    auto kern = gemv_kernel<FMT, WARPS>;
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return check_cuda(e, "qmm_gemv shared memory size");
+    }
+    const int tpr = (int)(K / Fmt<FMT>::tile_k);
+    const int items = (int)(N / (2 * kRowsPerGroup)) * p.splits;
+    cudaError_t e = launch_pdl(kern, dim3(p.grid), dim3(WARPS * 32), smem, st,
+                               (const uint8_t*)packed, x, y, partial, (int)N, (int)K, tpr, p.splits, items);
+    if (e != cudaSuccess) return check_cuda(e, "qmm_gemv launch");
+    if (p.splits > 1) {
+        e = launch_pdl(gemv_reduce_kernel, dim3((unsigned)((N + 255) / 256)), dim3(256), 0, st,
+                       (const float*)partial, y, (int)N, p.splits);
+        if (e != cudaSuccess) return check_cuda(e, "qmm_gemv reduce launch");
+    }
+    return QMM_OK;
+}
+
+qmm_status launch_gemv(int fmt, const void* packed, int64_t N, int64_t K, const uint16_t* x, uint16_t* y,
+                       void* ws, cudaStream_t st)
+{
+    const GemvPlan p = gemv_plan(fmt, N, K);
+    float* partial = (float*)ws;
+#define QMM_GEMV_CASE(F, W) \
+    if (fmt == F && p.warps == W) return launch_gemv_t<F, W>(p, packed, N, K, x, y, partial, st);
+    QMM_GEMV_CASE(QMM_Q4, 8)
+    QMM_GEMV_CASE(QMM_Q4, 16)
+    QMM_GEMV_CASE(QMM_Q8, 8)
+    QMM_GEMV_CASE(QMM_Q8, 16)
+#undef QMM_GEMV_CASE
+    return fail(QMM_ERR_UNSUPPORTED, "qmm_gemv: no kernel for this plan");
+}
+
+}  // namespace qmm

@@ -1,0 +1,202 @@
+"""Thin ctypes binding of libqmm.so (the C ABI declared in include/qmm.h).
+
+Argument marshalling only: every step of every product runs in the CUDA
+kernels of the library.  PyTorch is used for device memory and streams.  There
+is no CPU fallback: if the shared library cannot be loaded, or a call fails,
+an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import threading
+
+import torch
+
+Q4 = 4
+Q8 = 8
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libqmm.so")
+_lock = threading.Lock()
+_lib = None
+
+STATUS_NAMES = {
+    0: "QMM_OK", 1: "QMM_ERR_INVALID_ARG", 2: "QMM_ERR_SHAPE", 3: "QMM_ERR_ALIGNMENT",
+    4: "QMM_ERR_WORKSPACE", 5: "QMM_ERR_UNSUPPORTED", 6: "QMM_ERR_CUDA", 7: "QMM_ERR_DEVICE_TIMEOUT",
+}
+
+# every symbol include/qmm.h declares
+EXPORTS = (
+    "qmm_last_error", "qmm_version", "qmm_canonical_bytes", "qmm_packed_bytes", "qmm_pack",
+    "qmm_dequant", "qmm_gemv_workspace_bytes", "qmm_gemv", "qmm_gemm_workspace_bytes", "qmm_gemm",
+    "qmm_moe_workspace_bytes", "qmm_moe", "qmm_moe_route", "qmm_status_check",
+)
+
+
+class QmmError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__("%s: %s" % (STATUS_NAMES.get(status, status), message))
+        self.status = status
+        self.message = message
+
+
+class MoeArgs(ctypes.Structure):
+    _fields_ = [
+        ("T", ctypes.c_int32), ("H", ctypes.c_int32), ("I", ctypes.c_int32), ("E", ctypes.c_int32),
+        ("topk", ctypes.c_int32), ("fmt", ctypes.c_int32),
+        ("logits", ctypes.c_void_p), ("X", ctypes.c_void_p),
+        ("w_gate", ctypes.c_void_p), ("w_up", ctypes.c_void_p), ("w_down", ctypes.c_void_p),
+        ("out", ctypes.c_void_p),
+        ("topk_idx", ctypes.c_void_p), ("topk_w", ctypes.c_void_p),
+        ("perm", ctypes.c_void_p), ("expert_offsets", ctypes.c_void_p),
+        ("dbg_H", ctypes.c_void_p), ("dbg_D", ctypes.c_void_p),
+    ]
+
+
+def lib() -> ctypes.CDLL:
+    """Load libqmm.so (building it with nvcc first if it is not there)."""
+    global _lib
+    with _lock:
+        if _lib is None:
+            if not os.path.exists(LIB_PATH):
+                from . import _build
+                _build.build()
+            L = ctypes.CDLL(LIB_PATH)
+            i64, vp, ci, sz = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+            L.qmm_last_error.restype = ctypes.c_char_p
+            L.qmm_last_error.argtypes = []
+            L.qmm_version.restype = ci
+            L.qmm_canonical_bytes.restype = sz
+            L.qmm_canonical_bytes.argtypes = [ci, i64, i64]
+            L.qmm_packed_bytes.restype = sz
+            L.qmm_packed_bytes.argtypes = [ci, i64, i64]
+            L.qmm_pack.argtypes = [ci, vp, i64, i64, vp, vp]
+            L.qmm_dequant.argtypes = [ci, vp, i64, i64, vp, vp]
+            L.qmm_gemv_workspace_bytes.restype = sz
+            L.qmm_gemv_workspace_bytes.argtypes = [ci, i64, i64]
+            L.qmm_gemv.argtypes = [ci, vp, i64, i64, vp, vp, vp, sz, vp]
+            L.qmm_gemm_workspace_bytes.restype = sz
+            L.qmm_gemm_workspace_bytes.argtypes = [ci, i64, i64, i64]
+            L.qmm_gemm.argtypes = [ci, vp, i64, i64, vp, i64, vp, i64, i64, vp, sz, vp]
+            L.qmm_moe_workspace_bytes.restype = sz
+            L.qmm_moe_workspace_bytes.argtypes = [ctypes.POINTER(MoeArgs)]
+            L.qmm_moe.argtypes = [ctypes.POINTER(MoeArgs), vp, sz, vp]
+            L.qmm_moe_route.argtypes = [ctypes.POINTER(MoeArgs), vp, sz, vp]
+            L.qmm_status_check.argtypes = [vp, vp]
+            _lib = L
+    return _lib
+
+
+def last_error() -> str:
+    return lib().qmm_last_error().decode("utf-8", "replace")
+
+
+def _check(status: int):
+    if status != 0:
+        raise QmmError(status, last_error())
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _dp(t):
+    return 0 if t is None else t.data_ptr()
+
+
+def _nbytes(t) -> int:
+    return 0 if t is None else t.numel() * t.element_size()
+
+
+def version() -> int:
+    return lib().qmm_version()
+
+
+def canonical_bytes(fmt: int, N: int, K: int) -> int:
+    return lib().qmm_canonical_bytes(fmt, N, K)
+
+
+def packed_bytes(fmt: int, N: int, K: int) -> int:
+    n = lib().qmm_packed_bytes(fmt, N, K)
+    if n == 0:
+        raise QmmError(5, last_error())
+    return n
+
+
+def pack(fmt: int, canonical: torch.Tensor, N: int, K: int, out: torch.Tensor | None = None) -> torch.Tensor:
+    """canonical: uint8 CUDA tensor of canonical_bytes(fmt,N,K) bytes -> packed uint8 tensor."""
+    assert canonical.is_cuda and canonical.dtype == torch.uint8 and canonical.is_contiguous()
+    assert canonical.numel() == canonical_bytes(fmt, N, K)
+    if out is None:
+        out = torch.empty(packed_bytes(fmt, N, K), dtype=torch.uint8, device=canonical.device)
+    _check(lib().qmm_pack(fmt, canonical.data_ptr(), N, K, out.data_ptr(), _stream()))
+    return out
+
+
+def dequant(fmt: int, packed: torch.Tensor, N: int, K: int) -> torch.Tensor:
+    out = torch.empty((N, K), dtype=torch.float32, device=packed.device)
+    _check(lib().qmm_dequant(fmt, packed.data_ptr(), N, K, out.data_ptr(), _stream()))
+    return out
+
+
+def gemv_workspace_bytes(fmt: int, N: int, K: int) -> int:
+    return lib().qmm_gemv_workspace_bytes(fmt, N, K)
+
+
+def gemv(fmt: int, packed: torch.Tensor, N: int, K: int, x: torch.Tensor,
+         y: torch.Tensor | None = None, ws: torch.Tensor | None = None) -> torch.Tensor:
+    """y = W x.  x: fp16 [K] CUDA tensor; returns fp16 [N]."""
+    assert x.is_cuda and x.dtype == torch.float16 and x.numel() == K and x.is_contiguous()
+    if y is None:
+        y = torch.empty(N, dtype=torch.float16, device=x.device)
+    if ws is None:
+        need = gemv_workspace_bytes(fmt, N, K)
+        ws = torch.empty(need, dtype=torch.uint8, device=x.device) if need else None
+    _check(lib().qmm_gemv(fmt, packed.data_ptr(), N, K, x.data_ptr(), y.data_ptr(), _dp(ws), _nbytes(ws), _stream()))
+    return y
+
+
+def gemm_workspace_bytes(fmt: int, M: int, N: int, K: int) -> int:
+    return lib().qmm_gemm_workspace_bytes(fmt, M, N, K)
+
+
+def gemm(fmt: int, packed: torch.Tensor, N: int, K: int, X: torch.Tensor,
+         Y: torch.Tensor | None = None, ws: torch.Tensor | None = None) -> torch.Tensor:
+    """Y = X W^T.  X: fp16 [M,K] (row stride >= K); returns fp16 [M,N]."""
+    assert X.is_cuda and X.dtype == torch.float16 and X.dim() == 2 and X.shape[1] == K and X.stride(1) == 1
+    M = X.shape[0]
+    if Y is None:
+        Y = torch.empty((M, N), dtype=torch.float16, device=X.device)
+    assert Y.stride(1) == 1
+    if ws is None:
+        ws = torch.zeros(max(gemm_workspace_bytes(fmt, M, N, K), 256), dtype=torch.uint8, device=X.device)
+    _check(lib().qmm_gemm(fmt, packed.data_ptr(), N, K, X.data_ptr(), X.stride(0) if M > 1 else max(K, X.stride(0)),
+                          Y.data_ptr(), Y.stride(0) if M > 1 else max(N, Y.stride(0)), M,
+                          ws.data_ptr(), _nbytes(ws), _stream()))
+    return Y
+
+
+def moe_args(fmt, T, H, I, E, topk, logits, X, w_gate, w_up, w_down, out,
+             topk_idx=None, topk_w=None, perm=None, expert_offsets=None, dbg_H=None, dbg_D=None) -> MoeArgs:
+    return MoeArgs(T, H, I, E, topk, fmt, _dp(logits), _dp(X), _dp(w_gate), _dp(w_up), _dp(w_down), _dp(out),
+                   _dp(topk_idx), _dp(topk_w), _dp(perm), _dp(expert_offsets), _dp(dbg_H), _dp(dbg_D))
+
+
+def moe_workspace_bytes(args: MoeArgs) -> int:
+    n = lib().qmm_moe_workspace_bytes(ctypes.byref(args))
+    if n == 0:
+        raise QmmError(5, last_error())
+    return n
+
+
+def moe(args: MoeArgs, ws: torch.Tensor) -> None:
+    _check(lib().qmm_moe(ctypes.byref(args), ws.data_ptr(), _nbytes(ws), _stream()))
+
+
+def moe_route(args: MoeArgs, ws: torch.Tensor) -> None:
+    _check(lib().qmm_moe_route(ctypes.byref(args), ws.data_ptr(), _nbytes(ws), _stream()))
+
+
+def status_check(ws: torch.Tensor) -> None:
+    _check(lib().qmm_status_check(ws.data_ptr(), _stream()))

@@ -1,0 +1,163 @@
+"""GPU parity: qmm_pack / qmm_dequant / qmm_gemv against the CPU oracle.
+
+Weights must dequantise bit-exactly; every GEMV output must satisfy
+|y_gpu - y_ref| <= 2e-3 * sum_k |w x| + 1e-5 with y_ref, sum|w x| from the
+oracle's fp64 accumulation.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2607_00501_b200 import synth
+from tests import util
+
+pytestmark = pytest.mark.gpu
+Q4, Q8 = 4, 8
+
+
+@pytest.fixture(scope="module")
+def qmm():
+    from paper_2607_00501_b200 import qmm as _qmm
+    assert torch.cuda.is_available()
+    _qmm.lib()
+    return _qmm
+
+
+def packed_from(qmm, fmt, blocks, N, K):
+    return qmm.pack(fmt, util.dev(blocks), N, K)
+
+
+@pytest.mark.parametrize("fmt", [Q4, Q8])
+@pytest.mark.parametrize("N,K", [(128, 256), (384, 768), (256, 2048)])
+def test_dequant_bit_exact(qmm, oracle, fmt, N, K):
+    blocks, _, _ = util.random_blocks(synth, fmt, N, K, seed=N + K + fmt)
+    w_gpu = qmm.dequant(fmt, packed_from(qmm, fmt, blocks, N, K), N, K).cpu().numpy()
+    w_ref = oracle.dequant(fmt, blocks, N, K)
+    assert w_gpu.tobytes() == w_ref.tobytes()
+
+
+@pytest.mark.parametrize("fmt", [Q4, Q8])
+def test_dequant_every_code_and_scale_class(qmm, oracle, fmt):
+    # each row repeats every code value; scales sweep normal, subnormal, negative, zero
+    N, K = 128, 256
+    lo, hi = (-8, 8) if fmt == Q4 else (-128, 128)
+    codes = np.resize(np.arange(lo, hi), (N, K))
+    codes = np.roll(codes, np.arange(N)[:, None] % 7, axis=1) if False else codes
+    sb = np.resize(np.array([0x0001, 0x03FF, 0x0400, 0x2000, 0x3C00, 0x7BFF, 0x8001, 0xBC00, 0x0000, 0x8000],
+                            dtype=np.uint16), (N, K // 32))
+    blocks = synth.blocks_from_codes(fmt, sb, codes)
+    w_gpu = qmm.dequant(fmt, packed_from(qmm, fmt, blocks, N, K), N, K).cpu().numpy()
+    assert w_gpu.tobytes() == oracle.dequant(fmt, blocks, N, K).tobytes()
+
+
+def run_gemv(qmm, oracle, fmt, blocks, N, K, x, what):
+    y = qmm.gemv(fmt, packed_from(qmm, fmt, blocks, N, K), N, K, util.dev(x))
+    torch.cuda.synchronize()
+    y_ref, B = oracle.gemv(fmt, blocks, N, K, x)
+    return util.assert_within_tol(util.host_f64(y), y_ref, B, what), y
+
+
+@pytest.mark.parametrize("fmt", [Q4, Q8])
+@pytest.mark.parametrize("N,K", [(128, 256), (384, 512), (128, 8192), (2176, 1280)])
+def test_gemv_small_shapes(qmm, oracle, fmt, N, K):
+    blocks, _, _ = util.random_blocks(synth, fmt, N, K, seed=7 * N + K + fmt)
+    x = synth.activations(90, N + K, K)
+    run_gemv(qmm, oracle, fmt, blocks, N, K, x, "gemv %dx%d fmt %d" % (N, K, fmt))
+
+
+@pytest.mark.parametrize("fmt", [Q4, Q8])
+@pytest.mark.parametrize("force", ["8,1", "8,2", "8,8", "16,1", "16,2", "16,4"])
+def test_gemv_every_launch_geometry(qmm, oracle, fmt, force, monkeypatch):
+    # the same product through each block size and K split (split-K partials + fixed-order reduce)
+    monkeypatch.setenv("QMM_GEMV_FORCE", force)
+    N, K = 512, 4096
+    blocks = synth.quantize(fmt, synth.weights(91, fmt, N, K))
+    x = synth.activations(91, 7, K)
+    run_gemv(qmm, oracle, fmt, blocks, N, K, x, "gemv forced " + force)
+
+
+@pytest.mark.parametrize("fmt", [Q4, Q8])
+def test_gemv_integer_case_is_exact(qmm, fmt):
+    # unit scales and small integer activations: an integer matrix-vector product, exact in fp16 output
+    rng = np.random.default_rng(5 + fmt)
+    N, K = 256, 512
+    lo, hi = (-8, 8) if fmt == Q4 else (-127, 128)
+    codes = rng.integers(lo, hi, size=(N, K))
+    keep = rng.random((N, K)) < (0.25 if fmt == Q4 else 0.01)       # keep |y| < 2048
+    codes = np.where(keep, codes, 0)
+    xi = rng.integers(-2, 3, size=K)
+    ref = codes.astype(np.int64) @ xi.astype(np.int64)
+    assert np.abs(ref).max() < 2048
+    blocks = synth.blocks_from_codes(fmt, np.full((N, K // 32), 0x3C00, dtype=np.uint16), codes)
+    y = qmm.gemv(fmt, packed_from(qmm, fmt, blocks, N, K), N, K, util.dev(xi.astype(np.float16)))
+    assert np.array_equal(util.host_f64(y), ref.astype(np.float64))
+
+
+@pytest.mark.parametrize("fmt", [Q4, Q8])
+def test_gemv_one_hot_returns_column_and_zero_codes_give_zero(qmm, oracle, fmt):
+    N, K = 128, 512
+    blocks, codes, sb = util.random_blocks(synth, fmt, N, K, seed=33 + fmt, special_scales=False)
+    packed = packed_from(qmm, fmt, blocks, N, K)
+    W = oracle.dequant(fmt, blocks, N, K)
+    for k in (0, 1, 31, 32, 63, 64, 255, 511):
+        e = np.zeros(K, dtype=np.float16)
+        e[k] = 1
+        y = qmm.gemv(fmt, packed, N, K, util.dev(e)).cpu().numpy()
+        assert np.array_equal(y, W[:, k].astype(np.float16)), k
+    z = synth.blocks_from_codes(fmt, sb, np.zeros_like(codes))
+    y = qmm.gemv(fmt, packed_from(qmm, fmt, z, N, K), N, K, util.dev(synth.activations(1, 1, K)))
+    assert not y.cpu().numpy().any()
+
+
+def test_gemv_is_deterministic_and_stays_in_bounds(qmm, monkeypatch):
+    monkeypatch.setenv("QMM_GEMV_FORCE", "8,4")
+    N, K = 256, 2048
+    blocks = synth.quantize(Q4, synth.weights(92, 0, N, K))
+    packed = packed_from(qmm, Q4, blocks, N, K)
+    x = util.dev(synth.activations(92, 1, K))
+    guard = 64
+    buf = torch.full((N + 2 * guard,), 7.0, dtype=torch.float16, device="cuda")
+    need = qmm.gemv_workspace_bytes(Q4, N, K)
+    wsbuf = torch.full((need + 512,), 0x5A, dtype=torch.uint8, device="cuda")
+    y = buf[guard:guard + N]
+    qmm.gemv(Q4, packed, N, K, x, y=y, ws=wsbuf[256:256 + need])
+    first = y.clone()
+    for _ in range(5):
+        qmm.gemv(Q4, packed, N, K, x, y=y, ws=wsbuf[256:256 + need])
+        assert torch.equal(first, y)
+    assert torch.all(buf[:guard] == 7.0) and torch.all(buf[guard + N:] == 7.0)
+    assert torch.all(wsbuf[:256] == 0x5A) and torch.all(wsbuf[256 + need:] == 0x5A)
+
+
+def test_cfg0_q4_gemv_full_size(qmm, oracle):
+    c = synth.CFG0
+    blocks = synth.quantize(c["fmt"], synth.weights(c["seed"], 0, c["N"], c["K"]))
+    x = synth.activations(c["seed"], 1, c["K"])
+    run_gemv(qmm, oracle, c["fmt"], blocks, c["N"], c["K"], x, "cfg0")
+
+
+@pytest.mark.parametrize("fmt", [Q4, Q8])
+def test_cfg1_one_layer_full_size_unfused_and_fused(qmm, oracle, fmt):
+    layer = 3
+    acts = synth.cfg1_layer_acts(layer)
+    packed, refs = {}, {}
+    for name, N, K, act, w in synth.cfg1_layer_weights(layer):
+        blocks = synth.quantize(fmt, w)
+        packed[name] = packed_from(qmm, fmt, blocks, N, K)
+        y = qmm.gemv(fmt, packed[name], N, K, util.dev(acts[act]))
+        refs[name] = oracle.gemv(fmt, blocks, N, K, acts[act])
+        util.assert_within_tol(util.host_f64(y), refs[name][0], refs[name][1], "cfg1 %s" % name)
+    # fused launches: packed buffers with the same K concatenate into one matrix
+    for names, act in ((("q", "k", "v"), "x_attn"), (("gate", "up"), "x_ffn")):
+        Ntot = sum(packed[n].numel() for n in names) // (qmm.packed_bytes(fmt, 128, 2048) // 128)
+        y = qmm.gemv(fmt, torch.cat([packed[n] for n in names]), Ntot, 2048, util.dev(acts[act]))
+        y_ref = np.concatenate([refs[n][0] for n in names])
+        B = np.concatenate([refs[n][1] for n in names])
+        util.assert_within_tol(util.host_f64(y), y_ref, B, "cfg1 fused " + "+".join(names))
+
+
+def test_cfg2_q8_lm_head_full_size(qmm, oracle):
+    c = synth.CFG2
+    blocks = synth.quantize(c["fmt"], synth.weights(c["seed"], 0, c["N"], c["K"]))
+    x = synth.activations(c["seed"], 1, c["K"])
+    run_gemv(qmm, oracle, c["fmt"], blocks, c["N"], c["K"], x, "cfg2")

@@ -1,0 +1,115 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports
+every symbol the header declares, answers size queries and rejects bad
+arguments before anything is launched."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2607_00501_b200 import _build, qmm, synth
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def L():
+    _build.build()
+    return qmm.lib()
+
+
+def test_header_symbols_are_exported(L):
+    hdr = open(os.path.join(ROOT, "include", "qmm.h")).read()
+    hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
+    declared = set(re.findall(r"\b(qmm_[a-z_]+)\s*\(", hdr))
+    assert declared == set(qmm.EXPORTS)
+    for name in declared:
+        assert hasattr(L, name), name
+
+
+def test_version_and_sizes(L):
+    assert qmm.version() >= 100
+    assert qmm.canonical_bytes(4, 3072, 1024) == 1769472 == synth.canonical_bytes(4, 3072, 1024)
+    assert qmm.canonical_bytes(8, 128256, 3072) == 418627584
+    assert qmm.canonical_bytes(4, 128, 31) == 0
+    assert qmm.packed_bytes(4, 3072, 1024) == 1769472
+    assert qmm.packed_bytes(8, 128256, 3072) == 418627584
+    # packed buffers with the same K concatenate row-wise
+    assert qmm.packed_bytes(4, 2048, 2048) + 2 * qmm.packed_bytes(4, 512, 2048) == qmm.packed_bytes(4, 3072, 2048)
+
+
+@pytest.mark.parametrize("fmt,N,K,status", [
+    (5, 128, 256, 1), (4, 0, 256, 1), (4, 128, -256, 1), (4, 128, 100, 2), (4, 128, 288, 5), (4, 100, 256, 5),
+])
+def test_bad_shapes_are_rejected(L, fmt, N, K, status):
+    buf = (ctypes.c_char * 64)()
+    addr = ctypes.addressof(buf)
+    assert L.qmm_pack(fmt, addr, N, K, addr, None) == status
+    assert qmm.last_error()
+    assert L.qmm_gemv(fmt, addr, N, K, addr, addr, None, 0, None) == status
+    assert L.qmm_gemm(fmt, addr, N, K, addr, K, addr, N, 4, addr, 0, None) == status
+    with pytest.raises(qmm.QmmError):
+        qmm.packed_bytes(fmt, N, K)
+
+
+def test_null_and_misaligned_pointers(L):
+    buf = (ctypes.c_char * 512)()
+    a = (ctypes.addressof(buf) + 255) & ~255
+    assert L.qmm_pack(4, None, 128, 256, a, None) == 1
+    assert L.qmm_pack(4, a, 128, 256, a + 8, None) == 3
+    assert L.qmm_dequant(4, a, 128, 256, None, None) == 1
+    assert L.qmm_gemv(4, a, 128, 256, None, a, None, 0, None) == 1
+    assert L.qmm_gemv(4, a, 128, 256, a + 2, a, None, 0, None) == 3
+    assert L.qmm_gemv(4, a + 16, 128, 256, a, a, None, 0, None) == 3
+    assert "aligned" in qmm.last_error()
+    assert L.qmm_gemm(4, a, 128, 256, a, 255, a, 128, 4, a, 1 << 20, None) == 2     # ldx < K
+    assert L.qmm_gemm(4, a, 128, 256, a, 260, a, 128, 4, a, 1 << 20, None) == 3     # ldx % 8
+    assert L.qmm_gemm(4, a, 128, 256, a, 256, a, 128, -1, a, 1 << 20, None) == 1
+    assert L.qmm_gemm(4, a, 128, 256, a, 256, a, 128, 0, a, 0, None) == 0           # M = 0: nothing to do
+    assert L.qmm_gemm(4, a, 128, 256, a, 256, a, 128, 4, None, 0, None) == 4
+    assert L.qmm_status_check(None, None) == 1
+
+
+def test_gemv_workspace_rule(L, monkeypatch):
+    monkeypatch.setenv("QMM_GEMV_FORCE", "8,4")
+    need = qmm.gemv_workspace_bytes(4, 512, 2048)
+    assert need == 4 * 512 * 4
+    buf = (ctypes.c_char * 512)()
+    a = (ctypes.addressof(buf) + 255) & ~255
+    assert L.qmm_gemv(4, a, 512, 2048, a, a, None, 0, None) == 4
+    assert L.qmm_gemv(4, a, 512, 2048, a, a, a, need - 1, None) == 4
+    assert "workspace" in qmm.last_error()
+    monkeypatch.setenv("QMM_GEMV_FORCE", "8,1")
+    assert qmm.gemv_workspace_bytes(4, 512, 2048) == 0
+
+
+def test_moe_argument_checks(L):
+    buf = (ctypes.c_char * 512)()
+    a = (ctypes.addressof(buf) + 255) & ~255
+    ok = dict(fmt=4, T=4, H=2048, I=768, E=128, topk=8)
+
+    def args(**kw):
+        d = dict(ok, **kw)
+        return qmm.MoeArgs(d["T"], d["H"], d["I"], d["E"], d["topk"], d["fmt"], a, a, a, a, a, a, 0, 0, 0, 0, 0, 0)
+
+    assert L.qmm_moe(None, a, 0, None) == 1
+    assert L.qmm_moe(ctypes.byref(args(topk=200)), a, 1 << 30, None) == 2
+    assert L.qmm_moe(ctypes.byref(args(E=0)), a, 1 << 30, None) == 1
+    assert L.qmm_moe(ctypes.byref(args(H=2000)), a, 1 << 30, None) == 2
+    assert L.qmm_moe(ctypes.byref(args(I=96)), a, 1 << 30, None) == 5
+    assert L.qmm_moe(ctypes.byref(args()), a, 16, None) == 4
+    assert L.qmm_moe_workspace_bytes(ctypes.byref(args())) > 0
+    assert L.qmm_moe_workspace_bytes(ctypes.byref(args(fmt=3))) == 0
+
+
+def test_error_buffer_is_thread_local(L):
+    import threading
+    buf = (ctypes.c_char * 64)()
+    addr = ctypes.addressof(buf)
+    L.qmm_pack(4, addr, 128, 100, addr, None)
+    mine = qmm.last_error()
+    seen = []
+    t = threading.Thread(target=lambda: seen.append(qmm.last_error()))
+    t.start()
+    t.join()
+    assert "K=100" in mine and seen == [""]
