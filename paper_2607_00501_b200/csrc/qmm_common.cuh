@@ -111,19 +111,40 @@ __device__ __forceinline__ uint32_t as_u32(__half2 h)
     return *reinterpret_cast<uint32_t*>(&h);
 }
 
+// Bit constants of the Q4 unpack, held in registers.  (a & mask) | magic is one
+// LOP3 only when at most one of its operands is an immediate, so the values
+// are produced by opaque moves that the compiler cannot fold back into
+// immediates.
+struct Q4Consts {
+    uint32_t mask_lo, mask_hi, magic;
+    __device__ __forceinline__ void init()
+    {
+        asm volatile("mov.u32 %0, 0x000F000F;" : "=r"(mask_lo));
+        asm volatile("mov.u32 %0, 0x00F000F0;" : "=r"(mask_hi));
+        asm volatile("mov.u32 %0, 0x64006400;" : "=r"(magic));
+    }
+};
+
+__device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t b, uint32_t c)
+{
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(b), "r"(c));   // (a & b) | c
+    return d;
+}
+
 // Q4: the four element pairs of one packed word as exact integers q in fp16.
 // 0x6400 | u is the fp16 value 1024 + u; 0x6400 | (u << 4) is 1024 + 16 u.
 // (1024 + u) - 1032 = q and (1024 + 16 u) / 16 - 72 = q are both exact.
-__device__ __forceinline__ void q4_word_to_h2(uint32_t w, __half2 (&q)[4])
+__device__ __forceinline__ void q4_word_to_h2(uint32_t w, __half2 (&q)[4], const Q4Consts& k)
 {
     const __half2 c1032 = as_h2(0x64086408u);
     const __half2 c16th = as_h2(0x2C002C00u);
     const __half2 cm72 = as_h2(0xD480D480u);
     const uint32_t w8 = w >> 8;
-    q[0] = __hsub2(as_h2((w & 0x000F000Fu) | 0x64006400u), c1032);
-    q[1] = __hfma2(as_h2((w & 0x00F000F0u) | 0x64006400u), c16th, cm72);
-    q[2] = __hsub2(as_h2((w8 & 0x000F000Fu) | 0x64006400u), c1032);
-    q[3] = __hfma2(as_h2((w8 & 0x00F000F0u) | 0x64006400u), c16th, cm72);
+    q[0] = __hsub2(as_h2(and_or(w, k.mask_lo, k.magic)), c1032);
+    q[1] = __hfma2(as_h2(and_or(w, k.mask_hi, k.magic)), c16th, cm72);
+    q[2] = __hsub2(as_h2(and_or(w8, k.mask_lo, k.magic)), c1032);
+    q[3] = __hfma2(as_h2(and_or(w8, k.mask_hi, k.magic)), c16th, cm72);
 }
 
 // Q8: the two element pairs of one packed word (4 offset-binary bytes) as

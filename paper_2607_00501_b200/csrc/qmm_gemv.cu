@@ -50,7 +50,7 @@ __device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1
 
 // Q4: tile = 64 k.  acc[0..1] rows of P, acc[2..3] rows of Q (see above).
 __device__ __forceinline__ void tile_pair_mma_q4(const u32x8& cp, const u32x8& cq, uint2 sp, uint2 sq,
-                                                 const uint4* xt, float (&acc)[4])
+                                                 const uint4* xt, float (&acc)[4], const Q4Consts& kc)
 {
 #pragma unroll
     for (int b = 0; b < 2; ++b) {
@@ -59,8 +59,8 @@ __device__ __forceinline__ void tile_pair_mma_q4(const u32x8& cp, const u32x8& c
         for (int i = 0; i < 4; ++i) {
             const uint4 xv = xt[b * 4 + i];                      // activations k = 8(4b+i) .. +7
             __half2 p[4], q[4];
-            q4_word_to_h2(cp.v[b * 4 + i], p);
-            q4_word_to_h2(cq.v[b * 4 + i], q);
+            q4_word_to_h2(cp.v[b * 4 + i], p, kc);
+            q4_word_to_h2(cq.v[b * 4 + i], q, kc);
             mma16816(c, as_u32(p[0]), as_u32(q[0]), as_u32(p[1]), as_u32(q[1]), xv.x, xv.y);
             mma16816(c, as_u32(p[2]), as_u32(q[2]), as_u32(p[3]), as_u32(q[3]), xv.z, xv.w);
         }
@@ -183,6 +183,8 @@ gemv_kernel(const uint8_t* __restrict__ packed, const uint16_t* __restrict__ x,
     }
     __syncthreads();
     const uint4* xb = ((lane >> 2) == (lane & 3)) ? xs : zs;
+    Q4Consts kc;
+    kc.init();
 
     while (item < items) {
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
@@ -192,7 +194,7 @@ gemv_kernel(const uint8_t* __restrict__ packed, const uint16_t* __restrict__ x,
                 const int tt = t + u * WARPS;
                 if (tt < t_end) {
                     if constexpr (FMT == QMM_Q4)
-                        tile_pair_mma_q4(r.cp[u], r.cq[u], r.sp[u], r.sq[u], xb + tt * XV, acc);
+                        tile_pair_mma_q4(r.cp[u], r.cq[u], r.sp[u], r.sq[u], xb + tt * XV, acc, kc);
                     else
                         tile_pair_mma_q8(r.cp[u], r.cq[u], r.sp[u], r.sq[u], xb + tt * XV, acc);
                 }
