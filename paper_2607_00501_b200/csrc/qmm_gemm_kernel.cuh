@@ -1,0 +1,324 @@
+// qmm_gemm_kernel.cuh -- tensor-core product of packed Q4/Q8 weights with fp16
+// activations, shared by the dense prefill GEMM and the grouped expert GEMMs.
+//
+// The paper's prefill kernels are tiled GEMMs that dequantise in the inner
+// loop (Sec. 3.3, Sec. 3.4).  On B200 the contraction runs on tcgen05 tensor
+// cores, which cannot read 4/8-bit codes with fp16 block scales, so CUDA cores
+// expand codes to fp16 weights and hand them to the tensor core *through
+// tensor memory*: tcgen05.mma takes its A operand from TMEM, so the expanded
+// weights never touch shared memory or L2.
+//
+// Orientation.  Weights sit on the MMA M axis (128 rows = 128 TMEM lanes, one
+// weight row per lane -- the same "one row per lane" order the packed layout
+// has), tokens on the MMA N axis:  D[n, m] = sum_k W[n, k] * X[m, k].
+//
+// One thread block computes NA (1 or 2) weight tiles of 128 rows against one
+// tile of BN tokens; with NA = 2 both weight tiles reuse the same activation
+// tile (half the activation traffic; the gate and up matrices of an expert).
+//
+// Roles (warp specialised):
+//   warps 0 .. 4*NA-1  expanders: thread = one weight row; 32-byte code loads
+//                      straight from global/L2, unpack to fp16(d*q), tcgen05.st
+//                      into the A ring in TMEM; afterwards the epilogue.
+//   warp 4*NA          TMA producer: activation tiles -> shared-memory ring
+//                      (128-byte swizzle), one elected lane.
+//   warp 4*NA+1        MMA issuer: one elected lane issues tcgen05.mma
+//                      (M128 x N=BN x K16), frees ring slots with tcgen05.commit.
+//
+// TMEM columns: [0, NA*BN) fp32 accumulators, then STAGES slots of NA*32
+// columns (64 fp16 k-values per row and weight tile).
+//
+// Every mbarrier wait is bounded; on give-up the block raises an abort flag,
+// records QMM_ERR_DEVICE_TIMEOUT in the status word, stops issuing work, waits
+// (bounded) for its outstanding TMA loads, frees its TMEM and returns.
+#pragma once
+
+#include "qmm_common.cuh"
+#include "qmm_tc.cuh"
+
+namespace qmm {
+
+constexpr int kGemmBK = 64;          // k per pipeline stage
+constexpr int kGemmStages = 4;
+
+enum GemmEpilogue { kEpiStore = 0, kEpiSiluMul = 1 };
+
+struct GemmParams {
+    const uint8_t* w[2];             // packed weights of tile set 0 / 1 (expert 0)
+    int64_t w_expert_stride;         // bytes between experts (grouped), else 0
+    int N, K;                        // weight matrix [N, K] (per expert)
+    uint16_t* out;                   // [rows, ldo] fp16
+    int64_t ldo;
+    int a_col_offset;                // output column offset of tile set 1 (plain store epilogue)
+    int M;                           // rows of X / out (dense); capacity of the row space (grouped)
+    // grouped mode (tile_expert != nullptr): token tiles come from a device-built list
+    const int* tile_expert;          // [max_tiles] expert of token tile y
+    const int* tile_row0;            // [max_tiles] first permuted row of the tile
+    const int* tile_rows;            // [max_tiles] valid rows in the tile (<= BN)
+    const int* num_tiles;            // [1]
+    int* status;                     // device status word (0 = ok)
+};
+
+template <int BN, int NA>
+struct GemmSmem {
+    static constexpr int kBStage = BN * kGemmBK * 2;                       // bytes per activation stage
+    static constexpr int kBarriers = 3 * kGemmStages + 1;
+    static constexpr int kBytes = kGemmStages * kBStage + 1024 /*align*/ + 256;
+};
+
+__device__ __forceinline__ float silu_f(float g) { return g / (1.0f + __expf(-g)); }
+
+// One 64-k slice of a weight row as loaded (codes + scales), and its expansion
+// to fp16(d * q) pairs, k ascending.  Loading and expanding are separate so
+// that the loads of later slices can be in flight while one is expanded.
+template <int FMT> struct RawRow64;
+template <> struct RawRow64<QMM_Q4> {
+    u32x8 c;
+    uint32_t sc;
+    __device__ __forceinline__ void load(const uint8_t* tile_ptr, int lane)
+    {
+        c = ld_keep_256(tile_ptr + 32 * lane);
+        sc = ld_nc_u32(tile_ptr + kTileCodeBytes + 4 * lane);
+    }
+    __device__ __forceinline__ void expand(uint32_t (&out)[32], const Q4Consts& kc) const
+    {
+        const __half2 d0 = __half2half2(__low2half(as_h2(sc)));
+        const __half2 d1 = __half2half2(__high2half(as_h2(sc)));
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            __half2 q[4];
+            q4_word_to_h2(c.v[j], q, kc);
+            const __half2 d = j < 4 ? d0 : d1;
+#pragma unroll
+            for (int p = 0; p < 4; ++p) out[4 * j + p] = as_u32(__hmul2(q[p], d));
+        }
+    }
+};
+template <> struct RawRow64<QMM_Q8> {
+    u32x8 c[2];
+    uint16_t sc[2];
+    __device__ __forceinline__ void load(const uint8_t* tile_ptr, int lane)
+    {
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {                                     // two 32-k tiles
+            const uint8_t* tp = tile_ptr + t * kQ8TileBytes;
+            c[t] = ld_keep_256(tp + 32 * lane);
+            sc[t] = ld_nc_u16(tp + kTileCodeBytes + 2 * lane);
+        }
+    }
+    __device__ __forceinline__ void expand(uint32_t (&out)[32], const Q4Consts&) const
+    {
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+            const __half2 d = __half2half2(__ushort_as_half(sc[t]));
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                __half2 q[2];
+                q8_word_to_h2(c[t].v[j], q);
+                out[16 * t + 2 * j] = as_u32(__hmul2(q[0], d));
+                out[16 * t + 2 * j + 1] = as_u32(__hmul2(q[1], d));
+            }
+        }
+    }
+};
+
+constexpr int kGemmPrefetch = 4;     // weight slices in flight per expander thread
+
+template <int FMT, int BN, int NA, int EPI>
+__global__ void __launch_bounds__((4 * NA + 2) * 32, 1)
+gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
+{
+    using namespace tc;
+    constexpr int NEXP = 4 * NA;                      // expander warps
+    constexpr int TMA_WARP = NEXP, MMA_WARP = NEXP + 1;
+    constexpr int S = kGemmStages;
+    constexpr int A_COLS = NA * 32;                   // TMEM columns per A stage
+    constexpr int D_COLS = NA * BN;
+    constexpr int TMEM_COLS = (D_COLS + S * A_COLS) <= 128 ? 128 : (D_COLS + S * A_COLS) <= 256 ? 256 : 512;
+    static_assert(D_COLS + S * A_COLS <= 512, "tensor memory over-subscribed");
+    static_assert(BN % 16 == 0 && BN >= 16 && BN <= 256, "MMA N");
+    constexpr int B_STAGE = BN * kGemmBK * 2;
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t* smem_b = smem;                                               // S stages, 1024-aligned each
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S * B_STAGE);
+    uint64_t* a_full = bars;                                              // [S] expanders -> MMA
+    uint64_t* b_full = bars + S;                                          // [S] TMA -> MMA
+    uint64_t* empty = bars + 2 * S;                                       // [S] MMA -> producers
+    uint64_t* acc_full = bars + 3 * S;                                    // MMA -> epilogue
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3 * S + 1);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    // ---- which tile
+    const int n_tile = blockIdx.x;                                        // 128 weight rows (per tile set)
+    int expert = 0, row0, rows;
+    if (p.tile_expert != nullptr) {
+        pdl_wait();                                                       // the tile list is written upstream
+        if ((int)blockIdx.y >= *p.num_tiles) return;                      // uniform over the block
+        expert = p.tile_expert[blockIdx.y];
+        row0 = p.tile_row0[blockIdx.y];
+        rows = p.tile_rows[blockIdx.y];
+    } else {
+        row0 = blockIdx.y * BN;
+        rows = min(BN, p.M - row0);
+    }
+    const int num_kb = p.K / kGemmBK;
+
+    // ---- set-up
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(&a_full[s], NEXP);                                  // one arrival per expander warp
+            mbar_init(&b_full[s], 1);
+            mbar_init(&empty[s], 1);
+        }
+        mbar_init(acc_full, 1);
+        *abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == MMA_WARP) {
+        tmem_alloc(tmem_slot, TMEM_COLS);
+        tmem_relinquish();
+    }
+    if (warp == TMA_WARP && lane == 0) prefetch_tensormap(&x_map);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    pdl_launch_dependents();
+
+    if (warp < NEXP) {
+        // ================= expanders: weights -> fp16 -> TMEM A ring
+        const int a = warp >> 2;                                          // weight tile set
+        const int quarter = warp & 3;                                     // TMEM lane quarter
+        const int rg = n_tile * 4 + quarter;                              // row group of 32 rows
+        const int tpr = p.K / Fmt<FMT>::tile_k;
+        constexpr int TILES_PER_KB = kGemmBK / Fmt<FMT>::tile_k;
+        const uint8_t* wrow = p.w[a] + (size_t)expert * p.w_expert_stride + (size_t)rg * tpr * Fmt<FMT>::tile_bytes;
+        Q4Consts kc;
+        kc.init();
+        const size_t kb_bytes = (size_t)TILES_PER_KB * Fmt<FMT>::tile_bytes;
+        RawRow64<FMT> raw[kGemmPrefetch];
+#pragma unroll
+        for (int i = 0; i < kGemmPrefetch; ++i)
+            if (i < num_kb) raw[i].load(wrow + i * kb_bytes, lane);
+        bool ok = true;
+        for (int kb0 = 0; kb0 < num_kb && ok; kb0 += kGemmPrefetch) {
+#pragma unroll
+            for (int i = 0; i < kGemmPrefetch; ++i) {
+                const int kb = kb0 + i;
+                if (kb >= num_kb || !ok) break;
+                const int s = kb % S;
+                uint32_t vals[32];
+                raw[i].expand(vals, kc);
+                if (kb + kGemmPrefetch < num_kb) raw[i].load(wrow + (size_t)(kb + kGemmPrefetch) * kb_bytes, lane);
+                if (kb >= S) ok = mbar_wait(&empty[s], ((kb / S) - 1) & 1, abort_flag);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(D_COLS + s * A_COLS + a * 32);
+                tmem_st_32x32b_x32(taddr, vals);
+                tmem_wait_st();
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&a_full[s]);
+            }
+        }
+        if (!ok) *abort_flag = 1;
+
+        // ================= epilogue: TMEM -> registers -> global
+        if (p.out != nullptr) {
+            pdl_wait();                                                   // the output buffer may be in use upstream
+            bool acc_ok = ok && mbar_wait(acc_full, 0, abort_flag);
+            acc_ok = __all_sync(0xFFFFFFFFu, acc_ok);
+            if (!acc_ok) {
+                *abort_flag = 1;
+            } else if (EPI == kEpiStore || a == 0) {
+                tc_fence_after_sync();
+                const int n = n_tile * 128 + quarter * 32 + lane;         // weight row within the tile set
+                for (int c0 = 0; c0 < BN; c0 += 32) {
+                    if (c0 >= rows) break;                                // uniform
+                    uint32_t v[32];
+                    const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+                    tmem_ld_32x32b_x32(lane_addr + (uint32_t)(a * BN + c0), v);
+                    if (EPI == kEpiSiluMul) {
+                        uint32_t u[32];
+                        tmem_ld_32x32b_x32(lane_addr + (uint32_t)(BN + c0), u);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(silu_f(__uint_as_float(v[j])) * __uint_as_float(u[j]));
+                    } else {
+                        tmem_wait_ld();
+                    }
+                    uint16_t* o = p.out + (size_t)(row0 + c0) * p.ldo + (EPI == kEpiStore ? (size_t)a * p.a_col_offset : 0) + n;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (c0 + j < rows) o[(size_t)j * p.ldo] = __half_as_ushort(__float2half_rn(__uint_as_float(v[j])));
+                }
+            }
+        }
+    } else if (warp == TMA_WARP) {
+        // ================= TMA producer: activation tiles
+        if (lane == 0) {
+            pdl_wait();                                                   // activations come from the previous kernel
+            int issued = 0;
+            bool ok = true;
+            for (int kb = 0; kb < num_kb; ++kb) {
+                const int s = kb % S;
+                if (kb >= S) ok = mbar_wait(&empty[s], ((kb / S) - 1) & 1, abort_flag);
+                if (!ok) break;
+                mbar_arrive_expect_tx(&b_full[s], B_STAGE);
+                tma_load_2d(smem_b + s * B_STAGE, &x_map, kb * kGemmBK, row0, &b_full[s]);
+                issued = kb + 1;
+            }
+            if (!ok) {
+                *abort_flag = 1;
+                // let loads in flight land before the block's shared memory is released
+                for (int kb = max(0, issued - S); kb < issued; ++kb) {
+                    const long long t0 = clock64();
+                    while (!mbar_try_wait(&b_full[kb % S], (kb / S) & 1) && clock64() - t0 < kWaitLimitCycles) {}
+                }
+            }
+        }
+    } else {
+        // ================= MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = idesc_f16_m128(BN);
+            bool ok = true;
+            for (int kb = 0; kb < num_kb; ++kb) {
+                const int s = kb % S;
+                const uint32_t ph = (kb / S) & 1;
+                ok = mbar_wait(&a_full[s], ph, abort_flag) && mbar_wait(&b_full[s], ph, abort_flag);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t b_addr = smem_u32(smem_b + s * B_STAGE);
+#pragma unroll
+                for (int a = 0; a < NA; ++a) {
+#pragma unroll
+                    for (int k = 0; k < kGemmBK / 16; ++k) {
+                        const uint64_t bdesc = smem_desc_k_sw128(b_addr + k * 32);
+                        const uint32_t a_tmem = tmem_base + (uint32_t)(D_COLS + s * A_COLS + a * 32 + k * 8);
+                        mma_ts_f16(tmem_base + (uint32_t)(a * BN), a_tmem, bdesc, idesc, (kb | k) != 0);
+                    }
+                }
+                mma_commit(&empty[s]);                                    // slot reusable when these MMAs finish
+            }
+            if (ok) mma_commit(acc_full);
+            else *abort_flag = 1;
+        }
+    }
+
+    // ---- teardown
+    tc_fence_before_sync();
+    __syncthreads();
+    if (threadIdx.x == 0 && *abort_flag && p.status != nullptr) atomicExch(p.status, (int)QMM_ERR_DEVICE_TIMEOUT);
+    if (warp == MMA_WARP) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+}  // namespace qmm

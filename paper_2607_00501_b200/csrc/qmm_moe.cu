@@ -1,6 +1,370 @@
-// placeholder until the MoE path lands
-#include "qmm_common.cuh"
+// qmm_moe.cu -- top-k mixture-of-experts feed-forward layer on packed weights.
+//
+// The paper reports its largest prefill gains on mixture-of-experts models
+// (Sec. 4.3) and lists "mixture-of-experts specifics" among the things its
+// architecture descriptor carries (Sec. 3.1), but gives no algorithm; the
+// steps below are this library's definition (see include/qmm.h):
+//   route  -> stable permutation by (expert, token) -> gather rows ->
+//   grouped gate/up GEMM with SiLU*mul epilogue -> grouped down GEMM ->
+//   weighted combine in slot order.
+// Nothing synchronises with the host: the token-tile work list of the grouped
+// GEMMs is built on the device from the expert offsets.
+#include "qmm_gemm_kernel.cuh"
+
 namespace qmm {
-size_t moe_workspace_bytes(const qmm_moe_args*) { return 256; }
-qmm_status launch_moe(const qmm_moe_args*, void*, bool, cudaStream_t) { return fail(QMM_ERR_UNSUPPORTED, "qmm_moe: not built yet"); }
+
+qmm_status make_x_map(CUtensorMap* map, const uint16_t* X, int64_t rows, int64_t K, int64_t ld, int box_rows);
+qmm_status launch_tc_gemm(int fmt, int bn, int na, int epi, const CUtensorMap& map, const GemmParams& p, dim3 grid,
+                          cudaStream_t st);
+int pick_token_tile(int64_t rows);
+
+// ------------------------------------------------------------ workspace
+
+struct MoeWorkspace {
+    size_t status, counts, offsets, num_tiles, tile_expert, tile_row0, tile_rows;
+    size_t topk_idx, topk_w, perm, inv_perm, xp, hbuf, dbuf, total;
+    int bn, max_tiles;
+};
+
+static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+static MoeWorkspace moe_layout(const qmm_moe_args* a)
+{
+    MoeWorkspace w;
+    const size_t rows = (size_t)a->T * a->topk;
+    w.bn = pick_token_tile((int64_t)((rows + a->E - 1) / a->E));           // mean rows per expert
+    w.max_tiles = (int)((rows + w.bn - 1) / w.bn) + a->E;
+    size_t o = 0;
+    auto take = [&](size_t bytes) { const size_t at = o; o = align_up(o + bytes, 256); return at; };
+    w.status = take(256);
+    w.counts = take((size_t)a->E * 4);
+    w.offsets = take((size_t)(a->E + 1) * 4);
+    w.num_tiles = take(4);
+    w.tile_expert = take((size_t)w.max_tiles * 4);
+    w.tile_row0 = take((size_t)w.max_tiles * 4);
+    w.tile_rows = take((size_t)w.max_tiles * 4);
+    w.topk_idx = take(rows * 4);
+    w.topk_w = take(rows * 4);
+    w.perm = take(rows * 4);
+    w.inv_perm = take(rows * 4);
+    w.xp = take(rows * (size_t)a->H * 2);
+    w.hbuf = take(rows * (size_t)a->I * 2);
+    w.dbuf = take(rows * (size_t)a->H * 2);
+    w.total = o;
+    return w;
 }
+
+size_t moe_workspace_bytes(const qmm_moe_args* a) { return moe_layout(a).total; }
+
+// ---------------------------------------------------------------- route
+
+// One warp per token.  topk passes; each pass takes the largest remaining
+// logit, equal logits going to the lower expert index.  The weights are the
+// softmax over the selected logits in fp32.  Also counts rows per expert.
+template <int MAX_PER_LANE>
+__global__ void route_kernel(const float* __restrict__ logits, int T, int E, int topk,
+                             int* __restrict__ idx_out, float* __restrict__ w_out,
+                             int* __restrict__ idx_user, float* __restrict__ w_user, int* __restrict__ counts)
+{
+    pdl_launch_dependents();
+    pdl_wait();
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (warp >= T) return;
+    const float* l = logits + (size_t)warp * E;
+    float v[MAX_PER_LANE];
+#pragma unroll
+    for (int i = 0; i < MAX_PER_LANE; ++i) {
+        const int e = lane + 32 * i;
+        v[i] = e < E ? l[e] : -INFINITY;
+    }
+    unsigned taken = 0;                                   // bit i: v[i] already selected
+    float sel_val = 0.f, lmax = 0.f, denom = 0.f;         // lane j keeps the j-th selected logit
+    int sel_idx = 0;
+    for (int j = 0; j < topk; ++j) {
+        float best = -INFINITY;
+        int best_e = 0x7FFFFFFF;
+#pragma unroll
+        for (int i = 0; i < MAX_PER_LANE; ++i) {
+            const int e = lane + 32 * i;
+            if (e < E && !((taken >> i) & 1u) && (v[i] > best || (v[i] == best && e < best_e))) {
+                best = v[i];
+                best_e = e;
+            }
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            const float ob = __shfl_xor_sync(0xFFFFFFFFu, best, off);
+            const int oe = __shfl_xor_sync(0xFFFFFFFFu, best_e, off);
+            if (ob > best || (ob == best && oe < best_e)) {
+                best = ob;
+                best_e = oe;
+            }
+        }
+        if ((best_e & 31) == lane) taken |= 1u << (best_e >> 5);
+        if (j == 0) lmax = best;
+        if (lane == j) {
+            sel_val = best;
+            sel_idx = best_e;
+        }
+        denom += expf(best - lmax);                       // same value and order on every lane
+    }
+    if (lane < topk) {
+        const float w = expf(sel_val - lmax) / denom;
+        const size_t o = (size_t)warp * topk + lane;
+        idx_out[o] = sel_idx;
+        w_out[o] = w;
+        if (idx_user) idx_user[o] = sel_idx;
+        if (w_user) w_user[o] = w;
+        atomicAdd(&counts[sel_idx], 1);                   // a count: the order of the adds does not matter
+    }
+}
+
+// One block: exclusive scan of the per-expert counts -> expert_offsets, and the
+// token-tile list of the grouped GEMMs (expert, first row, valid rows).
+__global__ void offsets_kernel(const int* __restrict__ counts, int E, int bn,
+                               int* __restrict__ offsets, int* __restrict__ offsets_user,
+                               int* __restrict__ num_tiles, int* __restrict__ tile_expert,
+                               int* __restrict__ tile_row0, int* __restrict__ tile_rows)
+{
+    pdl_launch_dependents();
+    pdl_wait();
+    __shared__ int s_cnt[1024], s_off[1025], s_toff[1025];
+    const int e = threadIdx.x;
+    s_cnt[e] = e < E ? counts[e] : 0;
+    __syncthreads();
+    if (threadIdx.x == 0) {                               // E <= 1024: a serial scan is a few microseconds
+        int o = 0, t = 0;
+        for (int i = 0; i < E; ++i) {
+            s_off[i] = o;
+            s_toff[i] = t;
+            o += s_cnt[i];
+            t += (s_cnt[i] + bn - 1) / bn;
+        }
+        s_off[E] = o;
+        s_toff[E] = t;
+        *num_tiles = t;
+        offsets[E] = o;
+        if (offsets_user) offsets_user[E] = o;
+    }
+    __syncthreads();
+    if (e < E) {
+        offsets[e] = s_off[e];
+        if (offsets_user) offsets_user[e] = s_off[e];
+    }
+    if (e < E) {
+        const int nt = s_toff[e + 1] - s_toff[e];
+        for (int i = 0; i < nt; ++i) {
+            const int y = s_toff[e] + i;
+            tile_expert[y] = e;
+            tile_row0[y] = s_off[e] + i * bn;
+            tile_rows[y] = min(bn, s_cnt[e] - i * bn);
+        }
+    }
+}
+
+// One block per expert: walks the T*topk (token, slot) pairs in flat order and
+// appends those routed to this expert, which yields the stable order by
+// (expert, token).  perm[r] = flat index, inv_perm[flat] = r.
+__global__ void permute_kernel(const int* __restrict__ topk_idx, int total, const int* __restrict__ offsets,
+                               int* __restrict__ perm, int* __restrict__ perm_user, int* __restrict__ inv_perm)
+{
+    pdl_launch_dependents();
+    pdl_wait();
+    __shared__ int s_warp[8];
+    __shared__ int s_base;
+    const int e = blockIdx.x;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) s_base = offsets[e];
+    __syncthreads();
+    for (int start = 0; start < total; start += 256) {
+        const int i = start + threadIdx.x;
+        const bool mine = i < total && topk_idx[i] == e;
+        const unsigned ballot = __ballot_sync(0xFFFFFFFFu, mine);
+        if (lane == 0) s_warp[warp] = __popc(ballot);
+        __syncthreads();
+        int before = 0, all = 0;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) {
+            if (w < warp) before += s_warp[w];
+            all += s_warp[w];
+        }
+        if (mine) {
+            const int r = s_base + before + __popc(ballot & ((1u << lane) - 1u));
+            perm[r] = i;
+            if (perm_user) perm_user[r] = i;
+            inv_perm[i] = r;
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) s_base += all;
+        __syncthreads();
+    }
+}
+
+// One warp per permuted row: copy the token's activations into expert order.
+__global__ void gather_rows_kernel(const uint16_t* __restrict__ X, const int* __restrict__ perm, int total, int topk,
+                                   int H, uint16_t* __restrict__ Xp)
+{
+    pdl_launch_dependents();
+    pdl_wait();
+    const int r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (r >= total) return;
+    const int t = perm[r] / topk;
+    const uint4* src = reinterpret_cast<const uint4*>(X + (size_t)t * H);
+    uint4* dst = reinterpret_cast<uint4*>(Xp + (size_t)r * H);
+    for (int i = lane; i < H / 8; i += 32) dst[i] = src[i];
+}
+
+// out[t, :] = fp16( sum_j p[t, j] * D[inv_perm[t*topk + j], :] ), fp32, j ascending.
+// One block per token; each thread owns 8 consecutive columns.
+__global__ void combine_kernel(const uint16_t* __restrict__ D, const int* __restrict__ inv_perm,
+                               const float* __restrict__ topk_w, int topk, int H, uint16_t* __restrict__ out)
+{
+    pdl_launch_dependents();
+    pdl_wait();
+    const int t = blockIdx.x;
+    for (int c = threadIdx.x * 8; c < H; c += blockDim.x * 8) {
+        float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        for (int j = 0; j < topk; ++j) {
+            const int r = inv_perm[t * topk + j];
+            const float p = topk_w[t * topk + j];
+            const uint4 d = *reinterpret_cast<const uint4*>(D + (size_t)r * H + c);
+            const __half2* h = reinterpret_cast<const __half2*>(&d);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float2 f = __half22float2(h[i]);
+                acc[2 * i] = fmaf(p, f.x, acc[2 * i]);
+                acc[2 * i + 1] = fmaf(p, f.y, acc[2 * i + 1]);
+            }
+        }
+        uint4 o;
+        __half2* oh = reinterpret_cast<__half2*>(&o);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) oh[i] = __floats2half2_rn(acc[2 * i], acc[2 * i + 1]);
+        *reinterpret_cast<uint4*>(out + (size_t)t * H + c) = o;
+    }
+}
+
+// ------------------------------------------------------------------ host
+
+template <typename... Args>
+static cudaError_t launch_pdl(void (*kernel)(Args...), dim3 grid, dim3 block, cudaStream_t st, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
+qmm_status launch_moe(const qmm_moe_args* a, void* ws, bool route_only, cudaStream_t st)
+{
+    const MoeWorkspace w = moe_layout(a);
+    uint8_t* base = (uint8_t*)ws;
+    int* status = (int*)(base + w.status);
+    int* counts = (int*)(base + w.counts);
+    int* offsets = (int*)(base + w.offsets);
+    int* num_tiles = (int*)(base + w.num_tiles);
+    int* tile_expert = (int*)(base + w.tile_expert);
+    int* tile_row0 = (int*)(base + w.tile_row0);
+    int* tile_rows = (int*)(base + w.tile_rows);
+    int* topk_idx = (int*)(base + w.topk_idx);
+    float* topk_w = (float*)(base + w.topk_w);
+    int* perm = (int*)(base + w.perm);
+    int* inv_perm = (int*)(base + w.inv_perm);
+    uint16_t* xp = (uint16_t*)(base + w.xp);
+    uint16_t* hbuf = a->dbg_H ? a->dbg_H : (uint16_t*)(base + w.hbuf);
+    uint16_t* dbuf = a->dbg_D ? a->dbg_D : (uint16_t*)(base + w.dbuf);
+    const int total = a->T * a->topk;
+
+    cudaError_t e = cudaMemsetAsync(counts, 0, (size_t)a->E * 4, st);
+    if (e != cudaSuccess) return check_cuda(e, "qmm_moe clear counts");
+
+    // 1. routing
+    {
+        const int warps_per_block = 8;
+        const dim3 grid((a->T + warps_per_block - 1) / warps_per_block), block(warps_per_block * 32);
+        const int per_lane = (a->E + 31) / 32;
+        if (per_lane <= 4)
+            e = launch_pdl(route_kernel<4>, grid, block, st, a->logits, (int)a->T, (int)a->E, (int)a->topk, topk_idx, topk_w,
+                           a->topk_idx, a->topk_w, counts);
+        else
+            e = launch_pdl(route_kernel<32>, grid, block, st, a->logits, (int)a->T, (int)a->E, (int)a->topk, topk_idx, topk_w,
+                           a->topk_idx, a->topk_w, counts);
+        if (e != cudaSuccess) return check_cuda(e, "qmm_moe route launch");
+    }
+    // 2. offsets + tile list, stable permutation
+    e = launch_pdl(offsets_kernel, dim3(1), dim3(1024), st, (const int*)counts, (int)a->E, w.bn, offsets, a->expert_offsets,
+                   num_tiles, tile_expert, tile_row0, tile_rows);
+    if (e != cudaSuccess) return check_cuda(e, "qmm_moe offsets launch");
+    e = launch_pdl(permute_kernel, dim3(a->E), dim3(256), st, (const int*)topk_idx, total, (const int*)offsets, perm, a->perm,
+                   inv_perm);
+    if (e != cudaSuccess) return check_cuda(e, "qmm_moe permute launch");
+    if (route_only) return QMM_OK;
+
+    // 3. gather rows into expert order
+    e = launch_pdl(gather_rows_kernel, dim3((total + 7) / 8), dim3(256), st, a->X, (const int*)perm, total, (int)a->topk,
+                   (int)a->H, xp);
+    if (e != cudaSuccess) return check_cuda(e, "qmm_moe gather launch");
+
+    // 4. grouped gate/up GEMM with SiLU*mul epilogue -> Hm [total, I]
+    const size_t gu_stride = (size_t)(a->I / kRowsPerGroup) * (size_t)(a->H / tile_k_of(a->fmt)) * tile_bytes_of(a->fmt);
+    const size_t dn_stride = (size_t)(a->H / kRowsPerGroup) * (size_t)(a->I / tile_k_of(a->fmt)) * tile_bytes_of(a->fmt);
+    {
+        CUtensorMap map;
+        qmm_status s = make_x_map(&map, xp, total, a->H, a->H, w.bn);
+        if (s != QMM_OK) return s;
+        GemmParams p = {};
+        p.w[0] = (const uint8_t*)a->w_gate;
+        p.w[1] = (const uint8_t*)a->w_up;
+        p.w_expert_stride = (int64_t)gu_stride;
+        p.N = a->I;
+        p.K = a->H;
+        p.out = hbuf;
+        p.ldo = a->I;
+        p.a_col_offset = 0;
+        p.M = total;
+        p.tile_expert = tile_expert;
+        p.tile_row0 = tile_row0;
+        p.tile_rows = tile_rows;
+        p.num_tiles = num_tiles;
+        p.status = status;
+        s = launch_tc_gemm(a->fmt, w.bn, 2, kEpiSiluMul, map, p, dim3(a->I / 128, w.max_tiles), st);
+        if (s != QMM_OK) return s;
+    }
+    // 5. grouped down GEMM -> D [total, H]
+    {
+        CUtensorMap map;
+        qmm_status s = make_x_map(&map, hbuf, total, a->I, a->I, w.bn);
+        if (s != QMM_OK) return s;
+        const int na = (a->H % 256 == 0) ? 2 : 1;
+        GemmParams p = {};
+        p.w[0] = (const uint8_t*)a->w_down;
+        p.w[1] = na == 2 ? (const uint8_t*)a->w_down + dn_stride / 2 : nullptr;
+        p.w_expert_stride = (int64_t)dn_stride;
+        p.N = a->H;
+        p.K = a->I;
+        p.out = dbuf;
+        p.ldo = a->H;
+        p.a_col_offset = a->H / 2;
+        p.M = total;
+        p.tile_expert = tile_expert;
+        p.tile_row0 = tile_row0;
+        p.tile_rows = tile_rows;
+        p.num_tiles = num_tiles;
+        p.status = status;
+        s = launch_tc_gemm(a->fmt, w.bn, na, kEpiStore, map, p, dim3(a->H / (128 * na), w.max_tiles), st);
+        if (s != QMM_OK) return s;
+    }
+    // 6. weighted combine
+    e = launch_pdl(combine_kernel, dim3(a->T), dim3(256), st, (const uint16_t*)dbuf, (const int*)inv_perm, (const float*)topk_w,
+                   (int)a->topk, (int)a->H, a->out);
+    if (e != cudaSuccess) return check_cuda(e, "qmm_moe combine launch");
+    return QMM_OK;
+}
+
+}  // namespace qmm

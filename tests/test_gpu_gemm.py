@@ -1,0 +1,93 @@
+"""GPU parity: qmm_gemm (tcgen05 tensor cores, weights expanded through tensor
+memory) against the CPU oracle.  Every output must satisfy
+|Y_gpu - Y_ref| <= 2e-3 * sum_k |w x| + 1e-5."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2607_00501_b200 import synth
+from tests import util
+
+pytestmark = pytest.mark.gpu
+Q4, Q8 = 4, 8
+
+
+@pytest.fixture(scope="module")
+def qmm():
+    from paper_2607_00501_b200 import qmm as _qmm
+    assert torch.cuda.is_available()
+    _qmm.lib()
+    return _qmm
+
+
+def run_gemm(qmm, oracle, fmt, blocks, N, K, X, what, rows=None):
+    packed = qmm.pack(fmt, util.dev(blocks), N, K)
+    ws = torch.zeros(qmm.gemm_workspace_bytes(fmt, X.shape[0], N, K), dtype=torch.uint8, device="cuda")
+    Y = qmm.gemm(fmt, packed, N, K, util.dev(X), ws=ws)
+    qmm.status_check(ws)
+    Yh = util.host_f64(Y)
+    sel = np.arange(X.shape[0]) if rows is None else np.asarray(rows)
+    Y_ref, B = oracle.gemm(fmt, blocks, N, K, X[sel])
+    return util.assert_within_tol(Yh[sel], Y_ref, B, what)
+
+
+@pytest.mark.parametrize("fmt", [Q4, Q8])
+@pytest.mark.parametrize("M,N,K", [(128, 128, 256), (32, 256, 256), (1, 128, 512), (77, 384, 768), (130, 256, 1024),
+                                   (200, 640, 512), (64, 128, 4096)])
+def test_gemm_small_shapes(qmm, oracle, fmt, M, N, K):
+    blocks, _, _ = util.random_blocks(synth, fmt, N, K, seed=M + 3 * N + K + fmt, special_scales=False)
+    X = synth.activations(70, M + N + K, M, K)
+    run_gemm(qmm, oracle, fmt, blocks, N, K, X, "gemm M=%d N=%d K=%d fmt=%d" % (M, N, K, fmt))
+
+
+@pytest.mark.parametrize("fmt", [Q4, Q8])
+def test_gemm_integer_case_is_exact(qmm, fmt):
+    # unit scales, small integer activations: every product and partial sum is an exact integer
+    rng = np.random.default_rng(17 + fmt)
+    M, N, K = 96, 256, 512
+    lo, hi = (-8, 8) if fmt == Q4 else (-127, 128)
+    codes = np.where(rng.random((N, K)) < (0.25 if fmt == Q4 else 0.01), rng.integers(lo, hi, size=(N, K)), 0)
+    Xi = rng.integers(-2, 3, size=(M, K))
+    ref = Xi.astype(np.int64) @ codes.T.astype(np.int64)
+    assert np.abs(ref).max() < 2048
+    blocks = synth.blocks_from_codes(fmt, np.full((N, K // 32), 0x3C00, dtype=np.uint16), codes)
+    packed = qmm.pack(fmt, util.dev(blocks), N, K)
+    Y = qmm.gemm(fmt, packed, N, K, util.dev(Xi.astype(np.float16)))
+    assert np.array_equal(util.host_f64(Y), ref.astype(np.float64))
+
+
+def test_gemm_strided_inputs_and_guard_bytes(qmm, oracle):
+    M, N, K = 100, 256, 512
+    blocks = synth.quantize(Q4, synth.weights(71, 0, N, K))
+    packed = qmm.pack(Q4, util.dev(blocks), N, K)
+    X = synth.activations(71, 1, M, K)
+    Xbuf = torch.full((M, K + 64), 9.0, dtype=torch.float16, device="cuda")
+    Xbuf[:, :K] = util.dev(X)
+    Ybuf = torch.full((M + 2, N + 16), 5.0, dtype=torch.float16, device="cuda")
+    qmm.gemm(Q4, packed, N, K, Xbuf[:, :K], Y=Ybuf[1:M + 1, :N])
+    Y_ref, B = oracle.gemm(Q4, blocks, N, K, X)
+    util.assert_within_tol(util.host_f64(Ybuf[1:M + 1, :N]), Y_ref, B, "strided")
+    assert torch.all(Ybuf[0] == 5.0) and torch.all(Ybuf[M + 1] == 5.0) and torch.all(Ybuf[:, N:] == 5.0)
+
+
+def test_gemm_matches_gemv_rows(qmm):
+    # the M = 1 product through both kernels agrees to fp16 rounding of nearly equal fp32 sums
+    N, K = 384, 1024
+    blocks = synth.quantize(Q8, synth.weights(72, 0, N, K))
+    packed = qmm.pack(Q8, util.dev(blocks), N, K)
+    x = util.dev(synth.activations(72, 1, K))
+    y1 = qmm.gemv(Q8, packed, N, K, x).float()
+    y2 = qmm.gemm(Q8, packed, N, K, x.reshape(1, K)).float()[0]
+    assert torch.allclose(y1, y2, rtol=4e-3, atol=1e-3)
+
+
+@pytest.mark.parametrize("shape", synth.CFG3["shapes"])
+@pytest.mark.parametrize("M", synth.CFG3["Ms"])
+def test_cfg3_prefill_full_size_sampled_rows(qmm, oracle, shape, M):
+    name, N, K = shape
+    c = synth.CFG3
+    blocks = synth.quantize(c["fmt"], synth.weights(c["seed"], 0 if name == "gate_up" else 1, N, K))
+    X = synth.activations(c["seed"], 10 + M, M, K)
+    rng = np.random.default_rng(M + N)
+    rows = np.unique(np.concatenate([[0, M - 1, M // 2], rng.integers(0, M, size=13)]))
+    run_gemm(qmm, oracle, c["fmt"], blocks, N, K, X, "cfg3 %s M=%d" % (name, M), rows=rows)
