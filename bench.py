@@ -1,0 +1,502 @@
+#!/usr/bin/env python
+"""Benchmark of the block-quantised dequantise-and-multiply path on B200.
+
+`python bench.py --gpus N --steps K --warmup W` prints ONE JSON line.
+
+Headline (`value`): effective HBM GB/s of the decode GEMV stack -- a 16-layer,
+1B-class transformer's linear layers at M = 1, in Q4 and in Q8 (the second
+benchmark configuration): quantised-weight bytes read per step / step time.
+One step = one pass over both stacks (every q/k/v/o/gate/up/down product of all
+16 layers, once in Q4 and once in Q8).  Extra sections in the same line time
+the other parts of the path on their own workloads: the Q8 LM-head GEMV, the
+Q4 prefill GEMM (tensor cores) and the Q4 mixture-of-experts layer.
+
+`--impl reference` times the CPU oracle (a deliberately plain program) on a
+bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2607_00501_b200 import synth  # noqa: E402
+
+METRIC = "decode GEMV effective HBM bandwidth on quantised-weight bytes (Q4+Q8 16-layer stack)"
+UNIT = "GB/s"
+NOMINAL_BF16_TFLOPS = 2250.0
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# fused launches per layer: (name, constituent matrices, N, K, activation)
+FUSED = (("qkv", ("q", "k", "v"), 3072, 2048, "x_attn"), ("o", ("o",), 2048, 2048, "x_o"),
+         ("gate_up", ("gate", "up"), 16384, 2048, "x_ffn"), ("down", ("down",), 2048, 8192, "x_down"))
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {k: float(d[k]) for k in FALLBACK_PEAKS if k in d} | {"source": "measured"}
+    return dict(FALLBACK_PEAKS, source="fallback")
+
+
+# --------------------------------------------------------------------------
+# clocks
+# --------------------------------------------------------------------------
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            f = tempfile.NamedTemporaryFile("w", suffix=".csv", delete=False)
+            self.path = f.name
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, reasons, smax = [], set(), None
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1]))
+                    smax = float(f[2])
+                except ValueError:
+                    continue
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=smax, reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# --------------------------------------------------------------------------
+# workload construction
+# --------------------------------------------------------------------------
+
+def build_stack_host(layers: int, fmts, threads: int = 8):
+    """Canonical blocks of the decode stack: {fmt: [ {name: blocks} per layer ]} and activations per layer."""
+    def one(layer):
+        out = {f: {} for f in fmts}
+        for name, N, K, act, w in synth.cfg1_layer_weights(layer):
+            for f in fmts:
+                out[f][name] = synth.quantize(f, w)
+        return out, synth.cfg1_layer_acts(layer)
+    with ThreadPoolExecutor(max_workers=threads) as ex:
+        res = list(ex.map(one, range(layers)))
+    return {f: [r[0][f] for r in res] for f in fmts}, [r[1] for r in res]
+
+
+def stack_bytes(fmt):
+    return sum(synth.canonical_bytes(fmt, N, K) for _, N, K, _ in synth.CFG1_LAYER) * synth.CFG1["layers"]
+
+
+# --------------------------------------------------------------------------
+# multi-rank plumbing (weak scaling: every rank decodes its own tokens)
+# --------------------------------------------------------------------------
+
+def rank_activations(rank: int, host_acts):
+    """Rank 0 keeps the workload's activations; every other rank draws its own (same shapes,
+    its own seed) -- each rank stands for an independent decode request on the same weights."""
+    if rank == 0:
+        return host_acts
+    return [{k: synth.activations(synth.CFG1["seed"] + 1000 * rank, 17 * l + i, v.size)
+             for i, (k, v) in enumerate(a.items())} for l, a in enumerate(host_acts)]
+
+
+def max_over_ranks(dist, values, device):
+    """Element-wise maximum over all ranks (the job is as slow as its slowest rank)."""
+    import torch
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def whole_job_value(world: int, bytes_per_rank_step: int, ms_per_step: float) -> float:
+    """GB/s over all ranks: every rank moves bytes_per_rank_step per step."""
+    return world * bytes_per_rank_step / (ms_per_step * 1e-3) / 1e9
+
+
+# --------------------------------------------------------------------------
+# our arm
+# --------------------------------------------------------------------------
+
+def run_ours(args):
+    import torch
+    from paper_2607_00501_b200 import qmm
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group("nccl", device_id=torch.device("cuda", local))
+        dist = dist_mod
+    qmm.lib()
+    pk = peaks()
+    layers = synth.CFG1["layers"]
+    fmts = synth.CFG1["fmts"]
+
+    t_gen = time.time()
+    host_blocks, host_acts = build_stack_host(layers, fmts)
+    host_acts = rank_activations(rank, host_acts)
+    gen_s = time.time() - t_gen
+
+    # ---- device residency: packed weights (fused per launch), activations, outputs
+    def dev_u8(a):
+        return torch.from_numpy(a).cuda()
+
+    ops = {f: [] for f in fmts}                          # (N, K, packed, x, y, ws)
+    rows_of = {n: NN for n, NN, _, _ in synth.CFG1_LAYER}
+    x_dev = [{k: torch.from_numpy(v).cuda() for k, v in a.items()} for a in host_acts]
+    for f in fmts:
+        for l in range(layers):
+            for name, parts, N, K, act in FUSED:
+                packed = torch.cat([qmm.pack(f, dev_u8(host_blocks[f][l][p]), rows_of[p], K) for p in parts])
+                y = torch.empty(N, dtype=torch.float16, device="cuda")
+                need = qmm.gemv_workspace_bytes(f, N, K)
+                ws = torch.empty(max(need, 16), dtype=torch.uint8, device="cuda")
+                ops[f].append((N, K, packed, x_dev[l][act], y, ws))
+    torch.cuda.synchronize()
+    bytes_step = sum(stack_bytes(f) for f in fmts)
+    launches_per_step = sum(len(v) for v in ops.values())
+
+    nstreams = args.streams
+    main = torch.cuda.Stream()
+    side = [torch.cuda.Stream() for _ in range(nstreams)]
+
+    def issue_all():
+        """Every GEMV of both stacks.  The products are independent (each has its own seeded
+        activation vector), so they are spread over `nstreams` streams; within a stream,
+        consecutive launches are chained with programmatic dependent launch."""
+        flat = [(f,) + op for f in fmts for op in ops[f]]
+        if nstreams <= 1:
+            for f, N, K, w, x, y, ws in flat:
+                qmm.gemv(f, w, N, K, x, y=y, ws=ws)
+            return
+        ev = torch.cuda.Event()
+        ev.record(torch.cuda.current_stream())
+        for i, (f, N, K, w, x, y, ws) in enumerate(flat):
+            st = side[i % nstreams]
+            if i < nstreams:
+                st.wait_event(ev)
+            with torch.cuda.stream(st):
+                qmm.gemv(f, w, N, K, x, y=y, ws=ws)
+        for st in side:
+            e = torch.cuda.Event()
+            e.record(st)
+            torch.cuda.current_stream().wait_event(e)
+
+    with torch.cuda.stream(main):
+        issue_all()
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=main):
+            issue_all()
+
+        def barrier():
+            torch.cuda.synchronize()
+            if dist is not None:
+                dist.barrier()
+            torch.cuda.synchronize()
+
+        for _ in range(max(args.warmup, 3)):
+            graph.replay()
+        barrier()
+        sampler = ClockSampler(local)
+        if rank == 0:
+            sampler.start()
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+        evs[0].record()
+        for i in range(args.steps):
+            graph.replay()
+            evs[i + 1].record()
+        barrier()
+        step_ms = [evs[i].elapsed_time(evs[i + 1]) for i in range(args.steps)]
+        total_ms = evs[0].elapsed_time(evs[-1])
+        # keep the GPU busy a little longer so that the clock sampler sees load even for short runs
+        t_end = time.time() + 1.0
+        while time.time() < t_end:
+            graph.replay()
+        torch.cuda.synchronize()
+        clocks = sampler.stop() if rank == 0 else None
+
+        # ---- end to end through the C ABI with host buffers: H2D activations, D2H outputs, per step
+        pin_x = [{k: torch.from_numpy(v).pin_memory() for k, v in a.items()} for a in host_acts]
+        ys = [op[4] for f in fmts for op in ops[f]]
+        pin_y = [torch.empty(y.shape, dtype=y.dtype).pin_memory() for y in ys]
+        h2d = sum(v.numel() * 2 for a in pin_x for v in a.values())
+        d2h = sum(y.numel() * 2 for y in ys)
+
+        def e2e_step():
+            for l in range(layers):
+                for k in pin_x[l]:
+                    x_dev[l][k].copy_(pin_x[l][k], non_blocking=True)
+            graph.replay()
+            for src, dst in zip(ys, pin_y):
+                dst.copy_(src, non_blocking=True)
+
+        for _ in range(3):
+            e2e_step()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            e2e_step()
+        e1.record()
+        barrier()
+        e2e_ms = e0.elapsed_time(e1)
+
+    total_ms, e2e_ms = max_over_ranks(dist, [total_ms, e2e_ms], "cuda")
+    ms_per_step = total_ms / args.steps
+    value = whole_job_value(world, bytes_step, ms_per_step)
+    e2e_value = whole_job_value(world, bytes_step, e2e_ms / args.steps)
+
+    sections = {}
+    cpu = None
+    if rank == 0 and not args.no_sections:
+        sections = extra_sections(args, qmm, torch, pk, ops, fmts)
+    if rank == 0 and world == 1 and not args.no_cpu:
+        cpu = cpu_baseline(host_blocks, host_acts, fmts, budget_s=args.cpu_seconds)
+
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank != 0:
+        return
+    line = {
+        "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": round(ms_per_step, 5), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f16 x int4/int8 -> f32 accumulate", "data": "synthetic",
+        "config": {"workload": "cfg1: Q4+Q8 decode linear stack, 16 layers, M=1 (q,k,v fused; gate,up fused)",
+                   "launches_per_step": launches_per_step, "streams": nstreams,
+                   "bytes_per_step": bytes_step, "l2": "inputs larger than L2 (1.58 GB of weights per step)",
+                   "input_generation_s": round(gen_s, 1)},
+        "e2e": {"value": round(e2e_value, 1), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": launches_per_step * args.steps,
+        "clocks": clocks,
+        "roofline": {"bound": "hbm", "achieved": round(value / world, 1), "peak": pk["hbm_gbs"], "unit": "GB/s",
+                     "frac": round(value / world / pk["hbm_gbs"], 4), "traffic": None,
+                     "kernel": "gemv_kernel (all launches of the step)", "peak_source": pk["source"],
+                     "step_ms_min": round(min(step_ms), 5), "step_ms_max": round(max(step_ms), 5)},
+        "cpu_baseline": cpu,
+        "sections": sections,
+    }
+    print(json.dumps(line))
+
+
+def time_op(torch, fn, iters, flush=None):
+    """Median and best device time (ms) of fn() over iters runs, L2 flushed before each run."""
+    times = []
+    for _ in range(iters):
+        if flush is not None:
+            flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    return float(np.median(times)), float(min(times))
+
+
+def extra_sections(args, qmm, torch, pk, ops, fmts):
+    """The rest of the path on its own workloads (each L2-flushed between runs)."""
+    out = {}
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+    # per-format decode stacks, chained on one stream (dependent-decode mode)
+    for f in fmts:
+        g = torch.cuda.CUDAGraph()
+        s = torch.cuda.Stream()
+        with torch.cuda.stream(s):
+            for N, K, w, x, y, ws in ops[f][:4]:
+                qmm.gemv(f, w, N, K, x, y=y, ws=ws)
+            torch.cuda.synchronize()
+            with torch.cuda.graph(g, stream=s):
+                for N, K, w, x, y, ws in ops[f]:
+                    qmm.gemv(f, w, N, K, x, y=y, ws=ws)
+            med, best = time_op(torch, g.replay, 10)
+        b = stack_bytes(f)
+        out["decode_stack_q%d_chained" % f] = {"ms": round(med, 4), "GBps": round(b / med / 1e6, 1),
+                                                "frac_hbm": round(b / med / 1e6 / pk["hbm_gbs"], 4),
+                                                "launches": len(ops[f])}
+
+    # cfg2: Q8 LM head GEMV
+    c = synth.CFG2
+    blocks = synth.quantize(c["fmt"], synth.weights(c["seed"], 0, c["N"], c["K"]))
+    packed = qmm.pack(c["fmt"], dev(blocks), c["N"], c["K"])
+    x = dev(synth.activations(c["seed"], 1, c["K"]))
+    y = torch.empty(c["N"], dtype=torch.float16, device="cuda")
+    med, best = time_op(torch, lambda: qmm.gemv(c["fmt"], packed, c["N"], c["K"], x, y=y), 20, flush)
+    out["lm_head_q8_gemv"] = {"ms": round(med, 4), "GBps": round(blocks.nbytes / med / 1e6, 1),
+                              "frac_hbm": round(blocks.nbytes / med / 1e6 / pk["hbm_gbs"], 4)}
+    del packed, blocks
+
+    # cfg3: Q4 prefill GEMM sweep
+    c = synth.CFG3
+    gemm = {}
+    for name, N, K in c["shapes"]:
+        blocks = synth.quantize(c["fmt"], synth.weights(c["seed"], 0 if name == "gate_up" else 1, N, K))
+        packed = qmm.pack(c["fmt"], dev(blocks), N, K)
+        for M in c["Ms"]:
+            X = dev(synth.activations(c["seed"], 10 + M, M, K))
+            Y = torch.empty((M, N), dtype=torch.float16, device="cuda")
+            ws = torch.zeros(256, dtype=torch.uint8, device="cuda")
+            fn = lambda: qmm.gemm(c["fmt"], packed, N, K, X, Y=Y, ws=ws)
+            fn()
+            med, best = time_op(torch, fn, 10, flush)
+            tf = 2.0 * M * N * K / med / 1e9
+            gemm["%s_M%d" % (name, M)] = {"ms": round(med, 4), "TFLOPs": round(tf, 1),
+                                          "frac_tensor_measured": round(tf / pk["bf16_tflops"], 4),
+                                          "frac_tensor_nominal": round(tf / NOMINAL_BF16_TFLOPS, 4)}
+            qmm.status_check(ws)
+    out["prefill_gemm_q4"] = gemm
+
+    # cfg4: Q4 MoE layer
+    c = synth.CFG4
+    gate, up, down = synth.moe_expert_weights(c["seed"], c["fmt"], c["E"], c["H"], c["I"])
+    pg = qmm.pack(c["fmt"], dev(gate), c["E"] * c["I"], c["H"])
+    pu = qmm.pack(c["fmt"], dev(up), c["E"] * c["I"], c["H"])
+    pd = qmm.pack(c["fmt"], dev(down), c["E"] * c["H"], c["I"])
+    wbytes = gate.nbytes + up.nbytes + down.nbytes
+    moe = {}
+    for T in c["Ts"]:
+        X = dev(synth.activations(c["seed"], 100 + T, T, c["H"]))
+        lg = dev(synth.logits(c["seed"], 200 + T, T, c["E"]))
+        o = torch.empty((T, c["H"]), dtype=torch.float16, device="cuda")
+        a = qmm.moe_args(c["fmt"], T, c["H"], c["I"], c["E"], c["topk"], lg, X, pg, pu, pd, o)
+        ws = torch.zeros(qmm.moe_workspace_bytes(a), dtype=torch.uint8, device="cuda")
+        fn = lambda: qmm.moe(a, ws)
+        fn()
+        med, best = time_op(torch, fn, 10, flush)
+        qmm.status_check(ws)
+        fl = T * c["topk"] * 3 * 2.0 * c["H"] * c["I"]
+        touched = min(c["E"], T * c["topk"]) / c["E"] * wbytes if T * c["topk"] < c["E"] else wbytes
+        moe["T%d" % T] = {"ms": round(med, 4), "TFLOPs": round(fl / med / 1e9, 2),
+                          "frac_tensor_nominal": round(fl / med / 1e9 / NOMINAL_BF16_TFLOPS, 4),
+                          "hbm_floor_ms": round(touched / pk["hbm_gbs"] / 1e6, 4),
+                          "frac_of_hbm_floor": round(touched / pk["hbm_gbs"] / 1e6 / med, 4)}
+    out["moe_q4"] = moe
+    return out
+
+
+# --------------------------------------------------------------------------
+# CPU oracle legs
+# --------------------------------------------------------------------------
+
+def cpu_baseline(host_blocks, host_acts, fmts, budget_s=12.0):
+    """The oracle, as it stands, on the host cores: whole passes over the decode stack for ~budget_s."""
+    import oracle
+    shapes = {n: (N, K, a) for n, N, K, a in synth.CFG1_LAYER}
+    t0 = time.time()
+    done_bytes, done_layers = 0, 0
+    while time.time() - t0 < budget_s:
+        for l in range(len(host_acts)):
+            for f in fmts:
+                for name, (N, K, act) in shapes.items():
+                    oracle.gemv(f, host_blocks[f][l][name], N, K, host_acts[l][act])
+                    done_bytes += host_blocks[f][l][name].nbytes
+            done_layers += 1
+            if time.time() - t0 > budget_s:
+                break
+    dt = time.time() - t0
+    return {"value": round(done_bytes / dt / 1e9, 3), "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": "%d layer passes (%.2f passes over the 16-layer Q4+Q8 decode stack, every GEMV), %.1f s" %
+                      (done_layers, done_layers / len(host_acts), dt)}
+
+
+def run_reference(args):
+    """`--impl reference`: the CPU oracle on a bounded sample of the same workload per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    fmts = synth.CFG1["fmts"]
+    sample_layers = 1
+    host_blocks, host_acts = build_stack_host(sample_layers, fmts)
+    shapes = {n: (N, K, a) for n, N, K, a in synth.CFG1_LAYER}
+    nbytes = sum(host_blocks[f][0][n].nbytes for f in fmts for n in shapes)
+
+    def step():
+        for f in fmts:
+            for name, (N, K, act) in shapes.items():
+                oracle.gemv(f, host_blocks[f][0][name], N, K, host_acts[0][act])
+
+    for _ in range(max(args.warmup, 1)):
+        step()
+    t0 = time.time()
+    for _ in range(args.steps):
+        step()
+    dt = time.time() - t0
+    value = nbytes * args.steps / dt / 1e9
+    sample = "layer 0 of 16 of the Q4+Q8 decode stack per step (all 14 GEMVs), host cores"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": round(value, 3), "unit": UNIT,
+        "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": max(args.warmup, 1),
+        "ms_per_step": round(dt / args.steps * 1e3, 3), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64 accumulate (CPU oracle)", "data": "synthetic",
+        "config": {"workload": "cfg1: Q4+Q8 decode linear stack, 16 layers, M=1", "sample": sample},
+        "cpu_baseline": {"value": round(value, 3), "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": round(value, 3), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--streams", type=int, default=8, help="streams the independent GEMVs are spread over")
+    ap.add_argument("--no-sections", action="store_true", help="skip the LM-head / GEMM / MoE sections")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline")
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

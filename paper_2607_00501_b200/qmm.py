@@ -179,8 +179,11 @@ def gemm(fmt: int, packed: torch.Tensor, N: int, K: int, X: torch.Tensor,
 
 def moe_args(fmt, T, H, I, E, topk, logits, X, w_gate, w_up, w_down, out,
              topk_idx=None, topk_w=None, perm=None, expert_offsets=None, dbg_H=None, dbg_D=None) -> MoeArgs:
-    return MoeArgs(T, H, I, E, topk, fmt, _dp(logits), _dp(X), _dp(w_gate), _dp(w_up), _dp(w_down), _dp(out),
-                   _dp(topk_idx), _dp(topk_w), _dp(perm), _dp(expert_offsets), _dp(dbg_H), _dp(dbg_D))
+    a = MoeArgs(T, H, I, E, topk, fmt, _dp(logits), _dp(X), _dp(w_gate), _dp(w_up), _dp(w_down), _dp(out),
+                _dp(topk_idx), _dp(topk_w), _dp(perm), _dp(expert_offsets), _dp(dbg_H), _dp(dbg_D))
+    # the struct holds raw device pointers only: keep the tensors alive as long as the struct
+    a._keep = (logits, X, w_gate, w_up, w_down, out, topk_idx, topk_w, perm, expert_offsets, dbg_H, dbg_D)
+    return a
 
 
 def moe_workspace_bytes(args: MoeArgs) -> int:

@@ -1,0 +1,50 @@
+"""The N > 1 path of the benchmark on CPU: two gloo ranks (no GPU needed).
+
+Covers what differs between ranks: each rank draws its own activations, the
+step time is the maximum over ranks, the reported value is the whole-job sum,
+and the reference arm runs on rank 0 only."""
+import json
+import os
+import subprocess
+import sys
+
+import numpy as np
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+sys.path.insert(0, ROOT)
+
+
+def _worker(rank, world, port, out_dir):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    import bench
+    from paper_2607_00501_b200 import synth
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    base = [synth.cfg1_layer_acts(0)]
+    mine = bench.rank_activations(rank, base)
+    # rank r pretends its step took (1 + r) ms
+    total_ms, = bench.max_over_ranks(dist, [1.0 + rank], "cpu")
+    value = bench.whole_job_value(world, 1000, total_ms)
+    dist.barrier()
+    np.save(os.path.join(out_dir, "acts%d.npy" % rank), mine[0]["x_attn"])
+    json.dump({"total_ms": total_ms, "value": value}, open(os.path.join(out_dir, "r%d.json" % rank), "w"))
+    dist.destroy_process_group()
+
+
+def test_two_gloo_ranks(tmp_path):
+    world, port = 2, 29000 + os.getpid() % 2000
+    mp.spawn(_worker, args=(world, port, str(tmp_path)), nprocs=world, join=True)
+    r = [json.load(open(tmp_path / ("r%d.json" % i))) for i in range(world)]
+    assert r[0]["total_ms"] == r[1]["total_ms"] == 2.0           # the slowest rank sets the time
+    assert r[0]["value"] == 2 * 1000 / 2e-3 / 1e9                # whole-job bytes over that time
+    a0, a1 = np.load(tmp_path / "acts0.npy"), np.load(tmp_path / "acts1.npy")
+    assert a0.shape == a1.shape and not np.array_equal(a0, a1)   # every rank decodes its own token
+
+
+def test_reference_arm_runs_on_rank0_only():
+    env = dict(os.environ, RANK="1", WORLD_SIZE="2")
+    p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "1", "--warmup", "1"],
+                       env=env, capture_output=True, text=True, timeout=300)
+    assert p.returncode == 0 and p.stdout.strip() == ""
