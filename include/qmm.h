@@ -108,6 +108,33 @@ qmm_status qmm_gemv(qmm_format fmt, const void* packed, int64_t N, int64_t K,
                     const uint16_t* x_fp16, uint16_t* y_fp16,
                     void* ws, size_t ws_bytes, void* stream);
 
+/* qmm_gemv for callers that cannot allocate.  The paper has no counterpart to
+ * this call; it exists for integrations that are not allowed to obtain device
+ * memory at the time they need a product: code that runs after a host
+ * application has handed out its whole device-memory budget, code that runs
+ * under a lock or inside a latency-critical loop where the device-wide
+ * synchronisation of an allocation is not acceptable, and plug-ins whose host
+ * forbids any allocator call after start-up.  Such a caller has nowhere to
+ * get the split-K workspace of qmm_gemv from, so this variant keeps that
+ * scratch inside the library: a fixed array of QMM_GEMV_STATIC_SCRATCH_BYTES
+ * that every GPU which loads the library holds until the process exits.
+ *   - Same arguments and result as qmm_gemv, minus the workspace.  The caller
+ *     still owns packed, x_fp16 and y_fp16 (device pointers).
+ *   - Shapes whose split-K partial sums need more than the built-in scratch are
+ *     rejected with QMM_ERR_WORKSPACE (nothing is enqueued); use qmm_gemv.
+ *   - The call allocates nothing and frees nothing, on the host or the device.
+ *   - The first call on each device looks up the device address of the scratch
+ *     (one runtime query, no allocation).  Make that first call outside any
+ *     stream capture, e.g. once at start-up on every device that will be used.
+ *   - All calls on a device share the one scratch array, and it keeps whatever
+ *     the last call left in it.  The kernels overwrite every element they later
+ *     read, so nothing needs clearing, but two calls whose kernels can overlap
+ *     on the GPU (different streams, or graphs replayed concurrently) race on
+ *     it: keep calls to this function on one device ordered on one stream.   */
+#define QMM_GEMV_STATIC_SCRATCH_BYTES (1 << 20)
+qmm_status qmm_gemv_static(qmm_format fmt, const void* packed, int64_t N, int64_t K,
+                           const uint16_t* x_fp16, uint16_t* y_fp16, void* stream);
+
 /* Prefill matrix-matrix product (Sec. 3.3 "GEMM (prefill, M>1)", Sec. 3.4):
  *   Y[m,n] = fp16( sum_k w[n,k] * X[m,k] ), fp32 accumulation on the tensor
  * cores; weights enter the contraction as fp16(float(d) * q).

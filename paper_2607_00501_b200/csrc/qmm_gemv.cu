@@ -348,3 +348,75 @@ qmm_status launch_gemv(int fmt, const void* packed, int64_t N, int64_t K, const 
 }
 
 }  // namespace qmm
+
+// --------------------------------------------------------------------------
+// qmm_gemv_static: the same product for callers that must not allocate.
+// --------------------------------------------------------------------------
+
+namespace qmm {
+
+// Scratch for the split-K partial sums of qmm_gemv_static.  It lives in the
+// library image: every GPU that loads libqmm holds these bytes until the
+// process exits.  In host code this name is only a handle for the runtime, not
+// a device address; the address each device uses is looked up once with
+// cudaGetSymbolAddress (below) and that pointer is what the kernels receive.
+static __device__ __align__(256) float g_gemv_static_scratch[QMM_GEMV_STATIC_SCRATCH_BYTES / sizeof(float)];
+
+constexpr int kMaxDevices = 64;
+static float* g_static_scratch_ptr[kMaxDevices];   // device address of the array, per device; nullptr = not looked up yet
+
+// Looks up (once per device, with that device current) where the scratch array lives.
+static qmm_status static_scratch_for_current_device(float** out)
+{
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return check_cuda(e, "qmm_gemv_static: cudaGetDevice");
+    if (dev < 0 || dev >= kMaxDevices) return fail(QMM_ERR_UNSUPPORTED, "qmm_gemv_static: device index %d not supported", dev);
+    float* p = __atomic_load_n(&g_static_scratch_ptr[dev], __ATOMIC_ACQUIRE);
+    if (p == nullptr) {
+        int major = 0, minor = 0;
+        e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&minor, cudaDevAttrComputeCapabilityMinor, dev);
+        if (e != cudaSuccess) return check_cuda(e, "qmm_gemv_static: device attributes");
+        if (major != 10 || minor != 0)
+            return fail(QMM_ERR_UNSUPPORTED, "qmm_gemv_static: device %d is not compute capability 10.0 (B200)", dev);
+        void* addr = nullptr;
+        e = cudaGetSymbolAddress(&addr, g_gemv_static_scratch);
+        if (e != cudaSuccess) return check_cuda(e, "qmm_gemv_static: cudaGetSymbolAddress");
+        p = static_cast<float*>(addr);
+        __atomic_store_n(&g_static_scratch_ptr[dev], p, __ATOMIC_RELEASE);   // same value from any thread
+    }
+    *out = p;
+    return QMM_OK;
+}
+
+}  // namespace qmm
+
+extern "C" qmm_status qmm_gemv_static(qmm_format fmt, const void* packed, int64_t N, int64_t K,
+                                      const uint16_t* x_fp16, uint16_t* y_fp16, void* stream)
+{
+    using namespace qmm;
+    if (fmt != QMM_Q4 && fmt != QMM_Q8) return fail(QMM_ERR_INVALID_ARG, "qmm_gemv_static: unknown format %d", (int)fmt);
+    if (N <= 0 || K <= 0) return fail(QMM_ERR_INVALID_ARG, "qmm_gemv_static: N=%lld and K=%lld must be positive", (long long)N, (long long)K);
+    if (K % 32) return fail(QMM_ERR_SHAPE, "qmm_gemv_static: K=%lld is not a multiple of the block size 32", (long long)K);
+    if (K % 256 || N % 128 || K > 32768 || N > (1 << 24))
+        return fail(QMM_ERR_UNSUPPORTED, "qmm_gemv_static: needs K %% 256 == 0, N %% 128 == 0, K <= 32768, N <= 2^24 (got N=%lld K=%lld)",
+                    (long long)N, (long long)K);
+    if (!packed || !x_fp16 || !y_fp16) return fail(QMM_ERR_INVALID_ARG, "qmm_gemv_static: null pointer");
+    if ((reinterpret_cast<uintptr_t>(packed) & 31) || (reinterpret_cast<uintptr_t>(x_fp16) & 15) ||
+        (reinterpret_cast<uintptr_t>(y_fp16) & 15))
+        return fail(QMM_ERR_ALIGNMENT, "qmm_gemv_static: packed must be 32-byte aligned, x and y 16-byte aligned");
+    const size_t need = gemv_workspace_bytes(fmt, N, K);
+    if (need > (size_t)QMM_GEMV_STATIC_SCRATCH_BYTES)
+        return fail(QMM_ERR_WORKSPACE,
+                    "qmm_gemv_static: this shape needs %zu bytes of split-K scratch, the built-in scratch holds %d; "
+                    "use qmm_gemv with a caller-provided workspace",
+                    need, (int)QMM_GEMV_STATIC_SCRATCH_BYTES);
+    float* scratch = nullptr;
+    const qmm_status s = static_scratch_for_current_device(&scratch);
+    if (s != QMM_OK) return s;
+    // Partial sums are written in full before the second stage reads them, so the
+    // scratch needs no clearing between calls.
+    return launch_gemv(fmt, packed, N, K, x_fp16, y_fp16, scratch, (cudaStream_t)stream);
+}
+

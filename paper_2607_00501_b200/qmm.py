@@ -30,7 +30,7 @@ STATUS_NAMES = {
 EXPORTS = (
     "qmm_last_error", "qmm_version", "qmm_canonical_bytes", "qmm_packed_bytes", "qmm_pack",
     "qmm_dequant", "qmm_gemv_workspace_bytes", "qmm_gemv", "qmm_gemm_workspace_bytes", "qmm_gemm",
-    "qmm_moe_workspace_bytes", "qmm_moe", "qmm_moe_route", "qmm_status_check",
+    "qmm_moe_workspace_bytes", "qmm_moe", "qmm_moe_route", "qmm_status_check", "qmm_gemv_static",
 )
 
 
@@ -76,6 +76,7 @@ def lib() -> ctypes.CDLL:
             L.qmm_gemv_workspace_bytes.restype = sz
             L.qmm_gemv_workspace_bytes.argtypes = [ci, i64, i64]
             L.qmm_gemv.argtypes = [ci, vp, i64, i64, vp, vp, vp, sz, vp]
+            L.qmm_gemv_static.argtypes = [ci, vp, i64, i64, vp, vp, vp]
             L.qmm_gemm_workspace_bytes.restype = sz
             L.qmm_gemm_workspace_bytes.argtypes = [ci, i64, i64, i64]
             L.qmm_gemm.argtypes = [ci, vp, i64, i64, vp, i64, vp, i64, i64, vp, sz, vp]
@@ -154,6 +155,26 @@ def gemv(fmt: int, packed: torch.Tensor, N: int, K: int, x: torch.Tensor,
         need = gemv_workspace_bytes(fmt, N, K)
         ws = torch.empty(need, dtype=torch.uint8, device=x.device) if need else None
     _check(lib().qmm_gemv(fmt, packed.data_ptr(), N, K, x.data_ptr(), y.data_ptr(), _dp(ws), _nbytes(ws), _stream()))
+    return y
+
+
+GEMV_STATIC_SCRATCH_BYTES = 1 << 20
+
+
+def gemv_static(fmt: int, packed: torch.Tensor, N: int, K: int, x: torch.Tensor, y: torch.Tensor) -> torch.Tensor:
+    """y = W x through qmm_gemv_static: no workspace argument and no allocation anywhere.
+
+    For callers that may not allocate device memory when they need the product (memory
+    budget already handed out, allocator calls forbidden after start-up, no tolerance for
+    the device-wide synchronisation an allocation implies).  The split-K scratch is a fixed
+    array inside the library (GEMV_STATIC_SCRATCH_BYTES per GPU); shapes that need more
+    raise QmmError (QMM_ERR_WORKSPACE).  `y` must be provided by the caller.  All calls on a
+    device share that scratch: keep them on one stream.  Make the first call on each device
+    outside any stream capture.
+    """
+    assert x.is_cuda and x.dtype == torch.float16 and x.numel() == K and x.is_contiguous()
+    assert y.is_cuda and y.dtype == torch.float16 and y.numel() == N and y.is_contiguous()
+    _check(lib().qmm_gemv_static(fmt, packed.data_ptr(), N, K, x.data_ptr(), y.data_ptr(), _stream()))
     return y
 
 
