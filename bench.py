@@ -195,9 +195,20 @@ def run_ours(args):
                 need = qmm.gemv_workspace_bytes(f, N, K)
                 ws = torch.empty(max(need, 16), dtype=torch.uint8, device="cuda")
                 ops[f].append((N, K, packed, x_dev[l][act], y, ws))
+    # the same stack as one batched launch per format: every matrix its own problem (no fusion needed)
+    batch = {}
+    ys_batch = []
+    for f in fmts:
+        probs = []
+        for l in range(layers):
+            for name, N, K, act in synth.CFG1_LAYER:
+                y = torch.empty(N, dtype=torch.float16, device="cuda")
+                probs.append((qmm.pack(f, dev_u8(host_blocks[f][l][name]), N, K), N, K, x_dev[l][act], y))
+                ys_batch.append(y)
+        batch[f] = qmm.gemv_batch_problems(probs)
     torch.cuda.synchronize()
     bytes_step = sum(stack_bytes(f) for f in fmts)
-    launches_per_step = sum(len(v) for v in ops.values())
+    launches_per_step = len(fmts) if args.mode == "batch" else sum(len(v) for v in ops.values())
 
     nstreams = args.streams
     main = torch.cuda.Stream()
@@ -205,8 +216,13 @@ def run_ours(args):
 
     def issue_all():
         """Every GEMV of both stacks.  The products are independent (each has its own seeded
-        activation vector), so they are spread over `nstreams` streams; within a stream,
-        consecutive launches are chained with programmatic dependent launch."""
+        activation vector).  mode 'batch': one qmm_gemv_batch launch per format (112 problems each).
+        mode 'streams': one qmm_gemv launch per fused matrix, spread over `nstreams` streams; within
+        a stream consecutive launches are chained with programmatic dependent launch."""
+        if args.mode == "batch":
+            for f in fmts:
+                qmm.gemv_batch(f, batch[f])
+            return
         flat = [(f,) + op for f in fmts for op in ops[f]]
         if nstreams <= 1:
             for f, N, K, w, x, y, ws in flat:
@@ -261,7 +277,7 @@ def run_ours(args):
 
         # ---- end to end through the C ABI with host buffers: H2D activations, D2H outputs, per step
         pin_x = [{k: torch.from_numpy(v).pin_memory() for k, v in a.items()} for a in host_acts]
-        ys = [op[4] for f in fmts for op in ops[f]]
+        ys = ys_batch if args.mode == "batch" else [op[4] for f in fmts for op in ops[f]]
         pin_y = [torch.empty(y.shape, dtype=y.dtype).pin_memory() for y in ys]
         h2d = sum(v.numel() * 2 for a in pin_x for v in a.values())
         d2h = sum(y.numel() * 2 for y in ys)
@@ -306,8 +322,9 @@ def run_ours(args):
         "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": round(ms_per_step, 5), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f16 x int4/int8 -> f32 accumulate", "data": "synthetic",
-        "config": {"workload": "cfg1: Q4+Q8 decode linear stack, 16 layers, M=1 (q,k,v fused; gate,up fused)",
-                   "launches_per_step": launches_per_step, "streams": nstreams,
+        "config": {"workload": "cfg1: Q4+Q8 decode linear stack, 16 layers x 7 matrices, M=1",
+                   "mode": args.mode, "launches_per_step": launches_per_step,
+                   "streams": nstreams if args.mode == "streams" else 1,
                    "bytes_per_step": bytes_step, "l2": "inputs larger than L2 (1.58 GB of weights per step)",
                    "input_generation_s": round(gen_s, 1)},
         "e2e": {"value": round(e2e_value, 1), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
@@ -315,7 +332,7 @@ def run_ours(args):
         "clocks": clocks,
         "roofline": {"bound": "hbm", "achieved": round(value / world, 1), "peak": pk["hbm_gbs"], "unit": "GB/s",
                      "frac": round(value / world / pk["hbm_gbs"], 4), "traffic": None,
-                     "kernel": "gemv_kernel (all launches of the step)", "peak_source": pk["source"],
+                     "kernel": "gemv_batch_kernel (both launches of the step)" if args.mode == "batch" else "gemv_kernel (all launches of the step)", "peak_source": pk["source"],
                      "step_ms_min": round(min(step_ms), 5), "step_ms_max": round(max(step_ms), 5)},
         "cpu_baseline": cpu,
         "sections": sections,
@@ -344,7 +361,8 @@ def extra_sections(args, qmm, torch, pk, ops, fmts):
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
     dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
 
-    # per-format decode stacks, chained on one stream (dependent-decode mode)
+    # per-format decode stacks, one qmm_gemv launch per fused matrix, chained on one stream with
+    # programmatic dependent launch (a dependency between consecutive launches, as in a real decoder)
     for f in fmts:
         g = torch.cuda.CUDAGraph()
         s = torch.cuda.Stream()
@@ -487,7 +505,9 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--streams", type=int, default=8, help="streams the independent GEMVs are spread over")
+    ap.add_argument("--mode", default="batch", choices=["batch", "streams"],
+                    help="batch: one qmm_gemv_batch launch per format; streams: one qmm_gemv launch per matrix")
+    ap.add_argument("--streams", type=int, default=8, help="streams for --mode streams")
     ap.add_argument("--no-sections", action="store_true", help="skip the LM-head / GEMM / MoE sections")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)

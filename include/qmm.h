@@ -108,6 +108,23 @@ qmm_status qmm_gemv(qmm_format fmt, const void* packed, int64_t N, int64_t K,
                     const uint16_t* x_fp16, uint16_t* y_fp16,
                     void* ws, size_t ws_bytes, void* stream);
 
+/* Several independent decode products in one launch: y_i = W_i x_i for
+ * i < count, all in format fmt (Sec. 3.3: fusing what other runtimes dispatch
+ * as separate kernels matters most in decode, where each kernel is short).
+ * The products must be independent: every x_i is ready when the call's work
+ * starts, no y_i is another problem's input.  Shapes may differ.  Results are
+ * those of qmm_gemv up to the order of the fp32 additions.  No workspace.
+ *   problems  HOST array of `count` descriptors (read during the call only);
+ *             the pointers inside are device pointers with the alignment
+ *             rules of qmm_gemv; K <= 32768.                                */
+typedef struct {
+    const void* packed;        /* device, from qmm_pack                        */
+    const uint16_t* x_fp16;    /* device, K fp16 values                        */
+    uint16_t* y_fp16;          /* device, N fp16 values, written               */
+    int64_t N, K;
+} qmm_gemv_problem;
+qmm_status qmm_gemv_batch(qmm_format fmt, const qmm_gemv_problem* problems, int count, void* stream);
+
 /* qmm_gemv for callers that cannot allocate.  The paper has no counterpart to
  * this call; it exists for integrations that are not allowed to obtain device
  * memory at the time they need a product: code that runs after a host

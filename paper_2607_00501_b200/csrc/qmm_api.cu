@@ -36,6 +36,7 @@ qmm_status launch_dequant(int fmt, const void* packed, int64_t N, int64_t K, flo
 size_t gemv_workspace_bytes(int fmt, int64_t N, int64_t K);
 qmm_status launch_gemv(int fmt, const void* packed, int64_t N, int64_t K, const uint16_t* x, uint16_t* y,
                        void* ws, cudaStream_t st);
+qmm_status launch_gemv_batch(int fmt, const qmm_gemv_problem* probs, int count, cudaStream_t st);
 size_t gemm_workspace_bytes(int fmt, int64_t M, int64_t N, int64_t K);
 qmm_status launch_gemm(int fmt, const void* packed, int64_t N, int64_t K, const uint16_t* X, int64_t ldx,
                        uint16_t* Y, int64_t ldy, int64_t M, void* ws, cudaStream_t st);
@@ -149,6 +150,25 @@ qmm_status qmm_gemv(qmm_format fmt, const void* packed, int64_t N, int64_t K,
     }
     if ((s = check_device("qmm_gemv")) != QMM_OK) return s;
     return launch_gemv(fmt, packed, N, K, x_fp16, y_fp16, ws, (cudaStream_t)stream);
+}
+
+qmm_status qmm_gemv_batch(qmm_format fmt, const qmm_gemv_problem* problems, int count, void* stream)
+{
+    if (count < 0) return fail(QMM_ERR_INVALID_ARG, "qmm_gemv_batch: count=%d is negative", count);
+    if (count == 0) return QMM_OK;
+    if (!problems) return fail(QMM_ERR_INVALID_ARG, "qmm_gemv_batch: null problem list");
+    for (int i = 0; i < count; ++i) {
+        const qmm_gemv_problem& q = problems[i];
+        qmm_status s = check_matrix("qmm_gemv_batch", fmt, q.N, q.K);
+        if (s != QMM_OK) return s;
+        if (q.K > 32768) return fail(QMM_ERR_UNSUPPORTED, "qmm_gemv_batch: problem %d has K=%lld > 32768", i, (long long)q.K);
+        if (!q.packed || !q.x_fp16 || !q.y_fp16) return fail(QMM_ERR_INVALID_ARG, "qmm_gemv_batch: problem %d has a null pointer", i);
+        if (!aligned(q.packed, 32) || !aligned(q.x_fp16, 16) || !aligned(q.y_fp16, 16))
+            return fail(QMM_ERR_ALIGNMENT, "qmm_gemv_batch: problem %d: packed must be 32-byte, x and y 16-byte aligned", i);
+    }
+    qmm_status s = check_device("qmm_gemv_batch");
+    if (s != QMM_OK) return s;
+    return launch_gemv_batch(fmt, problems, count, (cudaStream_t)stream);
 }
 
 size_t qmm_gemm_workspace_bytes(qmm_format fmt, int64_t M, int64_t N, int64_t K)

@@ -236,6 +236,155 @@ gemv_kernel(const uint8_t* __restrict__ packed, const uint16_t* __restrict__ x,
     }
 }
 
+// ---------------------------------------------------------------- batch
+//
+// Many independent products in ONE launch (fused q/k/v, gate/up, all the
+// matrices of a layer whose inputs are ready...).  The paper's decode gains
+// come from issuing fewer, fused dispatches (Sec. 3.3); a launch per small
+// matrix cannot keep a B200's HBM busy -- a 2 MB matrix is 0.3 us of traffic,
+// a launch is several -- so the whole list is streamed by one persistent grid.
+//
+// Work unit = (problem, pair of row groups): 64 outputs, the block's warps
+// split its K range.  The list of units is cut into gridDim.x contiguous
+// ranges of equal *cost* (cost of a unit = its number of tiles), so blocks
+// finish together although problems differ in K.  No split-K, no workspace.
+
+constexpr int kMaxBatch = 128;
+
+struct BatchProblem {
+    const uint8_t* packed;
+    const uint16_t* x;
+    uint16_t* y;
+    int K;            // input features
+    int tpr;          // tiles per row
+    int pairs;        // N / 64
+    int cost_begin;   // tiles of all earlier problems
+};
+
+struct BatchParams {
+    int count;
+    int total_cost;
+    int max_k;
+    BatchProblem p[kMaxBatch];
+};
+
+template <int FMT, int WARPS>
+__global__ void __launch_bounds__(WARPS * 32, 768 / (WARPS * 32))
+gemv_batch_kernel(const __grid_constant__ BatchParams bp)
+{
+    extern __shared__ uint4 smem[];
+    uint4* xs = smem;
+    uint4* zs = smem + bp.max_k / 8;
+    float* red = reinterpret_cast<float*>(smem + bp.max_k / 4);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr int TB = Fmt<FMT>::tile_bytes;
+    constexpr int XV = Fmt<FMT>::tile_k / 8;
+    constexpr int STEP = kUnroll * WARPS;
+
+    // this block's range of the unit list, by cost
+    const int c0 = (int)(((long long)bp.total_cost * blockIdx.x) / gridDim.x);
+    const int c1 = (int)(((long long)bp.total_cost * (blockIdx.x + 1)) / gridDim.x);
+    int pi = 0;
+    while (pi < bp.count && bp.p[pi].cost_begin + bp.p[pi].pairs * bp.p[pi].tpr <= c0) ++pi;
+    int unit = 0;                                               // pair index within problem pi
+    if (pi < bp.count) {
+        const int rel = c0 - bp.p[pi].cost_begin;
+        unit = rel <= 0 ? 0 : (rel + bp.p[pi].tpr - 1) / bp.p[pi].tpr;
+        if (unit >= bp.p[pi].pairs) {
+            ++pi;
+            unit = 0;
+        }
+    }
+    // a unit belongs to the block whose range holds the unit's first tile
+    auto valid = [&](int p, int u) { return p < bp.count && bp.p[p].cost_begin + u * bp.p[p].tpr < c1; };
+
+    TileRegs<FMT> r;
+    int t = 0, t_end = 0;
+    const uint8_t* tiles_p = nullptr;
+    size_t group_bytes = 0;
+    auto open_unit = [&](int p, int u) {
+        group_bytes = (size_t)bp.p[p].tpr * TB;
+        tiles_p = bp.p[p].packed + 32 * lane + (size_t)(2 * u) * group_bytes;
+        t = warp;
+        t_end = bp.p[p].tpr;
+    };
+    auto load_group = [&]() {
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            const int tt = t + u * WARPS;
+            if (tt < t_end) {
+                const uint8_t* tp = tiles_p + (size_t)tt * TB;
+                const uint8_t* tq = tp + group_bytes;
+                r.cp[u] = ld_stream_256(tp);
+                r.cq[u] = ld_stream_256(tq);
+                r.sp[u] = load_scales<FMT>(tp - 32 * lane, lane);
+                r.sq[u] = load_scales<FMT>(tq - 32 * lane, lane);
+            }
+        }
+    };
+    bool have = valid(pi, unit);
+    if (have) {
+        open_unit(pi, unit);
+        load_group();
+    }
+
+    pdl_launch_dependents();
+    pdl_wait();                                                 // activations may come from the previous kernel
+    for (int i = threadIdx.x; i < bp.max_k / 8; i += WARPS * 32) zs[i] = make_uint4(0u, 0u, 0u, 0u);
+    if (have)
+        for (int i = threadIdx.x; i < bp.p[pi].K / 8; i += WARPS * 32) xs[i] = reinterpret_cast<const uint4*>(bp.p[pi].x)[i];
+    __syncthreads();
+    const uint4* xb = ((lane >> 2) == (lane & 3)) ? xs : zs;
+    Q4Consts kc;
+    kc.init();
+
+    while (have) {
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        while (t < t_end) {
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) {
+                const int tt = t + u * WARPS;
+                if (tt < t_end) {
+                    if constexpr (FMT == QMM_Q4)
+                        tile_pair_mma_q4(r.cp[u], r.cq[u], r.sp[u], r.sq[u], xb + tt * XV, acc, kc);
+                    else
+                        tile_pair_mma_q8(r.cp[u], r.cq[u], r.sp[u], r.sq[u], xb + tt * XV, acc);
+                }
+            }
+            t += STEP;
+            if (t < t_end) load_group();
+        }
+        const int done_p = pi, done_u = unit;
+        if (++unit >= bp.p[pi].pairs) {
+            ++pi;
+            unit = 0;
+        }
+        have = valid(pi, unit);
+        if (have) {                                             // next unit's loads fly during the reduction
+            open_unit(pi, unit);
+            load_group();
+        }
+        if ((lane & 3) < 2) {
+            const int row = (lane & ~3) + 2 * (lane & 1);
+            float* w = red + warp * 64;
+            w[row] = acc[0];
+            w[row + 1] = acc[1];
+            w[32 + row] = acc[2];
+            w[32 + row + 1] = acc[3];
+        }
+        __syncthreads();                                        // also: every warp is done with xs
+        if (threadIdx.x < 64) {
+            float sum = red[threadIdx.x];
+#pragma unroll
+            for (int w = 1; w < WARPS; ++w) sum += red[w * 64 + threadIdx.x];
+            bp.p[done_p].y[done_u * 64 + threadIdx.x] = __half_as_ushort(__float2half_rn(sum));
+        }
+        if (have && pi != done_p)                               // next unit reads another activation vector
+            for (int i = threadIdx.x; i < bp.p[pi].K / 8; i += WARPS * 32) xs[i] = reinterpret_cast<const uint4*>(bp.p[pi].x)[i];
+        __syncthreads();
+    }
+}
+
 // Second stage of split-K: y[n] = fp16(sum_s partial[s][n]), s ascending.
 __global__ void gemv_reduce_kernel(const float* __restrict__ partial, uint16_t* __restrict__ y, int N, int splits)
 {
@@ -328,6 +477,53 @@ static qmm_status launch_gemv_t(const GemvPlan& p, const void* packed, int64_t N
         e = launch_pdl(gemv_reduce_kernel, dim3((unsigned)((N + 255) / 256)), dim3(256), 0, st,
                        (const float*)partial, y, (int)N, p.splits);
         if (e != cudaSuccess) return check_cuda(e, "qmm_gemv reduce launch");
+    }
+    return QMM_OK;
+}
+
+// Host side of qmm_gemv_batch: up to kMaxBatch problems per launch.
+qmm_status launch_gemv_batch(int fmt, const qmm_gemv_problem* probs, int count, cudaStream_t st)
+{
+    for (int first = 0; first < count; first += kMaxBatch) {
+        const int n = count - first < kMaxBatch ? count - first : kMaxBatch;
+        BatchParams bp = {};
+        bp.count = n;
+        int cost = 0, max_k = 0;
+        for (int i = 0; i < n; ++i) {
+            const qmm_gemv_problem& q = probs[first + i];
+            BatchProblem& b = bp.p[i];
+            b.packed = (const uint8_t*)q.packed;
+            b.x = q.x_fp16;
+            b.y = q.y_fp16;
+            b.K = (int)q.K;
+            b.tpr = (int)(q.K / tile_k_of(fmt));
+            b.pairs = (int)(q.N / (2 * kRowsPerGroup));
+            b.cost_begin = cost;
+            if ((long long)cost + (long long)b.pairs * b.tpr > 0x7FFFFFFFLL)
+                return fail(QMM_ERR_UNSUPPORTED, "qmm_gemv_batch: batch too large for one launch");
+            cost += b.pairs * b.tpr;
+            if (b.K > max_k) max_k = b.K;
+        }
+        bp.total_cost = cost;
+        bp.max_k = max_k;
+        constexpr int WARPS = 8;
+        const size_t smem = (size_t)max_k * 4 + (size_t)WARPS * 64 * sizeof(float);
+        const int units = cost / (max_k / tile_k_of(fmt)) + 1;
+        int grid = kNumSMs * (768 / (WARPS * 32));
+        if (units < grid) grid = units;
+        cudaError_t e;
+        if (fmt == QMM_Q4) {
+            auto kern = gemv_batch_kernel<QMM_Q4, WARPS>;
+            if (smem > 48 * 1024 && (e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess)
+                return check_cuda(e, "qmm_gemv_batch shared memory size");
+            e = launch_pdl(kern, dim3(grid), dim3(WARPS * 32), smem, st, bp);
+        } else {
+            auto kern = gemv_batch_kernel<QMM_Q8, WARPS>;
+            if (smem > 48 * 1024 && (e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess)
+                return check_cuda(e, "qmm_gemv_batch shared memory size");
+            e = launch_pdl(kern, dim3(grid), dim3(WARPS * 32), smem, st, bp);
+        }
+        if (e != cudaSuccess) return check_cuda(e, "qmm_gemv_batch launch");
     }
     return QMM_OK;
 }

@@ -30,7 +30,7 @@ STATUS_NAMES = {
 EXPORTS = (
     "qmm_last_error", "qmm_version", "qmm_canonical_bytes", "qmm_packed_bytes", "qmm_pack",
     "qmm_dequant", "qmm_gemv_workspace_bytes", "qmm_gemv", "qmm_gemm_workspace_bytes", "qmm_gemm",
-    "qmm_moe_workspace_bytes", "qmm_moe", "qmm_moe_route", "qmm_status_check", "qmm_gemv_static",
+    "qmm_moe_workspace_bytes", "qmm_moe", "qmm_moe_route", "qmm_status_check", "qmm_gemv_static", "qmm_gemv_batch",
 )
 
 
@@ -39,6 +39,11 @@ class QmmError(RuntimeError):
         super().__init__("%s: %s" % (STATUS_NAMES.get(status, status), message))
         self.status = status
         self.message = message
+
+
+class GemvProblem(ctypes.Structure):
+    _fields_ = [("packed", ctypes.c_void_p), ("x_fp16", ctypes.c_void_p), ("y_fp16", ctypes.c_void_p),
+                ("N", ctypes.c_int64), ("K", ctypes.c_int64)]
 
 
 class MoeArgs(ctypes.Structure):
@@ -77,6 +82,7 @@ def lib() -> ctypes.CDLL:
             L.qmm_gemv_workspace_bytes.argtypes = [ci, i64, i64]
             L.qmm_gemv.argtypes = [ci, vp, i64, i64, vp, vp, vp, sz, vp]
             L.qmm_gemv_static.argtypes = [ci, vp, i64, i64, vp, vp, vp]
+            L.qmm_gemv_batch.argtypes = [ci, ctypes.POINTER(GemvProblem), ci, vp]
             L.qmm_gemm_workspace_bytes.restype = sz
             L.qmm_gemm_workspace_bytes.argtypes = [ci, i64, i64, i64]
             L.qmm_gemm.argtypes = [ci, vp, i64, i64, vp, i64, vp, i64, i64, vp, sz, vp]
@@ -156,6 +162,23 @@ def gemv(fmt: int, packed: torch.Tensor, N: int, K: int, x: torch.Tensor,
         ws = torch.empty(need, dtype=torch.uint8, device=x.device) if need else None
     _check(lib().qmm_gemv(fmt, packed.data_ptr(), N, K, x.data_ptr(), y.data_ptr(), _dp(ws), _nbytes(ws), _stream()))
     return y
+
+
+def gemv_batch_problems(problems):
+    """problems: iterable of (packed, N, K, x, y) tensors -> ctypes array for gemv_batch (keeps the tensors alive)."""
+    problems = list(problems)
+    arr = (GemvProblem * len(problems))()
+    for i, (packed, N, K, x, y) in enumerate(problems):
+        assert x.dtype == torch.float16 and x.numel() == K and y.dtype == torch.float16 and y.numel() == N
+        arr[i] = GemvProblem(packed.data_ptr(), x.data_ptr(), y.data_ptr(), N, K)
+    arr._keep = problems
+    return arr
+
+
+def gemv_batch(fmt: int, problems) -> None:
+    """All products y_i = W_i x_i of the list in one launch.  `problems` is the array made by
+    gemv_batch_problems (build it once and reuse it: the call only reads it)."""
+    _check(lib().qmm_gemv_batch(fmt, problems, len(problems), _stream()))
 
 
 GEMV_STATIC_SCRATCH_BYTES = 1 << 20

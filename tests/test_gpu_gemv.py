@@ -161,3 +161,56 @@ def test_cfg2_q8_lm_head_full_size(qmm, oracle):
     blocks = synth.quantize(c["fmt"], synth.weights(c["seed"], 0, c["N"], c["K"]))
     x = synth.activations(c["seed"], 1, c["K"])
     run_gemv(qmm, oracle, c["fmt"], blocks, c["N"], c["K"], x, "cfg2")
+
+
+@pytest.mark.parametrize("fmt", [Q4, Q8])
+def test_gemv_batch_mixed_shapes(qmm, oracle, fmt):
+    # one launch over problems that differ in N and K; each result held to the GEMV tolerance
+    shapes = [(128, 256), (384, 1024), (128, 8192), (640, 512), (256, 2048), (128, 256), (2176, 1280)]
+    probs, refs = [], []
+    for i, (N, K) in enumerate(shapes):
+        blocks = synth.quantize(fmt, synth.weights(95, 10 * fmt + i, N, K))
+        x = synth.activations(95, 100 + i, K)
+        y = torch.full((N,), 9.0, dtype=torch.float16, device="cuda")
+        probs.append((packed_from(qmm, fmt, blocks, N, K), N, K, util.dev(x), y))
+        refs.append(oracle.gemv(fmt, blocks, N, K, x))
+    arr = qmm.gemv_batch_problems(probs)
+    qmm.gemv_batch(fmt, arr)
+    torch.cuda.synchronize()
+    for (p, N, K, x, y), (y_ref, B) in zip(probs, refs):
+        util.assert_within_tol(util.host_f64(y), y_ref, B, "batch %dx%d" % (N, K))
+    first = [p[4].clone() for p in probs]
+    qmm.gemv_batch(fmt, arr)                                # deterministic
+    for f, p in zip(first, probs):
+        assert torch.equal(f, p[4])
+
+
+def test_gemv_batch_argument_checks(qmm):
+    buf = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
+    y = torch.zeros(128, dtype=torch.float16, device="cuda")
+    x = torch.zeros(256, dtype=torch.float16, device="cuda")
+    L = qmm.lib()
+    good = qmm.gemv_batch_problems([(buf, 128, 256, x, y)])
+    assert L.qmm_gemv_batch(4, good, 0, None) == 0
+    assert L.qmm_gemv_batch(4, good, -1, None) == 1
+    assert L.qmm_gemv_batch(4, None, 1, None) == 1
+    bad = (qmm.GemvProblem * 1)(qmm.GemvProblem(buf.data_ptr() + 8, x.data_ptr(), y.data_ptr(), 128, 256))
+    assert L.qmm_gemv_batch(4, bad, 1, None) == 3
+    bad = (qmm.GemvProblem * 1)(qmm.GemvProblem(buf.data_ptr(), x.data_ptr(), y.data_ptr(), 100, 256))
+    assert L.qmm_gemv_batch(4, bad, 1, None) == 5
+
+
+@pytest.mark.parametrize("fmt", [Q4, Q8])
+def test_cfg1_two_layers_full_size_in_one_batch(qmm, oracle, fmt):
+    probs, refs = [], []
+    for layer in (0, 15):
+        acts = synth.cfg1_layer_acts(layer)
+        for name, N, K, act, w in synth.cfg1_layer_weights(layer):
+            blocks = synth.quantize(fmt, w)
+            y = torch.empty(N, dtype=torch.float16, device="cuda")
+            probs.append((packed_from(qmm, fmt, blocks, N, K), N, K, util.dev(acts[act]), y))
+            refs.append((name, oracle.gemv(fmt, blocks, N, K, acts[act])))
+    qmm.gemv_batch(fmt, qmm.gemv_batch_problems(probs))
+    torch.cuda.synchronize()
+    for (p, N, K, x, y), (name, (y_ref, B)) in zip(probs, refs):
+        util.assert_within_tol(util.host_f64(y), y_ref, B, "cfg1 batch %s" % name)
