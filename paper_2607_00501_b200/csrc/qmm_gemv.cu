@@ -20,7 +20,10 @@
 
 namespace qmm {
 
-constexpr int kUnroll = 2;   // tile pairs in flight per warp (4 x 1 KiB of codes per warp)
+#ifndef QMM_GEMV_UNROLL
+#define QMM_GEMV_UNROLL 2
+#endif
+constexpr int kUnroll = QMM_GEMV_UNROLL;   // tile pairs in flight per warp (4 x 1 KiB of codes per warp)
 
 // D(16x8, fp32) += A(16x16, fp16, row) * B(16x8, fp16, col) on the warp-level tensor path.
 __device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
@@ -29,6 +32,15 @@ __device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1
     asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// Same, starting a new accumulation (C = 0) without spending instructions on zeroing registers.
+__device__ __forceinline__ void mma16816_zero(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                              uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+                 : "=f"(c[0]), "=f"(c[1]), "=f"(c[2]), "=f"(c[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.f));
 }
 
 // How a warp multiplies with one row per lane and no shuffles.
@@ -54,14 +66,17 @@ __device__ __forceinline__ void tile_pair_mma_q4(const u32x8& cp, const u32x8& c
 {
 #pragma unroll
     for (int b = 0; b < 2; ++b) {
-        float c[4] = {0.f, 0.f, 0.f, 0.f};
+        float c[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const uint4 xv = xt[b * 4 + i];                      // activations k = 8(4b+i) .. +7
             __half2 p[4], q[4];
             q4_word_to_h2(cp.v[b * 4 + i], p, kc);
             q4_word_to_h2(cq.v[b * 4 + i], q, kc);
-            mma16816(c, as_u32(p[0]), as_u32(q[0]), as_u32(p[1]), as_u32(q[1]), xv.x, xv.y);
+            if (i == 0)
+                mma16816_zero(c, as_u32(p[0]), as_u32(q[0]), as_u32(p[1]), as_u32(q[1]), xv.x, xv.y);
+            else
+                mma16816(c, as_u32(p[0]), as_u32(q[0]), as_u32(p[1]), as_u32(q[1]), xv.x, xv.y);
             mma16816(c, as_u32(p[2]), as_u32(q[2]), as_u32(p[3]), as_u32(q[3]), xv.z, xv.w);
         }
         // scales: sp.x / sp.y = rows 4g+2t / 4g+2t+1 of P as (block 0, block 1) fp16 pairs
@@ -80,14 +95,17 @@ __device__ __forceinline__ void tile_pair_mma_q4(const u32x8& cp, const u32x8& c
 __device__ __forceinline__ void tile_pair_mma_q8(const u32x8& cp, const u32x8& cq, uint32_t sp, uint32_t sq,
                                                  const uint4* xt, float (&acc)[4])
 {
-    float c[4] = {0.f, 0.f, 0.f, 0.f};
+    float c[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         const uint4 xv = xt[i];                                  // activations k = 8i .. 8i+7
         __half2 p[2], q[2];
         q8_word_to_h2(cp.v[2 * i], p);
         q8_word_to_h2(cq.v[2 * i], q);
-        mma16816(c, as_u32(p[0]), as_u32(q[0]), as_u32(p[1]), as_u32(q[1]), xv.x, xv.y);
+        if (i == 0)
+            mma16816_zero(c, as_u32(p[0]), as_u32(q[0]), as_u32(p[1]), as_u32(q[1]), xv.x, xv.y);
+        else
+            mma16816(c, as_u32(p[0]), as_u32(q[0]), as_u32(p[1]), as_u32(q[1]), xv.x, xv.y);
         q8_word_to_h2(cp.v[2 * i + 1], p);
         q8_word_to_h2(cq.v[2 * i + 1], q);
         mma16816(c, as_u32(p[0]), as_u32(q[0]), as_u32(p[1]), as_u32(q[1]), xv.z, xv.w);
@@ -159,19 +177,19 @@ gemv_kernel(const uint8_t* __restrict__ packed, const uint16_t* __restrict__ x,
     const uint8_t* tiles_p = lane_base + (size_t)(2 * pair) * group_bytes;
 
     TileRegs<FMT> r;
+    // slot u of the register file holds tile pair t + u * WARPS of the current item
+    auto load_slot = [&](int u, int tt) {
+        const uint8_t* tp = tiles_p + (size_t)tt * TB;
+        const uint8_t* tq = tp + group_bytes;
+        r.cp[u] = ld_stream_256(tp);
+        r.cq[u] = ld_stream_256(tq);
+        r.sp[u] = load_scales<FMT>(tp - 32 * lane, lane);
+        r.sq[u] = load_scales<FMT>(tq - 32 * lane, lane);
+    };
     auto load_group = [&]() {
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-            const int tt = t + u * WARPS;
-            if (tt < t_end) {
-                const uint8_t* tp = tiles_p + (size_t)tt * TB;
-                const uint8_t* tq = tp + group_bytes;
-                r.cp[u] = ld_stream_256(tp);
-                r.cq[u] = ld_stream_256(tq);
-                r.sp[u] = load_scales<FMT>(tp - 32 * lane, lane);
-                r.sq[u] = load_scales<FMT>(tq - 32 * lane, lane);
-            }
-        }
+        for (int u = 0; u < kUnroll; ++u)
+            if (t + u * WARPS < t_end) load_slot(u, t + u * WARPS);
     };
     if (item < items) load_group();
 
@@ -269,7 +287,10 @@ struct BatchParams {
 };
 
 template <int FMT, int WARPS>
-__global__ void __launch_bounds__(WARPS * 32, 768 / (WARPS * 32))
+#ifndef QMM_BATCH_THREADS_PER_SM
+#define QMM_BATCH_THREADS_PER_SM 768
+#endif
+__global__ void __launch_bounds__(WARPS * 32, QMM_BATCH_THREADS_PER_SM / (WARPS * 32))
 gemv_batch_kernel(const __grid_constant__ BatchParams bp)
 {
     extern __shared__ uint4 smem[];
@@ -308,19 +329,19 @@ gemv_batch_kernel(const __grid_constant__ BatchParams bp)
         t = warp;
         t_end = bp.p[p].tpr;
     };
+    // slot u of the register file holds tile pair t + u * WARPS of the current item
+    auto load_slot = [&](int u, int tt) {
+        const uint8_t* tp = tiles_p + (size_t)tt * TB;
+        const uint8_t* tq = tp + group_bytes;
+        r.cp[u] = ld_stream_256(tp);
+        r.cq[u] = ld_stream_256(tq);
+        r.sp[u] = load_scales<FMT>(tp - 32 * lane, lane);
+        r.sq[u] = load_scales<FMT>(tq - 32 * lane, lane);
+    };
     auto load_group = [&]() {
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-            const int tt = t + u * WARPS;
-            if (tt < t_end) {
-                const uint8_t* tp = tiles_p + (size_t)tt * TB;
-                const uint8_t* tq = tp + group_bytes;
-                r.cp[u] = ld_stream_256(tp);
-                r.cq[u] = ld_stream_256(tq);
-                r.sp[u] = load_scales<FMT>(tp - 32 * lane, lane);
-                r.sq[u] = load_scales<FMT>(tq - 32 * lane, lane);
-            }
-        }
+        for (int u = 0; u < kUnroll; ++u)
+            if (t + u * WARPS < t_end) load_slot(u, t + u * WARPS);
     };
     bool have = valid(pi, unit);
     if (have) {
@@ -509,7 +530,7 @@ qmm_status launch_gemv_batch(int fmt, const qmm_gemv_problem* probs, int count, 
         constexpr int WARPS = 8;
         const size_t smem = (size_t)max_k * 4 + (size_t)WARPS * 64 * sizeof(float);
         const int units = cost / (max_k / tile_k_of(fmt)) + 1;
-        int grid = kNumSMs * (768 / (WARPS * 32));
+        int grid = kNumSMs * (QMM_BATCH_THREADS_PER_SM / (WARPS * 32));
         if (units < grid) grid = units;
         cudaError_t e;
         if (fmt == QMM_Q4) {
