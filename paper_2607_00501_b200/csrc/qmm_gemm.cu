@@ -3,6 +3,8 @@
 // launch_tc_gemm, the grouped expert GEMMs of qmm_moe.
 #include "qmm_gemm_kernel.cuh"
 
+#include <stdlib.h>
+
 namespace qmm {
 
 // cuTensorMapEncodeTiled is reached through the runtime so that libqmm links
@@ -45,7 +47,7 @@ template <int FMT, int BN, int NA, int EPI>
 static qmm_status launch_t(const CUtensorMap& map, const GemmParams& p, dim3 grid, cudaStream_t st)
 {
     auto kern = gemm_kernel<FMT, BN, NA, EPI>;
-    constexpr int smem = GemmSmem<BN, NA>::kBytes;
+    constexpr int smem = GemmGeom<BN, NA>::kSmemBytes;
     static bool configured = false;                 // per instantiation; attribute is sticky per device context
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
@@ -54,7 +56,7 @@ static qmm_status launch_t(const CUtensorMap& map, const GemmParams& p, dim3 gri
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
-    cfg.blockDim = dim3((4 * NA + 2) * 32);
+    cfg.blockDim = dim3((4 * NA * kGemmPhases + 2) * 32);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -75,6 +77,7 @@ qmm_status launch_tc_gemm(int fmt, int bn, int na, int epi, const CUtensorMap& m
     QMM_TC_CASE(F, 32, 1, kEpiStore)      \
     QMM_TC_CASE(F, 64, 1, kEpiStore)      \
     QMM_TC_CASE(F, 128, 1, kEpiStore)     \
+    QMM_TC_CASE(F, 256, 1, kEpiStore)     \
     QMM_TC_CASE(F, 32, 2, kEpiStore)      \
     QMM_TC_CASE(F, 64, 2, kEpiStore)      \
     QMM_TC_CASE(F, 128, 2, kEpiStore)     \
@@ -99,8 +102,14 @@ size_t gemm_workspace_bytes(int, int64_t, int64_t, int64_t) { return 256; }
 qmm_status launch_gemm(int fmt, const void* packed, int64_t N, int64_t K, const uint16_t* X, int64_t ldx,
                        uint16_t* Y, int64_t ldy, int64_t M, void* ws, cudaStream_t st)
 {
-    const int bn = pick_token_tile(M);
-    const int na = (N % 256 == 0) ? 2 : 1;
+    int bn = pick_token_tile(M);
+    int na = (N % 256 == 0) ? 2 : 1;
+    if (const char* f = getenv("QMM_GEMM_NA")) {               // tuning sweeps
+        if (f[0] == '1') na = 1;
+    }
+    if (const char* f = getenv("QMM_GEMM_BN")) {
+        if (atoi(f) == 256 && M > 128) { bn = 256; na = 1; }
+    }
     CUtensorMap map;
     qmm_status s = make_x_map(&map, X, M, K, ldx, bn);
     if (s != QMM_OK) return s;
@@ -116,6 +125,7 @@ qmm_status launch_gemm(int fmt, const void* packed, int64_t N, int64_t K, const 
     p.a_col_offset = (int)(N / 2);
     p.M = (int)M;
     p.status = (int*)ws;
+    if (getenv("QMM_GEMM_TRACE")) p.trace = (long long*)((uint8_t*)ws + 256);   // tuning aid: needs a workspace of >= 256 + 4096 bytes
     const dim3 grid((unsigned)(N / (128 * na)), (unsigned)((M + bn - 1) / bn));
     return launch_tc_gemm(fmt, bn, na, kEpiStore, map, p, grid, st);
 }

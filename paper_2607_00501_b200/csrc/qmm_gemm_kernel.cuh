@@ -17,7 +17,8 @@
 // tile (half the activation traffic; the gate and up matrices of an expert).
 //
 // Roles (warp specialised):
-//   warps 0 .. 4*NA-1  expanders: thread = one weight row; 32-byte code loads
+//   warps 0 .. 8*NA-1  expanders (two per weight tile and lane quarter, alternating
+//                      stages): thread = one weight row; 32-byte code loads
 //                      straight from global/L2, unpack to fp16(d*q), tcgen05.st
 //                      into the A ring in TMEM; afterwards the epilogue.
 //   warp 4*NA          TMA producer: activation tiles -> shared-memory ring
@@ -39,7 +40,7 @@
 namespace qmm {
 
 constexpr int kGemmBK = 64;          // k per pipeline stage
-constexpr int kGemmStages = 4;
+constexpr int kGemmMaxStages = 6;     // pipeline depth is min(this, what tensor memory leaves for the weight ring)
 
 enum GemmEpilogue { kEpiStore = 0, kEpiSiluMul = 1 };
 
@@ -57,13 +58,22 @@ struct GemmParams {
     const int* tile_rows;            // [max_tiles] valid rows in the tile (<= BN)
     const int* num_tiles;            // [1]
     int* status;                     // device status word (0 = ok)
+    long long* trace;                // optional [block 0 only] clock64 samples for pipeline analysis (tuning aid), else null
 };
 
+// Pipeline geometry of one instantiation.  Tensor memory: half of the SM's 512 columns when the
+// accumulators leave room for it (two blocks per SM), else all of it; what the accumulators leave
+// is the weight ring.  A stage is one weight slot in TMEM plus one activation slot in shared memory.
 template <int BN, int NA>
-struct GemmSmem {
-    static constexpr int kBStage = BN * kGemmBK * 2;                       // bytes per activation stage
-    static constexpr int kBarriers = 3 * kGemmStages + 1;
-    static constexpr int kBytes = kGemmStages * kBStage + 1024 /*align*/ + 256;
+struct GemmGeom {
+    static constexpr int kACols = NA * 32;                                 // TMEM columns per weight slot
+    static constexpr int kDCols = NA * BN;                                 // accumulator columns
+    static constexpr int kTmemCols = kDCols <= 128 ? 256 : 512;
+    static constexpr int kFit = (kTmemCols - kDCols) / kACols;
+    static constexpr int kStages = kFit < kGemmMaxStages ? kFit : kGemmMaxStages;
+    static constexpr int kBStage = BN * kGemmBK * 2;                       // bytes per activation slot
+    static constexpr int kSmemBytes = kStages * kBStage + 1024 /*align*/ + 256;
+    static_assert(kStages >= 2, "tensor memory over-subscribed");
 };
 
 __device__ __forceinline__ float silu_f(float g) { return g / (1.0f + __expf(-g)); }
@@ -122,32 +132,33 @@ template <> struct RawRow64<QMM_Q8> {
     }
 };
 
-constexpr int kGemmPrefetch = 4;     // weight slices in flight per expander thread
+constexpr int kGemmPrefetch = 2;     // weight slices in flight per expander thread
+constexpr int kGemmPhases = 2;       // expander warps per (weight tile, lane quarter): they alternate pipeline stages
 
 template <int FMT, int BN, int NA, int EPI>
-__global__ void __launch_bounds__((4 * NA + 2) * 32, 1)
+__global__ void __launch_bounds__((4 * NA * kGemmPhases + 2) * 32, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
 {
     using namespace tc;
-    constexpr int NEXP = 4 * NA;                      // expander warps
+    constexpr int PH = kGemmPhases;
+    constexpr int NEXP = 4 * NA * PH;                 // expander warps
     constexpr int TMA_WARP = NEXP, MMA_WARP = NEXP + 1;
-    constexpr int S = kGemmStages;
-    constexpr int A_COLS = NA * 32;                   // TMEM columns per A stage
-    constexpr int D_COLS = NA * BN;
-    constexpr int TMEM_COLS = (D_COLS + S * A_COLS) <= 128 ? 128 : (D_COLS + S * A_COLS) <= 256 ? 256 : 512;
-    static_assert(D_COLS + S * A_COLS <= 512, "tensor memory over-subscribed");
+    using G = GemmGeom<BN, NA>;
+    constexpr int S = G::kStages;                     // pipeline depth
+    constexpr int A_COLS = G::kACols;
+    constexpr int D_COLS = G::kDCols;
+    constexpr int TMEM_COLS = G::kTmemCols;
     static_assert(BN % 16 == 0 && BN >= 16 && BN <= 256, "MMA N");
     constexpr int B_STAGE = BN * kGemmBK * 2;
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint8_t* smem_b = smem;                                               // S stages, 1024-aligned each
+    uint8_t* smem_b = smem;                                               // S slots, 1024-aligned each
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S * B_STAGE);
-    uint64_t* a_full = bars;                                              // [S] expanders -> MMA
-    uint64_t* b_full = bars + S;                                          // [S] TMA -> MMA
-    uint64_t* empty = bars + 2 * S;                                       // [S] MMA -> producers
-    uint64_t* acc_full = bars + 3 * S;                                    // MMA -> epilogue
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3 * S + 1);
+    uint64_t* full = bars;                                                // [S] expanders + TMA -> MMA
+    uint64_t* empty = bars + S;                                           // [S] MMA -> expanders, TMA
+    uint64_t* acc_full = bars + 2 * S;                                    // MMA -> epilogue
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 1);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -170,9 +181,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
     // ---- set-up
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
-            mbar_init(&a_full[s], NEXP);                                  // one arrival per expander warp
-            mbar_init(&b_full[s], 1);
-            mbar_init(&empty[s], 1);
+            mbar_init(&full[s], 4 * NA + 1);                              // the stage's expander warps + the TMA producer
+            mbar_init(&empty[s], 1);                                      // one tcgen05.commit
         }
         mbar_init(acc_full, 1);
         *abort_flag = 0;
@@ -192,8 +202,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
 
     if (warp < NEXP) {
         // ================= expanders: weights -> fp16 -> TMEM A ring
-        const int a = warp >> 2;                                          // weight tile set
         const int quarter = warp & 3;                                     // TMEM lane quarter
+        const int a = (warp >> 2) % NA;                                   // weight tile set
+        const int phase = (warp >> 2) / NA;                               // takes the stages kb = phase (mod PH)
         const int rg = n_tile * 4 + quarter;                              // row group of 32 rows
         const int tpr = p.K / Fmt<FMT>::tile_k;
         constexpr int TILES_PER_KB = kGemmBK / Fmt<FMT>::tile_k;
@@ -201,32 +212,48 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         Q4Consts kc;
         kc.init();
         const size_t kb_bytes = (size_t)TILES_PER_KB * Fmt<FMT>::tile_bytes;
+        const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);
         RawRow64<FMT> raw[kGemmPrefetch];
 #pragma unroll
         for (int i = 0; i < kGemmPrefetch; ++i)
-            if (i < num_kb) raw[i].load(wrow + i * kb_bytes, lane);
+            if (phase + i * PH < num_kb) raw[i].load(wrow + (size_t)(phase + i * PH) * kb_bytes, lane);
         bool ok = true;
-        for (int kb0 = 0; kb0 < num_kb && ok; kb0 += kGemmPrefetch) {
+        int pending = -1;                                                 // stage stored but not yet announced
+        // The store of one stage is announced (wait::st + arrive) only after the next stage has been
+        // expanded, so the tensor-memory write latency hides behind ALU work.
+        auto announce = [&]() {
+            if (pending >= 0) {
+                tmem_wait_st();
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&full[pending]);
+                pending = -1;
+            }
+        };
+        for (int kb0 = phase; kb0 < num_kb && ok; kb0 += kGemmPrefetch * PH) {
 #pragma unroll
             for (int i = 0; i < kGemmPrefetch; ++i) {
-                const int kb = kb0 + i;
+                const int kb = kb0 + i * PH;
                 if (kb >= num_kb || !ok) break;
                 const int s = kb % S;
                 uint32_t vals[32];
+                const bool tr = p.trace != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && kb < 64 && quarter == 0 && a == 0 && lane == 0;
+                if (tr) p.trace[kb * 8 + 4] = clock64();
                 raw[i].expand(vals, kc);
-                if (kb + kGemmPrefetch < num_kb) raw[i].load(wrow + (size_t)(kb + kGemmPrefetch) * kb_bytes, lane);
+                if (kb + kGemmPrefetch * PH < num_kb) raw[i].load(wrow + (size_t)(kb + kGemmPrefetch * PH) * kb_bytes, lane);
+                if (tr) p.trace[kb * 8 + 5] = clock64();
+                announce();
+                if (tr) p.trace[kb * 8 + 6] = clock64();
                 if (kb >= S) ok = mbar_wait(&empty[s], ((kb / S) - 1) & 1, abort_flag);
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
                 tc_fence_after_sync();
-                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(D_COLS + s * A_COLS + a * 32);
-                tmem_st_32x32b_x32(taddr, vals);
-                tmem_wait_st();
-                tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&a_full[s]);
+                tmem_st_32x32b_x32(lane_base + (uint32_t)(D_COLS + s * A_COLS + a * 32), vals);
+                if (tr) p.trace[kb * 8 + 7] = clock64();
+                pending = s;
             }
         }
+        if (ok) announce();
         if (!ok) *abort_flag = 1;
 
         // ================= epilogue: TMEM -> registers -> global
@@ -239,10 +266,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             } else if (EPI == kEpiStore || a == 0) {
                 tc_fence_after_sync();
                 const int n = n_tile * 128 + quarter * 32 + lane;         // weight row within the tile set
-                for (int c0 = 0; c0 < BN; c0 += 32) {
+                for (int c0 = phase * 32; c0 < BN; c0 += 32 * PH) {        // the phases share the column chunks
                     if (c0 >= rows) break;                                // uniform
                     uint32_t v[32];
-                    const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+                    const uint32_t lane_addr = lane_base;
                     tmem_ld_32x32b_x32(lane_addr + (uint32_t)(a * BN + c0), v);
                     if (EPI == kEpiSiluMul) {
                         uint32_t u[32];
@@ -270,16 +297,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                 const int s = kb % S;
                 if (kb >= S) ok = mbar_wait(&empty[s], ((kb / S) - 1) & 1, abort_flag);
                 if (!ok) break;
-                mbar_arrive_expect_tx(&b_full[s], B_STAGE);
-                tma_load_2d(smem_b + s * B_STAGE, &x_map, kb * kGemmBK, row0, &b_full[s]);
+                mbar_arrive_expect_tx(&full[s], B_STAGE);
+                tma_load_2d(smem_b + s * B_STAGE, &x_map, kb * kGemmBK, row0, &full[s]);
                 issued = kb + 1;
             }
             if (!ok) {
                 *abort_flag = 1;
                 // let loads in flight land before the block's shared memory is released
+                // (the same barrier also counts expander arrivals, so this can run into its time limit)
                 for (int kb = max(0, issued - S); kb < issued; ++kb) {
                     const long long t0 = clock64();
-                    while (!mbar_try_wait(&b_full[kb % S], (kb / S) & 1) && clock64() - t0 < kWaitLimitCycles) {}
+                    while (!mbar_try_wait(&full[kb % S], (kb / S) & 1) && clock64() - t0 < (1LL << 22)) {}
                 }
             }
         }
@@ -287,24 +315,28 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         // ================= MMA issuer
         if (lane == 0) {
             constexpr uint32_t idesc = idesc_f16_m128(BN);
+            const uint64_t desc0 = smem_desc_k_sw128(smem_u32(smem_b));   // slot 0, k-step 0
             bool ok = true;
             for (int kb = 0; kb < num_kb; ++kb) {
                 const int s = kb % S;
-                const uint32_t ph = (kb / S) & 1;
-                ok = mbar_wait(&a_full[s], ph, abort_flag) && mbar_wait(&b_full[s], ph, abort_flag);
+                const bool tr = p.trace != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && kb < 64;
+                if (tr) p.trace[kb * 8 + 0] = clock64();
+                ok = mbar_wait(&full[s], (kb / S) & 1, abort_flag);
+                if (tr) p.trace[kb * 8 + 2] = clock64();
                 if (!ok) break;
                 tc_fence_after_sync();
-                const uint32_t b_addr = smem_u32(smem_b + s * B_STAGE);
+                // descriptor start address is in 16-byte units: slot s is s * B_STAGE / 16 further, k-step k is 2 further
+                const uint64_t desc_s = desc0 + (uint64_t)(s * (B_STAGE >> 4));
+                const uint32_t a_s = tmem_base + (uint32_t)(D_COLS + s * A_COLS);
 #pragma unroll
                 for (int a = 0; a < NA; ++a) {
 #pragma unroll
-                    for (int k = 0; k < kGemmBK / 16; ++k) {
-                        const uint64_t bdesc = smem_desc_k_sw128(b_addr + k * 32);
-                        const uint32_t a_tmem = tmem_base + (uint32_t)(D_COLS + s * A_COLS + a * 32 + k * 8);
-                        mma_ts_f16(tmem_base + (uint32_t)(a * BN), a_tmem, bdesc, idesc, (kb | k) != 0);
-                    }
+                    for (int k = 0; k < kGemmBK / 16; ++k)
+                        mma_ts_f16(tmem_base + (uint32_t)(a * BN), a_s + (uint32_t)(a * 32 + k * 8), desc_s + (uint64_t)(k * 2), idesc,
+                                   (kb | k) != 0);
                 }
                 mma_commit(&empty[s]);                                    // slot reusable when these MMAs finish
+                if (tr) p.trace[kb * 8 + 3] = clock64();
             }
             if (ok) mma_commit(acc_full);
             else *abort_flag = 1;
