@@ -3,6 +3,7 @@
 // launch_tc_gemm, the grouped expert GEMMs of qmm_moe.
 #include "qmm_gemm_kernel.cuh"
 
+#include <stdio.h>
 #include <stdlib.h>
 
 namespace qmm {
@@ -56,7 +57,7 @@ static qmm_status launch_t(const CUtensorMap& map, const GemmParams& p, dim3 gri
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
-    cfg.blockDim = dim3((4 * NA * kGemmPhases + 2) * 32);
+    cfg.blockDim = dim3(kGemmThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -91,6 +92,17 @@ qmm_status launch_tc_gemm(int fmt, int bn, int na, int epi, const CUtensorMap& m
     return fail(QMM_ERR_UNSUPPORTED, "no tensor-core kernel for fmt=%d bn=%d na=%d epi=%d", fmt, bn, na, epi);
 }
 
+// Persistent grid: one block per SM (a block's 18 warps use most of the register file), never
+// more blocks than tiles (tiles <= 0: unknown on the host, the kernel reads the count).
+dim3 persistent_grid(int bn, int na, int64_t tiles)
+{
+    (void)bn;
+    (void)na;
+    int64_t g = kNumSMs;
+    if (tiles > 0 && tiles < g) g = tiles;
+    return dim3((unsigned)g);
+}
+
 int pick_token_tile(int64_t rows)
 {
     return rows <= 32 ? 32 : rows <= 64 ? 64 : 128;
@@ -102,13 +114,17 @@ size_t gemm_workspace_bytes(int, int64_t, int64_t, int64_t) { return 256; }
 qmm_status launch_gemm(int fmt, const void* packed, int64_t N, int64_t K, const uint16_t* X, int64_t ldx,
                        uint16_t* Y, int64_t ldy, int64_t M, void* ws, cudaStream_t st)
 {
-    int bn = pick_token_tile(M);
-    int na = (N % 256 == 0) ? 2 : 1;
-    if (const char* f = getenv("QMM_GEMM_NA")) {               // tuning sweeps
-        if (f[0] == '1') na = 1;
-    }
-    if (const char* f = getenv("QMM_GEMM_BN")) {
-        if (atoi(f) == 256 && M > 128) { bn = 256; na = 1; }
+    // Token tile: 256 (the widest MMA, N = 256) once M exceeds one 128-token tile; one weight tile
+    // per block, so that small problems spread over as many SMs as possible.
+    int bn = M > 128 ? 256 : pick_token_tile(M);
+    int na = 1;
+    if (const char* f = getenv("QMM_GEMM_FORCE")) {            // "bn,na" for tuning sweeps
+        int b = 0, a = 0;
+        if (sscanf(f, "%d,%d", &b, &a) == 2 && (a == 1 || (a == 2 && N % 256 == 0 && b <= 128)) &&
+            (b == 32 || b == 64 || b == 128 || (b == 256 && a == 1))) {
+            bn = b;
+            na = a;
+        }
     }
     CUtensorMap map;
     qmm_status s = make_x_map(&map, X, M, K, ldx, bn);
@@ -126,8 +142,8 @@ qmm_status launch_gemm(int fmt, const void* packed, int64_t N, int64_t K, const 
     p.M = (int)M;
     p.status = (int*)ws;
     if (getenv("QMM_GEMM_TRACE")) p.trace = (long long*)((uint8_t*)ws + 256);   // tuning aid: needs a workspace of >= 256 + 4096 bytes
-    const dim3 grid((unsigned)(N / (128 * na)), (unsigned)((M + bn - 1) / bn));
-    return launch_tc_gemm(fmt, bn, na, kEpiStore, map, p, grid, st);
+    const int64_t tiles = (N / (128 * na)) * ((M + bn - 1) / bn);
+    return launch_tc_gemm(fmt, bn, na, kEpiStore, map, p, persistent_grid(bn, na, tiles), st);
 }
 
 // Reads and clears the device status word (first int of a GEMM / MoE workspace).

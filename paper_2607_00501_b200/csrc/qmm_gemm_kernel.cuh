@@ -17,14 +17,17 @@
 // tile (half the activation traffic; the gate and up matrices of an expert).
 //
 // Roles (warp specialised):
-//   warps 0 .. 8*NA-1  expanders (two per weight tile and lane quarter, alternating
-//                      stages): thread = one weight row; 32-byte code loads
-//                      straight from global/L2, unpack to fp16(d*q), tcgen05.st
-//                      into the A ring in TMEM; afterwards the epilogue.
-//   warp 4*NA          TMA producer: activation tiles -> shared-memory ring
+//   warps 0 .. 7       expanders (8 / (4*NA) per weight tile and lane quarter,
+//                      alternating stages): thread = one weight row; 32-byte code
+//                      loads straight from global/L2, unpack to fp16(d*q),
+//                      tcgen05.st into the A ring in TMEM.
+//   warps 8 .. 15      epilogue: tcgen05.ld the accumulators, release them, store fp16.
+//   warp 16            TMA producer: activation tiles -> shared-memory ring
 //                      (128-byte swizzle), one elected lane.
-//   warp 4*NA+1        MMA issuer: one elected lane issues tcgen05.mma
+//   warp 17            MMA issuer: one elected lane issues tcgen05.mma
 //                      (M128 x N=BN x K16), frees ring slots with tcgen05.commit.
+// The kernel is persistent: a block loops over tiles and the pipeline runs on
+// across tile boundaries.
 //
 // TMEM columns: [0, NA*BN) fp32 accumulators, then STAGES slots of NA*32
 // columns (64 fp16 k-values per row and weight tile).
@@ -133,22 +136,32 @@ template <> struct RawRow64<QMM_Q8> {
 };
 
 constexpr int kGemmPrefetch = 2;     // weight slices in flight per expander thread
-constexpr int kGemmPhases = 2;       // expander warps per (weight tile, lane quarter): they alternate pipeline stages
+constexpr int kGemmExpWarps = 8;     // expander warps per block
+constexpr int kGemmEpiWarps = 8;     // epilogue warps per block (two per TMEM lane quarter)
+constexpr int kGemmThreads = (kGemmExpWarps + kGemmEpiWarps + 2) * 32;
 
+// Persistent, warp-specialised kernel.  Every block walks the tile list
+// t = blockIdx.x, blockIdx.x + gridDim.x, ...; tile t = (token tile t / n_tiles,
+// weight tile t % n_tiles), so blocks that run together share activation tiles.
+// The pipeline (stage counter, barrier phases) runs on across tiles: while the
+// epilogue warps drain the accumulators of tile i, the expanders and the TMA
+// producer already fill the ring for tile i+1.
 template <int FMT, int BN, int NA, int EPI>
-__global__ void __launch_bounds__((4 * NA * kGemmPhases + 2) * 32, 1)
+__global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
 {
     using namespace tc;
-    constexpr int PH = kGemmPhases;
-    constexpr int NEXP = 4 * NA * PH;                 // expander warps
-    constexpr int TMA_WARP = NEXP, MMA_WARP = NEXP + 1;
+    constexpr int NEXP = kGemmExpWarps;
+    constexpr int PH = NEXP / (4 * NA);               // expander warps per (weight tile, lane quarter): they alternate stages
+    constexpr int NEPI = kGemmEpiWarps;
+    constexpr int TMA_WARP = NEXP + NEPI, MMA_WARP = NEXP + NEPI + 1;
     using G = GemmGeom<BN, NA>;
     constexpr int S = G::kStages;                     // pipeline depth
     constexpr int A_COLS = G::kACols;
     constexpr int D_COLS = G::kDCols;
     constexpr int TMEM_COLS = G::kTmemCols;
-    static_assert(BN % 16 == 0 && BN >= 16 && BN <= 256, "MMA N");
+    static_assert(BN % 32 == 0 && BN >= 32 && BN <= 256, "token tile");
+    static_assert(PH >= 1 && NEXP % 4 == 0, "expander warps must cover the four lane quarters");
     constexpr int B_STAGE = BN * kGemmBK * 2;
 
     extern __shared__ uint8_t smem_raw[];
@@ -158,24 +171,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
     uint64_t* full = bars;                                                // [S] expanders + TMA -> MMA
     uint64_t* empty = bars + S;                                           // [S] MMA -> expanders, TMA
     uint64_t* acc_full = bars + 2 * S;                                    // MMA -> epilogue
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 1);
+    uint64_t* acc_empty = bars + 2 * S + 1;                               // epilogue -> MMA
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-
-    // ---- which tile
-    const int n_tile = blockIdx.x;                                        // 128 weight rows (per tile set)
-    int expert = 0, row0, rows;
-    if (p.tile_expert != nullptr) {
-        pdl_wait();                                                       // the tile list is written upstream
-        if ((int)blockIdx.y >= *p.num_tiles) return;                      // uniform over the block
-        expert = p.tile_expert[blockIdx.y];
-        row0 = p.tile_row0[blockIdx.y];
-        rows = p.tile_rows[blockIdx.y];
-    } else {
-        row0 = blockIdx.y * BN;
-        rows = min(BN, p.M - row0);
-    }
+    const bool grouped = p.tile_expert != nullptr;
+    if (grouped) pdl_wait();                                              // the tile list is written upstream
+    // plain store: the NA tile sets split the rows of one matrix; SiLU*mul: they are two matrices of N rows each
+    const int n_tiles = (EPI == kEpiSiluMul) ? p.N / 128 : p.N / (128 * NA);
+    const int m_tiles = grouped ? *p.num_tiles : (p.M + BN - 1) / BN;
+    const int total_tiles = n_tiles * m_tiles;
     const int num_kb = p.K / kGemmBK;
 
     // ---- set-up
@@ -185,6 +191,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             mbar_init(&empty[s], 1);                                      // one tcgen05.commit
         }
         mbar_init(acc_full, 1);
+        mbar_init(acc_empty, NEPI);
         *abort_flag = 0;
         fence_barrier_init();
     }
@@ -200,23 +207,32 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
 
     pdl_launch_dependents();
 
+    // token rows of tile t
+    auto tile_rows = [&](int t, int& n_tile, int& expert, int& row0, int& rows) {
+        n_tile = t % n_tiles;
+        const int mt = t / n_tiles;
+        if (grouped) {
+            expert = p.tile_expert[mt];
+            row0 = p.tile_row0[mt];
+            rows = p.tile_rows[mt];
+        } else {
+            expert = 0;
+            row0 = mt * BN;
+            rows = min(BN, p.M - row0);
+        }
+    };
+
     if (warp < NEXP) {
         // ================= expanders: weights -> fp16 -> TMEM A ring
         const int quarter = warp & 3;                                     // TMEM lane quarter
         const int a = (warp >> 2) % NA;                                   // weight tile set
-        const int phase = (warp >> 2) / NA;                               // takes the stages kb = phase (mod PH)
-        const int rg = n_tile * 4 + quarter;                              // row group of 32 rows
+        const int phase = (warp >> 2) / NA;                               // takes the stages g = phase (mod PH)
         const int tpr = p.K / Fmt<FMT>::tile_k;
         constexpr int TILES_PER_KB = kGemmBK / Fmt<FMT>::tile_k;
-        const uint8_t* wrow = p.w[a] + (size_t)expert * p.w_expert_stride + (size_t)rg * tpr * Fmt<FMT>::tile_bytes;
-        Q4Consts kc;
-        kc.init();
         const size_t kb_bytes = (size_t)TILES_PER_KB * Fmt<FMT>::tile_bytes;
         const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);
-        RawRow64<FMT> raw[kGemmPrefetch];
-#pragma unroll
-        for (int i = 0; i < kGemmPrefetch; ++i)
-            if (phase + i * PH < num_kb) raw[i].load(wrow + (size_t)(phase + i * PH) * kb_bytes, lane);
+        Q4Consts kc;
+        kc.init();
         bool ok = true;
         int pending = -1;                                                 // stage stored but not yet announced
         // The store of one stage is announced (wait::st + arrive) only after the next stage has been
@@ -230,84 +246,128 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                 pending = -1;
             }
         };
-        for (int kb0 = phase; kb0 < num_kb && ok; kb0 += kGemmPrefetch * PH) {
+        int g0 = 0;                                                       // stage counter at the start of the tile
+        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, g0 += num_kb) {
+            int n_tile, expert, row0, rows;
+            tile_rows(t, n_tile, expert, row0, rows);
+            const int rg = n_tile * 4 + quarter;                          // row group of 32 rows
+            const uint8_t* wrow = p.w[a] + (size_t)expert * p.w_expert_stride + (size_t)rg * tpr * Fmt<FMT>::tile_bytes;
+            RawRow64<FMT> raw[kGemmPrefetch];
 #pragma unroll
-            for (int i = 0; i < kGemmPrefetch; ++i) {
-                const int kb = kb0 + i * PH;
-                if (kb >= num_kb || !ok) break;
-                const int s = kb % S;
-                uint32_t vals[32];
-                const bool tr = p.trace != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && kb < 64 && quarter == 0 && a == 0 && lane == 0;
-                if (tr) p.trace[kb * 8 + 4] = clock64();
-                raw[i].expand(vals, kc);
-                if (kb + kGemmPrefetch * PH < num_kb) raw[i].load(wrow + (size_t)(kb + kGemmPrefetch * PH) * kb_bytes, lane);
-                if (tr) p.trace[kb * 8 + 5] = clock64();
-                announce();
-                if (tr) p.trace[kb * 8 + 6] = clock64();
-                if (kb >= S) ok = mbar_wait(&empty[s], ((kb / S) - 1) & 1, abort_flag);
-                ok = __all_sync(0xFFFFFFFFu, ok);
-                if (!ok) break;
-                tc_fence_after_sync();
-                tmem_st_32x32b_x32(lane_base + (uint32_t)(D_COLS + s * A_COLS + a * 32), vals);
-                if (tr) p.trace[kb * 8 + 7] = clock64();
-                pending = s;
-            }
-        }
-        if (ok) announce();
-        if (!ok) *abort_flag = 1;
-
-        // ================= epilogue: TMEM -> registers -> global
-        if (p.out != nullptr) {
-            pdl_wait();                                                   // the output buffer may be in use upstream
-            bool acc_ok = ok && mbar_wait(acc_full, 0, abort_flag);
-            acc_ok = __all_sync(0xFFFFFFFFu, acc_ok);
-            if (!acc_ok) {
-                *abort_flag = 1;
-            } else if (EPI == kEpiStore || a == 0) {
-                tc_fence_after_sync();
-                const int n = n_tile * 128 + quarter * 32 + lane;         // weight row within the tile set
-                for (int c0 = phase * 32; c0 < BN; c0 += 32 * PH) {        // the phases share the column chunks
-                    if (c0 >= rows) break;                                // uniform
-                    uint32_t v[32];
-                    const uint32_t lane_addr = lane_base;
-                    tmem_ld_32x32b_x32(lane_addr + (uint32_t)(a * BN + c0), v);
-                    if (EPI == kEpiSiluMul) {
-                        uint32_t u[32];
-                        tmem_ld_32x32b_x32(lane_addr + (uint32_t)(BN + c0), u);
-                        tmem_wait_ld();
+            for (int i = 0; i < kGemmPrefetch; ++i)
+                if (phase + i * PH < num_kb) raw[i].load(wrow + (size_t)(phase + i * PH) * kb_bytes, lane);
+            for (int kb0 = phase; kb0 < num_kb && ok; kb0 += kGemmPrefetch * PH) {
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(silu_f(__uint_as_float(v[j])) * __uint_as_float(u[j]));
-                    } else {
-                        tmem_wait_ld();
-                    }
-                    uint16_t* o = p.out + (size_t)(row0 + c0) * p.ldo + (EPI == kEpiStore ? (size_t)a * p.a_col_offset : 0) + n;
-#pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        if (c0 + j < rows) o[(size_t)j * p.ldo] = __half_as_ushort(__float2half_rn(__uint_as_float(v[j])));
+                for (int i = 0; i < kGemmPrefetch; ++i) {
+                    const int kb = kb0 + i * PH;
+                    if (kb >= num_kb || !ok) break;
+                    const int g = g0 + kb;
+                    const int s = g % S;
+                    uint32_t vals[32];
+                    raw[i].expand(vals, kc);
+                    if (kb + kGemmPrefetch * PH < num_kb) raw[i].load(wrow + (size_t)(kb + kGemmPrefetch * PH) * kb_bytes, lane);
+                    announce();
+                    if (g >= S) ok = mbar_wait(&empty[s], ((g / S) - 1) & 1, abort_flag);
+                    ok = __all_sync(0xFFFFFFFFu, ok);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    tmem_st_32x32b_x32(lane_base + (uint32_t)(D_COLS + s * A_COLS + a * 32), vals);
+                    pending = s;
                 }
             }
         }
+        if (ok) announce();
+        else *abort_flag = 1;
+    } else if (warp < NEXP + NEPI) {
+        // ================= epilogue: TMEM -> registers -> global
+        const int e = warp - NEXP;
+        const int quarter = e & 3;                                        // == warp & 3: the lanes this warp may read
+        const int half = e >> 2;                                          // which half of the token columns
+        const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);
+        constexpr int CH = BN >= 64 ? BN / 64 : 1;                        // 32-column chunks per warp (BN = 32: the second half idles)
+        constexpr int NOUT = (EPI == kEpiSiluMul) ? 1 : NA;               // output tiles per weight row
+        pdl_wait();                                                       // the output buffer may be in use upstream
+        bool ok = true;
+        int it = 0;
+        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
+            int n_tile, expert, row0, rows;
+            tile_rows(t, n_tile, expert, row0, rows);
+            ok = mbar_wait(acc_full, it & 1, abort_flag);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) break;
+            tc_fence_after_sync();
+            // fp16 results of this warp's columns, two tokens per register
+            uint32_t packed[NOUT][CH][16];
+#pragma unroll
+            for (int o = 0; o < NOUT; ++o) {
+#pragma unroll
+                for (int c = 0; c < CH; ++c) {
+                    const int c0 = (half * CH + c) * 32;
+                    if (c0 < BN && c0 < rows) {                           // uniform over the warp
+                        uint32_t v[32];
+                        tmem_ld_32x32b_x32(lane_base + (uint32_t)(o * BN + c0), v);
+                        if (EPI == kEpiSiluMul) {
+                            uint32_t u[32];
+                            tmem_ld_32x32b_x32(lane_base + (uint32_t)(BN + c0), u);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(silu_f(__uint_as_float(v[j])) * __uint_as_float(u[j]));
+                        } else {
+                            tmem_wait_ld();
+                        }
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            packed[o][c][j] = as_u32(__floats2half2_rn(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1])));
+                    }
+                }
+            }
+            // the accumulators are in registers: the next tile may overwrite them
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_empty);
+            const int n = n_tile * 128 + quarter * 32 + lane;             // weight row within the tile set
+#pragma unroll
+            for (int o = 0; o < NOUT; ++o) {
+#pragma unroll
+                for (int c = 0; c < CH; ++c) {
+                    const int c0 = (half * CH + c) * 32;
+                    if (c0 < BN && c0 < rows) {
+                        uint16_t* out = p.out + (size_t)(row0 + c0) * p.ldo + (size_t)o * p.a_col_offset + n;
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            if (c0 + 2 * j < rows) out[(size_t)(2 * j) * p.ldo] = (uint16_t)(packed[o][c][j] & 0xFFFFu);
+                            if (c0 + 2 * j + 1 < rows) out[(size_t)(2 * j + 1) * p.ldo] = (uint16_t)(packed[o][c][j] >> 16);
+                        }
+                    }
+                }
+            }
+        }
+        if (!ok) *abort_flag = 1;
     } else if (warp == TMA_WARP) {
         // ================= TMA producer: activation tiles
         if (lane == 0) {
             pdl_wait();                                                   // activations come from the previous kernel
-            int issued = 0;
+            int issued = 0, g = 0;
             bool ok = true;
-            for (int kb = 0; kb < num_kb; ++kb) {
-                const int s = kb % S;
-                if (kb >= S) ok = mbar_wait(&empty[s], ((kb / S) - 1) & 1, abort_flag);
-                if (!ok) break;
-                mbar_arrive_expect_tx(&full[s], B_STAGE);
-                tma_load_2d(smem_b + s * B_STAGE, &x_map, kb * kGemmBK, row0, &full[s]);
-                issued = kb + 1;
+            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+                int n_tile, expert, row0, rows;
+                tile_rows(t, n_tile, expert, row0, rows);
+                for (int kb = 0; kb < num_kb; ++kb, ++g) {
+                    const int s = g % S;
+                    if (g >= S) ok = mbar_wait(&empty[s], ((g / S) - 1) & 1, abort_flag);
+                    if (!ok) break;
+                    mbar_arrive_expect_tx(&full[s], B_STAGE);
+                    tma_load_2d(smem_b + s * B_STAGE, &x_map, kb * kGemmBK, row0, &full[s]);
+                    issued = g + 1;
+                }
             }
             if (!ok) {
                 *abort_flag = 1;
                 // let loads in flight land before the block's shared memory is released
                 // (the same barrier also counts expander arrivals, so this can run into its time limit)
-                for (int kb = max(0, issued - S); kb < issued; ++kb) {
+                for (int q = max(0, issued - S); q < issued; ++q) {
                     const long long t0 = clock64();
-                    while (!mbar_try_wait(&full[kb % S], (kb / S) & 1) && clock64() - t0 < (1LL << 22)) {}
+                    while (!mbar_try_wait(&full[q % S], (q / S) & 1) && clock64() - t0 < (1LL << 22)) {}
                 }
             }
         }
@@ -317,29 +377,37 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             constexpr uint32_t idesc = idesc_f16_m128(BN);
             const uint64_t desc0 = smem_desc_k_sw128(smem_u32(smem_b));   // slot 0, k-step 0
             bool ok = true;
-            for (int kb = 0; kb < num_kb; ++kb) {
-                const int s = kb % S;
-                const bool tr = p.trace != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && kb < 64;
-                if (tr) p.trace[kb * 8 + 0] = clock64();
-                ok = mbar_wait(&full[s], (kb / S) & 1, abort_flag);
-                if (tr) p.trace[kb * 8 + 2] = clock64();
-                if (!ok) break;
-                tc_fence_after_sync();
-                // descriptor start address is in 16-byte units: slot s is s * B_STAGE / 16 further, k-step k is 2 further
-                const uint64_t desc_s = desc0 + (uint64_t)(s * (B_STAGE >> 4));
-                const uint32_t a_s = tmem_base + (uint32_t)(D_COLS + s * A_COLS);
-#pragma unroll
-                for (int a = 0; a < NA; ++a) {
-#pragma unroll
-                    for (int k = 0; k < kGemmBK / 16; ++k)
-                        mma_ts_f16(tmem_base + (uint32_t)(a * BN), a_s + (uint32_t)(a * 32 + k * 8), desc_s + (uint64_t)(k * 2), idesc,
-                                   (kb | k) != 0);
+            int g = 0, it = 0;
+            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
+                if (it > 0) {                                             // the epilogue must have read the accumulators
+                    ok = mbar_wait(acc_empty, (it - 1) & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after_sync();
                 }
-                mma_commit(&empty[s]);                                    // slot reusable when these MMAs finish
-                if (tr) p.trace[kb * 8 + 3] = clock64();
+                for (int kb = 0; kb < num_kb; ++kb, ++g) {
+                    const int s = g % S;
+                    const bool tr = p.trace != nullptr && blockIdx.x == 0 && g < 64;
+                    if (tr) p.trace[g * 8 + 0] = clock64();
+                    ok = mbar_wait(&full[s], (g / S) & 1, abort_flag);
+                    if (tr) p.trace[g * 8 + 2] = clock64();
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    // descriptor start address is in 16-byte units: slot s is s * B_STAGE / 16 further, k-step k is 2 further
+                    const uint64_t desc_s = desc0 + (uint64_t)(s * (B_STAGE >> 4));
+                    const uint32_t a_s = tmem_base + (uint32_t)(D_COLS + s * A_COLS);
+#pragma unroll
+                    for (int a = 0; a < NA; ++a) {
+#pragma unroll
+                        for (int k = 0; k < kGemmBK / 16; ++k)
+                            mma_ts_f16(tmem_base + (uint32_t)(a * BN), a_s + (uint32_t)(a * 32 + k * 8), desc_s + (uint64_t)(k * 2), idesc,
+                                       (kb | k) != 0);
+                    }
+                    mma_commit(&empty[s]);                                // slot reusable when these MMAs finish
+                    if (tr) p.trace[g * 8 + 3] = clock64();
+                }
+                if (ok) mma_commit(acc_full);                             // accumulators of this tile are complete
             }
-            if (ok) mma_commit(acc_full);
-            else *abort_flag = 1;
+            if (!ok) *abort_flag = 1;
         }
     }
 

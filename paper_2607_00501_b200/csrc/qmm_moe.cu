@@ -17,6 +17,7 @@ qmm_status make_x_map(CUtensorMap* map, const uint16_t* X, int64_t rows, int64_t
 qmm_status launch_tc_gemm(int fmt, int bn, int na, int epi, const CUtensorMap& map, const GemmParams& p, dim3 grid,
                           cudaStream_t st);
 int pick_token_tile(int64_t rows);
+dim3 persistent_grid(int bn, int na, int64_t tiles);
 
 // ------------------------------------------------------------ workspace
 
@@ -333,7 +334,7 @@ qmm_status launch_moe(const qmm_moe_args* a, void* ws, bool route_only, cudaStre
         p.tile_rows = tile_rows;
         p.num_tiles = num_tiles;
         p.status = status;
-        s = launch_tc_gemm(a->fmt, w.bn, 2, kEpiSiluMul, map, p, dim3(a->I / 128, w.max_tiles), st);
+        s = launch_tc_gemm(a->fmt, w.bn, 2, kEpiSiluMul, map, p, persistent_grid(w.bn, 2, 0), st);
         if (s != QMM_OK) return s;
     }
     // 5. grouped down GEMM -> D [total, H]
@@ -357,7 +358,7 @@ qmm_status launch_moe(const qmm_moe_args* a, void* ws, bool route_only, cudaStre
         p.tile_rows = tile_rows;
         p.num_tiles = num_tiles;
         p.status = status;
-        s = launch_tc_gemm(a->fmt, w.bn, na, kEpiStore, map, p, dim3(a->H / (128 * na), w.max_tiles), st);
+        s = launch_tc_gemm(a->fmt, w.bn, na, kEpiStore, map, p, persistent_grid(w.bn, na, 0), st);
         if (s != QMM_OK) return s;
     }
     // 6. weighted combine
