@@ -36,6 +36,10 @@ from paper_2607_00501_b200 import synth  # noqa: E402
 METRIC = "decode GEMV effective HBM bandwidth on quantised-weight bytes (Q4+Q8 16-layer stack)"
 UNIT = "GB/s"
 NOMINAL_BF16_TFLOPS = 2250.0
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of gemv_batch_kernel on this workload, from the
+# ncu captures summarised in profiles/gemv_batch_kernel_q{4,8}_cfg1_stack.md (algorithmic bytes: 547 356 672 /
+# 1 033 895 936).  Only reported, never used in a computation.
+NCU_DRAM_TRAFFIC = {synth.Q4: 552_050_000, synth.Q8: 1_038_200_000}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 # fused launches per layer: (name, constituent matrices, N, K, activation)
@@ -196,7 +200,8 @@ def run_ours(args):
             d[k] = x_all[off:off + n]
             off += n
         x_dev.append(d)
-    for f in fmts:
+    need_fused = args.mode == "streams" or not args.no_sections     # fused per-matrix launches: streams mode, chained sections
+    for f in (fmts if need_fused else ()):
         for l in range(layers):
             for name, parts, N, K, act in FUSED:
                 packed = torch.cat([qmm.pack(f, dev_u8(host_blocks[f][l][p]), rows_of[p], K) for p in parts])
@@ -278,6 +283,25 @@ def run_ours(args):
         barrier()
         step_ms = [evs[i].elapsed_time(evs[i + 1]) for i in range(args.steps)]
         total_ms = evs[0].elapsed_time(evs[-1])
+        # the two kernels of the step timed one by one (same launches, one format at a time)
+        per_kernel = {}
+        if args.mode == "batch":
+            for f in fmts:
+                for _ in range(3):
+                    qmm.gemv_batch(f, batch[f])
+                k0, k1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda.synchronize()
+                k0.record()
+                for _ in range(args.steps):
+                    qmm.gemv_batch(f, batch[f])
+                k1.record()
+                torch.cuda.synchronize()
+                us = k0.elapsed_time(k1) * 1e3 / args.steps
+                per_kernel["gemv_batch_kernel<Q%d>" % f] = {
+                    "avg_launch_us": round(us, 2), "algorithmic_bytes": stack_bytes(f),
+                    "achieved_GBps": round(stack_bytes(f) / us / 1e3, 1),
+                    "frac": round(stack_bytes(f) / us / 1e3 / pk["hbm_gbs"], 4),
+                    "ncu_dram_traffic_bytes": NCU_DRAM_TRAFFIC[f]}
         # keep the GPU busy a little longer so that the clock sampler sees load even for short runs
         t_end = time.time() + 1.0
         while time.time() < t_end:
@@ -339,7 +363,9 @@ def run_ours(args):
         "gpu_launches": launches_per_step * args.steps,
         "clocks": clocks,
         "roofline": {"bound": "hbm", "achieved": round(value / world, 1), "peak": pk["hbm_gbs"], "unit": "GB/s",
-                     "frac": round(value / world / pk["hbm_gbs"], 4), "traffic": None,
+                     "frac": round(value / world / pk["hbm_gbs"], 4),
+                     "traffic": sum(NCU_DRAM_TRAFFIC[f] for f in fmts) if args.mode == "batch" else None,
+                     "algorithmic_bytes": bytes_step, "per_kernel": per_kernel,
                      "kernel": "gemv_batch_kernel (both launches of the step)" if args.mode == "batch" else "gemv_kernel (all launches of the step)", "peak_source": pk["source"],
                      "step_ms_min": round(min(step_ms), 5), "step_ms_max": round(max(step_ms), 5)},
         "cpu_baseline": cpu,
@@ -507,6 +533,57 @@ def run_reference(args):
     }))
 
 
+def run_case(args):
+    """`--case NAME`: a few launches of one kernel on its benchmark workload and nothing else, so that a
+    profiler can be pointed at it (`ncu -k regex:... python bench.py --case gemm_q4_M2048`).  Prints no JSON."""
+    import torch
+    from paper_2607_00501_b200 import qmm
+    torch.cuda.set_device(0)
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    name = args.case
+    reps = 4
+    if name in ("gemv_batch_q4", "gemv_batch_q8"):
+        f = synth.Q4 if name.endswith("q4") else synth.Q8
+        host_blocks, host_acts = build_stack_host(synth.CFG1["layers"], (f,))
+        probs = []
+        for l in range(synth.CFG1["layers"]):
+            for mname, N, K, act in synth.CFG1_LAYER:
+                probs.append((qmm.pack(f, dev(host_blocks[f][l][mname]), N, K), N, K, dev(host_acts[l][act]),
+                              torch.empty(N, dtype=torch.float16, device="cuda")))
+        arr = qmm.gemv_batch_problems(probs)
+        for _ in range(reps):
+            qmm.gemv_batch(f, arr)
+    elif name.startswith("gemm_q4_M"):
+        c = synth.CFG3
+        M = int(name.split("_M")[1])
+        _, N, K = c["shapes"][0]
+        packed = qmm.pack(c["fmt"], dev(synth.quantize(c["fmt"], synth.weights(c["seed"], 0, N, K))), N, K)
+        X = dev(synth.activations(c["seed"], 10 + M, M, K))
+        Y = torch.empty((M, N), dtype=torch.float16, device="cuda")
+        ws = torch.zeros(256, dtype=torch.uint8, device="cuda")
+        for _ in range(reps):
+            qmm.gemm(c["fmt"], packed, N, K, X, Y=Y, ws=ws)
+        qmm.status_check(ws)
+    elif name.startswith("moe_q4_T"):
+        c = synth.CFG4
+        T = int(name.split("_T")[1])
+        gate, up, down = synth.moe_expert_weights(c["seed"], c["fmt"], c["E"], c["H"], c["I"])
+        pg, pu = qmm.pack(c["fmt"], dev(gate), c["E"] * c["I"], c["H"]), qmm.pack(c["fmt"], dev(up), c["E"] * c["I"], c["H"])
+        pd = qmm.pack(c["fmt"], dev(down), c["E"] * c["H"], c["I"])
+        X = dev(synth.activations(c["seed"], 100 + T, T, c["H"]))
+        lg = dev(synth.logits(c["seed"], 200 + T, T, c["E"]))
+        o = torch.empty((T, c["H"]), dtype=torch.float16, device="cuda")
+        a = qmm.moe_args(c["fmt"], T, c["H"], c["I"], c["E"], c["topk"], lg, X, pg, pu, pd, o)
+        ws = torch.zeros(qmm.moe_workspace_bytes(a), dtype=torch.uint8, device="cuda")
+        for _ in range(reps):
+            qmm.moe(a, ws)
+        qmm.status_check(ws)
+    else:
+        raise SystemExit("unknown --case %r (gemv_batch_q4, gemv_batch_q8, gemm_q4_M<M>, moe_q4_T<T>)" % name)
+    torch.cuda.synchronize()
+    print("case %s: %d launches done" % (name, reps), file=sys.stderr)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -519,7 +596,11 @@ def main():
     ap.add_argument("--no-sections", action="store_true", help="skip the LM-head / GEMM / MoE sections")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--case", default=None, help="profiling aid: run a few launches of one kernel and exit (see run_case)")
     args = ap.parse_args()
+    if args.case:
+        run_case(args)
+        return
     if args.impl == "reference":
         run_reference(args)
     else:
