@@ -373,28 +373,32 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         }
     } else {
         // ================= MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc = idesc_f16_m128(BN);
-            const uint64_t desc0 = smem_desc_k_sw128(smem_u32(smem_b));   // slot 0, k-step 0
-            bool ok = true;
-            int g = 0, it = 0;
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
-                if (it > 0) {                                             // the epilogue must have read the accumulators
-                    ok = mbar_wait(acc_empty, (it - 1) & 1, abort_flag);
-                    if (!ok) break;
-                    tc_fence_after_sync();
-                }
-                for (int kb = 0; kb < num_kb; ++kb, ++g) {
-                    const int s = g % S;
-                    const bool tr = p.trace != nullptr && blockIdx.x == 0 && g < 64;
-                    if (tr) p.trace[g * 8 + 0] = clock64();
-                    ok = mbar_wait(&full[s], (g / S) & 1, abort_flag);
-                    if (tr) p.trace[g * 8 + 2] = clock64();
-                    if (!ok) break;
-                    tc_fence_after_sync();
-                    // descriptor start address is in 16-byte units: slot s is s * B_STAGE / 16 further, k-step k is 2 further
-                    const uint64_t desc_s = desc0 + (uint64_t)(s * (B_STAGE >> 4));
-                    const uint32_t a_s = tmem_base + (uint32_t)(D_COLS + s * A_COLS);
+        // The whole warp runs the loop converged (so that addresses and descriptors stay warp-uniform
+        // values); one elected lane issues the MMAs and the commits.
+        constexpr uint32_t idesc = idesc_f16_m128(BN);
+        const uint64_t desc0 = smem_desc_k_sw128(smem_u32(smem_b));       // slot 0, k-step 0
+        bool ok = true;
+        int g = 0, it = 0;
+        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
+            if (it > 0) {                                                 // the epilogue must have read the accumulators
+                ok = mbar_wait(acc_empty, (it - 1) & 1, abort_flag);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
+                tc_fence_after_sync();
+            }
+            for (int kb = 0; kb < num_kb; ++kb, ++g) {
+                const int s = g % S;
+                const bool tr = p.trace != nullptr && blockIdx.x == 0 && g < 64 && lane == 0;
+                if (tr) p.trace[g * 8 + 0] = clock64();
+                ok = mbar_wait(&full[s], (g / S) & 1, abort_flag);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (tr) p.trace[g * 8 + 2] = clock64();
+                if (!ok) break;
+                tc_fence_after_sync();
+                // descriptor start address is in 16-byte units: slot s is s * B_STAGE / 16 further, k-step k is 2 further
+                const uint64_t desc_s = desc0 + (uint64_t)(s * (B_STAGE >> 4));
+                const uint32_t a_s = tmem_base + (uint32_t)(D_COLS + s * A_COLS);
+                if (elect_one()) {
 #pragma unroll
                     for (int a = 0; a < NA; ++a) {
 #pragma unroll
@@ -403,12 +407,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                                        (kb | k) != 0);
                     }
                     mma_commit(&empty[s]);                                // slot reusable when these MMAs finish
-                    if (tr) p.trace[g * 8 + 3] = clock64();
                 }
-                if (ok) mma_commit(acc_full);                             // accumulators of this tile are complete
+                __syncwarp();
+                if (tr) p.trace[g * 8 + 3] = clock64();
             }
-            if (!ok) *abort_flag = 1;
+            if (ok && elect_one()) mma_commit(acc_full);                  // accumulators of this tile are complete
+            __syncwarp();
         }
+        if (!ok) *abort_flag = 1;
     }
 
     // ---- teardown
