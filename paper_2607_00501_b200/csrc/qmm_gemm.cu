@@ -3,6 +3,7 @@
 // launch_tc_gemm, the grouped expert GEMMs of qmm_moe.
 #include "qmm_gemm_kernel.cuh"
 
+#include <math.h>
 #include <stdio.h>
 #include <stdlib.h>
 
@@ -57,7 +58,7 @@ static qmm_status launch_t(const CUtensorMap& map, const GemmParams& p, dim3 gri
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
-    cfg.blockDim = dim3(kGemmThreads);
+    cfg.blockDim = dim3(GemmGeom<BN, NA>::kThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -82,9 +83,11 @@ qmm_status launch_tc_gemm(int fmt, int bn, int na, int epi, const CUtensorMap& m
     QMM_TC_CASE(F, 32, 2, kEpiStore)      \
     QMM_TC_CASE(F, 64, 2, kEpiStore)      \
     QMM_TC_CASE(F, 128, 2, kEpiStore)     \
+    QMM_TC_CASE(F, 160, 2, kEpiStore)     \
     QMM_TC_CASE(F, 32, 2, kEpiSiluMul)    \
     QMM_TC_CASE(F, 64, 2, kEpiSiluMul)    \
-    QMM_TC_CASE(F, 128, 2, kEpiSiluMul)
+    QMM_TC_CASE(F, 128, 2, kEpiSiluMul)   \
+    QMM_TC_CASE(F, 160, 2, kEpiSiluMul)
     QMM_TC_FMT(QMM_Q4)
     QMM_TC_FMT(QMM_Q8)
 #undef QMM_TC_FMT
@@ -106,6 +109,16 @@ dim3 persistent_grid(int bn, int na, int64_t tiles)
 int pick_token_tile(int64_t rows)
 {
     return rows <= 32 ? 32 : rows <= 64 ? 64 : 128;
+}
+
+// Token tile of the grouped (per-expert) GEMMs: the smallest tile that holds the mean number of rows
+// per expert plus three standard deviations of a uniform routing (binomial), so that almost every
+// expert is one tile.  160 is the widest two-accumulator tile that leaves tensor memory for a 3-slot ring.
+int pick_expert_tile(int64_t total_rows, int experts)
+{
+    const double mean = (double)total_rows / experts;
+    const double want = mean + 3.0 * sqrt(mean) + 1.0;
+    return want <= 32 ? 32 : want <= 64 ? 64 : want <= 128 ? 128 : 160;
 }
 
 // The workspace of qmm_gemm holds only the device status word.

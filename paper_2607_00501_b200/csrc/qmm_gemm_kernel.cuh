@@ -17,14 +17,15 @@
 // tile (half the activation traffic; the gate and up matrices of an expert).
 //
 // Roles (warp specialised):
-//   warps 0 .. 7       expanders (8 / (4*NA) per weight tile and lane quarter,
-//                      alternating stages): thread = one weight row; 32-byte code
-//                      loads straight from global/L2, unpack to fp16(d*q),
+//   expanders (8 warps): 8 / (4*NA) per weight tile and lane quarter,
+//                      alternating stages; thread = one weight row; 32-byte
+//                      code loads straight from global/L2, unpack to fp16(d*q),
 //                      tcgen05.st into the A ring in TMEM.
-//   warps 8 .. 15      epilogue: tcgen05.ld the accumulators, release them, store fp16.
-//   warp 16            TMA producer: activation tiles -> shared-memory ring
-//                      (128-byte swizzle), one elected lane.
-//   warp 17            MMA issuer: one elected lane issues tcgen05.mma
+//   epilogue (8 warps, two per lane quarter): tcgen05.ld the accumulators,
+//                      release them, store fp16.
+//   TMA producer (1 warp): activation tiles -> shared-memory ring (128-byte
+//                      swizzle), one elected lane.
+//   MMA issuer (1 warp, converged): one elected lane issues tcgen05.mma
 //                      (M128 x N=BN x K16), frees ring slots with tcgen05.commit.
 // The kernel is persistent: a block loops over tiles and the pipeline runs on
 // across tile boundaries.
@@ -76,10 +77,16 @@ struct GemmGeom {
     static constexpr int kStages = kFit < kGemmMaxStages ? kFit : kGemmMaxStages;
     static constexpr int kBStage = BN * kGemmBK * 2;                       // bytes per activation slot
     static constexpr int kSmemBytes = kStages * kBStage + 1024 /*align*/ + 256;
+    // Warp roles: 8 expanders, 8 epilogue warps (two per TMEM lane quarter), TMA producer, MMA issuer.
+    static constexpr int kExpWarps = 8;
+    static constexpr int kEpiWarps = 8;
+    static constexpr int kThreads = (kExpWarps + kEpiWarps + 2) * 32;
     static_assert(kStages >= 2, "tensor memory over-subscribed");
 };
 
-__device__ __forceinline__ float silu_f(float g) { return g / (1.0f + __expf(-g)); }
+// silu(g) = g / (1 + exp(-g)) with the fast exponential and reciprocal (relative error ~1e-6,
+// far inside the fp16 rounding of the result; exp(-g) = inf for g < -88 gives -0, the right limit).
+__device__ __forceinline__ float silu_f(float g) { return __fdividef(g, 1.0f + __expf(-g)); }
 
 // One 64-k slice of a weight row as loaded (codes + scales), and its expansion
 // to fp16(d * q) pairs, k ascending.  Loading and expanding are separate so
@@ -136,9 +143,7 @@ template <> struct RawRow64<QMM_Q8> {
 };
 
 constexpr int kGemmPrefetch = 2;     // weight slices in flight per expander thread
-constexpr int kGemmExpWarps = 8;     // expander warps per block
-constexpr int kGemmEpiWarps = 8;     // epilogue warps per block (two per TMEM lane quarter)
-constexpr int kGemmThreads = (kGemmExpWarps + kGemmEpiWarps + 2) * 32;
+constexpr int kGemmL2Ahead = 12;     // stages of a row group's weight stream requested into L2 ahead of use
 
 // Persistent, warp-specialised kernel.  Every block walks the tile list
 // t = blockIdx.x, blockIdx.x + gridDim.x, ...; tile t = (token tile t / n_tiles,
@@ -147,15 +152,15 @@ constexpr int kGemmThreads = (kGemmExpWarps + kGemmEpiWarps + 2) * 32;
 // epilogue warps drain the accumulators of tile i, the expanders and the TMA
 // producer already fill the ring for tile i+1.
 template <int FMT, int BN, int NA, int EPI>
-__global__ void __launch_bounds__(kGemmThreads, 1)
+__global__ void __launch_bounds__(GemmGeom<BN, NA>::kThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
 {
     using namespace tc;
-    constexpr int NEXP = kGemmExpWarps;
-    constexpr int PH = NEXP / (4 * NA);               // expander warps per (weight tile, lane quarter): they alternate stages
-    constexpr int NEPI = kGemmEpiWarps;
-    constexpr int TMA_WARP = NEXP + NEPI, MMA_WARP = NEXP + NEPI + 1;
     using G = GemmGeom<BN, NA>;
+    constexpr int NEXP = G::kExpWarps;
+    constexpr int PH = NEXP / (4 * NA);               // expander warps per (weight tile, lane quarter): they alternate stages
+    constexpr int NEPI = G::kEpiWarps;
+    constexpr int TMA_WARP = NEXP + NEPI, MMA_WARP = NEXP + NEPI + 1;
     constexpr int S = G::kStages;                     // pipeline depth
     constexpr int A_COLS = G::kACols;
     constexpr int D_COLS = G::kDCols;
@@ -252,6 +257,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             tile_rows(t, n_tile, expert, row0, rows);
             const int rg = n_tile * 4 + quarter;                          // row group of 32 rows
             const uint8_t* wrow = p.w[a] + (size_t)expert * p.w_expert_stride + (size_t)rg * tpr * Fmt<FMT>::tile_bytes;
+            // The weight stream of a row group is contiguous: ask L2 for it kGemmL2Ahead stages ahead
+            // (expert weights come from HBM; two register-held slices alone do not cover that latency).
+            if (lane == 0 && phase == 0) {
+                const int ahead = num_kb < kGemmL2Ahead ? num_kb : kGemmL2Ahead;
+                l2_prefetch(wrow, (uint32_t)(ahead * kb_bytes));
+            }
             RawRow64<FMT> raw[kGemmPrefetch];
 #pragma unroll
             for (int i = 0; i < kGemmPrefetch; ++i)
@@ -264,15 +275,22 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                     const int g = g0 + kb;
                     const int s = g % S;
                     uint32_t vals[32];
+                    const bool tr = p.trace != nullptr && blockIdx.x == 0 && g < 64 && quarter == 0 && a == 0 && lane == 0;
+                    if (tr) p.trace[g * 8 + 4] = clock64();
                     raw[i].expand(vals, kc);
                     if (kb + kGemmPrefetch * PH < num_kb) raw[i].load(wrow + (size_t)(kb + kGemmPrefetch * PH) * kb_bytes, lane);
+                    if (lane == 0 && kb + kGemmL2Ahead < num_kb) l2_prefetch(wrow + (size_t)(kb + kGemmL2Ahead) * kb_bytes, (uint32_t)kb_bytes);
+                    if (tr) p.trace[g * 8 + 5] = clock64();
                     announce();
+                    if (tr) p.trace[g * 8 + 6] = clock64();
                     if (g >= S) ok = mbar_wait(&empty[s], ((g / S) - 1) & 1, abort_flag);
                     ok = __all_sync(0xFFFFFFFFu, ok);
                     if (!ok) break;
                     tc_fence_after_sync();
+                    if (tr) p.trace[g * 8 + 7] = clock64();
                     tmem_st_32x32b_x32(lane_base + (uint32_t)(D_COLS + s * A_COLS + a * 32), vals);
                     pending = s;
+                    if (PH == 1) announce();          // a lone warp per weight rows: nothing to overlap the store with
                 }
             }
         }
@@ -282,13 +300,45 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         // ================= epilogue: TMEM -> registers -> global
         const int e = warp - NEXP;
         const int quarter = e & 3;                                        // == warp & 3: the lanes this warp may read
-        const int half = e >> 2;                                          // which half of the token columns
+        constexpr int GROUPS = NEPI / 4;                                  // warps per lane quarter: they split the token columns
+        const int grp = e >> 2;
         const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);
-        constexpr int CH = BN >= 64 ? BN / 64 : 1;                        // 32-column chunks per warp (BN = 32: the second half idles)
+        constexpr int NCH = BN / 32;                                      // 32-column chunks of the tile
+        constexpr int CH = (NCH + GROUPS - 1) / GROUPS;                   // chunks per warp
         constexpr int NOUT = (EPI == kEpiSiluMul) ? 1 : NA;               // output tiles per weight row
+        constexpr bool HOLD = (NOUT * CH <= 6);                           // few chunks: read all, release, then store
         pdl_wait();                                                       // the output buffer may be in use upstream
         bool ok = true;
         int it = 0;
+        // one 32-column chunk of output tile o: accumulators -> fp16 pairs (two tokens per register)
+        auto read_chunk = [&](int o, int c0, uint32_t (&dst)[16]) {
+            uint32_t v[32];
+            tmem_ld_32x32b_x32(lane_base + (uint32_t)(o * BN + c0), v);
+            if (EPI == kEpiSiluMul) {
+                uint32_t u[32];
+                tmem_ld_32x32b_x32(lane_base + (uint32_t)(BN + c0), u);
+                tmem_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(silu_f(__uint_as_float(v[j])) * __uint_as_float(u[j]));
+            } else {
+                tmem_wait_ld();
+            }
+#pragma unroll
+            for (int j = 0; j < 16; ++j) dst[j] = as_u32(__floats2half2_rn(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1])));
+        };
+        auto store_chunk = [&](int o, int c0, int row0, int rows, int n, const uint32_t (&src)[16]) {
+            uint16_t* out = p.out + (size_t)(row0 + c0) * p.ldo + (size_t)o * p.a_col_offset + n;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                if (c0 + 2 * j < rows) out[(size_t)(2 * j) * p.ldo] = (uint16_t)(src[j] & 0xFFFFu);
+                if (c0 + 2 * j + 1 < rows) out[(size_t)(2 * j + 1) * p.ldo] = (uint16_t)(src[j] >> 16);
+            }
+        };
+        auto release = [&]() {                                            // the next tile may overwrite the accumulators
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_empty);
+        };
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
             int n_tile, expert, row0, rows;
             tile_rows(t, n_tile, expert, row0, rows);
@@ -296,50 +346,47 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
             tc_fence_after_sync();
-            // fp16 results of this warp's columns, two tokens per register
-            uint32_t packed[NOUT][CH][16];
-#pragma unroll
-            for (int o = 0; o < NOUT; ++o) {
-#pragma unroll
-                for (int c = 0; c < CH; ++c) {
-                    const int c0 = (half * CH + c) * 32;
-                    if (c0 < BN && c0 < rows) {                           // uniform over the warp
-                        uint32_t v[32];
-                        tmem_ld_32x32b_x32(lane_base + (uint32_t)(o * BN + c0), v);
-                        if (EPI == kEpiSiluMul) {
-                            uint32_t u[32];
-                            tmem_ld_32x32b_x32(lane_base + (uint32_t)(BN + c0), u);
-                            tmem_wait_ld();
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(silu_f(__uint_as_float(v[j])) * __uint_as_float(u[j]));
-                        } else {
-                            tmem_wait_ld();
-                        }
-#pragma unroll
-                        for (int j = 0; j < 16; ++j)
-                            packed[o][c][j] = as_u32(__floats2half2_rn(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1])));
-                    }
-                }
-            }
-            // the accumulators are in registers: the next tile may overwrite them
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(acc_empty);
             const int n = n_tile * 128 + quarter * 32 + lane;             // weight row within the tile set
+            if constexpr (HOLD) {
+                uint32_t packed[NOUT][CH][16];
 #pragma unroll
-            for (int o = 0; o < NOUT; ++o) {
+                for (int o = 0; o < NOUT; ++o) {
 #pragma unroll
-                for (int c = 0; c < CH; ++c) {
-                    const int c0 = (half * CH + c) * 32;
-                    if (c0 < BN && c0 < rows) {
-                        uint16_t* out = p.out + (size_t)(row0 + c0) * p.ldo + (size_t)o * p.a_col_offset + n;
+                    for (int c = 0; c < CH; ++c) {
+                        const int c0 = (grp * CH + c) * 32;
+                        if (c0 < BN && c0 < rows) read_chunk(o, c0, packed[o][c]);   // uniform over the warp
+                    }
+                }
+                release();
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            if (c0 + 2 * j < rows) out[(size_t)(2 * j) * p.ldo] = (uint16_t)(packed[o][c][j] & 0xFFFFu);
-                            if (c0 + 2 * j + 1 < rows) out[(size_t)(2 * j + 1) * p.ldo] = (uint16_t)(packed[o][c][j] >> 16);
+                for (int o = 0; o < NOUT; ++o) {
+#pragma unroll
+                    for (int c = 0; c < CH; ++c) {
+                        const int c0 = (grp * CH + c) * 32;
+                        if (c0 < BN && c0 < rows) store_chunk(o, c0, row0, rows, n, packed[o][c]);
+                    }
+                }
+            } else {
+                // many chunks: stream them (read, store), release after the last read
+                uint32_t buf[16];
+                bool pending = false;
+                int po = 0, pc0 = 0;
+#pragma unroll
+                for (int o = 0; o < NOUT; ++o) {
+#pragma unroll
+                    for (int c = 0; c < CH; ++c) {
+                        const int c0 = (grp * CH + c) * 32;
+                        if (c0 < BN && c0 < rows) {
+                            if (pending) store_chunk(po, pc0, row0, rows, n, buf);
+                            read_chunk(o, c0, buf);
+                            pending = true;
+                            po = o;
+                            pc0 = c0;
                         }
                     }
                 }
+                release();
+                if (pending) store_chunk(po, pc0, row0, rows, n, buf);
             }
         }
         if (!ok) *abort_flag = 1;

@@ -4,26 +4,28 @@
 // (Sec. 4.3) and lists "mixture-of-experts specifics" among the things its
 // architecture descriptor carries (Sec. 3.1), but gives no algorithm; the
 // steps below are this library's definition (see include/qmm.h):
-//   route  -> stable permutation by (expert, token) -> gather rows ->
+//   route  -> expert offsets + stable permutation by (expert, token) -> gather rows ->
 //   grouped gate/up GEMM with SiLU*mul epilogue -> grouped down GEMM ->
 //   weighted combine in slot order.
 // Nothing synchronises with the host: the token-tile work list of the grouped
 // GEMMs is built on the device from the expert offsets.
 #include "qmm_gemm_kernel.cuh"
 
+#include <stdlib.h>
+
 namespace qmm {
 
 qmm_status make_x_map(CUtensorMap* map, const uint16_t* X, int64_t rows, int64_t K, int64_t ld, int box_rows);
 qmm_status launch_tc_gemm(int fmt, int bn, int na, int epi, const CUtensorMap& map, const GemmParams& p, dim3 grid,
                           cudaStream_t st);
-int pick_token_tile(int64_t rows);
+int pick_expert_tile(int64_t total_rows, int experts);
 dim3 persistent_grid(int bn, int na, int64_t tiles);
 
 // ------------------------------------------------------------ workspace
 
 struct MoeWorkspace {
     size_t status, counts, offsets, num_tiles, tile_expert, tile_row0, tile_rows;
-    size_t topk_idx, topk_w, perm, inv_perm, xp, hbuf, dbuf, total;
+    size_t topk_idx, topk_w, perm, inv_perm, xp, hbuf, dbuf, trace, total;
     int bn, max_tiles;
 };
 
@@ -33,7 +35,7 @@ static MoeWorkspace moe_layout(const qmm_moe_args* a)
 {
     MoeWorkspace w;
     const size_t rows = (size_t)a->T * a->topk;
-    w.bn = pick_token_tile((int64_t)((rows + a->E - 1) / a->E));           // mean rows per expert
+    w.bn = pick_expert_tile((int64_t)rows, a->E);
     w.max_tiles = (int)((rows + w.bn - 1) / w.bn) + a->E;
     size_t o = 0;
     auto take = [&](size_t bytes) { const size_t at = o; o = align_up(o + bytes, 256); return at; };
@@ -51,6 +53,7 @@ static MoeWorkspace moe_layout(const qmm_moe_args* a)
     w.xp = take(rows * (size_t)a->H * 2);
     w.hbuf = take(rows * (size_t)a->I * 2);
     w.dbuf = take(rows * (size_t)a->H * 2);
+    w.trace = take(4096);                                  // pipeline trace of the gate/up GEMM (tuning aid, QMM_GEMM_TRACE)
     w.total = o;
     return w;
 }
@@ -120,64 +123,71 @@ __global__ void route_kernel(const float* __restrict__ logits, int T, int E, int
     }
 }
 
-// One block: exclusive scan of the per-expert counts -> expert_offsets, and the
-// token-tile list of the grouped GEMMs (expert, first row, valid rows).
-__global__ void offsets_kernel(const int* __restrict__ counts, int E, int bn,
-                               int* __restrict__ offsets, int* __restrict__ offsets_user,
-                               int* __restrict__ num_tiles, int* __restrict__ tile_expert,
-                               int* __restrict__ tile_row0, int* __restrict__ tile_rows)
-{
-    pdl_launch_dependents();
-    pdl_wait();
-    __shared__ int s_cnt[1024], s_off[1025], s_toff[1025];
-    const int e = threadIdx.x;
-    s_cnt[e] = e < E ? counts[e] : 0;
-    __syncthreads();
-    if (threadIdx.x == 0) {                               // E <= 1024: a serial scan is a few microseconds
-        int o = 0, t = 0;
-        for (int i = 0; i < E; ++i) {
-            s_off[i] = o;
-            s_toff[i] = t;
-            o += s_cnt[i];
-            t += (s_cnt[i] + bn - 1) / bn;
-        }
-        s_off[E] = o;
-        s_toff[E] = t;
-        *num_tiles = t;
-        offsets[E] = o;
-        if (offsets_user) offsets_user[E] = o;
-    }
-    __syncthreads();
-    if (e < E) {
-        offsets[e] = s_off[e];
-        if (offsets_user) offsets_user[e] = s_off[e];
-    }
-    if (e < E) {
-        const int nt = s_toff[e + 1] - s_toff[e];
-        for (int i = 0; i < nt; ++i) {
-            const int y = s_toff[e] + i;
-            tile_expert[y] = e;
-            tile_row0[y] = s_off[e] + i * bn;
-            tile_rows[y] = min(bn, s_cnt[e] - i * bn);
-        }
-    }
-}
-
-// One block per expert: walks the T*topk (token, slot) pairs in flat order and
-// appends those routed to this expert, which yields the stable order by
+// One block per expert e (1024 threads).  First the block derives what the
+// exclusive scan over the per-expert counts gives expert e -- its first row
+// (expert_offsets[e]) and its first token tile -- by summing the counts of the
+// experts before it, and writes its entries of the token-tile list of the
+// grouped GEMMs.  Then it walks the T*topk (token, slot) pairs in flat order
+// and appends those routed to e, which yields the stable order by
 // (expert, token).  perm[r] = flat index, inv_perm[flat] = r.
-__global__ void permute_kernel(const int* __restrict__ topk_idx, int total, const int* __restrict__ offsets,
-                               int* __restrict__ perm, int* __restrict__ perm_user, int* __restrict__ inv_perm)
+constexpr int kPermuteThreads = 1024;
+
+__global__ void __launch_bounds__(kPermuteThreads)
+permute_kernel(const int* __restrict__ topk_idx, int total, const int* __restrict__ counts, int E, int bn,
+               int* __restrict__ offsets, int* __restrict__ offsets_user, int* __restrict__ num_tiles,
+               int* __restrict__ tile_expert, int* __restrict__ tile_row0, int* __restrict__ tile_rows,
+               int* __restrict__ perm, int* __restrict__ perm_user, int* __restrict__ inv_perm)
 {
     pdl_launch_dependents();
     pdl_wait();
-    __shared__ int s_warp[8];
+    __shared__ int s_warp[kPermuteThreads / 32];
+    __shared__ int s_rows[kPermuteThreads / 32], s_tiles[kPermuteThreads / 32];
     __shared__ int s_base;
     const int e = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (threadIdx.x == 0) s_base = offsets[e];
+
+    // rows and token tiles of the experts before e (E <= 1024: one count per thread)
+    int rows_before = 0, tiles_before = 0;
+    if ((int)threadIdx.x < e) {
+        const int c = counts[threadIdx.x];
+        rows_before = c;
+        tiles_before = (c + bn - 1) / bn;
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        rows_before += __shfl_xor_sync(0xFFFFFFFFu, rows_before, off);
+        tiles_before += __shfl_xor_sync(0xFFFFFFFFu, tiles_before, off);
+    }
+    if (lane == 0) {
+        s_rows[warp] = rows_before;
+        s_tiles[warp] = tiles_before;
+    }
     __syncthreads();
-    for (int start = 0; start < total; start += 256) {
+    if (threadIdx.x == 0) {
+        int r0 = 0, t0 = 0;
+        for (int w = 0; w < kPermuteThreads / 32; ++w) {
+            r0 += s_rows[w];
+            t0 += s_tiles[w];
+        }
+        const int mine = counts[e];
+        const int nt = (mine + bn - 1) / bn;
+        s_base = r0;
+        offsets[e] = r0;
+        if (offsets_user) offsets_user[e] = r0;
+        for (int i = 0; i < nt; ++i) {
+            tile_expert[t0 + i] = e;
+            tile_row0[t0 + i] = r0 + i * bn;
+            tile_rows[t0 + i] = min(bn, mine - i * bn);
+        }
+        if (e == E - 1) {
+            offsets[E] = r0 + mine;
+            if (offsets_user) offsets_user[E] = r0 + mine;
+            *num_tiles = t0 + nt;
+        }
+    }
+    __syncthreads();
+
+    for (int start = 0; start < total; start += kPermuteThreads) {
         const int i = start + threadIdx.x;
         const bool mine = i < total && topk_idx[i] == e;
         const unsigned ballot = __ballot_sync(0xFFFFFFFFu, mine);
@@ -185,9 +195,10 @@ __global__ void permute_kernel(const int* __restrict__ topk_idx, int total, cons
         __syncthreads();
         int before = 0, all = 0;
 #pragma unroll
-        for (int w = 0; w < 8; ++w) {
-            if (w < warp) before += s_warp[w];
-            all += s_warp[w];
+        for (int w = 0; w < kPermuteThreads / 32; ++w) {
+            const int c = s_warp[w];
+            if (w < warp) before += c;
+            all += c;
         }
         if (mine) {
             const int r = s_base + before + __popc(ballot & ((1u << lane) - 1u));
@@ -298,11 +309,9 @@ qmm_status launch_moe(const qmm_moe_args* a, void* ws, bool route_only, cudaStre
                            a->topk_idx, a->topk_w, counts);
         if (e != cudaSuccess) return check_cuda(e, "qmm_moe route launch");
     }
-    // 2. offsets + tile list, stable permutation
-    e = launch_pdl(offsets_kernel, dim3(1), dim3(1024), st, (const int*)counts, (int)a->E, w.bn, offsets, a->expert_offsets,
-                   num_tiles, tile_expert, tile_row0, tile_rows);
-    if (e != cudaSuccess) return check_cuda(e, "qmm_moe offsets launch");
-    e = launch_pdl(permute_kernel, dim3(a->E), dim3(256), st, (const int*)topk_idx, total, (const int*)offsets, perm, a->perm,
+    // 2. expert offsets, token-tile list and stable permutation (one block per expert)
+    e = launch_pdl(permute_kernel, dim3(a->E), dim3(kPermuteThreads), st, (const int*)topk_idx, total, (const int*)counts,
+                   (int)a->E, w.bn, offsets, a->expert_offsets, num_tiles, tile_expert, tile_row0, tile_rows, perm, a->perm,
                    inv_perm);
     if (e != cudaSuccess) return check_cuda(e, "qmm_moe permute launch");
     if (route_only) return QMM_OK;
@@ -334,6 +343,7 @@ qmm_status launch_moe(const qmm_moe_args* a, void* ws, bool route_only, cudaStre
         p.tile_rows = tile_rows;
         p.num_tiles = num_tiles;
         p.status = status;
+        if (getenv("QMM_GEMM_TRACE")) p.trace = (long long*)(base + w.trace);
         s = launch_tc_gemm(a->fmt, w.bn, 2, kEpiSiluMul, map, p, persistent_grid(w.bn, 2, 0), st);
         if (s != QMM_OK) return s;
     }
