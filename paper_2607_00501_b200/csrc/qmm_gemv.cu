@@ -406,6 +406,131 @@ gemv_batch_kernel(const __grid_constant__ BatchParams bp)
     }
 }
 
+// ------------------------------------------------------- MoE decode rows
+//
+// The expert products of a mixture-of-experts layer when only a few tokens are
+// in flight (decode): every permuted row r = (token, expert) is a GEMV against
+// its expert's matrices, found on the device from the routing result.
+//   GATE_UP: unit = (row r, 32 outputs): the warp's row-group pair is
+//            (gate rows, up rows) of the same 32 outputs, so one pass yields
+//            G and U; the block writes h = fp16(silu(G) * U).  x = X[token(r)].
+//   DOWN:    unit = (row r, 64 outputs) of the down matrix.  x = Hm[r].
+struct MoeGemvParams {
+    const uint8_t* w0;          // GATE_UP: gate matrices; DOWN: down matrices (expert-major, packed)
+    const uint8_t* w1;          // GATE_UP: up matrices
+    int64_t expert_stride;      // bytes between experts
+    const uint16_t* x;          // GATE_UP: X [T, K]; DOWN: Hm [rows, K]
+    uint16_t* out;              // GATE_UP: Hm [rows, N]; DOWN: D [rows, N]
+    const int* perm;            // [rows] flat (token, slot) index of permuted row r
+    const int* topk_idx;        // [T*topk]
+    int rows, topk, N, K;       // N, K of one expert matrix
+};
+
+enum { kMoeGateUp = 0, kMoeDown = 1 };
+
+template <int FMT, int MODE, int WARPS>
+__global__ void __launch_bounds__(WARPS * 32, 768 / (WARPS * 32))
+moe_gemv_kernel(const MoeGemvParams p)
+{
+    extern __shared__ uint4 smem[];
+    uint4* xs = smem;
+    uint4* zs = smem + p.K / 8;
+    float* red = reinterpret_cast<float*>(smem + p.K / 4);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr int TB = Fmt<FMT>::tile_bytes;
+    constexpr int XV = Fmt<FMT>::tile_k / 8;
+    constexpr int STEP = kUnroll * WARPS;
+    constexpr int OUT_PER_UNIT = MODE == kMoeGateUp ? 32 : 64;
+    const int tpr = p.K / Fmt<FMT>::tile_k;
+    const int units_per_row = p.N / OUT_PER_UNIT;
+    const int units = p.rows * units_per_row;
+    const size_t group_bytes = (size_t)tpr * TB;
+
+    pdl_launch_dependents();
+    pdl_wait();                                                 // routing result and activations are written upstream
+    for (int i = threadIdx.x; i < p.K / 8; i += WARPS * 32) zs[i] = make_uint4(0u, 0u, 0u, 0u);
+    const uint4* xb = ((lane >> 2) == (lane & 3)) ? xs : zs;
+    Q4Consts kc;
+    kc.init();
+
+    int cur_row = -1;
+    for (int u = blockIdx.x; u < units; u += gridDim.x) {
+        const int r = u / units_per_row, j = u - r * units_per_row;
+        const int flat = p.perm[r];
+        const int e = p.topk_idx[flat];
+        if (r != cur_row) {                                     // stage this row's activation vector
+            __syncthreads();
+            const uint16_t* xr = MODE == kMoeGateUp ? p.x + (size_t)(flat / p.topk) * p.K : p.x + (size_t)r * p.K;
+            for (int i = threadIdx.x; i < p.K / 8; i += WARPS * 32) xs[i] = reinterpret_cast<const uint4*>(xr)[i];
+            __syncthreads();
+            cur_row = r;
+        }
+        const uint8_t *tiles_p, *tiles_q;
+        if (MODE == kMoeGateUp) {
+            tiles_p = p.w0 + (size_t)e * p.expert_stride + (size_t)j * group_bytes + 32 * lane;
+            tiles_q = p.w1 + (size_t)e * p.expert_stride + (size_t)j * group_bytes + 32 * lane;
+        } else {
+            tiles_p = p.w0 + (size_t)e * p.expert_stride + (size_t)(2 * j) * group_bytes + 32 * lane;
+            tiles_q = tiles_p + group_bytes;
+        }
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int t = warp; t < tpr; t += STEP) {
+            TileRegs<FMT> rg;
+#pragma unroll
+            for (int q = 0; q < kUnroll; ++q) {
+                const int tt = t + q * WARPS;
+                if (tt < tpr) {
+                    const uint8_t* tp = tiles_p + (size_t)tt * TB;
+                    const uint8_t* tq = tiles_q + (size_t)tt * TB;
+                    rg.cp[q] = ld_stream_256(tp);
+                    rg.cq[q] = ld_stream_256(tq);
+                    rg.sp[q] = load_scales<FMT>(tp - 32 * lane, lane);
+                    rg.sq[q] = load_scales<FMT>(tq - 32 * lane, lane);
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < kUnroll; ++q) {
+                const int tt = t + q * WARPS;
+                if (tt < tpr) {
+                    if constexpr (FMT == QMM_Q4)
+                        tile_pair_mma_q4(rg.cp[q], rg.cq[q], rg.sp[q], rg.sq[q], xb + tt * XV, acc, kc);
+                    else
+                        tile_pair_mma_q8(rg.cp[q], rg.cq[q], rg.sp[q], rg.sq[q], xb + tt * XV, acc);
+                }
+            }
+        }
+        if ((lane & 3) < 2) {
+            const int row = (lane & ~3) + 2 * (lane & 1);
+            float* w = red + warp * 64;
+            w[row] = acc[0];
+            w[row + 1] = acc[1];
+            w[32 + row] = acc[2];
+            w[32 + row + 1] = acc[3];
+        }
+        __syncthreads();
+        if (MODE == kMoeGateUp) {
+            if (threadIdx.x < 32) {                             // red[.. 0..31] = G, red[.. 32..63] = U
+                float g = red[threadIdx.x], up = red[32 + threadIdx.x];
+#pragma unroll
+                for (int w = 1; w < WARPS; ++w) {
+                    g += red[w * 64 + threadIdx.x];
+                    up += red[w * 64 + 32 + threadIdx.x];
+                }
+                const float h = (g / (1.0f + expf(-g))) * up;
+                p.out[(size_t)r * p.N + j * 32 + threadIdx.x] = __half_as_ushort(__float2half_rn(h));
+            }
+        } else {
+            if (threadIdx.x < 64) {
+                float sum = red[threadIdx.x];
+#pragma unroll
+                for (int w = 1; w < WARPS; ++w) sum += red[w * 64 + threadIdx.x];
+                p.out[(size_t)r * p.N + j * 64 + threadIdx.x] = __half_as_ushort(__float2half_rn(sum));
+            }
+        }
+        __syncthreads();
+    }
+}
+
 // Second stage of split-K: y[n] = fp16(sum_s partial[s][n]), s ascending.
 __global__ void gemv_reduce_kernel(const float* __restrict__ partial, uint16_t* __restrict__ y, int N, int splits)
 {
@@ -500,6 +625,42 @@ static qmm_status launch_gemv_t(const GemvPlan& p, const void* packed, int64_t N
         if (e != cudaSuccess) return check_cuda(e, "qmm_gemv reduce launch");
     }
     return QMM_OK;
+}
+
+// Expert products of the MoE layer for a handful of rows (decode): see moe_gemv_kernel.
+qmm_status launch_moe_gemv(int fmt, bool gate_up, const void* w0, const void* w1, int64_t expert_stride,
+                           const uint16_t* x, uint16_t* out, const int* perm, const int* topk_idx,
+                           int rows, int topk, int N, int K, cudaStream_t st)
+{
+    constexpr int WARPS = 8;
+    MoeGemvParams p;
+    p.w0 = (const uint8_t*)w0;
+    p.w1 = (const uint8_t*)w1;
+    p.expert_stride = expert_stride;
+    p.x = x;
+    p.out = out;
+    p.perm = perm;
+    p.topk_idx = topk_idx;
+    p.rows = rows;
+    p.topk = topk;
+    p.N = N;
+    p.K = K;
+    const size_t smem = (size_t)K * 4 + (size_t)WARPS * 64 * sizeof(float);
+    const int units = rows * (N / (gate_up ? 32 : 64));
+    const int grid = units < kNumSMs * 3 ? units : kNumSMs * 3;
+    cudaError_t e = cudaSuccess;
+#define QMM_MOE_GEMV(F, M)                                                                                        \
+    {                                                                                                             \
+        auto kern = moe_gemv_kernel<F, M, WARPS>;                                                                 \
+        if (smem > 48 * 1024) e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+        if (e == cudaSuccess) e = launch_pdl(kern, dim3(grid), dim3(WARPS * 32), smem, st, p);                    \
+    }
+    if (fmt == QMM_Q4 && gate_up) QMM_MOE_GEMV(QMM_Q4, kMoeGateUp)
+    else if (fmt == QMM_Q4) QMM_MOE_GEMV(QMM_Q4, kMoeDown)
+    else if (gate_up) QMM_MOE_GEMV(QMM_Q8, kMoeGateUp)
+    else QMM_MOE_GEMV(QMM_Q8, kMoeDown)
+#undef QMM_MOE_GEMV
+    return check_cuda(e, "qmm_moe decode GEMV launch");
 }
 
 // Host side of qmm_gemv_batch: up to kMaxBatch problems per launch.

@@ -19,6 +19,13 @@ qmm_status make_x_map(CUtensorMap* map, const uint16_t* X, int64_t rows, int64_t
 qmm_status launch_tc_gemm(int fmt, int bn, int na, int epi, const CUtensorMap& map, const GemmParams& p, dim3 grid,
                           cudaStream_t st);
 int pick_expert_tile(int64_t total_rows, int experts);
+qmm_status launch_moe_gemv(int fmt, bool gate_up, const void* w0, const void* w1, int64_t expert_stride,
+                           const uint16_t* x, uint16_t* out, const int* perm, const int* topk_idx,
+                           int rows, int topk, int N, int K, cudaStream_t st);
+
+// Up to this many (token, expert) rows the expert products run as GEMVs (each row streams its expert's
+// matrices once); above it, as grouped tensor-core GEMMs (each expert's matrices are read once per layer).
+constexpr int kMoeGemvMaxRows = 32;
 dim3 persistent_grid(int bn, int na, int64_t tiles);
 
 // ------------------------------------------------------------ workspace
@@ -62,19 +69,13 @@ size_t moe_workspace_bytes(const qmm_moe_args* a) { return moe_layout(a).total; 
 
 // ---------------------------------------------------------------- route
 
-// One warp per token.  topk passes; each pass takes the largest remaining
-// logit, equal logits going to the lower expert index.  The weights are the
-// softmax over the selected logits in fp32.  Also counts rows per expert.
+// Routing of one token by one warp.  topk passes; each pass takes the largest
+// remaining logit, equal logits going to the lower expert index.  The weights
+// are the softmax over the selected logits in fp32.  On return lane j < topk
+// holds the j-th selected expert and its weight.
 template <int MAX_PER_LANE>
-__global__ void route_kernel(const float* __restrict__ logits, int T, int E, int topk,
-                             int* __restrict__ idx_out, float* __restrict__ w_out,
-                             int* __restrict__ idx_user, float* __restrict__ w_user, int* __restrict__ counts)
+__device__ __forceinline__ void route_token(const float* __restrict__ l, int E, int topk, int lane, int& sel_idx, float& sel_w)
 {
-    pdl_launch_dependents();
-    pdl_wait();
-    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-    if (warp >= T) return;
-    const float* l = logits + (size_t)warp * E;
     float v[MAX_PER_LANE];
 #pragma unroll
     for (int i = 0; i < MAX_PER_LANE; ++i) {
@@ -83,7 +84,7 @@ __global__ void route_kernel(const float* __restrict__ logits, int T, int E, int
     }
     unsigned taken = 0;                                   // bit i: v[i] already selected
     float sel_val = 0.f, lmax = 0.f, denom = 0.f;         // lane j keeps the j-th selected logit
-    int sel_idx = 0;
+    sel_idx = 0;
     for (int j = 0; j < topk; ++j) {
         float best = -INFINITY;
         int best_e = 0x7FFFFFFF;
@@ -112,14 +113,78 @@ __global__ void route_kernel(const float* __restrict__ logits, int T, int E, int
         }
         denom += expf(best - lmax);                       // same value and order on every lane
     }
+    sel_w = expf(sel_val - lmax) / denom;
+}
+
+// One warp per token; also counts rows per expert.
+template <int MAX_PER_LANE>
+__global__ void route_kernel(const float* __restrict__ logits, int T, int E, int topk,
+                             int* __restrict__ idx_out, float* __restrict__ w_out,
+                             int* __restrict__ idx_user, float* __restrict__ w_user, int* __restrict__ counts)
+{
+    pdl_launch_dependents();
+    pdl_wait();
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (warp >= T) return;
+    int sel_idx;
+    float w;
+    route_token<MAX_PER_LANE>(logits + (size_t)warp * E, E, topk, lane, sel_idx, w);
     if (lane < topk) {
-        const float w = expf(sel_val - lmax) / denom;
         const size_t o = (size_t)warp * topk + lane;
         idx_out[o] = sel_idx;
         w_out[o] = w;
         if (idx_user) idx_user[o] = sel_idx;
         if (w_user) w_user[o] = w;
         atomicAdd(&counts[sel_idx], 1);                   // a count: the order of the adds does not matter
+    }
+}
+
+// Decode-sized layers (T * topk <= 32): routing, expert offsets and the stable
+// permutation in ONE block, so that the layer is four dependent launches.
+// Warp t routes token t; then one warp ranks the <= 32 (token, slot) pairs by
+// (expert, flat index) and every thread e derives expert_offsets[e].
+template <int MAX_PER_LANE>
+__global__ void __launch_bounds__(1024)
+route_small_kernel(const float* __restrict__ logits, int T, int E, int topk,
+                   int* __restrict__ idx_out, float* __restrict__ w_out, int* __restrict__ idx_user, float* __restrict__ w_user,
+                   int* __restrict__ offsets, int* __restrict__ offsets_user,
+                   int* __restrict__ perm, int* __restrict__ perm_user, int* __restrict__ inv_perm)
+{
+    pdl_launch_dependents();
+    pdl_wait();
+    __shared__ int s_e[32];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int total = T * topk;
+    if (warp < T) {
+        int sel_idx;
+        float w;
+        route_token<MAX_PER_LANE>(logits + (size_t)warp * E, E, topk, lane, sel_idx, w);
+        if (lane < topk) {
+            const int o = warp * topk + lane;
+            idx_out[o] = sel_idx;
+            w_out[o] = w;
+            if (idx_user) idx_user[o] = sel_idx;
+            if (w_user) w_user[o] = w;
+            s_e[o] = sel_idx;
+        }
+    }
+    __syncthreads();
+    if (warp == 0 && lane < total) {                       // rank of pair `lane` in the (expert, flat index) order
+        const int mine = s_e[lane];
+        int r = 0;
+        for (int j = 0; j < total; ++j) {
+            const int other = s_e[j];
+            r += (other < mine || (other == mine && j < lane)) ? 1 : 0;
+        }
+        perm[r] = lane;
+        if (perm_user) perm_user[r] = lane;
+        inv_perm[lane] = r;
+    }
+    for (int e = threadIdx.x; e <= E; e += blockDim.x) {   // rows of the experts before e
+        int c = 0;
+        for (int j = 0; j < total; ++j) c += s_e[j] < e ? 1 : 0;
+        offsets[e] = c;
+        if (offsets_user) offsets_user[e] = c;
     }
 }
 
@@ -293,14 +358,24 @@ qmm_status launch_moe(const qmm_moe_args* a, void* ws, bool route_only, cudaStre
     uint16_t* dbuf = a->dbg_D ? a->dbg_D : (uint16_t*)(base + w.dbuf);
     const int total = a->T * a->topk;
 
-    cudaError_t e = cudaMemsetAsync(counts, 0, (size_t)a->E * 4, st);
-    if (e != cudaSuccess) return check_cuda(e, "qmm_moe clear counts");
-
-    // 1. routing
-    {
+    cudaError_t e;
+    const int per_lane = (a->E + 31) / 32;
+    // decode-sized: one block does steps 1-2 and the expert products run as GEMVs
+    const bool small = total <= kMoeGemvMaxRows && a->T <= 32 && a->H <= 32768 && a->I <= 32768;
+    if (small) {
+        if (per_lane <= 4)
+            e = launch_pdl(route_small_kernel<4>, dim3(1), dim3(1024), st, a->logits, (int)a->T, (int)a->E, (int)a->topk, topk_idx,
+                           topk_w, a->topk_idx, a->topk_w, offsets, a->expert_offsets, perm, a->perm, inv_perm);
+        else
+            e = launch_pdl(route_small_kernel<32>, dim3(1), dim3(1024), st, a->logits, (int)a->T, (int)a->E, (int)a->topk, topk_idx,
+                           topk_w, a->topk_idx, a->topk_w, offsets, a->expert_offsets, perm, a->perm, inv_perm);
+        if (e != cudaSuccess) return check_cuda(e, "qmm_moe route launch");
+    } else {
+        e = cudaMemsetAsync(counts, 0, (size_t)a->E * 4, st);
+        if (e != cudaSuccess) return check_cuda(e, "qmm_moe clear counts");
+        // 1. routing
         const int warps_per_block = 8;
         const dim3 grid((a->T + warps_per_block - 1) / warps_per_block), block(warps_per_block * 32);
-        const int per_lane = (a->E + 31) / 32;
         if (per_lane <= 4)
             e = launch_pdl(route_kernel<4>, grid, block, st, a->logits, (int)a->T, (int)a->E, (int)a->topk, topk_idx, topk_w,
                            a->topk_idx, a->topk_w, counts);
@@ -308,13 +383,30 @@ qmm_status launch_moe(const qmm_moe_args* a, void* ws, bool route_only, cudaStre
             e = launch_pdl(route_kernel<32>, grid, block, st, a->logits, (int)a->T, (int)a->E, (int)a->topk, topk_idx, topk_w,
                            a->topk_idx, a->topk_w, counts);
         if (e != cudaSuccess) return check_cuda(e, "qmm_moe route launch");
+        // 2. expert offsets, token-tile list and stable permutation (one block per expert)
+        e = launch_pdl(permute_kernel, dim3(a->E), dim3(kPermuteThreads), st, (const int*)topk_idx, total, (const int*)counts,
+                       (int)a->E, w.bn, offsets, a->expert_offsets, num_tiles, tile_expert, tile_row0, tile_rows, perm, a->perm,
+                       inv_perm);
+        if (e != cudaSuccess) return check_cuda(e, "qmm_moe permute launch");
     }
-    // 2. expert offsets, token-tile list and stable permutation (one block per expert)
-    e = launch_pdl(permute_kernel, dim3(a->E), dim3(kPermuteThreads), st, (const int*)topk_idx, total, (const int*)counts,
-                   (int)a->E, w.bn, offsets, a->expert_offsets, num_tiles, tile_expert, tile_row0, tile_rows, perm, a->perm,
-                   inv_perm);
-    if (e != cudaSuccess) return check_cuda(e, "qmm_moe permute launch");
     if (route_only) return QMM_OK;
+
+    const size_t gu_stride = (size_t)(a->I / kRowsPerGroup) * (size_t)(a->H / tile_k_of(a->fmt)) * tile_bytes_of(a->fmt);
+    const size_t dn_stride = (size_t)(a->H / kRowsPerGroup) * (size_t)(a->I / tile_k_of(a->fmt)) * tile_bytes_of(a->fmt);
+
+    if (small) {
+        // decode: a few rows -> GEMV path (gate/up with SiLU*mul, down), then the combine
+        qmm_status s = launch_moe_gemv(a->fmt, true, a->w_gate, a->w_up, (int64_t)gu_stride, a->X, hbuf, perm, topk_idx, total,
+                                       (int)a->topk, (int)a->I, (int)a->H, st);
+        if (s != QMM_OK) return s;
+        s = launch_moe_gemv(a->fmt, false, a->w_down, nullptr, (int64_t)dn_stride, hbuf, dbuf, perm, topk_idx, total,
+                            (int)a->topk, (int)a->H, (int)a->I, st);
+        if (s != QMM_OK) return s;
+        e = launch_pdl(combine_kernel, dim3(a->T), dim3(256), st, (const uint16_t*)dbuf, (const int*)inv_perm,
+                       (const float*)topk_w, (int)a->topk, (int)a->H, a->out);
+        if (e != cudaSuccess) return check_cuda(e, "qmm_moe combine launch");
+        return QMM_OK;
+    }
 
     // 3. gather rows into expert order
     e = launch_pdl(gather_rows_kernel, dim3((total + 7) / 8), dim3(256), st, a->X, (const int*)perm, total, (int)a->topk,
@@ -322,8 +414,6 @@ qmm_status launch_moe(const qmm_moe_args* a, void* ws, bool route_only, cudaStre
     if (e != cudaSuccess) return check_cuda(e, "qmm_moe gather launch");
 
     // 4. grouped gate/up GEMM with SiLU*mul epilogue -> Hm [total, I]
-    const size_t gu_stride = (size_t)(a->I / kRowsPerGroup) * (size_t)(a->H / tile_k_of(a->fmt)) * tile_bytes_of(a->fmt);
-    const size_t dn_stride = (size_t)(a->H / kRowsPerGroup) * (size_t)(a->I / tile_k_of(a->fmt)) * tile_bytes_of(a->fmt);
     {
         CUtensorMap map;
         qmm_status s = make_x_map(&map, xp, total, a->H, a->H, w.bn);
