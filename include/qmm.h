@@ -28,7 +28,9 @@
  *   - Supported shapes: K a multiple of 256, N a multiple of 128, M >= 1
  *     (M = 0 / T = 0 is accepted and does nothing).  Other shapes return
  *     QMM_ERR_UNSUPPORTED.  There is no CPU fallback and no other GPU target.
- *   - Device pointers must be 16-byte aligned.
+ *   - Device pointers must be 16-byte aligned; packed weight buffers 32-byte.
+ *   - Workspaces of qmm_gemm and qmm_moe start with a status word: zero-fill a
+ *     workspace once after allocating it.
  *
  * Canonical block format (what qmm_pack reads)
  *   Q4 block, 18 bytes: uint16 d (fp16 bits, little endian), uint8 qs[16];
