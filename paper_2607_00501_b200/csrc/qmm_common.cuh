@@ -156,18 +156,6 @@ __device__ __forceinline__ void q8_word_to_h2(uint32_t w, __half2 (&q)[2])
     q[1] = __hsub2(as_h2(__byte_perm(w, 0x64646464u, 0x4342)), c1152);
 }
 
-// acc += q * x with fp16 inputs widened exactly and one fp32 rounding.
-__device__ __forceinline__ void fma_f16_f32(float& acc, __half a, __half b)
-{
-    asm("fma.rn.f32.f16 %0, %1, %2, %0;" : "+f"(acc) : "h"(__half_as_ushort(a)), "h"(__half_as_ushort(b)));
-}
-
-__device__ __forceinline__ void dot2_f32(float& acc0, float& acc1, __half2 q, __half2 x)
-{
-    fma_f16_f32(acc0, __low2half(q), __low2half(x));
-    fma_f16_f32(acc1, __high2half(q), __high2half(x));
-}
-
 // Programmatic dependent launch: let the next kernel in the stream start its
 // prologue now / wait until the previous kernel's writes are visible.
 __device__ __forceinline__ void pdl_launch_dependents()

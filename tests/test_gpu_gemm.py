@@ -70,6 +70,19 @@ def test_gemm_strided_inputs_and_guard_bytes(qmm, oracle):
     assert torch.all(Ybuf[0] == 5.0) and torch.all(Ybuf[M + 1] == 5.0) and torch.all(Ybuf[:, N:] == 5.0)
 
 
+def test_status_word_is_decoded_and_cleared(qmm):
+    # the kernels write QMM_ERR_DEVICE_TIMEOUT (7) into the workspace's status word when a bounded wait
+    # gives up; here the word is set by hand to check the host side: report once, then clear
+    ws = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    qmm.status_check(ws)
+    ws.view(torch.int32)[0] = 7
+    with pytest.raises(qmm.QmmError) as ei:
+        qmm.status_check(ws)
+    assert ei.value.status == 7 and "bounded wait" in ei.value.message
+    qmm.status_check(ws)
+    assert int(ws.view(torch.int32)[0]) == 0
+
+
 def test_gemm_matches_gemv_rows(qmm):
     # the M = 1 product through both kernels agrees to fp16 rounding of nearly equal fp32 sums
     N, K = 384, 1024

@@ -62,6 +62,7 @@ def test_null_and_misaligned_pointers(L):
     assert L.qmm_gemv(4, a, 128, 256, a + 2, a, None, 0, None) == 3
     assert L.qmm_gemv(4, a + 16, 128, 256, a, a, None, 0, None) == 3
     assert "aligned" in qmm.last_error()
+    assert L.qmm_gemv(4, a, 128, 65536, a, a, None, 0, None) == 5                  # K beyond the GEMV's shared-memory staging
     assert L.qmm_gemm(4, a, 128, 256, a, 255, a, 128, 4, a, 1 << 20, None) == 2     # ldx < K
     assert L.qmm_gemm(4, a, 128, 256, a, 260, a, 128, 4, a, 1 << 20, None) == 3     # ldx % 8
     assert L.qmm_gemm(4, a, 128, 256, a, 256, a, 128, -1, a, 1 << 20, None) == 1

@@ -395,3 +395,41 @@ def test_moe_tokens_subset_equals_full(oracle):
     full = oracle.moe_tokens(Q8, lg, X, gate, up, down, H, I, E, k, np.arange(T))
     sub = oracle.moe_tokens(Q8, lg, X, gate, up, down, H, I, E, k, np.array([4, 1]))
     assert np.array_equal(sub, full[[4, 1]])
+
+
+# ------------------------------------------------------- property tests
+
+from hypothesis import assume, given, settings, strategies as st  # noqa: E402
+
+
+@settings(max_examples=60, deadline=None)
+@given(st.lists(st.floats(min_value=-4.0, max_value=4.0, allow_nan=False, width=32), min_size=32, max_size=32),
+       st.sampled_from([Q4, Q8]))
+def test_property_quantise_block_roundtrip(oracle, vals, fmt):
+    w = np.array(vals, dtype=np.float32).reshape(1, 32)
+    blk = oracle.quantize(fmt, w)
+    assert np.array_equal(blk, synth.quantize(fmt, w))               # both quantisers, any block
+    assume(np.abs(w).max() >= 1e-2)                                  # half-step bound: scales in fp16's normal range
+    d = float(npref.scales_bits(fmt, blk, 1, 32).view(np.float16)[0, 0])
+    wq = oracle.dequant(fmt, blk, 1, 32).astype(np.float64)
+    assert np.all(np.abs(w.astype(np.float64) - wq) <= d / 2 * (1 + 2.0**-10) + 1e-30)
+    assert np.array_equal(wq, npref.decode(fmt, blk, 1, 32))
+
+
+@settings(max_examples=40, deadline=None)
+@given(st.integers(1, 9), st.integers(2, 12), st.integers(0, 2**31 - 1))
+def test_property_routing_and_permutation(oracle, T, E, seed):
+    rng = np.random.default_rng(seed)
+    k = int(rng.integers(1, E + 1))
+    lg = rng.integers(-3, 4, size=(T, E)).astype(np.float32)          # small integers: many ties
+    idx, p = oracle.route(lg, k)
+    for t in range(T):
+        order = sorted(range(E), key=lambda e: (-float(lg[t, e]), e))[:k]
+        assert idx[t].tolist() == order
+        assert abs(p[t].sum() - 1.0) < 1e-12
+    perm, offs = oracle.permute(idx, E)
+    flat = idx.reshape(-1)
+    assert sorted(perm.tolist()) == list(range(T * k))
+    keys = [(int(flat[i]), int(i)) for i in perm]
+    assert keys == sorted(keys)
+    assert offs.tolist() == [int((flat < e).sum()) for e in range(E + 1)]
