@@ -433,7 +433,7 @@ def extra_sections(args, qmm, torch, pk, ops, fmts):
         for M in c["Ms"]:
             X = dev(synth.activations(c["seed"], 10 + M, M, K))
             Y = torch.empty((M, N), dtype=torch.float16, device="cuda")
-            ws = torch.zeros(256, dtype=torch.uint8, device="cuda")
+            ws = torch.zeros(qmm.gemm_workspace_bytes(c["fmt"], M, N, K), dtype=torch.uint8, device="cuda")
             fn = lambda: qmm.gemm(c["fmt"], packed, N, K, X, Y=Y, ws=ws)
             fn()
             med, best = time_op(torch, fn, 10, flush)
@@ -560,7 +560,7 @@ def run_case(args):
         packed = qmm.pack(c["fmt"], dev(synth.quantize(c["fmt"], synth.weights(c["seed"], 0, N, K))), N, K)
         X = dev(synth.activations(c["seed"], 10 + M, M, K))
         Y = torch.empty((M, N), dtype=torch.float16, device="cuda")
-        ws = torch.zeros(256, dtype=torch.uint8, device="cuda")
+        ws = torch.zeros(qmm.gemm_workspace_bytes(c["fmt"], M, N, K), dtype=torch.uint8, device="cuda")
         for _ in range(reps):
             qmm.gemm(c["fmt"], packed, N, K, X, Y=Y, ws=ws)
         qmm.status_check(ws)

@@ -121,24 +121,88 @@ int pick_expert_tile(int64_t total_rows, int experts)
     return want <= 32 ? 32 : want <= 64 ? 64 : want <= 128 ? 128 : 160;
 }
 
-// The workspace of qmm_gemm holds only the device status word.
-size_t gemm_workspace_bytes(int, int64_t, int64_t, int64_t) { return 256; }
+// Second stage of the split-K GEMM: Y[m][n] = fp16(sum_s partial[s][m][n]), s ascending (fixed order).
+__global__ void gemm_splitk_reduce_kernel(const float* __restrict__ partial, uint16_t* __restrict__ Y, int M, int N,
+                                          int64_t ldy, int splits)
+{
+    pdl_launch_dependents();
+    pdl_wait();
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;      // one thread: 8 consecutive n of one m
+    const int per_row = N / 8;
+    if (i >= (int64_t)M * per_row) return;
+    const int m = (int)(i / per_row), n = (int)(i % per_row) * 8;
+    float acc[8];
+    const float4* src = reinterpret_cast<const float4*>(partial + (size_t)m * N + n);
+    float4 a = src[0], b = src[1];
+    acc[0] = a.x; acc[1] = a.y; acc[2] = a.z; acc[3] = a.w;
+    acc[4] = b.x; acc[5] = b.y; acc[6] = b.z; acc[7] = b.w;
+    for (int s = 1; s < splits; ++s) {
+        src = reinterpret_cast<const float4*>(partial + ((size_t)s * M + m) * N + n);
+        a = src[0];
+        b = src[1];
+        acc[0] += a.x; acc[1] += a.y; acc[2] += a.z; acc[3] += a.w;
+        acc[4] += b.x; acc[5] += b.y; acc[6] += b.z; acc[7] += b.w;
+    }
+    uint4 o;
+    __half2* oh = reinterpret_cast<__half2*>(&o);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) oh[j] = __floats2half2_rn(acc[2 * j], acc[2 * j + 1]);
+    uint16_t* dst = Y + (size_t)m * ldy + n;
+    if ((reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
+        *reinterpret_cast<uint4*>(dst) = o;
+    } else {                                                              // a row pitch that is not a multiple of 8
+        const uint16_t* oh16 = reinterpret_cast<const uint16_t*>(&o);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) dst[j] = oh16[j];
+    }
+}
+
+// Shape -> tiling of the dense GEMM.
+struct GemmPlan {
+    int bn, na, splits;
+};
+
+// Token tile: 256 (the widest MMA, N = 256) once M exceeds one 128-token tile; one weight tile per
+// block.  When the tiles cannot cover the SMs, the K range is split across blocks (fp32 partial
+// sums in the workspace, a second stage adds them in a fixed order), as long as every split keeps
+// at least 8 k-blocks and an even number of them.
+static GemmPlan gemm_plan(int64_t M, int64_t N, int64_t K)
+{
+    GemmPlan p;
+    p.bn = M > 128 ? 256 : pick_token_tile(M);
+    p.na = 1;
+    p.splits = 1;
+    const int64_t tiles = (N / 128) * ((M + p.bn - 1) / p.bn);
+    const int num_kb = (int)(K / kGemmBK);
+    while (tiles * p.splits * 2 <= kNumSMs && num_kb % (p.splits * 2) == 0 && num_kb / (p.splits * 2) >= 8 &&
+           (num_kb / (p.splits * 2)) % 2 == 0)
+        p.splits *= 2;
+    if (const char* f = getenv("QMM_GEMM_FORCE")) {            // "bn,na[,splits]" for tuning sweeps and tests
+        int b = 0, a = 0, sp = 1;
+        const int got = sscanf(f, "%d,%d,%d", &b, &a, &sp);
+        if (got >= 2 && (a == 1 || (a == 2 && N % 256 == 0 && b <= 128)) &&
+            (b == 32 || b == 64 || b == 128 || (b == 256 && a == 1))) {
+            p.bn = b;
+            p.na = a;
+            p.splits = 1;
+            if (got == 3 && sp >= 1 && num_kb % sp == 0 && (num_kb / sp) % 2 == 0) p.splits = sp;
+        }
+    }
+    return p;
+}
+
+// Workspace of qmm_gemm: the device status word, then the split-K partial sums.
+size_t gemm_workspace_bytes(int, int64_t M, int64_t N, int64_t K)
+{
+    const GemmPlan p = gemm_plan(M, N, K);
+    return 256 + (p.splits > 1 ? (size_t)p.splits * (size_t)M * (size_t)N * sizeof(float) : 0);
+}
 
 qmm_status launch_gemm(int fmt, const void* packed, int64_t N, int64_t K, const uint16_t* X, int64_t ldx,
                        uint16_t* Y, int64_t ldy, int64_t M, void* ws, cudaStream_t st)
 {
-    // Token tile: 256 (the widest MMA, N = 256) once M exceeds one 128-token tile; one weight tile
-    // per block, so that small problems spread over as many SMs as possible.
-    int bn = M > 128 ? 256 : pick_token_tile(M);
-    int na = 1;
-    if (const char* f = getenv("QMM_GEMM_FORCE")) {            // "bn,na" for tuning sweeps
-        int b = 0, a = 0;
-        if (sscanf(f, "%d,%d", &b, &a) == 2 && (a == 1 || (a == 2 && N % 256 == 0 && b <= 128)) &&
-            (b == 32 || b == 64 || b == 128 || (b == 256 && a == 1))) {
-            bn = b;
-            na = a;
-        }
-    }
+    const GemmPlan plan = gemm_plan(M, N, K);
+    const int bn = plan.bn, na = plan.na;
     CUtensorMap map;
     qmm_status s = make_x_map(&map, X, M, K, ldx, bn);
     if (s != QMM_OK) return s;
@@ -150,13 +214,30 @@ qmm_status launch_gemm(int fmt, const void* packed, int64_t N, int64_t K, const 
     p.N = (int)N;
     p.K = (int)K;
     p.out = Y;
-    p.ldo = ldy;
+    p.ldo = plan.splits > 1 ? N : ldy;                                    // partial sums are [split][M][N], dense
     p.a_col_offset = (int)(N / 2);
     p.M = (int)M;
+    p.splits = plan.splits;
+    p.partial = plan.splits > 1 ? (float*)((uint8_t*)ws + 256) : nullptr;
     p.status = (int*)ws;
-    if (getenv("QMM_GEMM_TRACE")) p.trace = (long long*)((uint8_t*)ws + 256);   // tuning aid: needs a workspace of >= 256 + 4096 bytes
-    const int64_t tiles = (N / (128 * na)) * ((M + bn - 1) / bn);
-    return launch_tc_gemm(fmt, bn, na, kEpiStore, map, p, persistent_grid(bn, na, tiles), st);
+    if (getenv("QMM_GEMM_TRACE") && plan.splits == 1)
+        p.trace = (long long*)((uint8_t*)ws + 256);                       // tuning aid: needs a workspace of >= 256 + 4096 bytes
+    const int64_t tiles = (N / (128 * na)) * ((M + bn - 1) / bn) * plan.splits;
+    s = launch_tc_gemm(fmt, bn, na, kEpiStore, map, p, persistent_grid(bn, na, tiles), st);
+    if (s != QMM_OK || plan.splits == 1) return s;
+    cudaLaunchConfig_t cfg = {};
+    const int64_t threads = M * (N / 8);
+    cfg.gridDim = dim3((unsigned)((threads + 255) / 256));
+    cfg.blockDim = dim3(256);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return check_cuda(cudaLaunchKernelEx(&cfg, gemm_splitk_reduce_kernel, (const float*)p.partial, Y, (int)M, (int)N,
+                                         (int64_t)ldy, plan.splits),
+                      "qmm_gemm split-K reduce launch");
 }
 
 // Reads and clears the device status word (first int of a GEMM / MoE workspace).

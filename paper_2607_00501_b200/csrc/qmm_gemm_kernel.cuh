@@ -61,6 +61,8 @@ struct GemmParams {
     const int* tile_row0;            // [max_tiles] first permuted row of the tile
     const int* tile_rows;            // [max_tiles] valid rows in the tile (<= BN)
     const int* num_tiles;            // [1]
+    int splits;                      // K splits (dense only, >= 1): > 1 -> fp32 partial sums go to `partial`
+    float* partial;                  // [splits][M][N-wide rows] fp32, when splits > 1
     int* status;                     // device status word (0 = ok)
     long long* trace;                // optional [block 0 only] clock64 samples for pipeline analysis (tuning aid), else null
 };
@@ -186,8 +188,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
     // plain store: the NA tile sets split the rows of one matrix; SiLU*mul: they are two matrices of N rows each
     const int n_tiles = (EPI == kEpiSiluMul) ? p.N / 128 : p.N / (128 * NA);
     const int m_tiles = grouped ? *p.num_tiles : (p.M + BN - 1) / BN;
-    const int total_tiles = n_tiles * m_tiles;
-    const int num_kb = p.K / kGemmBK;
+    const int splits = grouped || p.splits < 1 ? 1 : p.splits;           // K splits: a tile is (token tile, weight tile, split)
+    const int total_tiles = n_tiles * m_tiles * splits;
+    const int num_kb = p.K / kGemmBK / splits;                            // k-blocks per tile
 
     // ---- set-up
     if (threadIdx.x == 0) {
@@ -213,7 +216,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
     pdl_launch_dependents();
 
     // token rows of tile t
-    auto tile_rows = [&](int t, int& n_tile, int& expert, int& row0, int& rows) {
+    auto tile_rows = [&](int t, int& n_tile, int& expert, int& row0, int& rows, int& ks) {
+        ks = t % splits;
+        t /= splits;
         n_tile = t % n_tiles;
         const int mt = t / n_tiles;
         if (grouped) {
@@ -253,10 +258,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         };
         int g0 = 0;                                                       // stage counter at the start of the tile
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, g0 += num_kb) {
-            int n_tile, expert, row0, rows;
-            tile_rows(t, n_tile, expert, row0, rows);
+            int n_tile, expert, row0, rows, ks;
+            tile_rows(t, n_tile, expert, row0, rows, ks);
             const int rg = n_tile * 4 + quarter;                          // row group of 32 rows
-            const uint8_t* wrow = p.w[a] + (size_t)expert * p.w_expert_stride + (size_t)rg * tpr * Fmt<FMT>::tile_bytes;
+            const uint8_t* wrow = p.w[a] + (size_t)expert * p.w_expert_stride + (size_t)rg * tpr * Fmt<FMT>::tile_bytes +
+                                  (size_t)ks * num_kb * kb_bytes;          // this split's part of the row group's stream
             // The weight stream of a row group is contiguous: ask L2 for it kGemmL2Ahead stages ahead
             // (expert weights come from HBM; two register-held slices alone do not cover that latency).
             if (lane == 0 && phase == 0) {
@@ -340,14 +346,36 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             if (lane == 0) mbar_arrive(acc_empty);
         };
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
-            int n_tile, expert, row0, rows;
-            tile_rows(t, n_tile, expert, row0, rows);
+            int n_tile, expert, row0, rows, ks;
+            tile_rows(t, n_tile, expert, row0, rows, ks);
             ok = mbar_wait(acc_full, it & 1, abort_flag);
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
             tc_fence_after_sync();
             const int n = n_tile * 128 + quarter * 32 + lane;             // weight row within the tile set
-            if constexpr (HOLD) {
+            if (splits > 1) {
+                // split-K: fp32 partial sums of this split, [split][token][weight row]; a second kernel adds the splits
+                if constexpr (EPI == kEpiStore) {
+                    float* pbase = p.partial + ((size_t)ks * p.M + row0) * p.ldo + n;
+#pragma unroll
+                    for (int o = 0; o < NOUT; ++o) {
+#pragma unroll
+                        for (int c = 0; c < CH; ++c) {
+                            const int c0 = (grp * CH + c) * 32;
+                            if (c0 < BN && c0 < rows) {
+                                uint32_t v[32];
+                                tmem_ld_32x32b_x32(lane_base + (uint32_t)(o * BN + c0), v);
+                                tmem_wait_ld();
+                                float* dst = pbase + (size_t)c0 * p.ldo + (size_t)o * p.a_col_offset;
+#pragma unroll
+                                for (int j = 0; j < 32; ++j)
+                                    if (c0 + j < rows) dst[(size_t)j * p.ldo] = __uint_as_float(v[j]);
+                            }
+                        }
+                    }
+                }
+                release();
+            } else if constexpr (HOLD) {
                 uint32_t packed[NOUT][CH][16];
 #pragma unroll
                 for (int o = 0; o < NOUT; ++o) {
@@ -397,14 +425,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             int issued = 0, g = 0;
             bool ok = true;
             for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-                int n_tile, expert, row0, rows;
-                tile_rows(t, n_tile, expert, row0, rows);
+                int n_tile, expert, row0, rows, ks;
+                tile_rows(t, n_tile, expert, row0, rows, ks);
                 for (int kb = 0; kb < num_kb; ++kb, ++g) {
                     const int s = g % S;
                     if (g >= S) ok = mbar_wait(&empty[s], ((g / S) - 1) & 1, abort_flag);
                     if (!ok) break;
                     mbar_arrive_expect_tx(&full[s], B_STAGE);
-                    tma_load_2d(smem_b + s * B_STAGE, &x_map, kb * kGemmBK, row0, &full[s]);
+                    tma_load_2d(smem_b + s * B_STAGE, &x_map, (ks * num_kb + kb) * kGemmBK, row0, &full[s]);
                     issued = g + 1;
                 }
             }

@@ -83,6 +83,27 @@ def test_status_word_is_decoded_and_cleared(qmm):
     assert int(ws.view(torch.int32)[0]) == 0
 
 
+@pytest.mark.parametrize("fmt", [Q4, Q8])
+@pytest.mark.parametrize("force,M,N,K", [("128,1,2", 100, 256, 2048), ("32,1,4", 7, 128, 4096), ("256,1,2", 300, 384, 1024),
+                                         (None, 48, 256, 8192), (None, 256, 128, 4096)])
+def test_gemm_split_k(qmm, oracle, monkeypatch, fmt, force, M, N, K):
+    """K range cut across blocks, fp32 partial sums added in a fixed order by a second kernel."""
+    if force is None:
+        monkeypatch.delenv("QMM_GEMM_FORCE", raising=False)
+    else:
+        monkeypatch.setenv("QMM_GEMM_FORCE", force)
+    assert qmm.gemm_workspace_bytes(fmt, M, N, K) > 256           # these shapes do take the split path
+    blocks, _, _ = util.random_blocks(synth, fmt, N, K, seed=M + N + K + fmt, special_scales=False)
+    X = synth.activations(71, M + N + K, M, K)
+    run_gemm(qmm, oracle, fmt, blocks, N, K, X, "split-K gemm M=%d N=%d K=%d fmt=%d" % (M, N, K, fmt))
+    # same bits on every call
+    packed = qmm.pack(fmt, util.dev(blocks), N, K)
+    Xd = util.dev(X)
+    first = qmm.gemm(fmt, packed, N, K, Xd).cpu()
+    for _ in range(3):
+        assert torch.equal(first, qmm.gemm(fmt, packed, N, K, Xd).cpu())
+
+
 def test_gemm_matches_gemv_rows(qmm):
     # the M = 1 product through both kernels agrees to fp16 rounding of nearly equal fp32 sums
     N, K = 384, 1024
