@@ -79,6 +79,8 @@ qmm_status launch_tc_gemm(int fmt, int bn, int na, int epi, const CUtensorMap& m
     QMM_TC_CASE(F, 32, 1, kEpiStore)      \
     QMM_TC_CASE(F, 64, 1, kEpiStore)      \
     QMM_TC_CASE(F, 128, 1, kEpiStore)     \
+    QMM_TC_CASE(F, 160, 1, kEpiStore)     \
+    QMM_TC_CASE(F, 192, 1, kEpiStore)     \
     QMM_TC_CASE(F, 256, 1, kEpiStore)     \
     QMM_TC_CASE(F, 32, 2, kEpiStore)      \
     QMM_TC_CASE(F, 64, 2, kEpiStore)      \
@@ -121,81 +123,116 @@ int pick_expert_tile(int64_t total_rows, int experts)
     return want <= 32 ? 32 : want <= 64 ? 64 : want <= 128 ? 128 : 160;
 }
 
-// Second stage of the split-K GEMM: Y[m][n] = fp16(sum_s partial[s][m][n]), s ascending (fixed order).
-__global__ void gemm_splitk_reduce_kernel(const float* __restrict__ partial, uint16_t* __restrict__ Y, int M, int N,
-                                          int64_t ldy, int splits)
+// Adds the partial sums of the tiles that the dense GEMM cut across blocks, contributors in
+// ascending order (a fixed order: same bits on every call), and stores fp16.  Used when tiles
+// are cut into many pieces (few tiles, long K), where the whole GPU does the sum faster than
+// the last contributor of every tile.  Block (t, y): token columns [8 y, 8 y + 8) of tile t; a
+// thread adds one float4 (4 weight rows of one token) per output tile, so every load is in flight at once.
+__global__ void gemm_cut_reduce_kernel(const float* __restrict__ partial, uint16_t* __restrict__ Y, int64_t ldy, int M,
+                                       int bn, int nout, int a_col_offset, int n_tiles, int KB, int U)
 {
     pdl_launch_dependents();
     pdl_wait();
-    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;      // one thread: 8 consecutive n of one m
-    const int per_row = N / 8;
-    if (i >= (int64_t)M * per_row) return;
-    const int m = (int)(i / per_row), n = (int)(i % per_row) * 8;
-    float acc[8];
-    const float4* src = reinterpret_cast<const float4*>(partial + (size_t)m * N + n);
-    float4 a = src[0], b = src[1];
-    acc[0] = a.x; acc[1] = a.y; acc[2] = a.z; acc[3] = a.w;
-    acc[4] = b.x; acc[5] = b.y; acc[6] = b.z; acc[7] = b.w;
-    for (int s = 1; s < splits; ++s) {
-        src = reinterpret_cast<const float4*>(partial + ((size_t)s * M + m) * N + n);
-        a = src[0];
-        b = src[1];
-        acc[0] += a.x; acc[1] += a.y; acc[2] += a.z; acc[3] += a.w;
-        acc[4] += b.x; acc[5] += b.y; acc[6] += b.z; acc[7] += b.w;
-    }
-    uint4 o;
-    __half2* oh = reinterpret_cast<__half2*>(&o);
-#pragma unroll
-    for (int j = 0; j < 4; ++j) oh[j] = __floats2half2_rn(acc[2 * j], acc[2 * j + 1]);
-    uint16_t* dst = Y + (size_t)m * ldy + n;
-    if ((reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
-        *reinterpret_cast<uint4*>(dst) = o;
-    } else {                                                              // a row pitch that is not a multiple of 8
-        const uint16_t* oh16 = reinterpret_cast<const uint16_t*>(&o);
-#pragma unroll
-        for (int j = 0; j < 8; ++j) dst[j] = oh16[j];
+    const int t = blockIdx.x, c0 = blockIdx.y * 8;
+    const int n_tile = t % n_tiles, row0 = (t / n_tiles) * bn;
+    const int rows = min(bn, M - row0);
+    if (c0 >= rows) return;
+    const long long tb = (long long)t * KB;
+    const int first = (int)(tb / U);
+    const int cn = (int)((tb + KB - 1) / U) - first + 1;
+    if (cn == 1) return;                                                  // a whole tile: stored by the GEMM itself
+    const size_t slot = (size_t)nout * bn * 128;
+    const int r4 = threadIdx.x & 31, j = threadIdx.x >> 5;                 // 4 weight rows, token column
+    if (c0 + j >= rows) return;
+    for (int o = 0; o < nout; ++o) {
+        const size_t off = (size_t)(o * bn + c0 + j) * 128 + r4 * 4;
+        float4 acc = __ldcg(reinterpret_cast<const float4*>(partial + (size_t)(2 * first + 1) * slot + off));
+        for (int c = 1; c < cn; ++c) {
+            const float4 v = __ldcg(reinterpret_cast<const float4*>(partial + (size_t)(2 * (first + c)) * slot + off));
+            acc.x += v.x;
+            acc.y += v.y;
+            acc.z += v.z;
+            acc.w += v.w;
+        }
+        uint2 h;
+        *reinterpret_cast<__half2*>(&h.x) = __floats2half2_rn(acc.x, acc.y);
+        *reinterpret_cast<__half2*>(&h.y) = __floats2half2_rn(acc.z, acc.w);
+        *reinterpret_cast<uint2*>(Y + (size_t)(row0 + c0 + j) * ldy + (size_t)o * a_col_offset + n_tile * 128 + r4 * 4) = h;
     }
 }
 
-// Shape -> tiling of the dense GEMM.
+// Shape -> tiling and work split of the dense GEMM.
 struct GemmPlan {
-    int bn, na, splits;
+    int bn, na;
+    int units;          // (tile, k-block) units per block
+    int grid;           // blocks
+    bool cut;           // some tile is shared between blocks (needs the partial-sum slots)
+    bool reduce_kernel; // cut tiles are summed by a second kernel (else by their last contributor)
 };
 
-// Token tile: 256 (the widest MMA, N = 256) once M exceeds one 128-token tile; one weight tile per
-// block.  When the tiles cannot cover the SMs, the K range is split across blocks (fp32 partial
-// sums in the workspace, a second stage adds them in a fixed order), as long as every split keeps
-// at least 8 k-blocks and an even number of them.
+// Workspace of qmm_gemm: [0, 4) status word, [256, 8192) arrival counters of the cut tiles,
+// [8192, 16384) trace samples (tuning aid), then the partial-sum slots.
+constexpr size_t kGemmWsCounters = 256, kGemmWsTrace = 8192, kGemmWsHeader = 16384;
+static_assert(kGemmWsCounters + (size_t)kNumSMs * 8 * sizeof(int) <= kGemmWsTrace, "counter area");
+
+// Token tile: 256 (the widest MMA, N = 256) once M exceeds one 128-token tile, else the smallest
+// that holds M; one weight tile per block.  The (tile, k-block) units are dealt to the blocks in
+// equal contiguous shares:
+//   tiles <= SMs / 2: every tile is cut into equal pieces, one per block, as many as the SMs can
+//                     take at once; a second kernel adds the pieces;
+//   tiles <  SMs:     whole tiles (cutting gains less than the exposed sum at the end costs);
+//   tiles >= SMs:     one share per SM, whatever tiles it crosses; a block computes its two cut
+//                     tiles first, and the last contributor of a cut tile adds the pieces while
+//                     whole tiles are still being computed.
 static GemmPlan gemm_plan(int64_t M, int64_t N, int64_t K)
 {
     GemmPlan p;
     p.bn = M > 128 ? 256 : pick_token_tile(M);
     p.na = 1;
-    p.splits = 1;
-    const int64_t tiles = (N / 128) * ((M + p.bn - 1) / p.bn);
-    const int num_kb = (int)(K / kGemmBK);
-    while (tiles * p.splits * 2 <= kNumSMs && num_kb % (p.splits * 2) == 0 && num_kb / (p.splits * 2) >= 8 &&
-           (num_kb / (p.splits * 2)) % 2 == 0)
-        p.splits *= 2;
-    if (const char* f = getenv("QMM_GEMM_FORCE")) {            // "bn,na[,splits]" for tuning sweeps and tests
-        int b = 0, a = 0, sp = 1;
-        const int got = sscanf(f, "%d,%d,%d", &b, &a, &sp);
+    int force_units = 0, force_reduce = -1;
+    if (const char* f = getenv("QMM_GEMM_FORCE")) {            // "bn,na[,units[,second kernel 0/1]]" for tuning sweeps and tests
+        int b = 0, a = 0, u = 0, r = -1;
+        const int got = sscanf(f, "%d,%d,%d,%d", &b, &a, &u, &r);
         if (got >= 2 && (a == 1 || (a == 2 && N % 256 == 0 && b <= 128)) &&
-            (b == 32 || b == 64 || b == 128 || (b == 256 && a == 1))) {
+            (b == 32 || b == 64 || b == 128 || ((b == 160 || b == 192 || b == 256) && a == 1))) {
             p.bn = b;
             p.na = a;
-            p.splits = 1;
-            if (got == 3 && sp >= 1 && num_kb % sp == 0 && (num_kb / sp) % 2 == 0) p.splits = sp;
+            if (got >= 3 && u >= 1) force_units = u;
+            if (got >= 4) force_reduce = r != 0;
         }
     }
+    const int64_t tiles = (N / (128 * p.na)) * ((M + p.bn - 1) / p.bn);
+    const int64_t KB = K / kGemmBK;
+    const int64_t total = tiles * KB;
+    int64_t units;
+    p.reduce_kernel = false;
+    if (tiles * 2 <= kNumSMs) {
+        // the largest number of equal pieces per tile that the SMs can take at once, every piece
+        // worth a pipeline fill and an epilogue (>= 8 k-blocks)
+        int64_t pieces = 1;
+        for (int64_t d = 2; d * tiles <= kNumSMs; ++d)
+            if (KB % d == 0 && KB / d >= 8) pieces = d;
+        units = KB / pieces;
+        p.reduce_kernel = true;
+    } else if (tiles < kNumSMs) {
+        units = KB;
+    } else {
+        units = (total + kNumSMs - 1) / kNumSMs;
+    }
+    if (force_units) units = force_units;
+    if (force_reduce >= 0) p.reduce_kernel = force_reduce != 0;
+    p.units = (int)units;
+    p.grid = (int)((total + units - 1) / units);
+    p.cut = units % KB != 0;
+    if (!p.cut) p.reduce_kernel = false;
     return p;
 }
 
-// Workspace of qmm_gemm: the device status word, then the split-K partial sums.
 size_t gemm_workspace_bytes(int, int64_t M, int64_t N, int64_t K)
 {
+    if (M == 0) return kGemmWsHeader;
     const GemmPlan p = gemm_plan(M, N, K);
-    return 256 + (p.splits > 1 ? (size_t)p.splits * (size_t)M * (size_t)N * sizeof(float) : 0);
+    return kGemmWsHeader + (p.cut ? (size_t)2 * p.grid * p.na * p.bn * 128 * sizeof(float) : 0);
 }
 
 qmm_status launch_gemm(int fmt, const void* packed, int64_t N, int64_t K, const uint16_t* X, int64_t ldx,
@@ -203,6 +240,8 @@ qmm_status launch_gemm(int fmt, const void* packed, int64_t N, int64_t K, const 
 {
     const GemmPlan plan = gemm_plan(M, N, K);
     const int bn = plan.bn, na = plan.na;
+    if (plan.grid > kNumSMs && plan.cut && !plan.reduce_kernel)   // (only a forced unit count can ask for this)
+        return fail(QMM_ERR_UNSUPPORTED, "qmm_gemm: %d blocks with cut tiles exceed the counter area", plan.grid);
     CUtensorMap map;
     qmm_status s = make_x_map(&map, X, M, K, ldx, bn);
     if (s != QMM_OK) return s;
@@ -214,20 +253,20 @@ qmm_status launch_gemm(int fmt, const void* packed, int64_t N, int64_t K, const 
     p.N = (int)N;
     p.K = (int)K;
     p.out = Y;
-    p.ldo = plan.splits > 1 ? N : ldy;                                    // partial sums are [split][M][N], dense
+    p.ldo = ldy;
     p.a_col_offset = (int)(N / 2);
     p.M = (int)M;
-    p.splits = plan.splits;
-    p.partial = plan.splits > 1 ? (float*)((uint8_t*)ws + 256) : nullptr;
+    p.units_per_block = plan.units;
+    p.counters = plan.reduce_kernel ? nullptr : (int*)((uint8_t*)ws + kGemmWsCounters);
+    p.partial = (float*)((uint8_t*)ws + kGemmWsHeader);
     p.status = (int*)ws;
-    if (getenv("QMM_GEMM_TRACE") && plan.splits == 1)
-        p.trace = (long long*)((uint8_t*)ws + 256);                       // tuning aid: needs a workspace of >= 256 + 4096 bytes
-    const int64_t tiles = (N / (128 * na)) * ((M + bn - 1) / bn) * plan.splits;
-    s = launch_tc_gemm(fmt, bn, na, kEpiStore, map, p, persistent_grid(bn, na, tiles), st);
-    if (s != QMM_OK || plan.splits == 1) return s;
+    if (getenv("QMM_GEMM_TRACE")) p.trace = (long long*)((uint8_t*)ws + kGemmWsTrace);   // tuning aid
+    s = launch_tc_gemm(fmt, bn, na, kEpiStore, map, p, dim3((unsigned)plan.grid), st);
+    if (s != QMM_OK || !plan.reduce_kernel) return s;
+    const int n_tiles = (int)(N / (128 * na));
+    const int64_t tiles = (int64_t)n_tiles * ((M + bn - 1) / bn);
     cudaLaunchConfig_t cfg = {};
-    const int64_t threads = M * (N / 8);
-    cfg.gridDim = dim3((unsigned)((threads + 255) / 256));
+    cfg.gridDim = dim3((unsigned)tiles, (unsigned)(bn / 8));
     cfg.blockDim = dim3(256);
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -235,9 +274,9 @@ qmm_status launch_gemm(int fmt, const void* packed, int64_t N, int64_t K, const 
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return check_cuda(cudaLaunchKernelEx(&cfg, gemm_splitk_reduce_kernel, (const float*)p.partial, Y, (int)M, (int)N,
-                                         (int64_t)ldy, plan.splits),
-                      "qmm_gemm split-K reduce launch");
+    return check_cuda(cudaLaunchKernelEx(&cfg, gemm_cut_reduce_kernel, (const float*)p.partial, Y, (int64_t)ldy, (int)M, bn, na,
+                                         p.a_col_offset, n_tiles, (int)(K / kGemmBK), plan.units),
+                      "qmm_gemm partial-sum kernel launch");
 }
 
 // Reads and clears the device status word (first int of a GEMM / MoE workspace).

@@ -30,8 +30,8 @@
 // The kernel is persistent: a block loops over tiles and the pipeline runs on
 // across tile boundaries.
 //
-// TMEM columns: [0, NA*BN) fp32 accumulators, then STAGES slots of NA*32
-// columns (64 fp16 k-values per row and weight tile).
+// TMEM columns: one or two accumulator buffers of NA*BN fp32 columns, then
+// STAGES slots of NA*32 columns (64 fp16 k-values per row and weight tile).
 //
 // Every mbarrier wait is bounded; on give-up the block raises an abort flag,
 // records QMM_ERR_DEVICE_TIMEOUT in the status word, stops issuing work, waits
@@ -61,8 +61,13 @@ struct GemmParams {
     const int* tile_row0;            // [max_tiles] first permuted row of the tile
     const int* tile_rows;            // [max_tiles] valid rows in the tile (<= BN)
     const int* num_tiles;            // [1]
-    int splits;                      // K splits (dense only, >= 1): > 1 -> fp32 partial sums go to `partial`
-    float* partial;                  // [splits][M][N-wide rows] fp32, when splits > 1
+    // dense mode, work split by k-blocks ("stream-K"): block b owns the units [b*U, (b+1)*U) of the
+    // tile-major sequence of (tile, k-block) units; a tile cut by a block boundary is summed from the
+    // fp32 partial results of its contributors by whichever of them finishes last, in contributor order
+    int units_per_block;             // U; 0 = whole tiles, t = blockIdx.x, blockIdx.x + gridDim.x, ...
+    float* partial;                  // [2 * gridDim.x] slots of NA*BN*128 floats (U > 0 and some tile is cut)
+    int* counters;                   // [gridDim.x * epilogue warps] arrival counts, zero between launches; null: the
+                                     // contributors only store their partial sums and a second kernel adds them
     int* status;                     // device status word (0 = ok)
     long long* trace;                // optional [block 0 only] clock64 samples for pipeline analysis (tuning aid), else null
 };
@@ -74,8 +79,11 @@ template <int BN, int NA>
 struct GemmGeom {
     static constexpr int kACols = NA * 32;                                 // TMEM columns per weight slot
     static constexpr int kDCols = NA * BN;                                 // accumulator columns
-    static constexpr int kTmemCols = kDCols <= 128 ? 256 : 512;
-    static constexpr int kFit = (kTmemCols - kDCols) / kACols;
+    static constexpr int kTmemCols = 512;                                  // all of it: one block per SM (registers)
+    // two accumulator buffers (the epilogue of one piece overlaps the MMAs of the next) when a ring
+    // of at least four weight slots still fits beside them
+    static constexpr int kAccBufs = (2 * kDCols + 4 * kACols <= kTmemCols) ? 2 : 1;
+    static constexpr int kFit = (kTmemCols - kAccBufs * kDCols) / kACols;
     static constexpr int kStages = kFit < kGemmMaxStages ? kFit : kGemmMaxStages;
     static constexpr int kBStage = BN * kGemmBK * 2;                       // bytes per activation slot
     static constexpr int kSmemBytes = kStages * kBStage + 1024 /*align*/ + 256;
@@ -147,12 +155,22 @@ template <> struct RawRow64<QMM_Q8> {
 constexpr int kGemmPrefetch = 2;     // weight slices in flight per expander thread
 constexpr int kGemmL2Ahead = 12;     // stages of a row group's weight stream requested into L2 ahead of use
 
-// Persistent, warp-specialised kernel.  Every block walks the tile list
-// t = blockIdx.x, blockIdx.x + gridDim.x, ...; tile t = (token tile t / n_tiles,
-// weight tile t % n_tiles), so blocks that run together share activation tiles.
-// The pipeline (stage counter, barrier phases) runs on across tiles: while the
-// epilogue warps drain the accumulators of tile i, the expanders and the TMA
-// producer already fill the ring for tile i+1.
+// One piece of work of a block: k-blocks [kb0, kb1) of one output tile.  `cn` blocks contribute to
+// the tile (block indices first .. first + cn - 1, k ascending); cn == 1: the piece is the whole tile.
+struct GemmWork {
+    int n_tile, expert, row0, rows;
+    int kb0, kb1;
+    int first, cn;
+};
+
+// Persistent, warp-specialised kernel.  Tile t = (token tile t / n_tiles, weight
+// tile t % n_tiles).  Grouped mode: every block walks the tile list t =
+// blockIdx.x, blockIdx.x + gridDim.x, ... so blocks that run together share
+// activation tiles.  Dense mode: every block takes an equal, contiguous share
+// of all (tile, k-block) units, so the SMs finish together whatever the tile
+// count.  The pipeline (stage counter, barrier phases) runs on across pieces:
+// while the epilogue warps drain the accumulators of piece i, the expanders
+// and the TMA producer already fill the ring for piece i+1.
 template <int FMT, int BN, int NA, int EPI>
 __global__ void __launch_bounds__(GemmGeom<BN, NA>::kThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
@@ -167,6 +185,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
     constexpr int A_COLS = G::kACols;
     constexpr int D_COLS = G::kDCols;
     constexpr int TMEM_COLS = G::kTmemCols;
+    constexpr int AB = G::kAccBufs;                   // accumulator buffers: piece i uses buffer i % AB
+    constexpr int RING0 = AB * D_COLS;                // first TMEM column of the weight ring
     static_assert(BN % 32 == 0 && BN >= 32 && BN <= 256, "token tile");
     static_assert(PH >= 1 && NEXP % 4 == 0, "expander warps must cover the four lane quarters");
     constexpr int B_STAGE = BN * kGemmBK * 2;
@@ -177,9 +197,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S * B_STAGE);
     uint64_t* full = bars;                                                // [S] expanders + TMA -> MMA
     uint64_t* empty = bars + S;                                           // [S] MMA -> expanders, TMA
-    uint64_t* acc_full = bars + 2 * S;                                    // MMA -> epilogue
-    uint64_t* acc_empty = bars + 2 * S + 1;                               // epilogue -> MMA
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 2);
+    uint64_t* acc_full = bars + 2 * S;                                    // [2] MMA -> epilogue
+    uint64_t* acc_empty = bars + 2 * S + 2;                               // [2] epilogue -> MMA
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 4);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -188,9 +208,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
     // plain store: the NA tile sets split the rows of one matrix; SiLU*mul: they are two matrices of N rows each
     const int n_tiles = (EPI == kEpiSiluMul) ? p.N / 128 : p.N / (128 * NA);
     const int m_tiles = grouped ? *p.num_tiles : (p.M + BN - 1) / BN;
-    const int splits = grouped || p.splits < 1 ? 1 : p.splits;           // K splits: a tile is (token tile, weight tile, split)
-    const int total_tiles = n_tiles * m_tiles * splits;
-    const int num_kb = p.K / kGemmBK / splits;                            // k-blocks per tile
+    const int total_tiles = n_tiles * m_tiles;
+    const int KB = p.K / kGemmBK;                                         // k-blocks per tile
+    const int U = grouped ? 0 : p.units_per_block;
 
     // ---- set-up
     if (threadIdx.x == 0) {
@@ -198,8 +218,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             mbar_init(&full[s], 4 * NA + 1);                              // the stage's expander warps + the TMA producer
             mbar_init(&empty[s], 1);                                      // one tcgen05.commit
         }
-        mbar_init(acc_full, 1);
-        mbar_init(acc_empty, NEPI);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&acc_full[b], 1);
+            mbar_init(&acc_empty[b], NEPI);
+        }
         *abort_flag = 0;
         fence_barrier_init();
     }
@@ -215,21 +237,48 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
 
     pdl_launch_dependents();
 
-    // token rows of tile t
-    auto tile_rows = [&](int t, int& n_tile, int& expert, int& row0, int& rows, int& ks) {
-        ks = t % splits;
-        t /= splits;
-        n_tile = t % n_tiles;
+    // i-th piece of work of this block (every role walks the same sequence); false past the last
+    auto get_work = [&](int i, GemmWork& w) -> bool {
+        int t;
+        if (U > 0) {
+            const long long u0 = (long long)blockIdx.x * U;
+            const long long u1 = min(u0 + U, (long long)total_tiles * KB);
+            if (u0 >= u1) return false;
+            // Tiles the share touches: first .. last.  Order of work: the cut tile at the head of the
+            // share, the cut tile at its tail, then the whole tiles -- cut tiles are then completed
+            // (by this block or a neighbour) while whole tiles are still being computed.
+            const int t_first = (int)(u0 / KB), t_last = (int)((u1 - 1) / KB);
+            if (i > t_last - t_first) return false;
+            const int hc = u0 > (long long)t_first * KB ? 1 : 0;
+            const int tc = (t_last > t_first && u1 < (long long)(t_last + 1) * KB) ? 1 : 0;
+            if (hc && i == 0) t = t_first;
+            else if (tc && i == hc) t = t_last;
+            else t = t_first + i - tc;
+            const long long tb = (long long)t * KB;                       // first unit of tile t
+            w.kb0 = (int)max(u0 - tb, 0LL);
+            w.kb1 = (int)min(u1 - tb, (long long)KB);
+            w.first = (int)(tb / U);
+            w.cn = (int)((tb + KB - 1) / U) - w.first + 1;
+        } else {
+            t = blockIdx.x + i * gridDim.x;
+            if (t >= total_tiles) return false;
+            w.kb0 = 0;
+            w.kb1 = KB;
+            w.first = blockIdx.x;
+            w.cn = 1;
+        }
+        w.n_tile = t % n_tiles;
         const int mt = t / n_tiles;
         if (grouped) {
-            expert = p.tile_expert[mt];
-            row0 = p.tile_row0[mt];
-            rows = p.tile_rows[mt];
+            w.expert = p.tile_expert[mt];
+            w.row0 = p.tile_row0[mt];
+            w.rows = p.tile_rows[mt];
         } else {
-            expert = 0;
-            row0 = mt * BN;
-            rows = min(BN, p.M - row0);
+            w.expert = 0;
+            w.row0 = mt * BN;
+            w.rows = min(BN, p.M - w.row0);
         }
+        return true;
     };
 
     if (warp < NEXP) {
@@ -256,13 +305,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                 pending = -1;
             }
         };
-        int g0 = 0;                                                       // stage counter at the start of the tile
-        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, g0 += num_kb) {
-            int n_tile, expert, row0, rows, ks;
-            tile_rows(t, n_tile, expert, row0, rows, ks);
-            const int rg = n_tile * 4 + quarter;                          // row group of 32 rows
-            const uint8_t* wrow = p.w[a] + (size_t)expert * p.w_expert_stride + (size_t)rg * tpr * Fmt<FMT>::tile_bytes +
-                                  (size_t)ks * num_kb * kb_bytes;          // this split's part of the row group's stream
+        int g0 = 0;                                                       // stage counter at the start of the piece
+        GemmWork w;
+        for (int i = 0; ok && get_work(i, w); ++i) {
+            const int num_kb = w.kb1 - w.kb0;
+            const int rg = w.n_tile * 4 + quarter;                        // row group of 32 rows
+            const uint8_t* wrow = p.w[a] + (size_t)w.expert * p.w_expert_stride + (size_t)rg * tpr * Fmt<FMT>::tile_bytes +
+                                  (size_t)w.kb0 * kb_bytes;                // this piece's part of the row group's stream
             // The weight stream of a row group is contiguous: ask L2 for it kGemmL2Ahead stages ahead
             // (expert weights come from HBM; two register-held slices alone do not cover that latency).
             if (lane == 0 && phase == 0) {
@@ -294,11 +343,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                     if (!ok) break;
                     tc_fence_after_sync();
                     if (tr) p.trace[g * 8 + 7] = clock64();
-                    tmem_st_32x32b_x32(lane_base + (uint32_t)(D_COLS + s * A_COLS + a * 32), vals);
+                    tmem_st_32x32b_x32(lane_base + (uint32_t)(RING0 + s * A_COLS + a * 32), vals);
                     pending = s;
                     if (PH == 1) announce();          // a lone warp per weight rows: nothing to overlap the store with
                 }
             }
+            g0 += num_kb;
         }
         if (ok) announce();
         else *abort_flag = 1;
@@ -308,13 +358,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         const int quarter = e & 3;                                        // == warp & 3: the lanes this warp may read
         constexpr int GROUPS = NEPI / 4;                                  // warps per lane quarter: they split the token columns
         const int grp = e >> 2;
-        const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);
+        uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);   // + the piece's accumulator buffer
+        int buf = 0;
         constexpr int NCH = BN / 32;                                      // 32-column chunks of the tile
         constexpr int CH = (NCH + GROUPS - 1) / GROUPS;                   // chunks per warp
         constexpr int NOUT = (EPI == kEpiSiluMul) ? 1 : NA;               // output tiles per weight row
         constexpr bool HOLD = (NOUT * CH <= 6);                           // few chunks: read all, release, then store
         pdl_wait();                                                       // the output buffer may be in use upstream
-        bool ok = true;
+        bool ok = true, etr = false;
         int it = 0;
         // one 32-column chunk of output tile o: accumulators -> fp16 pairs (two tokens per register)
         auto read_chunk = [&](int o, int c0, uint32_t (&dst)[16]) {
@@ -343,20 +394,30 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         auto release = [&]() {                                            // the next tile may overwrite the accumulators
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(acc_empty);
+            if (lane == 0) mbar_arrive(&acc_empty[buf]);
+            if (etr) p.trace[(it * 4 + 2) * 8 + 1] = clock64();
         };
-        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
-            int n_tile, expert, row0, rows, ks;
-            tile_rows(t, n_tile, expert, row0, rows, ks);
-            ok = mbar_wait(acc_full, it & 1, abort_flag);
+        GemmWork w;
+        for (; ok && get_work(it, w); ++it) {
+            const int row0 = w.row0, rows = w.rows;
+            buf = it % AB;
+            lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * D_COLS);
+            ok = mbar_wait(&acc_full[buf], (it / AB) & 1, abort_flag);
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
             tc_fence_after_sync();
-            const int n = n_tile * 128 + quarter * 32 + lane;             // weight row within the tile set
-            if (splits > 1) {
-                // split-K: fp32 partial sums of this split, [split][token][weight row]; a second kernel adds the splits
+            etr = p.trace != nullptr && blockIdx.x == 0 && it < 16 && e == 0 && lane == 0;
+            if (etr) p.trace[(it * 4 + 1) * 8 + 1] = clock64();
+            const int n = w.n_tile * 128 + quarter * 32 + lane;           // weight row within the tile set
+            if (w.cn > 1) {
+                // A tile cut by block boundaries.  Every contributor stores its fp32 partial sums
+                // ([output tile][token column][128 weight rows], this warp's slice of them), then counts
+                // itself in; the warp that arrives last adds the slices of all contributors in
+                // contributor order (so the sum does not depend on who was last) and stores the output.
                 if constexpr (EPI == kEpiStore) {
-                    float* pbase = p.partial + ((size_t)ks * p.M + row0) * p.ldo + n;
+                    constexpr size_t SLOT = (size_t)NOUT * BN * 128;      // floats per partial slot
+                    auto slot_of = [&](int c) { return p.partial + (size_t)(2 * c + (c == w.first ? 1 : 0)) * SLOT + quarter * 32 + lane; };
+                    float* mine = slot_of((int)blockIdx.x);
 #pragma unroll
                     for (int o = 0; o < NOUT; ++o) {
 #pragma unroll
@@ -366,15 +427,52 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                                 uint32_t v[32];
                                 tmem_ld_32x32b_x32(lane_base + (uint32_t)(o * BN + c0), v);
                                 tmem_wait_ld();
-                                float* dst = pbase + (size_t)c0 * p.ldo + (size_t)o * p.a_col_offset;
+                                float* dst = mine + (size_t)(o * BN + c0) * 128;
 #pragma unroll
-                                for (int j = 0; j < 32; ++j)
-                                    if (c0 + j < rows) dst[(size_t)j * p.ldo] = __uint_as_float(v[j]);
+                                for (int j = 0; j < 32; ++j) __stcg(dst + j * 128, __uint_as_float(v[j]));
                             }
                         }
                     }
+                    release();
+                    int seen = -1;
+                    int* cnt = nullptr;
+                    if (p.counters != nullptr) {
+                        __threadfence();
+                        __syncwarp();
+                        cnt = p.counters + w.first * NEPI + e;
+                        if (lane == 0) seen = atomicAdd(cnt, 1);
+                        seen = __shfl_sync(0xFFFFFFFFu, seen, 0);
+                    }
+                    if (seen == w.cn - 1) {
+                        if (lane == 0) *cnt = 0;                          // nobody else touches it in this launch
+                        __threadfence();
+#pragma unroll
+                        for (int o = 0; o < NOUT; ++o) {
+#pragma unroll
+                            for (int c = 0; c < CH; ++c) {
+                                const int c0 = (grp * CH + c) * 32;
+                                if (c0 < BN && c0 < rows) {
+                                    float acc[32];
+                                    const size_t off = (size_t)(o * BN + c0) * 128;
+                                    const float* src = slot_of(w.first) + off;
+#pragma unroll
+                                    for (int j = 0; j < 32; ++j) acc[j] = __ldcg(src + j * 128);
+                                    for (int cc = 1; cc < w.cn; ++cc) {
+                                        src = slot_of(w.first + cc) + off;
+#pragma unroll
+                                        for (int j = 0; j < 32; ++j) acc[j] += __ldcg(src + j * 128);
+                                    }
+                                    uint32_t h[16];
+#pragma unroll
+                                    for (int j = 0; j < 16; ++j) h[j] = as_u32(__floats2half2_rn(acc[2 * j], acc[2 * j + 1]));
+                                    store_chunk(o, c0, row0, rows, n, h);
+                                }
+                            }
+                        }
+                    }
+                } else {
+                    release();                                            // (grouped products are never cut)
                 }
-                release();
             } else if constexpr (HOLD) {
                 uint32_t packed[NOUT][CH][16];
 #pragma unroll
@@ -424,15 +522,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             pdl_wait();                                                   // activations come from the previous kernel
             int issued = 0, g = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-                int n_tile, expert, row0, rows, ks;
-                tile_rows(t, n_tile, expert, row0, rows, ks);
-                for (int kb = 0; kb < num_kb; ++kb, ++g) {
+            GemmWork w;
+            for (int i = 0; ok && get_work(i, w); ++i) {
+                for (int kb = w.kb0; kb < w.kb1; ++kb, ++g) {
                     const int s = g % S;
                     if (g >= S) ok = mbar_wait(&empty[s], ((g / S) - 1) & 1, abort_flag);
                     if (!ok) break;
                     mbar_arrive_expect_tx(&full[s], B_STAGE);
-                    tma_load_2d(smem_b + s * B_STAGE, &x_map, (ks * num_kb + kb) * kGemmBK, row0, &full[s]);
+                    tma_load_2d(smem_b + s * B_STAGE, &x_map, kb * kGemmBK, w.row0, &full[s]);
                     issued = g + 1;
                 }
             }
@@ -454,40 +551,76 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         const uint64_t desc0 = smem_desc_k_sw128(smem_u32(smem_b));       // slot 0, k-step 0
         bool ok = true;
         int g = 0, it = 0;
-        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
-            if (it > 0) {                                                 // the epilogue must have read the accumulators
-                ok = mbar_wait(acc_empty, (it - 1) & 1, abort_flag);
+        int s = 0;                                                        // ring slot of stage g and the parity of its
+        uint32_t par = 0;                                                 // "full" barrier, carried across pieces
+        GemmWork w;
+        for (; ok && get_work(it, w); ++it) {
+            const int buf = it % AB;
+            if (it >= AB) {                                               // the epilogue must have read this buffer's previous piece
+                ok = mbar_wait(&acc_empty[buf], ((it / AB) - 1) & 1, abort_flag);
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
                 tc_fence_after_sync();
+                if (p.trace != nullptr && blockIdx.x == 0 && it <= 16 && lane == 0) p.trace[((it - AB) * 4 + 3) * 8 + 1] = clock64();
             }
-            for (int kb = 0; kb < num_kb; ++kb, ++g) {
-                const int s = g % S;
-                const bool tr = p.trace != nullptr && blockIdx.x == 0 && g < 64 && lane == 0;
-                if (tr) p.trace[g * 8 + 0] = clock64();
-                ok = mbar_wait(&full[s], (g / S) & 1, abort_flag);
+            const uint32_t d_tmem = tmem_base + (uint32_t)(buf * D_COLS);
+            // Two stages per round when the piece has them: the barrier polls, the warp vote and the
+            // fence are paid once per 128 k, which keeps this loop ahead of the tensor pipe for
+            // token tiles narrower than 256 too.
+            for (int kb = w.kb0; kb < w.kb1;) {
+                const int n = w.kb1 - kb >= 2 ? 2 : 1;
+                int s1 = s + 1;
+                uint32_t par1 = par;
+                if (s1 == S) {
+                    s1 = 0;
+                    par1 ^= 1;
+                }
+                const bool tr = p.trace != nullptr && blockIdx.x == 0 && g + 1 < 64 && lane == 0;
+                if (tr) p.trace[g * 8 + 0] = p.trace[(g + 1) * 8 + 0] = clock64();
+                ok = mbar_wait(&full[s], par, abort_flag);
+                if (n == 2 && ok) ok = mbar_wait(&full[s1], par1, abort_flag);
                 ok = __all_sync(0xFFFFFFFFu, ok);
-                if (tr) p.trace[g * 8 + 2] = clock64();
+                if (tr) p.trace[g * 8 + 2] = p.trace[(g + 1) * 8 + 2] = clock64();
                 if (!ok) break;
                 tc_fence_after_sync();
-                // descriptor start address is in 16-byte units: slot s is s * B_STAGE / 16 further, k-step k is 2 further
-                const uint64_t desc_s = desc0 + (uint64_t)(s * (B_STAGE >> 4));
-                const uint32_t a_s = tmem_base + (uint32_t)(D_COLS + s * A_COLS);
                 if (elect_one()) {
 #pragma unroll
-                    for (int a = 0; a < NA; ++a) {
+                    for (int j = 0; j < 2; ++j) {
+                        if (j < n) {
+                            const int sj = j == 0 ? s : s1;
+                            // descriptor start address is in 16-byte units: slot s is s * B_STAGE / 16 further, k-step k is 2 further
+                            const uint64_t desc_s = desc0 + (uint64_t)(sj * (B_STAGE >> 4));
+                            const uint32_t a_s = tmem_base + (uint32_t)(RING0 + sj * A_COLS);
 #pragma unroll
-                        for (int k = 0; k < kGemmBK / 16; ++k)
-                            mma_ts_f16(tmem_base + (uint32_t)(a * BN), a_s + (uint32_t)(a * 32 + k * 8), desc_s + (uint64_t)(k * 2), idesc,
-                                       (kb | k) != 0);
+                            for (int a = 0; a < NA; ++a) {
+#pragma unroll
+                                for (int k = 0; k < kGemmBK / 16; ++k)
+                                    mma_ts_f16(d_tmem + (uint32_t)(a * BN), a_s + (uint32_t)(a * 32 + k * 8), desc_s + (uint64_t)(k * 2),
+                                               idesc, kb + j != w.kb0 || k != 0);
+                            }
+                            mma_commit(&empty[sj]);                       // slot reusable when these MMAs finish
+                        }
                     }
-                    mma_commit(&empty[s]);                                // slot reusable when these MMAs finish
                 }
                 __syncwarp();
-                if (tr) p.trace[g * 8 + 3] = clock64();
+                if (tr) p.trace[g * 8 + 3] = p.trace[(g + 1) * 8 + 3] = clock64();
+                kb += n;
+                g += n;
+                if (n == 2) {
+                    s = s1 + 1;
+                    par = par1;
+                    if (s == S) {
+                        s = 0;
+                        par ^= 1;
+                    }
+                } else {
+                    s = s1;
+                    par = par1;
+                }
             }
-            if (ok && elect_one()) mma_commit(acc_full);                  // accumulators of this tile are complete
+            if (ok && elect_one()) mma_commit(&acc_full[buf]);            // accumulators of this piece are complete
             __syncwarp();
+            if (p.trace != nullptr && blockIdx.x == 0 && it < 16 && lane == 0) p.trace[(it * 4 + 0) * 8 + 1] = clock64();
         }
         if (!ok) *abort_flag = 1;
     }
