@@ -45,10 +45,10 @@ qmm_status make_x_map(CUtensorMap* map, const uint16_t* X, int64_t rows, int64_t
     return QMM_OK;
 }
 
-template <int FMT, int BN, int NA, int EPI>
+template <int FMT, int BN, int NA, int EPI, bool DENSE>
 static qmm_status launch_t(const CUtensorMap& map, const GemmParams& p, dim3 grid, cudaStream_t st)
 {
-    auto kern = gemm_kernel<FMT, BN, NA, EPI>;
+    auto kern = gemm_kernel<FMT, BN, NA, EPI, DENSE>;
     constexpr int smem = GemmGeom<BN, NA>::kSmemBytes;
     static bool configured = false;                 // per instantiation; attribute is sticky per device context
     if (!configured) {
@@ -69,32 +69,38 @@ static qmm_status launch_t(const CUtensorMap& map, const GemmParams& p, dim3 gri
     return check_cuda(cudaLaunchKernelEx(&cfg, kern, map, p), "tensor-core GEMM launch");
 }
 
-// Launch one tensor-core product.  bn in {32, 64, 128}; na in {1, 2}; epi as GemmEpilogue.
-qmm_status launch_tc_gemm(int fmt, int bn, int na, int epi, const CUtensorMap& map, const GemmParams& p, dim3 grid,
-                          cudaStream_t st)
+// Launch one tensor-core product.  Dense (qmm_gemm): one weight tile set, token tiles of 32 .. 256,
+// plain store.  Grouped (expert products): token tiles of 32 .. 160 from a device-built list, one
+// or two weight tile sets, plain store or SiLU*mul.
+qmm_status launch_tc_gemm(int fmt, int bn, int na, int epi, bool dense, const CUtensorMap& map, const GemmParams& p,
+                          dim3 grid, cudaStream_t st)
 {
-#define QMM_TC_CASE(F, B, A, E) \
-    if (fmt == F && bn == B && na == A && epi == E) return launch_t<F, B, A, E>(map, p, grid, st);
-#define QMM_TC_FMT(F)                     \
-    QMM_TC_CASE(F, 32, 1, kEpiStore)      \
-    QMM_TC_CASE(F, 64, 1, kEpiStore)      \
-    QMM_TC_CASE(F, 128, 1, kEpiStore)     \
-    QMM_TC_CASE(F, 160, 1, kEpiStore)     \
-    QMM_TC_CASE(F, 192, 1, kEpiStore)     \
-    QMM_TC_CASE(F, 256, 1, kEpiStore)     \
-    QMM_TC_CASE(F, 32, 2, kEpiStore)      \
-    QMM_TC_CASE(F, 64, 2, kEpiStore)      \
-    QMM_TC_CASE(F, 128, 2, kEpiStore)     \
-    QMM_TC_CASE(F, 160, 2, kEpiStore)     \
-    QMM_TC_CASE(F, 32, 2, kEpiSiluMul)    \
-    QMM_TC_CASE(F, 64, 2, kEpiSiluMul)    \
-    QMM_TC_CASE(F, 128, 2, kEpiSiluMul)   \
-    QMM_TC_CASE(F, 160, 2, kEpiSiluMul)
+#define QMM_TC_CASE(F, B, A, E, D) \
+    if (fmt == F && bn == B && na == A && epi == E && dense == D) return launch_t<F, B, A, E, D>(map, p, grid, st);
+#define QMM_TC_FMT(F)                            \
+    QMM_TC_CASE(F, 32, 1, kEpiStore, true)       \
+    QMM_TC_CASE(F, 64, 1, kEpiStore, true)       \
+    QMM_TC_CASE(F, 128, 1, kEpiStore, true)      \
+    QMM_TC_CASE(F, 160, 1, kEpiStore, true)      \
+    QMM_TC_CASE(F, 192, 1, kEpiStore, true)      \
+    QMM_TC_CASE(F, 256, 1, kEpiStore, true)      \
+    QMM_TC_CASE(F, 32, 1, kEpiStore, false)      \
+    QMM_TC_CASE(F, 64, 1, kEpiStore, false)      \
+    QMM_TC_CASE(F, 128, 1, kEpiStore, false)     \
+    QMM_TC_CASE(F, 160, 1, kEpiStore, false)     \
+    QMM_TC_CASE(F, 32, 2, kEpiStore, false)      \
+    QMM_TC_CASE(F, 64, 2, kEpiStore, false)      \
+    QMM_TC_CASE(F, 128, 2, kEpiStore, false)     \
+    QMM_TC_CASE(F, 160, 2, kEpiStore, false)     \
+    QMM_TC_CASE(F, 32, 2, kEpiSiluMul, false)    \
+    QMM_TC_CASE(F, 64, 2, kEpiSiluMul, false)    \
+    QMM_TC_CASE(F, 128, 2, kEpiSiluMul, false)   \
+    QMM_TC_CASE(F, 160, 2, kEpiSiluMul, false)
     QMM_TC_FMT(QMM_Q4)
     QMM_TC_FMT(QMM_Q8)
 #undef QMM_TC_FMT
 #undef QMM_TC_CASE
-    return fail(QMM_ERR_UNSUPPORTED, "no tensor-core kernel for fmt=%d bn=%d na=%d epi=%d", fmt, bn, na, epi);
+    return fail(QMM_ERR_UNSUPPORTED, "no tensor-core kernel for fmt=%d bn=%d na=%d epi=%d dense=%d", fmt, bn, na, epi, (int)dense);
 }
 
 // Persistent grid: one block per SM (a block's 18 warps use most of the register file), never
@@ -124,9 +130,7 @@ int pick_expert_tile(int64_t total_rows, int experts)
 }
 
 // Adds the partial sums of the tiles that the dense GEMM cut across blocks, contributors in
-// ascending order (a fixed order: same bits on every call), and stores fp16.  Used when tiles
-// are cut into many pieces (few tiles, long K), where the whole GPU does the sum faster than
-// the last contributor of every tile.  Block (t, y): token columns [8 y, 8 y + 8) of tile t; a
+// ascending order (a fixed order: same bits on every call), and stores fp16.  Block (t, y): token columns [8 y, 8 y + 8) of tile t; a
 // thread adds one float4 (4 weight rows of one token) per output tile, so every load is in flight at once.
 __global__ void gemm_cut_reduce_kernel(const float* __restrict__ partial, uint16_t* __restrict__ Y, int64_t ldy, int M,
                                        int bn, int nout, int a_col_offset, int n_tiles, int KB, int U)
@@ -166,46 +170,40 @@ struct GemmPlan {
     int bn, na;
     int units;          // (tile, k-block) units per block
     int grid;           // blocks
-    bool cut;           // some tile is shared between blocks (needs the partial-sum slots)
-    bool reduce_kernel; // cut tiles are summed by a second kernel (else by their last contributor)
+    bool cut;           // some tile is shared between blocks: partial-sum slots and the second kernel
 };
 
-// Workspace of qmm_gemm: [0, 4) status word, [256, 8192) arrival counters of the cut tiles,
-// [8192, 16384) trace samples (tuning aid), then the partial-sum slots.
-constexpr size_t kGemmWsCounters = 256, kGemmWsTrace = 8192, kGemmWsHeader = 16384;
-static_assert(kGemmWsCounters + (size_t)kNumSMs * 8 * sizeof(int) <= kGemmWsTrace, "counter area");
+// Workspace of qmm_gemm: [0, 4) status word, [4096, 8192) trace samples (tuning aid), then the
+// partial-sum slots.
+constexpr size_t kGemmWsTrace = 4096, kGemmWsHeader = 8192;
 
 // Token tile: 256 (the widest MMA, N = 256) once M exceeds one 128-token tile, else the smallest
 // that holds M; one weight tile per block.  The (tile, k-block) units are dealt to the blocks in
 // equal contiguous shares:
 //   tiles <= SMs / 2: every tile is cut into equal pieces, one per block, as many as the SMs can
 //                     take at once; a second kernel adds the pieces;
-//   tiles <  SMs:     whole tiles (cutting gains less than the exposed sum at the end costs);
-//   tiles >= SMs:     one share per SM, whatever tiles it crosses; a block computes its two cut
-//                     tiles first, and the last contributor of a cut tile adds the pieces while
-//                     whole tiles are still being computed.
+//   otherwise:        whole tiles, the same number for every block.  (Shares that cut tiles were
+//                     measured here too: the fp32 partial traffic costs more than the idle SMs
+//                     of the last round.)
 static GemmPlan gemm_plan(int64_t M, int64_t N, int64_t K)
 {
     GemmPlan p;
     p.bn = M > 128 ? 256 : pick_token_tile(M);
     p.na = 1;
-    int force_units = 0, force_reduce = -1;
-    if (const char* f = getenv("QMM_GEMM_FORCE")) {            // "bn,na[,units[,second kernel 0/1]]" for tuning sweeps and tests
-        int b = 0, a = 0, u = 0, r = -1;
-        const int got = sscanf(f, "%d,%d,%d,%d", &b, &a, &u, &r);
-        if (got >= 2 && (a == 1 || (a == 2 && N % 256 == 0 && b <= 128)) &&
-            (b == 32 || b == 64 || b == 128 || ((b == 160 || b == 192 || b == 256) && a == 1))) {
+    int force_units = 0;
+    if (const char* f = getenv("QMM_GEMM_FORCE")) {            // "bn,na[,units]" for tuning sweeps and tests
+        int b = 0, a = 0, u = 0;
+        const int got = sscanf(f, "%d,%d,%d", &b, &a, &u);
+        if (got >= 2 && a == 1 && (b == 32 || b == 64 || b == 128 || b == 160 || b == 192 || b == 256)) {
             p.bn = b;
             p.na = a;
             if (got >= 3 && u >= 1) force_units = u;
-            if (got >= 4) force_reduce = r != 0;
         }
     }
     const int64_t tiles = (N / (128 * p.na)) * ((M + p.bn - 1) / p.bn);
     const int64_t KB = K / kGemmBK;
     const int64_t total = tiles * KB;
     int64_t units;
-    p.reduce_kernel = false;
     if (tiles * 2 <= kNumSMs) {
         // the largest number of equal pieces per tile that the SMs can take at once, every piece
         // worth a pipeline fill and an epilogue (>= 8 k-blocks)
@@ -213,18 +211,13 @@ static GemmPlan gemm_plan(int64_t M, int64_t N, int64_t K)
         for (int64_t d = 2; d * tiles <= kNumSMs; ++d)
             if (KB % d == 0 && KB / d >= 8) pieces = d;
         units = KB / pieces;
-        p.reduce_kernel = true;
-    } else if (tiles < kNumSMs) {
-        units = KB;
     } else {
-        units = (total + kNumSMs - 1) / kNumSMs;
+        units = KB * ((tiles + kNumSMs - 1) / kNumSMs);       // whole tiles, the same number for every block
     }
     if (force_units) units = force_units;
-    if (force_reduce >= 0) p.reduce_kernel = force_reduce != 0;
     p.units = (int)units;
     p.grid = (int)((total + units - 1) / units);
     p.cut = units % KB != 0;
-    if (!p.cut) p.reduce_kernel = false;
     return p;
 }
 
@@ -240,8 +233,6 @@ qmm_status launch_gemm(int fmt, const void* packed, int64_t N, int64_t K, const 
 {
     const GemmPlan plan = gemm_plan(M, N, K);
     const int bn = plan.bn, na = plan.na;
-    if (plan.grid > kNumSMs && plan.cut && !plan.reduce_kernel)   // (only a forced unit count can ask for this)
-        return fail(QMM_ERR_UNSUPPORTED, "qmm_gemm: %d blocks with cut tiles exceed the counter area", plan.grid);
     CUtensorMap map;
     qmm_status s = make_x_map(&map, X, M, K, ldx, bn);
     if (s != QMM_OK) return s;
@@ -257,12 +248,11 @@ qmm_status launch_gemm(int fmt, const void* packed, int64_t N, int64_t K, const 
     p.a_col_offset = (int)(N / 2);
     p.M = (int)M;
     p.units_per_block = plan.units;
-    p.counters = plan.reduce_kernel ? nullptr : (int*)((uint8_t*)ws + kGemmWsCounters);
     p.partial = (float*)((uint8_t*)ws + kGemmWsHeader);
     p.status = (int*)ws;
     if (getenv("QMM_GEMM_TRACE")) p.trace = (long long*)((uint8_t*)ws + kGemmWsTrace);   // tuning aid
-    s = launch_tc_gemm(fmt, bn, na, kEpiStore, map, p, dim3((unsigned)plan.grid), st);
-    if (s != QMM_OK || !plan.reduce_kernel) return s;
+    s = launch_tc_gemm(fmt, bn, na, kEpiStore, true, map, p, dim3((unsigned)plan.grid), st);
+    if (s != QMM_OK || !plan.cut) return s;
     const int n_tiles = (int)(N / (128 * na));
     const int64_t tiles = (int64_t)n_tiles * ((M + bn - 1) / bn);
     cudaLaunchConfig_t cfg = {};

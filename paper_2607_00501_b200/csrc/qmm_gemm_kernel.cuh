@@ -22,7 +22,8 @@
 //                      code loads straight from global/L2, unpack to fp16(d*q),
 //                      tcgen05.st into the A ring in TMEM.
 //   epilogue (8 warps, two per lane quarter): tcgen05.ld the accumulators,
-//                      release them, store fp16.
+//                      convert, stage the tile in shared memory, release the
+//                      accumulators, then store the tile with 16-byte rows.
 //   TMA producer (1 warp): activation tiles -> shared-memory ring (128-byte
 //                      swizzle), one elected lane.
 //   MMA issuer (1 warp, converged): one elected lane issues tcgen05.mma
@@ -61,13 +62,11 @@ struct GemmParams {
     const int* tile_row0;            // [max_tiles] first permuted row of the tile
     const int* tile_rows;            // [max_tiles] valid rows in the tile (<= BN)
     const int* num_tiles;            // [1]
-    // dense mode, work split by k-blocks ("stream-K"): block b owns the units [b*U, (b+1)*U) of the
-    // tile-major sequence of (tile, k-block) units; a tile cut by a block boundary is summed from the
-    // fp32 partial results of its contributors by whichever of them finishes last, in contributor order
-    int units_per_block;             // U; 0 = whole tiles, t = blockIdx.x, blockIdx.x + gridDim.x, ...
-    float* partial;                  // [2 * gridDim.x] slots of NA*BN*128 floats (U > 0 and some tile is cut)
-    int* counters;                   // [gridDim.x * epilogue warps] arrival counts, zero between launches; null: the
-                                     // contributors only store their partial sums and a second kernel adds them
+    // dense mode: block b owns the units [b*U, (b+1)*U) of the tile-major sequence of (tile, k-block)
+    // units; the pieces of a tile cut by a block boundary go to `partial` as fp32 and a second
+    // kernel adds them
+    int units_per_block;             // U
+    float* partial;                  // [2 * gridDim.x] slots of NA*BN*128 floats (when some tile is cut)
     int* status;                     // device status word (0 = ok)
     long long* trace;                // optional [block 0 only] clock64 samples for pipeline analysis (tuning aid), else null
 };
@@ -84,9 +83,14 @@ struct GemmGeom {
     // of at least four weight slots still fits beside them
     static constexpr int kAccBufs = (2 * kDCols + 4 * kACols <= kTmemCols) ? 2 : 1;
     static constexpr int kFit = (kTmemCols - kAccBufs * kDCols) / kACols;
-    static constexpr int kStages = kFit < kGemmMaxStages ? kFit : kGemmMaxStages;
     static constexpr int kBStage = BN * kGemmBK * 2;                       // bytes per activation slot
-    static constexpr int kSmemBytes = kStages * kBStage + 1024 /*align*/ + 256;
+    // the epilogue stages a finished tile in shared memory as fp16 [output tile][token][128 weight rows]
+    static constexpr int kStaging = NA * BN * 128 * 2;
+    static constexpr int kSmemMax = 227 * 1024;                            // per block on sm_100
+    static constexpr int kSmemFit = (kSmemMax - 1024 - 256 - kStaging) / kBStage;
+    static constexpr int kFit2 = kFit < kSmemFit ? kFit : kSmemFit;
+    static constexpr int kStages = kFit2 < kGemmMaxStages ? kFit2 : kGemmMaxStages;
+    static constexpr int kSmemBytes = kStages * kBStage + kStaging + 1024 /*align*/ + 256;
     // Warp roles: 8 expanders, 8 epilogue warps (two per TMEM lane quarter), TMA producer, MMA issuer.
     static constexpr int kExpWarps = 8;
     static constexpr int kEpiWarps = 8;
@@ -163,6 +167,34 @@ struct GemmWork {
     int first, cn;
 };
 
+// Epilogue of a piece of a tile that block boundaries cut (dense mode): store this warp's slice
+// of the fp32 partial sums ([output tile][token column][128 weight rows]) and free the
+// accumulators.  A second kernel adds the pieces of every cut tile in a fixed order.
+template <int BN, int NOUT, int CH>
+__device__ __noinline__ void cut_tile_epilogue(const GemmParams& p, const GemmWork& w, uint32_t lane_base, int quarter, int grp,
+                                               int lane, uint64_t* acc_empty_bar)
+{
+    using namespace tc;
+    constexpr size_t SLOT = (size_t)NOUT * BN * 128;                      // floats per partial slot
+    // slot of this block's piece: 2 b + 1 for the piece that starts a tile, 2 b for one that continues it
+    float* mine = p.partial + (size_t)(2 * blockIdx.x + ((int)blockIdx.x == w.first ? 1 : 0)) * SLOT + quarter * 32 + lane;
+#pragma unroll 1
+    for (int oc = 0; oc < NOUT * CH; ++oc) {
+        const int o = oc / CH, c0 = (grp * CH + oc % CH) * 32;
+        if (c0 < BN && c0 < w.rows) {
+            uint32_t v[32];
+            tmem_ld_32x32b_x32(lane_base + (uint32_t)(o * BN + c0), v);
+            tmem_wait_ld();
+            float* dst = mine + (size_t)(o * BN + c0) * 128;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) __stcg(dst + j * 128, __uint_as_float(v[j]));
+        }
+    }
+    tc_fence_before_sync();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(acc_empty_bar);                            // the accumulators may be overwritten
+}
+
 // Persistent, warp-specialised kernel.  Tile t = (token tile t / n_tiles, weight
 // tile t % n_tiles).  Grouped mode: every block walks the tile list t =
 // blockIdx.x, blockIdx.x + gridDim.x, ... so blocks that run together share
@@ -171,7 +203,7 @@ struct GemmWork {
 // count.  The pipeline (stage counter, barrier phases) runs on across pieces:
 // while the epilogue warps drain the accumulators of piece i, the expanders
 // and the TMA producer already fill the ring for piece i+1.
-template <int FMT, int BN, int NA, int EPI>
+template <int FMT, int BN, int NA, int EPI, bool DENSE>
 __global__ void __launch_bounds__(GemmGeom<BN, NA>::kThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
 {
@@ -194,16 +226,19 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* smem_b = smem;                                               // S slots, 1024-aligned each
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S * B_STAGE);
+    uint8_t* staging = smem + S * B_STAGE;                                // finished tile, fp16 [output tile][token][128 rows]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(staging + G::kStaging);
     uint64_t* full = bars;                                                // [S] expanders + TMA -> MMA
     uint64_t* empty = bars + S;                                           // [S] MMA -> expanders, TMA
     uint64_t* acc_full = bars + 2 * S;                                    // [2] MMA -> epilogue
     uint64_t* acc_empty = bars + 2 * S + 2;                               // [2] epilogue -> MMA
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 4);
+    uint64_t* stg_full = bars + 2 * S + 4;                                // epilogue warps: tile staged
+    uint64_t* stg_empty = bars + 2 * S + 5;                               // epilogue warps: staged tile stored
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 6);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const bool grouped = p.tile_expert != nullptr;
+    constexpr bool grouped = !DENSE;                                      // token tiles come from a device-built list
     if (grouped) pdl_wait();                                              // the tile list is written upstream
     // plain store: the NA tile sets split the rows of one matrix; SiLU*mul: they are two matrices of N rows each
     const int n_tiles = (EPI == kEpiSiluMul) ? p.N / 128 : p.N / (128 * NA);
@@ -222,6 +257,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             mbar_init(&acc_full[b], 1);
             mbar_init(&acc_empty[b], NEPI);
         }
+        mbar_init(stg_full, NEPI);
+        mbar_init(stg_empty, NEPI);
         *abort_flag = 0;
         fence_barrier_init();
     }
@@ -363,35 +400,21 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         constexpr int NCH = BN / 32;                                      // 32-column chunks of the tile
         constexpr int CH = (NCH + GROUPS - 1) / GROUPS;                   // chunks per warp
         constexpr int NOUT = (EPI == kEpiSiluMul) ? 1 : NA;               // output tiles per weight row
-        constexpr bool HOLD = (NOUT * CH <= 6);                           // few chunks: read all, release, then store
         pdl_wait();                                                       // the output buffer may be in use upstream
         bool ok = true, etr = false;
-        int it = 0;
-        // one 32-column chunk of output tile o: accumulators -> fp16 pairs (two tokens per register)
-        auto read_chunk = [&](int o, int c0, uint32_t (&dst)[16]) {
-            uint32_t v[32];
-            tmem_ld_32x32b_x32(lane_base + (uint32_t)(o * BN + c0), v);
-            if (EPI == kEpiSiluMul) {
-                uint32_t u[32];
-                tmem_ld_32x32b_x32(lane_base + (uint32_t)(BN + c0), u);
-                tmem_wait_ld();
-#pragma unroll
-                for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(silu_f(__uint_as_float(v[j])) * __uint_as_float(u[j]));
-            } else {
-                tmem_wait_ld();
-            }
-#pragma unroll
-            for (int j = 0; j < 16; ++j) dst[j] = as_u32(__floats2half2_rn(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1])));
-        };
-        auto store_chunk = [&](int o, int c0, int row0, int rows, int n, const uint32_t (&src)[16]) {
-            uint16_t* out = p.out + (size_t)(row0 + c0) * p.ldo + (size_t)o * p.a_col_offset + n;
+        int it = 0, staged = 0;                                           // pieces seen / tiles that went through the staging buffer
+        const uint32_t stg_lane = smem_u32(staging) + (uint32_t)((quarter * 32 + lane) * 2);   // this thread's weight row
+        // 32 tokens (one chunk) of this thread's weight row -> staging[o][c0 + j][row]
+        auto stage_chunk = [&](int o, int c0, const uint32_t (&v)[32]) {
+            const uint32_t dst = stg_lane + (uint32_t)((o * BN + c0) * 256);
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
-                if (c0 + 2 * j < rows) out[(size_t)(2 * j) * p.ldo] = (uint16_t)(src[j] & 0xFFFFu);
-                if (c0 + 2 * j + 1 < rows) out[(size_t)(2 * j + 1) * p.ldo] = (uint16_t)(src[j] >> 16);
+                const uint32_t h = as_u32(__floats2half2_rn(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1])));
+                st_shared_b16(dst + (uint32_t)(2 * j * 256), (uint16_t)(h & 0xFFFFu));
+                st_shared_b16(dst + (uint32_t)((2 * j + 1) * 256), (uint16_t)(h >> 16));
             }
         };
-        auto release = [&]() {                                            // the next tile may overwrite the accumulators
+        auto release = [&]() {                                            // the next piece may overwrite the accumulators
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty[buf]);
@@ -399,7 +422,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         };
         GemmWork w;
         for (; ok && get_work(it, w); ++it) {
-            const int row0 = w.row0, rows = w.rows;
+            const int rows = w.rows;
             buf = it % AB;
             lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * D_COLS);
             ok = mbar_wait(&acc_full[buf], (it / AB) & 1, abort_flag);
@@ -408,112 +431,72 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             tc_fence_after_sync();
             etr = p.trace != nullptr && blockIdx.x == 0 && it < 16 && e == 0 && lane == 0;
             if (etr) p.trace[(it * 4 + 1) * 8 + 1] = clock64();
-            const int n = w.n_tile * 128 + quarter * 32 + lane;           // weight row within the tile set
-            if (w.cn > 1) {
-                // A tile cut by block boundaries.  Every contributor stores its fp32 partial sums
-                // ([output tile][token column][128 weight rows], this warp's slice of them), then counts
-                // itself in; the warp that arrives last adds the slices of all contributors in
-                // contributor order (so the sum does not depend on who was last) and stores the output.
-                if constexpr (EPI == kEpiStore) {
-                    constexpr size_t SLOT = (size_t)NOUT * BN * 128;      // floats per partial slot
-                    auto slot_of = [&](int c) { return p.partial + (size_t)(2 * c + (c == w.first ? 1 : 0)) * SLOT + quarter * 32 + lane; };
-                    float* mine = slot_of((int)blockIdx.x);
+            if (DENSE && w.cn > 1) {
+                // a tile cut by block boundaries (dense mode only): out of line, so that its registers
+                // do not weigh on the common path
+                if constexpr (DENSE) cut_tile_epilogue<BN, NOUT, CH>(p, w, lane_base, quarter, grp, lane, &acc_empty[buf]);
+                continue;
+            }
+            if (staged > 0) {                                             // the previous staged tile must have been stored
+                ok = mbar_wait(stg_empty, (staged - 1) & 1, abort_flag);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
+            }
+            if constexpr (EPI == kEpiSiluMul) {
 #pragma unroll
-                    for (int o = 0; o < NOUT; ++o) {
+                for (int c = 0; c < CH; ++c) {
+                    const int c0 = (grp * CH + c) * 32;
+                    if (c0 < BN && c0 < rows) {                           // uniform over the warp
+                        uint32_t g[32], u[32];
+                        tmem_ld_32x32b_x32(lane_base + (uint32_t)c0, g);
+                        tmem_ld_32x32b_x32(lane_base + (uint32_t)(BN + c0), u);
+                        tmem_wait_ld();
 #pragma unroll
-                        for (int c = 0; c < CH; ++c) {
-                            const int c0 = (grp * CH + c) * 32;
-                            if (c0 < BN && c0 < rows) {
-                                uint32_t v[32];
-                                tmem_ld_32x32b_x32(lane_base + (uint32_t)(o * BN + c0), v);
-                                tmem_wait_ld();
-                                float* dst = mine + (size_t)(o * BN + c0) * 128;
-#pragma unroll
-                                for (int j = 0; j < 32; ++j) __stcg(dst + j * 128, __uint_as_float(v[j]));
-                            }
-                        }
-                    }
-                    release();
-                    int seen = -1;
-                    int* cnt = nullptr;
-                    if (p.counters != nullptr) {
-                        __threadfence();
-                        __syncwarp();
-                        cnt = p.counters + w.first * NEPI + e;
-                        if (lane == 0) seen = atomicAdd(cnt, 1);
-                        seen = __shfl_sync(0xFFFFFFFFu, seen, 0);
-                    }
-                    if (seen == w.cn - 1) {
-                        if (lane == 0) *cnt = 0;                          // nobody else touches it in this launch
-                        __threadfence();
-#pragma unroll
-                        for (int o = 0; o < NOUT; ++o) {
-#pragma unroll
-                            for (int c = 0; c < CH; ++c) {
-                                const int c0 = (grp * CH + c) * 32;
-                                if (c0 < BN && c0 < rows) {
-                                    float acc[32];
-                                    const size_t off = (size_t)(o * BN + c0) * 128;
-                                    const float* src = slot_of(w.first) + off;
-#pragma unroll
-                                    for (int j = 0; j < 32; ++j) acc[j] = __ldcg(src + j * 128);
-                                    for (int cc = 1; cc < w.cn; ++cc) {
-                                        src = slot_of(w.first + cc) + off;
-#pragma unroll
-                                        for (int j = 0; j < 32; ++j) acc[j] += __ldcg(src + j * 128);
-                                    }
-                                    uint32_t h[16];
-#pragma unroll
-                                    for (int j = 0; j < 16; ++j) h[j] = as_u32(__floats2half2_rn(acc[2 * j], acc[2 * j + 1]));
-                                    store_chunk(o, c0, row0, rows, n, h);
-                                }
-                            }
-                        }
-                    }
-                } else {
-                    release();                                            // (grouped products are never cut)
-                }
-            } else if constexpr (HOLD) {
-                uint32_t packed[NOUT][CH][16];
-#pragma unroll
-                for (int o = 0; o < NOUT; ++o) {
-#pragma unroll
-                    for (int c = 0; c < CH; ++c) {
-                        const int c0 = (grp * CH + c) * 32;
-                        if (c0 < BN && c0 < rows) read_chunk(o, c0, packed[o][c]);   // uniform over the warp
-                    }
-                }
-                release();
-#pragma unroll
-                for (int o = 0; o < NOUT; ++o) {
-#pragma unroll
-                    for (int c = 0; c < CH; ++c) {
-                        const int c0 = (grp * CH + c) * 32;
-                        if (c0 < BN && c0 < rows) store_chunk(o, c0, row0, rows, n, packed[o][c]);
+                        for (int j = 0; j < 32; ++j) g[j] = __float_as_uint(silu_f(__uint_as_float(g[j])) * __uint_as_float(u[j]));
+                        stage_chunk(0, c0, g);
                     }
                 }
             } else {
-                // many chunks: stream them (read, store), release after the last read
-                uint32_t buf[16];
-                bool pending = false;
-                int po = 0, pc0 = 0;
+                // two chunk loads in flight per wait (an invalid second chunk re-reads the first and is dropped)
 #pragma unroll
                 for (int o = 0; o < NOUT; ++o) {
 #pragma unroll
-                    for (int c = 0; c < CH; ++c) {
-                        const int c0 = (grp * CH + c) * 32;
-                        if (c0 < BN && c0 < rows) {
-                            if (pending) store_chunk(po, pc0, row0, rows, n, buf);
-                            read_chunk(o, c0, buf);
-                            pending = true;
-                            po = o;
-                            pc0 = c0;
+                    for (int c = 0; c < CH; c += 2) {
+                        const int c0 = (grp * CH + c) * 32, c1 = c0 + 32;
+                        const bool v0 = c0 < BN && c0 < rows, v1 = c + 1 < CH && c1 < BN && c1 < rows;
+                        if (v0) {
+                            uint32_t va[32], vb[32];
+                            tmem_ld_32x32b_x32(lane_base + (uint32_t)(o * BN + c0), va);
+                            tmem_ld_32x32b_x32(lane_base + (uint32_t)(o * BN + (v1 ? c1 : c0)), vb);
+                            tmem_wait_ld();
+                            stage_chunk(o, c0, va);
+                            if (v1) stage_chunk(o, c1, vb);
                         }
                     }
                 }
-                release();
-                if (pending) store_chunk(po, pc0, row0, rows, n, buf);
             }
+            release();
+            // all eight warps staged -> store the tile: two token rows (2 x 256 bytes) per warp instruction
+            __syncwarp();
+            if (lane == 0) mbar_arrive(stg_full);
+            ok = mbar_wait(stg_full, staged & 1, abort_flag);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) break;
+            {
+                const int half = lane >> 4, seg = lane & 15;              // row of the pair, 16-byte segment of the row
+                uint16_t* out = p.out + (size_t)w.row0 * p.ldo + (size_t)w.n_tile * 128 + seg * 8;
+                const uint32_t src = smem_u32(staging) + (uint32_t)(seg * 16);
+#pragma unroll
+                for (int o = 0; o < NOUT; ++o) {
+                    for (int r = 2 * e + half; r < rows; r += 2 * NEPI) {
+                        const uint4 v = ld_shared_v4(src + (uint32_t)((o * BN + r) * 256));
+                        *reinterpret_cast<uint4*>(out + (size_t)r * p.ldo + (size_t)o * p.a_col_offset) = v;
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(stg_empty);
+            ++staged;
         }
         if (!ok) *abort_flag = 1;
     } else if (warp == TMA_WARP) {
@@ -564,11 +547,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                 if (p.trace != nullptr && blockIdx.x == 0 && it <= 16 && lane == 0) p.trace[((it - AB) * 4 + 3) * 8 + 1] = clock64();
             }
             const uint32_t d_tmem = tmem_base + (uint32_t)(buf * D_COLS);
-            // Two stages per round when the piece has them: the barrier polls, the warp vote and the
-            // fence are paid once per 128 k, which keeps this loop ahead of the tensor pipe for
-            // token tiles narrower than 256 too.
+            // Two stages per round when the ring is deep enough and the piece has them: the barrier
+            // polls, the warp vote and the fence are paid once per 128 k.
             for (int kb = w.kb0; kb < w.kb1;) {
-                const int n = w.kb1 - kb >= 2 ? 2 : 1;
+                const int n = (S >= 6 && w.kb1 - kb >= 2) ? 2 : 1;         // (a short ring is consumed one stage at a time)
                 int s1 = s + 1;
                 uint32_t par1 = par;
                 if (s1 == S) {

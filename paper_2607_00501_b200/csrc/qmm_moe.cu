@@ -16,8 +16,8 @@
 namespace qmm {
 
 qmm_status make_x_map(CUtensorMap* map, const uint16_t* X, int64_t rows, int64_t K, int64_t ld, int box_rows);
-qmm_status launch_tc_gemm(int fmt, int bn, int na, int epi, const CUtensorMap& map, const GemmParams& p, dim3 grid,
-                          cudaStream_t st);
+qmm_status launch_tc_gemm(int fmt, int bn, int na, int epi, bool dense, const CUtensorMap& map, const GemmParams& p,
+                          dim3 grid, cudaStream_t st);
 int pick_expert_tile(int64_t total_rows, int experts);
 qmm_status launch_moe_gemv(int fmt, bool gate_up, const void* w0, const void* w1, int64_t expert_stride,
                            const uint16_t* x, uint16_t* out, const int* perm, const int* topk_idx,
@@ -434,7 +434,7 @@ qmm_status launch_moe(const qmm_moe_args* a, void* ws, bool route_only, cudaStre
         p.num_tiles = num_tiles;
         p.status = status;
         if (getenv("QMM_GEMM_TRACE")) p.trace = (long long*)(base + w.trace);
-        s = launch_tc_gemm(a->fmt, w.bn, 2, kEpiSiluMul, map, p, persistent_grid(w.bn, 2, 0), st);
+        s = launch_tc_gemm(a->fmt, w.bn, 2, kEpiSiluMul, false, map, p, persistent_grid(w.bn, 2, 0), st);
         if (s != QMM_OK) return s;
     }
     // 5. grouped down GEMM -> D [total, H]
@@ -458,7 +458,7 @@ qmm_status launch_moe(const qmm_moe_args* a, void* ws, bool route_only, cudaStre
         p.tile_rows = tile_rows;
         p.num_tiles = num_tiles;
         p.status = status;
-        s = launch_tc_gemm(a->fmt, w.bn, na, kEpiStore, map, p, persistent_grid(w.bn, na, 0), st);
+        s = launch_tc_gemm(a->fmt, w.bn, na, kEpiStore, false, map, p, persistent_grid(w.bn, na, 0), st);
         if (s != QMM_OK) return s;
     }
     // 6. weighted combine
