@@ -49,7 +49,7 @@ template <int FMT, int BN, int NA, int EPI, bool DENSE>
 static qmm_status launch_t(const CUtensorMap& map, const GemmParams& p, dim3 grid, cudaStream_t st)
 {
     auto kern = gemm_kernel<FMT, BN, NA, EPI, DENSE>;
-    constexpr int smem = GemmGeom<BN, NA>::kSmemBytes;
+    constexpr int smem = GemmGeom<BN, NA, EPI>::kSmemBytes;
     static bool configured = false;                 // per instantiation; attribute is sticky per device context
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
@@ -58,7 +58,7 @@ static qmm_status launch_t(const CUtensorMap& map, const GemmParams& p, dim3 gri
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
-    cfg.blockDim = dim3(GemmGeom<BN, NA>::kThreads);
+    cfg.blockDim = dim3(GemmGeom<BN, NA, EPI>::kThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];

@@ -74,7 +74,7 @@ struct GemmParams {
 // Pipeline geometry of one instantiation.  Tensor memory: half of the SM's 512 columns when the
 // accumulators leave room for it (two blocks per SM), else all of it; what the accumulators leave
 // is the weight ring.  A stage is one weight slot in TMEM plus one activation slot in shared memory.
-template <int BN, int NA>
+template <int BN, int NA, int EPI>
 struct GemmGeom {
     static constexpr int kACols = NA * 32;                                 // TMEM columns per weight slot
     static constexpr int kDCols = NA * BN;                                 // accumulator columns
@@ -84,8 +84,9 @@ struct GemmGeom {
     static constexpr int kAccBufs = (2 * kDCols + 4 * kACols <= kTmemCols) ? 2 : 1;
     static constexpr int kFit = (kTmemCols - kAccBufs * kDCols) / kACols;
     static constexpr int kBStage = BN * kGemmBK * 2;                       // bytes per activation slot
-    // the epilogue stages a finished tile in shared memory as fp16 [output tile][token][128 weight rows]
-    static constexpr int kStaging = NA * BN * 128 * 2;
+    // the epilogue stages a finished tile in shared memory, [tile set][token][128 weight rows]: fp16
+    // outputs (plain store), or the fp32 gate and up accumulators (SiLU*mul is applied on the way out)
+    static constexpr int kStaging = NA * BN * 128 * (EPI == kEpiSiluMul ? 4 : 2);
     static constexpr int kSmemMax = 227 * 1024;                            // per block on sm_100
     static constexpr int kSmemFit = (kSmemMax - 1024 - 256 - kStaging) / kBStage;
     static constexpr int kFit2 = kFit < kSmemFit ? kFit : kSmemFit;
@@ -204,11 +205,11 @@ __device__ __noinline__ void cut_tile_epilogue(const GemmParams& p, const GemmWo
 // while the epilogue warps drain the accumulators of piece i, the expanders
 // and the TMA producer already fill the ring for piece i+1.
 template <int FMT, int BN, int NA, int EPI, bool DENSE>
-__global__ void __launch_bounds__(GemmGeom<BN, NA>::kThreads, 1)
+__global__ void __launch_bounds__(GemmGeom<BN, NA, EPI>::kThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
 {
     using namespace tc;
-    using G = GemmGeom<BN, NA>;
+    using G = GemmGeom<BN, NA, EPI>;
     constexpr int NEXP = G::kExpWarps;
     constexpr int PH = NEXP / (4 * NA);               // expander warps per (weight tile, lane quarter): they alternate stages
     constexpr int NEPI = G::kEpiWarps;
@@ -443,6 +444,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                 if (!ok) break;
             }
             if constexpr (EPI == kEpiSiluMul) {
+                // gate and up accumulators go to the staging buffer as they are (fp32); SiLU*mul is
+                // applied when the tile is stored, after the accumulators have been handed back
 #pragma unroll
                 for (int c = 0; c < CH; ++c) {
                     const int c0 = (grp * CH + c) * 32;
@@ -451,9 +454,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                         tmem_ld_32x32b_x32(lane_base + (uint32_t)c0, g);
                         tmem_ld_32x32b_x32(lane_base + (uint32_t)(BN + c0), u);
                         tmem_wait_ld();
+                        const uint32_t dg = smem_u32(staging) + (uint32_t)(c0 * 512 + (quarter * 32 + lane) * 4);
+                        const uint32_t du = dg + (uint32_t)(BN * 512);
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) g[j] = __float_as_uint(silu_f(__uint_as_float(g[j])) * __uint_as_float(u[j]));
-                        stage_chunk(0, c0, g);
+                        for (int j = 0; j < 32; ++j) {
+                            st_shared_b32(dg + (uint32_t)(j * 512), g[j]);
+                            st_shared_b32(du + (uint32_t)(j * 512), u[j]);
+                        }
                     }
                 }
             } else {
@@ -482,7 +489,21 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             ok = mbar_wait(stg_full, staged & 1, abort_flag);
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
-            {
+            if constexpr (EPI == kEpiSiluMul) {
+                // one token row (128 weight rows: 4 per lane) per warp instruction
+                uint16_t* out = p.out + (size_t)w.row0 * p.ldo + (size_t)w.n_tile * 128 + lane * 4;
+                const uint32_t src = smem_u32(staging) + (uint32_t)(lane * 16);
+                for (int r = e; r < rows; r += NEPI) {
+                    const uint4 g = ld_shared_v4(src + (uint32_t)(r * 512));
+                    const uint4 u = ld_shared_v4(src + (uint32_t)((BN + r) * 512));
+                    uint2 h;
+                    h.x = as_u32(__floats2half2_rn(silu_f(__uint_as_float(g.x)) * __uint_as_float(u.x),
+                                                   silu_f(__uint_as_float(g.y)) * __uint_as_float(u.y)));
+                    h.y = as_u32(__floats2half2_rn(silu_f(__uint_as_float(g.z)) * __uint_as_float(u.z),
+                                                   silu_f(__uint_as_float(g.w)) * __uint_as_float(u.w)));
+                    *reinterpret_cast<uint2*>(out + (size_t)r * p.ldo) = h;
+                }
+            } else {
                 const int half = lane >> 4, seg = lane & 15;              // row of the pair, 16-byte segment of the row
                 uint16_t* out = p.out + (size_t)w.row0 * p.ldo + (size_t)w.n_tile * 128 + seg * 8;
                 const uint32_t src = smem_u32(staging) + (uint32_t)(seg * 16);

@@ -193,9 +193,10 @@ route_small_kernel(const float* __restrict__ logits, int T, int E, int topk,
 // (expert_offsets[e]) and its first token tile -- by summing the counts of the
 // experts before it, and writes its entries of the token-tile list of the
 // grouped GEMMs.  Then it walks the T*topk (token, slot) pairs in flat order
-// and appends those routed to e, which yields the stable order by
-// (expert, token).  perm[r] = flat index, inv_perm[flat] = r.
+// (a contiguous run per thread) and appends those routed to e, which yields the
+// stable order by (expert, token).  perm[r] = flat index, inv_perm[flat] = r.
 constexpr int kPermuteThreads = 1024;
+constexpr int kPermutePer = 16;       // (token, slot) pairs per thread and pass
 
 __global__ void __launch_bounds__(kPermuteThreads)
 permute_kernel(const int* __restrict__ topk_idx, int total, const int* __restrict__ counts, int E, int bn,
@@ -252,11 +253,31 @@ permute_kernel(const int* __restrict__ topk_idx, int total, const int* __restric
     }
     __syncthreads();
 
-    for (int start = 0; start < total; start += kPermuteThreads) {
-        const int i = start + threadIdx.x;
-        const bool mine = i < total && topk_idx[i] == e;
-        const unsigned ballot = __ballot_sync(0xFFFFFFFFu, mine);
-        if (lane == 0) s_warp[warp] = __popc(ballot);
+    // A thread takes kPermutePer consecutive pairs (all loads in flight at once), counts those routed
+    // to e, and a block-wide exclusive scan of the counts gives where its matches go.
+    for (int pass0 = 0; pass0 < total; pass0 += kPermuteThreads * kPermutePer) {
+        const int i0 = pass0 + (int)threadIdx.x * kPermutePer;
+        unsigned mask = 0;
+        if (i0 + kPermutePer <= total) {
+            int4 v[kPermutePer / 4];
+#pragma unroll
+            for (int q = 0; q < kPermutePer / 4; ++q) v[q] = reinterpret_cast<const int4*>(topk_idx + i0)[q];
+#pragma unroll
+            for (int q = 0; q < kPermutePer / 4; ++q)
+                mask |= (unsigned)(v[q].x == e) << (4 * q) | (unsigned)(v[q].y == e) << (4 * q + 1) |
+                        (unsigned)(v[q].z == e) << (4 * q + 2) | (unsigned)(v[q].w == e) << (4 * q + 3);
+        } else {
+            for (int j = 0; j < kPermutePer; ++j)
+                if (i0 + j < total && topk_idx[i0 + j] == e) mask |= 1u << j;
+        }
+        const int cnt = __popc(mask);
+        int incl = cnt;                                                   // inclusive scan inside the warp
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+            if (lane >= off) incl += up;
+        }
+        if (lane == 31) s_warp[warp] = incl;
         __syncthreads();
         int before = 0, all = 0;
 #pragma unroll
@@ -265,11 +286,14 @@ permute_kernel(const int* __restrict__ topk_idx, int total, const int* __restric
             if (w < warp) before += c;
             all += c;
         }
-        if (mine) {
-            const int r = s_base + before + __popc(ballot & ((1u << lane) - 1u));
-            perm[r] = i;
-            if (perm_user) perm_user[r] = i;
-            inv_perm[i] = r;
+        int r = s_base + before + incl - cnt;
+        while (mask) {
+            const int j = __ffs(mask) - 1;
+            mask &= mask - 1;
+            perm[r] = i0 + j;
+            if (perm_user) perm_user[r] = i0 + j;
+            inv_perm[i0 + j] = r;
+            ++r;
         }
         __syncthreads();
         if (threadIdx.x == 0) s_base += all;
