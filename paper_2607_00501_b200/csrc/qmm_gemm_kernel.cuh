@@ -92,9 +92,10 @@ struct GemmGeom {
     static constexpr int kFit2 = kFit < kSmemFit ? kFit : kSmemFit;
     static constexpr int kStages = kFit2 < kGemmMaxStages ? kFit2 : kGemmMaxStages;
     static constexpr int kSmemBytes = kStages * kBStage + kStaging + 1024 /*align*/ + 256;
-    // Warp roles: 8 expanders, 8 epilogue warps (two per TMEM lane quarter), TMA producer, MMA issuer.
-    static constexpr int kExpWarps = 8;
-    static constexpr int kEpiWarps = 8;
+    // Warp roles: expanders, epilogue warps (one or two per TMEM lane quarter), TMA producer, MMA
+    // issuer.  Narrow token tiles are bound by the expansion, not by the epilogue: 16 + 4 there.
+    static constexpr int kExpWarps = BN <= 64 ? 16 : 8;
+    static constexpr int kEpiWarps = BN <= 64 ? 4 : 8;
     static constexpr int kThreads = (kExpWarps + kEpiWarps + 2) * 32;
     static_assert(kStages >= 2, "tensor memory over-subscribed");
 };
