@@ -178,7 +178,8 @@ struct GemmPlan {
 constexpr size_t kGemmWsTrace = 4096, kGemmWsHeader = 8192;
 
 // Token tile: 256 (the widest MMA, N = 256) once M exceeds one 128-token tile, else the smallest
-// that holds M; one weight tile per block.  The (tile, k-block) units are dealt to the blocks in
+// that holds M -- or half / a quarter of that when this yields between 3/4 and one round of whole
+// tiles; one weight tile per block.  The (tile, k-block) units are dealt to the blocks in
 // equal contiguous shares:
 //   tiles <= SMs / 2: every tile is cut into equal pieces, one per block, as many as the SMs can
 //                     take at once; a second kernel adds the pieces;
@@ -190,6 +191,15 @@ static GemmPlan gemm_plan(int64_t M, int64_t N, int64_t K)
     GemmPlan p;
     p.bn = M > 128 ? 256 : pick_token_tile(M);
     p.na = 1;
+    // a narrower token tile that fills one round of the SMs with whole tiles beats cutting K
+    // (no partial sums, no second kernel)
+    for (int cand = p.bn / 2; cand >= 64 && (N / 128) * ((M + p.bn - 1) / p.bn) * 2 <= kNumSMs; cand /= 2) {
+        const int64_t t = (N / 128) * ((M + cand - 1) / cand);
+        if (t * 4 >= (int64_t)kNumSMs * 3 && t <= kNumSMs) {
+            p.bn = cand;
+            break;
+        }
+    }
     int force_units = 0;
     if (const char* f = getenv("QMM_GEMM_FORCE")) {            // "bn,na[,units]" for tuning sweeps and tests
         int b = 0, a = 0, u = 0;
