@@ -84,6 +84,29 @@ def test_gemv_workspace_rule(L, monkeypatch):
     assert qmm.gemv_workspace_bytes(4, 512, 2048) == 0
 
 
+def test_gemm_workspace_rule(L, monkeypatch):
+    """The workspace is a fixed header, plus fp32 partial-sum slots exactly when the plan cuts tiles
+    along K (few output tiles); the plan is a pure function of the shape."""
+    monkeypatch.delenv("QMM_GEMM_FORCE", raising=False)
+    header = qmm.gemm_workspace_bytes(4, 2048, 8192, 3072)        # 512 whole tiles: nothing to add up
+    assert header == 8192
+    assert qmm.gemm_workspace_bytes(8, 2048, 8192, 3072) == header
+    assert qmm.gemm_workspace_bytes(4, 1024, 3072, 8192) == header    # 96 tiles: whole tiles, one round
+    assert qmm.gemm_workspace_bytes(4, 256, 8192, 3072) == header     # 128 tiles of 128 tokens instead of a K split
+    few = qmm.gemm_workspace_bytes(4, 256, 3072, 8192)                 # 24 tiles of 256 tokens: K cut in 4
+    assert few == header + 2 * 96 * 256 * 128 * 4
+    assert qmm.gemm_workspace_bytes(4, 256, 3072, 8192) == few         # same answer every time
+    tiny = qmm.gemm_workspace_bytes(4, 1, 128, 256)                    # one tile, 4 k-blocks: too short to cut
+    assert tiny == header
+    monkeypatch.setenv("QMM_GEMM_FORCE", "128,1,5")
+    forced = qmm.gemm_workspace_bytes(4, 100, 256, 2048)               # 2 tiles x 32 k-blocks in shares of 5: 13 blocks
+    assert forced == header + 2 * 13 * 128 * 128 * 4
+    buf = (ctypes.c_char * 512)()
+    a = (ctypes.addressof(buf) + 255) & ~255
+    assert L.qmm_gemm(4, a, 256, 2048, a, 2048, a, 256, 100, a, forced - 1, None) == 4
+    assert "workspace" in qmm.last_error()
+
+
 def test_moe_argument_checks(L):
     buf = (ctypes.c_char * 512)()
     a = (ctypes.addressof(buf) + 255) & ~255
