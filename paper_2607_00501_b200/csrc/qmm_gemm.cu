@@ -3,6 +3,7 @@
 // launch_tc_gemm, the grouped expert GEMMs of qmm_moe.
 #include "qmm_gemm_kernel.cuh"
 
+#include <atomic>
 #include <math.h>
 #include <stdio.h>
 #include <stdlib.h>
@@ -50,11 +51,15 @@ static qmm_status launch_t(const CUtensorMap& map, const GemmParams& p, dim3 gri
 {
     auto kern = gemm_kernel<FMT, BN, NA, EPI, DENSE>;
     constexpr int smem = GemmGeom<BN, NA, EPI>::kSmemBytes;
-    static bool configured = false;                 // per instantiation; attribute is sticky per device context
-    if (!configured) {
+    // the attribute is per device: remember which devices have it (per instantiation)
+    static std::atomic<uint64_t> configured{0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) dev = 0;
+    const uint64_t bit = dev < 64 ? (1ull << dev) : 0;
+    if (!(configured.load(std::memory_order_relaxed) & bit)) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return check_cuda(e, "tensor-core GEMM shared memory size");
-        configured = true;
+        configured.fetch_or(bit, std::memory_order_relaxed);
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
