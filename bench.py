@@ -482,6 +482,21 @@ def extra_sections(args, qmm, torch, pk, ops, fmts):
                               "frac_hbm": round(blocks.nbytes / med / 1e6 / pk["hbm_gbs"], 4)}
     del packed, blocks
 
+    # one cfg1 layer's feed-forward front half as a single launch: h = silu(Wgate x) * (Wup x)
+    for f in fmts:
+        wts = {name: (N, K, w) for name, N, K, act, w in synth.cfg1_layer_weights(0) if name in ("gate", "up")}
+        N, K, _ = wts["gate"]
+        pgate = qmm.pack(f, dev(synth.quantize(f, wts["gate"][2])), N, K)
+        pup = qmm.pack(f, dev(synth.quantize(f, wts["up"][2])), N, K)
+        xf = dev(synth.cfg1_layer_acts(0)["x_ffn"])
+        hf = torch.empty(N, dtype=torch.float16, device="cuda")
+        fn = lambda: qmm.gemv_gate_up(f, pgate, pup, N, K, xf, hf)
+        fn()
+        med, best = time_op(torch, fn, 10, flush)
+        b = 2 * synth.canonical_bytes(f, N, K)
+        out["ffn_gate_up_silu_q%d_gemv" % f] = {"ms": round(med, 4), "GBps": round(b / med / 1e6, 1),
+                                                 "frac_hbm": round(b / med / 1e6 / pk["hbm_gbs"], 4)}
+
     # cfg3: Q4 prefill GEMM sweep
     c = synth.CFG3
     gemm = {}

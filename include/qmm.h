@@ -127,6 +127,19 @@ typedef struct {
 } qmm_gemv_problem;
 qmm_status qmm_gemv_batch(qmm_format fmt, const qmm_gemv_problem* problems, int count, void* stream);
 
+/* Front half of a gated feed-forward block for one token, in one launch:
+ *     h[n] = fp16( silu(g[n]) * u[n] ),  g = W_gate x,  u = W_up x,
+ * g and u accumulated in fp32 and never rounded or written (the paper fuses
+ * operator sequences within the feed-forward block to save launches and
+ * round trips through memory, Sec. 3.3; it does not spell out which).
+ * silu(g) = g / (1 + exp(-g)).  W_gate and W_up are [N, K], packed separately.
+ *   packed_gate, packed_up  device, 32-byte aligned
+ *   x_fp16  device, [K] fp16;  h_fp16  device, [N] fp16, written
+ * K <= 32768.  No workspace.                                                 */
+qmm_status qmm_gemv_gate_up(qmm_format fmt, const void* packed_gate, const void* packed_up,
+                            int64_t N, int64_t K, const uint16_t* x_fp16, uint16_t* h_fp16,
+                            void* stream);
+
 /* qmm_gemv for callers that cannot allocate.  The paper has no counterpart to
  * this call; it exists for integrations that are not allowed to obtain device
  * memory at the time they need a product: code that runs after a host

@@ -37,6 +37,8 @@ size_t gemv_workspace_bytes(int fmt, int64_t N, int64_t K);
 qmm_status launch_gemv(int fmt, const void* packed, int64_t N, int64_t K, const uint16_t* x, uint16_t* y,
                        void* ws, cudaStream_t st);
 qmm_status launch_gemv_batch(int fmt, const qmm_gemv_problem* probs, int count, cudaStream_t st);
+qmm_status launch_gemv_gate_up(int fmt, const void* packed_gate, const void* packed_up, int64_t N, int64_t K,
+                               const uint16_t* x, uint16_t* h, cudaStream_t st);
 size_t gemm_workspace_bytes(int fmt, int64_t M, int64_t N, int64_t K);
 qmm_status launch_gemm(int fmt, const void* packed, int64_t N, int64_t K, const uint16_t* X, int64_t ldx,
                        uint16_t* Y, int64_t ldy, int64_t M, void* ws, cudaStream_t st);
@@ -150,6 +152,21 @@ qmm_status qmm_gemv(qmm_format fmt, const void* packed, int64_t N, int64_t K,
     }
     if ((s = check_device("qmm_gemv")) != QMM_OK) return s;
     return launch_gemv(fmt, packed, N, K, x_fp16, y_fp16, ws, (cudaStream_t)stream);
+}
+
+qmm_status qmm_gemv_gate_up(qmm_format fmt, const void* packed_gate, const void* packed_up, int64_t N, int64_t K,
+                            const uint16_t* x_fp16, uint16_t* h_fp16, void* stream)
+{
+    qmm_status s = check_matrix("qmm_gemv_gate_up", fmt, N, K);
+    if (s != QMM_OK) return s;
+    if (!packed_gate || !packed_up || !x_fp16 || !h_fp16) return fail(QMM_ERR_INVALID_ARG, "qmm_gemv_gate_up: null pointer");
+    if (!aligned(packed_gate, 32) || !aligned(packed_up, 32))
+        return fail(QMM_ERR_ALIGNMENT, "qmm_gemv_gate_up: packed matrices must be 32-byte aligned");
+    if (!aligned(x_fp16, 16) || !aligned(h_fp16, 16))
+        return fail(QMM_ERR_ALIGNMENT, "qmm_gemv_gate_up: x and h must be 16-byte aligned");
+    if (K > 32768) return fail(QMM_ERR_UNSUPPORTED, "qmm_gemv_gate_up: K=%lld > 32768", (long long)K);
+    if ((s = check_device("qmm_gemv_gate_up")) != QMM_OK) return s;
+    return launch_gemv_gate_up(fmt, packed_gate, packed_up, N, K, x_fp16, h_fp16, (cudaStream_t)stream);
 }
 
 qmm_status qmm_gemv_batch(qmm_format fmt, const qmm_gemv_problem* problems, int count, void* stream)

@@ -152,11 +152,15 @@ struct TileRegs {
 // So each warp issues the loads of its first group *before* waiting for the
 // previous kernel (programmatic dependent launch): the HBM latency of one
 // product hides behind the tail of the one before it.
-template <int FMT, int WARPS>
+//
+// GATEUP: the row-group pair of an item is (group j of `packed`, group j of `packed_up`) -- the gate
+// rows and the up rows of the same 32 outputs -- and the item writes h = fp16(silu(g) * u) for them
+// (no K split across blocks in this form).
+template <int FMT, int WARPS, bool GATEUP = false>
 __global__ void __launch_bounds__(WARPS * 32, 768 / (WARPS * 32))
 gemv_kernel(const uint8_t* __restrict__ packed, const uint16_t* __restrict__ x,
             uint16_t* __restrict__ y, float* __restrict__ partial,
-            int N, int K, int tiles_per_row, int splits, int items)
+            int N, int K, int tiles_per_row, int splits, int items, const uint8_t* __restrict__ packed_up)
 {
     extern __shared__ uint4 smem[];
     uint4* xs = smem;
@@ -170,17 +174,20 @@ gemv_kernel(const uint8_t* __restrict__ packed, const uint16_t* __restrict__ x,
     const int tps = tiles_per_row / splits;                     // tiles per item
     const size_t group_bytes = (size_t)tiles_per_row * TB;
     const uint8_t* lane_base = packed + 32 * lane;
+    // second row group of the pair: the next group of the same matrix, or the same group of the up matrix
+    const ptrdiff_t q_delta = GATEUP ? packed_up - packed : (ptrdiff_t)group_bytes;
+    constexpr int GROUPS_PER_ITEM = GATEUP ? 1 : 2;
 
     int item = blockIdx.x;
     int pair = item / splits, s = item - pair * splits;
     int t = s * tps + warp, t_end = (s + 1) * tps;
-    const uint8_t* tiles_p = lane_base + (size_t)(2 * pair) * group_bytes;
+    const uint8_t* tiles_p = lane_base + (size_t)(GROUPS_PER_ITEM * pair) * group_bytes;
 
     TileRegs<FMT> r;
     // slot u of the register file holds tile pair t + u * WARPS of the current item
     auto load_slot = [&](int u, int tt) {
         const uint8_t* tp = tiles_p + (size_t)tt * TB;
-        const uint8_t* tq = tp + group_bytes;
+        const uint8_t* tq = tp + q_delta;
         r.cp[u] = ld_stream_256(tp);
         r.cq[u] = ld_stream_256(tq);
         r.sp[u] = load_scales<FMT>(tp - 32 * lane, lane);
@@ -227,7 +234,7 @@ gemv_kernel(const uint8_t* __restrict__ packed, const uint16_t* __restrict__ x,
             s = item - pair * splits;
             t = s * tps + warp;
             t_end = (s + 1) * tps;
-            tiles_p = lane_base + (size_t)(2 * pair) * group_bytes;
+            tiles_p = lane_base + (size_t)(GROUPS_PER_ITEM * pair) * group_bytes;
             load_group();
         }
         // add the warps' partial sums in warp order
@@ -240,7 +247,17 @@ gemv_kernel(const uint8_t* __restrict__ packed, const uint16_t* __restrict__ x,
             w[32 + row + 1] = acc[3];
         }
         __syncthreads();
-        if (threadIdx.x < 64) {
+        if (GATEUP) {
+            if (threadIdx.x < 32) {                             // red[.. 0..31] = gate sums, red[.. 32..63] = up sums
+                float g = red[threadIdx.x], up = red[32 + threadIdx.x];
+#pragma unroll
+                for (int w = 1; w < WARPS; ++w) {
+                    g += red[w * 64 + threadIdx.x];
+                    up += red[w * 64 + 32 + threadIdx.x];
+                }
+                y[done_pair * 32 + threadIdx.x] = __half_as_ushort(__float2half_rn((g / (1.0f + expf(-g))) * up));
+            }
+        } else if (threadIdx.x < 64) {
             float sum = red[threadIdx.x];
 #pragma unroll
             for (int w = 1; w < WARPS; ++w) sum += red[w * 64 + threadIdx.x];
@@ -617,7 +634,7 @@ static qmm_status launch_gemv_t(const GemvPlan& p, const void* packed, int64_t N
     const int tpr = (int)(K / Fmt<FMT>::tile_k);
     const int items = (int)(N / (2 * kRowsPerGroup)) * p.splits;
     cudaError_t e = launch_pdl(kern, dim3(p.grid), dim3(WARPS * 32), smem, st,
-                               (const uint8_t*)packed, x, y, partial, (int)N, (int)K, tpr, p.splits, items);
+                               (const uint8_t*)packed, x, y, partial, (int)N, (int)K, tpr, p.splits, items, (const uint8_t*)nullptr);
     if (e != cudaSuccess) return check_cuda(e, "qmm_gemv launch");
     if (p.splits > 1) {
         e = launch_pdl(gemv_reduce_kernel, dim3((unsigned)((N + 255) / 256)), dim3(256), 0, st,
@@ -625,6 +642,32 @@ static qmm_status launch_gemv_t(const GemvPlan& p, const void* packed, int64_t N
         if (e != cudaSuccess) return check_cuda(e, "qmm_gemv reduce launch");
     }
     return QMM_OK;
+}
+
+// h = fp16(silu(W_gate x) * (W_up x)): gemv_kernel with (gate group, up group) pairs, one item per 32 outputs.
+qmm_status launch_gemv_gate_up(int fmt, const void* packed_gate, const void* packed_up, int64_t N, int64_t K,
+                               const uint16_t* x, uint16_t* h, cudaStream_t st)
+{
+    constexpr int WARPS = 8;
+    const size_t smem = (size_t)K * 4 + (size_t)WARPS * 64 * sizeof(float);
+    const int tpr = (int)(K / tile_k_of(fmt));
+    const int items = (int)(N / kRowsPerGroup);
+    const int grid = items < 3 * kNumSMs ? items : 3 * kNumSMs;
+    cudaError_t e = cudaSuccess;
+    if (fmt == QMM_Q4) {
+        auto kern = gemv_kernel<QMM_Q4, WARPS, true>;
+        if (smem > 48 * 1024) e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e == cudaSuccess)
+            e = launch_pdl(kern, dim3(grid), dim3(WARPS * 32), smem, st, (const uint8_t*)packed_gate, x, h, (float*)nullptr, (int)N,
+                           (int)K, tpr, 1, items, (const uint8_t*)packed_up);
+    } else {
+        auto kern = gemv_kernel<QMM_Q8, WARPS, true>;
+        if (smem > 48 * 1024) e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e == cudaSuccess)
+            e = launch_pdl(kern, dim3(grid), dim3(WARPS * 32), smem, st, (const uint8_t*)packed_gate, x, h, (float*)nullptr, (int)N,
+                           (int)K, tpr, 1, items, (const uint8_t*)packed_up);
+    }
+    return check_cuda(e, "qmm_gemv_gate_up launch");
 }
 
 // Expert products of the MoE layer for a handful of rows (decode): see moe_gemv_kernel.

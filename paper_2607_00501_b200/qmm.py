@@ -31,6 +31,7 @@ EXPORTS = (
     "qmm_last_error", "qmm_version", "qmm_canonical_bytes", "qmm_packed_bytes", "qmm_pack",
     "qmm_dequant", "qmm_gemv_workspace_bytes", "qmm_gemv", "qmm_gemm_workspace_bytes", "qmm_gemm",
     "qmm_moe_workspace_bytes", "qmm_moe", "qmm_moe_route", "qmm_status_check", "qmm_gemv_static", "qmm_gemv_batch",
+    "qmm_gemv_gate_up",
 )
 
 
@@ -82,6 +83,7 @@ def lib() -> ctypes.CDLL:
             L.qmm_gemv_workspace_bytes.argtypes = [ci, i64, i64]
             L.qmm_gemv.argtypes = [ci, vp, i64, i64, vp, vp, vp, sz, vp]
             L.qmm_gemv_static.argtypes = [ci, vp, i64, i64, vp, vp, vp]
+            L.qmm_gemv_gate_up.argtypes = [ci, vp, vp, i64, i64, vp, vp, vp]
             L.qmm_gemv_batch.argtypes = [ci, ctypes.POINTER(GemvProblem), ci, vp]
             L.qmm_gemm_workspace_bytes.restype = sz
             L.qmm_gemm_workspace_bytes.argtypes = [ci, i64, i64, i64]
@@ -182,6 +184,17 @@ def gemv_batch(fmt: int, problems) -> None:
 
 
 GEMV_STATIC_SCRATCH_BYTES = 1 << 20
+
+
+def gemv_gate_up(fmt: int, packed_gate: torch.Tensor, packed_up: torch.Tensor, N: int, K: int, x: torch.Tensor,
+                 h: torch.Tensor | None = None) -> torch.Tensor:
+    """h = fp16(silu(W_gate x) * (W_up x)) in one launch (both products kept in fp32 until the end)."""
+    assert x.is_cuda and x.dtype == torch.float16 and x.numel() == K and x.is_contiguous()
+    if h is None:
+        h = torch.empty(N, dtype=torch.float16, device=x.device)
+    assert h.is_cuda and h.dtype == torch.float16 and h.numel() == N and h.is_contiguous()
+    _check(lib().qmm_gemv_gate_up(fmt, packed_gate.data_ptr(), packed_up.data_ptr(), N, K, x.data_ptr(), h.data_ptr(), _stream()))
+    return h
 
 
 def gemv_static(fmt: int, packed: torch.Tensor, N: int, K: int, x: torch.Tensor, y: torch.Tensor) -> torch.Tensor:

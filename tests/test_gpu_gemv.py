@@ -156,6 +156,51 @@ def test_cfg1_one_layer_full_size_unfused_and_fused(qmm, oracle, fmt):
         util.assert_within_tol(util.host_f64(y), y_ref, B, "cfg1 fused " + "+".join(names))
 
 
+def check_gate_up(qmm, oracle, fmt, gate_blocks, up_blocks, N, K, x, what):
+    """h = silu(Wg x) * (Wu x): both products held to the per-product tolerance through the bound
+    it implies for h (|silu'| <= 1.1), plus the fp16 rounding of h."""
+    h = qmm.gemv_gate_up(fmt, packed_from(qmm, fmt, gate_blocks, N, K), packed_from(qmm, fmt, up_blocks, N, K), N, K, util.dev(x))
+    G, BG = oracle.gemv(fmt, gate_blocks, N, K, x)
+    U, BU = oracle.gemv(fmt, up_blocks, N, K, x)
+    tolG, tolU = util.RTOL_SUMABS * BG + util.ATOL, util.RTOL_SUMABS * BU + util.ATOL
+    sG = oracle.silu(G)
+    h_ref = sG * U
+    bound = 1.1 * tolG * np.abs(U) + np.abs(sG) * tolU + 1.1 * tolG * tolU + 2.0**-11 * np.abs(h_ref)
+    worst = float(np.max(np.abs(util.host_f64(h) - h_ref) / bound))
+    assert worst <= 1.0, "%s: %.3f of bound" % (what, worst)
+    return worst
+
+
+@pytest.mark.parametrize("fmt", [Q4, Q8])
+@pytest.mark.parametrize("N,K", [(128, 256), (384, 1280), (2176, 512)])
+def test_gemv_gate_up_small_shapes(qmm, oracle, fmt, N, K):
+    # (weights of the configs' distribution: with arbitrary scales silu(g) * u leaves the fp16 range)
+    gate = synth.quantize(fmt, synth.weights(92, N + K, N, K))
+    up = synth.quantize(fmt, synth.weights(93, N + K, N, K))
+    x = synth.activations(91, N + K, K)
+    check_gate_up(qmm, oracle, fmt, gate, up, N, K, x, "gate_up %dx%d fmt %d" % (N, K, fmt))
+
+
+@pytest.mark.parametrize("fmt", [Q4, Q8])
+def test_gemv_gate_up_cfg1_layer_full_size(qmm, oracle, fmt):
+    layer = 5
+    acts = synth.cfg1_layer_acts(layer)
+    w = {name: (N, K, synth.quantize(fmt, wt)) for name, N, K, act, wt in synth.cfg1_layer_weights(layer) if name in ("gate", "up")}
+    N, K, gate = w["gate"]
+    check_gate_up(qmm, oracle, fmt, gate, w["up"][2], N, K, acts["x_ffn"], "cfg1 gate_up fused with SiLU*mul")
+
+
+def test_gemv_gate_up_argument_checks(qmm):
+    a = torch.zeros(4096, dtype=torch.uint8, device="cuda")
+    x = torch.zeros(256, dtype=torch.float16, device="cuda")
+    h = torch.zeros(128, dtype=torch.float16, device="cuda")
+    L = qmm.lib()
+    assert L.qmm_gemv_gate_up(Q4, a.data_ptr(), a.data_ptr(), 128, 200, x.data_ptr(), h.data_ptr(), None) in (2, 5)   # K % 256
+    assert L.qmm_gemv_gate_up(Q4, a.data_ptr() + 8, a.data_ptr(), 128, 256, x.data_ptr(), h.data_ptr(), None) == 3    # alignment
+    assert L.qmm_gemv_gate_up(Q4, a.data_ptr(), None, 128, 256, x.data_ptr(), h.data_ptr(), None) == 1                # null
+    assert "null" in qmm.last_error()
+
+
 def test_cfg2_q8_lm_head_full_size(qmm, oracle):
     c = synth.CFG2
     blocks = synth.quantize(c["fmt"], synth.weights(c["seed"], 0, c["N"], c["K"]))
