@@ -497,51 +497,55 @@ def extra_sections(args, qmm, torch, pk, ops, fmts):
         out["ffn_gate_up_silu_q%d_gemv" % f] = {"ms": round(med, 4), "GBps": round(b / med / 1e6, 1),
                                                  "frac_hbm": round(b / med / 1e6 / pk["hbm_gbs"], 4)}
 
-    # cfg3: Q4 prefill GEMM sweep
+    # cfg3: prefill GEMM sweep (Q4 as the config says; Q8 = the same kernels with the byte expander,
+    # measured at the two largest M)
     c = synth.CFG3
-    gemm = {}
-    for name, N, K in c["shapes"]:
-        blocks = synth.quantize(c["fmt"], synth.weights(c["seed"], 0 if name == "gate_up" else 1, N, K))
-        packed = qmm.pack(c["fmt"], dev(blocks), N, K)
-        for M in c["Ms"]:
-            X = dev(synth.activations(c["seed"], 10 + M, M, K))
-            Y = torch.empty((M, N), dtype=torch.float16, device="cuda")
-            ws = torch.zeros(qmm.gemm_workspace_bytes(c["fmt"], M, N, K), dtype=torch.uint8, device="cuda")
-            fn = lambda: qmm.gemm(c["fmt"], packed, N, K, X, Y=Y, ws=ws)
+    for f, Ms in ((c["fmt"], c["Ms"]), (synth.Q8, c["Ms"][-2:])):
+        gemm = {}
+        for name, N, K in c["shapes"]:
+            blocks = synth.quantize(f, synth.weights(c["seed"], 0 if name == "gate_up" else 1, N, K))
+            packed = qmm.pack(f, dev(blocks), N, K)
+            for M in Ms:
+                X = dev(synth.activations(c["seed"], 10 + M, M, K))
+                Y = torch.empty((M, N), dtype=torch.float16, device="cuda")
+                ws = torch.zeros(qmm.gemm_workspace_bytes(f, M, N, K), dtype=torch.uint8, device="cuda")
+                fn = lambda: qmm.gemm(f, packed, N, K, X, Y=Y, ws=ws)
+                fn()
+                med, best = time_op(torch, fn, 10, flush)
+                tf = 2.0 * M * N * K / med / 1e9
+                gemm["%s_M%d" % (name, M)] = {"ms": round(med, 4), "TFLOPs": round(tf, 1),
+                                              "frac_tensor_measured": round(tf / pk["bf16_tflops"], 4),
+                                              "frac_tensor_nominal": round(tf / NOMINAL_BF16_TFLOPS, 4)}
+                qmm.status_check(ws)
+        out["prefill_gemm_q%d" % f] = gemm
+
+    # cfg4: MoE layer (Q4 as the config says; Q8 at the largest T)
+    c = synth.CFG4
+    for f, Ts in ((c["fmt"], c["Ts"]), (synth.Q8, c["Ts"][-1:])):
+        gate, up, down = synth.moe_expert_weights(c["seed"], f, c["E"], c["H"], c["I"])
+        pg = qmm.pack(f, dev(gate), c["E"] * c["I"], c["H"])
+        pu = qmm.pack(f, dev(up), c["E"] * c["I"], c["H"])
+        pd = qmm.pack(f, dev(down), c["E"] * c["H"], c["I"])
+        wbytes = gate.nbytes + up.nbytes + down.nbytes
+        moe = {}
+        for T in Ts:
+            X = dev(synth.activations(c["seed"], 100 + T, T, c["H"]))
+            lg = dev(synth.logits(c["seed"], 200 + T, T, c["E"]))
+            o = torch.empty((T, c["H"]), dtype=torch.float16, device="cuda")
+            a = qmm.moe_args(f, T, c["H"], c["I"], c["E"], c["topk"], lg, X, pg, pu, pd, o)
+            ws = torch.zeros(qmm.moe_workspace_bytes(a), dtype=torch.uint8, device="cuda")
+            fn = lambda: qmm.moe(a, ws)
             fn()
             med, best = time_op(torch, fn, 10, flush)
-            tf = 2.0 * M * N * K / med / 1e9
-            gemm["%s_M%d" % (name, M)] = {"ms": round(med, 4), "TFLOPs": round(tf, 1),
-                                          "frac_tensor_measured": round(tf / pk["bf16_tflops"], 4),
-                                          "frac_tensor_nominal": round(tf / NOMINAL_BF16_TFLOPS, 4)}
             qmm.status_check(ws)
-    out["prefill_gemm_q4"] = gemm
-
-    # cfg4: Q4 MoE layer
-    c = synth.CFG4
-    gate, up, down = synth.moe_expert_weights(c["seed"], c["fmt"], c["E"], c["H"], c["I"])
-    pg = qmm.pack(c["fmt"], dev(gate), c["E"] * c["I"], c["H"])
-    pu = qmm.pack(c["fmt"], dev(up), c["E"] * c["I"], c["H"])
-    pd = qmm.pack(c["fmt"], dev(down), c["E"] * c["H"], c["I"])
-    wbytes = gate.nbytes + up.nbytes + down.nbytes
-    moe = {}
-    for T in c["Ts"]:
-        X = dev(synth.activations(c["seed"], 100 + T, T, c["H"]))
-        lg = dev(synth.logits(c["seed"], 200 + T, T, c["E"]))
-        o = torch.empty((T, c["H"]), dtype=torch.float16, device="cuda")
-        a = qmm.moe_args(c["fmt"], T, c["H"], c["I"], c["E"], c["topk"], lg, X, pg, pu, pd, o)
-        ws = torch.zeros(qmm.moe_workspace_bytes(a), dtype=torch.uint8, device="cuda")
-        fn = lambda: qmm.moe(a, ws)
-        fn()
-        med, best = time_op(torch, fn, 10, flush)
-        qmm.status_check(ws)
-        fl = T * c["topk"] * 3 * 2.0 * c["H"] * c["I"]
-        touched = min(c["E"], T * c["topk"]) / c["E"] * wbytes if T * c["topk"] < c["E"] else wbytes
-        moe["T%d" % T] = {"ms": round(med, 4), "TFLOPs": round(fl / med / 1e9, 2),
-                          "frac_tensor_nominal": round(fl / med / 1e9 / NOMINAL_BF16_TFLOPS, 4),
-                          "hbm_floor_ms": round(touched / pk["hbm_gbs"] / 1e6, 4),
-                          "frac_of_hbm_floor": round(touched / pk["hbm_gbs"] / 1e6 / med, 4)}
-    out["moe_q4"] = moe
+            fl = T * c["topk"] * 3 * 2.0 * c["H"] * c["I"]
+            touched = min(c["E"], T * c["topk"]) / c["E"] * wbytes if T * c["topk"] < c["E"] else wbytes
+            moe["T%d" % T] = {"ms": round(med, 4), "TFLOPs": round(fl / med / 1e9, 2),
+                              "frac_tensor_nominal": round(fl / med / 1e9 / NOMINAL_BF16_TFLOPS, 4),
+                              "hbm_floor_ms": round(touched / pk["hbm_gbs"] / 1e6, 4),
+                              "frac_of_hbm_floor": round(touched / pk["hbm_gbs"] / 1e6 / med, 4)}
+        out["moe_q%d" % f] = moe
+        del pg, pu, pd, gate, up, down
     return out
 
 
