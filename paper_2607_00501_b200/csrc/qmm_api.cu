@@ -35,7 +35,7 @@ qmm_status launch_pack(int fmt, const void* canon, int64_t N, int64_t K, void* p
 qmm_status launch_dequant(int fmt, const void* packed, int64_t N, int64_t K, float* w_out, cudaStream_t st);
 size_t gemv_workspace_bytes(int fmt, int64_t N, int64_t K);
 qmm_status launch_gemv(int fmt, const void* packed, int64_t N, int64_t K, const uint16_t* x, uint16_t* y,
-                       void* ws, cudaStream_t st);
+                       void* ws, bool allow_cluster, cudaStream_t st);
 qmm_status launch_gemv_batch(int fmt, const qmm_gemv_problem* probs, int count, cudaStream_t st);
 qmm_status launch_gemv_gate_up(int fmt, const void* packed_gate, const void* packed_up, int64_t N, int64_t K,
                                const uint16_t* x, uint16_t* h, cudaStream_t st);
@@ -151,7 +151,7 @@ qmm_status qmm_gemv(qmm_format fmt, const void* packed, int64_t N, int64_t K,
         if (!aligned(ws, 16)) return fail(QMM_ERR_ALIGNMENT, "qmm_gemv: workspace must be 16-byte aligned");
     }
     if ((s = check_device("qmm_gemv")) != QMM_OK) return s;
-    return launch_gemv(fmt, packed, N, K, x_fp16, y_fp16, ws, (cudaStream_t)stream);
+    return launch_gemv(fmt, packed, N, K, x_fp16, y_fp16, ws, true, (cudaStream_t)stream);
 }
 
 qmm_status qmm_gemv_gate_up(qmm_format fmt, const void* packed_gate, const void* packed_up, int64_t N, int64_t K,

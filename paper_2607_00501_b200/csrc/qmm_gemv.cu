@@ -138,6 +138,25 @@ __device__ __forceinline__ uint32_t load_scales<QMM_Q8>(const uint8_t* tile, int
     return ld_nc_u32(tile + kTileCodeBytes + 2 * row);
 }
 
+// Thread-block cluster helpers of the split-K form without workspace.
+constexpr int kMaxClusterSplits = 8;                            // portable cluster size (room in shared memory)
+constexpr int kPlanClusterSplits = 4;                           // what the plan asks for: clusters of 8 measured slower to schedule
+
+// Store to the same shared-memory location in the cluster's first block.
+__device__ __forceinline__ void st_cluster_rank0(float* local_ptr, float v)
+{
+    uint32_t local = static_cast<uint32_t>(__cvta_generic_to_shared(local_ptr)), remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, 0;" : "=r"(remote) : "r"(local));
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(v) : "memory");
+}
+
+// Barrier over all threads of the cluster (hardware barrier; the blocks of a cluster are co-scheduled).
+__device__ __forceinline__ void cluster_sync()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 // Codes and scales of kUnroll tile pairs held in registers.
 template <int FMT>
 struct TileRegs {
@@ -153,6 +172,12 @@ struct TileRegs {
 // previous kernel (programmatic dependent launch): the HBM latency of one
 // product hides behind the tail of the one before it.
 //
+// K split across blocks (splits > 1), two forms.  With `partial`: fp32 partial sums go to the workspace
+// and gemv_reduce_kernel adds them.  Without (partial == nullptr): the `splits` blocks of an item are a
+// thread-block cluster; each writes its 64 sums into the shared memory of the cluster's first block
+// (distributed shared memory), which adds them in split order after a cluster barrier and writes y --
+// no workspace, no second launch, same bits on every call.
+//
 // GATEUP: the row-group pair of an item is (group j of `packed`, group j of `packed_up`) -- the gate
 // rows and the up rows of the same 32 outputs -- and the item writes h = fp16(silu(g) * u) for them
 // (no K split across blocks in this form).
@@ -166,6 +191,9 @@ gemv_kernel(const uint8_t* __restrict__ packed, const uint16_t* __restrict__ x,
     uint4* xs = smem;
     uint4* zs = smem + K / 8;
     float* red = reinterpret_cast<float*>(smem + K / 4);
+    float* cred = red + WARPS * 64;                             // cluster form: [2][kMaxClusterSplits][64] in the first block
+    const bool clustered = !GATEUP && splits > 1 && partial == nullptr;
+    int cluster_round = 0;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     constexpr int TB = Fmt<FMT>::tile_bytes;
     constexpr int XV = Fmt<FMT>::tile_k / 8;                    // uint4 of activations per tile
@@ -257,6 +285,22 @@ gemv_kernel(const uint8_t* __restrict__ packed, const uint16_t* __restrict__ x,
                 }
                 y[done_pair * 32 + threadIdx.x] = __half_as_ushort(__float2half_rn((g / (1.0f + expf(-g))) * up));
             }
+        } else if (clustered) {
+            // every block of the cluster runs the same sequence of items, one split each
+            float* slot = cred + (cluster_round & 1) * (kMaxClusterSplits * 64);
+            if (threadIdx.x < 64) {
+                float sum = red[threadIdx.x];
+#pragma unroll
+                for (int w = 1; w < WARPS; ++w) sum += red[w * 64 + threadIdx.x];
+                st_cluster_rank0(slot + done_s * 64 + threadIdx.x, sum);
+            }
+            cluster_sync();
+            if (done_s == 0 && threadIdx.x < 64) {
+                float total = slot[threadIdx.x];
+                for (int sp = 1; sp < splits; ++sp) total += slot[sp * 64 + threadIdx.x];
+                y[done_pair * 64 + threadIdx.x] = __half_as_ushort(__float2half_rn(total));
+            }
+            ++cluster_round;                                    // (two slots: the next item's sums do not wait for this read)
         } else if (threadIdx.x < 64) {
             float sum = red[threadIdx.x];
 #pragma unroll
@@ -571,7 +615,7 @@ struct GemvPlan {
 // Shape -> launch geometry.  The aim is >= ~2 resident blocks' worth of loads
 // on every SM: prefer more warps per block, and split K across blocks only
 // when the row groups alone cannot cover the SMs.
-GemvPlan gemv_plan(int fmt, int64_t N, int64_t K)
+GemvPlan gemv_plan(int fmt, int64_t N, int64_t K, bool cluster)
 {
     GemvPlan p;
     const int tpr = (int)(K / tile_k_of(fmt));
@@ -582,7 +626,8 @@ GemvPlan gemv_plan(int fmt, int64_t N, int64_t K)
     if ((int64_t)groups * tpr >= (int64_t)kNumSMs * 64 * 4 && warps > 8) warps = 8;
     else if ((int64_t)groups * tpr >= (int64_t)kNumSMs * 64 && warps > 16) warps = 16;
     int splits = 1;
-    while (groups * splits < kNumSMs && tpr / (splits * 2) >= warps && (tpr % (splits * 2)) == 0 && splits < 16)
+    const int max_splits = cluster ? kPlanClusterSplits : 16;
+    while (groups * splits < kNumSMs && tpr / (splits * 2) >= warps && (tpr % (splits * 2)) == 0 && splits < max_splits)
         splits *= 2;
     if (const char* f = getenv("QMM_GEMV_FORCE")) {           // "warps,splits" for sweeps
         int w = 0, s = 0;
@@ -601,7 +646,7 @@ GemvPlan gemv_plan(int fmt, int64_t N, int64_t K)
 
 size_t gemv_workspace_bytes(int fmt, int64_t N, int64_t K)
 {
-    const GemvPlan p = gemv_plan(fmt, N, K);
+    const GemvPlan p = gemv_plan(fmt, N, K, false);            // the two-kernel form (the cluster form needs none)
     return p.splits > 1 ? (size_t)p.splits * (size_t)N * sizeof(float) : 0;
 }
 
@@ -623,9 +668,13 @@ static cudaError_t launch_pdl(void (*kernel)(Args...), dim3 grid, dim3 block, si
 
 template <int FMT, int WARPS>
 static qmm_status launch_gemv_t(const GemvPlan& p, const void* packed, int64_t N, int64_t K,
-                                const uint16_t* x, uint16_t* y, float* partial, cudaStream_t st)
+                                const uint16_t* x, uint16_t* y, float* partial, bool allow_cluster, cudaStream_t st)
 {
-    const size_t smem = (size_t)K * 4 + (size_t)WARPS * 64 * sizeof(float);
+    // K split over up to 8 blocks: the blocks of an item form a cluster and add their sums through
+    // distributed shared memory; more splits (or a caller that brings its own scratch): partial sums
+    // in memory and a second kernel
+    const bool cluster = allow_cluster && p.splits > 1 && p.splits <= kMaxClusterSplits;
+    const size_t smem = (size_t)K * 4 + (size_t)WARPS * 64 * sizeof(float) + (cluster ? 2 * kMaxClusterSplits * 64 * sizeof(float) : 0);
     auto kern = gemv_kernel<FMT, WARPS>;
     if (smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -633,6 +682,25 @@ static qmm_status launch_gemv_t(const GemvPlan& p, const void* packed, int64_t N
     }
     const int tpr = (int)(K / Fmt<FMT>::tile_k);
     const int items = (int)(N / (2 * kRowsPerGroup)) * p.splits;
+    if (cluster) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(p.grid / p.splits * p.splits));      // whole clusters
+        cfg.blockDim = dim3(WARPS * 32);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[2];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = (unsigned)p.splits;
+        attr[1].val.clusterDim.y = 1;
+        attr[1].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 2;
+        return check_cuda(cudaLaunchKernelEx(&cfg, kern, (const uint8_t*)packed, x, y, (float*)nullptr, (int)N, (int)K, tpr, p.splits,
+                                             items, (const uint8_t*)nullptr),
+                          "qmm_gemv cluster launch");
+    }
     cudaError_t e = launch_pdl(kern, dim3(p.grid), dim3(WARPS * 32), smem, st,
                                (const uint8_t*)packed, x, y, partial, (int)N, (int)K, tpr, p.splits, items, (const uint8_t*)nullptr);
     if (e != cudaSuccess) return check_cuda(e, "qmm_gemv launch");
@@ -754,12 +822,13 @@ qmm_status launch_gemv_batch(int fmt, const qmm_gemv_problem* probs, int count, 
 }
 
 qmm_status launch_gemv(int fmt, const void* packed, int64_t N, int64_t K, const uint16_t* x, uint16_t* y,
-                       void* ws, cudaStream_t st)
+                       void* ws, bool allow_cluster, cudaStream_t st)
 {
-    const GemvPlan p = gemv_plan(fmt, N, K);
+    if (getenv("QMM_GEMV_NO_CLUSTER")) allow_cluster = false;          // tuning aid / tests of the two-kernel form
+    const GemvPlan p = gemv_plan(fmt, N, K, allow_cluster);
     float* partial = (float*)ws;
 #define QMM_GEMV_CASE(F, W) \
-    if (fmt == F && p.warps == W) return launch_gemv_t<F, W>(p, packed, N, K, x, y, partial, st);
+    if (fmt == F && p.warps == W) return launch_gemv_t<F, W>(p, packed, N, K, x, y, partial, allow_cluster, st);
     QMM_GEMV_CASE(QMM_Q4, 8)
     QMM_GEMV_CASE(QMM_Q4, 16)
     QMM_GEMV_CASE(QMM_Q8, 8)
@@ -838,6 +907,6 @@ extern "C" qmm_status qmm_gemv_static(qmm_format fmt, const void* packed, int64_
     if (s != QMM_OK) return s;
     // Partial sums are written in full before the second stage reads them, so the
     // scratch needs no clearing between calls.
-    return launch_gemv(fmt, packed, N, K, x_fp16, y_fp16, scratch, (cudaStream_t)stream);
+    return launch_gemv(fmt, packed, N, K, x_fp16, y_fp16, scratch, false, (cudaStream_t)stream);
 }
 

@@ -66,14 +66,23 @@ def test_gemv_small_shapes(qmm, oracle, fmt, N, K):
 
 
 @pytest.mark.parametrize("fmt", [Q4, Q8])
-@pytest.mark.parametrize("force", ["8,1", "8,2", "8,8", "16,1", "16,2", "16,4"])
-def test_gemv_every_launch_geometry(qmm, oracle, fmt, force, monkeypatch):
-    # the same product through each block size and K split (split-K partials + fixed-order reduce)
+@pytest.mark.parametrize("force", ["8,1", "8,2", "8,8", "16,1", "16,2", "16,4", "8,16"])
+@pytest.mark.parametrize("two_kernels", [False, True])
+def test_gemv_every_launch_geometry(qmm, oracle, fmt, force, two_kernels, monkeypatch):
+    # the same product through each block size and K split; a K split over up to 8 blocks adds the
+    # blocks' sums through the shared memory of a thread-block cluster, otherwise (more splits, or
+    # on request) through fp32 partials in the workspace and a second kernel -- both in a fixed order
     monkeypatch.setenv("QMM_GEMV_FORCE", force)
+    if two_kernels:
+        monkeypatch.setenv("QMM_GEMV_NO_CLUSTER", "1")
+    else:
+        monkeypatch.delenv("QMM_GEMV_NO_CLUSTER", raising=False)
     N, K = 512, 4096
     blocks = synth.quantize(fmt, synth.weights(91, fmt, N, K))
     x = synth.activations(91, 7, K)
-    run_gemv(qmm, oracle, fmt, blocks, N, K, x, "gemv forced " + force)
+    _, y = run_gemv(qmm, oracle, fmt, blocks, N, K, x, "gemv forced " + force)
+    _, y2 = run_gemv(qmm, oracle, fmt, blocks, N, K, x, "gemv forced " + force)
+    assert torch.equal(y, y2)                              # same bits on every call
 
 
 @pytest.mark.parametrize("fmt", [Q4, Q8])
