@@ -98,8 +98,9 @@ qmm_status qmm_dequant(qmm_format fmt, const void* packed, int64_t N, int64_t K,
 /* Decode matrix-vector product (Sec. 3.3, "GEMV (decode, M=1)"):
  *   y[n] = fp16( sum_b float(d[n,b]) * sum_{i<32} q[n,b,i] * x[32 b + i] ),
  * accumulated in fp32.  When N is too small to occupy the GPU the K range is
- * split across thread blocks, fp32 partial sums go to the workspace and a
- * second stage adds them in a fixed order.
+ * split across thread blocks and their sums are added in a fixed order:
+ * inside a thread-block cluster through shared memory, or (more than 8
+ * splits) through fp32 partial sums in the workspace and a second stage.
  *   packed    device, from qmm_pack, read only
  *   x_fp16    device, K fp16 values (bit patterns), read only
  *   y_fp16    device, N fp16 values, written
