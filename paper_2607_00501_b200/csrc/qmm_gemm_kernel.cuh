@@ -332,18 +332,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         Q4Consts kc;
         kc.init();
         bool ok = true;
-        int pending = -1;                                                 // stage stored but not yet announced
-        // The store of one stage is announced (wait::st + arrive) only after the next stage has been
-        // expanded, so the tensor-memory write latency hides behind ALU work.
-        auto announce = [&]() {
-            if (pending >= 0) {
-                tmem_wait_st();
-                tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&full[pending]);
-                pending = -1;
-            }
-        };
         int g0 = 0;                                                       // stage counter at the start of the piece
         GemmWork w;
         for (int i = 0; ok && get_work(i, w); ++i) {
@@ -375,7 +363,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                     if (kb + kGemmPrefetch * PH < num_kb) raw[i].load(wrow + (size_t)(kb + kGemmPrefetch * PH) * kb_bytes, lane);
                     if (lane == 0 && kb + kGemmL2Ahead < num_kb) l2_prefetch(wrow + (size_t)(kb + kGemmL2Ahead) * kb_bytes, (uint32_t)kb_bytes);
                     if (tr) p.trace[g * 8 + 5] = clock64();
-                    announce();
                     if (tr) p.trace[g * 8 + 6] = clock64();
                     if (g >= S) ok = mbar_wait(&empty[s], ((g / S) - 1) & 1, abort_flag);
                     ok = __all_sync(0xFFFFFFFFu, ok);
@@ -383,14 +370,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                     tc_fence_after_sync();
                     if (tr) p.trace[g * 8 + 7] = clock64();
                     tmem_st_32x32b_x32(lane_base + (uint32_t)(RING0 + s * A_COLS + a * 32), vals);
-                    pending = s;
-                    if (PH == 1) announce();          // a lone warp per weight rows: nothing to overlap the store with
+                    // announce the slot at once: deferring the wait for the store behind the next
+                    // expansion was measured and costs more in slot turn-around than the ~85 cycles it hides
+                    tmem_wait_st();
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&full[s]);
                 }
             }
             g0 += num_kb;
         }
-        if (ok) announce();
-        else *abort_flag = 1;
+        if (!ok) *abort_flag = 1;
     } else if (warp < NEXP + NEPI) {
         // ================= epilogue: TMEM -> registers -> global
         const int e = warp - NEXP;
