@@ -158,8 +158,14 @@ template <> struct RawRow64<QMM_Q8> {
     }
 };
 
-constexpr int kGemmPrefetch = 2;     // weight slices in flight per expander thread
-constexpr int kGemmL2Ahead = 12;     // stages of a row group's weight stream requested into L2 ahead of use
+#ifndef QMM_GEMM_PREFETCH
+#define QMM_GEMM_PREFETCH 2
+#endif
+#ifndef QMM_GEMM_L2_AHEAD
+#define QMM_GEMM_L2_AHEAD 6
+#endif
+constexpr int kGemmPrefetch = QMM_GEMM_PREFETCH;   // weight slices in flight per expander thread
+constexpr int kGemmL2Ahead = QMM_GEMM_L2_AHEAD;    // stages of a row group's weight stream requested into L2 ahead of use
 
 // One piece of work of a block: k-blocks [kb0, kb1) of one output tile.  `cn` blocks contribute to
 // the tile (block indices first .. first + cn - 1, k ascending); cn == 1: the piece is the whole tile.
