@@ -205,6 +205,16 @@ static GemmPlan gemm_plan(int64_t M, int64_t N, int64_t K)
             break;
         }
     }
+    // many tiles: 256 tokens (N = 256 MMAs at the tensor rate, but one accumulator buffer: ~2 400 cycles
+    // of hand-over per tile) or 192 (two accumulator buffers, ~470 cycles per stage against 515):
+    // whichever needs fewer cycles for its rounds of whole tiles on the SMs
+    if (p.bn == 256 && (N / 128) * ((M + 255) / 256) * 2 > kNumSMs) {
+        const int64_t kb = K / kGemmBK;
+        const int64_t t256 = (N / 128) * ((M + 255) / 256), t192 = (N / 128) * ((M + 191) / 192);
+        const int64_t c256 = ((t256 + kNumSMs - 1) / kNumSMs) * (kb * 515 + 2400);
+        const int64_t c192 = ((t192 + kNumSMs - 1) / kNumSMs) * (kb * 470 + 300);
+        if (c192 < c256) p.bn = 192;
+    }
     int force_units = 0;
     if (const char* f = getenv("QMM_GEMM_FORCE")) {            // "bn,na[,units]" for tuning sweeps and tests
         int b = 0, a = 0, u = 0;
