@@ -242,6 +242,7 @@ static qmm_status moe_entry(const char* who, const qmm_moe_args* a, void* ws, si
 {
     qmm_status s = check_moe(who, a);
     if (s != QMM_OK) return s;
+    if (a->T == 0) return QMM_OK;                               // nothing to do: no tensor or workspace is touched
     if (!a->logits) return fail(QMM_ERR_INVALID_ARG, "%s: logits is null", who);
     if (!route_only && (!a->X || !a->w_gate || !a->w_up || !a->w_down || !a->out))
         return fail(QMM_ERR_INVALID_ARG, "%s: null tensor pointer", who);
@@ -252,7 +253,6 @@ static qmm_status moe_entry(const char* who, const qmm_moe_args* a, void* ws, si
     if (!ws || ws_bytes < need)
         return fail(QMM_ERR_WORKSPACE, "%s: workspace of %zu bytes needed, %zu given", who, need, ws ? ws_bytes : (size_t)0);
     if (!aligned(ws, 256)) return fail(QMM_ERR_ALIGNMENT, "%s: workspace must be 256-byte aligned", who);
-    if (a->T == 0) return QMM_OK;
     if ((s = check_device(who)) != QMM_OK) return s;
     return launch_moe(a, ws, route_only, (cudaStream_t)stream);
 }

@@ -107,6 +107,22 @@ def test_gemm_workspace_rule(L, monkeypatch):
     assert "workspace" in qmm.last_error()
 
 
+def test_empty_inputs_are_accepted_and_do_nothing(L):
+    """M = 0 and T = 0 return QMM_OK before anything is launched (so no GPU is needed to see it);
+    negative sizes are argument errors."""
+    buf = (ctypes.c_char * 512)()
+    a = (ctypes.addressof(buf) + 255) & ~255
+    assert L.qmm_gemm(4, a, 128, 256, a, 256, a, 128, 0, None, 0, None) == 0
+    assert L.qmm_gemm(4, a, 128, 256, a, 256, a, 128, -1, None, 0, None) == 1
+    assert L.qmm_gemv_batch(4, None, 0, None) == 0
+    assert L.qmm_gemv_batch(4, None, -1, None) == 1
+    m = qmm.MoeArgs(0, 2048, 768, 128, 8, 4, a, a, a, a, a, a, None, None, None, None, None, None)
+    assert L.qmm_moe(ctypes.byref(m), None, 0, None) == 0
+    assert L.qmm_moe_route(ctypes.byref(m), None, 0, None) == 0
+    m.T = -1
+    assert L.qmm_moe(ctypes.byref(m), None, 0, None) == 1
+
+
 def test_moe_argument_checks(L):
     buf = (ctypes.c_char * 512)()
     a = (ctypes.addressof(buf) + 255) & ~255
