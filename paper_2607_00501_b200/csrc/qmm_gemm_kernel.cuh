@@ -401,16 +401,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         pdl_wait();                                                       // the output buffer may be in use upstream
         bool ok = true, etr = false;
         int it = 0, staged = 0;                                           // pieces seen / tiles that went through the staging buffer
-        const uint32_t stg_lane = smem_u32(staging) + (uint32_t)((quarter * 32 + lane) * 2);   // this thread's weight row
-        // 32 tokens (one chunk) of this thread's weight row -> staging[o][c0 + j][row]
+        const uint32_t stg_lane = smem_u32(staging) + (uint32_t)((quarter * 32 + lane) * 4);   // this thread's weight row
+        // 32 tokens (one chunk) of this thread's weight row -> staging[o][(c0 + 2j) / 2][row] as fp16
+        // pairs (tokens 2j, 2j+1 of one weight row share a 32-bit word: one store per converted pair)
         auto stage_chunk = [&](int o, int c0, const uint32_t (&v)[32]) {
-            const uint32_t dst = stg_lane + (uint32_t)((o * BN + c0) * 256);
+            const uint32_t dst = stg_lane + (uint32_t)(((o * BN + c0) >> 1) * 512);
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-                const uint32_t h = as_u32(__floats2half2_rn(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1])));
-                st_shared_b16(dst + (uint32_t)(2 * j * 256), (uint16_t)(h & 0xFFFFu));
-                st_shared_b16(dst + (uint32_t)((2 * j + 1) * 256), (uint16_t)(h >> 16));
-            }
+            for (int j = 0; j < 16; ++j)
+                st_shared_b32(dst + (uint32_t)(j * 512),
+                              as_u32(__floats2half2_rn(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]))));
         };
         auto release = [&]() {                                            // the next piece may overwrite the accumulators
             tc_fence_before_sync();
@@ -501,13 +500,22 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                     *reinterpret_cast<uint2*>(out + (size_t)r * p.ldo) = h;
                 }
             } else {
-                const int half = lane >> 4, seg = lane & 15;              // row of the pair, 16-byte segment of the row
+                // lanes 0-15: token row r, lanes 16-31: row r + 1 (the same staged words, the other half);
+                // a lane gathers the 8 weight rows of its 16-byte output segment from 8 words
+                const int half = lane >> 4, seg = lane & 15;
                 uint16_t* out = p.out + (size_t)w.row0 * p.ldo + (size_t)w.n_tile * 128 + seg * 8;
-                const uint32_t src = smem_u32(staging) + (uint32_t)(seg * 16);
+                const uint32_t src = smem_u32(staging) + (uint32_t)(seg * 32);
+                const uint32_t sel = half ? 0x7632u : 0x5410u;            // high / low fp16 of two words
 #pragma unroll
                 for (int o = 0; o < NOUT; ++o) {
                     for (int r = 2 * e + half; r < rows; r += 2 * NEPI) {
-                        const uint4 v = ld_shared_v4(src + (uint32_t)((o * BN + r) * 256));
+                        const uint32_t a = src + (uint32_t)(((o * BN + r) >> 1) * 512);
+                        const uint4 w0 = ld_shared_v4(a), w1 = ld_shared_v4(a + 16);
+                        uint4 v;
+                        v.x = __byte_perm(w0.x, w0.y, sel);
+                        v.y = __byte_perm(w0.z, w0.w, sel);
+                        v.z = __byte_perm(w1.x, w1.y, sel);
+                        v.w = __byte_perm(w1.z, w1.w, sel);
                         *reinterpret_cast<uint4*>(out + (size_t)r * p.ldo + (size_t)o * p.a_col_offset) = v;
                     }
                 }
