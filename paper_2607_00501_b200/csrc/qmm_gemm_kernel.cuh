@@ -17,17 +17,20 @@
 // tile (half the activation traffic; the gate and up matrices of an expert).
 //
 // Roles (warp specialised):
-//   expanders (8 warps): 8 / (4*NA) per weight tile and lane quarter,
-//                      alternating stages; thread = one weight row; 32-byte
-//                      code loads straight from global/L2, unpack to fp16(d*q),
-//                      tcgen05.st into the A ring in TMEM.
-//   epilogue (8 warps, two per lane quarter): tcgen05.ld the accumulators,
-//                      convert, stage the tile in shared memory, release the
-//                      accumulators, then store the tile with 16-byte rows.
+//   expanders (8 warps; 16 for token tiles of 64 and narrower): several per
+//                      weight tile and lane quarter, alternating stages;
+//                      thread = one weight row; 32-byte code loads straight
+//                      from global/L2, unpack to fp16(d*q), tcgen05.st into the
+//                      A ring in TMEM.
+//   epilogue (8 warps, two per lane quarter; 4 for narrow tiles): tcgen05.ld
+//                      the accumulators, convert, stage the tile in shared
+//                      memory, release the accumulators, then store the tile
+//                      with 16-byte row segments.
 //   TMA producer (1 warp): activation tiles -> shared-memory ring (128-byte
-//                      swizzle), one elected lane.
-//   MMA issuer (1 warp, converged): one elected lane issues tcgen05.mma
-//                      (M128 x N=BN x K16), frees ring slots with tcgen05.commit.
+//                      swizzle), one lane.
+//   MMA issuer (1 warp, converged): tcgen05.mma (M128 x N=BN x K16) and the
+//                      tcgen05.commit that frees a ring slot, predicated on one
+//                      elected lane (no divergent branch around them).
 // The kernel is persistent: a block loops over tiles and the pipeline runs on
 // across tile boundaries.
 //
