@@ -1,0 +1,61 @@
+"""GPU parity on seeded random shapes: every supported (N % 128 == 0, K % 256 == 0, any M / T)
+combination goes through the same tolerance as the fixed cases -- shapes nobody picked by hand."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2607_00501_b200 import synth
+from tests import util
+from tests.test_gpu_moe import Layer, check_stages, run_layer
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def qmm():
+    from paper_2607_00501_b200 import qmm as _qmm
+    assert torch.cuda.is_available()
+    _qmm.lib()
+    return _qmm
+
+
+
+@pytest.mark.parametrize("case", range(12))
+def test_random_gemv_shapes(qmm, oracle, case):
+    rng = np.random.default_rng([811, case])
+    fmt = int(rng.choice([4, 8]))
+    N, K = int(rng.integers(1, 24)) * 128, int(rng.integers(1, 33)) * 256
+    blocks = synth.quantize(fmt, synth.weights(812, case, N, K))
+    x = synth.activations(813, case, K)
+    y = qmm.gemv(fmt, qmm.pack(fmt, util.dev(blocks), N, K), N, K, util.dev(x))
+    y_ref, B = oracle.gemv(fmt, blocks, N, K, x)
+    util.assert_within_tol(util.host_f64(y), y_ref, B, "gemv fmt=%d N=%d K=%d" % (fmt, N, K))
+
+
+@pytest.mark.parametrize("case", range(16))
+def test_random_gemm_shapes(qmm, oracle, case):
+    rng = np.random.default_rng([821, case])
+    fmt = int(rng.choice([4, 8]))
+    M, N, K = int(rng.integers(1, 700)), int(rng.integers(1, 20)) * 128, int(rng.integers(1, 17)) * 256
+    blocks = synth.quantize(fmt, synth.weights(822, case, N, K))
+    X = synth.activations(823, case, M, K)
+    ws = torch.zeros(qmm.gemm_workspace_bytes(fmt, M, N, K), dtype=torch.uint8, device="cuda")
+    Y = qmm.gemm(fmt, qmm.pack(fmt, util.dev(blocks), N, K), N, K, util.dev(X), ws=ws)
+    qmm.status_check(ws)
+    Y_ref, B = oracle.gemm(fmt, blocks, N, K, X)
+    util.assert_within_tol(util.host_f64(Y), Y_ref, B, "gemm fmt=%d M=%d N=%d K=%d" % (fmt, M, N, K))
+
+
+@pytest.mark.parametrize("case", range(6))
+def test_random_moe_layers(qmm, oracle, case):
+    rng = np.random.default_rng([831, case])
+    fmt = int(rng.choice([4, 8]))
+    E = int(rng.choice([4, 8, 32, 128]))
+    topk = int(rng.integers(1, min(E, 8) + 1))
+    T, H, I = int(rng.integers(1, 300)), int(rng.integers(1, 5)) * 256, int(rng.integers(1, 5)) * 256
+    L = Layer(qmm, fmt, 832 + case, E, H, I)
+    X = synth.activations(833, case, T, H)
+    logits = synth.logits(834, case, T, E)
+    res = run_layer(qmm, L, logits, X, topk)
+    experts = sorted({int(e) for e in rng.integers(0, E, size=min(E, 6))})
+    check_stages(oracle, L, res, logits, X, topk, experts=experts, rows_per_expert=8, tokens=list(range(min(T, 5))))
