@@ -33,7 +33,7 @@ def run_gemm(qmm, oracle, fmt, blocks, N, K, X, what, rows=None):
 
 @pytest.mark.parametrize("fmt", [Q4, Q8])
 @pytest.mark.parametrize("M,N,K", [(128, 128, 256), (32, 256, 256), (1, 128, 512), (77, 384, 768), (130, 256, 1024),
-                                   (200, 640, 512), (64, 128, 4096), (700, 6400, 512), (1000, 1280, 256)])
+                                   (200, 640, 512), (64, 128, 4096), (700, 6400, 512), (1000, 1280, 256), (4100, 256, 256)])
 def test_gemm_small_shapes(qmm, oracle, fmt, M, N, K):
     blocks, _, _ = util.random_blocks(synth, fmt, N, K, seed=M + 3 * N + K + fmt, special_scales=False)
     X = synth.activations(70, M + N + K, M, K)

@@ -132,7 +132,7 @@ def check_end_to_end(oracle, L, res, logits, X, topk, tokens):
 @pytest.mark.parametrize("fmt", [Q4, Q8])
 @pytest.mark.parametrize("T,E,topk,H,I", [(1, 8, 2, 256, 256), (5, 8, 2, 256, 256), (4, 128, 8, 256, 256),
                                           (5, 128, 8, 512, 256), (37, 16, 4, 512, 256), (200, 8, 2, 256, 512),
-                                          (64, 32, 8, 256, 256)])
+                                          (64, 32, 8, 256, 256), (400, 4, 2, 256, 256)])
 def test_moe_small_layers_every_row(qmm, oracle, fmt, T, E, topk, H, I):
     L = Layer(qmm, fmt, 500 + T + E, E, H, I)
     X = synth.activations(501, T, T, H)
