@@ -606,13 +606,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                             // descriptor start address is in 16-byte units: slot s is s * B_STAGE / 16 further, k-step k is 2 further
                             const uint64_t desc_s = desc0 + (uint64_t)(sj * (B_STAGE >> 4));
                             const uint32_t a_s = tmem_base + (uint32_t)(RING0 + sj * A_COLS);
+                            static_assert(kGemmBK == 64, "four K = 16 steps per stage");
 #pragma unroll
-                            for (int a = 0; a < NA; ++a) {
-#pragma unroll
-                                for (int k = 0; k < kGemmBK / 16; ++k)
-                                    mma_ts_f16_sel(d_tmem + (uint32_t)(a * BN), a_s + (uint32_t)(a * 32 + k * 8), desc_s + (uint64_t)(k * 2),
-                                                   idesc, kb + j != w.kb0 || k != 0, sel);
-                            }
+                            for (int a = 0; a < NA; ++a)
+                                mma_ts_f16_stage(d_tmem + (uint32_t)(a * BN), a_s + (uint32_t)(a * 32), desc_s, idesc, kb + j != w.kb0, sel);
                             mma_commit_sel(&empty[sj], sel);              // slot reusable when these MMAs finish
                         }
                     }

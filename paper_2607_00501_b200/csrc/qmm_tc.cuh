@@ -204,34 +204,40 @@ __host__ __device__ constexpr uint32_t idesc_f16_m128(int n)
     return (1u << 4) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
 
-// D[tmem] (+)= A[tmem] * B[smem]^T, one K = 16 step.  One thread issues.
-__device__ __forceinline__ void mma_ts_f16(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, bool accumulate)
+// D[tmem] (+)= A[tmem] * B[smem]^T.  The MMAs and commits of the issuing warp are executed by the
+// whole converged warp with only the lane `sel != 0` acting (predicated instructions instead of a
+// divergent branch).
+//
+// All MMAs of one 64-k stage for one weight tile set (four K = 16 steps) in one block of
+// instructions: the predicates are set up once, the operands of the four steps are the first
+// step's plus constants (8 tensor-memory columns, 2 descriptor units per step).  `first_acc` =
+// accumulate flag of the first step (false at the start of a piece of work); the others accumulate.
+__device__ __forceinline__ void mma_ts_f16_stage(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, bool first_acc,
+                                                 uint32_t sel)
 {
     asm volatile(
         "{\n\t"
-        ".reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t"
-        "}\n"
-        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate)
-        : "memory");
-}
-
-// The same two operations executed by a whole converged warp with only the lane `sel != 0` issuing
-// (predicated instruction instead of a divergent branch).
-__device__ __forceinline__ void mma_ts_f16_sel(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, bool accumulate,
-                                               uint32_t sel)
-{
-    asm volatile(
-        "{\n\t"
-        ".reg .pred p, q;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
+        ".reg .pred q, p0, pt;\n\t"
+        ".reg .b32 a1, a2, a3;\n\t"
+        ".reg .b64 b1, b2, b3;\n\t"
         "setp.ne.b32 q, %5, 0;\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t"
+        "setp.ne.b32 p0, %4, 0;\n\t"
+        "setp.eq.b32 pt, %5, %5;\n\t"
+        "add.u32 a1, %1, 8;\n\t"
+        "add.u32 a2, %1, 16;\n\t"
+        "add.u32 a3, %1, 24;\n\t"
+        "add.u64 b1, %2, 2;\n\t"
+        "add.u64 b2, %2, 4;\n\t"
+        "add.u64 b3, %2, 6;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [a1], b1, %3, pt;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [a2], b2, %3, pt;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [a3], b3, %3, pt;\n\t"
         "}\n"
-        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate), "r"(sel)
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"((uint32_t)first_acc), "r"(sel)
         : "memory");
 }
+// Arrive on an mbarrier once every MMA issued so far by the acting lane has finished.
 __device__ __forceinline__ void mma_commit_sel(uint64_t* bar, uint32_t sel)
 {
     asm volatile(
@@ -242,13 +248,6 @@ __device__ __forceinline__ void mma_commit_sel(uint64_t* bar, uint32_t sel)
         "}\n"
         ::"r"(smem_u32(bar)), "r"(sel)
         : "memory");
-}
-
-// Arrive on an mbarrier once every MMA issued so far by this thread has finished.
-__device__ __forceinline__ void mma_commit(uint64_t* bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
-                 : "memory");
 }
 
 }  // namespace tc
