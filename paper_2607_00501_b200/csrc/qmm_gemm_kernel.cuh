@@ -167,6 +167,14 @@ template <> struct RawRow64<QMM_Q8> {
 #ifndef QMM_GEMM_L2_AHEAD
 #define QMM_GEMM_L2_AHEAD 6
 #endif
+// Clock samples of the issuing loop of block 0 (tuning aid): compiled in only with -DQMM_GEMM_TRACE_MMA=1,
+// because even a skipped sample costs the issuing warp instructions in its critical loop.
+#if defined(QMM_GEMM_TRACE_MMA) && QMM_GEMM_TRACE_MMA
+#define QMM_TRACE_MMA(slot) \
+    if (tracing && g + 1 < 64) p.trace[g * 8 + (slot)] = p.trace[(g + 1) * 8 + (slot)] = clock64();
+#else
+#define QMM_TRACE_MMA(slot)
+#endif
 constexpr int kGemmPrefetch = QMM_GEMM_PREFETCH;   // weight slices in flight per expander thread
 constexpr int kGemmL2Ahead = QMM_GEMM_L2_AHEAD;    // stages of a row group's weight stream requested into L2 ahead of use
 
@@ -338,6 +346,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         constexpr int TILES_PER_KB = kGemmBK / Fmt<FMT>::tile_k;
         const size_t kb_bytes = (size_t)TILES_PER_KB * Fmt<FMT>::tile_bytes;
         const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);
+        const uint8_t* wmat = (NA == 2 && a == 1) ? p.w[1] : p.w[0];      // (not p.w[a]: indexing a kernel parameter by a run-time value copies the parameters to local memory)
         Q4Consts kc;
         kc.init();
         bool ok = true;
@@ -346,7 +355,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         for (int i = 0; ok && get_work(i, w); ++i) {
             const int num_kb = w.kb1 - w.kb0;
             const int rg = w.n_tile * 4 + quarter;                        // row group of 32 rows
-            const uint8_t* wrow = p.w[a] + (size_t)w.expert * p.w_expert_stride + (size_t)rg * tpr * Fmt<FMT>::tile_bytes +
+            const uint8_t* wrow = wmat + (size_t)w.expert * p.w_expert_stride + (size_t)rg * tpr * Fmt<FMT>::tile_bytes +
                                   (size_t)w.kb0 * kb_bytes;                // this piece's part of the row group's stream
             // The weight stream of a row group is contiguous: ask L2 for it kGemmL2Ahead stages ahead
             // (expert weights come from HBM; two register-held slices alone do not cover that latency).
@@ -567,6 +576,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         // divergent branch: measured ~25 % less issue time per stage (operands stay warp-uniform).
         const uint32_t sel = elect_one() ? 1u : 0u;
         const bool tracing = p.trace != nullptr && blockIdx.x == 0 && lane == 0;
+        (void)tracing;
+        (void)g;
         int s = 0;                                                        // ring slot of stage g and the parity of its
         uint32_t par = 0;                                                 // "full" barrier, carried across pieces
         GemmWork w;
@@ -580,54 +591,64 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                 if (p.trace != nullptr && blockIdx.x == 0 && it <= 16 && lane == 0) p.trace[((it - AB) * 4 + 3) * 8 + 1] = clock64();
             }
             const uint32_t d_tmem = tmem_base + (uint32_t)(buf * D_COLS);
-            // Two stages per round when the ring is deep enough and the piece has them: the barrier
-            // polls, the warp vote and the fence are paid once per 128 k.
-            for (int kb = w.kb0; kb < w.kb1;) {
-                const int n = (S >= 6 && w.kb1 - kb >= 2) ? 2 : 1;         // (a short ring is consumed one stage at a time)
-                int s1 = s + 1;
-                uint32_t par1 = par;
-                if (s1 == S) {
-                    s1 = 0;
-                    par1 ^= 1;
-                }
-                const bool tr = tracing && g + 1 < 64;
-                if (tr) p.trace[g * 8 + 0] = p.trace[(g + 1) * 8 + 0] = clock64();
-                ok = mbar_wait(&full[s], par, abort_flag);
-                if (n == 2 && ok) ok = mbar_wait(&full[s1], par1, abort_flag);
-                ok = __all_sync(0xFFFFFFFFu, ok);
-                if (tr) p.trace[g * 8 + 2] = p.trace[(g + 1) * 8 + 2] = clock64();
-                if (!ok) break;
-                tc_fence_after_sync();
-                {
+            // One round of the loop = wait for the slot(s), vote, fence, MMAs, commit(s).  Two stages per
+            // round when the ring is deep enough (the polls, the vote and the fence are paid once per
+            // 128 k), then single stages for what is left of the piece.  Both bodies are straight-line
+            // code: a common body with a run-time stage count per round was measured at ~100 cycles more
+            // per stage in the issuing warp, which the short MMA queue does not hide.
+            static_assert(kGemmBK == 64, "four K = 16 steps per stage");
+            // MMAs of stage kb from ring slot sj (descriptor start address is in 16-byte units: slot s is
+            // s * B_STAGE / 16 further), then the commit that frees the slot
+            auto issue_stage = [&](int sj, bool acc) {
+                const uint64_t desc_s = desc0 + (uint64_t)(sj * (B_STAGE >> 4));
+                const uint32_t a_s = tmem_base + (uint32_t)(RING0 + sj * A_COLS);
 #pragma unroll
-                    for (int j = 0; j < 2; ++j) {
-                        if (j < n) {                                      // uniform
-                            const int sj = j == 0 ? s : s1;
-                            // descriptor start address is in 16-byte units: slot s is s * B_STAGE / 16 further, k-step k is 2 further
-                            const uint64_t desc_s = desc0 + (uint64_t)(sj * (B_STAGE >> 4));
-                            const uint32_t a_s = tmem_base + (uint32_t)(RING0 + sj * A_COLS);
-                            static_assert(kGemmBK == 64, "four K = 16 steps per stage");
-#pragma unroll
-                            for (int a = 0; a < NA; ++a)
-                                mma_ts_f16_stage(d_tmem + (uint32_t)(a * BN), a_s + (uint32_t)(a * 32), desc_s, idesc, kb + j != w.kb0, sel);
-                            mma_commit_sel(&empty[sj], sel);              // slot reusable when these MMAs finish
-                        }
+                for (int a = 0; a < NA; ++a) mma_ts_f16_stage(d_tmem + (uint32_t)(a * BN), a_s + (uint32_t)(a * 32), desc_s, idesc, acc, sel);
+                mma_commit_sel(&empty[sj], sel);                          // slot reusable when these MMAs finish
+            };
+            int kb = w.kb0;
+            if constexpr (S >= 6) {
+                for (; kb + 2 <= w.kb1 && ok; kb += 2) {
+                    int s1 = s + 1;
+                    uint32_t par1 = par;
+                    if (s1 == S) {
+                        s1 = 0;
+                        par1 ^= 1;
                     }
-                }
-                __syncwarp();
-                if (tr) p.trace[g * 8 + 3] = p.trace[(g + 1) * 8 + 3] = clock64();
-                kb += n;
-                g += n;
-                if (n == 2) {
+                    QMM_TRACE_MMA(0)
+                    ok = mbar_wait(&full[s], par, abort_flag);
+                    if (ok) ok = mbar_wait(&full[s1], par1, abort_flag);
+                    ok = __all_sync(0xFFFFFFFFu, ok);
+                    QMM_TRACE_MMA(2)
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    issue_stage(s, kb != w.kb0);
+                    issue_stage(s1, true);
+                    __syncwarp();
+                    QMM_TRACE_MMA(3)
+                    g += 2;
                     s = s1 + 1;
                     par = par1;
                     if (s == S) {
                         s = 0;
                         par ^= 1;
                     }
-                } else {
-                    s = s1;
-                    par = par1;
+                }
+            }
+            for (; kb < w.kb1 && ok; ++kb) {
+                QMM_TRACE_MMA(0)
+                ok = mbar_wait(&full[s], par, abort_flag);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                QMM_TRACE_MMA(2)
+                if (!ok) break;
+                tc_fence_after_sync();
+                issue_stage(s, kb != w.kb0);
+                __syncwarp();
+                QMM_TRACE_MMA(3)
+                ++g;
+                if (++s == S) {
+                    s = 0;
+                    par ^= 1;
                 }
             }
             if (ok) mma_commit_sel(&acc_full[buf], sel);                  // accumulators of this piece are complete
