@@ -48,6 +48,7 @@
 namespace qmm {
 
 constexpr int kGemmBK = 64;          // k per pipeline stage
+constexpr int kGemmMaxStagesB = 8;    // depth of the activation ring where it is a ring of its own
 constexpr int kGemmMaxStages = 6;     // pipeline depth is min(this, what tensor memory leaves for the weight ring)
 
 enum GemmEpilogue { kEpiStore = 0, kEpiSiluMul = 1 };
@@ -87,20 +88,28 @@ struct GemmGeom {
     static constexpr int kAccBufs = (2 * kDCols + 4 * kACols <= kTmemCols) ? 2 : 1;
     static constexpr int kFit = (kTmemCols - kAccBufs * kDCols) / kACols;
     static constexpr int kBStage = BN * kGemmBK * 2;                       // bytes per activation slot
-    // the epilogue stages a finished tile in shared memory, [tile set][token][128 weight rows]: fp16
-    // outputs (plain store), or the fp32 gate and up accumulators (SiLU*mul is applied on the way out)
-    static constexpr int kStaging = NA * BN * 128 * (EPI == kEpiSiluMul ? 4 : 2);
+    // the epilogue stages a finished tile in shared memory as fp16, [tile set][token pair][128 weight
+    // rows] (32-bit words of two tokens): the outputs (plain store), or the gate and up accumulators
+    // (SiLU*mul is applied on the way out)
+    static constexpr int kStaging = NA * BN * 128 * 2;
     static constexpr int kSmemMax = 227 * 1024;                            // per block on sm_100
-    static constexpr int kSmemFit = (kSmemMax - 1024 - 256 - kStaging) / kBStage;
-    static constexpr int kFit2 = kFit < kSmemFit ? kFit : kSmemFit;
-    static constexpr int kStages = kFit2 < kGemmMaxStages ? kFit2 : kGemmMaxStages;
-    static constexpr int kSmemBytes = kStages * kBStage + kStaging + 1024 /*align*/ + 256;
+    static constexpr int kSmemFit = (kSmemMax - 1024 - 512 - kStaging) / kBStage;
+    // With two weight tile sets tensor memory leaves a ring of three or four weight slots; an
+    // activation tile takes ~1 800 cycles from the TMA request to its barrier, so a ring that shallow
+    // for the activations bounds a stage at (MMA time + that latency) / slots.  The activation tiles
+    // then get a ring of their own in shared memory with barriers of their own (kSplit), as deep as
+    // shared memory allows; else one ring and one pair of barriers per stage serve both operands.
+    static constexpr bool kSplit = NA == 2 && BN >= 128;                   // (narrower tiles: the extra waits and commits cost the issuing loop more than the latency they hide)
+    static constexpr int kFit2 = kSplit ? kFit : (kFit < kSmemFit ? kFit : kSmemFit);
+    static constexpr int kStages = kFit2 < kGemmMaxStages ? kFit2 : kGemmMaxStages;             // weight slots (and activation slots unless kSplit)
+    static constexpr int kStagesB = !kSplit ? kStages : (kSmemFit < kGemmMaxStagesB ? kSmemFit : kGemmMaxStagesB);
+    static constexpr int kSmemBytes = kStagesB * kBStage + kStaging + 1024 /*align*/ + 512;
     // Warp roles: expanders, epilogue warps (one or two per TMEM lane quarter), TMA producer, MMA
     // issuer.  Narrow token tiles are bound by the expansion, not by the epilogue: 16 + 4 there.
-    static constexpr int kExpWarps = BN <= 64 ? 16 : 8;
-    static constexpr int kEpiWarps = BN <= 64 ? 4 : 8;
+    static constexpr int kExpWarps = (BN <= 64 || NA == 2) ? 16 : 8;
+    static constexpr int kEpiWarps = (BN <= 64 || NA == 2) ? 4 : 8;
     static constexpr int kThreads = (kExpWarps + kEpiWarps + 2) * 32;
-    static_assert(kStages >= 2, "tensor memory over-subscribed");
+    static_assert(kStages >= 2 && kStagesB >= 2, "tensor memory or shared memory over-subscribed");
 };
 
 // silu(g) = g / (1 + exp(-g)) with the fast exponential and reciprocal (relative error ~1e-6,
@@ -232,7 +241,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
     constexpr int PH = NEXP / (4 * NA);               // expander warps per (weight tile, lane quarter): they alternate stages
     constexpr int NEPI = G::kEpiWarps;
     constexpr int TMA_WARP = NEXP + NEPI, MMA_WARP = NEXP + NEPI + 1;
-    constexpr int S = G::kStages;                     // pipeline depth
+    constexpr int S = G::kStages;                     // pipeline depth (weight slots)
+    constexpr bool SPLIT = G::kSplit;                 // activation tiles in a ring of their own
+    constexpr int SB = G::kStagesB;                   // its depth (== S unless SPLIT)
     constexpr int A_COLS = G::kACols;
     constexpr int D_COLS = G::kDCols;
     constexpr int TMEM_COLS = G::kTmemCols;
@@ -245,7 +256,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* smem_b = smem;                                               // S slots, 1024-aligned each
-    uint8_t* staging = smem + S * B_STAGE;                                // finished tile, fp16 [output tile][token][128 rows]
+    uint8_t* staging = smem + SB * B_STAGE;                               // finished tile, fp16 [output tile][token pair][128 rows]
     uint64_t* bars = reinterpret_cast<uint64_t*>(staging + G::kStaging);
     uint64_t* full = bars;                                                // [S] expanders + TMA -> MMA
     uint64_t* empty = bars + S;                                           // [S] MMA -> expanders, TMA
@@ -253,7 +264,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
     uint64_t* acc_empty = bars + 2 * S + 2;                               // [2] epilogue -> MMA
     uint64_t* stg_full = bars + 2 * S + 4;                                // epilogue warps: tile staged
     uint64_t* stg_empty = bars + 2 * S + 5;                               // epilogue warps: staged tile stored
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 6);
+    uint64_t* full_b = bars + 2 * S + 6;                                  // [SB] TMA -> MMA          (SPLIT only)
+    uint64_t* empty_b = bars + 2 * S + 6 + SB;                            // [SB] MMA -> TMA          (SPLIT only)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 6 + 2 * SB);
+    static_assert((2 * S + 6 + 2 * SB + 1) * 8 <= 512, "barrier area");
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -269,9 +283,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
     // ---- set-up
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
-            mbar_init(&full[s], 4 * NA + 1);                              // the stage's expander warps + the TMA producer
+            mbar_init(&full[s], 4 * NA + (SPLIT ? 0 : 1));                // the stage's expander warps (+ the TMA producer)
             mbar_init(&empty[s], 1);                                      // one tcgen05.commit
         }
+        if (SPLIT)
+            for (int s = 0; s < SB; ++s) {
+                mbar_init(&full_b[s], 1);                                 // the TMA producer (+ its bytes)
+                mbar_init(&empty_b[s], 1);                                // one tcgen05.commit
+            }
         for (int b = 0; b < 2; ++b) {
             mbar_init(&acc_full[b], 1);
             mbar_init(&acc_empty[b], NEPI);
@@ -410,6 +429,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         constexpr int NCH = BN / 32;                                      // 32-column chunks of the tile
         constexpr int CH = (NCH + GROUPS - 1) / GROUPS;                   // chunks per warp
         constexpr int NOUT = (EPI == kEpiSiluMul) ? 1 : NA;               // output tiles per weight row
+        constexpr int NSTG = NA;                                          // tile sets that go through the staging buffer
         pdl_wait();                                                       // the output buffer may be in use upstream
         bool ok = true, etr = false;
         int it = 0, staged = 0;                                           // pieces seen / tiles that went through the staging buffer
@@ -451,30 +471,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
             }
-            if constexpr (EPI == kEpiSiluMul) {
-                // gate and up accumulators go to the staging buffer as they are (fp32); SiLU*mul is
-                // applied when the tile is stored, after the accumulators have been handed back
-#pragma unroll
-                for (int c = 0; c < CH; ++c) {
-                    const int c0 = (grp * CH + c) * 32;
-                    if (c0 < BN && c0 < rows) {                           // uniform over the warp
-                        uint32_t g[32], u[32];
-                        tmem_ld_32x32b_x32(lane_base + (uint32_t)c0, g);
-                        tmem_ld_32x32b_x32(lane_base + (uint32_t)(BN + c0), u);
-                        tmem_wait_ld();
-                        const uint32_t dg = smem_u32(staging) + (uint32_t)(c0 * 512 + (quarter * 32 + lane) * 4);
-                        const uint32_t du = dg + (uint32_t)(BN * 512);
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            st_shared_b32(dg + (uint32_t)(j * 512), g[j]);
-                            st_shared_b32(du + (uint32_t)(j * 512), u[j]);
-                        }
-                    }
-                }
-            } else {
+            {
+                // (SiLU*mul: the gate and up accumulators are staged as fp16 and combined when the tile
+                // is stored, after the accumulators have been handed back)
                 // two chunk loads in flight per wait (an invalid second chunk re-reads the first and is dropped)
 #pragma unroll
-                for (int o = 0; o < NOUT; ++o) {
+                for (int o = 0; o < NSTG; ++o) {
 #pragma unroll
                     for (int c = 0; c < CH; c += 2) {
                         const int c0 = (grp * CH + c) * 32, c1 = c0 + 32;
@@ -498,18 +500,32 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
             if constexpr (EPI == kEpiSiluMul) {
-                // one token row (128 weight rows: 4 per lane) per warp instruction
+                // two token rows per warp instruction: a lane combines the gate and up values of its 4
+                // weight rows for tokens 2 rp, 2 rp + 1 (one 16-byte read each) and stores 8 bytes per row
                 uint16_t* out = p.out + (size_t)w.row0 * p.ldo + (size_t)w.n_tile * 128 + lane * 4;
                 const uint32_t src = smem_u32(staging) + (uint32_t)(lane * 16);
-                for (int r = e; r < rows; r += NEPI) {
-                    const uint4 g = ld_shared_v4(src + (uint32_t)(r * 512));
-                    const uint4 u = ld_shared_v4(src + (uint32_t)((BN + r) * 512));
+                auto silu_mul = [](uint32_t g, uint32_t u, float& lo, float& hi) {    // words of two tokens
+                    const float2 gf = __half22float2(as_h2(g)), uf = __half22float2(as_h2(u));
+                    lo = silu_f(gf.x) * uf.x;
+                    hi = silu_f(gf.y) * uf.y;
+                };
+                for (int rp = e; 2 * rp < rows; rp += NEPI) {
+                    const uint4 g = ld_shared_v4(src + (uint32_t)(rp * 512));
+                    const uint4 u = ld_shared_v4(src + (uint32_t)(((BN >> 1) + rp) * 512));
+                    float a0, b0, a1, b1, a2, b2, a3, b3;                 // a: token 2 rp, b: token 2 rp + 1
+                    silu_mul(g.x, u.x, a0, b0);
+                    silu_mul(g.y, u.y, a1, b1);
+                    silu_mul(g.z, u.z, a2, b2);
+                    silu_mul(g.w, u.w, a3, b3);
                     uint2 h;
-                    h.x = as_u32(__floats2half2_rn(silu_f(__uint_as_float(g.x)) * __uint_as_float(u.x),
-                                                   silu_f(__uint_as_float(g.y)) * __uint_as_float(u.y)));
-                    h.y = as_u32(__floats2half2_rn(silu_f(__uint_as_float(g.z)) * __uint_as_float(u.z),
-                                                   silu_f(__uint_as_float(g.w)) * __uint_as_float(u.w)));
-                    *reinterpret_cast<uint2*>(out + (size_t)r * p.ldo) = h;
+                    h.x = as_u32(__floats2half2_rn(a0, a1));
+                    h.y = as_u32(__floats2half2_rn(a2, a3));
+                    *reinterpret_cast<uint2*>(out + (size_t)(2 * rp) * p.ldo) = h;
+                    if (2 * rp + 1 < rows) {
+                        h.x = as_u32(__floats2half2_rn(b0, b1));
+                        h.y = as_u32(__floats2half2_rn(b2, b3));
+                        *reinterpret_cast<uint2*>(out + (size_t)(2 * rp + 1) * p.ldo) = h;
+                    }
                 }
             } else {
                 // lanes 0-15: token row r, lanes 16-31: row r + 1 (the same staged words, the other half);
@@ -546,11 +562,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             GemmWork w;
             for (int i = 0; ok && get_work(i, w); ++i) {
                 for (int kb = w.kb0; kb < w.kb1; ++kb, ++g) {
-                    const int s = g % S;
-                    if (g >= S) ok = mbar_wait(&empty[s], ((g / S) - 1) & 1, abort_flag);
+                    const int s = g % SB;
+                    uint64_t* slot_full = SPLIT ? &full_b[s] : &full[s];
+                    if (g >= SB) ok = mbar_wait(SPLIT ? &empty_b[s] : &empty[s], ((g / SB) - 1) & 1, abort_flag);
                     if (!ok) break;
-                    mbar_arrive_expect_tx(&full[s], B_STAGE);
-                    tma_load_2d(smem_b + s * B_STAGE, &x_map, kb * kGemmBK, w.row0, &full[s]);
+                    mbar_arrive_expect_tx(slot_full, B_STAGE);
+                    tma_load_2d(smem_b + s * B_STAGE, &x_map, kb * kGemmBK, w.row0, slot_full);
                     issued = g + 1;
                 }
             }
@@ -558,9 +575,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                 *abort_flag = 1;
                 // let loads in flight land before the block's shared memory is released
                 // (the same barrier also counts expander arrivals, so this can run into its time limit)
-                for (int q = max(0, issued - S); q < issued; ++q) {
+                for (int q = max(0, issued - SB); q < issued; ++q) {
                     const long long t0 = clock64();
-                    while (!mbar_try_wait(&full[q % S], (q / S) & 1) && clock64() - t0 < (1LL << 22)) {}
+                    while (!mbar_try_wait(SPLIT ? &full_b[q % SB] : &full[q % S], (q / SB) & 1) && clock64() - t0 < (1LL << 22)) {}
                 }
             }
         }
@@ -580,6 +597,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         (void)g;
         int s = 0;                                                        // ring slot of stage g and the parity of its
         uint32_t par = 0;                                                 // "full" barrier, carried across pieces
+        int sb = 0;                                                       // the same for the activation ring (SPLIT)
+        uint32_t parb = 0;
         GemmWork w;
         for (; ok && get_work(it, w); ++it) {
             const int buf = it % AB;
@@ -600,11 +619,18 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             // MMAs of stage kb from ring slot sj (descriptor start address is in 16-byte units: slot s is
             // s * B_STAGE / 16 further), then the commit that frees the slot
             auto issue_stage = [&](int sj, bool acc) {
-                const uint64_t desc_s = desc0 + (uint64_t)(sj * (B_STAGE >> 4));
+                const uint64_t desc_s = desc0 + (uint64_t)((SPLIT ? sb : sj) * (B_STAGE >> 4));
                 const uint32_t a_s = tmem_base + (uint32_t)(RING0 + sj * A_COLS);
 #pragma unroll
                 for (int a = 0; a < NA; ++a) mma_ts_f16_stage(d_tmem + (uint32_t)(a * BN), a_s + (uint32_t)(a * 32), desc_s, idesc, acc, sel);
                 mma_commit_sel(&empty[sj], sel);                          // slot reusable when these MMAs finish
+                if constexpr (SPLIT) mma_commit_sel(&empty_b[sb], sel);
+            };
+            auto next_b = [&]() {                                         // advance the activation ring (SPLIT)
+                if (++sb == SB) {
+                    sb = 0;
+                    parb ^= 1;
+                }
             };
             int kb = w.kb0;
             if constexpr (S >= 6) {
@@ -618,12 +644,24 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                     QMM_TRACE_MMA(0)
                     ok = mbar_wait(&full[s], par, abort_flag);
                     if (ok) ok = mbar_wait(&full[s1], par1, abort_flag);
+                    if constexpr (SPLIT) {
+                        int sb1 = sb + 1;
+                        uint32_t parb1 = parb;
+                        if (sb1 == SB) {
+                            sb1 = 0;
+                            parb1 ^= 1;
+                        }
+                        if (ok) ok = mbar_wait(&full_b[sb], parb, abort_flag);
+                        if (ok) ok = mbar_wait(&full_b[sb1], parb1, abort_flag);
+                    }
                     ok = __all_sync(0xFFFFFFFFu, ok);
                     QMM_TRACE_MMA(2)
                     if (!ok) break;
                     tc_fence_after_sync();
                     issue_stage(s, kb != w.kb0);
+                    if constexpr (SPLIT) next_b();
                     issue_stage(s1, true);
+                    if constexpr (SPLIT) next_b();
                     __syncwarp();
                     QMM_TRACE_MMA(3)
                     g += 2;
@@ -638,6 +676,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             for (; kb < w.kb1 && ok; ++kb) {
                 QMM_TRACE_MMA(0)
                 ok = mbar_wait(&full[s], par, abort_flag);
+                if constexpr (SPLIT) {
+                    if (ok) ok = mbar_wait(&full_b[sb], parb, abort_flag);
+                }
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 QMM_TRACE_MMA(2)
                 if (!ok) break;
@@ -650,6 +691,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                     s = 0;
                     par ^= 1;
                 }
+                if constexpr (SPLIT) next_b();
             }
             if (ok) mma_commit_sel(&acc_full[buf], sel);                  // accumulators of this piece are complete
             __syncwarp();
