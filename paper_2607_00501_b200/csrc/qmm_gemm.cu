@@ -138,15 +138,15 @@ int pick_expert_tile(int64_t total_rows, int experts)
 // ascending order (a fixed order: same bits on every call), and stores fp16.  Block (t, y): token columns [8 y, 8 y + 8) of tile t; a
 // thread adds one float4 (4 weight rows of one token) per output tile, so every load is in flight at once.
 __global__ void gemm_cut_reduce_kernel(const float* __restrict__ partial, uint16_t* __restrict__ Y, int64_t ldy, int M,
-                                       int bn, int nout, int a_col_offset, int n_tiles, int KB, int U)
+                                       int bn, int nout, int a_col_offset, int n_tiles, int KB, int U, int t0)
 {
     pdl_launch_dependents();
     pdl_wait();
-    const int t = blockIdx.x, c0 = blockIdx.y * 8;
+    const int t = t0 + blockIdx.x, c0 = blockIdx.y * 8;                   // the tiles dealt in unit shares start at t0
     const int n_tile = t % n_tiles, row0 = (t / n_tiles) * bn;
     const int rows = min(bn, M - row0);
     if (c0 >= rows) return;
-    const long long tb = (long long)t * KB;
+    const long long tb = (long long)blockIdx.x * KB;
     const int first = (int)(tb / U);
     const int cn = (int)((tb + KB - 1) / U) - first + 1;
     if (cn == 1) return;                                                  // a whole tile: stored by the GEMM itself
@@ -173,10 +173,36 @@ __global__ void gemm_cut_reduce_kernel(const float* __restrict__ partial, uint16
 // Shape -> tiling and work split of the dense GEMM.
 struct GemmPlan {
     int bn, na;
-    int units;          // (tile, k-block) units per block
+    int whole;          // tiles dealt whole, the same number to every block (a multiple of grid)
+    int units;          // (tile, k-block) units per block of the remaining tiles
     int grid;           // blocks
     bool cut;           // some tile is shared between blocks: partial-sum slots and the second kernel
 };
+
+// Cycles of one block for `tiles` tiles of `kb` k-blocks on the SMs: whole rounds, then the last,
+// partly filled round either as whole tiles or -- when that saves more than the partial sums and
+// the second kernel cost (~18 000 cycles, measured) -- cut into equal shares of its (tile, k-block) units.
+struct RoundCost {
+    int64_t cycles;
+    bool cut_tail;
+};
+static RoundCost round_cost(int64_t tiles, int64_t kb, int64_t stage, int64_t handover)
+{
+    const int64_t tile = kb * stage + handover;
+    const int64_t rounds = tiles / kNumSMs, tail = tiles % kNumSMs;
+    RoundCost r = {rounds * tile, false};
+    if (tail == 0) return r;
+    int64_t share = (tail * kb + kNumSMs - 1) / kNumSMs;
+    if (share < 8) share = 8;
+    const int64_t cut = share * stage + 2 * handover + 18000;
+    if (rounds >= 1 && cut < tile) {
+        r.cycles += cut;
+        r.cut_tail = true;
+    } else {
+        r.cycles += tile;
+    }
+    return r;
+}
 
 // Workspace of qmm_gemm: [0, 4) status word, [4096, 8192) trace samples (tuning aid), then the
 // partial-sum slots.
@@ -211,9 +237,7 @@ static GemmPlan gemm_plan(int64_t M, int64_t N, int64_t K)
     if (p.bn == 256 && (N / 128) * ((M + 255) / 256) * 2 > kNumSMs) {
         const int64_t kb = K / kGemmBK;
         const int64_t t256 = (N / 128) * ((M + 255) / 256), t192 = (N / 128) * ((M + 191) / 192);
-        const int64_t c256 = ((t256 + kNumSMs - 1) / kNumSMs) * (kb * 515 + 2400);
-        const int64_t c192 = ((t192 + kNumSMs - 1) / kNumSMs) * (kb * 470 + 300);
-        if (c192 < c256) p.bn = 192;
+        if (round_cost(t192, kb, 470, 300).cycles < round_cost(t256, kb, 515, 2400).cycles) p.bn = 192;
     }
     int force_units = 0;
     if (const char* f = getenv("QMM_GEMM_FORCE")) {            // "bn,na[,units]" for tuning sweeps and tests
@@ -229,6 +253,22 @@ static GemmPlan gemm_plan(int64_t M, int64_t N, int64_t K)
     const int64_t KB = K / kGemmBK;
     const int64_t total = tiles * KB;
     int64_t units;
+    p.whole = 0;
+    p.grid = 0;
+    if (tiles * 2 > kNumSMs && !force_units) {
+        // whole tiles, the same number for every block; the tiles of the last, partly filled round
+        // are cut into equal shares of their units when round_cost says that pays
+        const RoundCost rc = p.bn == 256 ? round_cost(tiles, KB, 515, 2400) : round_cost(tiles, KB, 470, 300);
+        if (rc.cut_tail && getenv("QMM_GEMM_NO_TAIL_CUT") == nullptr) {
+            p.grid = kNumSMs;
+            p.whole = (int)(tiles / kNumSMs) * kNumSMs;
+            units = ((tiles - p.whole) * KB + kNumSMs - 1) / kNumSMs;
+            if (units < 8) units = 8;
+            p.units = (int)units;
+            p.cut = true;
+            return p;
+        }
+    }
     if (tiles * 2 <= kNumSMs) {
         // the largest number of equal pieces per tile that the SMs can take at once, every piece
         // worth a pipeline fill and an epilogue (>= 8 k-blocks)
@@ -272,6 +312,7 @@ qmm_status launch_gemm(int fmt, const void* packed, int64_t N, int64_t K, const 
     p.ldo = ldy;
     p.a_col_offset = (int)(N / 2);
     p.M = (int)M;
+    p.whole_tiles = plan.whole;
     p.units_per_block = plan.units;
     p.partial = (float*)((uint8_t*)ws + kGemmWsHeader);
     p.status = (int*)ws;
@@ -281,7 +322,7 @@ qmm_status launch_gemm(int fmt, const void* packed, int64_t N, int64_t K, const 
     const int n_tiles = (int)(N / (128 * na));
     const int64_t tiles = (int64_t)n_tiles * ((M + bn - 1) / bn);
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)tiles, (unsigned)(bn / 8));
+    cfg.gridDim = dim3((unsigned)(tiles - plan.whole), (unsigned)(bn / 8));
     cfg.blockDim = dim3(256);
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -290,7 +331,7 @@ qmm_status launch_gemm(int fmt, const void* packed, int64_t N, int64_t K, const 
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return check_cuda(cudaLaunchKernelEx(&cfg, gemm_cut_reduce_kernel, (const float*)p.partial, Y, (int64_t)ldy, (int)M, bn, na,
-                                         p.a_col_offset, n_tiles, (int)(K / kGemmBK), plan.units),
+                                         p.a_col_offset, n_tiles, (int)(K / kGemmBK), plan.units, plan.whole),
                       "qmm_gemm partial-sum kernel launch");
 }
 

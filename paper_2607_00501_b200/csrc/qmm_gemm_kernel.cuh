@@ -66,10 +66,11 @@ struct GemmParams {
     const int* tile_row0;            // [max_tiles] first permuted row of the tile
     const int* tile_rows;            // [max_tiles] valid rows in the tile (<= BN)
     const int* num_tiles;            // [1]
-    // dense mode: block b owns the units [b*U, (b+1)*U) of the tile-major sequence of (tile, k-block)
-    // units; the pieces of a tile cut by a block boundary go to `partial` as fp32 and a second
-    // kernel adds them
-    int units_per_block;             // U
+    // dense mode: block b takes whole_tiles / grid whole tiles, then the units [b*U, (b+1)*U) of the
+    // tile-major sequence of (tile, k-block) units of the remaining tiles; the pieces of a tile cut
+    // by a block boundary go to `partial` as fp32 and a second kernel adds them
+    int whole_tiles;                 // the first whole_tiles tiles (a multiple of the grid size) are dealt whole, contiguously
+    int units_per_block;             // U: share of the (tile, k-block) units of the other tiles
     float* partial;                  // [2 * gridDim.x] slots of NA*BN*128 floats (when some tile is cut)
     int* status;                     // device status word (0 = ok)
     long long* trace;                // optional [block 0 only] clock64 samples for pipeline analysis (tuning aid), else null
@@ -315,9 +316,18 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
     // i-th piece of work of this block (every role walks the same sequence); false past the last
     auto get_work = [&](int i, GemmWork& w) -> bool {
         int t;
-        if (U > 0) {
+        const int whole = DENSE ? p.whole_tiles / (int)gridDim.x : 0;     // whole tiles of this block, taken first
+        if (DENSE && i < whole) {
+            t = (int)blockIdx.x * whole + i;
+            w.kb0 = 0;
+            w.kb1 = KB;
+            w.first = blockIdx.x;
+            w.cn = 1;
+        } else if (U > 0) {
+            i -= whole;
+            const int t0 = DENSE ? p.whole_tiles : 0;                     // the tiles below are counted from here
             const long long u0 = (long long)blockIdx.x * U;
-            const long long u1 = min(u0 + U, (long long)total_tiles * KB);
+            const long long u1 = min(u0 + U, (long long)(total_tiles - t0) * KB);
             if (u0 >= u1) return false;
             // Tiles the share touches: first .. last.  Order of work: the cut tile at the head of the
             // share, the cut tile at its tail, then the whole tiles -- cut tiles are then completed
@@ -334,6 +344,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             w.kb1 = (int)min(u1 - tb, (long long)KB);
             w.first = (int)(tb / U);
             w.cn = (int)((tb + KB - 1) / U) - w.first + 1;
+            t += t0;
         } else {
             t = blockIdx.x + i * gridDim.x;
             if (t >= total_tiles) return false;

@@ -106,6 +106,32 @@ def test_gemm_tiles_cut_across_blocks(qmm, oracle, monkeypatch, fmt, force, M, N
         assert torch.equal(first, qmm.gemm(fmt, packed, N, K, Xd).cpu())
 
 
+@pytest.mark.parametrize("fmt", [Q4, Q8])
+def test_gemm_last_round_cut_into_shares(qmm, oracle, monkeypatch, fmt):
+    """Many tiles, a nearly empty last round and a long K: every block takes its whole tiles, then an
+    equal share of the units of the last round's tiles (here 152 tiles on 148 SMs: 4 tiles in shares
+    of 8 of their 128 k-blocks), which the second kernel adds up.  Rows of the cut tiles and of whole tiles are checked."""
+    monkeypatch.delenv("QMM_GEMM_FORCE", raising=False)
+    monkeypatch.delenv("QMM_GEMM_NO_TAIL_CUT", raising=False)
+    M, N, K = 2048, 2432, 8192
+    assert qmm.gemm_workspace_bytes(fmt, M, N, K) == 8192 + 2 * 148 * 256 * 128 * 4
+    blocks, _, _ = util.random_blocks(synth, fmt, N, K, seed=5 + fmt, special_scales=False)
+    X = synth.activations(73, fmt, M, K)
+    rows = np.array([0, 255, 256, 1000, 1791, 1792, 1800, 1919, 2000, 2047])     # the last token tile holds the cut tiles
+    run_gemm(qmm, oracle, fmt, blocks, N, K, X, "cut last round fmt=%d" % fmt, rows=rows)
+    packed = qmm.pack(fmt, util.dev(blocks), N, K)
+    Xd = util.dev(X)
+    first = qmm.gemm(fmt, packed, N, K, Xd).cpu()
+    for _ in range(2):
+        assert torch.equal(first, qmm.gemm(fmt, packed, N, K, Xd).cpu())
+    # the same product with the last round left whole agrees to fp16 rounding of nearly equal fp32 sums
+    monkeypatch.setenv("QMM_GEMM_NO_TAIL_CUT", "1")
+    assert qmm.gemm_workspace_bytes(fmt, M, N, K) == 8192
+    whole = qmm.gemm(fmt, packed, N, K, Xd).cpu()
+    assert torch.equal(first[:1792], whole[:1792])                                # whole tiles: identical
+    assert float((first.float() - whole.float()).abs().max()) <= 2e-3 * float(whole.float().abs().max())
+
+
 def test_gemm_matches_gemv_rows(qmm):
     # the M = 1 product through both kernels agrees to fp16 rounding of nearly equal fp32 sums
     N, K = 384, 1024

@@ -96,6 +96,8 @@ def test_gemm_workspace_rule(L, monkeypatch):
     few = qmm.gemm_workspace_bytes(4, 256, 3072, 8192)                 # 24 tiles of 256 tokens: K cut in 4
     assert few == header + 2 * 96 * 256 * 128 * 4
     assert qmm.gemm_workspace_bytes(4, 256, 3072, 8192) == few         # same answer every time
+    # 192 tiles of 128 k-blocks: one whole tile per block, the 44 tiles of the second round in equal shares
+    assert qmm.gemm_workspace_bytes(4, 2048, 3072, 8192) == header + 2 * 148 * 256 * 128 * 4
     tiny = qmm.gemm_workspace_bytes(4, 1, 128, 256)                    # one tile, 4 k-blocks: too short to cut
     assert tiny == header
     monkeypatch.setenv("QMM_GEMM_FORCE", "128,1,5")
