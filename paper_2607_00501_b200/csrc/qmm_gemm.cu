@@ -50,7 +50,7 @@ template <int FMT, int BN, int NA, int EPI, bool DENSE>
 static qmm_status launch_t(const CUtensorMap& map, const GemmParams& p, dim3 grid, cudaStream_t st)
 {
     auto kern = gemm_kernel<FMT, BN, NA, EPI, DENSE>;
-    constexpr int smem = GemmGeom<BN, NA, EPI>::kSmemBytes;
+    constexpr int smem = GemmGeom<BN, NA, EPI, FMT>::kSmemBytes;
     // the attribute is per device: remember which devices have it (per instantiation)
     static std::atomic<uint64_t> configured{0};
     int dev = 0;
@@ -63,7 +63,7 @@ static qmm_status launch_t(const CUtensorMap& map, const GemmParams& p, dim3 gri
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
-    cfg.blockDim = dim3(GemmGeom<BN, NA, EPI>::kThreads);
+    cfg.blockDim = dim3(GemmGeom<BN, NA, EPI, FMT>::kThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];

@@ -79,7 +79,7 @@ struct GemmParams {
 // Pipeline geometry of one instantiation.  Tensor memory: half of the SM's 512 columns when the
 // accumulators leave room for it (two blocks per SM), else all of it; what the accumulators leave
 // is the weight ring.  A stage is one weight slot in TMEM plus one activation slot in shared memory.
-template <int BN, int NA, int EPI>
+template <int BN, int NA, int EPI, int FMT>
 struct GemmGeom {
     static constexpr int kACols = NA * 32;                                 // TMEM columns per weight slot
     static constexpr int kDCols = NA * BN;                                 // accumulator columns
@@ -106,9 +106,14 @@ struct GemmGeom {
     static constexpr int kStagesB = !kSplit ? kStages : (kSmemFit < kGemmMaxStagesB ? kSmemFit : kGemmMaxStagesB);
     static constexpr int kSmemBytes = kStagesB * kBStage + kStaging + 1024 /*align*/ + 512;
     // Warp roles: expanders, epilogue warps (one or two per TMEM lane quarter), TMA producer, MMA
-    // issuer.  Narrow token tiles are bound by the expansion, not by the epilogue: 16 + 4 there.
-    static constexpr int kExpWarps = (BN <= 64 || NA == 2) ? 16 : 8;
-    static constexpr int kEpiWarps = (BN <= 64 || NA == 2) ? 4 : 8;
+    // issuer.  Narrow token tiles are bound by the expansion, not by the epilogue: 16 + 4 there,
+    // and for two tile sets of 4-bit weights.
+    // (two tile sets: every stage needs eight warp-stages of expansion, which eight warps do not
+    // deliver in the 640 cycles of its MMAs; the 8-bit format's expanders need the 96 registers that
+    // only the smaller block leaves them)
+    static constexpr bool kManyExpanders = BN <= 64 || (NA == 2 && FMT == QMM_Q4);
+    static constexpr int kExpWarps = kManyExpanders ? 16 : 8;
+    static constexpr int kEpiWarps = kManyExpanders ? 4 : 8;
     static constexpr int kThreads = (kExpWarps + kEpiWarps + 2) * 32;
     static_assert(kStages >= 2 && kStagesB >= 2, "tensor memory or shared memory over-subscribed");
 };
@@ -233,11 +238,11 @@ __device__ __noinline__ void cut_tile_epilogue(const GemmParams& p, const GemmWo
 // while the epilogue warps drain the accumulators of piece i, the expanders
 // and the TMA producer already fill the ring for piece i+1.
 template <int FMT, int BN, int NA, int EPI, bool DENSE>
-__global__ void __launch_bounds__(GemmGeom<BN, NA, EPI>::kThreads, 1)
+__global__ void __launch_bounds__(GemmGeom<BN, NA, EPI, FMT>::kThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
 {
     using namespace tc;
-    using G = GemmGeom<BN, NA, EPI>;
+    using G = GemmGeom<BN, NA, EPI, FMT>;
     constexpr int NEXP = G::kExpWarps;
     constexpr int PH = NEXP / (4 * NA);               // expander warps per (weight tile, lane quarter): they alternate stages
     constexpr int NEPI = G::kEpiWarps;
