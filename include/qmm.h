@@ -174,10 +174,12 @@ qmm_status qmm_gemv_static(qmm_format fmt, const void* packed, int64_t N, int64_
  *   X_fp16  device, [M, ldx] fp16 row-major, ldx >= K, ldx % 8 == 0
  *   Y_fp16  device, [M, ldy] fp16 row-major, ldy >= N, ldy % 8 == 0, written
  *   ws      device, at least qmm_gemm_workspace_bytes(...) bytes: the status
- *           word and, for shapes with too few output tiles to occupy the SMs,
- *           the fp32 partial sums of the pieces the K range is cut into
- *           (added in a fixed order by a second kernel, so results are the
- *           same bits on every call)                                         */
+ *           word and, for shapes whose output tiles (or the tiles of their
+ *           last round) do not occupy the SMs, the fp32 partial sums of the
+ *           pieces the K range of those tiles is cut into (added in a fixed
+ *           order by a second kernel, so results are the same bits on every
+ *           call).  8 KB for most shapes, up to two slots of one output tile
+ *           per SM (39 MB) where tiles are cut                               */
 size_t qmm_gemm_workspace_bytes(qmm_format fmt, int64_t M, int64_t N, int64_t K);
 qmm_status qmm_gemm(qmm_format fmt, const void* packed, int64_t N, int64_t K,
                     const uint16_t* X_fp16, int64_t ldx,
