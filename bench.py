@@ -544,6 +544,23 @@ def extra_sections(args, qmm, torch, pk, ops, fmts):
                               "frac_tensor_nominal": round(fl / med / 1e9 / NOMINAL_BF16_TFLOPS, 4),
                               "hbm_floor_ms": round(touched / pk["hbm_gbs"] / 1e6, 4),
                               "frac_of_hbm_floor": round(touched / pk["hbm_gbs"] / 1e6 / med, 4)}
+        if f == c["fmt"]:
+            # not a config: the same layer under an uneven expert load (a fixed N(0, 1.5^2) bias per
+            # expert on the seeded logits; trained routers are skewed, the config's iid logits are not)
+            T = c["Ts"][-1]
+            bias = np.random.default_rng([c["seed"], 999]).standard_normal(c["E"]).astype(np.float32) * 1.5
+            X = dev(synth.activations(c["seed"], 100 + T, T, c["H"]))
+            lg = dev(synth.logits(c["seed"], 200 + T, T, c["E"]) + bias[None, :])
+            o = torch.empty((T, c["H"]), dtype=torch.float16, device="cuda")
+            a = qmm.moe_args(f, T, c["H"], c["I"], c["E"], c["topk"], lg, X, pg, pu, pd, o)
+            ws = torch.zeros(qmm.moe_workspace_bytes(a), dtype=torch.uint8, device="cuda")
+            fn = lambda: qmm.moe(a, ws)
+            fn()
+            med, best = time_op(torch, fn, 10, flush)
+            qmm.status_check(ws)
+            fl = T * c["topk"] * 3 * 2.0 * c["H"] * c["I"]
+            moe["T%d_skewed_load" % T] = {"ms": round(med, 4), "TFLOPs": round(fl / med / 1e9, 2),
+                                          "frac_tensor_nominal": round(fl / med / 1e9 / NOMINAL_BF16_TFLOPS, 4)}
         out["moe_q%d" % f] = moe
         del pg, pu, pd, gate, up, down
     return out
