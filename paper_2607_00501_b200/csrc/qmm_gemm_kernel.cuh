@@ -114,7 +114,11 @@ struct GemmGeom {
     static constexpr bool kManyExpanders = BN <= 64 || (NA == 2 && FMT == QMM_Q4);
     static constexpr int kExpWarps = kManyExpanders ? 16 : 8;
     static constexpr int kEpiWarps = kManyExpanders ? 4 : 8;
-    static constexpr int kThreads = (kExpWarps + kEpiWarps + 2) * 32;
+    // one MMA-issuing warp per weight tile set: each has its own accumulators, so nothing orders
+    // their MMAs, and the loop that feeds the tensor pipe (the critical path with two tile sets: it
+    // competes with four expander warps for its scheduler) runs in two halves side by side
+    static constexpr int kIssuers = NA;
+    static constexpr int kThreads = (kExpWarps + kEpiWarps + 1 + kIssuers) * 32;
     static_assert(kStages >= 2 && kStagesB >= 2, "tensor memory or shared memory over-subscribed");
 };
 
@@ -246,7 +250,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
     constexpr int NEXP = G::kExpWarps;
     constexpr int PH = NEXP / (4 * NA);               // expander warps per (weight tile, lane quarter): they alternate stages
     constexpr int NEPI = G::kEpiWarps;
-    constexpr int TMA_WARP = NEXP + NEPI, MMA_WARP = NEXP + NEPI + 1;
+    constexpr int TMA_WARP = NEXP + NEPI, MMA_WARP = NEXP + NEPI + 1;   // issuers: warps MMA_WARP .. MMA_WARP + NISS - 1
+    constexpr int NISS = G::kIssuers;
     constexpr int S = G::kStages;                     // pipeline depth (weight slots)
     constexpr bool SPLIT = G::kSplit;                 // activation tiles in a ring of their own
     constexpr int SB = G::kStagesB;                   // its depth (== S unless SPLIT)
@@ -290,15 +295,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
             mbar_init(&full[s], 4 * NA + (SPLIT ? 0 : 1));                // the stage's expander warps (+ the TMA producer)
-            mbar_init(&empty[s], 1);                                      // one tcgen05.commit
+            mbar_init(&empty[s], NISS);                                   // one tcgen05.commit per issuing warp
         }
         if (SPLIT)
             for (int s = 0; s < SB; ++s) {
                 mbar_init(&full_b[s], 1);                                 // the TMA producer (+ its bytes)
-                mbar_init(&empty_b[s], 1);                                // one tcgen05.commit
+                mbar_init(&empty_b[s], NISS);                             // one tcgen05.commit per issuing warp
             }
         for (int b = 0; b < 2; ++b) {
-            mbar_init(&acc_full[b], 1);
+            mbar_init(&acc_full[b], NISS);
             mbar_init(&acc_empty[b], NEPI);
         }
         mbar_init(stg_full, NEPI);
@@ -603,12 +608,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         // values); one elected lane issues the MMAs and the commits.
         constexpr uint32_t idesc = idesc_f16_m128(BN);
         const uint64_t desc0 = smem_desc_k_sw128(smem_u32(smem_b));       // slot 0, k-step 0
+        const int ia = warp - MMA_WARP;                                   // which issuer
         bool ok = true;
         int g = 0, it = 0;
         // The issuing lane.  The MMAs and commits below are predicated on it instead of sitting in a
         // divergent branch: measured ~25 % less issue time per stage (operands stay warp-uniform).
         const uint32_t sel = elect_one() ? 1u : 0u;
-        const bool tracing = p.trace != nullptr && blockIdx.x == 0 && lane == 0;
+        const bool tracing = p.trace != nullptr && blockIdx.x == 0 && lane == 0 && warp == MMA_WARP;
         (void)tracing;
         (void)g;
         int s = 0;                                                        // ring slot of stage g and the parity of its
@@ -623,7 +629,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
                 tc_fence_after_sync();
-                if (p.trace != nullptr && blockIdx.x == 0 && it <= 16 && lane == 0) p.trace[((it - AB) * 4 + 3) * 8 + 1] = clock64();
+                if (p.trace != nullptr && blockIdx.x == 0 && it <= 16 && lane == 0 && warp == MMA_WARP) p.trace[((it - AB) * 4 + 3) * 8 + 1] = clock64();
             }
             const uint32_t d_tmem = tmem_base + (uint32_t)(buf * D_COLS);
             // One round of the loop = wait for the slot(s), vote, fence, MMAs, commit(s).  Two stages per
@@ -638,7 +644,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                 const uint64_t desc_s = desc0 + (uint64_t)((SPLIT ? sb : sj) * (B_STAGE >> 4));
                 const uint32_t a_s = tmem_base + (uint32_t)(RING0 + sj * A_COLS);
 #pragma unroll
-                for (int a = 0; a < NA; ++a) mma_ts_f16_stage(d_tmem + (uint32_t)(a * BN), a_s + (uint32_t)(a * 32), desc_s, idesc, acc, sel);
+                for (int a = 0; a < NA / NISS; ++a)                       // this warp's tile set(s)
+                    mma_ts_f16_stage(d_tmem + (uint32_t)((ia + a * NISS) * BN), a_s + (uint32_t)((ia + a * NISS) * 32), desc_s, idesc, acc, sel);
                 mma_commit_sel(&empty[sj], sel);                          // slot reusable when these MMAs finish
                 if constexpr (SPLIT) mma_commit_sel(&empty_b[sb], sel);
             };
@@ -711,7 +718,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             }
             if (ok) mma_commit_sel(&acc_full[buf], sel);                  // accumulators of this piece are complete
             __syncwarp();
-            if (p.trace != nullptr && blockIdx.x == 0 && it < 16 && lane == 0) p.trace[(it * 4 + 0) * 8 + 1] = clock64();
+            if (p.trace != nullptr && blockIdx.x == 0 && it < 16 && lane == 0 && warp == MMA_WARP) p.trace[(it * 4 + 0) * 8 + 1] = clock64();
         }
         if (!ok) *abort_flag = 1;
     }
