@@ -117,7 +117,7 @@ struct GemmGeom {
     // one MMA-issuing warp per weight tile set: each has its own accumulators, so nothing orders
     // their MMAs, and the loop that feeds the tensor pipe (the critical path with two tile sets: it
     // competes with four expander warps for its scheduler) runs in two halves side by side
-    static constexpr int kIssuers = NA;
+    static constexpr int kIssuers = (NA == 2 && FMT == QMM_Q4) ? 2 : 1;   // (8-bit weights: measured 3 % slower with two)
     static constexpr int kThreads = (kExpWarps + kEpiWarps + 1 + kIssuers) * 32;
     static_assert(kStages >= 2 && kStagesB >= 2, "tensor memory or shared memory over-subscribed");
 };
