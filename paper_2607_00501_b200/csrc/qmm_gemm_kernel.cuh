@@ -100,7 +100,9 @@ struct GemmGeom {
     // for the activations bounds a stage at (MMA time + that latency) / slots.  The activation tiles
     // then get a ring of their own in shared memory with barriers of their own (kSplit), as deep as
     // shared memory allows; else one ring and one pair of barriers per stage serve both operands.
-    static constexpr bool kSplit = NA == 2 && BN >= 128;                   // (narrower tiles: the extra waits and commits cost the issuing loop more than the latency they hide)
+    // (also the 192-token tile with its two accumulator buffers: four weight slots.  Narrower tiles:
+    // the extra waits and commits cost the issuing loop more than the latency they hide.)
+    static constexpr bool kSplit = (NA == 2 && BN >= 128) || (NA == 1 && BN == 192);
     static constexpr int kFit2 = kSplit ? kFit : (kFit < kSmemFit ? kFit : kSmemFit);
     static constexpr int kStages = kFit2 < kGemmMaxStages ? kFit2 : kGemmMaxStages;             // weight slots (and activation slots unless kSplit)
     static constexpr int kStagesB = !kSplit ? kStages : (kSmemFit < kGemmMaxStagesB ? kSmemFit : kGemmMaxStagesB);
