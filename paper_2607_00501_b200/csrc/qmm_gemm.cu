@@ -174,6 +174,7 @@ __global__ void gemm_cut_reduce_kernel(const float* __restrict__ partial, uint16
 struct GemmPlan {
     int bn, na;
     int whole;          // tiles dealt whole, the same number to every block (a multiple of grid)
+    bool halves;        // the remaining tiles are dealt as half tiles (BN / 2 tokens each)
     int units;          // (tile, k-block) units per block of the remaining tiles
     int grid;           // blocks
     bool cut;           // some tile is shared between blocks: partial-sum slots and the second kernel
@@ -185,17 +186,23 @@ struct GemmPlan {
 struct RoundCost {
     int64_t cycles;
     bool cut_tail;
+    bool halve_tail;    // instead: the last round's tiles as two half tiles each (256-token tiles, at most SMs / 2 of them)
 };
 static RoundCost round_cost(int64_t tiles, int64_t kb, int64_t stage, int64_t handover)
 {
     const int64_t tile = kb * stage + handover;
     const int64_t rounds = tiles / kNumSMs, tail = tiles % kNumSMs;
-    RoundCost r = {rounds * tile, false};
+    RoundCost r = {rounds * tile, false, false};
     if (tail == 0) return r;
     int64_t share = (tail * kb + kNumSMs - 1) / kNumSMs;
     if (share < 8) share = 8;
     const int64_t cut = share * stage + 2 * handover + 18000;
-    if (rounds >= 1 && cut < tile) {
+    // half tiles (N = 128 MMAs in the 256-token kernel): ~470 cycles per stage, measured
+    const int64_t halves = (stage == 515 && 2 * tail <= kNumSMs) ? kb * 470 + handover : tile + 1;
+    if (rounds >= 1 && halves < tile && halves <= cut) {
+        r.cycles += halves;
+        r.halve_tail = true;
+    } else if (rounds >= 1 && cut < tile) {
         r.cycles += cut;
         r.cut_tail = true;
     } else {
@@ -255,10 +262,19 @@ static GemmPlan gemm_plan(int64_t M, int64_t N, int64_t K)
     int64_t units;
     p.whole = 0;
     p.grid = 0;
+    p.halves = false;
     if (tiles * 2 > kNumSMs && !force_units) {
         // whole tiles, the same number for every block; the tiles of the last, partly filled round
         // are cut into equal shares of their units when round_cost says that pays
         const RoundCost rc = p.bn == 256 ? round_cost(tiles, KB, 515, 2400) : round_cost(tiles, KB, 470, 300);
+        if (rc.halve_tail && getenv("QMM_GEMM_NO_TAIL_CUT") == nullptr) {
+            p.grid = kNumSMs;
+            p.whole = (int)(tiles / kNumSMs) * kNumSMs;
+            p.halves = true;
+            p.units = (int)KB;
+            p.cut = false;
+            return p;
+        }
         if (rc.cut_tail && getenv("QMM_GEMM_NO_TAIL_CUT") == nullptr) {
             p.grid = kNumSMs;
             p.whole = (int)(tiles / kNumSMs) * kNumSMs;
@@ -313,6 +329,7 @@ qmm_status launch_gemm(int fmt, const void* packed, int64_t N, int64_t K, const 
     p.a_col_offset = (int)(N / 2);
     p.M = (int)M;
     p.whole_tiles = plan.whole;
+    p.tail_halves = plan.halves ? 1 : 0;
     p.units_per_block = plan.units;
     p.partial = (float*)((uint8_t*)ws + kGemmWsHeader);
     p.status = (int*)ws;

@@ -70,6 +70,7 @@ struct GemmParams {
     // tile-major sequence of (tile, k-block) units of the remaining tiles; the pieces of a tile cut
     // by a block boundary go to `partial` as fp32 and a second kernel adds them
     int whole_tiles;                 // the first whole_tiles tiles (a multiple of the grid size) are dealt whole, contiguously
+    int tail_halves;                 // != 0: the remaining tiles are dealt as halves of BN / 2 tokens, one after the other over the blocks
     int units_per_block;             // U: share of the (tile, k-block) units of the other tiles
     float* partial;                  // [2 * gridDim.x] slots of NA*BN*128 floats (when some tile is cut)
     int* status;                     // device status word (0 = ok)
@@ -203,6 +204,7 @@ constexpr int kGemmL2Ahead = QMM_GEMM_L2_AHEAD;    // stages of a row group's we
 // the tile (block indices first .. first + cn - 1, k ascending); cn == 1: the piece is the whole tile.
 struct GemmWork {
     int n_tile, expert, row0, rows;
+    int n_mma;                       // token columns the MMAs of this piece compute (the tile width, or half of it)
     int kb0, kb1;
     int first, cn;
 };
@@ -328,8 +330,20 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
     // i-th piece of work of this block (every role walks the same sequence); false past the last
     auto get_work = [&](int i, GemmWork& w) -> bool {
         int t;
+        int half = -1;                                                    // >= 0: which half of the tile's tokens
         const int whole = DENSE ? p.whole_tiles / (int)gridDim.x : 0;     // whole tiles of this block, taken first
-        if (DENSE && i < whole) {
+        if (DENSE && i >= whole && p.tail_halves) {
+            // the tiles of the last, partly filled round as half tiles (no partial sums: each half is a
+            // product of its own; its weights are expanded twice)
+            const int j = (int)blockIdx.x + (i - whole) * (int)gridDim.x;
+            if (j >= 2 * (total_tiles - p.whole_tiles)) return false;
+            t = p.whole_tiles + (j >> 1);
+            half = j & 1;
+            w.kb0 = 0;
+            w.kb1 = KB;
+            w.first = blockIdx.x;
+            w.cn = 1;
+        } else if (DENSE && i < whole) {
             t = (int)blockIdx.x * whole + i;
             w.kb0 = 0;
             w.kb1 = KB;
@@ -375,6 +389,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             w.expert = 0;
             w.row0 = mt * BN;
             w.rows = min(BN, p.M - w.row0);
+        }
+        w.n_mma = BN;
+        if (DENSE && half >= 0) {
+            w.n_mma = BN / 2;
+            w.row0 += half * (BN / 2);
+            w.rows = max(0, min(BN / 2, p.M - w.row0));
         }
         return true;
     };
@@ -608,7 +628,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         // ================= MMA issuer
         // The whole warp runs the loop converged (so that addresses and descriptors stay warp-uniform
         // values); one elected lane issues the MMAs and the commits.
-        constexpr uint32_t idesc = idesc_f16_m128(BN);
         const uint64_t desc0 = smem_desc_k_sw128(smem_u32(smem_b));       // slot 0, k-step 0
         const int ia = warp - MMA_WARP;                                   // which issuer
         bool ok = true;
@@ -634,6 +653,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                 if (p.trace != nullptr && blockIdx.x == 0 && it <= 16 && lane == 0 && warp == MMA_WARP) p.trace[((it - AB) * 4 + 3) * 8 + 1] = clock64();
             }
             const uint32_t d_tmem = tmem_base + (uint32_t)(buf * D_COLS);
+            const uint32_t idesc = DENSE ? idesc_f16_m128(w.n_mma) : idesc_f16_m128(BN);   // (half tiles of a dense product's last round: N = BN / 2)
             // One round of the loop = wait for the slot(s), vote, fence, MMAs, commit(s).  Two stages per
             // round when the ring is deep enough (the polls, the vote and the fence are paid once per
             // 128 k), then single stages for what is left of the piece.  Both bodies are straight-line

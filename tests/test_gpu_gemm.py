@@ -132,6 +132,29 @@ def test_gemm_last_round_cut_into_shares(qmm, oracle, monkeypatch, fmt):
     assert float((first.float() - whole.float()).abs().max()) <= 2e-3 * float(whole.float().abs().max())
 
 
+@pytest.mark.parametrize("fmt", [Q4, Q8])
+@pytest.mark.parametrize("M", [2048, 1990, 1900])
+def test_gemm_last_round_as_half_tiles(qmm, oracle, monkeypatch, fmt, M):
+    """152 tiles of 256 tokens on 148 SMs, short K: the four tiles of the second round run as eight
+    half tiles (MMAs of 128 token columns), each a product of its own -- so the result is the same
+    bits as with whole tiles.  M = 1990 leaves the second half of the last token tile ragged,
+    M = 1900 leaves it empty."""
+    monkeypatch.delenv("QMM_GEMM_FORCE", raising=False)
+    monkeypatch.delenv("QMM_GEMM_NO_TAIL_CUT", raising=False)
+    N, K = 2432, 512
+    assert qmm.gemm_workspace_bytes(fmt, M, N, K) == 8192                         # no partial sums
+    blocks, _, _ = util.random_blocks(synth, fmt, N, K, seed=9 + fmt, special_scales=False)
+    X = synth.activations(74, fmt, M, K)
+    rows = np.unique(np.concatenate([[0, 255, 1000, 1791], np.arange(1792, M, 7), [M - 1]]))
+    run_gemm(qmm, oracle, fmt, blocks, N, K, X, "half tiles fmt=%d M=%d" % (fmt, M), rows=rows)
+    packed = qmm.pack(fmt, util.dev(blocks), N, K)
+    Xd = util.dev(X)
+    halves = qmm.gemm(fmt, packed, N, K, Xd).cpu()
+    monkeypatch.setenv("QMM_GEMM_NO_TAIL_CUT", "1")
+    whole = qmm.gemm(fmt, packed, N, K, Xd).cpu()
+    assert torch.equal(halves, whole)
+
+
 def test_gemm_matches_gemv_rows(qmm):
     # the M = 1 product through both kernels agrees to fp16 rounding of nearly equal fp32 sums
     N, K = 384, 1024
