@@ -653,7 +653,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                 if (p.trace != nullptr && blockIdx.x == 0 && it <= 16 && lane == 0 && warp == MMA_WARP) p.trace[((it - AB) * 4 + 3) * 8 + 1] = clock64();
             }
             const uint32_t d_tmem = tmem_base + (uint32_t)(buf * D_COLS);
-            const uint32_t idesc = DENSE ? idesc_f16_m128(w.n_mma) : idesc_f16_m128(BN);   // (half tiles of a dense product's last round: N = BN / 2)
+            // The MMAs' N: dense, the tile width (or half of it for half tiles of the last round);
+            // grouped, the tile's valid rows rounded up to 16 -- the tensor time of a partly filled
+            // expert tile shrinks with it, and the columns beyond are never read.
+            const uint32_t idesc = DENSE ? idesc_f16_m128(w.n_mma) : idesc_f16_m128(min(BN, (w.rows + 15) & ~15));
             // One round of the loop = wait for the slot(s), vote, fence, MMAs, commit(s).  Two stages per
             // round when the ring is deep enough (the polls, the vote and the fence are paid once per
             // 128 k), then single stages for what is left of the piece.  Both bodies are straight-line
