@@ -204,7 +204,7 @@ constexpr int kGemmL2Ahead = QMM_GEMM_L2_AHEAD;    // stages of a row group's we
 // the tile (block indices first .. first + cn - 1, k ascending); cn == 1: the piece is the whole tile.
 struct GemmWork {
     int n_tile, expert, row0, rows;
-    int n_mma;                       // token columns the MMAs of this piece compute (the tile width, or half of it)
+    int n_mma;                       // token columns the MMAs of this piece compute: rows rounded up to 16
     int kb0, kb1;
     int first, cn;
 };
@@ -390,12 +390,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             w.row0 = mt * BN;
             w.rows = min(BN, p.M - w.row0);
         }
-        w.n_mma = BN;
         if (DENSE && half >= 0) {
-            w.n_mma = BN / 2;
             w.row0 += half * (BN / 2);
             w.rows = max(0, min(BN / 2, p.M - w.row0));
         }
+        w.n_mma = max(16, min(BN, (w.rows + 15) & ~15));                  // valid rows rounded up to the MMA's granularity
         return true;
     };
 
@@ -653,10 +652,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                 if (p.trace != nullptr && blockIdx.x == 0 && it <= 16 && lane == 0 && warp == MMA_WARP) p.trace[((it - AB) * 4 + 3) * 8 + 1] = clock64();
             }
             const uint32_t d_tmem = tmem_base + (uint32_t)(buf * D_COLS);
-            // The MMAs' N: dense, the tile width (or half of it for half tiles of the last round);
-            // grouped, the tile's valid rows rounded up to 16 -- the tensor time of a partly filled
-            // expert tile shrinks with it, and the columns beyond are never read.
-            const uint32_t idesc = DENSE ? idesc_f16_m128(w.n_mma) : idesc_f16_m128(min(BN, (w.rows + 15) & ~15));
+            // The MMAs' N is the piece's valid token rows rounded up to 16 (a partly filled expert tile,
+            // the ragged last token tile of a dense product, a half tile of its last round): the tensor
+            // time shrinks with it, and the columns beyond are never read.
+            const uint32_t idesc = idesc_f16_m128(w.n_mma);
             // One round of the loop = wait for the slot(s), vote, fence, MMAs, commit(s).  Two stages per
             // round when the ring is deep enough (the polls, the vote and the fence are paid once per
             // 128 k), then single stages for what is left of the piece.  Both bodies are straight-line
