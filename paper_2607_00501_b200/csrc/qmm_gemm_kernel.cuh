@@ -17,18 +17,21 @@
 // tile (half the activation traffic; the gate and up matrices of an expert).
 //
 // Roles (warp specialised):
-//   expanders (8 warps; 16 for token tiles of 64 and narrower): several per
-//                      weight tile and lane quarter, alternating stages;
-//                      thread = one weight row; 32-byte code loads straight
-//                      from global/L2, unpack to fp16(d*q), tcgen05.st into the
-//                      A ring in TMEM.
-//   epilogue (8 warps, two per lane quarter; 4 for narrow tiles): tcgen05.ld
-//                      the accumulators, convert, stage the tile in shared
-//                      memory, release the accumulators, then store the tile
-//                      with 16-byte row segments.
+//   expanders (8 warps; 16 for token tiles of 64 and narrower and for two tile
+//                      sets of 4-bit weights): several per weight tile and lane
+//                      quarter, alternating stages; thread = one weight row;
+//                      32-byte code loads straight from global/L2, unpack to
+//                      fp16(d*q), tcgen05.st into the A ring in TMEM.
+//   epilogue (8 warps, two per lane quarter; 4 where there are 16 expanders):
+//                      tcgen05.ld the accumulators, convert, stage the tile in
+//                      shared memory as fp16, release the accumulators, then
+//                      store the tile with 16-byte row segments (or SiLU*mul of
+//                      the staged gate and up values).
 //   TMA producer (1 warp): activation tiles -> shared-memory ring (128-byte
 //                      swizzle), one lane.
-//   MMA issuer (1 warp, converged): tcgen05.mma (M128 x N=BN x K16) and the
+//   MMA issuer (1 warp, converged; one per tile set for two tile sets of 4-bit
+//                      weights): tcgen05.mma (M128 x N x K16, N = the piece's
+//                      valid token rows rounded up to 16) and the
 //                      tcgen05.commit that frees a ring slot, predicated on one
 //                      elected lane (no divergent branch around them).
 // The kernel is persistent: a block loops over tiles and the pipeline runs on
@@ -36,6 +39,9 @@
 //
 // TMEM columns: one or two accumulator buffers of NA*BN fp32 columns, then
 // STAGES slots of NA*32 columns (64 fp16 k-values per row and weight tile).
+// Activation tiles share those stages (one `full` and one `empty` barrier per
+// stage for both operands) except where tensor memory leaves only 3-4 weight
+// slots: there they have a deeper ring and barriers of their own (kSplit).
 //
 // Every mbarrier wait is bounded; on give-up the block raises an abort flag,
 // records QMM_ERR_DEVICE_TIMEOUT in the status word, stops issuing work, waits
@@ -240,9 +246,12 @@ __device__ __noinline__ void cut_tile_epilogue(const GemmParams& p, const GemmWo
 // Persistent, warp-specialised kernel.  Tile t = (token tile t / n_tiles, weight
 // tile t % n_tiles).  Grouped mode: every block walks the tile list t =
 // blockIdx.x, blockIdx.x + gridDim.x, ... so blocks that run together share
-// activation tiles.  Dense mode: every block takes an equal, contiguous share
-// of all (tile, k-block) units, so the SMs finish together whatever the tile
-// count.  The pipeline (stage counter, barrier phases) runs on across pieces:
+// activation tiles.  Dense mode: every block takes the same number of whole
+// tiles; the tiles that are left (all of them when there are few) are dealt
+// either as equal contiguous shares of their (tile, k-block) units -- pieces
+// of a tile cut by a share boundary go to fp32 partial sums -- or as half
+// tiles of BN / 2 tokens, as the host's plan says.
+// The pipeline (stage counter, barrier phases) runs on across pieces:
 // while the epilogue warps drain the accumulators of piece i, the expanders
 // and the TMA producer already fill the ring for piece i+1.
 template <int FMT, int BN, int NA, int EPI, bool DENSE>
