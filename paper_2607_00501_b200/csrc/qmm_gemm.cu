@@ -217,13 +217,15 @@ constexpr size_t kGemmWsTrace = 4096, kGemmWsHeader = 8192;
 
 // Token tile: 256 (the widest MMA, N = 256) once M exceeds one 128-token tile, else the smallest
 // that holds M -- or half / a quarter of that when this yields between 3/4 and one round of whole
-// tiles; one weight tile per block.  The (tile, k-block) units are dealt to the blocks in
-// equal contiguous shares:
-//   tiles <= SMs / 2: every tile is cut into equal pieces, one per block, as many as the SMs can
-//                     take at once; a second kernel adds the pieces;
-//   otherwise:        whole tiles, the same number for every block.  (Shares that cut tiles were
-//                     measured here too: the fp32 partial traffic costs more than the idle SMs
-//                     of the last round.)
+// tiles; one weight tile per block.  Work split:
+//   tiles <= SMs / 2: every tile is cut into equal pieces along K, one per block, as many as the
+//                     SMs can take at once; a second kernel adds the pieces;
+//   otherwise:        whole tiles, the same number for every block, and for the tiles of the
+//                     last, partly filled round the cheapest of (round_cost): whole tiles on
+//                     some of the SMs; equal shares of their (tile, k-block) units on all SMs
+//                     (partial sums + second kernel); two half tiles each (256-token tiles, at
+//                     most SMs / 2 of them left).  Cutting *every* tile into shares was measured
+//                     too: the fp32 partial traffic costs more than it saves.
 static GemmPlan gemm_plan(int64_t M, int64_t N, int64_t K)
 {
     GemmPlan p;
