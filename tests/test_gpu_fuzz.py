@@ -46,6 +46,42 @@ def test_random_gemm_shapes(qmm, oracle, case):
     util.assert_within_tol(util.host_f64(Y), Y_ref, B, "gemm fmt=%d M=%d N=%d K=%d" % (fmt, M, N, K))
 
 
+@pytest.mark.parametrize("case", range(10))
+def test_random_many_tile_gemm_plans_agree(qmm, oracle, monkeypatch, case):
+    """Shapes with more output tiles than SMs: the plan gives every block whole tiles and treats the
+    last, partly filled round in one of three ways (whole tiles, half tiles, shares of the K range with
+    partial sums).  Whatever it picks must agree with the whole-tile plan -- bit for bit unless partial
+    sums are added in another order -- be the same on every call, and pass the oracle on sampled rows."""
+    rng = np.random.default_rng([841, case])
+    fmt = int(rng.choice([4, 8]))
+    while True:
+        M, N, K = int(rng.integers(600, 4600)), int(rng.integers(4, 40)) * 128, int(rng.integers(1, 33)) * 256
+        if (N // 128) * ((M + 255) // 256) > 148:
+            break
+    monkeypatch.delenv("QMM_GEMM_FORCE", raising=False)
+    monkeypatch.delenv("QMM_GEMM_NO_TAIL_CUT", raising=False)
+    blocks, _, _ = util.random_blocks(synth, fmt, N, K, seed=842 + case, special_scales=False)
+    X = synth.activations(843, case, M, K)
+    packed, Xd = qmm.pack(fmt, util.dev(blocks), N, K), util.dev(X)
+    need = qmm.gemm_workspace_bytes(fmt, M, N, K)
+    ws = torch.zeros(need, dtype=torch.uint8, device="cuda")
+    Y = qmm.gemm(fmt, packed, N, K, Xd, ws=ws)
+    qmm.status_check(ws)
+    assert torch.equal(Y, qmm.gemm(fmt, packed, N, K, Xd, ws=ws))
+    rows = np.unique(np.concatenate([[0, M - 1, M - 129 if M > 129 else 0], rng.integers(0, M, size=5)]))
+    Y_ref, B = oracle.gemm(fmt, blocks, N, K, X[rows])
+    util.assert_within_tol(util.host_f64(Y)[rows], Y_ref, B, "gemm fmt=%d M=%d N=%d K=%d" % (fmt, M, N, K))
+    monkeypatch.setenv("QMM_GEMM_NO_TAIL_CUT", "1")
+    need_whole = qmm.gemm_workspace_bytes(fmt, M, N, K)
+    ws2 = torch.zeros(need_whole, dtype=torch.uint8, device="cuda")
+    Y2 = qmm.gemm(fmt, packed, N, K, Xd, ws=ws2)
+    qmm.status_check(ws2)
+    if need == need_whole:                                                        # no partial sums: same arithmetic
+        assert torch.equal(Y, Y2)
+    else:
+        assert float((Y.float() - Y2.float()).abs().max()) <= 2e-3 * float(Y2.float().abs().max())
+
+
 @pytest.mark.parametrize("case", range(6))
 def test_random_moe_layers(qmm, oracle, case):
     rng = np.random.default_rng([831, case])
