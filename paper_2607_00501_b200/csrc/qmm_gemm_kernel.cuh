@@ -57,6 +57,11 @@ constexpr int kGemmBK = 64;          // k per pipeline stage
 constexpr int kGemmMaxStagesB = 8;    // depth of the activation ring where it is a ring of its own
 constexpr int kGemmMaxStages = 6;     // pipeline depth is min(this, what tensor memory leaves for the weight ring)
 
+#ifndef QMM_GEMM_PREFETCH
+#define QMM_GEMM_PREFETCH 2
+#endif
+constexpr int kGemmPrefetch = QMM_GEMM_PREFETCH;   // weight slices in flight per expander thread (default)
+
 enum GemmEpilogue { kEpiStore = 0, kEpiSiluMul = 1 };
 
 struct GemmParams {
@@ -116,17 +121,20 @@ struct GemmGeom {
     static constexpr int kSmemBytes = kStagesB * kBStage + kStaging + 1024 /*align*/ + 512;
     // Warp roles: expanders, epilogue warps (one or two per TMEM lane quarter), TMA producer, MMA
     // issuer.  Narrow token tiles are bound by the expansion, not by the epilogue: 16 + 4 there,
-    // and for two tile sets of 4-bit weights.
+    // and for two tile sets.
     // (two tile sets: every stage needs eight warp-stages of expansion, which eight warps do not
-    // deliver in the 640 cycles of its MMAs; the 8-bit format's expanders need the 96 registers that
-    // only the smaller block leaves them)
-    static constexpr bool kManyExpanders = BN <= 64 || (NA == 2 && FMT == QMM_Q4);
+    // deliver in the 640 cycles of its MMAs)
+    static constexpr bool kManyExpanders = BN <= 64 || NA == 2;
+    // weight slices in flight per expander thread: the 8-bit format's slices are twice as many registers,
+    // so where 16 expander warps leave 80 registers per thread it keeps one (each warp then works on
+    // every other stage of its tile set, so the loads are as far ahead in time)
+    static constexpr int kPrefetch = (FMT == QMM_Q8 && kManyExpanders) ? 1 : kGemmPrefetch;
     static constexpr int kExpWarps = kManyExpanders ? 16 : 8;
     static constexpr int kEpiWarps = kManyExpanders ? 4 : 8;
     // one MMA-issuing warp per weight tile set: each has its own accumulators, so nothing orders
     // their MMAs, and the loop that feeds the tensor pipe (the critical path with two tile sets: it
     // competes with four expander warps for its scheduler) runs in two halves side by side
-    static constexpr int kIssuers = (NA == 2 && FMT == QMM_Q4) ? 2 : 1;   // (8-bit weights: measured 3 % slower with two)
+    static constexpr int kIssuers = NA;
     static constexpr int kThreads = (kExpWarps + kEpiWarps + 1 + kIssuers) * 32;
     static_assert(kStages >= 2 && kStagesB >= 2, "tensor memory or shared memory over-subscribed");
 };
@@ -189,9 +197,6 @@ template <> struct RawRow64<QMM_Q8> {
     }
 };
 
-#ifndef QMM_GEMM_PREFETCH
-#define QMM_GEMM_PREFETCH 2
-#endif
 #ifndef QMM_GEMM_L2_AHEAD
 #define QMM_GEMM_L2_AHEAD 6
 #endif
@@ -203,7 +208,6 @@ template <> struct RawRow64<QMM_Q8> {
 #else
 #define QMM_TRACE_MMA(slot)
 #endif
-constexpr int kGemmPrefetch = QMM_GEMM_PREFETCH;   // weight slices in flight per expander thread
 constexpr int kGemmL2Ahead = QMM_GEMM_L2_AHEAD;    // stages of a row group's weight stream requested into L2 ahead of use
 
 // One piece of work of a block: k-blocks [kb0, kb1) of one output tile.  `cn` blocks contribute to
@@ -265,6 +269,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
     constexpr int NEPI = G::kEpiWarps;
     constexpr int TMA_WARP = NEXP + NEPI, MMA_WARP = NEXP + NEPI + 1;   // issuers: warps MMA_WARP .. MMA_WARP + NISS - 1
     constexpr int NISS = G::kIssuers;
+    constexpr int PREF = G::kPrefetch;                // weight slices in flight per expander thread
     constexpr int S = G::kStages;                     // pipeline depth (weight slots)
     constexpr bool SPLIT = G::kSplit;                 // activation tiles in a ring of their own
     constexpr int SB = G::kStagesB;                   // its depth (== S unless SPLIT)
@@ -433,13 +438,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                 const int ahead = num_kb < kGemmL2Ahead ? num_kb : kGemmL2Ahead;
                 l2_prefetch(wrow, (uint32_t)(ahead * kb_bytes));
             }
-            RawRow64<FMT> raw[kGemmPrefetch];
+            RawRow64<FMT> raw[PREF];
 #pragma unroll
-            for (int i = 0; i < kGemmPrefetch; ++i)
+            for (int i = 0; i < PREF; ++i)
                 if (phase + i * PH < num_kb) raw[i].load(wrow + (size_t)(phase + i * PH) * kb_bytes, lane);
-            for (int kb0 = phase; kb0 < num_kb && ok; kb0 += kGemmPrefetch * PH) {
+            for (int kb0 = phase; kb0 < num_kb && ok; kb0 += PREF * PH) {
 #pragma unroll
-                for (int i = 0; i < kGemmPrefetch; ++i) {
+                for (int i = 0; i < PREF; ++i) {
                     const int kb = kb0 + i * PH;
                     if (kb >= num_kb || !ok) break;
                     const int g = g0 + kb;
@@ -448,7 +453,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                     const bool tr = p.trace != nullptr && blockIdx.x == 0 && g < 64 && quarter == 0 && a == 0 && lane == 0;
                     if (tr) p.trace[g * 8 + 4] = clock64();
                     raw[i].expand(vals, kc);
-                    if (kb + kGemmPrefetch * PH < num_kb) raw[i].load(wrow + (size_t)(kb + kGemmPrefetch * PH) * kb_bytes, lane);
+                    if (kb + PREF * PH < num_kb) raw[i].load(wrow + (size_t)(kb + PREF * PH) * kb_bytes, lane);
                     if (lane == 0 && kb + kGemmL2Ahead < num_kb) l2_prefetch(wrow + (size_t)(kb + kGemmL2Ahead) * kb_bytes, (uint32_t)kb_bytes);
                     if (tr) p.trace[g * 8 + 5] = clock64();
                     if (tr) p.trace[g * 8 + 6] = clock64();
