@@ -125,10 +125,11 @@ struct GemmGeom {
     // (two tile sets: every stage needs eight warp-stages of expansion, which eight warps do not
     // deliver in the 640 cycles of its MMAs)
     static constexpr bool kManyExpanders = BN <= 64 || NA == 2;
-    // weight slices in flight per expander thread: the 8-bit format's slices are twice as many registers,
-    // so where 16 expander warps leave 80 registers per thread it keeps one (each warp then works on
-    // every other stage of its tile set, so the loads are as far ahead in time)
-    static constexpr int kPrefetch = (FMT == QMM_Q8 && kManyExpanders) ? 1 : kGemmPrefetch;
+    // weight slices in flight per expander thread: one where there are 16 expander warps (each warp
+    // then works on every second or fourth stage of its tile set, so its loads are as far ahead in
+    // time as two slices with half the warps; measured 2-4 % faster for the 4-bit format, and the
+    // 8-bit format's slices, twice the registers, only fit the 80 registers per thread this way)
+    static constexpr int kPrefetch = kManyExpanders ? 1 : kGemmPrefetch;
     static constexpr int kExpWarps = kManyExpanders ? 16 : 8;
     static constexpr int kEpiWarps = kManyExpanders ? 4 : 8;
     // one MMA-issuing warp per weight tile set: each has its own accumulators, so nothing orders
