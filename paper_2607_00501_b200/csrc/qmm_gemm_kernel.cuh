@@ -18,7 +18,7 @@
 //
 // Roles (warp specialised):
 //   expanders (8 warps; 16 for token tiles of 64 and narrower and for two tile
-//                      sets of 4-bit weights): several per weight tile and lane
+//                      sets): several per weight tile and lane
 //                      quarter, alternating stages; thread = one weight row;
 //                      32-byte code loads straight from global/L2, unpack to
 //                      fp16(d*q), tcgen05.st into the A ring in TMEM.
@@ -29,8 +29,8 @@
 //                      the staged gate and up values).
 //   TMA producer (1 warp): activation tiles -> shared-memory ring (128-byte
 //                      swizzle), one lane.
-//   MMA issuer (1 warp, converged; one per tile set for two tile sets of 4-bit
-//                      weights): tcgen05.mma (M128 x N x K16, N = the piece's
+//   MMA issuer (1 warp per weight tile set, converged): tcgen05.mma
+//                      (M128 x N x K16, N = the piece's
 //                      valid token rows rounded up to 16) and the
 //                      tcgen05.commit that frees a ring slot, predicated on one
 //                      elected lane (no divergent branch around them).
