@@ -31,6 +31,13 @@
  *   - Device pointers must be 16-byte aligned; packed weight buffers 32-byte.
  *   - Workspaces of qmm_gemm and qmm_moe start with a status word: zero-fill a
  *     workspace once after allocating it.
+ *   - Packed weights are read before the product kernels wait for the work
+ *     that precedes them in the stream (their loads overlap the tail of the
+ *     previous kernel).  A packed buffer must therefore be complete when a
+ *     product call that reads it is enqueued: written by qmm_pack, a copy or
+ *     any ordinary kernel earlier in the same stream is fine; a kernel that
+ *     triggers programmatic dependent launch before it has written the
+ *     weights is not.
  *
  * Canonical block format (what qmm_pack reads)
  *   Q4 block, 18 bytes: uint16 d (fp16 bits, little endian), uint8 qs[16];
@@ -40,6 +47,20 @@
  *   Row n of W holds K/32 consecutive blocks; rows are consecutive; block b of
  *   row n covers k in [32 b, 32 b + 32).  Weight value: float(d) * q (exact in
  *   fp32).  Scales must be finite.
+ *
+ * Accuracy.  With y_ref and sum|w x| evaluated exactly, every output of every
+ * product satisfies |y - y_ref| <= 2e-3 * sum_k |w_k x_k| + 1e-5.  The GEMVs
+ * (qmm_gemv*, decode-sized qmm_moe) multiply integer codes by activations
+ * exactly and apply the scale in fp32, so this holds for every finite scale.
+ * The tensor-core products (qmm_gemm, qmm_moe with more than 32 token-expert
+ * rows) feed each weight to the tensor core as fp16(float(d) * q), which adds
+ * two limits:
+ *   - |d| * max|q| must stay below 65504 (|d| < 8188 for Q4, < 511.75 for Q8),
+ *     else the weight becomes inf; qmm_packed_check reports such scales;
+ *   - a weight with |d * q| < 2^-14 is a subnormal fp16 and carries an absolute
+ *     error of up to 2^-25 instead of a relative one, so the bound becomes
+ *     2e-3 * sum|w x| + 1e-5 + 2^-25 * sum_k |x_k| over such weights (scales of
+ *     N(0, 0.02) data are >= 1.8e-4: the extra term never applies to them).
  */
 #ifndef QMM_H
 #define QMM_H
@@ -59,7 +80,8 @@ typedef enum {
     QMM_ERR_WORKSPACE = 4,     /* workspace missing or smaller than *_workspace_bytes   */
     QMM_ERR_UNSUPPORTED = 5,   /* valid problem outside what the kernels cover          */
     QMM_ERR_CUDA = 6,          /* a CUDA runtime/driver call failed (message has it)    */
-    QMM_ERR_DEVICE_TIMEOUT = 7 /* a bounded wait inside a kernel gave up                */
+    QMM_ERR_DEVICE_TIMEOUT = 7,/* a bounded wait inside a kernel gave up                */
+    QMM_ERR_BAD_WEIGHTS = 8    /* qmm_packed_check: not a packed buffer of that format  */
 } qmm_status;
 
 typedef enum { QMM_Q4 = 4, QMM_Q8 = 8 } qmm_format;
@@ -69,11 +91,14 @@ typedef enum { QMM_Q4 = 4, QMM_Q8 = 8 } qmm_format;
  * NULL; valid until the next failing call on the same thread.               */
 const char* qmm_last_error(void);
 
-/* Library version, major * 10000 + minor * 100 + patch.                     */
+/* Library version, major * 10000 + minor * 100 + patch (the paper's runtime is
+ * reached through a versioned C API, Sec. 3).                               */
 int qmm_version(void);
 
 /* Bytes of the canonical block stream for W[N,K]: N * (K/32) * 18 (Q4) or
- * * 34 (Q8).  0 if the arguments are invalid.                               */
+ * * 34 (Q8).  0 if the arguments are invalid.  (Size queries exist so that the
+ * caller can allocate everything up front and the hot path allocates
+ * nothing, Sec. 3.2.)                                                       */
 size_t qmm_canonical_bytes(qmm_format fmt, int64_t N, int64_t K);
 
 /* Bytes of the device layout produced by qmm_pack (opaque, position
@@ -90,10 +115,29 @@ size_t qmm_packed_bytes(qmm_format fmt, int64_t N, int64_t K);
 qmm_status qmm_pack(qmm_format fmt, const void* canonical, int64_t N, int64_t K,
                     void* packed, void* stream);
 
-/* Validation aid: device layout -> fp32 W[N,K] row-major, w = float(d) * q.
+/* Validation aid: device layout -> fp32 W[N,K] row-major, w = float(d) * q --
+ * the materialised weights that the fused kernels never write (Sec. 3.3
+ * describes dequantisation inside the product's inner loop instead).
  *   packed  device, read only;  w_out  device, N*K floats, written.        */
 qmm_status qmm_dequant(qmm_format fmt, const void* packed, int64_t N, int64_t K,
                        float* w_out, void* stream);
+
+/* Plausibility check of a packed buffer (off the hot path; the product calls
+ * themselves cannot tell a packed buffer from other bytes, because the device
+ * layout has no header: packed_bytes == canonical_bytes, and buffers
+ * concatenate).  A kernel looks at every scale where the layout of `fmt` and
+ * [N, K] puts it; if one is inf / NaN or at least 65504 / max|q| in magnitude
+ * (see "Accuracy" above) it writes QMM_ERR_BAD_WEIGHTS to the status word at
+ * the start of `ws`, which the next qmm_status_check(ws, stream) returns.
+ * Canonical bytes passed as packed, or a buffer of the other format, put code
+ * bytes where scales belong and fail within a few hundred values; a buffer
+ * that passes has finite, tensor-core-safe scales and nothing more is implied.
+ * The paper's loader validates a converted model file once at load time
+ * (Sec. 3.1); this is the same step for one matrix.
+ *   packed  device, read only;  ws  device, >= 16 bytes, zeroed once (any
+ *   qmm_gemm / qmm_moe workspace will do).                                  */
+qmm_status qmm_packed_check(qmm_format fmt, const void* packed, int64_t N, int64_t K,
+                            void* ws, void* stream);
 
 /* Decode matrix-vector product (Sec. 3.3, "GEMV (decode, M=1)"):
  *   y[n] = fp16( sum_b float(d[n,b]) * sum_{i<32} q[n,b,i] * x[32 b + i] ),
@@ -105,7 +149,9 @@ qmm_status qmm_dequant(qmm_format fmt, const void* packed, int64_t N, int64_t K,
  *   x_fp16    device, K fp16 values (bit patterns), read only
  *   y_fp16    device, N fp16 values, written
  *   ws        device, at least qmm_gemv_workspace_bytes(fmt,N,K) bytes; may be
- *             NULL when that size is 0.  Contents are scratch.              */
+ *             NULL when that size is 0, which it is whenever the K split (if
+ *             any) fits a cluster.  Contents are scratch.  (The size query
+ *             follows Sec. 3.2: all memory is obtained before the hot path.) */
 size_t qmm_gemv_workspace_bytes(qmm_format fmt, int64_t N, int64_t K);
 qmm_status qmm_gemv(qmm_format fmt, const void* packed, int64_t N, int64_t K,
                     const uint16_t* x_fp16, uint16_t* y_fp16,
@@ -157,8 +203,12 @@ qmm_status qmm_gemv_gate_up(qmm_format fmt, const void* packed_gate, const void*
  *     rejected with QMM_ERR_WORKSPACE (nothing is enqueued); use qmm_gemv.
  *   - The call allocates nothing and frees nothing, on the host or the device.
  *   - The first call on each device looks up the device address of the scratch
- *     (one runtime query, no allocation).  Make that first call outside any
- *     stream capture, e.g. once at start-up on every device that will be used.
+ *     (one runtime query, no allocation by this library).  If the CUDA runtime
+ *     loads modules lazily, that first use is also when it places the
+ *     library's image -- this array included -- on the device, which can fail
+ *     for lack of memory like any module load.  Make that first call outside
+ *     any stream capture, e.g. once at start-up on every device that will be
+ *     used.
  *   - All calls on a device share the one scratch array, and it keeps whatever
  *     the last call left in it.  The kernels overwrite every element they later
  *     read, so nothing needs clearing, but two calls whose kernels can overlap
@@ -179,7 +229,7 @@ qmm_status qmm_gemv_static(qmm_format fmt, const void* packed, int64_t N, int64_
  *           pieces the K range of those tiles is cut into (added in a fixed
  *           order by a second kernel, so results are the same bits on every
  *           call).  8 KB for most shapes, up to two slots of one output tile
- *           per SM (39 MB) where tiles are cut                               */
+ *           per SM (39 MB) where tiles are cut.  (Size query: Sec. 3.2.)     */
 size_t qmm_gemm_workspace_bytes(qmm_format fmt, int64_t M, int64_t N, int64_t K);
 qmm_status qmm_gemm(qmm_format fmt, const void* packed, int64_t N, int64_t K,
                     const uint16_t* X_fp16, int64_t ldx,
@@ -216,16 +266,46 @@ typedef struct {
     uint16_t* dbg_D;               /* [T*topk, H] fp16 in permuted row order, optional  */
 } qmm_moe_args;
 
-size_t qmm_moe_workspace_bytes(const qmm_moe_args* args);   /* host pointer to args */
+/* Workspace size for these arguments (host pointer to args; only the sizes are
+ * read).  Obtained once, before the hot path (Sec. 3.2).                     */
+size_t qmm_moe_workspace_bytes(const qmm_moe_args* args);
 /* Steps 1-5.  ws: device, >= qmm_moe_workspace_bytes(args).                  */
 qmm_status qmm_moe(const qmm_moe_args* args, void* ws, size_t ws_bytes, void* stream);
-/* Steps 1-2 only; fills the optional routing outputs that are non-NULL.      */
+/* Steps 1-2 only; fills the optional routing outputs that are non-NULL.  (The
+ * paper lists routing among the mixture-of-experts specifics its architecture
+ * descriptor carries, Sec. 3.1, without giving the rule; the rule is above.)  */
 qmm_status qmm_moe_route(const qmm_moe_args* args, void* ws, size_t ws_bytes, void* stream);
 
-/* Waits for `stream`, then reports whether any kernel that used `ws` gave up
- * on a bounded wait (QMM_ERR_DEVICE_TIMEOUT) since the workspace was last
- * cleared by this call.  ws: device workspace of qmm_gemm or qmm_moe.        */
+/* Waits for `stream`, then reports what the kernels that used `ws` recorded in
+ * its status word since this call last cleared it: QMM_ERR_DEVICE_TIMEOUT if a
+ * bounded wait gave up, QMM_ERR_BAD_WEIGHTS from qmm_packed_check, else QMM_OK.
+ * The only call that synchronises; errors otherwise travel through the static
+ * thread-local buffer of qmm_last_error (Sec. 3.2).
+ *   ws: device workspace of qmm_gemm, qmm_moe or qmm_packed_check.           */
 qmm_status qmm_status_check(void* ws, void* stream);
+
+/* ---- debug entry points (tests and tuning; no counterpart in the paper) ----
+ *
+ * qmm_debug_config sets a process-wide knob that forces a launch geometry;
+ * none changes a result beyond the order of fp32 additions.  The library
+ * reads no environment variable.  Not synchronised: call it while no other
+ * thread is inside the library.  name == NULL resets every knob; value NULL,
+ * "" or "0" clears the named one.
+ *   "gemv_force"       "warps,splits"  block size (8 | 16 warps) and K split of qmm_gemv
+ *   "gemv_no_cluster"  "1"             K split through workspace partial sums + second kernel
+ *   "gemm_force"       "bn[,units]"    token tile and (tile, k-block) units per block of qmm_gemm
+ *   "gemm_no_tail_cut" "1"             last, partly filled round of tiles left whole
+ *   "moe_no_fuse"      "1"             decode-sized qmm_moe as separate route / product / combine launches
+ */
+qmm_status qmm_debug_config(const char* name, const char* value);
+
+/* Exercises the give-up path of the kernels' bounded waits without any other
+ * work in flight: one warp waits on a barrier that nothing completes for
+ * limit_cycles clock cycles (1 .. 2^24, i.e. at most ~10 ms), then records
+ * QMM_ERR_DEVICE_TIMEOUT in the status word at the start of ws, as a GEMM
+ * kernel whose pipeline stalled would.  The next qmm_status_check(ws, stream)
+ * returns it; the context stays usable.  ws: device, >= 16 bytes.           */
+qmm_status qmm_debug_wait_give_up(void* ws, int64_t limit_cycles, void* stream);
 
 #ifdef __cplusplus
 }

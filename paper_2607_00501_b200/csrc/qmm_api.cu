@@ -33,7 +33,7 @@ qmm_status check_cuda(cudaError_t e, const char* what)
 // defined in the kernel files
 qmm_status launch_pack(int fmt, const void* canon, int64_t N, int64_t K, void* packed, cudaStream_t st);
 qmm_status launch_dequant(int fmt, const void* packed, int64_t N, int64_t K, float* w_out, cudaStream_t st);
-size_t gemv_workspace_bytes(int fmt, int64_t N, int64_t K);
+size_t gemv_workspace_bytes(int fmt, int64_t N, int64_t K, bool allow_cluster);
 qmm_status launch_gemv(int fmt, const void* packed, int64_t N, int64_t K, const uint16_t* x, uint16_t* y,
                        void* ws, bool allow_cluster, cudaStream_t st);
 qmm_status launch_gemv_batch(int fmt, const qmm_gemv_problem* probs, int count, cudaStream_t st);
@@ -45,6 +45,10 @@ qmm_status launch_gemm(int fmt, const void* packed, int64_t N, int64_t K, const 
 size_t moe_workspace_bytes(const qmm_moe_args* a);
 qmm_status launch_moe(const qmm_moe_args* a, void* ws, bool route_only, cudaStream_t st);
 qmm_status status_check(void* ws, cudaStream_t st);
+qmm_status launch_packed_check(int fmt, const void* packed, int64_t N, int64_t K, int* status, cudaStream_t st);
+qmm_status launch_wait_give_up(int* status, long long limit_cycles, cudaStream_t st);
+
+DebugKnobs g_knobs = {};
 
 static bool fmt_ok(int fmt) { return fmt == QMM_Q4 || fmt == QMM_Q8; }
 
@@ -131,7 +135,7 @@ qmm_status qmm_dequant(qmm_format fmt, const void* packed, int64_t N, int64_t K,
 size_t qmm_gemv_workspace_bytes(qmm_format fmt, int64_t N, int64_t K)
 {
     if (check_matrix("qmm_gemv_workspace_bytes", fmt, N, K) != QMM_OK) return 0;
-    return gemv_workspace_bytes(fmt, N, K);
+    return gemv_workspace_bytes(fmt, N, K, true);
 }
 
 qmm_status qmm_gemv(qmm_format fmt, const void* packed, int64_t N, int64_t K,
@@ -144,7 +148,7 @@ qmm_status qmm_gemv(qmm_format fmt, const void* packed, int64_t N, int64_t K,
     if (!aligned(x_fp16, 16) || !aligned(y_fp16, 16))
         return fail(QMM_ERR_ALIGNMENT, "qmm_gemv: x and y must be 16-byte aligned");
     if (K > 32768) return fail(QMM_ERR_UNSUPPORTED, "qmm_gemv: K=%lld > 32768", (long long)K);
-    const size_t need = gemv_workspace_bytes(fmt, N, K);
+    const size_t need = gemv_workspace_bytes(fmt, N, K, true);
     if (need > 0) {
         if (!ws || ws_bytes < need)
             return fail(QMM_ERR_WORKSPACE, "qmm_gemv: workspace of %zu bytes needed, %zu given", need, ws ? ws_bytes : (size_t)0);
@@ -271,6 +275,68 @@ qmm_status qmm_status_check(void* ws, void* stream)
 {
     if (!ws) return fail(QMM_ERR_INVALID_ARG, "qmm_status_check: null workspace");
     return status_check(ws, (cudaStream_t)stream);
+}
+
+qmm_status qmm_packed_check(qmm_format fmt, const void* packed, int64_t N, int64_t K, void* ws, void* stream)
+{
+    qmm_status s = check_matrix("qmm_packed_check", fmt, N, K);
+    if (s != QMM_OK) return s;
+    if (!packed || !ws) return fail(QMM_ERR_INVALID_ARG, "qmm_packed_check: null pointer");
+    if (!aligned(packed, 32)) return fail(QMM_ERR_ALIGNMENT, "qmm_packed_check: packed must be 32-byte aligned");
+    if (!aligned(ws, 16)) return fail(QMM_ERR_ALIGNMENT, "qmm_packed_check: workspace must be 16-byte aligned");
+    if ((s = check_device("qmm_packed_check")) != QMM_OK) return s;
+    return launch_packed_check(fmt, packed, N, K, (int*)ws, (cudaStream_t)stream);
+}
+
+qmm_status qmm_debug_config(const char* name, const char* value)
+{
+    if (!name) {                                                // reset every knob
+        g_knobs = DebugKnobs{};
+        return QMM_OK;
+    }
+    const bool off = value == nullptr || value[0] == 0 || strcmp(value, "0") == 0;
+    if (strcmp(name, "gemv_force") == 0) {
+        int w = 0, sp = 0;
+        if (off) {
+            g_knobs.gemv_warps = g_knobs.gemv_splits = 0;
+            return QMM_OK;
+        }
+        if (sscanf(value, "%d,%d", &w, &sp) != 2 || (w != 8 && w != 16) || sp < 1 || sp > 64)
+            return fail(QMM_ERR_INVALID_ARG, "qmm_debug_config: gemv_force wants \"warps,splits\" with warps 8 or 16, 1 <= splits <= 64");
+        g_knobs.gemv_warps = w;
+        g_knobs.gemv_splits = sp;
+        return QMM_OK;
+    }
+    if (strcmp(name, "gemm_force") == 0) {
+        int b = 0, u = 0;
+        if (off) {
+            g_knobs.gemm_bn = g_knobs.gemm_units = 0;
+            return QMM_OK;
+        }
+        const int got = sscanf(value, "%d,%d", &b, &u);
+        if (got < 1 || !(b == 32 || b == 64 || b == 128 || b == 160 || b == 192 || b == 256) || (got == 2 && u < 1))
+            return fail(QMM_ERR_INVALID_ARG, "qmm_debug_config: gemm_force wants \"bn[,units]\" with bn in {32,64,128,160,192,256}");
+        g_knobs.gemm_bn = b;
+        g_knobs.gemm_units = got == 2 ? u : 0;
+        return QMM_OK;
+    }
+    int* flag = strcmp(name, "gemv_no_cluster") == 0    ? &g_knobs.gemv_no_cluster
+                : strcmp(name, "gemm_no_tail_cut") == 0 ? &g_knobs.gemm_no_tail_cut
+                : strcmp(name, "moe_no_fuse") == 0      ? &g_knobs.moe_no_fuse
+                                                        : nullptr;
+    if (!flag) return fail(QMM_ERR_INVALID_ARG, "qmm_debug_config: unknown knob \"%s\"", name);
+    *flag = off ? 0 : 1;
+    return QMM_OK;
+}
+
+qmm_status qmm_debug_wait_give_up(void* ws, int64_t limit_cycles, void* stream)
+{
+    if (!ws) return fail(QMM_ERR_INVALID_ARG, "qmm_debug_wait_give_up: null workspace");
+    if (limit_cycles < 1 || limit_cycles > (1LL << 24))
+        return fail(QMM_ERR_INVALID_ARG, "qmm_debug_wait_give_up: limit of %lld cycles outside [1, 2^24]", (long long)limit_cycles);
+    qmm_status s = check_device("qmm_debug_wait_give_up");
+    if (s != QMM_OK) return s;
+    return launch_wait_give_up((int*)ws, (long long)limit_cycles, (cudaStream_t)stream);
 }
 
 }  // extern "C"

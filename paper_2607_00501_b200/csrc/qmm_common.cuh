@@ -57,6 +57,19 @@ __host__ __device__ inline int tile_bytes_of(int fmt) { return fmt == QMM_Q4 ? k
 qmm_status fail(qmm_status code, const char* fmt, ...);
 qmm_status check_cuda(cudaError_t e, const char* what);
 
+// Debug knobs set through qmm_debug_config (tests and tuning sweeps force launch geometries
+// with them; none changes a result beyond the order of fp32 additions).  Plain process-wide
+// values, all zero by default: the launch path reads them and nothing else -- no environment
+// variable is looked at after the library is loaded.
+struct DebugKnobs {
+    int gemv_warps, gemv_splits;    // 0: the plan decides
+    int gemv_no_cluster;            // split-K GEMV through workspace partial sums and a second kernel
+    int gemm_bn, gemm_units;        // token tile / (tile, k-block) units per block of the dense GEMM; 0: the plan decides
+    int gemm_no_tail_cut;           // leave the tiles of the last, partly filled round whole
+    int moe_no_fuse;                // decode-sized MoE layers as four separate launches
+};
+extern DebugKnobs g_knobs;
+
 // ---------------------------------------------------------------- loads
 
 struct __align__(32) u32x8 {

@@ -6,7 +6,6 @@
 #include <atomic>
 #include <math.h>
 #include <stdio.h>
-#include <stdlib.h>
 
 namespace qmm {
 
@@ -249,14 +248,9 @@ static GemmPlan gemm_plan(int64_t M, int64_t N, int64_t K)
         if (round_cost(t192, kb, 470, 300).cycles < round_cost(t256, kb, 515, 2400).cycles) p.bn = 192;
     }
     int force_units = 0;
-    if (const char* f = getenv("QMM_GEMM_FORCE")) {            // "bn,na[,units]" for tuning sweeps and tests
-        int b = 0, a = 0, u = 0;
-        const int got = sscanf(f, "%d,%d,%d", &b, &a, &u);
-        if (got >= 2 && a == 1 && (b == 32 || b == 64 || b == 128 || b == 160 || b == 192 || b == 256)) {
-            p.bn = b;
-            p.na = a;
-            if (got >= 3 && u >= 1) force_units = u;
-        }
+    if (g_knobs.gemm_bn) {                                      // forced by qmm_debug_config("gemm_force", "bn[,units]")
+        p.bn = g_knobs.gemm_bn;
+        force_units = g_knobs.gemm_units;
     }
     const int64_t tiles = (N / (128 * p.na)) * ((M + p.bn - 1) / p.bn);
     const int64_t KB = K / kGemmBK;
@@ -269,7 +263,7 @@ static GemmPlan gemm_plan(int64_t M, int64_t N, int64_t K)
         // whole tiles, the same number for every block; the tiles of the last, partly filled round
         // are cut into equal shares of their units when round_cost says that pays
         const RoundCost rc = p.bn == 256 ? round_cost(tiles, KB, 515, 2400) : round_cost(tiles, KB, 470, 300);
-        if (rc.halve_tail && getenv("QMM_GEMM_NO_TAIL_CUT") == nullptr) {
+        if (rc.halve_tail && !g_knobs.gemm_no_tail_cut) {
             p.grid = kNumSMs;
             p.whole = (int)(tiles / kNumSMs) * kNumSMs;
             p.halves = true;
@@ -277,7 +271,7 @@ static GemmPlan gemm_plan(int64_t M, int64_t N, int64_t K)
             p.cut = false;
             return p;
         }
-        if (rc.cut_tail && getenv("QMM_GEMM_NO_TAIL_CUT") == nullptr) {
+        if (rc.cut_tail && !g_knobs.gemm_no_tail_cut) {
             p.grid = kNumSMs;
             p.whole = (int)(tiles / kNumSMs) * kNumSMs;
             units = ((tiles - p.whole) * KB + kNumSMs - 1) / kNumSMs;
@@ -335,7 +329,9 @@ qmm_status launch_gemm(int fmt, const void* packed, int64_t N, int64_t K, const 
     p.units_per_block = plan.units;
     p.partial = (float*)((uint8_t*)ws + kGemmWsHeader);
     p.status = (int*)ws;
-    if (getenv("QMM_GEMM_TRACE")) p.trace = (long long*)((uint8_t*)ws + kGemmWsTrace);   // tuning aid
+#if QMM_GEMM_TRACE
+    p.trace = (long long*)((uint8_t*)ws + kGemmWsTrace);                   // tuning builds only
+#endif
     s = launch_tc_gemm(fmt, bn, na, kEpiStore, true, map, p, dim3((unsigned)plan.grid), st);
     if (s != QMM_OK || !plan.cut) return s;
     const int n_tiles = (int)(N / (128 * na));
@@ -354,6 +350,33 @@ qmm_status launch_gemm(int fmt, const void* packed, int64_t N, int64_t K, const 
                       "qmm_gemm partial-sum kernel launch");
 }
 
+// Debug aid: the give-up path of the bounded waits on its own.  One warp waits on an mbarrier that
+// nobody ever arrives on, with a short limit; no TMA load and no tensor-core operation is in flight, so
+// giving up has nothing to unwind.  The kernel then does what the GEMM kernels do on give-up: raise
+// the abort flag, write QMM_ERR_DEVICE_TIMEOUT to the status word, return.
+__global__ void wait_give_up_kernel(int* status, long long limit_cycles)
+{
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        tc::mbar_init(&bar, 1);
+        abort_flag = 0;
+        tc::fence_barrier_init();
+    }
+    __syncthreads();
+    bool ok = tc::mbar_wait(&bar, 0, &abort_flag, limit_cycles);
+    ok = __all_sync(0xFFFFFFFFu, ok);
+    if (!ok) abort_flag = 1;
+    __syncthreads();
+    if (threadIdx.x == 0 && abort_flag) atomicExch(status, (int)QMM_ERR_DEVICE_TIMEOUT);
+}
+
+qmm_status launch_wait_give_up(int* status, long long limit_cycles, cudaStream_t st)
+{
+    wait_give_up_kernel<<<1, 32, 0, st>>>(status, limit_cycles);
+    return check_cuda(cudaGetLastError(), "qmm_debug_wait_give_up launch");
+}
+
 // Reads and clears the device status word (first int of a GEMM / MoE workspace).
 qmm_status status_check(void* ws, cudaStream_t st)
 {
@@ -367,6 +390,8 @@ qmm_status status_check(void* ws, cudaStream_t st)
         if (e != cudaSuccess) return check_cuda(e, "qmm_status_check");
         if (h == QMM_ERR_DEVICE_TIMEOUT)
             return fail(QMM_ERR_DEVICE_TIMEOUT, "a kernel gave up on a bounded wait (pipeline barrier never completed)");
+        if (h == QMM_ERR_BAD_WEIGHTS)
+            return fail(QMM_ERR_BAD_WEIGHTS, "qmm_packed_check found a scale that is inf/NaN or out of range: not a packed buffer of that format and shape");
         return fail(QMM_ERR_CUDA, "device status word holds unexpected value %d", h);
     }
     return QMM_OK;

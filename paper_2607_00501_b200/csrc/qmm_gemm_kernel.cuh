@@ -85,7 +85,7 @@ struct GemmParams {
     int units_per_block;             // U: share of the (tile, k-block) units of the other tiles
     float* partial;                  // [2 * gridDim.x] slots of NA*BN*128 floats (when some tile is cut)
     int* status;                     // device status word (0 = ok)
-    long long* trace;                // optional [block 0 only] clock64 samples for pipeline analysis (tuning aid), else null
+    long long* trace;                // clock64 samples of block 0 in -DQMM_GEMM_TRACE=1 builds; unused (null) otherwise
 };
 
 // Pipeline geometry of one instantiation.  Tensor memory: half of the SM's 512 columns when the
@@ -201,9 +201,19 @@ template <> struct RawRow64<QMM_Q8> {
 #ifndef QMM_GEMM_L2_AHEAD
 #define QMM_GEMM_L2_AHEAD 6
 #endif
-// Clock samples of the issuing loop of block 0 (tuning aid): compiled in only with -DQMM_GEMM_TRACE_MMA=1,
-// because even a skipped sample costs the issuing warp instructions in its critical loop.
-#if defined(QMM_GEMM_TRACE_MMA) && QMM_GEMM_TRACE_MMA
+// Clock samples of block 0's pipeline (tuning aid) exist only in builds with -DQMM_GEMM_TRACE=1: the
+// shipped kernels carry no trace code.  The issuing loop's own samples need -DQMM_GEMM_TRACE_MMA=1 as
+// well, because even a skipped sample costs the issuing warp instructions in its critical loop.
+#ifndef QMM_GEMM_TRACE
+#define QMM_GEMM_TRACE 0
+#endif
+#if QMM_GEMM_TRACE
+#define QMM_TRACE_AT(cond, idx) \
+    if (cond) p.trace[idx] = clock64();
+#else
+#define QMM_TRACE_AT(cond, idx)
+#endif
+#if QMM_GEMM_TRACE && defined(QMM_GEMM_TRACE_MMA) && QMM_GEMM_TRACE_MMA
 #define QMM_TRACE_MMA(slot) \
     if (tracing && g + 1 < 64) p.trace[g * 8 + (slot)] = p.trace[(g + 1) * 8 + (slot)] = clock64();
 #else
@@ -451,18 +461,18 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                     const int g = g0 + kb;
                     const int s = g % S;
                     uint32_t vals[32];
-                    const bool tr = p.trace != nullptr && blockIdx.x == 0 && g < 64 && quarter == 0 && a == 0 && lane == 0;
-                    if (tr) p.trace[g * 8 + 4] = clock64();
+                    [[maybe_unused]] const bool tr = QMM_GEMM_TRACE && p.trace != nullptr && blockIdx.x == 0 && g < 64 && quarter == 0 && a == 0 && lane == 0;
+                    QMM_TRACE_AT(tr, g * 8 + 4)
                     raw[i].expand(vals, kc);
                     if (kb + PREF * PH < num_kb) raw[i].load(wrow + (size_t)(kb + PREF * PH) * kb_bytes, lane);
                     if (lane == 0 && kb + kGemmL2Ahead < num_kb) l2_prefetch(wrow + (size_t)(kb + kGemmL2Ahead) * kb_bytes, (uint32_t)kb_bytes);
-                    if (tr) p.trace[g * 8 + 5] = clock64();
-                    if (tr) p.trace[g * 8 + 6] = clock64();
+                    QMM_TRACE_AT(tr, g * 8 + 5)
+                    QMM_TRACE_AT(tr, g * 8 + 6)
                     if (g >= S) ok = mbar_wait(&empty[s], ((g / S) - 1) & 1, abort_flag);
                     ok = __all_sync(0xFFFFFFFFu, ok);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    if (tr) p.trace[g * 8 + 7] = clock64();
+                    QMM_TRACE_AT(tr, g * 8 + 7)
                     tmem_st_32x32b_x32(lane_base + (uint32_t)(RING0 + s * A_COLS + a * 32), vals);
                     // announce the slot at once: deferring the wait for the store behind the next
                     // expansion was measured and costs more in slot turn-around than the ~85 cycles it hides
@@ -488,7 +498,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         constexpr int NOUT = (EPI == kEpiSiluMul) ? 1 : NA;               // output tiles per weight row
         constexpr int NSTG = NA;                                          // tile sets that go through the staging buffer
         pdl_wait();                                                       // the output buffer may be in use upstream
-        bool ok = true, etr = false;
+        bool ok = true;
+        [[maybe_unused]] bool etr = false;
         int it = 0, staged = 0;                                           // pieces seen / tiles that went through the staging buffer
         const uint32_t stg_lane = smem_u32(staging) + (uint32_t)((quarter * 32 + lane) * 4);   // this thread's weight row
         // 32 tokens (one chunk) of this thread's weight row -> staging[o][(c0 + 2j) / 2][row] as fp16
@@ -504,7 +515,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty[buf]);
-            if (etr) p.trace[(it * 4 + 2) * 8 + 1] = clock64();
+            QMM_TRACE_AT(etr, (it * 4 + 2) * 8 + 1)
         };
         GemmWork w;
         for (; ok && get_work(it, w); ++it) {
@@ -515,8 +526,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
             tc_fence_after_sync();
-            etr = p.trace != nullptr && blockIdx.x == 0 && it < 16 && e == 0 && lane == 0;
-            if (etr) p.trace[(it * 4 + 1) * 8 + 1] = clock64();
+            etr = QMM_GEMM_TRACE && p.trace != nullptr && blockIdx.x == 0 && it < 16 && e == 0 && lane == 0;
+            QMM_TRACE_AT(etr, (it * 4 + 1) * 8 + 1)
             if (DENSE && w.cn > 1) {
                 // a tile cut by block boundaries (dense mode only): out of line, so that its registers
                 // do not weigh on the common path
@@ -649,8 +660,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         // The issuing lane.  The MMAs and commits below are predicated on it instead of sitting in a
         // divergent branch: measured ~25 % less issue time per stage (operands stay warp-uniform).
         const uint32_t sel = elect_one() ? 1u : 0u;
-        const bool tracing = p.trace != nullptr && blockIdx.x == 0 && lane == 0 && warp == MMA_WARP;
-        (void)tracing;
+        [[maybe_unused]] const bool tracing = QMM_GEMM_TRACE && p.trace != nullptr && blockIdx.x == 0 && lane == 0 && warp == MMA_WARP;
         (void)g;
         int s = 0;                                                        // ring slot of stage g and the parity of its
         uint32_t par = 0;                                                 // "full" barrier, carried across pieces
@@ -664,7 +674,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
                 tc_fence_after_sync();
-                if (p.trace != nullptr && blockIdx.x == 0 && it <= 16 && lane == 0 && warp == MMA_WARP) p.trace[((it - AB) * 4 + 3) * 8 + 1] = clock64();
+                QMM_TRACE_AT(tracing && it <= 16, ((it - AB) * 4 + 3) * 8 + 1)
             }
             const uint32_t d_tmem = tmem_base + (uint32_t)(buf * D_COLS);
             // The MMAs' N is the piece's valid token rows rounded up to 16 (a partly filled expert tile,
@@ -757,7 +767,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             }
             if (ok) mma_commit_sel(&acc_full[buf], sel);                  // accumulators of this piece are complete
             __syncwarp();
-            if (p.trace != nullptr && blockIdx.x == 0 && it < 16 && lane == 0 && warp == MMA_WARP) p.trace[(it * 4 + 0) * 8 + 1] = clock64();
+            QMM_TRACE_AT(tracing && it < 16, (it * 4 + 0) * 8 + 1)
         }
         if (!ok) *abort_flag = 1;
     }

@@ -16,7 +16,6 @@
 #include "qmm_common.cuh"
 
 #include <stdio.h>
-#include <stdlib.h>
 
 namespace qmm {
 
@@ -629,12 +628,9 @@ GemvPlan gemv_plan(int fmt, int64_t N, int64_t K, bool cluster)
     const int max_splits = cluster ? kPlanClusterSplits : 16;
     while (groups * splits < kNumSMs && tpr / (splits * 2) >= warps && (tpr % (splits * 2)) == 0 && splits < max_splits)
         splits *= 2;
-    if (const char* f = getenv("QMM_GEMV_FORCE")) {           // "warps,splits" for sweeps
-        int w = 0, s = 0;
-        if (sscanf(f, "%d,%d", &w, &s) == 2 && (w == 8 || w == 16) && s >= 1 && tpr % s == 0) {
-            warps = w;
-            splits = s;
-        }
+    if (g_knobs.gemv_warps && tpr % g_knobs.gemv_splits == 0) {   // forced by qmm_debug_config("gemv_force", "warps,splits")
+        warps = g_knobs.gemv_warps;
+        splits = g_knobs.gemv_splits;
     }
     p.warps = warps;
     p.splits = splits;
@@ -644,10 +640,14 @@ GemvPlan gemv_plan(int fmt, int64_t N, int64_t K, bool cluster)
     return p;
 }
 
-size_t gemv_workspace_bytes(int fmt, int64_t N, int64_t K)
+// Workspace of the K split.  The cluster form (up to kMaxClusterSplits blocks per item, sums added
+// through distributed shared memory) needs none; the two-kernel form holds fp32 partial sums [splits][N].
+size_t gemv_workspace_bytes(int fmt, int64_t N, int64_t K, bool allow_cluster)
 {
-    const GemvPlan p = gemv_plan(fmt, N, K, false);            // the two-kernel form (the cluster form needs none)
-    return p.splits > 1 ? (size_t)p.splits * (size_t)N * sizeof(float) : 0;
+    if (g_knobs.gemv_no_cluster) allow_cluster = false;
+    const GemvPlan p = gemv_plan(fmt, N, K, allow_cluster);
+    if (p.splits <= 1 || (allow_cluster && p.splits <= kMaxClusterSplits)) return 0;
+    return (size_t)p.splits * (size_t)N * sizeof(float);
 }
 
 template <typename... Args>
@@ -824,7 +824,7 @@ qmm_status launch_gemv_batch(int fmt, const qmm_gemv_problem* probs, int count, 
 qmm_status launch_gemv(int fmt, const void* packed, int64_t N, int64_t K, const uint16_t* x, uint16_t* y,
                        void* ws, bool allow_cluster, cudaStream_t st)
 {
-    if (getenv("QMM_GEMV_NO_CLUSTER")) allow_cluster = false;          // tuning aid / tests of the two-kernel form
+    if (g_knobs.gemv_no_cluster) allow_cluster = false;               // tests of the two-kernel form
     const GemvPlan p = gemv_plan(fmt, N, K, allow_cluster);
     float* partial = (float*)ws;
 #define QMM_GEMV_CASE(F, W) \
@@ -896,7 +896,7 @@ extern "C" qmm_status qmm_gemv_static(qmm_format fmt, const void* packed, int64_
     if ((reinterpret_cast<uintptr_t>(packed) & 31) || (reinterpret_cast<uintptr_t>(x_fp16) & 15) ||
         (reinterpret_cast<uintptr_t>(y_fp16) & 15))
         return fail(QMM_ERR_ALIGNMENT, "qmm_gemv_static: packed must be 32-byte aligned, x and y 16-byte aligned");
-    const size_t need = gemv_workspace_bytes(fmt, N, K);
+    const size_t need = gemv_workspace_bytes(fmt, N, K, false);       // always the two-kernel form here
     if (need > (size_t)QMM_GEMV_STATIC_SCRATCH_BYTES)
         return fail(QMM_ERR_WORKSPACE,
                     "qmm_gemv_static: this shape needs %zu bytes of split-K scratch, the built-in scratch holds %d; "

@@ -11,8 +11,6 @@
 // GEMMs is built on the device from the expert offsets.
 #include "qmm_gemm_kernel.cuh"
 
-#include <stdlib.h>
-
 namespace qmm {
 
 qmm_status make_x_map(CUtensorMap* map, const uint16_t* X, int64_t rows, int64_t K, int64_t ld, int box_rows);
@@ -457,7 +455,9 @@ qmm_status launch_moe(const qmm_moe_args* a, void* ws, bool route_only, cudaStre
         p.tile_rows = tile_rows;
         p.num_tiles = num_tiles;
         p.status = status;
-        if (getenv("QMM_GEMM_TRACE")) p.trace = (long long*)(base + w.trace);
+#if QMM_GEMM_TRACE
+        p.trace = (long long*)(base + w.trace);                            // tuning builds only
+#endif
         s = launch_tc_gemm(a->fmt, w.bn, 2, kEpiSiluMul, false, map, p, persistent_grid(w.bn, 2, 0), st);
         if (s != QMM_OK) return s;
     }

@@ -105,6 +105,48 @@ __global__ void dequant_kernel(const uint8_t* __restrict__ packed, float* __rest
     }
 }
 
+// Plausibility check of a packed buffer: one thread per (row, tile) looks at the row's scale(s) where
+// the layout of `FMT` puts them.  A scale that is inf / NaN, or so large that |d| * max|q| leaves the
+// fp16 range (the tensor-core products multiply d * q in fp16), marks the buffer as bad.  Bytes that are
+// not a packed buffer of this format and shape (canonical blocks, the other format) put code bytes where
+// scales are expected, and code bytes fail this test within a few hundred values.
+template <int FMT>
+__global__ void packed_check_kernel(const uint8_t* __restrict__ packed, int64_t N, int64_t tiles_per_row, int* __restrict__ status)
+{
+    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= N * tiles_per_row) return;
+    const int64_t tile_idx = idx / kRowsPerGroup;                         // tiles are consecutive in memory
+    const int r = (int)(idx % kRowsPerGroup);
+    const uint8_t* tile = packed + tile_idx * Fmt<FMT>::tile_bytes;
+    constexpr float kMaxAbs = FMT == QMM_Q4 ? 65504.0f / 8.0f : 65504.0f / 128.0f;
+    bool bad = false;
+    auto look = [&](uint16_t bits) {
+        const float d = __half2float(__ushort_as_half(bits));
+        bad |= !(fabsf(d) < kMaxAbs);                                     // also true for NaN
+    };
+    if (FMT == QMM_Q4) {
+        const uint32_t dd = *reinterpret_cast<const uint32_t*>(tile + kTileCodeBytes + 4 * r);
+        look((uint16_t)(dd & 0xFFFFu));
+        look((uint16_t)(dd >> 16));
+    } else {
+        look(*reinterpret_cast<const uint16_t*>(tile + kTileCodeBytes + 2 * r));
+    }
+    if (bad) atomicExch(status, (int)QMM_ERR_BAD_WEIGHTS);
+}
+
+qmm_status launch_packed_check(int fmt, const void* packed, int64_t N, int64_t K, int* status, cudaStream_t st)
+{
+    const int64_t tpr = K / tile_k_of(fmt);
+    const int64_t total = N * tpr;
+    const int threads = 256;
+    const int64_t blocks = (total + threads - 1) / threads;
+    if (fmt == QMM_Q4)
+        packed_check_kernel<QMM_Q4><<<(unsigned)blocks, threads, 0, st>>>((const uint8_t*)packed, N, tpr, status);
+    else
+        packed_check_kernel<QMM_Q8><<<(unsigned)blocks, threads, 0, st>>>((const uint8_t*)packed, N, tpr, status);
+    return check_cuda(cudaGetLastError(), "qmm_packed_check launch");
+}
+
 qmm_status launch_pack(int fmt, const void* canon, int64_t N, int64_t K, void* packed, cudaStream_t st)
 {
     const int64_t tpr = K / tile_k_of(fmt);

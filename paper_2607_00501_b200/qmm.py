@@ -24,6 +24,7 @@ _lib = None
 STATUS_NAMES = {
     0: "QMM_OK", 1: "QMM_ERR_INVALID_ARG", 2: "QMM_ERR_SHAPE", 3: "QMM_ERR_ALIGNMENT",
     4: "QMM_ERR_WORKSPACE", 5: "QMM_ERR_UNSUPPORTED", 6: "QMM_ERR_CUDA", 7: "QMM_ERR_DEVICE_TIMEOUT",
+    8: "QMM_ERR_BAD_WEIGHTS",
 }
 
 # every symbol include/qmm.h declares
@@ -31,7 +32,7 @@ EXPORTS = (
     "qmm_last_error", "qmm_version", "qmm_canonical_bytes", "qmm_packed_bytes", "qmm_pack",
     "qmm_dequant", "qmm_gemv_workspace_bytes", "qmm_gemv", "qmm_gemm_workspace_bytes", "qmm_gemm",
     "qmm_moe_workspace_bytes", "qmm_moe", "qmm_moe_route", "qmm_status_check", "qmm_gemv_static", "qmm_gemv_batch",
-    "qmm_gemv_gate_up",
+    "qmm_gemv_gate_up", "qmm_packed_check", "qmm_debug_config", "qmm_debug_wait_give_up",
 )
 
 
@@ -93,6 +94,9 @@ def lib() -> ctypes.CDLL:
             L.qmm_moe.argtypes = [ctypes.POINTER(MoeArgs), vp, sz, vp]
             L.qmm_moe_route.argtypes = [ctypes.POINTER(MoeArgs), vp, sz, vp]
             L.qmm_status_check.argtypes = [vp, vp]
+            L.qmm_packed_check.argtypes = [ci, vp, i64, i64, vp, vp]
+            L.qmm_debug_config.argtypes = [ctypes.c_char_p, ctypes.c_char_p]
+            L.qmm_debug_wait_give_up.argtypes = [vp, i64, vp]
             _lib = L
     return _lib
 
@@ -260,3 +264,18 @@ def moe_route(args: MoeArgs, ws: torch.Tensor) -> None:
 
 def status_check(ws: torch.Tensor) -> None:
     _check(lib().qmm_status_check(ws.data_ptr(), _stream()))
+
+
+def packed_check(fmt: int, packed: torch.Tensor, N: int, K: int, ws: torch.Tensor) -> None:
+    """Enqueue the plausibility check of a packed buffer; status_check(ws) reports the verdict."""
+    _check(lib().qmm_packed_check(fmt, packed.data_ptr(), N, K, ws.data_ptr(), _stream()))
+
+
+def debug_config(name: str | None, value: str | None = None) -> None:
+    """Set (or with value None clear) a debug knob; name None resets all of them."""
+    enc = lambda v: None if v is None else str(v).encode()
+    _check(lib().qmm_debug_config(enc(name), enc(value)))
+
+
+def debug_wait_give_up(ws: torch.Tensor, limit_cycles: int) -> None:
+    _check(lib().qmm_debug_wait_give_up(ws.data_ptr(), int(limit_cycles), _stream()))

@@ -17,3 +17,12 @@ def oracle():
     import oracle as _oracle
     _oracle.build()
     return _oracle
+
+
+@pytest.fixture(autouse=True)
+def _reset_debug_knobs():
+    """Forced launch geometries (qmm_debug_config) never leak from one test into the next."""
+    yield
+    mod = sys.modules.get("paper_2607_00501_b200.qmm")
+    if mod is not None and mod._lib is not None:
+        mod.debug_config(None)

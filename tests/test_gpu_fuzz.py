@@ -47,7 +47,7 @@ def test_random_gemm_shapes(qmm, oracle, case):
 
 
 @pytest.mark.parametrize("case", range(10))
-def test_random_many_tile_gemm_plans_agree(qmm, oracle, monkeypatch, case):
+def test_random_many_tile_gemm_plans_agree(qmm, oracle, case):
     """Shapes with more output tiles than SMs: the plan gives every block whole tiles and treats the
     last, partly filled round in one of three ways (whole tiles, half tiles, shares of the K range with
     partial sums).  Whatever it picks must agree with the whole-tile plan -- bit for bit unless partial
@@ -58,8 +58,7 @@ def test_random_many_tile_gemm_plans_agree(qmm, oracle, monkeypatch, case):
         M, N, K = int(rng.integers(600, 4600)), int(rng.integers(4, 40)) * 128, int(rng.integers(1, 33)) * 256
         if (N // 128) * ((M + 255) // 256) > 148:
             break
-    monkeypatch.delenv("QMM_GEMM_FORCE", raising=False)
-    monkeypatch.delenv("QMM_GEMM_NO_TAIL_CUT", raising=False)
+    qmm.debug_config(None)
     blocks, _, _ = util.random_blocks(synth, fmt, N, K, seed=842 + case, special_scales=False)
     X = synth.activations(843, case, M, K)
     packed, Xd = qmm.pack(fmt, util.dev(blocks), N, K), util.dev(X)
@@ -71,7 +70,7 @@ def test_random_many_tile_gemm_plans_agree(qmm, oracle, monkeypatch, case):
     rows = np.unique(np.concatenate([[0, M - 1, M - 129 if M > 129 else 0], rng.integers(0, M, size=5)]))
     Y_ref, B = oracle.gemm(fmt, blocks, N, K, X[rows])
     util.assert_within_tol(util.host_f64(Y)[rows], Y_ref, B, "gemm fmt=%d M=%d N=%d K=%d" % (fmt, M, N, K))
-    monkeypatch.setenv("QMM_GEMM_NO_TAIL_CUT", "1")
+    qmm.debug_config("gemm_no_tail_cut", "1")
     need_whole = qmm.gemm_workspace_bytes(fmt, M, N, K)
     ws2 = torch.zeros(need_whole, dtype=torch.uint8, device="cuda")
     Y2 = qmm.gemm(fmt, packed, N, K, Xd, ws=ws2)

@@ -68,15 +68,12 @@ def test_gemv_small_shapes(qmm, oracle, fmt, N, K):
 @pytest.mark.parametrize("fmt", [Q4, Q8])
 @pytest.mark.parametrize("force", ["8,1", "8,2", "8,8", "16,1", "16,2", "16,4", "8,16"])
 @pytest.mark.parametrize("two_kernels", [False, True])
-def test_gemv_every_launch_geometry(qmm, oracle, fmt, force, two_kernels, monkeypatch):
+def test_gemv_every_launch_geometry(qmm, oracle, fmt, force, two_kernels):
     # the same product through each block size and K split; a K split over up to 8 blocks adds the
     # blocks' sums through the shared memory of a thread-block cluster, otherwise (more splits, or
     # on request) through fp32 partials in the workspace and a second kernel -- both in a fixed order
-    monkeypatch.setenv("QMM_GEMV_FORCE", force)
-    if two_kernels:
-        monkeypatch.setenv("QMM_GEMV_NO_CLUSTER", "1")
-    else:
-        monkeypatch.delenv("QMM_GEMV_NO_CLUSTER", raising=False)
+    qmm.debug_config("gemv_force", force)
+    qmm.debug_config("gemv_no_cluster", "1" if two_kernels else None)
     N, K = 512, 4096
     blocks = synth.quantize(fmt, synth.weights(91, fmt, N, K))
     x = synth.activations(91, 7, K)
@@ -118,8 +115,10 @@ def test_gemv_one_hot_returns_column_and_zero_codes_give_zero(qmm, oracle, fmt):
     assert not y.cpu().numpy().any()
 
 
-def test_gemv_is_deterministic_and_stays_in_bounds(qmm, monkeypatch):
-    monkeypatch.setenv("QMM_GEMV_FORCE", "8,4")
+@pytest.mark.parametrize("two_kernels", [False, True])
+def test_gemv_is_deterministic_and_stays_in_bounds(qmm, two_kernels):
+    qmm.debug_config("gemv_force", "8,4")
+    qmm.debug_config("gemv_no_cluster", "1" if two_kernels else None)
     N, K = 256, 2048
     blocks = synth.quantize(Q4, synth.weights(92, 0, N, K))
     packed = packed_from(qmm, Q4, blocks, N, K)
@@ -127,6 +126,7 @@ def test_gemv_is_deterministic_and_stays_in_bounds(qmm, monkeypatch):
     guard = 64
     buf = torch.full((N + 2 * guard,), 7.0, dtype=torch.float16, device="cuda")
     need = qmm.gemv_workspace_bytes(Q4, N, K)
+    assert need == (4 * N * 4 if two_kernels else 0)       # the cluster form adds its sums in shared memory
     wsbuf = torch.full((need + 512,), 0x5A, dtype=torch.uint8, device="cuda")
     y = buf[guard:guard + N]
     qmm.gemv(Q4, packed, N, K, x, y=y, ws=wsbuf[256:256 + need])
@@ -268,3 +268,32 @@ def test_cfg1_two_layers_full_size_in_one_batch(qmm, oracle, fmt):
     torch.cuda.synchronize()
     for (p, N, K, x, y), (name, (y_ref, B)) in zip(probs, refs):
         util.assert_within_tol(util.host_f64(y), y_ref, B, "cfg1 batch %s" % name)
+
+
+@pytest.mark.parametrize("fmt", [Q4, Q8])
+def test_cfg1_whole_stack_in_one_batch_as_benchmarked(qmm, oracle, fmt):
+    """The launch the benchmark times: all 112 matrices of the 16-layer stack as one qmm_gemv_batch
+    call, every output of every problem held to the GEMV tolerance against the oracle."""
+    from concurrent.futures import ThreadPoolExecutor
+    layers = synth.CFG1["layers"]
+
+    def host_layer(layer):
+        return [(name, N, K, act, synth.quantize(fmt, w)) for name, N, K, act, w in synth.cfg1_layer_weights(layer)]
+
+    with ThreadPoolExecutor(max_workers=8) as ex:
+        host = list(ex.map(host_layer, range(layers)))
+    probs, meta = [], []
+    for layer in range(layers):
+        acts = synth.cfg1_layer_acts(layer)
+        for name, N, K, act, blocks in host[layer]:
+            y = torch.full((N,), 9.0, dtype=torch.float16, device="cuda")
+            probs.append((packed_from(qmm, fmt, blocks, N, K), N, K, util.dev(acts[act]), y))
+            meta.append((layer, name, N, K, blocks, acts[act]))
+    assert len(probs) == 112
+    qmm.gemv_batch(fmt, qmm.gemv_batch_problems(probs))
+    torch.cuda.synchronize()
+    worst = 0.0
+    for (p, N, K, x, y), (layer, name, _, _, blocks, xh) in zip(probs, meta):
+        y_ref, B = oracle.gemv(fmt, blocks, N, K, xh)
+        worst = max(worst, util.assert_within_tol(util.host_f64(y), y_ref, B, "cfg1 stack, layer %d %s" % (layer, name)))
+    assert worst > 0

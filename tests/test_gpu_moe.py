@@ -30,9 +30,9 @@ def qmm():
 class Layer:
     """Expert weights of one MoE layer on host (canonical) and device (packed)."""
 
-    def __init__(self, qmm, fmt, seed, E, H, I):
+    def __init__(self, qmm, fmt, seed, E, H, I, blocks=None):
         self.fmt, self.E, self.H, self.I = fmt, E, H, I
-        self.gate, self.up, self.down = synth.moe_expert_weights(seed, fmt, E, H, I)
+        self.gate, self.up, self.down = blocks if blocks is not None else synth.moe_expert_weights(seed, fmt, E, H, I)
         self.p_gate = qmm.pack(fmt, util.dev(self.gate), E * I, H)
         self.p_up = qmm.pack(fmt, util.dev(self.up), E * I, H)
         self.p_down = qmm.pack(fmt, util.dev(self.down), E * H, I)
@@ -122,11 +122,21 @@ def check_stages(oracle, L, res, logits, X, topk, experts, rows_per_expert=None,
 
 
 def check_end_to_end(oracle, L, res, logits, X, topk, tokens):
-    """All-fp64 layer output; bound composed from the per-stage bounds (loose by design)."""
-    ref = oracle.moe_tokens(L.fmt, logits, X, L.gate, L.up, L.down, L.H, L.I, L.E, topk, np.asarray(tokens))
+    """The layer output against the all-fp64 layer (no intermediate rounding), within the bound composed
+    from the per-product tolerance of every stage (util.moe_composed_bound)."""
+    tokens = np.asarray(tokens)
+    ref = oracle.moe_tokens(L.fmt, logits, X, L.gate, L.up, L.down, L.H, L.I, L.E, topk, tokens)
+    ref2, bound = util.moe_composed_bound(oracle, L.fmt, logits, X, L.gate, L.up, L.down, L.H, L.I, L.E, topk, tokens)
+    assert np.allclose(ref, ref2, rtol=1e-10, atol=1e-12)
+    err = np.abs(res["out"][tokens].astype(np.float64) - ref)
+    worst = float(np.max(err / bound))
+    assert worst <= 1.0, "end to end: %.3f of the composed bound" % worst
+    # The composed bound is a worst case over every stage (each product's tolerance is relative to
+    # sum|w x|, ~10x the result when signs cancel); an error that large would still mean a broken
+    # layer, so the output is also held to 2 % of the token's largest component.
     scale = np.maximum(np.abs(ref).max(axis=1, keepdims=True), 1e-3)
-    err = np.abs(res["out"][np.asarray(tokens)].astype(np.float64) - ref)
     assert np.all(err <= 2e-2 * scale + 1e-4)
+    return worst
 
 
 @pytest.mark.parametrize("fmt", [Q4, Q8])
@@ -154,6 +164,24 @@ def test_moe_expert_without_tokens_and_skewed_load(qmm, oracle):
     res = run_layer(qmm, L, logits, X, topk)
     assert res["expert_offsets"][6] == res["expert_offsets"][5]
     check_stages(oracle, L, res, logits, X, topk, experts=range(E))
+
+
+@pytest.mark.parametrize("fmt", [Q4, Q8])
+@pytest.mark.parametrize("T", [3, 120])
+def test_moe_negative_and_zero_scales(qmm, oracle, fmt, T):
+    """Expert weights with arbitrary codes and one block in 16 carrying a negative, zero or -0 scale,
+    through the decode-sized path (T = 3: GEMVs) and the grouped tensor-core products (T = 120), at the
+    stage-wise tolerances."""
+    E, topk, H, I = 8, 2, 256, 512
+    mk = lambda seed, rows, cols: util.random_blocks(synth, fmt, rows, cols, seed=seed, special_scales="no_subnormal",
+                                                     scale_bits=(0x1000, 0x2400))[0]      # 2^-11 .. 2^-6
+    L = Layer(qmm, fmt, 0, E, H, I, blocks=(mk(640 + fmt, E * I, H), mk(641 + fmt, E * I, H), mk(642 + fmt, E * H, I)))
+    X = synth.activations(643, T, T, H)
+    logits = synth.logits(644, T, T, E)
+    res = run_layer(qmm, L, logits, X, topk)
+    assert np.all(np.isfinite(res["out"].astype(np.float64)))
+    check_stages(oracle, L, res, logits, X, topk, experts=range(E))
+    check_end_to_end(oracle, L, res, logits, X, topk, tokens=range(min(T, 4)))
 
 
 def test_moe_route_only_and_determinism(qmm, oracle):

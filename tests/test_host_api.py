@@ -71,8 +71,14 @@ def test_null_and_misaligned_pointers(L):
     assert L.qmm_status_check(None, None) == 1
 
 
-def test_gemv_workspace_rule(L, monkeypatch):
-    monkeypatch.setenv("QMM_GEMV_FORCE", "8,4")
+def test_gemv_workspace_rule(L):
+    assert qmm.gemv_workspace_bytes(4, 512, 2048) == 0            # the plan's K split fits a cluster: no workspace
+    qmm.debug_config("gemv_force", "8,4")
+    assert qmm.gemv_workspace_bytes(4, 512, 2048) == 0            # forced 4-way split: still a cluster
+    qmm.debug_config("gemv_force", "8,16")
+    assert qmm.gemv_workspace_bytes(4, 512, 8192) == 16 * 512 * 4  # beyond a cluster: partial sums in the workspace
+    qmm.debug_config("gemv_force", "8,4")
+    qmm.debug_config("gemv_no_cluster", "1")
     need = qmm.gemv_workspace_bytes(4, 512, 2048)
     assert need == 4 * 512 * 4
     buf = (ctypes.c_char * 512)()
@@ -80,14 +86,32 @@ def test_gemv_workspace_rule(L, monkeypatch):
     assert L.qmm_gemv(4, a, 512, 2048, a, a, None, 0, None) == 4
     assert L.qmm_gemv(4, a, 512, 2048, a, a, a, need - 1, None) == 4
     assert "workspace" in qmm.last_error()
-    monkeypatch.setenv("QMM_GEMV_FORCE", "8,1")
+    qmm.debug_config("gemv_force", "8,1")
     assert qmm.gemv_workspace_bytes(4, 512, 2048) == 0
 
 
-def test_gemm_workspace_rule(L, monkeypatch):
+def test_debug_config_rejects_what_it_does_not_know(L):
+    assert L.qmm_debug_config(b"no_such_knob", b"1") == 1
+    assert "unknown knob" in qmm.last_error()
+    assert L.qmm_debug_config(b"gemv_force", b"12,1") == 1
+    assert L.qmm_debug_config(b"gemm_force", b"100") == 1
+    assert L.qmm_debug_config(b"gemm_force", b"128,0") == 1
+    assert L.qmm_debug_config(b"gemm_force", b"128,5") == 0
+    assert L.qmm_debug_config(None, None) == 0
+    buf = (ctypes.c_char * 512)()
+    a = (ctypes.addressof(buf) + 255) & ~255
+    assert L.qmm_debug_wait_give_up(None, 1000, None) == 1
+    assert L.qmm_debug_wait_give_up(a, 0, None) == 1
+    assert L.qmm_debug_wait_give_up(a, 1 << 30, None) == 1
+    assert L.qmm_packed_check(4, None, 128, 256, a, None) == 1
+    assert L.qmm_packed_check(4, a, 128, 100, a, None) == 2
+    assert L.qmm_packed_check(4, a + 16, 128, 256, a, None) == 3
+
+
+def test_gemm_workspace_rule(L):
     """The workspace is a fixed header, plus fp32 partial-sum slots exactly when the plan cuts tiles
     along K (few output tiles); the plan is a pure function of the shape."""
-    monkeypatch.delenv("QMM_GEMM_FORCE", raising=False)
+    qmm.debug_config(None)
     header = qmm.gemm_workspace_bytes(4, 2048, 8192, 3072)        # 512 whole tiles: nothing to add up
     assert header == 8192
     assert qmm.gemm_workspace_bytes(8, 2048, 8192, 3072) == header
@@ -100,7 +124,7 @@ def test_gemm_workspace_rule(L, monkeypatch):
     assert qmm.gemm_workspace_bytes(4, 2048, 3072, 8192) == header + 2 * 148 * 256 * 128 * 4
     tiny = qmm.gemm_workspace_bytes(4, 1, 128, 256)                    # one tile, 4 k-blocks: too short to cut
     assert tiny == header
-    monkeypatch.setenv("QMM_GEMM_FORCE", "128,1,5")
+    qmm.debug_config("gemm_force", "128,5")
     forced = qmm.gemm_workspace_bytes(4, 100, 256, 2048)               # 2 tiles x 32 k-blocks in shares of 5: 13 blocks
     assert forced == header + 2 * 13 * 128 * 128 * 4
     buf = (ctypes.c_char * 512)()

@@ -433,3 +433,45 @@ def test_property_routing_and_permutation(oracle, T, E, seed):
     keys = [(int(flat[i]), int(i)) for i in perm]
     assert keys == sorted(keys)
     assert offs.tolist() == [int((flat < e).sum()) for e in range(E + 1)]
+
+
+def test_composed_moe_bound_reproduces_the_layer_and_scales_with_the_tolerance(oracle):
+    """The helper that composes the end-to-end bound of a mixture-of-experts layer from the per-product
+    tolerances recomputes the layer stage by stage: its reference must be the oracle's all-fp64 layer, and
+    its bound must be positive, dominated by the propagated gate/up term, and small against the output."""
+    from tests import util
+    fmt, T, E, topk, H, I = 4, 5, 8, 2, 256, 256
+    gate, up, down = synth.moe_expert_weights(901, fmt, E, H, I)
+    X = synth.activations(901, 1, T, H)
+    lg = synth.logits(901, 2, T, E)
+    tokens = np.arange(T)
+    ref = oracle.moe_tokens(fmt, lg, X, gate, up, down, H, I, E, topk, tokens)
+    ref2, bound = util.moe_composed_bound(oracle, fmt, lg, X, gate, up, down, H, I, E, topk, tokens)
+    assert np.allclose(ref, ref2, rtol=1e-12, atol=1e-15)
+    assert np.all(bound > 1e-5)
+    # never tighter than the combine's own tolerance, and not vacuous
+    assert np.all(bound >= 2e-3 * np.abs(ref) + 1e-5)
+    assert np.median(bound) < np.abs(ref).max()
+    # token 0 once more with the independent numpy decoder and plain matrix products
+    from tests import npref
+    idx, p = oracle.route(lg, topk)
+    x = X[0].astype(np.float64)
+    tol = lambda B: 2e-3 * B + 1e-5
+    want = np.zeros(H)
+    gu, dn = len(gate) // E, len(down) // E
+    mag = np.zeros(H)
+    for j in range(topk):
+        e = int(idx[0, j])
+        Wg, Wu = npref.decode(fmt, gate[e * gu:(e + 1) * gu], I, H), npref.decode(fmt, up[e * gu:(e + 1) * gu], I, H)
+        Wd = npref.decode(fmt, down[e * dn:(e + 1) * dn], H, I)
+        G, U = Wg @ x, Wu @ x
+        BG, BU = np.abs(Wg) @ np.abs(x), np.abs(Wu) @ np.abs(x)
+        sG = G / (1 + np.exp(-G))
+        h = sG * U
+        E_h = 1.1 * tol(BG) * np.abs(U) + np.abs(sG) * tol(BU) + 1.1 * tol(BG) * tol(BU) + 2.0**-11 * np.abs(h)
+        E_D = 2e-3 * (np.abs(Wd) @ np.abs(h)) + 1.002 * (np.abs(Wd) @ E_h) + 1e-5
+        D = Wd @ h
+        want += p[0, j] * E_D + 2e-3 * p[0, j] * (np.abs(D) + E_D)
+        mag += np.abs(D) + E_D
+    want += 1e-5 + 1e-6 * mag
+    assert np.allclose(bound[0], want, rtol=1e-9, atol=0)
