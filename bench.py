@@ -36,10 +36,13 @@ from paper_2607_00501_b200 import synth  # noqa: E402
 METRIC = "decode GEMV effective HBM bandwidth on quantised-weight bytes (Q4+Q8 16-layer stack)"
 UNIT = "GB/s"
 NOMINAL_BF16_TFLOPS = 2250.0
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of gemv_batch_kernel on this workload, from the
-# ncu captures summarised in profiles/gemv_batch_kernel_q{4,8}_cfg1_stack.md (algorithmic bytes: 547 356 672 /
-# 1 033 895 936).  Only reported, never used in a computation.
+NOMINAL_HBM_GBS = 8000.0
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of gemv_batch_kernel on this workload: a RECORDED
+# figure from one ncu capture per format of `bench.py --case gemv_batch_q4|q8` (algorithmic bytes:
+# 547 356 672 / 1 033 895 936).  It is reported beside the live timings, never used in a computation, and
+# does not change when the kernel does -- re-capture after changing gemv_batch_kernel.
 NCU_DRAM_TRAFFIC = {synth.Q4: 552_050_000, synth.Q8: 1_038_200_000}
+NCU_DRAM_TRAFFIC_SOURCE = "recorded from an ncu capture of --case gemv_batch_q4 / gemv_batch_q8; not measured in this run"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 # fused launches per layer: (name, constituent matrices, N, K, activation)
@@ -60,53 +63,68 @@ def peaks():
 # --------------------------------------------------------------------------
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
-    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+    """Samples nvidia-smi clocks and throttle reasons while a timed region runs (read-only queries).
+    Every sample carries nvidia-smi's own timestamp, so that one sampler can serve several regions:
+    stop() summarises all samples, window(t0, t1) those taken between two time.time() values."""
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    REASONS = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
 
-    def __init__(self, gpu_index: int):
+    def __init__(self, gpu_index: int, interval_ms: int = 100):
         self.gpu = gpu_index
+        self.interval_ms = interval_ms
         self.proc = None
         self.path = None
+        self.rows = []                  # (unix time, sm MHz, max sm MHz, power W, active reasons)
 
     def start(self):
         try:
             f = tempfile.NamedTemporaryFile("w", suffix=".csv", delete=False)
             self.path = f.name
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.Q,
-                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=f, stderr=subprocess.DEVNULL)
+                                          "--format=csv,noheader,nounits", "-lms", str(self.interval_ms)],
+                                         stdout=f, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
-    def stop(self):
+    @staticmethod
+    def summarise(rows):
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if rows:
+            reasons = sorted({r for row in rows for r in row[4]})
+            out.update(sm_mhz=float(np.median([r[1] for r in rows])), sm_max_mhz=rows[-1][2], reasons=reasons,
+                       samples=len(rows), power_w_max=max(r[3] for r in rows))
+        return out
+
+    def stop(self):
         if self.proc is None:
-            return out
+            return self.summarise([])
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, reasons, smax = [], set(), None
+        import datetime
         try:
             for line in open(self.path):
                 f = [x.strip() for x in line.split(",")]
                 if len(f) < 9:
                     continue
                 try:
-                    sm.append(float(f[1]))
-                    smax = float(f[2])
+                    ts = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                    row = (ts, float(f[1]), float(f[2]), float(f[3]),
+                           [n for n, v in zip(self.REASONS, f[5:9]) if v.lower().startswith("active")])
                 except ValueError:
                     continue
-                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
-                    if v.lower().startswith("active"):
-                        reasons.add(name)
+                self.rows.append(row)
             os.unlink(self.path)
         except Exception:
             pass
-        if sm:
-            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=smax, reasons=sorted(reasons), samples=len(sm))
-        return out
+        return self.summarise(self.rows)
+
+    def window(self, t0: float, t1: float):
+        """Summary of the samples taken between two time.time() values (call after stop())."""
+        return self.summarise([r for r in self.rows if t0 <= r[0] <= t1])
 
 
 # --------------------------------------------------------------------------
@@ -397,7 +415,7 @@ def run_ours(args):
     sections = {}
     cpu = None
     if rank == 0 and not args.no_sections:
-        sections = extra_sections(args, qmm, torch, pk, ops, fmts)
+        sections = extra_sections(args, qmm, torch, pk, ops, fmts, gpu_index=local)
     if rank == 0 and world == 1 and not args.no_cpu:
         cpu = cpu_baseline(host_blocks, host_acts, fmts, budget_s=args.cpu_seconds)
 
@@ -423,6 +441,8 @@ def run_ours(args):
         "roofline": {"bound": "hbm", "achieved": round(value / world, 1), "peak": pk["hbm_gbs"], "unit": "GB/s",
                      "frac": round(value / world / pk["hbm_gbs"], 4),
                      "traffic": sum(NCU_DRAM_TRAFFIC[f] for f in fmts) if args.mode == "batch" else None,
+                     "traffic_source": NCU_DRAM_TRAFFIC_SOURCE if args.mode == "batch" else None,
+                     "frac_of_nominal_8000": round(value / world / NOMINAL_HBM_GBS, 4),
                      "algorithmic_bytes": bytes_step, "per_kernel": per_kernel,
                      "kernel": "gemv_batch_kernel (both launches of the step)" if args.mode == "batch" else "gemv_kernel (all launches of the step)", "peak_source": pk["source"],
                      "step_ms_min": round(min(step_ms), 5), "step_ms_max": round(max(step_ms), 5)},
@@ -447,11 +467,57 @@ def time_op(torch, fn, iters, flush=None):
     return float(np.median(times)), float(min(times))
 
 
-def extra_sections(args, qmm, torch, pk, ops, fmts):
-    """The rest of the path on its own workloads (each L2-flushed between runs)."""
+def measure(torch, fn, flush, iters=10, sustain_s=0.12):
+    """One workload: cold (L2 flushed before every run: median and best of `iters`), then back to back
+    without flushing for ~sustain_s (the L2-warm, sustained figure; the clock sampler's samples of this
+    window are attached by attach_clocks)."""
+    fn()
+    med, best = time_op(torch, fn, iters, flush)
+    n = max(10, int(sustain_s * 1e3 / max(med, 1e-3)))
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    t0 = time.time()
+    e0.record()
+    for _ in range(n):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    t1 = time.time()
+    return {"ms": round(med, 4), "ms_best": round(best, 4), "ms_warm": round(e0.elapsed_time(e1) / n, 4), "_win": (t0, t1)}
+
+
+def attach_clocks(node, sampler):
+    """Replace every "_win" left by measure() with the SM clock seen in that window."""
+    if isinstance(node, dict):
+        if "_win" in node:
+            w = sampler.window(*node.pop("_win"))
+            node["sm_mhz_warm_run"] = w["sm_mhz"]
+            if w["reasons"]:
+                node["clock_reasons"] = w["reasons"]
+        for v in node.values():
+            attach_clocks(v, sampler)
+
+
+def tensor_fracs(tf, pk):
+    """TFLOP/s against the three tensor denominators: measured burst, measured sustained, nominal."""
+    return {"TFLOPs": round(tf, 1), "frac_tensor_measured": round(tf / pk["bf16_tflops"], 4),
+            "frac_tensor_sustained": round(tf / pk["bf16_tflops_sustained"], 4),
+            "frac_tensor_nominal": round(tf / NOMINAL_BF16_TFLOPS, 4)}
+
+
+def hbm_fracs(nbytes, ms, pk):
+    gbs = nbytes / ms / 1e6
+    return {"GBps": round(gbs, 1), "frac_hbm": round(gbs / pk["hbm_gbs"], 4), "frac_hbm_nominal": round(gbs / NOMINAL_HBM_GBS, 4)}
+
+
+def extra_sections(args, qmm, torch, pk, ops, fmts, gpu_index=0):
+    """The rest of the path on its own workloads.  Every entry: `ms` = median device time with L2 flushed
+    before each run, `ms_warm` = back to back without flushing (with the SM clock seen during that run)."""
     out = {}
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
     dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    sampler = ClockSampler(gpu_index, interval_ms=20)
+    sampler.start()
 
     # per-format decode stacks, one qmm_gemv launch per fused matrix, chained on one stream with
     # programmatic dependent launch (a dependency between consecutive launches, as in a real decoder)
@@ -467,9 +533,45 @@ def extra_sections(args, qmm, torch, pk, ops, fmts):
                     qmm.gemv(f, w, N, K, x, y=y, ws=ws)
             med, best = time_op(torch, g.replay, 10)
         b = stack_bytes(f)
-        out["decode_stack_q%d_chained" % f] = {"ms": round(med, 4), "GBps": round(b / med / 1e6, 1),
-                                                "frac_hbm": round(b / med / 1e6 / pk["hbm_gbs"], 4),
-                                                "launches": len(ops[f])}
+        out["decode_stack_q%d_chained" % f] = dict({"ms": round(med, 4), "launches": len(ops[f])}, **hbm_fracs(b, med, pk))
+
+    # cfg0: one small Q4 GEMV (1.77 MB of weights: 0.27 us of HBM traffic, far below a launch).  Steady
+    # state = 300 distinct packed copies (531 MB, larger than L2) so that every product streams from HBM:
+    # as 300 chained launches in one graph, and as qmm_gemv_batch launches over the same 300 problems.
+    c = synth.CFG0
+    copies = 300
+    blocks = synth.quantize(c["fmt"], synth.weights(c["seed"], 0, c["N"], c["K"]))
+    one = qmm.pack(c["fmt"], dev(blocks), c["N"], c["K"])
+    many = one.repeat(copies).reshape(copies, -1)
+    x0 = dev(synth.activations(c["seed"], 1, c["K"]))
+    y0 = torch.empty((copies, c["N"]), dtype=torch.float16, device="cuda")
+    nb = blocks.nbytes
+
+    def graph_of(fn_i):
+        g, st = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+        with torch.cuda.stream(st):
+            fn_i(0)
+            torch.cuda.synchronize()
+            with torch.cuda.graph(g, stream=st):
+                for i in range(copies):
+                    fn_i(i)
+        return g
+
+    g_cold = graph_of(lambda i: qmm.gemv(c["fmt"], many[i], c["N"], c["K"], x0, y=y0[i]))
+    g_warm = graph_of(lambda i: qmm.gemv(c["fmt"], many[0], c["N"], c["K"], x0, y=y0[i]))
+    arr = qmm.gemv_batch_problems([(many[i], c["N"], c["K"], x0, y0[i]) for i in range(copies)])
+    cfg0 = {"bytes_per_gemv": nb, "copies": copies}
+    med, _ = time_op(torch, g_cold.replay, 10)
+    cfg0["chained_launches_hbm_cold"] = dict({"us_per_gemv": round(med * 1e3 / copies, 3)}, **hbm_fracs(nb * copies, med, pk))
+    med, _ = time_op(torch, g_warm.replay, 10)
+    cfg0["chained_launches_l2_warm"] = {"us_per_gemv": round(med * 1e3 / copies, 3), "GBps_from_l2": round(nb * copies / med / 1e6, 1)}
+    med, _ = time_op(torch, lambda: qmm.gemv_batch(c["fmt"], arr), 10)
+    cfg0["batched_hbm_cold"] = dict({"us_per_gemv": round(med * 1e3 / copies, 3), "launches": (copies + 127) // 128},
+                                    **hbm_fracs(nb * copies, med, pk))
+    med, best = time_op(torch, lambda: qmm.gemv(c["fmt"], many[7], c["N"], c["K"], x0, y=y0[7]), 20, flush)
+    cfg0["isolated_launch_cold"] = dict({"us": round(med * 1e3, 3), "us_best": round(best * 1e3, 3)}, **hbm_fracs(nb, med, pk))
+    out["cfg0_q4_gemv"] = cfg0
+    del many, y0, g_cold, g_warm, arr
 
     # cfg2: Q8 LM head GEMV
     c = synth.CFG2
@@ -477,9 +579,8 @@ def extra_sections(args, qmm, torch, pk, ops, fmts):
     packed = qmm.pack(c["fmt"], dev(blocks), c["N"], c["K"])
     x = dev(synth.activations(c["seed"], 1, c["K"]))
     y = torch.empty(c["N"], dtype=torch.float16, device="cuda")
-    med, best = time_op(torch, lambda: qmm.gemv(c["fmt"], packed, c["N"], c["K"], x, y=y), 20, flush)
-    out["lm_head_q8_gemv"] = {"ms": round(med, 4), "GBps": round(blocks.nbytes / med / 1e6, 1),
-                              "frac_hbm": round(blocks.nbytes / med / 1e6 / pk["hbm_gbs"], 4)}
+    m = measure(torch, lambda: qmm.gemv(c["fmt"], packed, c["N"], c["K"], x, y=y), flush, iters=20)
+    out["lm_head_q8_gemv"] = dict(m, **hbm_fracs(blocks.nbytes, m["ms"], pk))
     del packed, blocks
 
     # one cfg1 layer's feed-forward front half as a single launch: h = silu(Wgate x) * (Wup x)
@@ -494,13 +595,12 @@ def extra_sections(args, qmm, torch, pk, ops, fmts):
         fn()
         med, best = time_op(torch, fn, 10, flush)
         b = 2 * synth.canonical_bytes(f, N, K)
-        out["ffn_gate_up_silu_q%d_gemv" % f] = {"ms": round(med, 4), "GBps": round(b / med / 1e6, 1),
-                                                 "frac_hbm": round(b / med / 1e6 / pk["hbm_gbs"], 4)}
+        out["ffn_gate_up_silu_q%d_gemv" % f] = dict({"ms": round(med, 4)}, **hbm_fracs(b, med, pk))
 
-    # cfg3: prefill GEMM sweep (Q4 as the config says; Q8 = the same kernels with the byte expander,
-    # measured at the two largest M)
+    # cfg3: prefill GEMM sweep (Q4 as the config says, plus the small-batch sizes below one token tile;
+    # Q8 = the same kernels with the byte expander, measured at the two largest M)
     c = synth.CFG3
-    for f, Ms in ((c["fmt"], c["Ms"]), (synth.Q8, c["Ms"][-2:])):
+    for f, Ms in ((c["fmt"], (16, 32, 64) + tuple(c["Ms"])), (synth.Q8, c["Ms"][-2:])):
         gemm = {}
         for name, N, K in c["shapes"]:
             blocks = synth.quantize(f, synth.weights(c["seed"], 0 if name == "gate_up" else 1, N, K))
@@ -509,18 +609,30 @@ def extra_sections(args, qmm, torch, pk, ops, fmts):
                 X = dev(synth.activations(c["seed"], 10 + M, M, K))
                 Y = torch.empty((M, N), dtype=torch.float16, device="cuda")
                 ws = torch.zeros(qmm.gemm_workspace_bytes(f, M, N, K), dtype=torch.uint8, device="cuda")
-                fn = lambda: qmm.gemm(f, packed, N, K, X, Y=Y, ws=ws)
-                fn()
-                med, best = time_op(torch, fn, 10, flush)
-                tf = 2.0 * M * N * K / med / 1e9
-                gemm["%s_M%d" % (name, M)] = {"ms": round(med, 4), "TFLOPs": round(tf, 1),
-                                              "frac_tensor_measured": round(tf / pk["bf16_tflops"], 4),
-                                              "frac_tensor_nominal": round(tf / NOMINAL_BF16_TFLOPS, 4)}
+                m = measure(torch, lambda: qmm.gemm(f, packed, N, K, X, Y=Y, ws=ws), flush)
+                tf = 2.0 * M * N * K / m["ms"] / 1e9
+                floor_ms = max(2.0 * M * N * K / pk["bf16_tflops"] / 1e9, (blocks.nbytes + 2 * M * (N + K)) / pk["hbm_gbs"] / 1e6)
+                gemm["%s_M%d" % (name, M)] = dict(m, roofline_floor_ms=round(floor_ms, 4), frac_of_floor=round(floor_ms / m["ms"], 4),
+                                                  **tensor_fracs(tf, pk))
                 qmm.status_check(ws)
         out["prefill_gemm_q%d" % f] = gemm
 
     # cfg4: MoE layer (Q4 as the config says; Q8 at the largest T)
     c = synth.CFG4
+
+    def moe_entry(f, T, lg, pg, pu, pd, wbytes):
+        X = dev(synth.activations(c["seed"], 100 + T, T, c["H"]))
+        o = torch.empty((T, c["H"]), dtype=torch.float16, device="cuda")
+        a = qmm.moe_args(f, T, c["H"], c["I"], c["E"], c["topk"], dev(lg), X, pg, pu, pd, o)
+        ws = torch.zeros(qmm.moe_workspace_bytes(a), dtype=torch.uint8, device="cuda")
+        m = measure(torch, lambda: qmm.moe(a, ws), flush)
+        qmm.status_check(ws)
+        fl = T * c["topk"] * 3 * 2.0 * c["H"] * c["I"]
+        touched = min(1.0, T * c["topk"] / c["E"]) * wbytes + 4 * T * c["H"] + 4 * T * c["E"]
+        floor_ms = max(fl / pk["bf16_tflops"] / 1e9, touched / pk["hbm_gbs"] / 1e6)
+        return dict(m, hbm_floor_ms=round(touched / pk["hbm_gbs"] / 1e6, 4), roofline_floor_ms=round(floor_ms, 4),
+                    frac_of_floor=round(floor_ms / m["ms"], 4), **tensor_fracs(fl / m["ms"] / 1e9, pk))
+
     for f, Ts in ((c["fmt"], c["Ts"]), (synth.Q8, c["Ts"][-1:])):
         gate, up, down = synth.moe_expert_weights(c["seed"], f, c["E"], c["H"], c["I"])
         pg = qmm.pack(f, dev(gate), c["E"] * c["I"], c["H"])
@@ -529,40 +641,17 @@ def extra_sections(args, qmm, torch, pk, ops, fmts):
         wbytes = gate.nbytes + up.nbytes + down.nbytes
         moe = {}
         for T in Ts:
-            X = dev(synth.activations(c["seed"], 100 + T, T, c["H"]))
-            lg = dev(synth.logits(c["seed"], 200 + T, T, c["E"]))
-            o = torch.empty((T, c["H"]), dtype=torch.float16, device="cuda")
-            a = qmm.moe_args(f, T, c["H"], c["I"], c["E"], c["topk"], lg, X, pg, pu, pd, o)
-            ws = torch.zeros(qmm.moe_workspace_bytes(a), dtype=torch.uint8, device="cuda")
-            fn = lambda: qmm.moe(a, ws)
-            fn()
-            med, best = time_op(torch, fn, 10, flush)
-            qmm.status_check(ws)
-            fl = T * c["topk"] * 3 * 2.0 * c["H"] * c["I"]
-            touched = min(c["E"], T * c["topk"]) / c["E"] * wbytes if T * c["topk"] < c["E"] else wbytes
-            moe["T%d" % T] = {"ms": round(med, 4), "TFLOPs": round(fl / med / 1e9, 2),
-                              "frac_tensor_nominal": round(fl / med / 1e9 / NOMINAL_BF16_TFLOPS, 4),
-                              "hbm_floor_ms": round(touched / pk["hbm_gbs"] / 1e6, 4),
-                              "frac_of_hbm_floor": round(touched / pk["hbm_gbs"] / 1e6 / med, 4)}
+            moe["T%d" % T] = moe_entry(f, T, synth.logits(c["seed"], 200 + T, T, c["E"]), pg, pu, pd, wbytes)
         if f == c["fmt"]:
             # not a config: the same layer under an uneven expert load (a fixed N(0, 1.5^2) bias per
             # expert on the seeded logits; trained routers are skewed, the config's iid logits are not)
             T = c["Ts"][-1]
             bias = np.random.default_rng([c["seed"], 999]).standard_normal(c["E"]).astype(np.float32) * 1.5
-            X = dev(synth.activations(c["seed"], 100 + T, T, c["H"]))
-            lg = dev(synth.logits(c["seed"], 200 + T, T, c["E"]) + bias[None, :])
-            o = torch.empty((T, c["H"]), dtype=torch.float16, device="cuda")
-            a = qmm.moe_args(f, T, c["H"], c["I"], c["E"], c["topk"], lg, X, pg, pu, pd, o)
-            ws = torch.zeros(qmm.moe_workspace_bytes(a), dtype=torch.uint8, device="cuda")
-            fn = lambda: qmm.moe(a, ws)
-            fn()
-            med, best = time_op(torch, fn, 10, flush)
-            qmm.status_check(ws)
-            fl = T * c["topk"] * 3 * 2.0 * c["H"] * c["I"]
-            moe["T%d_skewed_load" % T] = {"ms": round(med, 4), "TFLOPs": round(fl / med / 1e9, 2),
-                                          "frac_tensor_nominal": round(fl / med / 1e9 / NOMINAL_BF16_TFLOPS, 4)}
+            moe["T%d_skewed_load" % T] = moe_entry(f, T, synth.logits(c["seed"], 200 + T, T, c["E"]) + bias[None, :], pg, pu, pd, wbytes)
         out["moe_q%d" % f] = moe
         del pg, pu, pd, gate, up, down
+    sampler.stop()
+    attach_clocks(out, sampler)
     return out
 
 
@@ -598,15 +687,17 @@ def run_reference(args):
         return
     import oracle
     fmts = synth.CFG1["fmts"]
-    sample_layers = 1
-    host_blocks, host_acts = build_stack_host(sample_layers, fmts)
+    layers = synth.CFG1["layers"]
+    host_blocks, host_acts = build_stack_host(layers, fmts)
     shapes = {n: (N, K, a) for n, N, K, a in synth.CFG1_LAYER}
-    nbytes = sum(host_blocks[f][0][n].nbytes for f in fmts for n in shapes)
+    nbytes = sum(host_blocks[f][l][n].nbytes for f in fmts for l in range(layers) for n in shapes)
+    assert nbytes == sum(stack_bytes(f) for f in fmts)
 
     def step():
-        for f in fmts:
-            for name, (N, K, act) in shapes.items():
-                oracle.gemv(f, host_blocks[f][0][name], N, K, host_acts[0][act])
+        for l in range(layers):
+            for f in fmts:
+                for name, (N, K, act) in shapes.items():
+                    oracle.gemv(f, host_blocks[f][l][name], N, K, host_acts[l][act])
 
     for _ in range(max(args.warmup, 1)):
         step()
@@ -615,13 +706,14 @@ def run_reference(args):
         step()
     dt = time.time() - t0
     value = nbytes * args.steps / dt / 1e9
-    sample = "layer 0 of 16 of the Q4+Q8 decode stack per step (all 14 GEMVs), host cores"
+    sample = "the whole Q4+Q8 decode stack per step (all 16 layers, 224 GEMVs), host cores"
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": round(value, 3), "unit": UNIT,
         "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": max(args.warmup, 1),
         "ms_per_step": round(dt / args.steps * 1e3, 3), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64 accumulate (CPU oracle)", "data": "synthetic",
-        "config": {"workload": "cfg1: Q4+Q8 decode linear stack, 16 layers, M=1", "sample": sample},
+        "config": {"workload": "cfg1: Q4+Q8 decode linear stack, 16 layers x 7 matrices, M=1", "sample": sample,
+                   "bytes_per_step": nbytes},
         "cpu_baseline": {"value": round(value, 3), "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": round(value, 3), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
@@ -629,7 +721,10 @@ def run_reference(args):
 
 def run_case(args):
     """`--case NAME`: a few launches of one kernel on its benchmark workload and nothing else, so that a
-    profiler can be pointed at it (`ncu -k regex:... python bench.py --case gemm_q4_M2048`).  Prints no JSON."""
+    profiler can be pointed at it.  Prints no JSON.  Under ncu the flag `--clock-control none` is
+    mandatory (without it ncu locks the GPU's clocks, and a killed ncu leaves them locked for the next
+    user of a shared GPU); capture one kernel and a few launches:
+    `ncu --clock-control none -k regex:gemm_kernel -s 2 -c 2 python bench.py --case gemm_q4_M2048`."""
     import torch
     from paper_2607_00501_b200 import qmm
     torch.cuda.set_device(0)
@@ -647,40 +742,97 @@ def run_case(args):
         arr = qmm.gemv_batch_problems(probs)
         for _ in range(reps):
             qmm.gemv_batch(f, arr)
-    elif name.startswith("gemm_q4_M"):
+    elif name == "gemv_lm_head_q8":
+        c = synth.CFG2
+        packed = qmm.pack(c["fmt"], dev(synth.quantize(c["fmt"], synth.weights(c["seed"], 0, c["N"], c["K"]))), c["N"], c["K"])
+        x = dev(synth.activations(c["seed"], 1, c["K"]))
+        y = torch.empty(c["N"], dtype=torch.float16, device="cuda")
+        for _ in range(reps):
+            qmm.gemv(c["fmt"], packed, c["N"], c["K"], x, y=y)
+    elif name in ("gemv_kv_q4", "gemv_kv_q8"):
+        # the k / v projection of the decode stack: 512 rows do not fill the SMs, so K is split over a
+        # thread-block cluster.  64 distinct copies (37-70 MB) so that a few launches are not all L2 hits.
+        f = synth.Q4 if name.endswith("q4") else synth.Q8
+        N, K = 512, 2048
+        one = qmm.pack(f, dev(synth.quantize(f, synth.weights(1, 1, N, K))), N, K)
+        many = one.repeat(64).reshape(64, -1)
+        x = dev(synth.activations(1, 1000, K))
+        y = torch.empty(N, dtype=torch.float16, device="cuda")
+        for i in range(8):
+            qmm.gemv(f, many[i * 8], N, K, x, y=y)
+    elif name.startswith("gemm_q") and "_M" in name:
+        # gemm_q4_M2048 (gate/up shape), gemm_q8_M1024, gemm_q4_down_M512 ...
         c = synth.CFG3
+        f = synth.Q4 if name.startswith("gemm_q4") else synth.Q8
         M = int(name.split("_M")[1])
-        _, N, K = c["shapes"][0]
-        packed = qmm.pack(c["fmt"], dev(synth.quantize(c["fmt"], synth.weights(c["seed"], 0, N, K))), N, K)
+        which = 1 if "_down_" in name else 0
+        _, N, K = c["shapes"][which]
+        packed = qmm.pack(f, dev(synth.quantize(f, synth.weights(c["seed"], which, N, K))), N, K)
         X = dev(synth.activations(c["seed"], 10 + M, M, K))
         Y = torch.empty((M, N), dtype=torch.float16, device="cuda")
-        ws = torch.zeros(qmm.gemm_workspace_bytes(c["fmt"], M, N, K), dtype=torch.uint8, device="cuda")
+        ws = torch.zeros(qmm.gemm_workspace_bytes(f, M, N, K), dtype=torch.uint8, device="cuda")
         for _ in range(reps):
-            qmm.gemm(c["fmt"], packed, N, K, X, Y=Y, ws=ws)
+            qmm.gemm(f, packed, N, K, X, Y=Y, ws=ws)
         qmm.status_check(ws)
-    elif name.startswith("moe_q4_T"):
+    elif name.startswith("moe_q") and "_T" in name:
         c = synth.CFG4
+        f = synth.Q4 if name.startswith("moe_q4") else synth.Q8
         T = int(name.split("_T")[1])
-        gate, up, down = synth.moe_expert_weights(c["seed"], c["fmt"], c["E"], c["H"], c["I"])
-        pg, pu = qmm.pack(c["fmt"], dev(gate), c["E"] * c["I"], c["H"]), qmm.pack(c["fmt"], dev(up), c["E"] * c["I"], c["H"])
-        pd = qmm.pack(c["fmt"], dev(down), c["E"] * c["H"], c["I"])
+        gate, up, down = synth.moe_expert_weights(c["seed"], f, c["E"], c["H"], c["I"])
+        pg, pu = qmm.pack(f, dev(gate), c["E"] * c["I"], c["H"]), qmm.pack(f, dev(up), c["E"] * c["I"], c["H"])
+        pd = qmm.pack(f, dev(down), c["E"] * c["H"], c["I"])
         X = dev(synth.activations(c["seed"], 100 + T, T, c["H"]))
         lg = dev(synth.logits(c["seed"], 200 + T, T, c["E"]))
         o = torch.empty((T, c["H"]), dtype=torch.float16, device="cuda")
-        a = qmm.moe_args(c["fmt"], T, c["H"], c["I"], c["E"], c["topk"], lg, X, pg, pu, pd, o)
+        a = qmm.moe_args(f, T, c["H"], c["I"], c["E"], c["topk"], lg, X, pg, pu, pd, o)
         ws = torch.zeros(qmm.moe_workspace_bytes(a), dtype=torch.uint8, device="cuda")
         for _ in range(reps):
             qmm.moe(a, ws)
         qmm.status_check(ws)
     else:
-        raise SystemExit("unknown --case %r (gemv_batch_q4, gemv_batch_q8, gemm_q4_M<M>, moe_q4_T<T>)" % name)
+        raise SystemExit("unknown --case %r (gemv_batch_q4|q8, gemv_lm_head_q8, gemv_kv_q4|q8, gemm_q4|q8[_down]_M<M>, "
+                         "moe_q4|q8_T<T>)" % name)
     torch.cuda.synchronize()
     print("case %s: %d launches done" % (name, reps), file=sys.stderr)
+
+
+def launch_ranks(n: int, argv) -> int:
+    """`--gpus N` without a launcher: start N ranks of this script under torch.distributed.run on this
+    node (one process per GPU, rendezvous on 127.0.0.1), exactly as an external launcher would."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(n),
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+    return subprocess.call(cmd)
+
+
+def run_dry(args):
+    """`--dry-run-cpu`: the multi-rank plumbing of the benchmark with no GPU and no kernels (gloo): every
+    rank draws its own activations, pretends its step took (1 + rank) ms, the ranks agree on the maximum
+    and rank 0 prints the whole-job line.  Exists so that the launcher and the N > 1 bookkeeping can be
+    tested where there is no GPU; the line says "dry_run": true and carries no measurement."""
+    import torch.distributed as dist
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        dist.init_process_group("gloo")
+    acts = rank_activations(rank, [synth.cfg1_layer_acts(0)])
+    ms, = max_over_ranks(dist if world > 1 else None, [1.0 + rank], "cpu")
+    value = whole_job_value(world, 1000, ms)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps({"dry_run": True, "n_gpus": world, "gpus_arg": args.gpus, "ms_per_step": ms, "value": value,
+                          "scaling": "weak", "x_attn_checksum": float(np.abs(acts[0]["x_attn"].astype(np.float64)).sum())}))
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--dry-run-cpu", action="store_true", help="test aid: multi-rank plumbing only, gloo, no GPU (see run_dry)")
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -694,6 +846,16 @@ def main():
     args = ap.parse_args()
     if args.case:
         run_case(args)
+        return
+    world_env = os.environ.get("WORLD_SIZE")
+    if world_env is None and args.gpus > 1:
+        # not under a launcher: start the N ranks here (each re-enters main() with WORLD_SIZE set)
+        sys.exit(launch_ranks(args.gpus, sys.argv[1:]))
+    if world_env is not None and int(world_env) != args.gpus and int(os.environ.get("RANK", "0")) == 0:
+        print("bench.py: --gpus %d but the launcher started %s ranks; using the launcher's count" % (args.gpus, world_env),
+              file=sys.stderr)
+    if args.dry_run_cpu:
+        run_dry(args)
         return
     if args.impl == "reference":
         run_reference(args)
