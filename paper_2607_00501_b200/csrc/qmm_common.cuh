@@ -70,6 +70,15 @@ struct DebugKnobs {
 };
 extern DebugKnobs g_knobs;
 
+// Arguments of the decode-sized mixture-of-experts layer (host side; see moe_small_gate_up_kernel).
+struct MoeSmallHost {
+    const float* logits; const uint16_t* X; const void *w_gate, *w_up, *w_down; int64_t gu_stride, dn_stride;
+    uint16_t *hbuf, *dbg_D, *out; int T, E, topk, H, I;
+    int* idx_ws; float* w_ws; int *perm_ws, *inv_ws, *offsets_ws;
+    int* idx_user; float* w_user; int *perm_user, *offsets_user;
+};
+
+
 // ---------------------------------------------------------------- loads
 
 struct __align__(32) u32x8 {

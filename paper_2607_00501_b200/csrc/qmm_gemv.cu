@@ -14,6 +14,7 @@
 // and a second kernel adds the splits in ascending order (fixed order, so the
 // result does not depend on scheduling).
 #include "qmm_common.cuh"
+#include "qmm_route.cuh"
 
 #include <stdio.h>
 
@@ -591,6 +592,287 @@ moe_gemv_kernel(const MoeGemvParams p)
     }
 }
 
+// ------------------------------------------- MoE decode layer in two launches
+//
+// Decode-sized layers (T * topk <= 32 rows, topk <= 8).  Four dependent launches of ~5 us each
+// (route, gate/up, down, combine) around ~3 us of weight traffic is what a layer per-launch costs;
+// the paper's decode argument is exactly that such dispatch cost, not bytes, dominates short kernels
+// (Sec. 3.3).  Here the layer is two launches:
+//   A: every block routes all T tokens itself (T * E logits: a few KB, ~1 us) instead of waiting for a
+//      routing kernel, then runs its gate/up units with the SiLU*mul epilogue; block 0 also writes the
+//      routing results (indices, weights, permutation, offsets) for the caller.
+//   B: a thread-block cluster per (token, 64 output columns); cluster rank j takes the token's j-th
+//      expert, multiplies the expert's 64 down rows with Hm[row(t, j)], rounds to fp16 (the library's
+//      D), and the cluster's first block adds p_j * D_j in slot order through distributed shared
+//      memory and writes `out` -- D never leaves the SMs and no combine kernel runs.  B routes again
+//      from the logits (an input that is complete before A started), so its blocks know their expert
+//      and prefetch its weights *before* they wait for A's Hm.
+struct MoeSmallParams {
+    const float* logits;        // [T, E]
+    const uint16_t* X;          // [T, H]
+    const uint8_t *w_gate, *w_up, *w_down;
+    int64_t gu_stride, dn_stride;   // bytes between experts
+    uint16_t* hbuf;             // [T*topk, I] permuted row order (workspace or dbg_H)
+    uint16_t* dbg_D;            // [T*topk, H] optional export of D
+    uint16_t* out;              // [T, H]
+    int T, E, topk, H, I;
+    int* idx_ws;                // workspace copies of the routing result (read by nothing downstream, kept for qmm_moe_route parity)
+    float* w_ws;
+    int *perm_ws, *inv_ws, *offsets_ws;
+    int* idx_user;              // optional exports
+    float* w_user;
+    int *perm_user, *offsets_user;
+};
+
+// Routing + stable permutation of all T * topk <= 32 (token, slot) pairs by the whole block.
+// s_e / s_w: expert and weight of flat pair t * topk + j; s_perm[r] = flat pair of permuted row r;
+// s_inv[flat] = r.  Same selection rule and arithmetic as route_kernel, so every block (and the
+// separate routing kernels) get the same bits.
+template <int MAX_PER_LANE, int WARPS>
+__device__ __forceinline__ void route_all(const float* __restrict__ logits, int T, int E, int topk,
+                                          int* s_e, float* s_w, int* s_perm, int* s_inv)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int total = T * topk;
+    for (int t = warp; t < T; t += WARPS) {
+        int sel_idx;
+        float w;
+        route_token<MAX_PER_LANE>(logits + (size_t)t * E, E, topk, lane, sel_idx, w);
+        if (lane < topk) {
+            s_e[t * topk + lane] = sel_idx;
+            s_w[t * topk + lane] = w;
+        }
+    }
+    __syncthreads();
+    if ((int)threadIdx.x < total) {                          // rank of this pair in the (expert, flat index) order
+        const int mine = s_e[threadIdx.x];
+        int r = 0;
+        for (int j = 0; j < total; ++j) {
+            const int other = s_e[j];
+            r += (other < mine || (other == mine && j < (int)threadIdx.x)) ? 1 : 0;
+        }
+        s_perm[r] = threadIdx.x;
+        s_inv[threadIdx.x] = r;
+    }
+    __syncthreads();
+}
+
+template <int FMT, int MAX_PER_LANE, int WARPS>
+__global__ void __launch_bounds__(WARPS * 32, 768 / (WARPS * 32))
+moe_small_gate_up_kernel(const MoeSmallParams p)
+{
+    extern __shared__ uint4 smem[];
+    uint4* xs = smem;
+    uint4* zs = smem + p.H / 8;
+    float* red = reinterpret_cast<float*>(smem + p.H / 4);
+    __shared__ int s_e[32], s_perm[32], s_inv[32];
+    __shared__ float s_w[32];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr int TB = Fmt<FMT>::tile_bytes;
+    constexpr int XV = Fmt<FMT>::tile_k / 8;
+    constexpr int STEP = kUnroll * WARPS;
+    const int K = p.H, N = p.I;
+    const int tpr = K / Fmt<FMT>::tile_k;
+    const int units_per_row = N / 32;
+    const int total = p.T * p.topk;
+    const int units = total * units_per_row;
+    const size_t group_bytes = (size_t)tpr * TB;
+
+    pdl_wait();                                                 // logits and activations come from upstream
+    pdl_launch_dependents();
+    route_all<MAX_PER_LANE, WARPS>(p.logits, p.T, p.E, p.topk, s_e, s_w, s_perm, s_inv);
+    if (blockIdx.x == 0) {                                      // the routing result, for the caller and the workspace
+        if ((int)threadIdx.x < total) {
+            const int i = threadIdx.x;
+            p.idx_ws[i] = s_e[i];
+            p.w_ws[i] = s_w[i];
+            p.perm_ws[i] = s_perm[i];
+            p.inv_ws[i] = s_inv[i];
+            if (p.idx_user) p.idx_user[i] = s_e[i];
+            if (p.w_user) p.w_user[i] = s_w[i];
+            if (p.perm_user) p.perm_user[i] = s_perm[i];
+        }
+        for (int e = threadIdx.x; e <= p.E; e += WARPS * 32) {  // rows of the experts before e
+            int c = 0;
+            for (int j = 0; j < total; ++j) c += s_e[j] < e ? 1 : 0;
+            p.offsets_ws[e] = c;
+            if (p.offsets_user) p.offsets_user[e] = c;
+        }
+    }
+    for (int i = threadIdx.x; i < K / 8; i += WARPS * 32) zs[i] = make_uint4(0u, 0u, 0u, 0u);
+    const uint4* xb = ((lane >> 2) == (lane & 3)) ? xs : zs;
+    Q4Consts kc;
+    kc.init();
+
+    int cur_row = -1;
+    for (int u = blockIdx.x; u < units; u += gridDim.x) {
+        const int r = u / units_per_row, j = u - r * units_per_row;
+        const int flat = s_perm[r];
+        const int e = s_e[flat];
+        const uint8_t* tiles_p = p.w_gate + (size_t)e * p.gu_stride + (size_t)j * group_bytes + 32 * lane;
+        const uint8_t* tiles_q = p.w_up + (size_t)e * p.gu_stride + (size_t)j * group_bytes + 32 * lane;
+        TileRegs<FMT> rg;
+        auto load_group = [&](int t) {
+#pragma unroll
+            for (int q = 0; q < kUnroll; ++q) {
+                const int tt = t + q * WARPS;
+                if (tt < tpr) {
+                    const uint8_t* tp = tiles_p + (size_t)tt * TB;
+                    const uint8_t* tq = tiles_q + (size_t)tt * TB;
+                    rg.cp[q] = ld_stream_256(tp);
+                    rg.cq[q] = ld_stream_256(tq);
+                    rg.sp[q] = load_scales<FMT>(tp - 32 * lane, lane);
+                    rg.sq[q] = load_scales<FMT>(tq - 32 * lane, lane);
+                }
+            }
+        };
+        load_group(warp);                                       // weights fly while the activation row is staged
+        if (r != cur_row) {
+            __syncthreads();
+            const uint16_t* xr = p.X + (size_t)(flat / p.topk) * K;
+            for (int i = threadIdx.x; i < K / 8; i += WARPS * 32) xs[i] = reinterpret_cast<const uint4*>(xr)[i];
+            __syncthreads();
+            cur_row = r;
+        }
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int t = warp; t < tpr; t += STEP) {
+#pragma unroll
+            for (int q = 0; q < kUnroll; ++q) {
+                const int tt = t + q * WARPS;
+                if (tt < tpr) {
+                    if constexpr (FMT == QMM_Q4)
+                        tile_pair_mma_q4(rg.cp[q], rg.cq[q], rg.sp[q], rg.sq[q], xb + tt * XV, acc, kc);
+                    else
+                        tile_pair_mma_q8(rg.cp[q], rg.cq[q], rg.sp[q], rg.sq[q], xb + tt * XV, acc);
+                }
+            }
+            if (t + STEP < tpr) load_group(t + STEP);
+        }
+        if ((lane & 3) < 2) {
+            const int row = (lane & ~3) + 2 * (lane & 1);
+            float* w = red + warp * 64;
+            w[row] = acc[0];
+            w[row + 1] = acc[1];
+            w[32 + row] = acc[2];
+            w[32 + row + 1] = acc[3];
+        }
+        __syncthreads();
+        if (threadIdx.x < 32) {                                 // red[.. 0..31] = G, red[.. 32..63] = U
+            float g = red[threadIdx.x], up = red[32 + threadIdx.x];
+#pragma unroll
+            for (int w = 1; w < WARPS; ++w) {
+                g += red[w * 64 + threadIdx.x];
+                up += red[w * 64 + 32 + threadIdx.x];
+            }
+            const float h = (g / (1.0f + expf(-g))) * up;
+            p.hbuf[(size_t)r * N + j * 32 + threadIdx.x] = __half_as_ushort(__float2half_rn(h));
+        }
+        __syncthreads();
+    }
+}
+
+// Launch B (see above).  gridDim.x = T * (H / 64) * topk, cluster = topk blocks.
+template <int FMT, int MAX_PER_LANE, int WARPS>
+__global__ void __launch_bounds__(WARPS * 32, 768 / (WARPS * 32))
+moe_small_down_combine_kernel(const MoeSmallParams p)
+{
+    extern __shared__ uint4 smem[];
+    uint4* xs = smem;
+    uint4* zs = smem + p.I / 8;
+    float* red = reinterpret_cast<float*>(smem + p.I / 4);
+    float* cred = red + WARPS * 64;                             // [kMaxClusterSplits][64] in the cluster's first block
+    __shared__ int s_e[32], s_perm[32], s_inv[32];
+    __shared__ float s_w[32];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr int TB = Fmt<FMT>::tile_bytes;
+    constexpr int XV = Fmt<FMT>::tile_k / 8;
+    constexpr int STEP = kUnroll * WARPS;
+    const int K = p.I, N = p.H;
+    const int tpr = K / Fmt<FMT>::tile_k;
+    const size_t group_bytes = (size_t)tpr * TB;
+    // every block of the cluster has started once this barrier phase completes (awaited before the
+    // first store into the first block's shared memory)
+    asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
+    const int slot = blockIdx.x % p.topk;                       // rank in the cluster = the token's slot j
+    const int cu = blockIdx.x / p.topk;
+    const int col_groups = N / 64;
+    const int t = cu / col_groups, g = cu - t * col_groups;     // token, group of 64 output columns
+
+    // the logits are an input of the layer: complete before launch A started, so they can be read now
+    route_all<MAX_PER_LANE, WARPS>(p.logits, p.T, p.E, p.topk, s_e, s_w, s_perm, s_inv);
+    const int flat = t * p.topk + slot;
+    const int e = s_e[flat];
+    const int r = s_inv[flat];                                  // permuted row of (t, slot)
+    const uint8_t* tiles_p = p.w_down + (size_t)e * p.dn_stride + (size_t)(2 * g) * group_bytes + 32 * lane;
+    const uint8_t* tiles_q = tiles_p + group_bytes;
+    TileRegs<FMT> rg;
+    auto load_group = [&](int t0) {
+#pragma unroll
+        for (int q = 0; q < kUnroll; ++q) {
+            const int tt = t0 + q * WARPS;
+            if (tt < tpr) {
+                const uint8_t* tp = tiles_p + (size_t)tt * TB;
+                const uint8_t* tq = tiles_q + (size_t)tt * TB;
+                rg.cp[q] = ld_stream_256(tp);
+                rg.cq[q] = ld_stream_256(tq);
+                rg.sp[q] = load_scales<FMT>(tp - 32 * lane, lane);
+                rg.sq[q] = load_scales<FMT>(tq - 32 * lane, lane);
+            }
+        }
+    };
+    load_group(warp);                                           // the expert's weights, ahead of the wait for Hm
+    for (int i = threadIdx.x; i < K / 8; i += WARPS * 32) zs[i] = make_uint4(0u, 0u, 0u, 0u);
+
+    pdl_launch_dependents();
+    pdl_wait();                                                 // Hm is written by launch A
+    {
+        const uint16_t* xr = p.hbuf + (size_t)r * K;
+        for (int i = threadIdx.x; i < K / 8; i += WARPS * 32) xs[i] = __ldcg(reinterpret_cast<const uint4*>(xr) + i);
+    }
+    __syncthreads();
+    const uint4* xb = ((lane >> 2) == (lane & 3)) ? xs : zs;
+    Q4Consts kc;
+    kc.init();
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int t0 = warp; t0 < tpr; t0 += STEP) {
+#pragma unroll
+        for (int q = 0; q < kUnroll; ++q) {
+            const int tt = t0 + q * WARPS;
+            if (tt < tpr) {
+                if constexpr (FMT == QMM_Q4)
+                    tile_pair_mma_q4(rg.cp[q], rg.cq[q], rg.sp[q], rg.sq[q], xb + tt * XV, acc, kc);
+                else
+                    tile_pair_mma_q8(rg.cp[q], rg.cq[q], rg.sp[q], rg.sq[q], xb + tt * XV, acc);
+            }
+        }
+        if (t0 + STEP < tpr) load_group(t0 + STEP);
+    }
+    if ((lane & 3) < 2) {
+        const int row = (lane & ~3) + 2 * (lane & 1);
+        float* w = red + warp * 64;
+        w[row] = acc[0];
+        w[row + 1] = acc[1];
+        w[32 + row] = acc[2];
+        w[32 + row + 1] = acc[3];
+    }
+    __syncthreads();
+    asm volatile("barrier.cluster.wait.aligned;" ::: "memory");
+    if (threadIdx.x < 64) {
+        float sum = red[threadIdx.x];
+#pragma unroll
+        for (int w = 1; w < WARPS; ++w) sum += red[w * 64 + threadIdx.x];
+        const __half d = __float2half_rn(sum);                  // D is an fp16 tensor of the layer's definition
+        if (p.dbg_D) p.dbg_D[(size_t)r * N + g * 64 + threadIdx.x] = __half_as_ushort(d);
+        st_cluster_rank0(cred + slot * 64 + threadIdx.x, __half2float(d));
+    }
+    cluster_sync();
+    if (slot == 0 && threadIdx.x < 64) {                        // out = fp16(sum_j p_j * D_j), j ascending, as combine_kernel
+        float o = 0.f;
+        for (int j = 0; j < p.topk; ++j) o = fmaf(s_w[t * p.topk + j], cred[j * 64 + threadIdx.x], o);
+        p.out[(size_t)t * N + g * 64 + threadIdx.x] = __half_as_ushort(__float2half_rn(o));
+    }
+}
+
 // Second stage of split-K: y[n] = fp16(sum_s partial[s][n]), s ascending.
 __global__ void gemv_reduce_kernel(const float* __restrict__ partial, uint16_t* __restrict__ y, int N, int splits)
 {
@@ -772,6 +1054,76 @@ qmm_status launch_moe_gemv(int fmt, bool gate_up, const void* w0, const void* w1
     else QMM_MOE_GEMV(QMM_Q8, kMoeDown)
 #undef QMM_MOE_GEMV
     return check_cuda(e, "qmm_moe decode GEMV launch");
+}
+
+// Decode-sized MoE layer in two launches (see moe_small_gate_up_kernel).
+
+template <int FMT, int MPL>
+static qmm_status launch_moe_small_t(const MoeSmallParams& p, bool route_only, cudaStream_t st)
+{
+    constexpr int WARPS = 8;
+    const int total = p.T * p.topk;
+    {
+        auto kern = moe_small_gate_up_kernel<FMT, MPL, WARPS>;
+        const size_t smem = (size_t)p.H * 4 + (size_t)WARPS * 64 * sizeof(float);
+        cudaError_t e = cudaSuccess;
+        if (smem > 48 * 1024) e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return check_cuda(e, "qmm_moe decode gate/up shared memory size");
+        const int units = route_only ? 0 : total * (p.I / 32);
+        int grid = units < kNumSMs * 3 ? units : kNumSMs * 3;
+        if (grid < 1) grid = 1;                                 // block 0 always exports the routing result
+        MoeSmallParams q = p;
+        if (route_only) q.I = 0;                                // no units: routing only
+        e = launch_pdl(kern, dim3(grid), dim3(WARPS * 32), smem, st, q);
+        if (e != cudaSuccess) return check_cuda(e, "qmm_moe decode gate/up launch");
+    }
+    if (route_only) return QMM_OK;
+    {
+        auto kern = moe_small_down_combine_kernel<FMT, MPL, WARPS>;
+        const size_t smem = (size_t)p.I * 4 + (size_t)WARPS * 64 * sizeof(float) + kMaxClusterSplits * 64 * sizeof(float);
+        cudaError_t e = cudaSuccess;
+        if (smem > 48 * 1024) e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return check_cuda(e, "qmm_moe decode down shared memory size");
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(p.T * (p.H / 64) * p.topk));
+        cfg.blockDim = dim3(WARPS * 32);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[2];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = (unsigned)p.topk;
+        attr[1].val.clusterDim.y = 1;
+        attr[1].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 2;
+        e = cudaLaunchKernelEx(&cfg, kern, p);
+        if (e != cudaSuccess) return check_cuda(e, "qmm_moe decode down + combine launch");
+    }
+    return QMM_OK;
+}
+
+// Limits of the two-launch form: the pairs fit one warp's ranking pass, the experts of a token fit a
+// portable cluster, a row of X / Hm fits the shared-memory staging.
+bool moe_small_supported(int T, int topk, int H, int I)
+{
+    return T * topk <= 32 && topk <= kMaxClusterSplits && H <= 32768 && I <= 32768 && H % 64 == 0 && I % 32 == 0;
+}
+
+qmm_status launch_moe_small(int fmt, const MoeSmallHost& h, bool route_only, cudaStream_t st)
+{
+    MoeSmallParams p;
+    p.logits = h.logits; p.X = h.X;
+    p.w_gate = (const uint8_t*)h.w_gate; p.w_up = (const uint8_t*)h.w_up; p.w_down = (const uint8_t*)h.w_down;
+    p.gu_stride = h.gu_stride; p.dn_stride = h.dn_stride;
+    p.hbuf = h.hbuf; p.dbg_D = h.dbg_D; p.out = h.out;
+    p.T = h.T; p.E = h.E; p.topk = h.topk; p.H = h.H; p.I = h.I;
+    p.idx_ws = h.idx_ws; p.w_ws = h.w_ws; p.perm_ws = h.perm_ws; p.inv_ws = h.inv_ws; p.offsets_ws = h.offsets_ws;
+    p.idx_user = h.idx_user; p.w_user = h.w_user; p.perm_user = h.perm_user; p.offsets_user = h.offsets_user;
+    const bool narrow = (h.E + 31) / 32 <= 4;
+    if (fmt == QMM_Q4) return narrow ? launch_moe_small_t<QMM_Q4, 4>(p, route_only, st) : launch_moe_small_t<QMM_Q4, 32>(p, route_only, st);
+    return narrow ? launch_moe_small_t<QMM_Q8, 4>(p, route_only, st) : launch_moe_small_t<QMM_Q8, 32>(p, route_only, st);
 }
 
 // Host side of qmm_gemv_batch: up to kMaxBatch problems per launch.

@@ -10,6 +10,7 @@
 // Nothing synchronises with the host: the token-tile work list of the grouped
 // GEMMs is built on the device from the expert offsets.
 #include "qmm_gemm_kernel.cuh"
+#include "qmm_route.cuh"
 
 namespace qmm {
 
@@ -20,6 +21,9 @@ int pick_expert_tile(int64_t total_rows, int experts);
 qmm_status launch_moe_gemv(int fmt, bool gate_up, const void* w0, const void* w1, int64_t expert_stride,
                            const uint16_t* x, uint16_t* out, const int* perm, const int* topk_idx,
                            int rows, int topk, int N, int K, cudaStream_t st);
+
+bool moe_small_supported(int T, int topk, int H, int I);
+qmm_status launch_moe_small(int fmt, const MoeSmallHost& h, bool route_only, cudaStream_t st);
 
 // Up to this many (token, expert) rows the expert products run as GEMVs (each row streams its expert's
 // matrices once); above it, as grouped tensor-core GEMMs (each expert's matrices are read once per layer).
@@ -66,53 +70,6 @@ static MoeWorkspace moe_layout(const qmm_moe_args* a)
 size_t moe_workspace_bytes(const qmm_moe_args* a) { return moe_layout(a).total; }
 
 // ---------------------------------------------------------------- route
-
-// Routing of one token by one warp.  topk passes; each pass takes the largest
-// remaining logit, equal logits going to the lower expert index.  The weights
-// are the softmax over the selected logits in fp32.  On return lane j < topk
-// holds the j-th selected expert and its weight.
-template <int MAX_PER_LANE>
-__device__ __forceinline__ void route_token(const float* __restrict__ l, int E, int topk, int lane, int& sel_idx, float& sel_w)
-{
-    float v[MAX_PER_LANE];
-#pragma unroll
-    for (int i = 0; i < MAX_PER_LANE; ++i) {
-        const int e = lane + 32 * i;
-        v[i] = e < E ? l[e] : -INFINITY;
-    }
-    unsigned taken = 0;                                   // bit i: v[i] already selected
-    float sel_val = 0.f, lmax = 0.f, denom = 0.f;         // lane j keeps the j-th selected logit
-    sel_idx = 0;
-    for (int j = 0; j < topk; ++j) {
-        float best = -INFINITY;
-        int best_e = 0x7FFFFFFF;
-#pragma unroll
-        for (int i = 0; i < MAX_PER_LANE; ++i) {
-            const int e = lane + 32 * i;
-            if (e < E && !((taken >> i) & 1u) && (v[i] > best || (v[i] == best && e < best_e))) {
-                best = v[i];
-                best_e = e;
-            }
-        }
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) {
-            const float ob = __shfl_xor_sync(0xFFFFFFFFu, best, off);
-            const int oe = __shfl_xor_sync(0xFFFFFFFFu, best_e, off);
-            if (ob > best || (ob == best && oe < best_e)) {
-                best = ob;
-                best_e = oe;
-            }
-        }
-        if ((best_e & 31) == lane) taken |= 1u << (best_e >> 5);
-        if (j == 0) lmax = best;
-        if (lane == j) {
-            sel_val = best;
-            sel_idx = best_e;
-        }
-        denom += expf(best - lmax);                       // same value and order on every lane
-    }
-    sel_w = expf(sel_val - lmax) / denom;
-}
 
 // One warp per token; also counts rows per expert.
 template <int MAX_PER_LANE>
@@ -384,6 +341,19 @@ qmm_status launch_moe(const qmm_moe_args* a, void* ws, bool route_only, cudaStre
     const int per_lane = (a->E + 31) / 32;
     // decode-sized: one block does steps 1-2 and the expert products run as GEMVs
     const bool small = total <= kMoeGemvMaxRows && a->T <= 32 && a->H <= 32768 && a->I <= 32768;
+    const size_t gu_stride = (size_t)(a->I / kRowsPerGroup) * (size_t)(a->H / tile_k_of(a->fmt)) * tile_bytes_of(a->fmt);
+    const size_t dn_stride = (size_t)(a->H / kRowsPerGroup) * (size_t)(a->I / tile_k_of(a->fmt)) * tile_bytes_of(a->fmt);
+    if (small && !g_knobs.moe_no_fuse && moe_small_supported(a->T, a->topk, a->H, a->I)) {
+        // decode: the whole layer in two launches (routing inside the gate/up launch, combine inside the down launch)
+        MoeSmallHost h;
+        h.logits = a->logits; h.X = a->X; h.w_gate = a->w_gate; h.w_up = a->w_up; h.w_down = a->w_down;
+        h.gu_stride = (int64_t)gu_stride; h.dn_stride = (int64_t)dn_stride;
+        h.hbuf = hbuf; h.dbg_D = a->dbg_D; h.out = a->out;
+        h.T = a->T; h.E = a->E; h.topk = a->topk; h.H = a->H; h.I = a->I;
+        h.idx_ws = topk_idx; h.w_ws = topk_w; h.perm_ws = perm; h.inv_ws = inv_perm; h.offsets_ws = offsets;
+        h.idx_user = a->topk_idx; h.w_user = a->topk_w; h.perm_user = a->perm; h.offsets_user = a->expert_offsets;
+        return launch_moe_small(a->fmt, h, route_only, st);
+    }
     if (small) {
         if (per_lane <= 4)
             e = launch_pdl(route_small_kernel<4>, dim3(1), dim3(1024), st, a->logits, (int)a->T, (int)a->E, (int)a->topk, topk_idx,
@@ -412,9 +382,6 @@ qmm_status launch_moe(const qmm_moe_args* a, void* ws, bool route_only, cudaStre
         if (e != cudaSuccess) return check_cuda(e, "qmm_moe permute launch");
     }
     if (route_only) return QMM_OK;
-
-    const size_t gu_stride = (size_t)(a->I / kRowsPerGroup) * (size_t)(a->H / tile_k_of(a->fmt)) * tile_bytes_of(a->fmt);
-    const size_t dn_stride = (size_t)(a->H / kRowsPerGroup) * (size_t)(a->I / tile_k_of(a->fmt)) * tile_bytes_of(a->fmt);
 
     if (small) {
         // decode: a few rows -> GEMV path (gate/up with SiLU*mul, down), then the combine

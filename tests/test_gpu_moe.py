@@ -184,6 +184,31 @@ def test_moe_negative_and_zero_scales(qmm, oracle, fmt, T):
     check_end_to_end(oracle, L, res, logits, X, topk, tokens=range(min(T, 4)))
 
 
+@pytest.mark.parametrize("fmt", [Q4, Q8])
+@pytest.mark.parametrize("T,E,topk,H,I", [(1, 128, 8, 2048, 768), (4, 128, 8, 512, 256), (3, 16, 5, 256, 512), (32, 8, 1, 256, 256),
+                                          (2, 256, 7, 256, 256)])
+def test_moe_decode_two_launches_match_the_four_launch_form(qmm, oracle, fmt, T, E, topk, H, I):
+    """Decode-sized layers run as two launches (routing inside the gate/up launch, down product and
+    combine in one cluster kernel).  Forcing the separate route / gate-up / down / combine launches must
+    give the same routing, the same Hm and D, and the same output bits: both forms do the same
+    arithmetic in the same order."""
+    L = Layer(qmm, fmt, 650 + T + E + topk, E, H, I)
+    X = synth.activations(651, T + topk, T, H)
+    logits = synth.logits(652, T + E, T, E)
+    fused = run_layer(qmm, L, logits, X, topk)
+    check_stages(oracle, L, fused, logits, X, topk, experts=sorted(set(fused["topk_idx"].reshape(-1).tolist())))
+    check_end_to_end(oracle, L, fused, logits, X, topk, tokens=range(min(T, 3)))
+    qmm.debug_config("moe_no_fuse", "1")
+    plain = run_layer(qmm, L, logits, X, topk)
+    for k in ("topk_idx", "topk_w", "perm", "expert_offsets", "dbg_H", "dbg_D", "out"):
+        assert np.array_equal(fused[k], plain[k]), k
+    qmm.debug_config(None)
+    routed = run_layer(qmm, L, logits, X, topk, route_only=True)
+    for k in ("topk_idx", "topk_w", "perm", "expert_offsets"):
+        assert np.array_equal(fused[k], routed[k]), k
+    assert np.all(routed["out"] == 3.0)
+
+
 def test_moe_route_only_and_determinism(qmm, oracle):
     T, E, topk, H, I = 300, 128, 8, 256, 256
     L = Layer(qmm, Q4, 621, 1, H, I)                     # weights unused by the routing call
