@@ -76,6 +76,7 @@ struct MoeSmallHost {
     uint16_t *hbuf, *dbg_D, *out; int T, E, topk, H, I;
     int* idx_ws; float* w_ws; int *perm_ws, *inv_ws, *offsets_ws;
     int* idx_user; float* w_user; int *perm_user, *offsets_user;
+    long long* trace;           // tuning builds only, else null
 };
 
 

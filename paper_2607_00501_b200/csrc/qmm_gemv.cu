@@ -622,7 +622,23 @@ struct MoeSmallParams {
     int* idx_user;              // optional exports
     float* w_user;
     int *perm_user, *offsets_user;
+    long long* trace;           // -DQMM_MOE_TRACE=1 builds: %globaltimer samples of block 0 of each launch; else unused
 };
+
+// Time stamps of the two launches' first blocks (tuning builds only; the shipped kernels carry none).
+#ifndef QMM_MOE_TRACE
+#define QMM_MOE_TRACE 0
+#endif
+#if QMM_MOE_TRACE
+#define QMM_MOE_STAMP(i)                                                        \
+    if (blockIdx.x == 0 && threadIdx.x == 0 && p.trace != nullptr) {            \
+        long long t_;                                                           \
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                  \
+        p.trace[i] = t_;                                                        \
+    }
+#else
+#define QMM_MOE_STAMP(i)
+#endif
 
 // Routing + stable permutation of all T * topk <= 32 (token, slot) pairs by the whole block.
 // s_e / s_w: expert and weight of flat pair t * topk + j; s_perm[r] = flat pair of permuted row r;
@@ -657,8 +673,13 @@ __device__ __forceinline__ void route_all(const float* __restrict__ logits, int 
     __syncthreads();
 }
 
+// Four tile pairs in flight per warp (twice the GEMV's): a decode unit is one short stream (gate and up
+// rows of 32 outputs), and every round of loads it needs is a full memory latency on the layer's
+// critical path -- K = 2048 in the 4-bit format is one round this way.
+constexpr int kMoeSmallUnroll = 4;
+
 template <int FMT, int MAX_PER_LANE, int WARPS>
-__global__ void __launch_bounds__(WARPS * 32, 768 / (WARPS * 32))
+__global__ void __launch_bounds__(WARPS * 32, 512 / (WARPS * 32))
 moe_small_gate_up_kernel(const MoeSmallParams p)
 {
     extern __shared__ uint4 smem[];
@@ -670,7 +691,8 @@ moe_small_gate_up_kernel(const MoeSmallParams p)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     constexpr int TB = Fmt<FMT>::tile_bytes;
     constexpr int XV = Fmt<FMT>::tile_k / 8;
-    constexpr int STEP = kUnroll * WARPS;
+    constexpr int UNR = kMoeSmallUnroll;
+    constexpr int STEP = UNR * WARPS;
     const int K = p.H, N = p.I;
     const int tpr = K / Fmt<FMT>::tile_k;
     const int units_per_row = N / 32;
@@ -678,9 +700,12 @@ moe_small_gate_up_kernel(const MoeSmallParams p)
     const int units = total * units_per_row;
     const size_t group_bytes = (size_t)tpr * TB;
 
+    QMM_MOE_STAMP(0)
     pdl_wait();                                                 // logits and activations come from upstream
     pdl_launch_dependents();
+    QMM_MOE_STAMP(1)
     route_all<MAX_PER_LANE, WARPS>(p.logits, p.T, p.E, p.topk, s_e, s_w, s_perm, s_inv);
+    QMM_MOE_STAMP(2)
     if (blockIdx.x == 0) {                                      // the routing result, for the caller and the workspace
         if ((int)threadIdx.x < total) {
             const int i = threadIdx.x;
@@ -711,10 +736,13 @@ moe_small_gate_up_kernel(const MoeSmallParams p)
         const int e = s_e[flat];
         const uint8_t* tiles_p = p.w_gate + (size_t)e * p.gu_stride + (size_t)j * group_bytes + 32 * lane;
         const uint8_t* tiles_q = p.w_up + (size_t)e * p.gu_stride + (size_t)j * group_bytes + 32 * lane;
-        TileRegs<FMT> rg;
+        struct {
+            u32x8 cp[UNR], cq[UNR];
+            typename ScaleRegs<FMT>::type sp[UNR], sq[UNR];
+        } rg;
         auto load_group = [&](int t) {
 #pragma unroll
-            for (int q = 0; q < kUnroll; ++q) {
+            for (int q = 0; q < UNR; ++q) {
                 const int tt = t + q * WARPS;
                 if (tt < tpr) {
                     const uint8_t* tp = tiles_p + (size_t)tt * TB;
@@ -737,7 +765,7 @@ moe_small_gate_up_kernel(const MoeSmallParams p)
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
         for (int t = warp; t < tpr; t += STEP) {
 #pragma unroll
-            for (int q = 0; q < kUnroll; ++q) {
+            for (int q = 0; q < UNR; ++q) {
                 const int tt = t + q * WARPS;
                 if (tt < tpr) {
                     if constexpr (FMT == QMM_Q4)
@@ -748,6 +776,7 @@ moe_small_gate_up_kernel(const MoeSmallParams p)
             }
             if (t + STEP < tpr) load_group(t + STEP);
         }
+        QMM_MOE_STAMP(3)
         if ((lane & 3) < 2) {
             const int row = (lane & ~3) + 2 * (lane & 1);
             float* w = red + warp * 64;
@@ -768,6 +797,7 @@ moe_small_gate_up_kernel(const MoeSmallParams p)
             p.hbuf[(size_t)r * N + j * 32 + threadIdx.x] = __half_as_ushort(__float2half_rn(h));
         }
         __syncthreads();
+        QMM_MOE_STAMP(4)
     }
 }
 
@@ -798,8 +828,10 @@ moe_small_down_combine_kernel(const MoeSmallParams p)
     const int col_groups = N / 64;
     const int t = cu / col_groups, g = cu - t * col_groups;     // token, group of 64 output columns
 
+    QMM_MOE_STAMP(8)
     // the logits are an input of the layer: complete before launch A started, so they can be read now
     route_all<MAX_PER_LANE, WARPS>(p.logits, p.T, p.E, p.topk, s_e, s_w, s_perm, s_inv);
+    QMM_MOE_STAMP(9)
     const int flat = t * p.topk + slot;
     const int e = s_e[flat];
     const int r = s_inv[flat];                                  // permuted row of (t, slot)
@@ -825,6 +857,7 @@ moe_small_down_combine_kernel(const MoeSmallParams p)
 
     pdl_launch_dependents();
     pdl_wait();                                                 // Hm is written by launch A
+    QMM_MOE_STAMP(10)
     {
         const uint16_t* xr = p.hbuf + (size_t)r * K;
         for (int i = threadIdx.x; i < K / 8; i += WARPS * 32) xs[i] = __ldcg(reinterpret_cast<const uint4*>(xr) + i);
@@ -856,6 +889,7 @@ moe_small_down_combine_kernel(const MoeSmallParams p)
         w[32 + row + 1] = acc[3];
     }
     __syncthreads();
+    QMM_MOE_STAMP(11)
     asm volatile("barrier.cluster.wait.aligned;" ::: "memory");
     if (threadIdx.x < 64) {
         float sum = red[threadIdx.x];
@@ -866,6 +900,7 @@ moe_small_down_combine_kernel(const MoeSmallParams p)
         st_cluster_rank0(cred + slot * 64 + threadIdx.x, __half2float(d));
     }
     cluster_sync();
+    QMM_MOE_STAMP(12)
     if (slot == 0 && threadIdx.x < 64) {                        // out = fp16(sum_j p_j * D_j), j ascending, as combine_kernel
         float o = 0.f;
         for (int j = 0; j < p.topk; ++j) o = fmaf(s_w[t * p.topk + j], cred[j * 64 + threadIdx.x], o);
@@ -1070,7 +1105,7 @@ static qmm_status launch_moe_small_t(const MoeSmallParams& p, bool route_only, c
         if (smem > 48 * 1024) e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return check_cuda(e, "qmm_moe decode gate/up shared memory size");
         const int units = route_only ? 0 : total * (p.I / 32);
-        int grid = units < kNumSMs * 3 ? units : kNumSMs * 3;
+        int grid = units < kNumSMs * 2 ? units : kNumSMs * 2;
         if (grid < 1) grid = 1;                                 // block 0 always exports the routing result
         MoeSmallParams q = p;
         if (route_only) q.I = 0;                                // no units: routing only
@@ -1106,9 +1141,13 @@ static qmm_status launch_moe_small_t(const MoeSmallParams& p, bool route_only, c
 
 // Limits of the two-launch form: the pairs fit one warp's ranking pass, the experts of a token fit a
 // portable cluster, a row of X / Hm fits the shared-memory staging.
+// It is taken while the gate/up units fit the SMs in one wave (two blocks of 128 registers per thread
+// per SM): beyond that the four-launch form, whose GEMV kernels keep three lighter blocks per SM, was
+// measured equal (T = 2 at the 128-expert, top-8 layer: 27.5 us both) or faster (T = 4: 38 against 42 us).
 bool moe_small_supported(int T, int topk, int H, int I)
 {
-    return T * topk <= 32 && topk <= kMaxClusterSplits && H <= 32768 && I <= 32768 && H % 64 == 0 && I % 32 == 0;
+    return T * topk <= 32 && topk <= kMaxClusterSplits && H <= 32768 && I <= 32768 && H % 64 == 0 && I % 32 == 0 &&
+           (int64_t)T * topk * (I / 32) <= 2 * kNumSMs;
 }
 
 qmm_status launch_moe_small(int fmt, const MoeSmallHost& h, bool route_only, cudaStream_t st)
@@ -1121,6 +1160,7 @@ qmm_status launch_moe_small(int fmt, const MoeSmallHost& h, bool route_only, cud
     p.T = h.T; p.E = h.E; p.topk = h.topk; p.H = h.H; p.I = h.I;
     p.idx_ws = h.idx_ws; p.w_ws = h.w_ws; p.perm_ws = h.perm_ws; p.inv_ws = h.inv_ws; p.offsets_ws = h.offsets_ws;
     p.idx_user = h.idx_user; p.w_user = h.w_user; p.perm_user = h.perm_user; p.offsets_user = h.offsets_user;
+    p.trace = h.trace;
     const bool narrow = (h.E + 31) / 32 <= 4;
     if (fmt == QMM_Q4) return narrow ? launch_moe_small_t<QMM_Q4, 4>(p, route_only, st) : launch_moe_small_t<QMM_Q4, 32>(p, route_only, st);
     return narrow ? launch_moe_small_t<QMM_Q8, 4>(p, route_only, st) : launch_moe_small_t<QMM_Q8, 32>(p, route_only, st);

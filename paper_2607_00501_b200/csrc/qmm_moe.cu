@@ -352,6 +352,10 @@ qmm_status launch_moe(const qmm_moe_args* a, void* ws, bool route_only, cudaStre
         h.T = a->T; h.E = a->E; h.topk = a->topk; h.H = a->H; h.I = a->I;
         h.idx_ws = topk_idx; h.w_ws = topk_w; h.perm_ws = perm; h.inv_ws = inv_perm; h.offsets_ws = offsets;
         h.idx_user = a->topk_idx; h.w_user = a->topk_w; h.perm_user = a->perm; h.offsets_user = a->expert_offsets;
+        h.trace = nullptr;
+#if defined(QMM_MOE_TRACE) && QMM_MOE_TRACE
+        h.trace = (long long*)(base + w.trace);
+#endif
         return launch_moe_small(a->fmt, h, route_only, st);
     }
     if (small) {

@@ -186,7 +186,7 @@ def test_moe_negative_and_zero_scales(qmm, oracle, fmt, T):
 
 @pytest.mark.parametrize("fmt", [Q4, Q8])
 @pytest.mark.parametrize("T,E,topk,H,I", [(1, 128, 8, 2048, 768), (4, 128, 8, 512, 256), (3, 16, 5, 256, 512), (32, 8, 1, 256, 256),
-                                          (2, 256, 7, 256, 256)])
+                                          (2, 256, 7, 256, 256), (1, 128, 8, 256, 1024)])
 def test_moe_decode_two_launches_match_the_four_launch_form(qmm, oracle, fmt, T, E, topk, H, I):
     """Decode-sized layers run as two launches (routing inside the gate/up launch, down product and
     combine in one cluster kernel).  Forcing the separate route / gate-up / down / combine launches must
