@@ -218,6 +218,63 @@ qmm_status qmm_gemv_gate_up(qmm_format fmt, const void* packed_gate, const void*
 qmm_status qmm_gemv_static(qmm_format fmt, const void* packed, int64_t N, int64_t K,
                            const uint16_t* x_fp16, uint16_t* y_fp16, void* stream);
 
+/* A whole list of decode products -- dependent or not -- as ONE launch.
+ *
+ * The paper's decode loop prepares its dispatches once and replays them with
+ * nothing allocated and nothing decided on the hot path (Sec. 3.2), and fuses
+ * what other runtimes dispatch separately because a kernel per short product is
+ * what bounds decode (Sec. 3.3, Sec. 4.2).  Here a decode step's products are
+ * described once as a list of stages; stage i computes
+ *     QMM_CHAIN_LINEAR        y_i = fp16( W x )                     W [N, K]
+ *     QMM_CHAIN_GATE_UP_SILU  y_i = fp16( silu(W_gate x) * (W_up x) ),
+ *                              silu(g) = g / (1 + exp(-g)), W_gate, W_up [N, K]
+ * (fp32 accumulation) on x = a caller vector (x_stage < 0) or elements
+ * [x_offset, x_offset + K) of the output of an earlier stage -- the value as
+ * rounded to fp16, exactly what a separate qmm_gemv would have been given.
+ * Stages whose inputs are ready together run side by side; a stage that cannot
+ * occupy the GPU by its rows alone is cut along K, its partial sums added in a
+ * fixed order (same bits on every call).
+ *
+ * qmm_chain_build (set-up; synchronises `stream`; allocates host memory only)
+ * plans the work of every thread block, writes the plan into the caller's
+ * device buffer, clears the workspace and fills `info`.  qmm_chain_run is the
+ * hot-path call: one cooperative launch, no allocation, no synchronisation.
+ *   - plan: device, >= qmm_chain_plan_bytes; ws: device, >=
+ *     qmm_chain_workspace_bytes; both 256-byte aligned.  The plan holds
+ *     addresses inside `ws`, of the weights and of the x_fp16 / y_fp16 vectors:
+ *     all must stay where they are while the plan is used.  The workspace
+ *     starts with a status word (qmm_status_check(ws, stream) reports a
+ *     give-up of a bounded wait; after one, clear the workspace and rebuild).
+ *   - Launches that use one workspace must not overlap on the GPU.
+ *   - K <= 32768, K % 256 == 0, N % 128 == 0, x_offset % 8 == 0, <= 4096 stages.
+ *   - The launch needs every SM of the device for itself (one block per SM
+ *     must be resident at once); it fails with QMM_ERR_CUDA if that cannot be.
+ *   - y_fp16 (optional, device, [N] fp16) receives a plain copy of a stage's
+ *     output; outputs of stages without it stay internal.                     */
+typedef enum { QMM_CHAIN_LINEAR = 0, QMM_CHAIN_GATE_UP_SILU = 1 } qmm_chain_op;
+typedef struct {
+    int32_t op;                /* qmm_chain_op                                          */
+    int32_t x_stage;           /* < 0: x_fp16 below; else the index of an earlier stage */
+    int64_t x_offset;          /* first element of that stage's output used as x[0]     */
+    const uint16_t* x_fp16;    /* device, [K] fp16, ready when the launch starts        */
+    const void* packed;        /* device, from qmm_pack: W, or W_gate                   */
+    const void* packed_up;     /* device: W_up (QMM_CHAIN_GATE_UP_SILU), else NULL      */
+    int64_t N, K;
+    uint16_t* y_fp16;          /* device, [N] fp16, optional                            */
+} qmm_chain_stage;
+typedef struct {               /* filled by qmm_chain_build; plain data, may be copied  */
+    int32_t magic, fmt, stages, grid, threads, smem_bytes;
+    uint64_t plan_bytes, ws_bytes;
+    void* plan;
+    void* ws;
+} qmm_chain_info;
+size_t qmm_chain_plan_bytes(qmm_format fmt, const qmm_chain_stage* stages, int count);       /* host array */
+size_t qmm_chain_workspace_bytes(qmm_format fmt, const qmm_chain_stage* stages, int count);
+qmm_status qmm_chain_build(qmm_format fmt, const qmm_chain_stage* stages, int count,
+                           void* plan, size_t plan_bytes, void* ws, size_t ws_bytes,
+                           qmm_chain_info* info, void* stream);
+qmm_status qmm_chain_run(const qmm_chain_info* info, void* stream);
+
 /* Prefill matrix-matrix product (Sec. 3.3 "GEMM (prefill, M>1)", Sec. 3.4):
  *   Y[m,n] = fp16( sum_k w[n,k] * X[m,k] ), fp32 accumulation on the tensor
  * cores; weights enter the contraction as fp16(float(d) * q).

@@ -48,6 +48,12 @@ qmm_status status_check(void* ws, cudaStream_t st);
 qmm_status launch_packed_check(int fmt, const void* packed, int64_t N, int64_t K, int* status, cudaStream_t st);
 qmm_status launch_wait_give_up(int* status, long long limit_cycles, cudaStream_t st);
 
+size_t chain_plan_bytes(int fmt, const qmm_chain_stage* st, int count);
+size_t chain_workspace_bytes(int fmt, const qmm_chain_stage* st, int count);
+qmm_status chain_build(int fmt, const qmm_chain_stage* st, int count, void* plan, size_t plan_bytes, void* ws, size_t ws_bytes,
+                       qmm_chain_info* info, cudaStream_t stream);
+qmm_status chain_run(const qmm_chain_info* info, cudaStream_t stream);
+
 DebugKnobs g_knobs = {};
 
 static bool fmt_ok(int fmt) { return fmt == QMM_Q4 || fmt == QMM_Q8; }
@@ -275,6 +281,31 @@ qmm_status qmm_status_check(void* ws, void* stream)
 {
     if (!ws) return fail(QMM_ERR_INVALID_ARG, "qmm_status_check: null workspace");
     return status_check(ws, (cudaStream_t)stream);
+}
+
+size_t qmm_chain_plan_bytes(qmm_format fmt, const qmm_chain_stage* stages, int count)
+{
+    return chain_plan_bytes(fmt, stages, count);
+}
+
+size_t qmm_chain_workspace_bytes(qmm_format fmt, const qmm_chain_stage* stages, int count)
+{
+    return chain_workspace_bytes(fmt, stages, count);
+}
+
+qmm_status qmm_chain_build(qmm_format fmt, const qmm_chain_stage* stages, int count, void* plan, size_t plan_bytes,
+                           void* ws, size_t ws_bytes, qmm_chain_info* info, void* stream)
+{
+    qmm_status s = check_device("qmm_chain_build");
+    if (s != QMM_OK) return s;
+    return chain_build(fmt, stages, count, plan, plan_bytes, ws, ws_bytes, info, (cudaStream_t)stream);
+}
+
+qmm_status qmm_chain_run(const qmm_chain_info* info, void* stream)
+{
+    qmm_status s = check_device("qmm_chain_run");
+    if (s != QMM_OK) return s;
+    return chain_run(info, (cudaStream_t)stream);
 }
 
 qmm_status qmm_packed_check(qmm_format fmt, const void* packed, int64_t N, int64_t K, void* ws, void* stream)

@@ -33,6 +33,7 @@ EXPORTS = (
     "qmm_dequant", "qmm_gemv_workspace_bytes", "qmm_gemv", "qmm_gemm_workspace_bytes", "qmm_gemm",
     "qmm_moe_workspace_bytes", "qmm_moe", "qmm_moe_route", "qmm_status_check", "qmm_gemv_static", "qmm_gemv_batch",
     "qmm_gemv_gate_up", "qmm_packed_check", "qmm_debug_config", "qmm_debug_wait_give_up",
+    "qmm_chain_plan_bytes", "qmm_chain_workspace_bytes", "qmm_chain_build", "qmm_chain_run",
 )
 
 
@@ -46,6 +47,22 @@ class QmmError(RuntimeError):
 class GemvProblem(ctypes.Structure):
     _fields_ = [("packed", ctypes.c_void_p), ("x_fp16", ctypes.c_void_p), ("y_fp16", ctypes.c_void_p),
                 ("N", ctypes.c_int64), ("K", ctypes.c_int64)]
+
+
+class ChainStage(ctypes.Structure):
+    _fields_ = [("op", ctypes.c_int32), ("x_stage", ctypes.c_int32), ("x_offset", ctypes.c_int64),
+                ("x_fp16", ctypes.c_void_p), ("packed", ctypes.c_void_p), ("packed_up", ctypes.c_void_p),
+                ("N", ctypes.c_int64), ("K", ctypes.c_int64), ("y_fp16", ctypes.c_void_p)]
+
+
+class ChainInfo(ctypes.Structure):
+    _fields_ = [("magic", ctypes.c_int32), ("fmt", ctypes.c_int32), ("stages", ctypes.c_int32), ("grid", ctypes.c_int32),
+                ("threads", ctypes.c_int32), ("smem_bytes", ctypes.c_int32), ("plan_bytes", ctypes.c_uint64),
+                ("ws_bytes", ctypes.c_uint64), ("plan", ctypes.c_void_p), ("ws", ctypes.c_void_p)]
+
+
+CHAIN_LINEAR = 0
+CHAIN_GATE_UP_SILU = 1
 
 
 class MoeArgs(ctypes.Structure):
@@ -94,6 +111,12 @@ def lib() -> ctypes.CDLL:
             L.qmm_moe.argtypes = [ctypes.POINTER(MoeArgs), vp, sz, vp]
             L.qmm_moe_route.argtypes = [ctypes.POINTER(MoeArgs), vp, sz, vp]
             L.qmm_status_check.argtypes = [vp, vp]
+            L.qmm_chain_plan_bytes.restype = sz
+            L.qmm_chain_plan_bytes.argtypes = [ci, ctypes.POINTER(ChainStage), ci]
+            L.qmm_chain_workspace_bytes.restype = sz
+            L.qmm_chain_workspace_bytes.argtypes = [ci, ctypes.POINTER(ChainStage), ci]
+            L.qmm_chain_build.argtypes = [ci, ctypes.POINTER(ChainStage), ci, vp, sz, vp, sz, ctypes.POINTER(ChainInfo), vp]
+            L.qmm_chain_run.argtypes = [ctypes.POINTER(ChainInfo), vp]
             L.qmm_packed_check.argtypes = [ci, vp, i64, i64, vp, vp]
             L.qmm_debug_config.argtypes = [ctypes.c_char_p, ctypes.c_char_p]
             L.qmm_debug_wait_give_up.argtypes = [vp, i64, vp]
@@ -264,6 +287,42 @@ def moe_route(args: MoeArgs, ws: torch.Tensor) -> None:
 
 def status_check(ws: torch.Tensor) -> None:
     _check(lib().qmm_status_check(ws.data_ptr(), _stream()))
+
+
+class Chain:
+    """A planned list of decode products (qmm_chain_build); run() is the one-launch hot-path call.
+
+    stages: list of dicts with keys op, packed, N, K and either x (fp16 CUDA tensor) or x_stage (+ x_offset);
+    optional packed_up (gate/up stages) and y (fp16 CUDA tensor receiving a plain copy of the output).
+    The object keeps every tensor it refers to alive; the plan and workspace tensors are attributes."""
+
+    def __init__(self, fmt: int, stages):
+        self.fmt = fmt
+        self._keep = []
+        arr = (ChainStage * len(stages))()
+        for i, s in enumerate(stages):
+            x, y, up = s.get("x"), s.get("y"), s.get("packed_up")
+            if x is not None:
+                assert x.is_cuda and x.dtype == torch.float16 and x.is_contiguous() and x.numel() == s["K"]
+            if y is not None:
+                assert y.is_cuda and y.dtype == torch.float16 and y.is_contiguous() and y.numel() == s["N"]
+            arr[i] = ChainStage(s.get("op", CHAIN_LINEAR), -1 if x is not None else s["x_stage"], s.get("x_offset", 0),
+                                _dp(x), s["packed"].data_ptr(), _dp(up), s["N"], s["K"], _dp(y))
+            self._keep.append((x, y, up, s["packed"]))
+        self.stages = arr
+        L = lib()
+        plan_bytes = L.qmm_chain_plan_bytes(fmt, arr, len(arr))
+        ws_bytes = L.qmm_chain_workspace_bytes(fmt, arr, len(arr))
+        if plan_bytes == 0 or ws_bytes == 0:
+            raise QmmError(1, last_error())
+        self.plan = torch.empty(plan_bytes, dtype=torch.uint8, device="cuda")
+        self.ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+        self.info = ChainInfo()
+        _check(L.qmm_chain_build(fmt, arr, len(arr), self.plan.data_ptr(), plan_bytes, self.ws.data_ptr(), ws_bytes,
+                                 ctypes.byref(self.info), _stream()))
+
+    def run(self) -> None:
+        _check(lib().qmm_chain_run(ctypes.byref(self.info), _stream()))
 
 
 def packed_check(fmt: int, packed: torch.Tensor, N: int, K: int, ws: torch.Tensor) -> None:
