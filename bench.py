@@ -415,7 +415,7 @@ def run_ours(args):
     sections = {}
     cpu = None
     if rank == 0 and not args.no_sections:
-        sections = extra_sections(args, qmm, torch, pk, ops, fmts, gpu_index=local)
+        sections = extra_sections(args, qmm, torch, pk, ops, fmts, batch, gpu_index=local)
     if rank == 0 and world == 1 and not args.no_cpu:
         cpu = cpu_baseline(host_blocks, host_acts, fmts, budget_s=args.cpu_seconds)
 
@@ -510,18 +510,59 @@ def hbm_fracs(nbytes, ms, pk):
     return {"GBps": round(gbs, 1), "frac_hbm": round(gbs / pk["hbm_gbs"], 4), "frac_hbm_nominal": round(gbs / NOMINAL_HBM_GBS, 4)}
 
 
-def extra_sections(args, qmm, torch, pk, ops, fmts, gpu_index=0):
+def extra_sections(args, qmm, torch, pk, ops, fmts, batch, gpu_index=0):
     """The rest of the path on its own workloads.  Every entry: `ms` = median device time with L2 flushed
     before each run, `ms_warm` = back to back without flushing (with the SM clock seen during that run)."""
     out = {}
+    want = set(args.sections.split(",")) if args.sections else None
+    on = lambda name: want is None or name in want
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
     dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
     sampler = ClockSampler(gpu_index, interval_ms=20)
     sampler.start()
 
+    # the decode stack as ONE launch (qmm_chain): with the real dependencies of a decoder -- q/k/v, then o
+    # on the first 2048 of its outputs, then gate/up with SiLU*mul, then down, whose output is the next
+    # layer's input: 64 dependent stages -- and, for comparison, the same 112 matrices as independent products
+    for f in (fmts if on("chain") else ()):
+        layers = len(ops[f]) // 4
+        stages = []
+        for l in range(layers):
+            qkv, o, gu, down = ops[f][4 * l:4 * l + 4]                 # (N, K, packed, x, y, ws)
+            base = 4 * l
+            half = gu[2].numel() // 2
+            stages.append(dict(op=qmm.CHAIN_LINEAR, N=3072, K=2048, packed=qkv[2],
+                               **({"x": qkv[3]} if l == 0 else {"x_stage": base - 1, "x_offset": 0})))
+            stages.append(dict(op=qmm.CHAIN_LINEAR, N=2048, K=2048, packed=o[2], x_stage=base, x_offset=0))
+            stages.append(dict(op=qmm.CHAIN_GATE_UP_SILU, N=8192, K=2048, packed=gu[2][:half], packed_up=gu[2][half:],
+                               x_stage=base + 1, x_offset=0))
+            stages.append(dict(op=qmm.CHAIN_LINEAR, N=2048, K=8192, packed=down[2], x_stage=base + 2, x_offset=0,
+                               **({"y": down[4]} if l == layers - 1 else {})))
+        for name, st in (("dependent", stages),
+                         ("independent", [dict(op=qmm.CHAIN_LINEAR, N=N, K=K, packed=w, x=x, y=y) for (w, N, K, x, y) in batch[f]._keep])):
+            chain = qmm.Chain(f, st)
+            chain.run()
+            qmm.status_check(chain.ws)
+            g, sg = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+            fn = chain.run
+            try:
+                with torch.cuda.stream(sg):
+                    with torch.cuda.graph(g, stream=sg):
+                        chain.run()
+                fn = g.replay
+            except Exception:
+                pass                                                   # (timed as plain launches then)
+            med, best = time_op(torch, fn, 20)
+            qmm.status_check(chain.ws)
+            b = stack_bytes(f)
+            out["decode_stack_q%d_one_launch_%s" % (f, name)] = dict(
+                {"ms": round(med, 4), "ms_best": round(best, 4), "stages": len(st), "launches": 1,
+                 "as_graph": fn is not chain.run}, **hbm_fracs(b, med, pk))
+            del chain, g
+
     # per-format decode stacks, one qmm_gemv launch per fused matrix, chained on one stream with
     # programmatic dependent launch (a dependency between consecutive launches, as in a real decoder)
-    for f in fmts:
+    for f in (fmts if on("chained") else ()):
         g = torch.cuda.CUDAGraph()
         s = torch.cuda.Stream()
         with torch.cuda.stream(s):
@@ -538,6 +579,9 @@ def extra_sections(args, qmm, torch, pk, ops, fmts, gpu_index=0):
     # cfg0: one small Q4 GEMV (1.77 MB of weights: 0.27 us of HBM traffic, far below a launch).  Steady
     # state = 300 distinct packed copies (531 MB, larger than L2) so that every product streams from HBM:
     # as 300 chained launches in one graph, and as qmm_gemv_batch launches over the same 300 problems.
+    if not on("cfg0"):
+        return finish_sections(out, sampler) if not any(on(n) for n in ("lm_head", "ffn", "gemm", "moe")) else \
+            rest_of_sections(args, qmm, torch, pk, fmts, out, flush, dev, sampler, on)
     c = synth.CFG0
     copies = 300
     blocks = synth.quantize(c["fmt"], synth.weights(c["seed"], 0, c["N"], c["K"]))
@@ -572,7 +616,18 @@ def extra_sections(args, qmm, torch, pk, ops, fmts, gpu_index=0):
     cfg0["isolated_launch_cold"] = dict({"us": round(med * 1e3, 3), "us_best": round(best * 1e3, 3)}, **hbm_fracs(nb, med, pk))
     out["cfg0_q4_gemv"] = cfg0
     del many, y0, g_cold, g_warm, arr
+    return rest_of_sections(args, qmm, torch, pk, fmts, out, flush, dev, sampler, on)
 
+
+def finish_sections(out, sampler):
+    sampler.stop()
+    attach_clocks(out, sampler)
+    return out
+
+
+def rest_of_sections(args, qmm, torch, pk, fmts, out, flush, dev, sampler, on):
+    if not on("lm_head"):
+        return sections_ffn_on(args, qmm, torch, pk, fmts, out, flush, dev, sampler, on)
     # cfg2: Q8 LM head GEMV
     c = synth.CFG2
     blocks = synth.quantize(c["fmt"], synth.weights(c["seed"], 0, c["N"], c["K"]))
@@ -582,9 +637,12 @@ def extra_sections(args, qmm, torch, pk, ops, fmts, gpu_index=0):
     m = measure(torch, lambda: qmm.gemv(c["fmt"], packed, c["N"], c["K"], x, y=y), flush, iters=20)
     out["lm_head_q8_gemv"] = dict(m, **hbm_fracs(blocks.nbytes, m["ms"], pk))
     del packed, blocks
+    return sections_ffn_on(args, qmm, torch, pk, fmts, out, flush, dev, sampler, on)
 
+
+def sections_ffn_on(args, qmm, torch, pk, fmts, out, flush, dev, sampler, on):
     # one cfg1 layer's feed-forward front half as a single launch: h = silu(Wgate x) * (Wup x)
-    for f in fmts:
+    for f in (fmts if on("ffn") else ()):
         wts = {name: (N, K, w) for name, N, K, act, w in synth.cfg1_layer_weights(0) if name in ("gate", "up")}
         N, K, _ = wts["gate"]
         pgate = qmm.pack(f, dev(synth.quantize(f, wts["gate"][2])), N, K)
@@ -600,7 +658,7 @@ def extra_sections(args, qmm, torch, pk, ops, fmts, gpu_index=0):
     # cfg3: prefill GEMM sweep (Q4 as the config says, plus the small-batch sizes below one token tile;
     # Q8 = the same kernels with the byte expander, measured at the two largest M)
     c = synth.CFG3
-    for f, Ms in ((c["fmt"], (16, 32, 64) + tuple(c["Ms"])), (synth.Q8, c["Ms"][-2:])):
+    for f, Ms in (((c["fmt"], (16, 32, 64) + tuple(c["Ms"])), (synth.Q8, c["Ms"][-2:])) if on("gemm") else ()):
         gemm = {}
         for name, N, K in c["shapes"]:
             blocks = synth.quantize(f, synth.weights(c["seed"], 0 if name == "gate_up" else 1, N, K))
@@ -633,7 +691,7 @@ def extra_sections(args, qmm, torch, pk, ops, fmts, gpu_index=0):
         return dict(m, hbm_floor_ms=round(touched / pk["hbm_gbs"] / 1e6, 4), roofline_floor_ms=round(floor_ms, 4),
                     frac_of_floor=round(floor_ms / m["ms"], 4), **tensor_fracs(fl / m["ms"] / 1e9, pk))
 
-    for f, Ts in ((c["fmt"], c["Ts"]), (synth.Q8, c["Ts"][-1:])):
+    for f, Ts in (((c["fmt"], c["Ts"]), (synth.Q8, c["Ts"][-1:])) if on("moe") else ()):
         gate, up, down = synth.moe_expert_weights(c["seed"], f, c["E"], c["H"], c["I"])
         pg = qmm.pack(f, dev(gate), c["E"] * c["I"], c["H"])
         pu = qmm.pack(f, dev(up), c["E"] * c["I"], c["H"])
@@ -650,9 +708,7 @@ def extra_sections(args, qmm, torch, pk, ops, fmts, gpu_index=0):
             moe["T%d_skewed_load" % T] = moe_entry(f, T, synth.logits(c["seed"], 200 + T, T, c["E"]) + bias[None, :], pg, pu, pd, wbytes)
         out["moe_q%d" % f] = moe
         del pg, pu, pd, gate, up, down
-    sampler.stop()
-    attach_clocks(out, sampler)
-    return out
+    return finish_sections(out, sampler)
 
 
 # --------------------------------------------------------------------------
@@ -840,6 +896,8 @@ def main():
                     help="batch: one qmm_gemv_batch launch per format; streams: one qmm_gemv launch per matrix")
     ap.add_argument("--streams", type=int, default=8, help="streams for --mode streams")
     ap.add_argument("--no-sections", action="store_true", help="skip the LM-head / GEMM / MoE sections")
+    ap.add_argument("--sections", default=None,
+                    help="comma list of the sections to run (chain,chained,cfg0,lm_head,ffn,gemm,moe); default: all")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--case", default=None, help="profiling aid: run a few launches of one kernel and exit (see run_case)")

@@ -34,8 +34,11 @@
 
 namespace qmm {
 
-constexpr int kChainWarps = 16;                                 // consumer warps = tile pairs per ring slot
-constexpr int kChainThreads = (kChainWarps + 1) * 32;           // + the producer warp
+constexpr int kChainPairs = 16;                                 // tile pairs per ring slot
+constexpr int kChainConsumers = 20;                             // consumer warps (16 of them work on any one slot)
+constexpr int kChainPublishers = 2;                             // warps that reduce and publish a unit's 64 outputs
+constexpr int kChainThreads = (kChainConsumers + 1 + kChainPublishers) * 32;   // + the producer warp
+constexpr int kChainMaxSlices = 8;                              // K split of a stage: at most this many slices
 constexpr int kChainMaxSlots = 6;
 constexpr int kChainUnitCache = 160;                            // unit descriptors of a block kept in shared memory
 constexpr int kChainMaxK = 32768;
@@ -115,9 +118,9 @@ __device__ __forceinline__ int ld_volatile_int(const int* p)
     asm volatile("ld.volatile.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
-__device__ __forceinline__ void consumer_sync()                       // the 16 consumer warps only
+__device__ __forceinline__ void consumer_sync()                       // the consumer warps only
 {
-    asm volatile("bar.sync 1, %0;" ::"r"(kChainWarps * 32) : "memory");
+    asm volatile("bar.sync 1, %0;" ::"r"(kChainConsumers * 32) : "memory");
 }
 
 // Barrier of the consumer warps that also tells whether every one of their threads is still fine.
@@ -132,7 +135,7 @@ __device__ __forceinline__ bool consumer_all(bool ok)
         "selp.u32 %0, 1, 0, p;\n\t"
         "}\n"
         : "=r"(r)
-        : "r"((uint32_t)ok), "r"(kChainWarps * 32)
+        : "r"((uint32_t)ok), "r"(kChainConsumers * 32)
         : "memory");
     return r != 0;
 }
@@ -144,7 +147,8 @@ chain_kernel(const uint8_t* __restrict__ plan, uint8_t* ws)
     using namespace tc;
     constexpr int TB = Fmt<FMT>::tile_bytes;
     constexpr int XV = Fmt<FMT>::tile_k / 8;                          // uint4 of activations per tile
-    constexpr int SLOT = 2 * kChainWarps * TB;                        // bytes per ring slot: 16 tiles of P, 16 tiles of Q
+    constexpr int SLOT = 2 * kChainPairs * TB;                        // bytes per ring slot: 16 tiles of P, 16 tiles of Q
+    constexpr int NC = kChainConsumers;
     const ChainHeader* hd = reinterpret_cast<const ChainHeader*>(plan);
     const int* first = reinterpret_cast<const int*>(plan + hd->first_off);
     const ChainUnit* units = reinterpret_cast<const ChainUnit*>(plan + hd->units_off);
@@ -156,18 +160,24 @@ chain_kernel(const uint8_t* __restrict__ plan, uint8_t* ws)
     uint8_t* ring = smem;                                             // NS slots
     uint4* xs = reinterpret_cast<uint4*>(ring + (size_t)NS * SLOT);   // max_k fp16
     uint4* zs = xs + hd->max_k / 8;                                   // one tile of zeros
-    float* red = reinterpret_cast<float*>(zs + XV);                   // [16 warps][64]
-    uint64_t* full = reinterpret_cast<uint64_t*>(red + kChainWarps * 64);
-    uint64_t* empty = full + kChainMaxSlots;
-    volatile int* s_abort = reinterpret_cast<volatile int*>(empty + kChainMaxSlots);
+    float* red = reinterpret_cast<float*>(zs + XV);                   // [2][NC warps][64]: sums of a unit, double-buffered
+    uint64_t* full = reinterpret_cast<uint64_t*>(red + 2 * NC * 64);  // [slots] copies landed
+    uint64_t* empty = full + kChainMaxSlots;                          // [slots] consumers done
+    uint64_t* red_full = empty + kChainMaxSlots;                      // [2] every consumer warp has written its sums
+    uint64_t* red_empty = red_full + 2;                               // [2] the publishers have read them
+    volatile int* s_abort = reinterpret_cast<volatile int*>(red_empty + 2);
     volatile unsigned* s_epoch = reinterpret_cast<volatile unsigned*>(s_abort + 1);
-    ChainUnit* s_units = reinterpret_cast<ChainUnit*>(empty + kChainMaxSlots + 2);   // [kChainUnitCache]
+    ChainUnit* s_units = reinterpret_cast<ChainUnit*>(red_empty + 4); // [kChainUnitCache]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
         for (int s = 0; s < kChainMaxSlots; ++s) {
             mbar_init(&full[s], 1);                                   // the producer's arrive (+ the copies' bytes)
-            mbar_init(&empty[s], kChainWarps);                        // every consumer warp
+            mbar_init(&empty[s], kChainPairs);                        // the 16 consumer warps that work on the slot
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&red_full[b], NC);
+            mbar_init(&red_empty[b], kChainPublishers);
         }
         *s_abort = 0;
         // the tag of this launch: one more than the last completed launch's (all blocks read the same
@@ -190,8 +200,19 @@ chain_kernel(const uint8_t* __restrict__ plan, uint8_t* ws)
     auto unit_at = [&](int ui) -> const ChainUnit* {
         return ui - u_begin < kChainUnitCache ? s_units + (ui - u_begin) : units + ui;
     };
+    int polls = 0;
+    // true while a poll of another block's data may go on: nobody has given up and the time limit holds
+    auto may_wait = [&](long long t0) -> bool {
+        if (*s_abort) return false;
+        if ((++polls & 63) == 0) {
+            if (ld_volatile_int(&ctl->status) != 0) return false;
+            if (clock64() - t0 > kChainWaitCycles) return false;
+        }
+        return true;
+    };
+    bool gave_up = false;
 
-    if (warp == kChainWarps) {
+    if (warp == NC) {
         // ================= producer: weight tiles -> ring, in list order, as far ahead as the ring reaches
         if (lane == 0) {
             int g = 0;
@@ -201,20 +222,20 @@ chain_kernel(const uint8_t* __restrict__ plan, uint8_t* ws)
                 const uint8_t* wp = up->wp;
                 const uint8_t* wq = up->wq;
                 const int nt = up->nt;
-                for (int c = 0; c < nt && ok; c += kChainWarps, ++g) {
+                for (int c = 0; c < nt && ok; c += kChainPairs, ++g) {
                     const int s = g % NS;
                     if (g >= NS) ok = mbar_wait(&empty[s], ((g / NS) - 1) & 1, s_abort, kChainWaitCycles);
                     if (!ok) break;
-                    const int np = min(kChainWarps, nt - c);
+                    const int np = min(kChainPairs, nt - c);
                     uint8_t* dst = ring + (size_t)s * SLOT;
                     mbar_arrive_expect_tx(&full[s], (uint32_t)(2 * np * TB));
                     bulk_g2s(dst, wp + (size_t)c * TB, (uint32_t)(np * TB), &full[s]);
-                    bulk_g2s(dst + kChainWarps * TB, wq + (size_t)c * TB, (uint32_t)(np * TB), &full[s]);
+                    bulk_g2s(dst + kChainPairs * TB, wq + (size_t)c * TB, (uint32_t)(np * TB), &full[s]);
                 }
             }
             if (!ok) {
+                gave_up = true;
                 *s_abort = 1;
-                atomicExch(&ctl->status, (int)QMM_ERR_DEVICE_TIMEOUT);
                 // copies in flight must land before the block's shared memory is released
                 for (int q = max(0, g - NS); q < g; ++q) {
                     const long long t0 = clock64();
@@ -222,8 +243,82 @@ chain_kernel(const uint8_t* __restrict__ plan, uint8_t* ws)
                 }
             }
         }
+    } else if (warp > NC) {
+        // ================= publishers (64 threads): add the consumer warps' sums of a unit in warp order,
+        // finish K splits, publish.  Decoupled from the consumers, which are already on the next unit.
+        const int pt = threadIdx.x - (NC + 1) * 32;                   // output of the unit this thread owns
+        bool ok = true;
+        for (int ui = u_begin; ui < u_end && ok; ++ui) {
+            const ChainUnit& u = *unit_at(ui);
+            const int n = ui - u_begin, buf = n & 1;
+            ok = mbar_wait(&red_full[buf], (n >> 1) & 1, s_abort, kChainWaitCycles);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) break;
+            const float* r = red + buf * (NC * 64);
+            float v = 0.f;
+            bool publish = true;
+            if (u.kind == kUnitGateUp) {
+                const int o = pt & 31;
+                float gsum = r[o], usum = r[32 + o];
+#pragma unroll
+                for (int w = 1; w < NC; ++w) {
+                    gsum += r[w * 64 + o];
+                    usum += r[w * 64 + 32 + o];
+                }
+                v = (gsum / (1.0f + expf(-gsum))) * usum;
+                publish = pt < 32;
+            } else {
+                v = r[pt];
+#pragma unroll
+                for (int w = 1; w < NC; ++w) v += r[w * 64 + pt];
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&red_empty[buf]);              // the consumers may reuse this buffer
+            if (u.kind != kUnitGateUp && u.nslices > 1) {
+                if (u.slice + 1 < u.nslices) {
+                    st_word64(u.part + ((size_t)u.slice * 64 + pt) * 8, __float_as_uint(v), epoch);
+                    publish = false;
+                } else {
+                    // the last slice adds the unit's slices in ascending order (its own last); all loads of
+                    // a polling round are in flight together
+                    const int others = u.nslices - 1;
+                    uint2 w[kChainMaxSlices - 1];
+                    const long long t0 = clock64();
+#pragma unroll
+                    for (int sl = 0; sl < kChainMaxSlices - 1; ++sl)
+                        if (sl < others) w[sl] = ld_volatile_v2(u.part + ((size_t)sl * 64 + pt) * 8);
+#pragma unroll
+                    for (int sl = 0; sl < kChainMaxSlices - 1; ++sl) {
+                        if (sl >= others || !ok) continue;
+                        while (w[sl].y != epoch) {
+                            if (!may_wait(t0)) {
+                                ok = false;
+                                break;
+                            }
+                            w[sl] = ld_volatile_v2(u.part + ((size_t)sl * 64 + pt) * 8);
+                        }
+                    }
+                    float total = __uint_as_float(w[0].x);
+#pragma unroll
+                    for (int sl = 1; sl < kChainMaxSlices - 1; ++sl)
+                        if (sl < others) total += __uint_as_float(w[sl].x);
+                    v = total + v;
+                }
+            }
+            if (publish && ok) {
+                const unsigned hbits = __half_as_ushort(__float2half_rn(v));
+                st_word32(u.y_tag + (size_t)pt * 4, hbits | (tag16 << 16));
+                if (u.y_plain != nullptr) u.y_plain[pt] = (uint16_t)hbits;
+            }
+            ok = __all_sync(0xFFFFFFFFu, ok);
+        }
+        if (!ok) {
+            gave_up = true;
+            *s_abort = 1;
+        }
     } else {
-        // ================= consumers
+        // ================= consumers (NC warps).  A ring slot holds 16 tile pairs; the pairs of successive
+        // slots go round the NC warps (pair i of slot g to warp (16 g + i) mod NC), so all of them work.
         const bool diag = (lane >> 2) == (lane & 3);
         const uint4* xbase = diag ? xs : zs;
         const int xmul = diag ? XV : 0;                               // off-diagonal lanes read the one tile of zeros
@@ -231,49 +326,36 @@ chain_kernel(const uint8_t* __restrict__ plan, uint8_t* ws)
         kc.init();
         int g = 0;
         bool ok = true;
-        int polls = 0;
-        auto give_up = [&]() {
-            *s_abort = 1;
-            if (threadIdx.x == 0) atomicExch(&ctl->status, (int)QMM_ERR_DEVICE_TIMEOUT);
-        };
-        // true while waiting may go on: no other role or block has given up, and the time limit holds
-        auto may_wait = [&](long long t0) -> bool {
-            if (*s_abort) return false;
-            if ((++polls & 63) == 0) {
-                if (ld_volatile_int(&ctl->status) != 0) return false;
-                if (clock64() - t0 > kChainWaitCycles) return false;
-            }
-            return true;
-        };
-        // Control flow: every consumer thread passes the same sequence of consumer barriers.  A thread
-        // that gives up raises the abort flag (which ends every other wait of the block at once), keeps
-        // walking to the next barrier without working, and the barrier's vote takes all of them out together.
+        // Control flow: every consumer thread passes the same sequence of consumer barriers (they only
+        // surround the staging of an activation vector).  A thread that gives up raises the abort flag
+        // (which ends every other wait of the block at once) and walks on without working; the vote at
+        // the next staging barrier takes all of them out together.
         for (int ui = u_begin; ui < u_end; ++ui) {
             const ChainUnit& u = *unit_at(ui);
+            const int n = ui - u_begin, buf = n & 1;
             if (u.flags & kUnitNewX) {
-                // stage the activation range the following units of this block read
                 consumer_sync();                                      // every warp is done with the previous vector
                 const int v0 = u.xt0 * XV, v1 = (u.xt0 + u.xnt) * XV; // uint4 range of xs (8 fp16 each)
                 if (!u.x_tagged) {
-                    for (int i = v0 + (int)threadIdx.x; i < v1; i += kChainWarps * 32)
+                    for (int i = v0 + (int)threadIdx.x; i < v1; i += NC * 32)
                         xs[i] = __ldcg(reinterpret_cast<const uint4*>(u.x) + i);
-                } else {
+                } else if (ok) {
                     // tagged words {fp16, tag}: 8 values = two 16-byte loads; poll until every tag is this launch's
                     const long long t0 = clock64();
                     const unsigned want = tag16 << 16, m = 0xFFFF0000u;
-                    for (int i0 = v0; i0 < v1 && ok; i0 += 4 * kChainWarps * 32) {
-                        uint4 a[4], b[4];
+                    for (int i0 = v0; i0 < v1 && ok; i0 += 2 * NC * 32) {
+                        uint4 a[2], b[2];
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) {                 // all loads of the round in flight at once
-                            const int i = i0 + q * kChainWarps * 32 + (int)threadIdx.x;
+                        for (int q = 0; q < 2; ++q) {                 // all loads of the round in flight at once
+                            const int i = i0 + q * NC * 32 + (int)threadIdx.x;
                             if (i < v1) {
                                 a[q] = ld_volatile_v4(u.x + (size_t)i * 32);
                                 b[q] = ld_volatile_v4(u.x + (size_t)i * 32 + 16);
                             }
                         }
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            const int i = i0 + q * kChainWarps * 32 + (int)threadIdx.x;
+                        for (int q = 0; q < 2; ++q) {
+                            const int i = i0 + q * NC * 32 + (int)threadIdx.x;
                             if (i >= v1 || !ok) continue;
                             while (true) {
                                 const bool have = ((a[q].x & m) == want) && ((a[q].y & m) == want) && ((a[q].z & m) == want) &&
@@ -298,8 +380,9 @@ chain_kernel(const uint8_t* __restrict__ plan, uint8_t* ws)
                 if (!ok) break;
             }
             float acc[4] = {0.f, 0.f, 0.f, 0.f};
-            for (int c = 0; c < u.nt; c += kChainWarps, ++g) {
-                if (!ok) continue;                                    // gave up: walk on to the barrier below
+            for (int c = 0; c < u.nt; c += kChainPairs, ++g) {
+                const int pi = (warp - (g * kChainPairs) % NC + NC) % NC;      // this warp's pair of slot g, if < 16
+                if (!ok || pi >= kChainPairs) continue;
                 const int s = g % NS;
                 ok = mbar_wait(&full[s], (g / NS) & 1, s_abort, kChainWaitCycles);
                 ok = __all_sync(0xFFFFFFFFu, ok);
@@ -307,9 +390,9 @@ chain_kernel(const uint8_t* __restrict__ plan, uint8_t* ws)
                     *s_abort = 1;
                     continue;
                 }
-                if (c + warp < u.nt) {
-                    const uint8_t* tp = ring + (size_t)s * SLOT + (size_t)warp * TB;
-                    const uint8_t* tq = tp + kChainWarps * TB;
+                if (c + pi < u.nt) {
+                    const uint8_t* tp = ring + (size_t)s * SLOT + (size_t)pi * TB;
+                    const uint8_t* tq = tp + kChainPairs * TB;
                     // the two 16-byte halves in an order that keeps a quarter-warp's accesses on distinct banks
                     const int h = (lane >> 2) & 1;
                     u32x8 cp, cq;
@@ -325,7 +408,7 @@ chain_kernel(const uint8_t* __restrict__ plan, uint8_t* ws)
                         cq.v[4] = qhi.x; cq.v[5] = qhi.y; cq.v[6] = qhi.z; cq.v[7] = qhi.w;
                     }
                     const int row = (lane & ~3) + 2 * (lane & 1);     // the rows whose sums this lane receives
-                    const uint4* xt = xbase + (u.t0 + c + warp) * xmul;
+                    const uint4* xt = xbase + (u.t0 + c + pi) * xmul;
                     if constexpr (FMT == QMM_Q4) {
                         const uint2 sp = *reinterpret_cast<const uint2*>(tp + kTileCodeBytes + 4 * row);
                         const uint2 sq = *reinterpret_cast<const uint2*>(tq + kTileCodeBytes + 4 * row);
@@ -339,71 +422,33 @@ chain_kernel(const uint8_t* __restrict__ plan, uint8_t* ws)
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&empty[s]);                // this warp is done with the slot
             }
-            // add the warps' sums in warp order
-            if ((lane & 3) < 2) {
-                const int row = (lane & ~3) + 2 * (lane & 1);
-                float* w = red + warp * 64;
-                w[row] = acc[0];
-                w[row + 1] = acc[1];
-                w[32 + row] = acc[2];
-                w[32 + row + 1] = acc[3];
+            // hand the warp's sums to the publishers (buffer n & 1; its previous contents must have been read)
+            if (ok && n >= 2) {
+                ok = mbar_wait(&red_empty[buf], ((n >> 1) - 1) & 1, s_abort, kChainWaitCycles);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) *s_abort = 1;
             }
-            ok = consumer_all(ok);
-            if (!ok) break;
-            const int n_out = u.kind == kUnitGateUp ? 32 : 64;
-            if ((int)threadIdx.x < n_out) {
-                float v;
-                bool publish = true;
-                if (u.kind == kUnitGateUp) {
-                    float gsum = red[threadIdx.x], usum = red[32 + threadIdx.x];
-#pragma unroll
-                    for (int w = 1; w < kChainWarps; ++w) {
-                        gsum += red[w * 64 + threadIdx.x];
-                        usum += red[w * 64 + 32 + threadIdx.x];
-                    }
-                    v = (gsum / (1.0f + expf(-gsum))) * usum;
-                } else {
-                    v = red[threadIdx.x];
-#pragma unroll
-                    for (int w = 1; w < kChainWarps; ++w) v += red[w * 64 + threadIdx.x];
-                    if (u.nslices > 1) {
-                        if (u.slice + 1 < u.nslices) {
-                            st_word64(u.part + ((size_t)u.slice * 64 + threadIdx.x) * 8, __float_as_uint(v), epoch);
-                            publish = false;
-                        } else {
-                            // the last slice adds the unit's slices in ascending order (its own last)
-                            float total = 0.f;
-                            const long long t0 = clock64();
-                            for (int sl = 0; sl + 1 < u.nslices && ok; ++sl) {
-                                const uint8_t* src = u.part + ((size_t)sl * 64 + threadIdx.x) * 8;
-                                uint2 w = ld_volatile_v2(src);
-                                while (w.y != epoch) {
-                                    if (!may_wait(t0)) {
-                                        ok = false;
-                                        break;
-                                    }
-                                    w = ld_volatile_v2(src);
-                                }
-                                total = sl == 0 ? __uint_as_float(w.x) : total + __uint_as_float(w.x);
-                            }
-                            v = total + v;
-                            if (!ok) *s_abort = 1;
-                        }
-                    }
+            if (ok) {
+                if ((lane & 3) < 2) {
+                    const int row = (lane & ~3) + 2 * (lane & 1);
+                    float* w = red + buf * (NC * 64) + warp * 64;
+                    w[row] = acc[0];
+                    w[row + 1] = acc[1];
+                    w[32 + row] = acc[2];
+                    w[32 + row + 1] = acc[3];
                 }
-                if (publish && ok) {
-                    const unsigned hbits = __half_as_ushort(__float2half_rn(v));
-                    st_word32(u.y_tag + (size_t)threadIdx.x * 4, hbits | (tag16 << 16));
-                    if (u.y_plain != nullptr) u.y_plain[threadIdx.x] = (uint16_t)hbits;
-                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&red_full[buf]);
             }
-            ok = consumer_all(ok);                                    // `red` may be reused; a give-up above reaches everyone
-            if (!ok) break;
         }
-        if (!ok) give_up();
+        if (!ok) {
+            gave_up = true;
+            *s_abort = 1;
+        }
     }
 
     // ---- leave: the last block to arrive records the launch's tag for the next launch
+    if (gave_up) atomicExch(&ctl->status, (int)QMM_ERR_DEVICE_TIMEOUT);
     __syncthreads();
     if (threadIdx.x == 0) {
         __threadfence();
@@ -415,6 +460,10 @@ chain_kernel(const uint8_t* __restrict__ plan, uint8_t* ws)
         }
     }
 }
+
+}  // namespace qmm
+
+namespace qmm {
 
 // ------------------------------------------------------------------ host: the planner
 
@@ -498,16 +547,17 @@ static void plan_chain(int fmt, const qmm_chain_stage* st, int count, ChainLayou
             const int n_units = (int)(gu ? s.N / 32 : s.N / 64);
             const size_t group_bytes = (size_t)tpr * TB;
             // K split: the slice count that minimises (rounds of this stage's items on its share of the blocks)
-            // x (bytes of a slice), plus the price of the extra hop of the partial sums (~40 KB of streaming)
+            // x (bytes of a slice), plus the price of the extra hop of the partial sums through L2 (measured: about
+            // the time a block takes for 150 KB of weights, so only long-K stages with few rows are cut)
             int S = 1;
             if (!gu) {
                 const double share = std::max(1.0, (double)G * ((double)n_units * tpr) / (double)std::max(1LL, level_tiles));
                 double best = 1e30;
-                for (int cand = 1; cand <= 16; ++cand) {
+                for (int cand = 1; cand <= kChainMaxSlices; ++cand) {
                     const int per = (tpr + cand - 1) / cand;
                     if (cand > 1 && per < 4) break;
                     const double rounds = ceil((double)n_units * cand / share);
-                    const double est = rounds * per * 2.0 * TB + (cand > 1 ? 40000.0 : 0.0);
+                    const double est = rounds * per * 2.0 * TB + (cand > 1 ? 150000.0 : 0.0);
                     if (est < best - 1e-9) {
                         best = est;
                         S = cand;
@@ -552,19 +602,38 @@ static void plan_chain(int fmt, const qmm_chain_stage* st, int count, ChainLayou
                 }
             }
         }
-        // deal the items in order, equal cost per block; the block a share goes to rotates with the level
-        long long total = 0;
-        for (const Item& it : items) total += it.cost;
-        long long before = 0;
+        // Deal the items to the blocks.  Items that never wait for another block (whole units, and all
+        // slices of a split unit but the last) come first in every block's list, the last slices (which
+        // wait for the other slices of their unit) after them: when a block reaches one, the slices it
+        // needs were started by their blocks at the same time as its own and are done or nearly so.
+        // Many items: contiguous shares of equal cost (consecutive units of a stage stay together: one
+        // staging of the activation vector).  Few items (a level of a dependent chain): each item to the
+        // least loaded block, so that 128 items occupy 128 blocks.  The first block rotates with the level.
         const int rot = (int)(((long long)lv * 37) % G);
-        for (const Item& it : items) {
-            const long long mid2 = 2 * before + it.cost;                    // twice the item's midpoint
-            int b = (int)((mid2 * G) / (2 * std::max(1LL, total)));
-            if (b >= G) b = G - 1;
-            ChainUnit u = it.u;
-            u.pad[0] = it.stage;                                            // (host only: which stage's vector the unit reads)
-            per_block[(b + rot) % G].push_back(u);
-            before += it.cost;
+        std::vector<long long> load(G, 0);
+        const bool contiguous = (long long)items.size() >= 4LL * G;
+        for (int pass = 0; pass < 2; ++pass) {
+            long long total = 0, before = 0;
+            for (const Item& it : items)
+                if ((it.u.nslices > 1 && it.u.slice + 1 == it.u.nslices) == (pass == 1)) total += it.cost;
+            for (const Item& it : items) {
+                if ((it.u.nslices > 1 && it.u.slice + 1 == it.u.nslices) != (pass == 1)) continue;
+                int b;
+                if (contiguous) {
+                    const long long mid2 = 2 * before + it.cost;                // twice the item's midpoint
+                    b = (int)((mid2 * G) / (2 * std::max(1LL, total)));
+                    if (b >= G) b = G - 1;
+                    before += it.cost;
+                } else {
+                    b = 0;
+                    for (int k = 1; k < G; ++k)
+                        if (load[k] < load[b]) b = k;
+                }
+                load[b] += it.cost;
+                ChainUnit u = it.u;
+                u.pad[0] = it.stage;                                            // (host only: which stage's vector the unit reads)
+                per_block[(b + rot) % G].push_back(u);
+            }
         }
     }
     off = align_up(off, 256);
@@ -596,8 +665,8 @@ static void plan_chain(int fmt, const qmm_chain_stage* st, int count, ChainLayou
     L.ws_bytes = off;
     L.plan_bytes = align_up(sizeof(ChainHeader), 256) + align_up((size_t)(G + 1) * 4, 256) + L.units.size() * sizeof(ChainUnit);
     L.max_k = max_k;
-    const int slot = 2 * kChainWarps * TB;
-    const int fixed = 128 /*alignment*/ + max_k * 2 + (TK / 8) * 16 + kChainWarps * 64 * 4 + (2 * kChainMaxSlots + 2) * 8 +
+    const int slot = 2 * kChainPairs * TB;
+    const int fixed = 128 /*alignment*/ + max_k * 2 + (TK / 8) * 16 + 2 * kChainConsumers * 64 * 4 + (2 * kChainMaxSlots + 8) * 8 +
                       kChainUnitCache * (int)sizeof(ChainUnit) + 64;
     int ns = (227 * 1024 - fixed) / slot;
     L.n_slots = ns > kChainMaxSlots ? kChainMaxSlots : ns;
