@@ -18,6 +18,8 @@ import threading
 import numpy as np
 
 Q4 = 4
+Q5 = 5
+Q6 = 6
 Q8 = 8
 
 _HERE = os.path.dirname(os.path.abspath(__file__))

@@ -73,6 +73,8 @@ uint16_t orc_f2h(float f)
 size_t orc_block_bytes(int fmt)
 {
     if (fmt == ORC_Q4) return 18;
+    if (fmt == ORC_Q5) return 22;
+    if (fmt == ORC_Q6) return 26;
     if (fmt == ORC_Q8) return 34;
     return 0;
 }
@@ -103,6 +105,24 @@ static int decode_block(int fmt, const uint8_t* blk, float* w)
             int u = (i & 1) ? (byte >> 4) : (byte & 0x0F);
             w[i] = df * (float)(u - 8);
         }
+    } else if (fmt == ORC_Q5) {
+        /* d, then 4 bytes of fifth bits (bit i of the little-endian word: element i), then 16 bytes of low nibbles */
+        uint32_t hi = (uint32_t)blk[2] | ((uint32_t)blk[3] << 8) | ((uint32_t)blk[4] << 16) | ((uint32_t)blk[5] << 24);
+        for (i = 0; i < 32; ++i) {
+            uint8_t byte = blk[6 + i / 2];
+            int lo = (i & 1) ? (byte >> 4) : (byte & 0x0F);
+            int u = lo | (int)(((hi >> i) & 1u) << 4);
+            w[i] = df * (float)(u - 16);
+        }
+    } else if (fmt == ORC_Q6) {
+        /* d, then 8 bytes of high bit pairs (byte i/4, bits 2(i%4) and 2(i%4)+1: element i), then 16 bytes of low nibbles */
+        for (i = 0; i < 32; ++i) {
+            uint8_t byte = blk[10 + i / 2];
+            int lo = (i & 1) ? (byte >> 4) : (byte & 0x0F);
+            int hi2 = (blk[2 + i / 4] >> (2 * (i % 4))) & 3;
+            int u = lo | (hi2 << 4);
+            w[i] = df * (float)(u - 32);
+        }
     } else {
         for (i = 0; i < 32; ++i) {
             int q = (int)(int8_t)blk[2 + i];
@@ -120,8 +140,8 @@ int orc_quantize(int fmt, const float* w, int64_t N, int64_t K, uint8_t* blocks)
     if (!bb || !w || !blocks || N <= 0 || K <= 0 || K % 32) return 1;
     nb = K / 32;
     nblk = N * nb;
-    qmax = (fmt == ORC_Q4) ? 7.0f : 127.0f;
-    qmin = (fmt == ORC_Q4) ? -8.0f : -127.0f;
+    qmax = (fmt == ORC_Q4) ? 7.0f : (fmt == ORC_Q5) ? 15.0f : (fmt == ORC_Q6) ? 31.0f : 127.0f;
+    qmin = (fmt == ORC_Q4) ? -8.0f : (fmt == ORC_Q5) ? -16.0f : (fmt == ORC_Q6) ? -32.0f : -127.0f;
 #pragma omp parallel for schedule(static)
     for (g = 0; g < nblk; ++g) {
         const float* src = w + g * 32;
@@ -151,6 +171,17 @@ int orc_quantize(int fmt, const float* w, int64_t N, int64_t K, uint8_t* blocks)
         if (fmt == ORC_Q4) {
             for (i = 0; i < 16; ++i)
                 blk[2 + i] = (uint8_t)((q[2 * i] + 8) | ((q[2 * i + 1] + 8) << 4));
+        } else if (fmt == ORC_Q5) {
+            uint32_t hi = 0;
+            for (i = 0; i < 32; ++i) hi |= (uint32_t)(((q[i] + 16) >> 4) & 1) << i;
+            for (i = 0; i < 4; ++i) blk[2 + i] = (uint8_t)(hi >> (8 * i));
+            for (i = 0; i < 16; ++i)
+                blk[6 + i] = (uint8_t)(((q[2 * i] + 16) & 15) | (((q[2 * i + 1] + 16) & 15) << 4));
+        } else if (fmt == ORC_Q6) {
+            for (i = 0; i < 8; ++i) blk[2 + i] = 0;
+            for (i = 0; i < 32; ++i) blk[2 + i / 4] |= (uint8_t)((((q[i] + 32) >> 4) & 3) << (2 * (i % 4)));
+            for (i = 0; i < 16; ++i)
+                blk[10 + i] = (uint8_t)(((q[2 * i] + 32) & 15) | (((q[2 * i + 1] + 32) & 15) << 4));
         } else {
             for (i = 0; i < 32; ++i) blk[2 + i] = (uint8_t)(int8_t)q[i];
         }

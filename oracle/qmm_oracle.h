@@ -31,7 +31,7 @@
 extern "C" {
 #endif
 
-enum { ORC_Q4 = 4, ORC_Q8 = 8 };
+enum { ORC_Q4 = 4, ORC_Q5 = 5, ORC_Q6 = 6, ORC_Q8 = 8 };
 
 /* ---- fp16 <-> fp32, bit level (IEEE binary16, round to nearest even) ---- */
 float    orc_h2f(uint16_t h);
@@ -42,13 +42,21 @@ uint16_t orc_f2h(float f);
  *   element i in [0,32) has code q_i in [-8,7] stored as u_i = q_i + 8;
  *   qs[j] = u_{2j} | (u_{2j+1} << 4).
  * Q8 block, 34 bytes: uint16 d; int8 qs[32] (two's complement).
+ * Q5 block, 22 bytes: uint16 d; uint8 qh[4]; uint8 qs[16]; code q_i in [-16,15]
+ *   stored as u_i = q_i + 16: qs as in Q4 with the low four bits of u, bit i of
+ *   the little-endian 32-bit word qh = the fifth bit of u_i.
+ * Q6 block, 26 bytes: uint16 d; uint8 qh[8]; uint8 ql[16]; code q_i in [-32,31]
+ *   stored as u_i = q_i + 32: ql as in Q4 with the low four bits of u, bits
+ *   2(i%4), 2(i%4)+1 of qh[i/4] = the two high bits of u_i.
+ *   (The paper's library spans 2-bit to 16-bit formats, Sec. 3.3 / Sec. 4.1,
+ *   and gives no layout for any of them; these two are this library's.)
  * Matrix W[N,K]: row n holds K/32 consecutive blocks, rows consecutive.
  * Dequantised weight: w = h2f(d) * (float)q, which is exact in fp32.       */
-size_t orc_block_bytes(int fmt);                    /* 18 or 34, 0 if fmt unknown */
+size_t orc_block_bytes(int fmt);                    /* 18, 22, 26 or 34; 0 if fmt unknown */
 size_t orc_canonical_bytes(int fmt, int64_t N, int64_t K);
 
 /* Quantiser (inputs only; the GPU never quantises).  Per block, in fp32:
- * amax = max|w_i|; d = f2h(amax/QMAX), QMAX = 7 (Q4) or 127 (Q8);
+ * amax = max|w_i|; d = f2h(amax/QMAX), QMAX = 7 (Q4), 15 (Q5), 31 (Q6) or 127 (Q8);
  * df = h2f(d); df == 0 -> all codes 0; else q_i = clamp(rne(w_i/df)).
  * Returns 0 on success, nonzero on bad arguments.                          */
 int orc_quantize(int fmt, const float* w, int64_t N, int64_t K, uint8_t* blocks);

@@ -16,6 +16,10 @@ Canonical block format (32 elements along K):
   Q4: uint16 fp16 scale, then 16 bytes; element i has code q_i in [-8,7] stored
       as u_i = q_i + 8, byte j = u_{2j} | (u_{2j+1} << 4).            (18 bytes)
   Q8: uint16 fp16 scale, then 32 int8 codes in [-127,127].          (34 bytes)
+  Q5: uint16 fp16 scale, 4 bytes of fifth bits (bit i of the little-endian word:
+      element i), 16 bytes of low nibbles as in Q4; u_i = q_i + 16, q in [-16,15]. (22 bytes)
+  Q6: uint16 fp16 scale, 8 bytes of high bit pairs (bits 2(i%4), 2(i%4)+1 of byte
+      i/4: element i), 16 bytes of low nibbles; u_i = q_i + 32, q in [-32,31].     (26 bytes)
 Row n of W[N,K] holds K/32 consecutive blocks; rows are consecutive.
 """
 from __future__ import annotations
@@ -23,9 +27,12 @@ from __future__ import annotations
 import numpy as np
 
 Q4 = 4
+Q5 = 5
+Q6 = 6
 Q8 = 8
 BLOCK = 32
-BLOCK_BYTES = {Q4: 18, Q8: 34}
+BLOCK_BYTES = {Q4: 18, Q5: 22, Q6: 26, Q8: 34}
+QRANGE = {Q4: (-8, 7), Q5: (-16, 15), Q6: (-32, 31), Q8: (-127, 127)}     # what the quantiser emits (Q8 decodes -128 too)
 
 
 def canonical_bytes(fmt: int, N: int, K: int) -> int:
@@ -66,8 +73,7 @@ def quantize(fmt: int, w: np.ndarray, chunk_rows: int = 4096) -> np.ndarray:
     assert K % BLOCK == 0
     nb = K // BLOCK
     bb = BLOCK_BYTES[fmt]
-    qmax = np.float32(7 if fmt == Q4 else 127)
-    qmin = np.float32(-8 if fmt == Q4 else -127)
+    qmin, qmax = (np.float32(v) for v in QRANGE[fmt])
     out = np.empty((N * nb, bb), dtype=np.uint8)
     for r0 in range(0, N, chunk_rows):
         r1 = min(N, r0 + chunk_rows)
@@ -83,12 +89,29 @@ def quantize(fmt: int, w: np.ndarray, chunk_rows: int = 4096) -> np.ndarray:
         qi = q.astype(np.int8)
         o = out[r0 * nb:r1 * nb]
         o[:, 0:2] = d.view(np.uint16).astype("<u2").view(np.uint8).reshape(-1, 2)
-        if fmt == Q4:
-            u = (qi + 8).astype(np.uint8)
-            o[:, 2:] = u[:, 0::2] | (u[:, 1::2] << 4)
-        else:
-            o[:, 2:] = qi.view(np.uint8)
+        _store_codes(fmt, o, qi)
     return out.reshape(-1)
+
+
+def _store_codes(fmt: int, o: np.ndarray, q: np.ndarray) -> None:
+    """Write integer codes q [blocks, 32] into the code bytes of canonical blocks o [blocks, block bytes]."""
+    if fmt == Q8:
+        o[:, 2:] = q.astype(np.int8).view(np.uint8)
+        return
+    u = (q.astype(np.int16) - QRANGE[fmt][0]).astype(np.uint8)               # offset binary
+    lo = u & 15
+    nib = lo[:, 0::2] | (lo[:, 1::2] << 4)
+    if fmt == Q4:
+        o[:, 2:] = nib
+    elif fmt == Q5:
+        bit = (u >> 4).astype(np.uint32)
+        word = (bit << np.arange(32, dtype=np.uint32)[None, :]).sum(axis=1, dtype=np.uint32)
+        o[:, 2:6] = word.astype("<u4").view(np.uint8).reshape(-1, 4)
+        o[:, 6:] = nib
+    else:
+        two = (u >> 4).reshape(-1, 8, 4)
+        o[:, 2:10] = (two[:, :, 0] | (two[:, :, 1] << 2) | (two[:, :, 2] << 4) | (two[:, :, 3] << 6)).astype(np.uint8)
+        o[:, 10:] = nib
 
 
 def blocks_from_codes(fmt: int, scales_bits: np.ndarray, codes: np.ndarray) -> np.ndarray:
@@ -99,13 +122,9 @@ def blocks_from_codes(fmt: int, scales_bits: np.ndarray, codes: np.ndarray) -> n
     codes = np.asarray(codes).reshape(N * nb, BLOCK)
     out = np.empty((N * nb, BLOCK_BYTES[fmt]), dtype=np.uint8)
     out[:, 0:2] = scales_bits.reshape(-1).astype("<u2").view(np.uint8).reshape(-1, 2)
-    if fmt == Q4:
-        assert codes.min() >= -8 and codes.max() <= 7
-        u = (codes + 8).astype(np.uint8)
-        out[:, 2:] = u[:, 0::2] | (u[:, 1::2] << 4)
-    else:
-        assert codes.min() >= -128 and codes.max() <= 127
-        out[:, 2:] = codes.astype(np.int8).view(np.uint8)
+    lo, hi = (-128, 127) if fmt == Q8 else QRANGE[fmt]
+    assert codes.min() >= lo and codes.max() <= hi
+    _store_codes(fmt, out, codes)
     return out.reshape(-1)
 
 

@@ -17,7 +17,10 @@ from paper_2607_00501_b200 import synth
 from tests import npref
 
 GOLD = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "handbuilt.json")))
-Q4, Q8 = 4, 8
+Q4, Q5, Q6, Q8 = 4, 5, 6, 8
+FMTS = [Q4, Q5, Q6, Q8]
+QLO = {Q4: -8, Q5: -16, Q6: -32, Q8: -128}      # lowest code a block can hold
+QMAX = {Q4: 7, Q5: 15, Q6: 31, Q8: 127}
 
 
 def bits16(x):
@@ -108,6 +111,45 @@ def test_v2_q8_block(oracle):
     assert y[0] == g["x_iota"]["y"] and B[0] == g["x_iota"]["sum_abs"]
 
 
+@pytest.mark.parametrize("fmt,key,step", [(Q5, "V7_q5_block", 1), (Q6, "V8_q6_block", 2)])
+def test_v7_v8_q5_q6_blocks_bytes_and_products(oracle, fmt, key, step):
+    """Hand-typed bytes of a 5-bit and a 6-bit block: where the low nibbles and the high bits sit, the
+    offset, and the products the block gives with x = ones and x_i = i (derivations in the fixture)."""
+    g = GOLD[key]
+    raw = np.frombuffer(bytes.fromhex(g["canonical_hex"]), dtype=np.uint8)
+    assert raw.size == {Q5: 22, Q6: 26}[fmt]
+    d = float(np.array([bits16(g["scale_bits"])], dtype=np.uint16).view(np.float16)[0])
+    q = step * np.arange(32) - (16 if fmt == Q5 else 32)
+    assert oracle.dequant(fmt, raw, 1, 32)[0].tolist() == [d * v for v in q.tolist()]
+    # the block builders produce the same bytes from the codes
+    assert synth.blocks_from_codes(fmt, np.array([[bits16(g["scale_bits"])]], dtype=np.uint16), q.reshape(1, 32)).tobytes().hex() == g["canonical_hex"]
+    y, B = oracle.gemv(fmt, raw, 1, 32, np.ones(32, dtype=np.float16))
+    assert y[0] == g["x_ones"]["y"] and B[0] == g["x_ones"]["sum_abs"]
+    y, B = oracle.gemv(fmt, raw, 1, 32, np.arange(32, dtype=np.float16))
+    assert y[0] == g["x_iota"]["y"] and B[0] == g["x_iota"]["sum_abs"]
+
+
+def test_v8_q6_extreme_codes(oracle):
+    g = GOLD["V8_q6_block"]["extremes"]
+    raw = np.frombuffer(bytes.fromhex(g["hex"]), dtype=np.uint8)
+    w = oracle.dequant(Q6, raw, 1, 32)[0]
+    assert w[0] == g["w0"] and w[1] == g["w1"] and w[31] == g["w31"]
+    assert np.all(w[2:31] == -32.0)
+
+
+@pytest.mark.parametrize("fmt,key", [(Q5, "q5"), (Q6, "q6")])
+def test_v9_q5_q6_ties_to_even(oracle, fmt, key):
+    g = GOLD["V9_q5_q6_ties"][key]
+    d = float(np.array([bits16(g["scale_bits"])], dtype=np.uint16).view(np.float16)[0])
+    w = np.zeros((1, 32), dtype=np.float32)
+    w[0, :len(g["w_over_half_step"])] = np.array(g["w_over_half_step"], dtype=np.float32) * np.float32(d / 2)
+    for name, quant in _quantisers(oracle):
+        blk = quant(fmt, w)
+        assert npref.scales_bits(fmt, blk, 1, 32)[0, 0] == bits16(g["scale_bits"]), name
+        assert npref.codes(fmt, blk, 1, 32)[0, :len(g["codes"])].tolist() == g["codes"], name
+        assert not npref.codes(fmt, blk, 1, 32)[0, len(g["codes"]):].any(), name
+
+
 def test_q8_minus128_decodes(oracle):
     q = np.full((1, 32), -128)
     blk = synth.blocks_from_codes(Q8, np.array([[0x3C00]], dtype=np.uint16), q)
@@ -166,14 +208,14 @@ def test_zero_block_quantises_to_zero(oracle):
             assert not npref.scales_bits(fmt, blk, 2, 64).any(), name
 
 
-@pytest.mark.parametrize("fmt", [Q4, Q8])
+@pytest.mark.parametrize("fmt", FMTS)
 def test_two_quantisers_agree_bit_for_bit(oracle, fmt):
     w = synth.weights(77, fmt, 96, 256)
     w[3, 5] = 0.31      # an outlier block
     assert np.array_equal(oracle.quantize(fmt, w), synth.quantize(fmt, w))
 
 
-@pytest.mark.parametrize("fmt", [Q4, Q8])
+@pytest.mark.parametrize("fmt", FMTS)
 def test_roundtrip_within_half_step(oracle, fmt):
     w = synth.weights(5, fmt, 64, 512)
     blk = oracle.quantize(fmt, w)
@@ -182,7 +224,7 @@ def test_roundtrip_within_half_step(oracle, fmt):
     step = np.repeat(d, 32, axis=1)
     assert np.all(np.abs(w.astype(np.float64) - wq) <= step / 2 * (1 + 2.0**-10))
     c = npref.codes(fmt, blk, 64, 512).reshape(64, 16, 32)
-    qmax = 7 if fmt == Q4 else 127
+    qmax = QMAX[fmt]
     assert np.all(np.abs(c).max(axis=2) == qmax)        # the arg-max element gets +-QMAX
     assert c.min() >= -qmax                              # this quantiser never emits the lowest code
 
@@ -198,7 +240,7 @@ def test_dequant_product_is_exact_in_fp32():
 
 # ------------------------------------------------------------------ products
 
-@pytest.mark.parametrize("fmt", [Q4, Q8])
+@pytest.mark.parametrize("fmt", FMTS)
 def test_dequant_matches_independent_decoder(oracle, fmt):
     N, K = 48, 160
     w = synth.weights(9, fmt, N, K)
@@ -206,11 +248,11 @@ def test_dequant_matches_independent_decoder(oracle, fmt):
     assert np.array_equal(oracle.dequant(fmt, blk, N, K).astype(np.float64), npref.decode(fmt, blk, N, K))
 
 
-@pytest.mark.parametrize("fmt", [Q4, Q8])
+@pytest.mark.parametrize("fmt", FMTS)
 @pytest.mark.parametrize("N,K,M", [(32, 32, 1), (64, 96, 3), (96, 64, 5)])
 def test_gemm_matches_brute_force_loops(oracle, fmt, N, K, M):
     rng = np.random.default_rng(N * 1000 + K + M + fmt)
-    codes = rng.integers(-8 if fmt == Q4 else -127, 8 if fmt == Q4 else 128, size=(N, K))
+    codes = rng.integers(QLO[fmt], QMAX[fmt] + 1, size=(N, K))
     sb = rng.integers(0x1800, 0x3000, size=(N, K // 32)).astype(np.uint16)
     sb[0, 0] |= 0x8000                                  # one negative scale
     blk = synth.blocks_from_codes(fmt, sb, codes)
@@ -228,12 +270,12 @@ def test_gemm_matches_brute_force_loops(oracle, fmt, N, K, M):
             assert Y[m, n] == s and B[m, n] == a
 
 
-@pytest.mark.parametrize("fmt", [Q4, Q8])
+@pytest.mark.parametrize("fmt", FMTS)
 def test_unit_scales_reduce_to_integer_matmul(oracle, fmt):
     # scales = 1.0, small integer activations: the product is an integer matrix product.
     rng = np.random.default_rng(11 + fmt)
     N, K, M = 64, 128, 4
-    codes = rng.integers(-8 if fmt == Q4 else -127, 8 if fmt == Q4 else 128, size=(N, K))
+    codes = rng.integers(QLO[fmt], QMAX[fmt] + 1, size=(N, K))
     blk = synth.blocks_from_codes(fmt, np.full((N, K // 32), 0x3C00, dtype=np.uint16), codes)
     Xi = rng.integers(-4, 5, size=(M, K))
     Y, B = oracle.gemm(fmt, blk, N, K, Xi.astype(np.float16))
@@ -241,7 +283,7 @@ def test_unit_scales_reduce_to_integer_matmul(oracle, fmt):
     assert np.array_equal(B, (np.abs(Xi) @ np.abs(codes).T).astype(np.float64))
 
 
-@pytest.mark.parametrize("fmt", [Q4, Q8])
+@pytest.mark.parametrize("fmt", FMTS)
 def test_gemm_matches_numpy_float64_matmul(oracle, fmt):
     N, K, M = 128, 512, 7
     blk = oracle.quantize(fmt, synth.weights(21, fmt, N, K))
@@ -254,7 +296,7 @@ def test_gemm_matches_numpy_float64_matmul(oracle, fmt):
     assert np.allclose(B, Bn, rtol=1e-12, atol=0)
 
 
-@pytest.mark.parametrize("fmt", [Q4, Q8])
+@pytest.mark.parametrize("fmt", FMTS)
 def test_gemv_invariants(oracle, fmt):
     N, K = 64, 256
     blk = oracle.quantize(fmt, synth.weights(31, fmt, N, K))
@@ -404,7 +446,7 @@ from hypothesis import assume, given, settings, strategies as st  # noqa: E402
 
 @settings(max_examples=60, deadline=None)
 @given(st.lists(st.floats(min_value=-4.0, max_value=4.0, allow_nan=False, width=32), min_size=32, max_size=32),
-       st.sampled_from([Q4, Q8]))
+       st.sampled_from(FMTS))
 def test_property_quantise_block_roundtrip(oracle, vals, fmt):
     w = np.array(vals, dtype=np.float32).reshape(1, 32)
     blk = oracle.quantize(fmt, w)
