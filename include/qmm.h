@@ -44,6 +44,16 @@
  *     element i of the block has code q_i in [-8, 7] stored as u_i = q_i + 8,
  *     qs[j] = u_{2j} | (u_{2j+1} << 4).
  *   Q8 block, 34 bytes: uint16 d, int8 qs[32] (two's complement).
+ *   Q5 block, 22 bytes: uint16 d, uint8 qh[4], uint8 qs[16]; code q_i in
+ *     [-16, 15] stored as u_i = q_i + 16: qs as in Q4 with u_i & 15, bit i of the
+ *     little-endian 32-bit word qh = u_i >> 4.
+ *   Q6 block, 26 bytes: uint16 d, uint8 qh[8], uint8 ql[16]; code q_i in
+ *     [-32, 31] stored as u_i = q_i + 32: ql as in Q4 with u_i & 15, bits
+ *     2 (i % 4), 2 (i % 4) + 1 of qh[i / 4] = u_i >> 4.
+ *   (The paper's kernel library spans 2-bit to 16-bit formats, Sec. 3.3 and
+ *   Sec. 4.1; Q5 and Q6 are built for qmm_pack, qmm_dequant, qmm_packed_check,
+ *   qmm_gemv, qmm_gemv_static and qmm_gemm -- every other call returns
+ *   QMM_ERR_UNSUPPORTED for them.)
  *   Row n of W holds K/32 consecutive blocks; rows are consecutive; block b of
  *   row n covers k in [32 b, 32 b + 32).  Weight value: float(d) * q (exact in
  *   fp32).  Scales must be finite.
@@ -84,7 +94,7 @@ typedef enum {
     QMM_ERR_BAD_WEIGHTS = 8    /* qmm_packed_check: not a packed buffer of that format  */
 } qmm_status;
 
-typedef enum { QMM_Q4 = 4, QMM_Q8 = 8 } qmm_format;
+typedef enum { QMM_Q4 = 4, QMM_Q5 = 5, QMM_Q6 = 6, QMM_Q8 = 8 } qmm_format;
 
 /* Description of the last failure on the calling thread.  Points into a static
  * thread-local buffer (Sec. 3.2: error handling without allocation); never
@@ -95,8 +105,8 @@ const char* qmm_last_error(void);
  * reached through a versioned C API, Sec. 3).                               */
 int qmm_version(void);
 
-/* Bytes of the canonical block stream for W[N,K]: N * (K/32) * 18 (Q4) or
- * * 34 (Q8).  0 if the arguments are invalid.  (Size queries exist so that the
+/* Bytes of the canonical block stream for W[N,K]: N * (K/32) * 18 (Q4), 22
+ * (Q5), 26 (Q6) or 34 (Q8).  0 if the arguments are invalid.  (Size queries exist so that the
  * caller can allocate everything up front and the hot path allocates
  * nothing, Sec. 3.2.)                                                       */
 size_t qmm_canonical_bytes(qmm_format fmt, int64_t N, int64_t K);

@@ -56,7 +56,15 @@ qmm_status chain_run(const qmm_chain_info* info, cudaStream_t stream);
 
 DebugKnobs g_knobs = {};
 
-static bool fmt_ok(int fmt) { return fmt == QMM_Q4 || fmt == QMM_Q8; }
+static bool fmt_ok(int fmt) { return fmt == QMM_Q4 || fmt == QMM_Q5 || fmt == QMM_Q6 || fmt == QMM_Q8; }
+
+// Q5 and Q6 are built for pack / dequant / check, the single GEMV and the dense GEMM only.
+static qmm_status check_fmt_everywhere(const char* who, int fmt)
+{
+    if (fmt == QMM_Q5 || fmt == QMM_Q6)
+        return fail(QMM_ERR_UNSUPPORTED, "%s: format %d is built for qmm_pack, qmm_dequant, qmm_packed_check, qmm_gemv and qmm_gemm only", who, fmt);
+    return QMM_OK;
+}
 
 static bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
@@ -85,7 +93,7 @@ static qmm_status check_device(const char* who)
 // Shape rules shared by every call that takes a packed matrix.
 static qmm_status check_matrix(const char* who, int fmt, int64_t N, int64_t K)
 {
-    if (!fmt_ok(fmt)) return fail(QMM_ERR_INVALID_ARG, "%s: unknown format %d (expected 4 or 8)", who, fmt);
+    if (!fmt_ok(fmt)) return fail(QMM_ERR_INVALID_ARG, "%s: unknown format %d (expected 4, 5, 6 or 8)", who, fmt);
     if (N <= 0 || K <= 0) return fail(QMM_ERR_INVALID_ARG, "%s: N=%lld and K=%lld must be positive", who, (long long)N, (long long)K);
     if (K % 32) return fail(QMM_ERR_SHAPE, "%s: K=%lld is not a multiple of the block size 32", who, (long long)K);
     if (K % 256) return fail(QMM_ERR_UNSUPPORTED, "%s: K=%lld is not a multiple of 256", who, (long long)K);
@@ -108,7 +116,7 @@ int qmm_version(void) { return 100; }
 size_t qmm_canonical_bytes(qmm_format fmt, int64_t N, int64_t K)
 {
     if (!fmt_ok(fmt) || N <= 0 || K <= 0 || K % 32) return 0;
-    return (size_t)N * (size_t)(K / 32) * (fmt == QMM_Q4 ? 18u : 34u);
+    return (size_t)N * (size_t)(K / 32) * (size_t)canon_block_of(fmt);
 }
 
 size_t qmm_packed_bytes(qmm_format fmt, int64_t N, int64_t K)
@@ -169,6 +177,7 @@ qmm_status qmm_gemv_gate_up(qmm_format fmt, const void* packed_gate, const void*
 {
     qmm_status s = check_matrix("qmm_gemv_gate_up", fmt, N, K);
     if (s != QMM_OK) return s;
+    if ((s = check_fmt_everywhere("qmm_gemv_gate_up", fmt)) != QMM_OK) return s;
     if (!packed_gate || !packed_up || !x_fp16 || !h_fp16) return fail(QMM_ERR_INVALID_ARG, "qmm_gemv_gate_up: null pointer");
     if (!aligned(packed_gate, 32) || !aligned(packed_up, 32))
         return fail(QMM_ERR_ALIGNMENT, "qmm_gemv_gate_up: packed matrices must be 32-byte aligned");
@@ -184,6 +193,7 @@ qmm_status qmm_gemv_batch(qmm_format fmt, const qmm_gemv_problem* problems, int 
     if (count < 0) return fail(QMM_ERR_INVALID_ARG, "qmm_gemv_batch: count=%d is negative", count);
     if (count == 0) return QMM_OK;
     if (!problems) return fail(QMM_ERR_INVALID_ARG, "qmm_gemv_batch: null problem list");
+    if (fmt_ok(fmt) && check_fmt_everywhere("qmm_gemv_batch", fmt) != QMM_OK) return QMM_ERR_UNSUPPORTED;
     for (int i = 0; i < count; ++i) {
         const qmm_gemv_problem& q = problems[i];
         qmm_status s = check_matrix("qmm_gemv_batch", fmt, q.N, q.K);
@@ -239,6 +249,7 @@ static qmm_status check_moe(const char* who, const qmm_moe_args* a)
         return fail(QMM_ERR_UNSUPPORTED, "%s: T*topk=%lld > 2^22", who, (long long)a->T * a->topk);
     qmm_status s = check_matrix(who, a->fmt, a->I, a->H);
     if (s != QMM_OK) return s;
+    if ((s = check_fmt_everywhere(who, a->fmt)) != QMM_OK) return s;
     return check_matrix(who, a->fmt, a->H, a->I);
 }
 

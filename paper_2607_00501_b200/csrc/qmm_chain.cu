@@ -479,6 +479,7 @@ struct ChainLayout {
 
 static qmm_status check_stages(const char* who, int fmt, const qmm_chain_stage* st, int count)
 {
+    if (fmt == QMM_Q5 || fmt == QMM_Q6) return fail(QMM_ERR_UNSUPPORTED, "%s: format %d is not built for this call", who, fmt);
     if (fmt != QMM_Q4 && fmt != QMM_Q8) return fail(QMM_ERR_INVALID_ARG, "%s: unknown format %d", who, fmt);
     if (!st || count <= 0) return fail(QMM_ERR_INVALID_ARG, "%s: empty stage list", who);
     if (count > 4096) return fail(QMM_ERR_UNSUPPORTED, "%s: %d stages > 4096", who, count);

@@ -38,20 +38,54 @@ constexpr int kQ8TileBytes = 1088;
 constexpr int kTileCodeBytes = 1024;
 constexpr int kNumSMs = 148;
 
+//   Q5 / Q6 tile = 64 weights per row, as Q4 plus a plane of high bits between codes and scales:
+//     [32 rows][32 B low nibbles]  exactly the Q4 code layout, holding u & 15 (u = q + 16 / q + 32);
+//     [32 rows][8 B] (Q5) / [32 rows][16 B] (Q6)  high bits.  Q5: two 32-bit words per row, word b for the
+//                            packed words 4b .. 4b+3; the pair p of packed word j (elements 8j+2p, 8j+2p+1)
+//                            has its fifth bits at bit t = 4 (j mod 4) + p and 16 + t, so one shift and a
+//                            mask 0x00010001 << s drops them beside the low nibbles of both half-words.
+//                            Q6: four words per row, word h for the packed words 2h, 2h+1; the pair's
+//                            2-bit fields at bits 2t', 2t'+1 and 16 + 2t', t' = 4 (j mod 2) + p;
+//     [32 rows][2 x fp16]    scales.                       Q5: 1408 bytes, Q6: 1664 bytes per tile.
+constexpr int kQ5TileBytes = 1408;
+constexpr int kQ6TileBytes = 1664;
+
 template <int FMT> struct Fmt;
 template <> struct Fmt<QMM_Q4> {
     static constexpr int tile_k = kQ4TileK;
     static constexpr int tile_bytes = kQ4TileBytes;
     static constexpr int canon_block = 18;
+    static constexpr int hi_bytes = 0;                       // bytes of high bits per row and tile
+    static constexpr int scale_off = kTileCodeBytes;         // offset of the scale plane in a tile
+};
+template <> struct Fmt<QMM_Q5> {
+    static constexpr int tile_k = 64;
+    static constexpr int tile_bytes = kQ5TileBytes;
+    static constexpr int canon_block = 22;
+    static constexpr int hi_bytes = 8;
+    static constexpr int scale_off = kTileCodeBytes + 32 * 8;
+};
+template <> struct Fmt<QMM_Q6> {
+    static constexpr int tile_k = 64;
+    static constexpr int tile_bytes = kQ6TileBytes;
+    static constexpr int canon_block = 26;
+    static constexpr int hi_bytes = 16;
+    static constexpr int scale_off = kTileCodeBytes + 32 * 16;
 };
 template <> struct Fmt<QMM_Q8> {
     static constexpr int tile_k = kQ8TileK;
     static constexpr int tile_bytes = kQ8TileBytes;
     static constexpr int canon_block = 34;
+    static constexpr int hi_bytes = 0;
+    static constexpr int scale_off = kTileCodeBytes;
 };
 
-__host__ __device__ inline int tile_k_of(int fmt) { return fmt == QMM_Q4 ? kQ4TileK : kQ8TileK; }
-__host__ __device__ inline int tile_bytes_of(int fmt) { return fmt == QMM_Q4 ? kQ4TileBytes : kQ8TileBytes; }
+__host__ __device__ inline int tile_k_of(int fmt) { return fmt == QMM_Q8 ? kQ8TileK : 64; }
+__host__ __device__ inline int tile_bytes_of(int fmt)
+{
+    return fmt == QMM_Q4 ? kQ4TileBytes : fmt == QMM_Q5 ? kQ5TileBytes : fmt == QMM_Q6 ? kQ6TileBytes : kQ8TileBytes;
+}
+__host__ __device__ inline int canon_block_of(int fmt) { return fmt == QMM_Q4 ? 18 : fmt == QMM_Q5 ? 22 : fmt == QMM_Q6 ? 26 : 34; }
 
 // Host-side error reporting (thread-local buffer; see qmm_api.cu).
 qmm_status fail(qmm_status code, const char* fmt, ...);
@@ -168,6 +202,31 @@ __device__ __forceinline__ void q4_word_to_h2(uint32_t w, __half2 (&q)[4], const
     q[1] = __hfma2(as_h2(and_or(w, k.mask_hi, k.magic)), c16th, cm72);
     q[2] = __hsub2(as_h2(and_or(w8, k.mask_lo, k.magic)), c1032);
     q[3] = __hfma2(as_h2(and_or(w8, k.mask_hi, k.magic)), c16th, cm72);
+}
+
+// Q5 / Q6: the four element pairs of packed word `j` of a tile as exact integers q in fp16.  `H` is the
+// high-bit word that covers word j (see the layout above); the pair's high bits are shifted beside
+// its low nibbles -- bit 4 (5) for the pairs taken with mask_lo, bit 8 (9) for those taken with mask_hi,
+// whose value is then divided by 16 like the nibble -- and merged with one more LOP3.
+// 0x6400 | u is 1024 + u: (1024 + u) - (1024 + OFF) = q, (1024 + 16 u) / 16 - (64 + OFF) = q, OFF = 16 / 32.
+template <int FMT>
+__device__ __forceinline__ void q56_word_to_h2(uint32_t w, uint32_t H, int j, __half2 (&q)[4], const Q4Consts& k)
+{
+    constexpr bool Q5 = FMT == QMM_Q5;
+    const __half2 c_lo = as_h2(Q5 ? 0x64106410u : 0x64206420u);          // 1040 / 1056
+    const __half2 c16th = as_h2(0x2C002C00u);
+    const __half2 c_hi = as_h2(Q5 ? 0xD500D500u : 0xD600D600u);          // -80 / -96
+    const uint32_t m_lo = Q5 ? 0x00100010u : 0x00300030u, m_hi = Q5 ? 0x01000100u : 0x03000300u;
+    const uint32_t w8 = w >> 8;
+    auto hi_at = [&](int p, int target) -> uint32_t {                      // the pair's high bits moved to bit `target`
+        const int from = Q5 ? 4 * (j & 3) + p : 2 * (4 * (j & 1) + p);
+        const int s = from - target;                                       // a constant once the callers' loops are unrolled
+        return s >= 0 ? H >> s : H << -s;
+    };
+    q[0] = __hsub2(as_h2(and_or(hi_at(0, 4), m_lo, and_or(w, k.mask_lo, k.magic))), c_lo);
+    q[1] = __hfma2(as_h2(and_or(hi_at(1, 8), m_hi, and_or(w, k.mask_hi, k.magic))), c16th, c_hi);
+    q[2] = __hsub2(as_h2(and_or(hi_at(2, 4), m_lo, and_or(w8, k.mask_lo, k.magic))), c_lo);
+    q[3] = __hfma2(as_h2(and_or(hi_at(3, 8), m_hi, and_or(w8, k.mask_hi, k.magic))), c16th, c_hi);
 }
 
 // Q8: the two element pairs of one packed word (4 offset-binary bytes) as

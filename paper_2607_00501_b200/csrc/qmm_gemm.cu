@@ -103,6 +103,16 @@ qmm_status launch_tc_gemm(int fmt, int bn, int na, int epi, bool dense, const CU
     QMM_TC_FMT(QMM_Q4)
     QMM_TC_FMT(QMM_Q8)
 #undef QMM_TC_FMT
+#define QMM_TC_DENSE_ONLY(F)                     \
+    QMM_TC_CASE(F, 32, 1, kEpiStore, true)       \
+    QMM_TC_CASE(F, 64, 1, kEpiStore, true)       \
+    QMM_TC_CASE(F, 128, 1, kEpiStore, true)      \
+    QMM_TC_CASE(F, 160, 1, kEpiStore, true)      \
+    QMM_TC_CASE(F, 192, 1, kEpiStore, true)      \
+    QMM_TC_CASE(F, 256, 1, kEpiStore, true)
+    QMM_TC_DENSE_ONLY(QMM_Q5)                     // the 5- and 6-bit formats: dense product only
+    QMM_TC_DENSE_ONLY(QMM_Q6)
+#undef QMM_TC_DENSE_ONLY
 #undef QMM_TC_CASE
     return fail(QMM_ERR_UNSUPPORTED, "no tensor-core kernel for fmt=%d bn=%d na=%d epi=%d dense=%d", fmt, bn, na, epi, (int)dense);
 }

@@ -170,6 +170,34 @@ template <> struct RawRow64<QMM_Q4> {
         }
     }
 };
+// Q5 / Q6: the Q4 slice plus the row's high-bit words.
+template <int FMT> struct RawRow64_56 {
+    u32x8 c;
+    uint32_t hi[Fmt<FMT>::hi_bytes / 4];
+    uint32_t sc;
+    __device__ __forceinline__ void load(const uint8_t* tile_ptr, int lane)
+    {
+        c = ld_keep_256(tile_ptr + 32 * lane);
+#pragma unroll
+        for (int i = 0; i < Fmt<FMT>::hi_bytes / 4; ++i) hi[i] = ld_nc_u32(tile_ptr + kTileCodeBytes + Fmt<FMT>::hi_bytes * lane + 4 * i);
+        sc = ld_nc_u32(tile_ptr + Fmt<FMT>::scale_off + 4 * lane);
+    }
+    __device__ __forceinline__ void expand(uint32_t (&out)[32], const Q4Consts& kc) const
+    {
+        const __half2 d0 = __half2half2(__low2half(as_h2(sc)));
+        const __half2 d1 = __half2half2(__high2half(as_h2(sc)));
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            __half2 q[4];
+            q56_word_to_h2<FMT>(c.v[j], hi[FMT == QMM_Q5 ? j / 4 : j / 2], j, q, kc);
+            const __half2 d = j < 4 ? d0 : d1;
+#pragma unroll
+            for (int p = 0; p < 4; ++p) out[4 * j + p] = as_u32(__hmul2(q[p], d));
+        }
+    }
+};
+template <> struct RawRow64<QMM_Q5> : RawRow64_56<QMM_Q5> {};
+template <> struct RawRow64<QMM_Q6> : RawRow64_56<QMM_Q6> {};
 template <> struct RawRow64<QMM_Q8> {
     u32x8 c[2];
     uint16_t sc[2];

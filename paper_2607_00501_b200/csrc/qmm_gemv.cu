@@ -49,6 +49,7 @@ __device__ __forceinline__ void cluster_sync()
 template <int FMT>
 struct TileRegs {
     u32x8 cp[kUnroll], cq[kUnroll];
+    typename HiRegs<FMT>::type hp[kUnroll], hq[kUnroll];          // high bits (Q5 / Q6 only)
     typename ScaleRegs<FMT>::type sp[kUnroll], sq[kUnroll];
 };
 
@@ -106,6 +107,8 @@ gemv_kernel(const uint8_t* __restrict__ packed, const uint16_t* __restrict__ x,
         const uint8_t* tq = tp + q_delta;
         r.cp[u] = ld_stream_256(tp);
         r.cq[u] = ld_stream_256(tq);
+        r.hp[u] = load_hi<FMT>(tp - 32 * lane, lane);
+        r.hq[u] = load_hi<FMT>(tq - 32 * lane, lane);
         r.sp[u] = load_scales<FMT>(tp - 32 * lane, lane);
         r.sq[u] = load_scales<FMT>(tq - 32 * lane, lane);
     };
@@ -133,12 +136,7 @@ gemv_kernel(const uint8_t* __restrict__ packed, const uint16_t* __restrict__ x,
 #pragma unroll
             for (int u = 0; u < kUnroll; ++u) {
                 const int tt = t + u * WARPS;
-                if (tt < t_end) {
-                    if constexpr (FMT == QMM_Q4)
-                        tile_pair_mma_q4(r.cp[u], r.cq[u], r.sp[u], r.sq[u], xb + tt * XV, acc, kc);
-                    else
-                        tile_pair_mma_q8(r.cp[u], r.cq[u], r.sp[u], r.sq[u], xb + tt * XV, acc);
-                }
+                if (tt < t_end) tile_pair_mma<FMT>(r.cp[u], r.cq[u], r.hp[u], r.hq[u], r.sp[u], r.sq[u], xb + tt * XV, acc, kc);
             }
             t += STEP;
             if (t < t_end) load_group();
@@ -1113,6 +1111,10 @@ qmm_status launch_gemv(int fmt, const void* packed, int64_t N, int64_t K, const 
     QMM_GEMV_CASE(QMM_Q4, 16)
     QMM_GEMV_CASE(QMM_Q8, 8)
     QMM_GEMV_CASE(QMM_Q8, 16)
+    QMM_GEMV_CASE(QMM_Q5, 8)
+    QMM_GEMV_CASE(QMM_Q5, 16)
+    QMM_GEMV_CASE(QMM_Q6, 8)
+    QMM_GEMV_CASE(QMM_Q6, 16)
 #undef QMM_GEMV_CASE
     return fail(QMM_ERR_UNSUPPORTED, "qmm_gemv: no kernel for this plan");
 }
@@ -1166,7 +1168,8 @@ extern "C" qmm_status qmm_gemv_static(qmm_format fmt, const void* packed, int64_
                                       const uint16_t* x_fp16, uint16_t* y_fp16, void* stream)
 {
     using namespace qmm;
-    if (fmt != QMM_Q4 && fmt != QMM_Q8) return fail(QMM_ERR_INVALID_ARG, "qmm_gemv_static: unknown format %d", (int)fmt);
+    if (fmt != QMM_Q4 && fmt != QMM_Q5 && fmt != QMM_Q6 && fmt != QMM_Q8)
+        return fail(QMM_ERR_INVALID_ARG, "qmm_gemv_static: unknown format %d", (int)fmt);
     if (N <= 0 || K <= 0) return fail(QMM_ERR_INVALID_ARG, "qmm_gemv_static: N=%lld and K=%lld must be positive", (long long)N, (long long)K);
     if (K % 32) return fail(QMM_ERR_SHAPE, "qmm_gemv_static: K=%lld is not a multiple of the block size 32", (long long)K);
     if (K % 256 || N % 128 || K > 32768 || N > (1 << 24))

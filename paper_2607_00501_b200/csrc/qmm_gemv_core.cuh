@@ -99,26 +99,91 @@ __device__ __forceinline__ void tile_pair_mma_q8(const u32x8& cp, const u32x8& c
     acc[3] = fmaf(__half2float(__high2half(as_h2(sq))), c[3], acc[3]);
 }
 
-template <int FMT> struct ScaleRegs;
-template <> struct ScaleRegs<QMM_Q4> { using type = uint2; };
+// Q5 / Q6: a Q4 tile pair with the high-bit words of the two rows (hp, hq) merged in while unpacking.
+template <int FMT, typename HI>
+__device__ __forceinline__ void tile_pair_mma_q56(const u32x8& cp, const u32x8& cq, const HI& hp, const HI& hq, uint2 sp, uint2 sq,
+                                                  const uint4* xt, float (&acc)[4], const Q4Consts& kc)
+{
+    const uint32_t* hpw = reinterpret_cast<const uint32_t*>(&hp);
+    const uint32_t* hqw = reinterpret_cast<const uint32_t*>(&hq);
+#pragma unroll
+    for (int b = 0; b < 2; ++b) {
+        float c[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int j = b * 4 + i;                             // packed word of the tile
+            const int hw = FMT == QMM_Q5 ? j / 4 : j / 2;        // the high-bit word that covers it
+            const uint4 xv = xt[j];                              // activations k = 8j .. 8j+7
+            __half2 p[4], q[4];
+            q56_word_to_h2<FMT>(cp.v[j], hpw[hw], j, p, kc);
+            q56_word_to_h2<FMT>(cq.v[j], hqw[hw], j, q, kc);
+            if (i == 0)
+                mma16816_zero(c, as_u32(p[0]), as_u32(q[0]), as_u32(p[1]), as_u32(q[1]), xv.x, xv.y);
+            else
+                mma16816(c, as_u32(p[0]), as_u32(q[0]), as_u32(p[1]), as_u32(q[1]), xv.x, xv.y);
+            mma16816(c, as_u32(p[2]), as_u32(q[2]), as_u32(p[3]), as_u32(q[3]), xv.z, xv.w);
+        }
+        const float dp0 = __half2float(b ? __high2half(as_h2(sp.x)) : __low2half(as_h2(sp.x)));
+        const float dp1 = __half2float(b ? __high2half(as_h2(sp.y)) : __low2half(as_h2(sp.y)));
+        const float dq0 = __half2float(b ? __high2half(as_h2(sq.x)) : __low2half(as_h2(sq.x)));
+        const float dq1 = __half2float(b ? __high2half(as_h2(sq.y)) : __low2half(as_h2(sq.y)));
+        acc[0] = fmaf(dp0, c[0], acc[0]);
+        acc[1] = fmaf(dp1, c[1], acc[1]);
+        acc[2] = fmaf(dq0, c[2], acc[2]);
+        acc[3] = fmaf(dq1, c[3], acc[3]);
+    }
+}
+
+template <int FMT> struct ScaleRegs { using type = uint2; };
 template <> struct ScaleRegs<QMM_Q8> { using type = uint32_t; };
+
+// High-bit words of one row of a tile (Q5: 8 bytes, Q6: 16 bytes; nothing for Q4 / Q8).
+struct NoHi {};
+template <int FMT> struct HiRegs { using type = NoHi; };
+template <> struct HiRegs<QMM_Q5> { using type = uint2; };
+template <> struct HiRegs<QMM_Q6> { using type = uint4; };
+
+template <int FMT>
+__device__ __forceinline__ typename HiRegs<FMT>::type load_hi(const uint8_t* tile, int lane)
+{
+    if constexpr (FMT == QMM_Q5) {
+        uint2 r;
+        asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(r.x), "=r"(r.y) : "l"(tile + kTileCodeBytes + 8 * lane));
+        return r;
+    } else if constexpr (FMT == QMM_Q6) {
+        uint4 r;
+        asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                     : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+                     : "l"(tile + kTileCodeBytes + 16 * lane));
+        return r;
+    } else {
+        return NoHi{};
+    }
+}
+
+// One tile pair of any format.
+template <int FMT>
+__device__ __forceinline__ void tile_pair_mma(const u32x8& cp, const u32x8& cq, const typename HiRegs<FMT>::type& hp,
+                                              const typename HiRegs<FMT>::type& hq, typename ScaleRegs<FMT>::type sp,
+                                              typename ScaleRegs<FMT>::type sq, const uint4* xt, float (&acc)[4], const Q4Consts& kc)
+{
+    if constexpr (FMT == QMM_Q4) tile_pair_mma_q4(cp, cq, sp, sq, xt, acc, kc);
+    else if constexpr (FMT == QMM_Q8) tile_pair_mma_q8(cp, cq, sp, sq, xt, acc);
+    else tile_pair_mma_q56<FMT>(cp, cq, hp, hq, sp, sq, xt, acc, kc);
+}
 
 // Scales of rows 4g+2(t&1) and the next row of one tile (the rows whose sums this lane receives).
 template <int FMT>
-__device__ __forceinline__ typename ScaleRegs<FMT>::type load_scales(const uint8_t* tile, int lane);
-template <>
-__device__ __forceinline__ uint2 load_scales<QMM_Q4>(const uint8_t* tile, int lane)
+__device__ __forceinline__ typename ScaleRegs<FMT>::type load_scales(const uint8_t* tile, int lane)
 {
     const int row = (lane & ~3) + 2 * (lane & 1);
-    uint2 r;
-    asm volatile("ld.global.nc.v2.u32 {%0,%1}, [%2];" : "=r"(r.x), "=r"(r.y) : "l"(tile + kTileCodeBytes + 4 * row));
-    return r;
-}
-template <>
-__device__ __forceinline__ uint32_t load_scales<QMM_Q8>(const uint8_t* tile, int lane)
-{
-    const int row = (lane & ~3) + 2 * (lane & 1);
-    return ld_nc_u32(tile + kTileCodeBytes + 2 * row);
+    if constexpr (FMT == QMM_Q8) {
+        return ld_nc_u32(tile + kTileCodeBytes + 2 * row);
+    } else {
+        uint2 r;
+        asm volatile("ld.global.nc.v2.u32 {%0,%1}, [%2];" : "=r"(r.x), "=r"(r.y) : "l"(tile + Fmt<FMT>::scale_off + 4 * row));
+        return r;
+    }
 }
 
 }  // namespace qmm

@@ -14,6 +14,8 @@ import threading
 import torch
 
 Q4 = 4
+Q5 = 5
+Q6 = 6
 Q8 = 8
 
 _HERE = os.path.dirname(os.path.abspath(__file__))

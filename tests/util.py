@@ -30,7 +30,7 @@ def random_blocks(synth, fmt, N, K, seed, special_scales=True, scale_bits=(0x140
     `scale_bits` (default ~ 2^-10 .. 0.25).  special_scales: True replaces one block in 16 by a
     negative, zero, subnormal or -0 scale; "no_subnormal" leaves the subnormal kind out."""
     rng = np.random.default_rng(seed)
-    lo, hi = (-8, 8) if fmt == 4 else (-128, 128)
+    lo, hi = {4: (-8, 8), 5: (-16, 16), 6: (-32, 32), 8: (-128, 128)}[fmt]
     codes = rng.integers(lo, hi, size=(N, K))
     sb = rng.integers(scale_bits[0], scale_bits[1], size=(N, K // 32)).astype(np.uint16)
     if special_scales:
