@@ -580,7 +580,7 @@ def extra_sections(args, qmm, torch, pk, ops, fmts, batch, gpu_index=0):
     # state = 300 distinct packed copies (531 MB, larger than L2) so that every product streams from HBM:
     # as 300 chained launches in one graph, and as qmm_gemv_batch launches over the same 300 problems.
     if not on("cfg0"):
-        return finish_sections(out, sampler) if not any(on(n) for n in ("lm_head", "ffn", "gemm", "moe")) else \
+        return finish_sections(out, sampler) if not any(on(n) for n in ("lm_head", "ffn", "gemm", "formats", "moe")) else \
             rest_of_sections(args, qmm, torch, pk, fmts, out, flush, dev, sampler, on)
     c = synth.CFG0
     copies = 300
@@ -674,6 +674,30 @@ def sections_ffn_on(args, qmm, torch, pk, fmts, out, flush, dev, sampler, on):
                                                   **tensor_fracs(tf, pk))
                 qmm.status_check(ws)
         out["prefill_gemm_q%d" % f] = gemm
+
+    # not configs: the 5-bit and 6-bit formats through the same two kernel families (one decode-sized
+    # GEMV on the LM-head shape, one prefill GEMM on the gate/up shape at M = 2048)
+    for f in ((synth.Q5, synth.Q6) if on("formats") else ()):
+        e = {}
+        N, K = synth.CFG2["N"], synth.CFG2["K"]
+        blocks = synth.quantize(f, synth.weights(synth.CFG2["seed"], 0, N, K))
+        packed = qmm.pack(f, dev(blocks), N, K)
+        x = dev(synth.activations(synth.CFG2["seed"], 1, K))
+        y = torch.empty(N, dtype=torch.float16, device="cuda")
+        m = measure(torch, lambda: qmm.gemv(f, packed, N, K, x, y=y), flush, iters=20)
+        e["lm_head_gemv"] = dict(m, **hbm_fracs(blocks.nbytes, m["ms"], pk))
+        _, N, K = synth.CFG3["shapes"][0]
+        M = 2048
+        blocks = synth.quantize(f, synth.weights(synth.CFG3["seed"], 0, N, K))
+        packed = qmm.pack(f, dev(blocks), N, K)
+        X = dev(synth.activations(synth.CFG3["seed"], 10 + M, M, K))
+        Y = torch.empty((M, N), dtype=torch.float16, device="cuda")
+        ws = torch.zeros(qmm.gemm_workspace_bytes(f, M, N, K), dtype=torch.uint8, device="cuda")
+        m = measure(torch, lambda: qmm.gemm(f, packed, N, K, X, Y=Y, ws=ws), flush)
+        qmm.status_check(ws)
+        e["gemm_gate_up_M2048"] = dict(m, **tensor_fracs(2.0 * M * N * K / m["ms"] / 1e9, pk))
+        out["format_q%d" % f] = e
+        del packed, blocks
 
     # cfg4: MoE layer (Q4 as the config says; Q8 at the largest T)
     c = synth.CFG4
@@ -897,7 +921,7 @@ def main():
     ap.add_argument("--streams", type=int, default=8, help="streams for --mode streams")
     ap.add_argument("--no-sections", action="store_true", help="skip the LM-head / GEMM / MoE sections")
     ap.add_argument("--sections", default=None,
-                    help="comma list of the sections to run (chain,chained,cfg0,lm_head,ffn,gemm,moe); default: all")
+                    help="comma list of the sections to run (chain,chained,cfg0,lm_head,ffn,gemm,formats,moe); default: all")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--case", default=None, help="profiling aid: run a few launches of one kernel and exit (see run_case)")
