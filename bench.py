@@ -412,6 +412,38 @@ def run_ours(args):
     value = whole_job_value(world, bytes_step, ms_per_step)
     e2e_value = whole_job_value(world, bytes_step, e2e_ms / args.steps)
 
+    # N > 1 only: strong scaling of ONE matrix -- the Q8 LM head with its rows spread over the ranks and
+    # an all-gather of the fp16 outputs (every rank ends with the whole vector in its own memory)
+    sharded_section = None
+    if world > 1 and not args.no_sections:
+        try:
+            from paper_2607_00501_b200 import sharded
+            c = synth.CFG2
+            r0, r1 = sharded.shard_rows(c["N"], world, rank)
+            full = synth.weights(c["seed"], 0, c["N"], c["K"])
+            per_row = (c["K"] // 32) * synth.BLOCK_BYTES[c["fmt"]]
+            blocks = np.zeros(c["N"] * per_row, dtype=np.uint8)          # only this rank's rows are quantised
+            blocks.reshape(c["N"], per_row)[r0:r1] = synth.quantize(c["fmt"], full[r0:r1]).reshape(r1 - r0, per_row)
+            del full
+            op = sharded.RowShardedGemv(c["fmt"], blocks, c["N"], c["K"], device="cuda")
+            xs = torch.from_numpy(synth.activations(c["seed"], 1, c["K"])).cuda()
+            for _ in range(3):
+                op(xs)
+            torch.cuda.synchronize()
+            dist.barrier()
+            s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            s0.record()
+            for _ in range(args.steps):
+                op(xs)
+            s1.record()
+            torch.cuda.synchronize()
+            ms, = max_over_ranks(dist, [s0.elapsed_time(s1) / args.steps], "cuda")
+            nbytes = synth.canonical_bytes(c["fmt"], c["N"], c["K"])
+            sharded_section = {"ms": round(ms, 4), "GBps_whole_matrix": round(nbytes / ms / 1e6, 1), "ranks": world,
+                               "scaling": "strong", "exchange": "all_gather of %d fp16 outputs" % c["N"]}
+        except Exception as ex:                                          # never lose the headline line to this section
+            sharded_section = {"error": repr(ex)[:300]}
+
     sections = {}
     cpu = None
     if rank == 0 and not args.no_sections:
@@ -447,7 +479,7 @@ def run_ours(args):
                      "kernel": "gemv_batch_kernel (both launches of the step)" if args.mode == "batch" else "gemv_kernel (all launches of the step)", "peak_source": pk["source"],
                      "step_ms_min": round(min(step_ms), 5), "step_ms_max": round(max(step_ms), 5)},
         "cpu_baseline": cpu,
-        "sections": sections,
+        "sections": dict(sections, **({"lm_head_q8_row_sharded": sharded_section} if sharded_section else {})),
     }
     print(json.dumps(line))
 

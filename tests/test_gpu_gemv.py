@@ -297,3 +297,17 @@ def test_cfg1_whole_stack_in_one_batch_as_benchmarked(qmm, oracle, fmt):
         y_ref, B = oracle.gemv(fmt, blocks, N, K, xh)
         worst = max(worst, util.assert_within_tol(util.host_f64(y), y_ref, B, "cfg1 stack, layer %d %s" % (layer, name)))
     assert worst > 0
+
+
+def test_row_sharded_gemv_on_one_rank_is_the_plain_product(qmm, oracle):
+    """Without a process group the sharded operator holds every row and no collective runs (the
+    two-rank form is tested with gloo on CPU)."""
+    from paper_2607_00501_b200 import sharded
+    N, K = 640, 1024
+    blocks = synth.quantize(Q8, synth.weights(99, 0, N, K))
+    x = synth.activations(99, 1, K)
+    op = sharded.RowShardedGemv(Q8, blocks, N, K)
+    assert (op.r0, op.r1, op.world) == (0, N, 1)
+    y = op(util.dev(x))
+    y_ref, B = oracle.gemv(Q8, blocks, N, K, x)
+    util.assert_within_tol(util.host_f64(y), y_ref, B, "sharded, one rank")

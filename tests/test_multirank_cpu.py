@@ -62,3 +62,42 @@ def test_bench_gpus_flag_starts_the_ranks_itself():
     d = json.loads(lines[0])
     assert d["dry_run"] and d["n_gpus"] == 2 and d["gpus_arg"] == 2
     assert d["ms_per_step"] == 2.0 and d["value"] == 2 * 1000 / 2e-3 / 1e9
+
+
+def _sharded_worker(rank, world, port, out_dir):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    import oracle
+    from paper_2607_00501_b200 import sharded, synth
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    res = {}
+    for fmt, N, K in ((4, 384, 256), (8, 512, 512), (6, 256, 256)):       # 384 rows: 3 row blocks over 2 ranks (uneven)
+        blocks = synth.quantize(fmt, synth.weights(77, fmt, N, K))
+        x = synth.activations(77, 100 + fmt, K)
+        # the local product on CPU: the oracle's fp64 result rounded to fp16 stands in for the GPU kernel
+        prep = lambda f, b, n, k, dev: b
+        prod = lambda f, b, n, k, xv: torch.from_numpy(oracle.gemv(f, b, n, k, xv.numpy())[0].astype(np.float16))
+        op = sharded.RowShardedGemv(fmt, blocks, N, K, device="cpu", prepare=prep, product=prod)
+        y = op(torch.from_numpy(x))
+        res["%d_%d_%d" % (fmt, N, K)] = {"rows": [op.r0, op.r1], "y": y.numpy().view(np.uint16).tolist()}
+    dist.barrier()
+    json.dump(res, open(os.path.join(out_dir, "s%d.json" % rank), "w"))
+    dist.destroy_process_group()
+
+
+def test_row_sharded_gemv_two_ranks_equals_single_rank(tmp_path):
+    """Two gloo ranks each hold half of W's rows, multiply and all-gather the fp16 outputs: every rank
+    ends with the whole y, bit-identical to the unsharded product (rows are independent)."""
+    import oracle
+    from paper_2607_00501_b200 import sharded, synth
+    world, port = 2, 31000 + os.getpid() % 2000
+    mp.spawn(_sharded_worker, args=(world, port, str(tmp_path)), nprocs=world, join=True)
+    r = [json.load(open(tmp_path / ("s%d.json" % i))) for i in range(world)]
+    for fmt, N, K in ((4, 384, 256), (8, 512, 512), (6, 256, 256)):
+        key = "%d_%d_%d" % (fmt, N, K)
+        blocks = synth.quantize(fmt, synth.weights(77, fmt, N, K))
+        x = synth.activations(77, 100 + fmt, K)
+        whole = oracle.gemv(fmt, blocks, N, K, x)[0].astype(np.float16).view(np.uint16).tolist()
+        assert r[0][key]["y"] == whole and r[1][key]["y"] == whole
+        assert r[0][key]["rows"][0] == 0 and r[0][key]["rows"][1] == r[1][key]["rows"][0] and r[1][key]["rows"][1] == N
+    assert sharded.shard_rows(384, 2, 0) == (0, 256) and sharded.shard_rows(384, 2, 1) == (256, 384)
+    assert sharded.shard_rows(128, 4, 3) == (128, 128)                     # more ranks than row blocks: an empty share
