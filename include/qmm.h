@@ -331,6 +331,12 @@ typedef struct {
     int32_t* expert_offsets;       /* [E+1]     optional                                */
     uint16_t* dbg_H;               /* [T*topk, I] fp16 in permuted row order, optional  */
     uint16_t* dbg_D;               /* [T*topk, H] fp16 in permuted row order, optional  */
+    /* Optional router product (decode-sized layers, T * topk <= 32, E % 128 == 0): when
+     * w_router is non-NULL the logits are computed by the library, logits[t, e] =
+     * sum_k W_router[e, k] * X[t, k] accumulated and kept in fp32 (one more fused launch
+     * of the decode step, Sec. 3.3), and `logits` above is ignored (may be NULL).     */
+    const void* w_router;          /* packed [E, H] matrix in format fmt, or NULL       */
+    float* router_logits;          /* [T, E] fp32, optional export of those logits      */
 } qmm_moe_args;
 
 /* Workspace size for these arguments (host pointer to args; only the sizes are

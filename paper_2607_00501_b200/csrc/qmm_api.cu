@@ -36,7 +36,7 @@ qmm_status launch_dequant(int fmt, const void* packed, int64_t N, int64_t K, flo
 size_t gemv_workspace_bytes(int fmt, int64_t N, int64_t K, bool allow_cluster);
 qmm_status launch_gemv(int fmt, const void* packed, int64_t N, int64_t K, const uint16_t* x, uint16_t* y,
                        void* ws, bool allow_cluster, cudaStream_t st);
-qmm_status launch_gemv_batch(int fmt, const qmm_gemv_problem* probs, int count, cudaStream_t st);
+qmm_status launch_gemv_batch(int fmt, const qmm_gemv_problem* probs, int count, cudaStream_t st, bool out_f32);
 qmm_status launch_gemv_gate_up(int fmt, const void* packed_gate, const void* packed_up, int64_t N, int64_t K,
                                const uint16_t* x, uint16_t* h, cudaStream_t st);
 size_t gemm_workspace_bytes(int fmt, int64_t M, int64_t N, int64_t K);
@@ -205,7 +205,7 @@ qmm_status qmm_gemv_batch(qmm_format fmt, const qmm_gemv_problem* problems, int 
     }
     qmm_status s = check_device("qmm_gemv_batch");
     if (s != QMM_OK) return s;
-    return launch_gemv_batch(fmt, problems, count, (cudaStream_t)stream);
+    return launch_gemv_batch(fmt, problems, count, (cudaStream_t)stream, false);
 }
 
 size_t qmm_gemm_workspace_bytes(qmm_format fmt, int64_t M, int64_t N, int64_t K)
@@ -264,7 +264,15 @@ static qmm_status moe_entry(const char* who, const qmm_moe_args* a, void* ws, si
     qmm_status s = check_moe(who, a);
     if (s != QMM_OK) return s;
     if (a->T == 0) return QMM_OK;                               // nothing to do: no tensor or workspace is touched
-    if (!a->logits) return fail(QMM_ERR_INVALID_ARG, "%s: logits is null", who);
+    if (!a->logits && !a->w_router) return fail(QMM_ERR_INVALID_ARG, "%s: logits and w_router are both null", who);
+    if (a->w_router) {
+        if (!a->X) return fail(QMM_ERR_INVALID_ARG, "%s: w_router needs X", who);
+        if (!aligned(a->w_router, 32) || !aligned(a->router_logits, 16))
+            return fail(QMM_ERR_ALIGNMENT, "%s: w_router must be 32-byte, router_logits 16-byte aligned", who);
+        if (a->E % 128) return fail(QMM_ERR_UNSUPPORTED, "%s: w_router needs E %% 128 == 0 (got %d)", who, a->E);
+        if ((int64_t)a->T * a->topk > 32 || a->T > 32)
+            return fail(QMM_ERR_UNSUPPORTED, "%s: the router product is built for decode-sized layers (T * topk <= 32)", who);
+    }
     if (!route_only && (!a->X || !a->w_gate || !a->w_up || !a->w_down || !a->out))
         return fail(QMM_ERR_INVALID_ARG, "%s: null tensor pointer", who);
     if (!aligned(a->logits, 16) || !aligned(a->X, 16) || !aligned(a->out, 16) || !aligned(a->w_gate, 32) ||

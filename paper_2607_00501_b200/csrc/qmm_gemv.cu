@@ -230,6 +230,7 @@ struct BatchParams {
     int count;
     int total_cost;
     int max_k;
+    int out_f32;      // != 0: the y pointers are float*: outputs stay fp32 (router logits)
     BatchProblem p[kMaxBatch];
 };
 
@@ -345,7 +346,10 @@ gemv_batch_kernel(const __grid_constant__ BatchParams bp)
             float sum = red[threadIdx.x];
 #pragma unroll
             for (int w = 1; w < WARPS; ++w) sum += red[w * 64 + threadIdx.x];
-            bp.p[done_p].y[done_u * 64 + threadIdx.x] = __half_as_ushort(__float2half_rn(sum));
+            if (bp.out_f32)
+                reinterpret_cast<float*>(bp.p[done_p].y)[done_u * 64 + threadIdx.x] = sum;
+            else
+                bp.p[done_p].y[done_u * 64 + threadIdx.x] = __half_as_ushort(__float2half_rn(sum));
         }
         if (have && pi != done_p)                               // next unit reads another activation vector
             for (int i = threadIdx.x; i < bp.p[pi].K / 8; i += WARPS * 32) xs[i] = reinterpret_cast<const uint4*>(bp.p[pi].x)[i];
@@ -1053,12 +1057,13 @@ qmm_status launch_moe_small(int fmt, const MoeSmallHost& h, bool route_only, cud
 }
 
 // Host side of qmm_gemv_batch: up to kMaxBatch problems per launch.
-qmm_status launch_gemv_batch(int fmt, const qmm_gemv_problem* probs, int count, cudaStream_t st)
+qmm_status launch_gemv_batch(int fmt, const qmm_gemv_problem* probs, int count, cudaStream_t st, bool out_f32)
 {
     for (int first = 0; first < count; first += kMaxBatch) {
         const int n = count - first < kMaxBatch ? count - first : kMaxBatch;
         BatchParams bp = {};
         bp.count = n;
+        bp.out_f32 = out_f32 ? 1 : 0;
         int cost = 0, max_k = 0;
         for (int i = 0; i < n; ++i) {
             const qmm_gemv_problem& q = probs[first + i];

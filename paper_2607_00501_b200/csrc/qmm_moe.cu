@@ -24,6 +24,7 @@ qmm_status launch_moe_gemv(int fmt, bool gate_up, const void* w0, const void* w1
 
 bool moe_small_supported(int T, int topk, int H, int I);
 qmm_status launch_moe_small(int fmt, const MoeSmallHost& h, bool route_only, cudaStream_t st);
+qmm_status launch_gemv_batch(int fmt, const qmm_gemv_problem* probs, int count, cudaStream_t st, bool out_f32);
 
 // Up to this many (token, expert) rows the expert products run as GEMVs (each row streams its expert's
 // matrices once); above it, as grouped tensor-core GEMMs (each expert's matrices are read once per layer).
@@ -34,7 +35,7 @@ dim3 persistent_grid(int bn, int na, int64_t tiles);
 
 struct MoeWorkspace {
     size_t status, counts, offsets, num_tiles, tile_expert, tile_row0, tile_rows;
-    size_t topk_idx, topk_w, perm, inv_perm, xp, hbuf, dbuf, trace, total;
+    size_t topk_idx, topk_w, perm, inv_perm, xp, hbuf, dbuf, trace, logits, total;
     int bn, max_tiles;
 };
 
@@ -62,6 +63,7 @@ static MoeWorkspace moe_layout(const qmm_moe_args* a)
     w.xp = take(rows * (size_t)a->H * 2);
     w.hbuf = take(rows * (size_t)a->I * 2);
     w.dbuf = take(rows * (size_t)a->H * 2);
+    w.logits = take(a->w_router ? (size_t)a->T * a->E * 4 : 0);   // router logits when the library computes them
     w.trace = take(4096);                                  // pipeline trace of the gate/up GEMM (tuning aid, QMM_GEMM_TRACE)
     w.total = o;
     return w;
@@ -338,6 +340,22 @@ qmm_status launch_moe(const qmm_moe_args* a, void* ws, bool route_only, cudaStre
     const int total = a->T * a->topk;
 
     cudaError_t e;
+    const float* logits = a->logits;
+    if (a->w_router) {
+        // router product: T independent GEMVs of the [E, H] router matrix, fp32 outputs, one launch
+        float* lg = a->router_logits ? a->router_logits : (float*)(base + w.logits);
+        qmm_gemv_problem probs[32];
+        for (int t = 0; t < a->T; ++t) {
+            probs[t].packed = a->w_router;
+            probs[t].x_fp16 = a->X + (size_t)t * a->H;
+            probs[t].y_fp16 = (uint16_t*)(lg + (size_t)t * a->E);
+            probs[t].N = a->E;
+            probs[t].K = a->H;
+        }
+        qmm_status s = launch_gemv_batch(a->fmt, probs, a->T, st, true);
+        if (s != QMM_OK) return s;
+        logits = lg;
+    }
     const int per_lane = (a->E + 31) / 32;
     // decode-sized: one block does steps 1-2 and the expert products run as GEMVs
     const bool small = total <= kMoeGemvMaxRows && a->T <= 32 && a->H <= 32768 && a->I <= 32768;
@@ -346,7 +364,7 @@ qmm_status launch_moe(const qmm_moe_args* a, void* ws, bool route_only, cudaStre
     if (small && !g_knobs.moe_no_fuse && moe_small_supported(a->T, a->topk, a->H, a->I)) {
         // decode: the whole layer in two launches (routing inside the gate/up launch, combine inside the down launch)
         MoeSmallHost h;
-        h.logits = a->logits; h.X = a->X; h.w_gate = a->w_gate; h.w_up = a->w_up; h.w_down = a->w_down;
+        h.logits = logits; h.X = a->X; h.w_gate = a->w_gate; h.w_up = a->w_up; h.w_down = a->w_down;
         h.gu_stride = (int64_t)gu_stride; h.dn_stride = (int64_t)dn_stride;
         h.hbuf = hbuf; h.dbg_D = a->dbg_D; h.out = a->out;
         h.T = a->T; h.E = a->E; h.topk = a->topk; h.H = a->H; h.I = a->I;
@@ -360,10 +378,10 @@ qmm_status launch_moe(const qmm_moe_args* a, void* ws, bool route_only, cudaStre
     }
     if (small) {
         if (per_lane <= 4)
-            e = launch_pdl(route_small_kernel<4>, dim3(1), dim3(1024), st, a->logits, (int)a->T, (int)a->E, (int)a->topk, topk_idx,
+            e = launch_pdl(route_small_kernel<4>, dim3(1), dim3(1024), st, logits, (int)a->T, (int)a->E, (int)a->topk, topk_idx,
                            topk_w, a->topk_idx, a->topk_w, offsets, a->expert_offsets, perm, a->perm, inv_perm);
         else
-            e = launch_pdl(route_small_kernel<32>, dim3(1), dim3(1024), st, a->logits, (int)a->T, (int)a->E, (int)a->topk, topk_idx,
+            e = launch_pdl(route_small_kernel<32>, dim3(1), dim3(1024), st, logits, (int)a->T, (int)a->E, (int)a->topk, topk_idx,
                            topk_w, a->topk_idx, a->topk_w, offsets, a->expert_offsets, perm, a->perm, inv_perm);
         if (e != cudaSuccess) return check_cuda(e, "qmm_moe route launch");
     } else {

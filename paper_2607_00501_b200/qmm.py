@@ -77,6 +77,7 @@ class MoeArgs(ctypes.Structure):
         ("topk_idx", ctypes.c_void_p), ("topk_w", ctypes.c_void_p),
         ("perm", ctypes.c_void_p), ("expert_offsets", ctypes.c_void_p),
         ("dbg_H", ctypes.c_void_p), ("dbg_D", ctypes.c_void_p),
+        ("w_router", ctypes.c_void_p), ("router_logits", ctypes.c_void_p),
     ]
 
 
@@ -264,11 +265,13 @@ def gemm(fmt: int, packed: torch.Tensor, N: int, K: int, X: torch.Tensor,
 
 
 def moe_args(fmt, T, H, I, E, topk, logits, X, w_gate, w_up, w_down, out,
-             topk_idx=None, topk_w=None, perm=None, expert_offsets=None, dbg_H=None, dbg_D=None) -> MoeArgs:
+             topk_idx=None, topk_w=None, perm=None, expert_offsets=None, dbg_H=None, dbg_D=None,
+             w_router=None, router_logits=None) -> MoeArgs:
     a = MoeArgs(T, H, I, E, topk, fmt, _dp(logits), _dp(X), _dp(w_gate), _dp(w_up), _dp(w_down), _dp(out),
-                _dp(topk_idx), _dp(topk_w), _dp(perm), _dp(expert_offsets), _dp(dbg_H), _dp(dbg_D))
+                _dp(topk_idx), _dp(topk_w), _dp(perm), _dp(expert_offsets), _dp(dbg_H), _dp(dbg_D),
+                _dp(w_router), _dp(router_logits))
     # the struct holds raw device pointers only: keep the tensors alive as long as the struct
-    a._keep = (logits, X, w_gate, w_up, w_down, out, topk_idx, topk_w, perm, expert_offsets, dbg_H, dbg_D)
+    a._keep = (logits, X, w_gate, w_up, w_down, out, topk_idx, topk_w, perm, expert_offsets, dbg_H, dbg_D, w_router, router_logits)
     return a
 
 

@@ -209,6 +209,50 @@ def test_moe_decode_two_launches_match_the_four_launch_form(qmm, oracle, fmt, T,
     assert np.all(routed["out"] == 3.0)
 
 
+@pytest.mark.parametrize("fmt", [Q4, Q8])
+@pytest.mark.parametrize("T", [1, 4])
+def test_moe_decode_with_the_router_product_inside(qmm, oracle, fmt, T):
+    """The library computes the router logits itself (X times the packed [E, H] router matrix, fp32
+    outputs) ahead of the routing.  The exported logits are held to the product tolerance against the
+    oracle; everything downstream is then checked against the oracle fed with those very logits, so the
+    routing stays a bit-exact comparison."""
+    E, topk, H, I = 128, 8, 512, 256
+    L = Layer(qmm, fmt, 660 + T, E, H, I)
+    X = synth.activations(661, T, T, H)
+    wr = synth.quantize(fmt, synth.weights(662, fmt, E, H, std=0.05))
+    out = torch.full((T, H), 3.0, dtype=torch.float16, device="cuda")
+    o = dict(topk_idx=torch.full((T, topk), -1, dtype=torch.int32, device="cuda"),
+             topk_w=torch.zeros((T, topk), dtype=torch.float32, device="cuda"),
+             perm=torch.full((T * topk,), -1, dtype=torch.int32, device="cuda"),
+             expert_offsets=torch.full((E + 1,), -1, dtype=torch.int32, device="cuda"),
+             dbg_H=torch.zeros((T * topk, I), dtype=torch.float16, device="cuda"),
+             dbg_D=torch.zeros((T * topk, H), dtype=torch.float16, device="cuda"))
+    lg = torch.zeros((T, E), dtype=torch.float32, device="cuda")
+    args = qmm.moe_args(fmt, T, H, I, E, topk, None, util.dev(X), L.p_gate, L.p_up, L.p_down, out,
+                        w_router=qmm.pack(fmt, util.dev(wr), E, H), router_logits=lg, **o)
+    ws = torch.zeros(qmm.moe_workspace_bytes(args), dtype=torch.uint8, device="cuda")
+    qmm.moe(args, ws)
+    qmm.status_check(ws)
+    logits = lg.cpu().numpy()
+    ref, B = oracle.gemm(fmt, wr, E, H, X)
+    util.assert_within_tol(logits.astype(np.float64), ref, B, "router logits")
+    res = {k: v.cpu().numpy() for k, v in o.items()}
+    res["out"] = out.cpu().numpy()
+    check_stages(oracle, L, res, logits, X, topk, experts=sorted(set(res["topk_idx"].reshape(-1).tolist())))
+    check_end_to_end(oracle, L, res, logits, X, topk, tokens=range(T))
+    # without an export buffer the logits live in the workspace: same output
+    out2 = torch.empty_like(out)
+    args2 = qmm.moe_args(fmt, T, H, I, E, topk, None, util.dev(X), L.p_gate, L.p_up, L.p_down, out2,
+                         w_router=qmm.pack(fmt, util.dev(wr), E, H))
+    ws2 = torch.zeros(qmm.moe_workspace_bytes(args2), dtype=torch.uint8, device="cuda")
+    qmm.moe(args2, ws2)
+    assert torch.equal(out, out2)
+    # prefill-sized layers take caller logits only
+    big = qmm.moe_args(fmt, 64, H, I, E, topk, None, util.dev(synth.activations(1, 1, 64, H)), L.p_gate, L.p_up, L.p_down,
+                       torch.empty((64, H), dtype=torch.float16, device="cuda"), w_router=qmm.pack(fmt, util.dev(wr), E, H))
+    assert qmm.lib().qmm_moe(big, ws.data_ptr(), ws.numel(), None) == 5
+
+
 def test_moe_route_only_and_determinism(qmm, oracle):
     T, E, topk, H, I = 300, 128, 8, 256, 256
     L = Layer(qmm, Q4, 621, 1, H, I)                     # weights unused by the routing call

@@ -39,7 +39,7 @@ def test_version_and_sizes(L):
 
 
 @pytest.mark.parametrize("fmt,N,K,status", [
-    (5, 128, 256, 1), (4, 0, 256, 1), (4, 128, -256, 1), (4, 128, 100, 2), (4, 128, 288, 5), (4, 100, 256, 5),
+    (7, 128, 256, 1), (4, 0, 256, 1), (4, 128, -256, 1), (4, 128, 100, 2), (4, 128, 288, 5), (4, 100, 256, 5),
 ])
 def test_bad_shapes_are_rejected(L, fmt, N, K, status):
     buf = (ctypes.c_char * 64)()
