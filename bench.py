@@ -854,6 +854,34 @@ def run_case(args):
         arr = qmm.gemv_batch_problems(probs)
         for _ in range(reps):
             qmm.gemv_batch(f, arr)
+    elif name in ("chain_q4_dependent", "chain_q4_independent", "chain_q8_dependent", "chain_q8_independent"):
+        # four layers of the decode stack (137 / 258 MB of weights) through qmm_chain: as a dependent chain of
+        # 16 stages, or as 28 independent products
+        f = synth.Q4 if "_q4_" in name else synth.Q8
+        layers = 4
+        host_blocks, host_acts = build_stack_host(layers, (f,))
+        rows_of = {n: NN for n, NN, _, _ in synth.CFG1_LAYER}
+        stages = []
+        if name.endswith("independent"):
+            for l in range(layers):
+                for mname, N, K, act in synth.CFG1_LAYER:
+                    stages.append(dict(op=qmm.CHAIN_LINEAR, N=N, K=K, packed=qmm.pack(f, dev(host_blocks[f][l][mname]), N, K),
+                                       x=dev(host_acts[l][act]), y=torch.empty(N, dtype=torch.float16, device="cuda")))
+        else:
+            for l in range(layers):
+                pk_ = lambda parts, K: torch.cat([qmm.pack(f, dev(host_blocks[f][l][p]), rows_of[p], K) for p in parts])
+                base = 4 * l
+                stages.append(dict(op=qmm.CHAIN_LINEAR, N=3072, K=2048, packed=pk_(("q", "k", "v"), 2048),
+                                   **({"x": dev(host_acts[0]["x_attn"])} if l == 0 else {"x_stage": base - 1, "x_offset": 0})))
+                stages.append(dict(op=qmm.CHAIN_LINEAR, N=2048, K=2048, packed=pk_(("o",), 2048), x_stage=base, x_offset=0))
+                stages.append(dict(op=qmm.CHAIN_GATE_UP_SILU, N=8192, K=2048, packed=pk_(("gate",), 2048), packed_up=pk_(("up",), 2048),
+                                   x_stage=base + 1, x_offset=0))
+                stages.append(dict(op=qmm.CHAIN_LINEAR, N=2048, K=8192, packed=pk_(("down",), 8192), x_stage=base + 2, x_offset=0,
+                                   y=torch.empty(2048, dtype=torch.float16, device="cuda")))
+        chain = qmm.Chain(f, stages)
+        for _ in range(reps):
+            chain.run()
+        qmm.status_check(chain.ws)
     elif name == "gemv_lm_head_q8":
         c = synth.CFG2
         packed = qmm.pack(c["fmt"], dev(synth.quantize(c["fmt"], synth.weights(c["seed"], 0, c["N"], c["K"]))), c["N"], c["K"])
@@ -903,7 +931,7 @@ def run_case(args):
         qmm.status_check(ws)
     else:
         raise SystemExit("unknown --case %r (gemv_batch_q4|q8, gemv_lm_head_q8, gemv_kv_q4|q8, gemm_q4|q8[_down]_M<M>, "
-                         "moe_q4|q8_T<T>)" % name)
+                         "moe_q4|q8_T<T>, chain_q4|q8_dependent|independent)" % name)
     torch.cuda.synchronize()
     print("case %s: %d launches done" % (name, reps), file=sys.stderr)
 
