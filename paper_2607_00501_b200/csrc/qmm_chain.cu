@@ -118,6 +118,31 @@ __device__ __forceinline__ int ld_volatile_int(const int* p)
     asm volatile("ld.volatile.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
+// Bounded wait that parks the warp instead of spinning: mbarrier.try_wait with a suspend-time hint
+// lets the hardware hold the thread until the phase completes or the hint (in ns) has passed, so a
+// waiting warp issues a handful of instructions per microsecond and leaves the issue slots to the
+// warps that multiply.  Gives up like tc::mbar_wait: on the block's abort flag or after `limit` cycles.
+__device__ __forceinline__ bool mbar_wait_parked(uint64_t* bar, uint32_t parity, volatile int* abort, long long limit)
+{
+    const uint32_t addr = tc::smem_u32(bar);
+    const long long t0 = clock64();
+    while (true) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t"
+            ".reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t"
+            "}\n"
+            : "=r"(ok)
+            : "r"(addr), "r"(parity), "r"(1000u)
+            : "memory");
+        if (ok) return true;
+        if (*abort) return false;
+        if (clock64() - t0 > limit) return false;
+    }
+}
+
 __device__ __forceinline__ void consumer_sync()                       // the consumer warps only
 {
     asm volatile("bar.sync 1, %0;" ::"r"(kChainConsumers * 32) : "memory");
@@ -224,7 +249,7 @@ chain_kernel(const uint8_t* __restrict__ plan, uint8_t* ws)
                 const int nt = up->nt;
                 for (int c = 0; c < nt && ok; c += kChainPairs, ++g) {
                     const int s = g % NS;
-                    if (g >= NS) ok = mbar_wait(&empty[s], ((g / NS) - 1) & 1, s_abort, kChainWaitCycles);
+                    if (g >= NS) ok = mbar_wait_parked(&empty[s], ((g / NS) - 1) & 1, s_abort, kChainWaitCycles);
                     if (!ok) break;
                     const int np = min(kChainPairs, nt - c);
                     uint8_t* dst = ring + (size_t)s * SLOT;
@@ -251,7 +276,7 @@ chain_kernel(const uint8_t* __restrict__ plan, uint8_t* ws)
         for (int ui = u_begin; ui < u_end && ok; ++ui) {
             const ChainUnit& u = *unit_at(ui);
             const int n = ui - u_begin, buf = n & 1;
-            ok = mbar_wait(&red_full[buf], (n >> 1) & 1, s_abort, kChainWaitCycles);
+            ok = mbar_wait_parked(&red_full[buf], (n >> 1) & 1, s_abort, kChainWaitCycles);
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
             const float* r = red + buf * (NC * 64);
@@ -325,6 +350,7 @@ chain_kernel(const uint8_t* __restrict__ plan, uint8_t* ws)
         Q4Consts kc;
         kc.init();
         int g = 0;
+        int start = 0;                                                // (16 g) mod NC: the warp that takes pair 0 of slot g
         bool ok = true;
         // Control flow: every consumer thread passes the same sequence of consumer barriers (they only
         // surround the staging of an activation vector).  A thread that gives up raises the abort flag
@@ -380,17 +406,21 @@ chain_kernel(const uint8_t* __restrict__ plan, uint8_t* ws)
                 if (!ok) break;
             }
             float acc[4] = {0.f, 0.f, 0.f, 0.f};
-            for (int c = 0; c < u.nt; c += kChainPairs, ++g) {
-                const int pi = (warp - (g * kChainPairs) % NC + NC) % NC;      // this warp's pair of slot g, if < 16
+            const int nt = u.nt, t0u = u.t0;
+            for (int c = 0; c < nt; c += kChainPairs, ++g) {
+                int pi = warp - start;                                // this warp's pair of slot g, if < 16
+                if (pi < 0) pi += NC;
+                start += kChainPairs;
+                if (start >= NC) start -= NC;
                 if (!ok || pi >= kChainPairs) continue;
                 const int s = g % NS;
-                ok = mbar_wait(&full[s], (g / NS) & 1, s_abort, kChainWaitCycles);
+                ok = mbar_wait_parked(&full[s], (g / NS) & 1, s_abort, kChainWaitCycles);
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) {
                     *s_abort = 1;
                     continue;
                 }
-                if (c + pi < u.nt) {
+                if (c + pi < nt) {
                     const uint8_t* tp = ring + (size_t)s * SLOT + (size_t)pi * TB;
                     const uint8_t* tq = tp + kChainPairs * TB;
                     // the two 16-byte halves in an order that keeps a quarter-warp's accesses on distinct banks
@@ -408,7 +438,7 @@ chain_kernel(const uint8_t* __restrict__ plan, uint8_t* ws)
                         cq.v[4] = qhi.x; cq.v[5] = qhi.y; cq.v[6] = qhi.z; cq.v[7] = qhi.w;
                     }
                     const int row = (lane & ~3) + 2 * (lane & 1);     // the rows whose sums this lane receives
-                    const uint4* xt = xbase + (u.t0 + c + pi) * xmul;
+                    const uint4* xt = xbase + (t0u + c + pi) * xmul;
                     if constexpr (FMT == QMM_Q4) {
                         const uint2 sp = *reinterpret_cast<const uint2*>(tp + kTileCodeBytes + 4 * row);
                         const uint2 sq = *reinterpret_cast<const uint2*>(tq + kTileCodeBytes + 4 * row);
@@ -424,7 +454,7 @@ chain_kernel(const uint8_t* __restrict__ plan, uint8_t* ws)
             }
             // hand the warp's sums to the publishers (buffer n & 1; its previous contents must have been read)
             if (ok && n >= 2) {
-                ok = mbar_wait(&red_empty[buf], ((n >> 1) - 1) & 1, s_abort, kChainWaitCycles);
+                ok = mbar_wait_parked(&red_empty[buf], ((n >> 1) - 1) & 1, s_abort, kChainWaitCycles);
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) *s_abort = 1;
             }
