@@ -29,8 +29,10 @@
  *     (M = 0 / T = 0 is accepted and does nothing).  Other shapes return
  *     QMM_ERR_UNSUPPORTED.  There is no CPU fallback and no other GPU target.
  *   - Device pointers must be 16-byte aligned; packed weight buffers 32-byte.
- *   - Workspaces of qmm_gemm and qmm_moe start with a status word: zero-fill a
- *     workspace once after allocating it.
+ *   - Workspaces of qmm_gemm and qmm_moe start with a status word, and qmm_moe
+ *     keeps counters in its workspace that every complete call leaves at zero:
+ *     zero-fill a workspace once after allocating it, and again after a call on
+ *     it was reported as failed (qmm_status_check) or was abandoned midway.
  *   - Packed weights are read before the product kernels wait for the work
  *     that precedes them in the stream (their loads overlap the tail of the
  *     previous kernel).  A packed buffer must therefore be complete when a

@@ -84,6 +84,19 @@ struct GemmParams {
     int tail_halves;                 // != 0: the remaining tiles are dealt as halves of BN / 2 tokens, one after the other over the blocks
     int units_per_block;             // U: share of the (tile, k-block) units of the other tiles
     float* partial;                  // [2 * gridDim.x] slots of NA*BN*128 floats (when some tile is cut)
+    // Grouped products of one layer handed over tile by tile instead of kernel by kernel.  sync[0] is set
+    // once the token-tile list may be read; sync[1 + mt] counts the epilogue warps of the producing
+    // product (gate/up) that have stored their part of token tile mt.  The consuming product (down)
+    // starts under programmatic dependent launch on the SMs the producer's last round leaves idle, reads
+    // the list once sync[0] is set and loads token tile mt once its counter has reached sync_need.
+    int* sync;                       // null: plain kernel-to-kernel ordering
+    int sync_signal;                 // != 0: this launch sets sync[0] and counts its stored tiles
+    int sync_need;                   // > 0: this launch waits on sync[] instead of on the previous kernel
+    // Grouped mode, optional: tiles are handed out in ascending order from this device counter (zeroed
+    // by the caller) instead of in fixed strides, so that blocks which start late (the consuming
+    // product's blocks reach an SM only when the producer's block there has left) or which drew long
+    // tiles (uneven expert load) simply take fewer.
+    int* tile_counter;
     int* status;                     // device status word (0 = ok)
     long long* trace;                // clock64 samples of block 0 in -DQMM_GEMM_TRACE=1 builds; unused (null) otherwise
 };
@@ -252,7 +265,7 @@ constexpr int kGemmL2Ahead = QMM_GEMM_L2_AHEAD;    // stages of a row group's we
 // One piece of work of a block: k-blocks [kb0, kb1) of one output tile.  `cn` blocks contribute to
 // the tile (block indices first .. first + cn - 1, k ascending); cn == 1: the piece is the whole tile.
 struct GemmWork {
-    int n_tile, expert, row0, rows;
+    int n_tile, m_tile, expert, row0, rows;
     int n_mma;                       // token columns the MMAs of this piece compute: rows rounded up to 16
     int kb0, kb1;
     int first, cn;
@@ -334,13 +347,44 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
     uint64_t* stg_empty = bars + 2 * S + 5;                               // epilogue warps: staged tile stored
     uint64_t* full_b = bars + 2 * S + 6;                                  // [SB] TMA -> MMA          (SPLIT only)
     uint64_t* empty_b = bars + 2 * S + 6 + SB;                            // [SB] MMA -> TMA          (SPLIT only)
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 6 + 2 * SB);
-    static_assert((2 * S + 6 + 2 * SB + 1) * 8 <= 512, "barrier area");
+    uint64_t* seq_full = bars + 2 * S + 6 + 2 * SB;                       // [8] tile numbers drawn by the TMA lane (dynamic dealing)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 14 + 2 * SB);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    volatile int* seq = reinterpret_cast<volatile int*>(tmem_slot + 2);   // [8]
+    static_assert((2 * S + 14 + 2 * SB) * 8 + 8 + 32 <= 512, "barrier area");
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     constexpr bool grouped = !DENSE;                                      // token tiles come from a device-built list
-    if (grouped) pdl_wait();                                              // the tile list is written upstream
+    // the tile list is written upstream: wait for the previous kernel, or (hand-over by tiles) for the
+    // flag that the producing product sets once its own wait for the upstream kernels has returned
+    const bool by_tiles = grouped && p.sync != nullptr && p.sync_need > 0;
+    if (grouped && !by_tiles) {
+        pdl_wait();
+        if (p.sync != nullptr && p.sync_signal && blockIdx.x == 0 && threadIdx.x == 0) {
+            __threadfence();
+            atomicExch(p.sync, 1);
+        }
+    }
+    if (by_tiles) {
+        __shared__ int s_list_ok;
+        if (threadIdx.x == 0) {
+            const long long t0 = clock64();
+            int ok = 1;
+            while (*reinterpret_cast<volatile int*>(p.sync) == 0) {
+                if (clock64() - t0 > tc::kWaitLimitCycles) {
+                    ok = 0;
+                    break;
+                }
+            }
+            __threadfence();
+            s_list_ok = ok;
+        }
+        __syncthreads();
+        if (!s_list_ok) {                                                 // nothing is allocated or in flight yet
+            if (threadIdx.x == 0 && p.status != nullptr) atomicExch(p.status, (int)QMM_ERR_DEVICE_TIMEOUT);
+            return;
+        }
+    }
     // plain store: the NA tile sets split the rows of one matrix; SiLU*mul: they are two matrices of N rows each
     const int n_tiles = (EPI == kEpiSiluMul) ? p.N / 128 : p.N / (128 * NA);
     const int m_tiles = grouped ? *p.num_tiles : (p.M + BN - 1) / BN;
@@ -365,6 +409,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         }
         mbar_init(stg_full, NEPI);
         mbar_init(stg_empty, NEPI);
+        for (int q = 0; q < 8; ++q) mbar_init(&seq_full[q], 1);
         *abort_flag = 0;
         fence_barrier_init();
     }
@@ -425,7 +470,21 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             w.cn = (int)((tb + KB - 1) / U) - w.first + 1;
             t += t0;
         } else {
-            t = blockIdx.x + i * gridDim.x;
+            if (grouped && p.tile_counter != nullptr) {
+                // the TMA lane draws the block's i-th tile and publishes it to the other roles through a
+                // small ring (no role is ever more than a few tiles ahead of the epilogue, far fewer than 8)
+                const int slot = i & 7;
+                if (warp == TMA_WARP) {
+                    t = atomicAdd(p.tile_counter, 1);
+                    seq[slot] = t;
+                    mbar_arrive(&seq_full[slot]);
+                } else {
+                    if (!mbar_wait(&seq_full[slot], (i >> 3) & 1, abort_flag)) return false;
+                    t = seq[slot];
+                }
+            } else {
+                t = blockIdx.x + i * gridDim.x;
+            }
             if (t >= total_tiles) return false;
             w.kb0 = 0;
             w.kb1 = KB;
@@ -434,6 +493,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         }
         w.n_tile = t % n_tiles;
         const int mt = t / n_tiles;
+        w.m_tile = mt;
         if (grouped) {
             w.expert = p.tile_expert[mt];
             w.row0 = p.tile_row0[mt];
@@ -525,7 +585,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         constexpr int CH = (NCH + GROUPS - 1) / GROUPS;                   // chunks per warp
         constexpr int NOUT = (EPI == kEpiSiluMul) ? 1 : NA;               // output tiles per weight row
         constexpr int NSTG = NA;                                          // tile sets that go through the staging buffer
-        pdl_wait();                                                       // the output buffer may be in use upstream
+        if (!by_tiles) pdl_wait();                                        // the output buffer may be in use upstream
         bool ok = true;
         [[maybe_unused]] bool etr = false;
         int it = 0, staged = 0;                                           // pieces seen / tiles that went through the staging buffer
@@ -644,6 +704,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                     }
                 }
             }
+            if (grouped && p.sync != nullptr && p.sync_signal) {          // this warp's part of the token tile is stored
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) atomicAdd(p.sync + 1 + w.m_tile, 1);
+            }
             __syncwarp();
             if (lane == 0) mbar_arrive(stg_empty);
             ++staged;
@@ -652,11 +717,26 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
     } else if (warp == TMA_WARP) {
         // ================= TMA producer: activation tiles
         if (lane == 0) {
-            pdl_wait();                                                   // activations come from the previous kernel
+            if (!by_tiles) pdl_wait();                                    // activations come from the previous kernel
             int issued = 0, g = 0;
             bool ok = true;
             GemmWork w;
             for (int i = 0; ok && get_work(i, w); ++i) {
+                if (by_tiles) {
+                    // the rows of this token tile are complete once every epilogue warp of the producing
+                    // product has counted itself in for each of its weight tiles
+                    const volatile int* cnt = p.sync + 1 + w.m_tile;
+                    const long long t0 = clock64();
+                    while (*cnt < p.sync_need) {
+                        if (*abort_flag || clock64() - t0 > tc::kWaitLimitCycles) {
+                            ok = false;
+                            break;
+                        }
+                    }
+                    if (!ok) break;
+                    __threadfence();
+                    asm volatile("fence.proxy.async;" ::: "memory");     // the rows were written by ordinary stores, TMA reads them
+                }
                 for (int kb = w.kb0; kb < w.kb1; ++kb, ++g) {
                     const int s = g % SB;
                     uint64_t* slot_full = SPLIT ? &full_b[s] : &full[s];

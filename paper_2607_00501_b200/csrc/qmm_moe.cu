@@ -35,7 +35,7 @@ dim3 persistent_grid(int bn, int na, int64_t tiles);
 
 struct MoeWorkspace {
     size_t status, counts, offsets, num_tiles, tile_expert, tile_row0, tile_rows;
-    size_t topk_idx, topk_w, perm, inv_perm, xp, hbuf, dbuf, trace, logits, total;
+    size_t topk_idx, topk_w, perm, inv_perm, xp, hbuf, dbuf, trace, logits, sync, total;
     int bn, max_tiles;
 };
 
@@ -51,8 +51,9 @@ static MoeWorkspace moe_layout(const qmm_moe_args* a)
     auto take = [&](size_t bytes) { const size_t at = o; o = align_up(o + bytes, 256); return at; };
     w.status = take(256);
     w.counts = take((size_t)a->E * 4);
+    w.sync = take((size_t)(w.max_tiles + 3) * 4);          // hand-over of token tiles between the two grouped products (directly after counts: one memset clears both)
+    w.num_tiles = take(4);                                 // (counts, hand-over words and this are cleared by one memset per call)
     w.offsets = take((size_t)(a->E + 1) * 4);
-    w.num_tiles = take(4);
     w.tile_expert = take((size_t)w.max_tiles * 4);
     w.tile_row0 = take((size_t)w.max_tiles * 4);
     w.tile_rows = take((size_t)w.max_tiles * 4);
@@ -170,11 +171,14 @@ permute_kernel(const int* __restrict__ topk_idx, int total, const int* __restric
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
     // rows and token tiles of the experts before e (E <= 1024: one count per thread)
+    // (rows stay in expert order; the token tiles are listed busiest expert first, equal counts by
+    // expert index, so that the grouped products start their longest tiles first and end on short ones)
     int rows_before = 0, tiles_before = 0;
-    if ((int)threadIdx.x < e) {
+    const int mine_c = counts[e];
+    if ((int)threadIdx.x < E) {
         const int c = counts[threadIdx.x];
-        rows_before = c;
-        tiles_before = (c + bn - 1) / bn;
+        if ((int)threadIdx.x < e) rows_before = c;
+        if (c > mine_c || (c == mine_c && (int)threadIdx.x < e)) tiles_before = (c + bn - 1) / bn;
     }
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) {
@@ -205,8 +209,8 @@ permute_kernel(const int* __restrict__ topk_idx, int total, const int* __restric
         if (e == E - 1) {
             offsets[E] = r0 + mine;
             if (offsets_user) offsets_user[E] = r0 + mine;
-            *num_tiles = t0 + nt;
         }
+        if (t0 + nt > 0) atomicMax(num_tiles, t0 + nt);                   // the expert listed last closes the list (num_tiles is zeroed with the counts)
     }
     __syncthreads();
 
@@ -274,11 +278,17 @@ __global__ void gather_rows_kernel(const uint16_t* __restrict__ X, const int* __
 
 // out[t, :] = fp16( sum_j p[t, j] * D[inv_perm[t*topk + j], :] ), fp32, j ascending.
 // One block per token; each thread owns 8 consecutive columns.
+// The layer's last kernel also re-zeroes the words the next call counts in (rows per expert, tile
+// counters, hand-over words): every kernel that used them has finished once this one may run, and a
+// per-call memset node would sit in front of the routing kernel and keep it from overlapping its predecessor.
 __global__ void combine_kernel(const uint16_t* __restrict__ D, const int* __restrict__ inv_perm,
-                               const float* __restrict__ topk_w, int topk, int H, uint16_t* __restrict__ out)
+                               const float* __restrict__ topk_w, int topk, int H, uint16_t* __restrict__ out,
+                               int* __restrict__ clear_ptr, int clear_n)
 {
     pdl_launch_dependents();
     pdl_wait();
+    if (blockIdx.x == 0)
+        for (int i = threadIdx.x; i < clear_n; i += blockDim.x) clear_ptr[i] = 0;
     const int t = blockIdx.x;
     for (int c = threadIdx.x * 8; c < H; c += blockDim.x * 8) {
         float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
@@ -325,6 +335,7 @@ qmm_status launch_moe(const qmm_moe_args* a, void* ws, bool route_only, cudaStre
     uint8_t* base = (uint8_t*)ws;
     int* status = (int*)(base + w.status);
     int* counts = (int*)(base + w.counts);
+    int* tile_sync = (int*)(base + w.sync);
     int* offsets = (int*)(base + w.offsets);
     int* num_tiles = (int*)(base + w.num_tiles);
     int* tile_expert = (int*)(base + w.tile_expert);
@@ -385,8 +396,13 @@ qmm_status launch_moe(const qmm_moe_args* a, void* ws, bool route_only, cudaStre
                            topk_w, a->topk_idx, a->topk_w, offsets, a->expert_offsets, perm, a->perm, inv_perm);
         if (e != cudaSuccess) return check_cuda(e, "qmm_moe route launch");
     } else {
-        e = cudaMemsetAsync(counts, 0, (size_t)a->E * 4, st);
-        if (e != cudaSuccess) return check_cuda(e, "qmm_moe clear counts");
+        // counts, tile counters, hand-over words and the tile count start at zero: the workspace was zero-filled
+        // once by the caller and every complete call leaves them zero again (combine_kernel); a routing-only
+        // call has no last kernel of that kind and clears them itself, before and after
+        if (route_only) {
+            e = cudaMemsetAsync(counts, 0, (w.num_tiles - w.counts) + 4, st);
+            if (e != cudaSuccess) return check_cuda(e, "qmm_moe clear counts");
+        }
         // 1. routing
         const int warps_per_block = 8;
         const dim3 grid((a->T + warps_per_block - 1) / warps_per_block), block(warps_per_block * 32);
@@ -403,7 +419,13 @@ qmm_status launch_moe(const qmm_moe_args* a, void* ws, bool route_only, cudaStre
                        inv_perm);
         if (e != cudaSuccess) return check_cuda(e, "qmm_moe permute launch");
     }
-    if (route_only) return QMM_OK;
+    if (route_only) {
+        if (!small) {
+            e = cudaMemsetAsync(counts, 0, (w.num_tiles - w.counts) + 4, st);
+            if (e != cudaSuccess) return check_cuda(e, "qmm_moe clear counts");
+        }
+        return QMM_OK;
+    }
 
     if (small) {
         // decode: a few rows -> GEMV path (gate/up with SiLU*mul, down), then the combine
@@ -414,7 +436,7 @@ qmm_status launch_moe(const qmm_moe_args* a, void* ws, bool route_only, cudaStre
                             (int)a->topk, (int)a->H, (int)a->I, st);
         if (s != QMM_OK) return s;
         e = launch_pdl(combine_kernel, dim3(a->T), dim3(256), st, (const uint16_t*)dbuf, (const int*)inv_perm,
-                       (const float*)topk_w, (int)a->topk, (int)a->H, a->out);
+                       (const float*)topk_w, (int)a->topk, (int)a->H, a->out, (int*)nullptr, 0);
         if (e != cudaSuccess) return check_cuda(e, "qmm_moe combine launch");
         return QMM_OK;
     }
@@ -444,6 +466,9 @@ qmm_status launch_moe(const qmm_moe_args* a, void* ws, bool route_only, cudaStre
         p.tile_rows = tile_rows;
         p.num_tiles = num_tiles;
         p.status = status;
+        p.sync = tile_sync + 2;
+        p.sync_signal = 1;
+        if (!g_knobs.moe_no_fuse) p.tile_counter = tile_sync;
 #if QMM_GEMM_TRACE
         p.trace = (long long*)(base + w.trace);                            // tuning builds only
 #endif
@@ -471,12 +496,17 @@ qmm_status launch_moe(const qmm_moe_args* a, void* ws, bool route_only, cudaStre
         p.tile_rows = tile_rows;
         p.num_tiles = num_tiles;
         p.status = status;
+        if (!g_knobs.moe_no_fuse) {
+            p.sync = tile_sync + 2;
+            p.sync_need = (a->I / 128) * GemmGeom<128, 2, kEpiSiluMul, QMM_Q4>::kEpiWarps;   // weight tiles x epilogue warps of the gate/up product
+            p.tile_counter = tile_sync + 1;
+        }
         s = launch_tc_gemm(a->fmt, w.bn, na, kEpiStore, false, map, p, persistent_grid(w.bn, na, 0), st);
         if (s != QMM_OK) return s;
     }
     // 6. weighted combine
     e = launch_pdl(combine_kernel, dim3(a->T), dim3(256), st, (const uint16_t*)dbuf, (const int*)inv_perm, (const float*)topk_w,
-                   (int)a->topk, (int)a->H, a->out);
+                   (int)a->topk, (int)a->H, a->out, counts, (int)((w.num_tiles - w.counts) / 4 + 1));
     if (e != cudaSuccess) return check_cuda(e, "qmm_moe combine launch");
     return QMM_OK;
 }
