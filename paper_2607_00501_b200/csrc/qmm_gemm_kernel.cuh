@@ -97,6 +97,9 @@ struct GemmParams {
     // product's blocks reach an SM only when the producer's block there has left) or which drew long
     // tiles (uneven expert load) simply take fewer.
     int* tile_counter;
+    int list_ready;                  // != 0: the tile list was complete before this kernel could start (the upstream
+                                     // kernel lets its dependents go only after its own wait): no block-wide wait at the
+                                     // top, set-up and weight prefetch overlap the upstream kernel
     int* status;                     // device status word (0 = ok)
     long long* trace;                // clock64 samples of block 0 in -DQMM_GEMM_TRACE=1 builds; unused (null) otherwise
 };
@@ -358,7 +361,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
     // the tile list is written upstream: wait for the previous kernel, or (hand-over by tiles) for the
     // flag that the producing product sets once its own wait for the upstream kernels has returned
     const bool by_tiles = grouped && p.sync != nullptr && p.sync_need > 0;
-    if (grouped && !by_tiles) {
+    if (grouped && !by_tiles && !p.list_ready) {
         pdl_wait();
         if (p.sync != nullptr && p.sync_signal && blockIdx.x == 0 && threadIdx.x == 0) {
             __threadfence();
@@ -718,6 +721,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         // ================= TMA producer: activation tiles
         if (lane == 0) {
             if (!by_tiles) pdl_wait();                                    // activations come from the previous kernel
+            if (grouped && p.list_ready && p.sync != nullptr && p.sync_signal && blockIdx.x == 0) {
+                __threadfence();                                          // everything upstream is complete: the consuming product may read the list
+                atomicExch(p.sync, 1);
+            }
             int issued = 0, g = 0;
             bool ok = true;
             GemmWork w;

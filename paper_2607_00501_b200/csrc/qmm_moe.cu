@@ -266,8 +266,8 @@ permute_kernel(const int* __restrict__ topk_idx, int total, const int* __restric
 __global__ void gather_rows_kernel(const uint16_t* __restrict__ X, const int* __restrict__ perm, int total, int topk,
                                    int H, uint16_t* __restrict__ Xp)
 {
-    pdl_launch_dependents();
-    pdl_wait();
+    pdl_wait();                                       // first: once the dependents may start, the permutation kernel is
+    pdl_launch_dependents();                          // complete, so the grouped product reads the tile list without waiting
     const int r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     if (r >= total) return;
     const int t = perm[r] / topk;
@@ -468,6 +468,7 @@ qmm_status launch_moe(const qmm_moe_args* a, void* ws, bool route_only, cudaStre
         p.status = status;
         p.sync = tile_sync + 2;
         p.sync_signal = 1;
+        p.list_ready = 1;
         if (!g_knobs.moe_no_fuse) p.tile_counter = tile_sync;
 #if QMM_GEMM_TRACE
         p.trace = (long long*)(base + w.trace);                            // tuning builds only
