@@ -706,6 +706,20 @@ def sections_ffn_on(args, qmm, torch, pk, fmts, out, flush, dev, sampler, on):
                                                   **tensor_fracs(tf, pk))
                 qmm.status_check(ws)
         out["prefill_gemm_q%d" % f] = gemm
+    if on("gemm"):
+        # not configs: two shapes the tile plan was never tuned on (its cycle estimates come from the cfg3 shapes)
+        other = {}
+        for N, K in ((4096, 4096), (14336, 4096)):
+            blocks = synth.quantize(synth.Q4, synth.weights(33, N, N, K))
+            packed = qmm.pack(synth.Q4, dev(blocks), N, K)
+            for M in (512, 2048):
+                X = dev(synth.activations(33, M, M, K))
+                Y = torch.empty((M, N), dtype=torch.float16, device="cuda")
+                ws = torch.zeros(qmm.gemm_workspace_bytes(synth.Q4, M, N, K), dtype=torch.uint8, device="cuda")
+                m = measure(torch, lambda: qmm.gemm(synth.Q4, packed, N, K, X, Y=Y, ws=ws), flush)
+                qmm.status_check(ws)
+                other["N%d_K%d_M%d" % (N, K, M)] = dict(m, **tensor_fracs(2.0 * M * N * K / m["ms"] / 1e9, pk))
+        out["prefill_gemm_q4_other_shapes"] = other
 
     # not configs: the 5-bit and 6-bit formats through the same two kernel families (one decode-sized
     # GEMV on the LM-head shape, one prefill GEMM on the gate/up shape at M = 2048)

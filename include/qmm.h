@@ -54,7 +54,7 @@
  *     2 (i % 4), 2 (i % 4) + 1 of qh[i / 4] = u_i >> 4.
  *   (The paper's kernel library spans 2-bit to 16-bit formats, Sec. 3.3 and
  *   Sec. 4.1; Q5 and Q6 are built for qmm_pack, qmm_dequant, qmm_packed_check,
- *   qmm_gemv, qmm_gemv_static and qmm_gemm -- every other call returns
+ *   qmm_gemv, qmm_gemv_static, qmm_gemv_batch and qmm_gemm -- every other call returns
  *   QMM_ERR_UNSUPPORTED for them.)
  *   Row n of W holds K/32 consecutive blocks; rows are consecutive; block b of
  *   row n covers k in [32 b, 32 b + 32).  Weight value: float(d) * q (exact in

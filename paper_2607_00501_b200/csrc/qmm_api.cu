@@ -58,11 +58,11 @@ DebugKnobs g_knobs = {};
 
 static bool fmt_ok(int fmt) { return fmt == QMM_Q4 || fmt == QMM_Q5 || fmt == QMM_Q6 || fmt == QMM_Q8; }
 
-// Q5 and Q6 are built for pack / dequant / check, the single GEMV and the dense GEMM only.
+// Q5 and Q6 are built for pack / dequant / check, the single and the batched GEMV and the dense GEMM only.
 static qmm_status check_fmt_everywhere(const char* who, int fmt)
 {
     if (fmt == QMM_Q5 || fmt == QMM_Q6)
-        return fail(QMM_ERR_UNSUPPORTED, "%s: format %d is built for qmm_pack, qmm_dequant, qmm_packed_check, qmm_gemv and qmm_gemm only", who, fmt);
+        return fail(QMM_ERR_UNSUPPORTED, "%s: format %d is built for qmm_pack, qmm_dequant, qmm_packed_check, qmm_gemv, qmm_gemv_batch and qmm_gemm only", who, fmt);
     return QMM_OK;
 }
 
@@ -193,7 +193,6 @@ qmm_status qmm_gemv_batch(qmm_format fmt, const qmm_gemv_problem* problems, int 
     if (count < 0) return fail(QMM_ERR_INVALID_ARG, "qmm_gemv_batch: count=%d is negative", count);
     if (count == 0) return QMM_OK;
     if (!problems) return fail(QMM_ERR_INVALID_ARG, "qmm_gemv_batch: null problem list");
-    if (fmt_ok(fmt) && check_fmt_everywhere("qmm_gemv_batch", fmt) != QMM_OK) return QMM_ERR_UNSUPPORTED;
     for (int i = 0; i < count; ++i) {
         const qmm_gemv_problem& q = problems[i];
         qmm_status s = check_matrix("qmm_gemv_batch", fmt, q.N, q.K);

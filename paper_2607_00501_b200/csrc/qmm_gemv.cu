@@ -283,6 +283,8 @@ gemv_batch_kernel(const __grid_constant__ BatchParams bp)
         const uint8_t* tq = tp + group_bytes;
         r.cp[u] = ld_stream_256(tp);
         r.cq[u] = ld_stream_256(tq);
+        r.hp[u] = load_hi<FMT>(tp - 32 * lane, lane);
+        r.hq[u] = load_hi<FMT>(tq - 32 * lane, lane);
         r.sp[u] = load_scales<FMT>(tp - 32 * lane, lane);
         r.sq[u] = load_scales<FMT>(tq - 32 * lane, lane);
     };
@@ -313,12 +315,7 @@ gemv_batch_kernel(const __grid_constant__ BatchParams bp)
 #pragma unroll
             for (int u = 0; u < kUnroll; ++u) {
                 const int tt = t + u * WARPS;
-                if (tt < t_end) {
-                    if constexpr (FMT == QMM_Q4)
-                        tile_pair_mma_q4(r.cp[u], r.cq[u], r.sp[u], r.sq[u], xb + tt * XV, acc, kc);
-                    else
-                        tile_pair_mma_q8(r.cp[u], r.cq[u], r.sp[u], r.sq[u], xb + tt * XV, acc);
-                }
+                if (tt < t_end) tile_pair_mma<FMT>(r.cp[u], r.cq[u], r.hp[u], r.hq[u], r.sp[u], r.sq[u], xb + tt * XV, acc, kc);
             }
             t += STEP;
             if (t < t_end) load_group();
@@ -1088,17 +1085,18 @@ qmm_status launch_gemv_batch(int fmt, const qmm_gemv_problem* probs, int count, 
         int grid = kNumSMs * (QMM_BATCH_THREADS_PER_SM / (WARPS * 32));
         if (units < grid) grid = units;
         cudaError_t e;
-        if (fmt == QMM_Q4) {
-            auto kern = gemv_batch_kernel<QMM_Q4, WARPS>;
-            if (smem > 48 * 1024 && (e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess)
-                return check_cuda(e, "qmm_gemv_batch shared memory size");
-            e = launch_pdl(kern, dim3(grid), dim3(WARPS * 32), smem, st, bp);
-        } else {
-            auto kern = gemv_batch_kernel<QMM_Q8, WARPS>;
-            if (smem > 48 * 1024 && (e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess)
-                return check_cuda(e, "qmm_gemv_batch shared memory size");
-            e = launch_pdl(kern, dim3(grid), dim3(WARPS * 32), smem, st, bp);
-        }
+#define QMM_BATCH_CASE(F)                                                                                                          \
+    {                                                                                                                              \
+        auto kern = gemv_batch_kernel<F, WARPS>;                                                                                   \
+        if (smem > 48 * 1024 && (e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) \
+            return check_cuda(e, "qmm_gemv_batch shared memory size");                                                             \
+        e = launch_pdl(kern, dim3(grid), dim3(WARPS * 32), smem, st, bp);                                                          \
+    }
+        if (fmt == QMM_Q4) QMM_BATCH_CASE(QMM_Q4)
+        else if (fmt == QMM_Q5) QMM_BATCH_CASE(QMM_Q5)
+        else if (fmt == QMM_Q6) QMM_BATCH_CASE(QMM_Q6)
+        else QMM_BATCH_CASE(QMM_Q8)
+#undef QMM_BATCH_CASE
         if (e != cudaSuccess) return check_cuda(e, "qmm_gemv_batch launch");
     }
     return QMM_OK;

@@ -20,17 +20,18 @@ def qmm():
     return _qmm
 
 
-def build_chain(qmm, fmt, spec, seed):
+def build_chain(qmm, fmt, spec, seed, unit_variance=False):
     """spec: list of (op, N, K, source) with source = None (own caller vector) or (stage, offset).
     Returns (chain, host data per stage)."""
     stages, host = [], []
     for i, (op, N, K, src) in enumerate(spec):
         h = {"op": op, "N": N, "K": K, "src": src}
-        h["w"] = synth.quantize(fmt, synth.weights(seed, 10 * i, N, K))
+        std = K ** -0.5 if unit_variance else 0.02                    # (unit variance: magnitudes survive long chains)
+        h["w"] = synth.quantize(fmt, synth.weights(seed, 10 * i, N, K, std=std))
         d = {"op": op, "N": N, "K": K, "packed": qmm.pack(fmt, util.dev(h["w"]), N, K),
              "y": torch.full((N,), 7.0, dtype=torch.float16, device="cuda")}
         if op == qmm.CHAIN_GATE_UP_SILU:
-            h["w_up"] = synth.quantize(fmt, synth.weights(seed, 10 * i + 1, N, K))
+            h["w_up"] = synth.quantize(fmt, synth.weights(seed, 10 * i + 1, N, K, std=std))
             d["packed_up"] = qmm.pack(fmt, util.dev(h["w_up"]), N, K)
         if src is None:
             h["x"] = synth.activations(seed, 1000 + i, K)
@@ -115,6 +116,36 @@ def test_chain_of_independent_products_is_a_batch(qmm, oracle, fmt):
     chain.run()
     qmm.status_check(chain.ws)
     check_chain(qmm, oracle, fmt, stages, host, "independent")
+
+
+@pytest.mark.parametrize("case", range(8))
+def test_random_stage_graphs(qmm, oracle, case):
+    """Seeded random lists of stages: random shapes and operators, each stage reading a caller vector or a
+    random window of a random earlier stage -- levels of several stages, fan-out, K splits and whole
+    units mixed -- every stage against the oracle on the GPU's own intermediates, twice (same bits)."""
+    rng = np.random.default_rng([951, case])
+    fmt = int(rng.choice([4, 8]))
+    spec = []
+    for i in range(int(rng.integers(3, 14))):
+        op = GU if rng.random() < 0.25 else LIN
+        N = int(rng.integers(1, 17)) * 128
+        feasible = [j for j in range(i) if spec[j][1] >= 256]
+        if feasible and rng.random() < 0.7:
+            j = int(rng.choice(feasible))
+            K = int(rng.integers(1, min(spec[j][1], 4096) // 256 + 1)) * 256
+            off = int(rng.integers(0, (spec[j][1] - K) // 8 + 1)) * 8
+            spec.append((op, N, K, (j, off)))
+        else:
+            spec.append((op, N, int(rng.integers(1, 17)) * 256, None))
+    chain, stages, host = build_chain(qmm, fmt, spec, 960 + case, unit_variance=True)
+    chain.run()
+    qmm.status_check(chain.ws)
+    check_chain(qmm, oracle, fmt, stages, host, "random graph %d" % case)
+    first = [s["y"].clone() for s in stages]
+    chain.run()
+    torch.cuda.synchronize()
+    for a, s in zip(first, stages):
+        assert torch.equal(a, s["y"])
 
 
 def test_chain_argument_checks(qmm):

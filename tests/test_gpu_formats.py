@@ -127,6 +127,22 @@ def test_prefill_and_decode_shapes_of_the_configs(qmm, oracle, fmt):
         qmm.status_check(ws)
 
 
+@pytest.mark.parametrize("fmt", [Q5, Q6])
+def test_gemv_batch(qmm, oracle, fmt):
+    shapes = [(128, 256), (384, 1024), (128, 8192), (640, 512), (2176, 1280), (2048, 2048)]
+    probs, refs = [], []
+    for i, (N, K) in enumerate(shapes):
+        blocks = synth.quantize(fmt, synth.weights(94, 10 * fmt + i, N, K))
+        x = synth.activations(94, 100 + i, K)
+        y = torch.full((N,), 9.0, dtype=torch.float16, device="cuda")
+        probs.append((qmm.pack(fmt, util.dev(blocks), N, K), N, K, util.dev(x), y))
+        refs.append(oracle.gemv(fmt, blocks, N, K, x))
+    qmm.gemv_batch(fmt, qmm.gemv_batch_problems(probs))
+    torch.cuda.synchronize()
+    for (p, N, K, x, y), (y_ref, B) in zip(probs, refs):
+        util.assert_within_tol(util.host_f64(y), y_ref, B, "batch fmt=%d %dx%d" % (fmt, N, K))
+
+
 def test_calls_not_built_for_these_formats_say_so(qmm):
     L = qmm.lib()
     w = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
@@ -134,7 +150,6 @@ def test_calls_not_built_for_these_formats_say_so(qmm):
     y = torch.zeros(128, dtype=torch.float16, device="cuda")
     for fmt in (Q5, Q6):
         assert L.qmm_gemv_gate_up(fmt, w.data_ptr(), w.data_ptr(), 128, 256, x.data_ptr(), y.data_ptr(), None) == 5
-        assert L.qmm_gemv_batch(fmt, qmm.gemv_batch_problems([(w, 128, 256, x, y)]), 1, None) == 5
         st = (qmm.ChainStage * 1)(qmm.ChainStage(0, -1, 0, x.data_ptr(), w.data_ptr(), None, 128, 256, None))
         assert L.qmm_chain_plan_bytes(fmt, st, 1) == 0 and "not built" in qmm.last_error()
         a = qmm.moe_args(fmt, 4, 256, 256, 8, 2, x, x, w, w, w, y)
