@@ -311,3 +311,28 @@ def test_row_sharded_gemv_on_one_rank_is_the_plain_product(qmm, oracle):
     y = op(util.dev(x))
     y_ref, B = oracle.gemv(Q8, blocks, N, K, x)
     util.assert_within_tol(util.host_f64(y), y_ref, B, "sharded, one rank")
+
+
+@pytest.mark.parametrize("fmt", [Q4, Q8])
+def test_gemv_batch_of_many_short_products(qmm, oracle, fmt):
+    """Enough short-K products for every warp of the grid to own units of its own (the one-warp-per-unit
+    form of the batched kernel): 100 products of mixed shapes, every output against the oracle."""
+    shapes = [(3072, 1024), (512, 256), (1024, 512), (640, 1024 if fmt == Q4 else 512)]
+    probs, refs = [], []
+    for i in range(100):
+        N, K = shapes[i % len(shapes)]
+        blocks = synth.quantize(fmt, synth.weights(120, 1000 * fmt + i, N, K))
+        x = synth.activations(121, i, K)
+        y = torch.full((N,), 9.0, dtype=torch.float16, device="cuda")
+        probs.append((packed_from(qmm, fmt, blocks, N, K), N, K, util.dev(x), y))
+        refs.append(oracle.gemv(fmt, blocks, N, K, x))
+    arr = qmm.gemv_batch_problems(probs)
+    qmm.gemv_batch(fmt, arr)
+    torch.cuda.synchronize()
+    for (p, N, K, x, y), (y_ref, B) in zip(probs, refs):
+        util.assert_within_tol(util.host_f64(y), y_ref, B, "short batch %dx%d" % (N, K))
+    first = [p[4].clone() for p in probs]
+    qmm.gemv_batch(fmt, arr)
+    torch.cuda.synchronize()
+    for f, p in zip(first, probs):
+        assert torch.equal(f, p[4])
