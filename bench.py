@@ -687,10 +687,11 @@ def sections_ffn_on(args, qmm, torch, pk, fmts, out, flush, dev, sampler, on):
         b = 2 * synth.canonical_bytes(f, N, K)
         out["ffn_gate_up_silu_q%d_gemv" % f] = dict({"ms": round(med, 4)}, **hbm_fracs(b, med, pk))
 
-    # cfg3: prefill GEMM sweep (Q4 as the config says, plus the small-batch sizes below one token tile;
-    # Q8 = the same kernels with the byte expander, measured at the two largest M)
+    # cfg3: prefill GEMM sweep (Q4 as the config says, plus the small-batch sizes below one token tile:
+    # M <= 8 runs on the few-token kernel, whose bound is the HBM stream of W; Q8 = the same kernels with
+    # the byte expander, measured at M = 4 and the two largest M)
     c = synth.CFG3
-    for f, Ms in (((c["fmt"], (16, 32, 64) + tuple(c["Ms"])), (synth.Q8, c["Ms"][-2:])) if on("gemm") else ()):
+    for f, Ms in (((c["fmt"], (2, 4, 8, 16, 32, 64) + tuple(c["Ms"])), (synth.Q8, (4,) + tuple(c["Ms"][-2:]))) if on("gemm") else ()):
         gemm = {}
         for name, N, K in c["shapes"]:
             blocks = synth.quantize(f, synth.weights(c["seed"], 0 if name == "gate_up" else 1, N, K))
@@ -703,7 +704,7 @@ def sections_ffn_on(args, qmm, torch, pk, fmts, out, flush, dev, sampler, on):
                 tf = 2.0 * M * N * K / m["ms"] / 1e9
                 floor_ms = max(2.0 * M * N * K / pk["bf16_tflops"] / 1e9, (blocks.nbytes + 2 * M * (N + K)) / pk["hbm_gbs"] / 1e6)
                 gemm["%s_M%d" % (name, M)] = dict(m, roofline_floor_ms=round(floor_ms, 4), frac_of_floor=round(floor_ms / m["ms"], 4),
-                                                  **tensor_fracs(tf, pk))
+                                                  **(hbm_fracs(blocks.nbytes, m["ms"], pk) if M <= 8 else tensor_fracs(tf, pk)))
                 qmm.status_check(ws)
         out["prefill_gemm_q%d" % f] = gemm
     if on("gemm"):

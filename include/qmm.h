@@ -370,6 +370,7 @@ qmm_status qmm_status_check(void* ws, void* stream);
  *   "gemv_no_cluster"  "1"             K split through workspace partial sums + second kernel
  *   "gemm_force"       "bn[,units]"    token tile and (tile, k-block) units per block of qmm_gemm
  *   "gemm_no_tail_cut" "1"             last, partly filled round of tiles left whole
+ *   "gemm_no_small"    "1"             M <= 8 through the tensor-core kernel, not the few-token kernel
  *   "moe_no_fuse"      "1"             decode-sized qmm_moe as separate route / product / combine launches
  */
 qmm_status qmm_debug_config(const char* name, const char* value);

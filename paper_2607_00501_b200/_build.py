@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 BUILD = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libqmm.so")
-SOURCES = ("qmm_api.cu", "qmm_pack.cu", "qmm_gemv.cu", "qmm_gemm.cu", "qmm_moe.cu", "qmm_chain.cu")
+SOURCES = ("qmm_api.cu", "qmm_pack.cu", "qmm_gemv.cu", "qmm_gemm.cu", "qmm_gemm_small.cu", "qmm_moe.cu", "qmm_chain.cu")
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
               "-Xcompiler", "-fPIC", "-DQMM_BUILD"]
 

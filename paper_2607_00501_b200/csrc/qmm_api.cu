@@ -371,6 +371,7 @@ qmm_status qmm_debug_config(const char* name, const char* value)
     }
     int* flag = strcmp(name, "gemv_no_cluster") == 0    ? &g_knobs.gemv_no_cluster
                 : strcmp(name, "gemm_no_tail_cut") == 0 ? &g_knobs.gemm_no_tail_cut
+                : strcmp(name, "gemm_no_small") == 0    ? &g_knobs.gemm_no_small
                 : strcmp(name, "moe_no_fuse") == 0      ? &g_knobs.moe_no_fuse
                                                         : nullptr;
     if (!flag) return fail(QMM_ERR_INVALID_ARG, "qmm_debug_config: unknown knob \"%s\"", name);

@@ -100,6 +100,7 @@ struct DebugKnobs {
     int gemv_no_cluster;            // split-K GEMV through workspace partial sums and a second kernel
     int gemm_bn, gemm_units;        // token tile / (tile, k-block) units per block of the dense GEMM; 0: the plan decides
     int gemm_no_tail_cut;           // leave the tiles of the last, partly filled round whole
+    int gemm_no_small;              // M <= 8 through the tensor-core prefill kernel instead of the few-token kernel
     int moe_no_fuse;                // decode-sized MoE layers as four separate launches
 };
 extern DebugKnobs g_knobs;

@@ -308,6 +308,11 @@ static GemmPlan gemm_plan(int64_t M, int64_t N, int64_t K)
     return p;
 }
 
+// defined in qmm_gemm_small.cu
+bool gemm_small_supported(int fmt, int64_t M);
+qmm_status launch_gemm_small(int fmt, const void* packed, int64_t N, int64_t K, const uint16_t* X, int64_t ldx,
+                             uint16_t* Y, int64_t ldy, int64_t M, cudaStream_t st);
+
 size_t gemm_workspace_bytes(int, int64_t M, int64_t N, int64_t K)
 {
     if (M == 0) return kGemmWsHeader;
@@ -318,6 +323,8 @@ size_t gemm_workspace_bytes(int, int64_t M, int64_t N, int64_t K)
 qmm_status launch_gemm(int fmt, const void* packed, int64_t N, int64_t K, const uint16_t* X, int64_t ldx,
                        uint16_t* Y, int64_t ldy, int64_t M, void* ws, cudaStream_t st)
 {
+    // a handful of tokens: bound by streaming W once, like decode -- the few-token kernel
+    if (gemm_small_supported(fmt, M)) return launch_gemm_small(fmt, packed, N, K, X, ldx, Y, ldy, M, st);
     const GemmPlan plan = gemm_plan(M, N, K);
     const int bn = plan.bn, na = plan.na;
     CUtensorMap map;

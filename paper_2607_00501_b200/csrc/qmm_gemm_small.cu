@@ -1,0 +1,448 @@
+// qmm_gemm_small.cu -- Y[M, N] = X[M, K] W^T for a handful of tokens (M <= 8): a decode step of a
+// small batch, or the tail of a prefill chunk.
+//
+// At these sizes the product is bound by streaming W once, exactly like the single-token product
+// (Sec. 3.3: decode is memory-bound), so it runs on the decode kernels' inner product rather than on
+// the prefill kernel, whose 128-row tiles and fp16 expansion cost the same whatever M is: codes are
+// streamed into registers, unpacked once, and multiplied by eight tokens per warp-level MMA (see FragRegs).
+//
+// Work item = (pair of row groups, K split): 64 outputs for every token; the block's warps split the
+// item's K range, their sums are added in warp order.  K is split across blocks only when the row
+// groups alone cannot cover the SMs; the blocks of an item are then a thread-block cluster and add
+// their sums through the shared memory of its first block, in split order: no workspace, no second
+// launch, the same bits on every call.
+#include "qmm_gemv_core.cuh"
+
+namespace qmm {
+
+constexpr int kSmallUnroll = 2;             // tile pairs in flight per warp
+constexpr int kSmallWarps = 8;
+constexpr int kSmallMaxSplits = 8;          // portable cluster size
+constexpr int kSmallMaxTokens = 8;          // one group of eight tokens per MMA
+
+// How a warp multiplies a tile pair by up to eight tokens with one MMA per 256 weights.
+//
+// The single-token kernels give every lane one matrix row and pay for it with a sparse B operand.
+// Here the codes are streamed the same way (32 bytes per lane = one row of the tile, the widest loads)
+// but then transposed inside the warp through a 2 KiB patch of shared memory: every lane stores its
+// row, and ldmatrix hands lane l = 4g + t, of each of the four rows 4g .. 4g+3 of both row groups
+// (P, Q), the packed words t and t + 4: one 8-k chunk of each 32-element block (Q8: 4-k chunks of the
+// tile's one block).  For row i of the four, the lane's words are then exactly its share of a 16 x 16
+// A fragment whose MMA row g is matrix row 4g+i of P, MMA row g+8 the same row of Q, and whose 16 k
+// are the chunk t of every lane t -- all inside one quantisation block, so the block's scale still
+// multiplies the fp32 sum afterwards and the integer products stay exact.  B is dense: lane (g, t)
+// supplies token g's activations for chunk t (one 16-byte shared-memory load per block and token group,
+// shared by the four rows).  D[g][2t, 2t+1] / D[g+8][..] are row 4g+i of P / Q for tokens 2t, 2t+1.
+template <int FMT>
+struct SmallSlot {                                              // one tile pair in flight
+    static constexpr int HW = FMT == QMM_Q5 || FMT == QMM_Q6 ? 2 : 0;
+    u32x8 cp, cq;                                               // the lane's row of P and of Q
+    uint32_t hp[4][HW ? HW : 1], hq[4][HW ? HW : 1];            // high-bit words covering words t, t+4 of rows 4g+i (Q5 / Q6)
+    uint32_t sp[FMT == QMM_Q8 ? 2 : 4], sq[FMT == QMM_Q8 ? 2 : 4];   // scales of rows 4g .. 4g+3 (fp16; Q8: one per row, else two)
+};
+
+template <int FMT>
+struct FragRegs {
+    uint32_t wp[4][2], wq[4][2];                                // [row i][block b]: word t + 4b of row 4g+i
+};
+
+__device__ __forceinline__ uint2 ld_nc_u32x2(const void* p)
+{
+    uint2 r;
+    asm volatile("ld.global.nc.v2.u32 {%0,%1}, [%2];" : "=r"(r.x), "=r"(r.y) : "l"(p));
+    return r;
+}
+__device__ __forceinline__ uint4 ld_nc_u32x4(const void* p)
+{
+    uint4 r;
+    asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+    return r;
+}
+
+// tile_p / tile_q: start of the tile of row group P / Q (not offset by lane).
+template <int FMT>
+__device__ __forceinline__ void load_slot(SmallSlot<FMT>& r, const uint8_t* tile_p, const uint8_t* tile_q, int lane)
+{
+    const int g = lane >> 2, t = lane & 3;
+    r.cp = ld_stream_256(tile_p + 32 * lane);
+    r.cq = ld_stream_256(tile_q + 32 * lane);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int row = 4 * g + i;
+        if constexpr (FMT == QMM_Q5) {                          // word j is covered by high-bit word j / 4
+            const uint2 a = ld_nc_u32x2(tile_p + kTileCodeBytes + 8 * row), b = ld_nc_u32x2(tile_q + kTileCodeBytes + 8 * row);
+            r.hp[i][0] = a.x, r.hp[i][1] = a.y, r.hq[i][0] = b.x, r.hq[i][1] = b.y;
+        } else if constexpr (FMT == QMM_Q6) {                   // word j is covered by high-bit word j / 2
+            r.hp[i][0] = ld_nc_u32(tile_p + kTileCodeBytes + 16 * row + 4 * (t >> 1));
+            r.hp[i][1] = ld_nc_u32(tile_p + kTileCodeBytes + 16 * row + 4 * (t >> 1) + 8);
+            r.hq[i][0] = ld_nc_u32(tile_q + kTileCodeBytes + 16 * row + 4 * (t >> 1));
+            r.hq[i][1] = ld_nc_u32(tile_q + kTileCodeBytes + 16 * row + 4 * (t >> 1) + 8);
+        }
+    }
+    if constexpr (FMT == QMM_Q8) {
+        const uint2 a = ld_nc_u32x2(tile_p + Fmt<FMT>::scale_off + 8 * g), b = ld_nc_u32x2(tile_q + Fmt<FMT>::scale_off + 8 * g);
+        r.sp[0] = a.x, r.sp[1] = a.y, r.sq[0] = b.x, r.sq[1] = b.y;
+    } else {
+        const uint4 a = ld_nc_u32x4(tile_p + Fmt<FMT>::scale_off + 16 * g), b = ld_nc_u32x4(tile_q + Fmt<FMT>::scale_off + 16 * g);
+        r.sp[0] = a.x, r.sp[1] = a.y, r.sp[2] = a.z, r.sp[3] = a.w;
+        r.sq[0] = b.x, r.sq[1] = b.y, r.sq[2] = b.z, r.sq[3] = b.w;
+    }
+}
+
+// The transposition.  `patch`: the warp's 2 KiB of shared memory as a 32-bit shared address.  Row r of
+// the tile is stored as two 16-byte halves at 128 (r / 4) + 16 (((2 (r % 4) + h)) ^ (r / 4)): the XOR
+// spreads the eight rows that one ldmatrix matrix reads (rows 4g+i, g = 0..7, same i and h) over all
+// banks, and keeps the stores of a quarter-warp apart as well.  Matrix (i, h) of eight 16-byte rows
+// then gives lane (g, t) the 32-bit word t of half h of row 4g+i.
+__device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+{
+    asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& d0, uint32_t& d1, uint32_t& d2, uint32_t& d3)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(d0), "=r"(d1), "=r"(d2), "=r"(d3) : "r"(addr) : "memory");
+}
+
+template <int FMT>
+__device__ __forceinline__ void transpose_slot(const SmallSlot<FMT>& r, FragRegs<FMT>& f, uint32_t patch, int lane)
+{
+    const int wg = lane >> 2, wi = lane & 3;                    // the row this lane stores: 4 wg + wi
+    const uint32_t st0 = patch + 128 * wg + 16 * ((2 * wi) ^ wg), st1 = patch + 128 * wg + 16 * ((2 * wi + 1) ^ wg);
+    const int mg = lane & 7, mj = lane >> 3;                    // ldmatrix: this lane addresses row mg of matrix mj
+    const uint32_t ld0 = patch + 128 * mg + 16 * ((2 * mj) ^ mg), ld1 = patch + 128 * mg + 16 * ((2 * mj + 1) ^ mg);
+    __syncwarp();                                               // the previous tile's reads are done
+    sts128(st0, r.cp.v[0], r.cp.v[1], r.cp.v[2], r.cp.v[3]);
+    sts128(st1, r.cp.v[4], r.cp.v[5], r.cp.v[6], r.cp.v[7]);
+    sts128(st0 + 1024, r.cq.v[0], r.cq.v[1], r.cq.v[2], r.cq.v[3]);
+    sts128(st1 + 1024, r.cq.v[4], r.cq.v[5], r.cq.v[6], r.cq.v[7]);
+    __syncwarp();
+    ldmatrix_x4(ld0, f.wp[0][0], f.wp[1][0], f.wp[2][0], f.wp[3][0]);
+    ldmatrix_x4(ld1, f.wp[0][1], f.wp[1][1], f.wp[2][1], f.wp[3][1]);
+    ldmatrix_x4(ld0 + 1024, f.wq[0][0], f.wq[1][0], f.wq[2][0], f.wq[3][0]);
+    ldmatrix_x4(ld1 + 1024, f.wq[0][1], f.wq[1][1], f.wq[2][1], f.wq[3][1]);
+}
+
+// q56_word_to_h2 for a word whose index within its high-bit word (jq = j & 3 for Q5, j & 1 for Q6) is
+// known only at run time: the high-bit word is first shifted down to that word's bits, the per-pair
+// shifts are then constants.
+template <int FMT>
+__device__ __forceinline__ void q56_word_to_h2_dyn(uint32_t w, uint32_t H, int jq, __half2 (&q)[4], const Q4Consts& k)
+{
+    constexpr bool Q5 = FMT == QMM_Q5;
+    const __half2 c_lo = as_h2(Q5 ? 0x64106410u : 0x64206420u);          // 1040 / 1056
+    const __half2 c16th = as_h2(0x2C002C00u);
+    const __half2 c_hi = as_h2(Q5 ? 0xD500D500u : 0xD600D600u);          // -80 / -96
+    const uint32_t m_lo = Q5 ? 0x00100010u : 0x00300030u, m_hi = Q5 ? 0x01000100u : 0x03000300u;
+    const uint32_t w8 = w >> 8;
+    const uint32_t Hs = H >> (Q5 ? 4 * jq : 8 * jq);
+    auto hi_at = [&](int p, int target) -> uint32_t {                      // pair p's high bits moved to bit `target`
+        const int s = (Q5 ? p : 2 * p) - target;
+        return s >= 0 ? Hs >> s : Hs << -s;
+    };
+    q[0] = __hsub2(as_h2(and_or(hi_at(0, 4), m_lo, and_or(w, k.mask_lo, k.magic))), c_lo);
+    q[1] = __hfma2(as_h2(and_or(hi_at(1, 8), m_hi, and_or(w, k.mask_hi, k.magic))), c16th, c_hi);
+    q[2] = __hsub2(as_h2(and_or(hi_at(2, 4), m_lo, and_or(w8, k.mask_lo, k.magic))), c_lo);
+    q[3] = __hfma2(as_h2(and_or(hi_at(3, 8), m_hi, and_or(w8, k.mask_hi, k.magic))), c16th, c_hi);
+}
+
+// xg[n]: the lane's activation pointer of token group n (token 8n+g, or zeros), in uint4 units;
+// x_off: first chunk of this tile.  acc[n][i][0..1]: row 4g+i of P for tokens 8n+2t, 8n+2t+1;
+// acc[n][i][2..3]: the same row of Q.
+template <int FMT, int NG>
+__device__ __forceinline__ void frag_mma(const SmallSlot<FMT>& r, const FragRegs<FMT>& f, const uint4* const (&xg)[NG], int x_off, int t,
+                                         float (&acc)[NG][4][4], const Q4Consts& kc)
+{
+    constexpr int BLOCKS = FMT == QMM_Q8 ? 1 : 2;
+#pragma unroll
+    for (int b = 0; b < BLOCKS; ++b) {
+        uint4 xv[NG];
+#pragma unroll
+        for (int n = 0; n < NG; ++n) {
+            if constexpr (FMT == QMM_Q8) {
+                // words t and 4 + t of the row are k = 4t .. 4t+3 and 16 + 4t .. 16 + 4t+3 of the tile
+                const uint2* x2 = reinterpret_cast<const uint2*>(xg[n] + x_off);
+                const uint2 lo = x2[t], hi = x2[4 + t];
+                xv[n] = make_uint4(lo.x, lo.y, hi.x, hi.y);
+            } else {
+                xv[n] = xg[n][x_off + 4 * b + t];
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            __half2 p[4], q[4];
+            if constexpr (FMT == QMM_Q8) {
+                __half2 a[2];
+                q8_word_to_h2(f.wp[i][0], a);
+                p[0] = a[0], p[1] = a[1];
+                q8_word_to_h2(f.wp[i][1], a);
+                p[2] = a[0], p[3] = a[1];
+                q8_word_to_h2(f.wq[i][0], a);
+                q[0] = a[0], q[1] = a[1];
+                q8_word_to_h2(f.wq[i][1], a);
+                q[2] = a[0], q[3] = a[1];
+            } else if constexpr (FMT == QMM_Q4) {
+                q4_word_to_h2(f.wp[i][b], p, kc);
+                q4_word_to_h2(f.wq[i][b], q, kc);
+            } else {
+                // word j = t + 4b of the row; only j's position inside its high-bit word matters
+                const int jq = FMT == QMM_Q5 ? (t & 3) : (t & 1);
+                q56_word_to_h2_dyn<FMT>(f.wp[i][b], r.hp[i][b], jq, p, kc);
+                q56_word_to_h2_dyn<FMT>(f.wq[i][b], r.hq[i][b], jq, q, kc);
+            }
+            float dp, dq;
+            if constexpr (FMT == QMM_Q8) {
+                const __half2 hp2 = as_h2(r.sp[i >> 1]), hq2 = as_h2(r.sq[i >> 1]);
+                dp = __half2float((i & 1) ? __high2half(hp2) : __low2half(hp2));
+                dq = __half2float((i & 1) ? __high2half(hq2) : __low2half(hq2));
+            } else {
+                dp = __half2float(b ? __high2half(as_h2(r.sp[i])) : __low2half(as_h2(r.sp[i])));
+                dq = __half2float(b ? __high2half(as_h2(r.sq[i])) : __low2half(as_h2(r.sq[i])));
+            }
+#pragma unroll
+            for (int n = 0; n < NG; ++n) {
+                float c[4];
+                mma16816_zero(c, as_u32(p[0]), as_u32(q[0]), as_u32(p[1]), as_u32(q[1]), xv[n].x, xv[n].y);
+                mma16816(c, as_u32(p[2]), as_u32(q[2]), as_u32(p[3]), as_u32(q[3]), xv[n].z, xv[n].w);
+                acc[n][i][0] = fmaf(dp, c[0], acc[n][i][0]);
+                acc[n][i][1] = fmaf(dp, c[1], acc[n][i][1]);
+                acc[n][i][2] = fmaf(dq, c[2], acc[n][i][2]);
+                acc[n][i][3] = fmaf(dq, c[3], acc[n][i][3]);
+            }
+        }
+    }
+}
+
+// Dynamic shared memory: WARPS * 2 KiB of transposition patches, activations of the block's K range
+// for M tokens, the same number of fp16 zeros once, WARPS * 8*NG * 64 floats for the warps' sums, and
+// (cluster form, used in the first block) 2 * kSmallMaxSplits * 8*NG * 64 floats.
+template <int FMT, int NG>
+__global__ void __launch_bounds__(kSmallWarps * 32, 2)
+gemm_small_kernel(const uint8_t* __restrict__ packed, const uint16_t* __restrict__ X, int64_t ldx,
+                  uint16_t* __restrict__ Y, int64_t ldy, int M, int K, int tiles_per_row, int splits, int items)
+{
+    constexpr int WARPS = kSmallWarps, NT = 8 * NG;
+    constexpr int TB = Fmt<FMT>::tile_bytes;
+    constexpr int XV = Fmt<FMT>::tile_k / 8;                    // uint4 of activations per tile
+    constexpr int STEP = kSmallUnroll * WARPS;
+    extern __shared__ uint4 smem[];
+    const int tps = tiles_per_row / splits;                     // tiles per item
+    const int kr8 = tps * XV;                                   // uint4 of one token's activations in the block's K range
+    uint4* xs = smem + WARPS * 128;                             // [M][kr8], behind the warps' patches
+    uint4* zs = xs + M * kr8;                                   // [kr8]
+    float* red = reinterpret_cast<float*>(zs + kr8);
+    float* cred = red + WARPS * NT * 64;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, t4 = lane & 3;
+    const bool clustered = splits > 1;
+    int cluster_round = 0;
+
+    const size_t group_bytes = (size_t)tiles_per_row * TB;
+    int item = blockIdx.x;
+    int pair = item / splits;
+    const int s = item - pair * splits;                         // the same for every item of this block (grid = whole clusters)
+    int t = s * tps + warp;
+    const int t_end = (s + 1) * tps;
+    const uint8_t* tiles_p = packed + (size_t)(2 * pair) * group_bytes;
+
+    SmallSlot<FMT> r[kSmallUnroll];
+    const uint32_t patch = static_cast<uint32_t>(__cvta_generic_to_shared(smem + warp * 128));
+    auto load_group = [&]() {
+#pragma unroll
+        for (int u = 0; u < kSmallUnroll; ++u) {
+            const int tt = t + u * WARPS;
+            if (tt < t_end) load_slot<FMT>(r[u], tiles_p + (size_t)tt * TB, tiles_p + (size_t)tt * TB + group_bytes, lane);
+        }
+    };
+    if (item < items) load_group();                             // weights never depend on the previous kernel
+
+    pdl_launch_dependents();
+    pdl_wait();                                                 // X may come from the previous kernel
+    for (int i = threadIdx.x; i < kr8; i += WARPS * 32) zs[i] = make_uint4(0u, 0u, 0u, 0u);
+    {
+        // all of a thread's loads in flight before the first store (the rows are short: latency, not bandwidth)
+        const int total = M * kr8;
+        const uint4* x0 = reinterpret_cast<const uint4*>(X) + s * kr8;
+        const int64_t ldx8 = ldx / 8;
+        for (int base = threadIdx.x; base < total; base += 4 * WARPS * 32) {
+            uint4 v[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int i = base + u * WARPS * 32;
+                if (i < total) {
+                    const int m = i / kr8;
+                    v[u] = x0[m * ldx8 + (i - m * kr8)];
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int i = base + u * WARPS * 32;
+                if (i < total) xs[i] = v[u];
+            }
+        }
+    }
+    __syncthreads();
+    const uint4* xg[NG];
+#pragma unroll
+    for (int n = 0; n < NG; ++n) xg[n] = 8 * n + g < M ? xs + (8 * n + g) * kr8 : zs;
+    Q4Consts kc;
+    kc.init();
+
+    while (item < items) {
+        float acc[NG][4][4];
+#pragma unroll
+        for (int n = 0; n < NG; ++n)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) acc[n][i][0] = acc[n][i][1] = acc[n][i][2] = acc[n][i][3] = 0.f;
+        while (t < t_end) {
+#pragma unroll
+            for (int u = 0; u < kSmallUnroll; ++u) {
+                const int tt = t + u * WARPS;
+                if (tt < t_end) {                               // (warp-uniform)
+                    FragRegs<FMT> f;
+                    transpose_slot<FMT>(r[u], f, patch, lane);
+                    frag_mma<FMT, NG>(r[u], f, xg, (tt - s * tps) * XV, t4, acc, kc);
+                }
+            }
+            t += STEP;
+            if (t < t_end) load_group();
+        }
+        const int done_pair = pair;
+        item += gridDim.x;
+        if (item < items) {                                     // next item's loads fly during the reduction
+            pair = item / splits;
+            t = s * tps + warp;
+            tiles_p = packed + (size_t)(2 * pair) * group_bytes;
+            load_group();
+        }
+        // red[warp][token][64]: rows 0..31 of P, then of Q
+#pragma unroll
+        for (int n = 0; n < NG; ++n)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                float* w = red + (warp * NT + 8 * n + 2 * t4) * 64 + 4 * g + i;
+                w[0] = acc[n][i][0];
+                w[64] = acc[n][i][1];
+                w[32] = acc[n][i][2];
+                w[64 + 32] = acc[n][i][3];
+            }
+        __syncthreads();
+        const int live = (M < NT ? M : NT) * 64;                // sums of tokens that exist
+        if (!clustered) {
+            for (int i = threadIdx.x; i < live; i += WARPS * 32) {
+                float sum = red[i];
+#pragma unroll
+                for (int w = 1; w < WARPS; ++w) sum += red[w * NT * 64 + i];
+                Y[(size_t)(i >> 6) * ldy + done_pair * 64 + (i & 63)] = __half_as_ushort(__float2half_rn(sum));
+            }
+        } else {
+            // every block of the cluster runs the same sequence of pairs, one split each
+            float* slot = cred + (cluster_round & 1) * (kSmallMaxSplits * NT * 64);
+            for (int i = threadIdx.x; i < live; i += WARPS * 32) {
+                float sum = red[i];
+#pragma unroll
+                for (int w = 1; w < WARPS; ++w) sum += red[w * NT * 64 + i];
+                st_cluster_rank0(slot + s * NT * 64 + i, sum);
+            }
+            cluster_sync();
+            if (s == 0) {
+                for (int i = threadIdx.x; i < live; i += WARPS * 32) {
+                    float total = slot[i];
+                    for (int sp = 1; sp < splits; ++sp) total += slot[sp * NT * 64 + i];
+                    Y[(size_t)(i >> 6) * ldy + done_pair * 64 + (i & 63)] = __half_as_ushort(__float2half_rn(total));
+                }
+            }
+            ++cluster_round;                                    // two slots: the next item's sums do not wait for this read
+        }
+        __syncthreads();
+    }
+}
+
+// ------------------------------------------------------------------ host
+
+bool gemm_small_supported(int fmt, int64_t M)
+{
+    (void)fmt;
+    return M >= 1 && M <= kSmallMaxTokens && !g_knobs.gemm_no_small;
+}
+
+qmm_status launch_gemv(int fmt, const void* packed, int64_t N, int64_t K, const uint16_t* x, uint16_t* y,
+                       void* ws, bool allow_cluster, cudaStream_t st);
+size_t gemv_workspace_bytes(int fmt, int64_t N, int64_t K, bool allow_cluster);
+
+struct SmallPlan {
+    int splits, grid;
+    size_t smem;
+};
+
+static SmallPlan small_plan(int fmt, int64_t M, int64_t N, int64_t K)
+{
+    const int ng = (int)((M + 7) / 8), nt = 8 * ng;
+    const int tpr = (int)(K / tile_k_of(fmt));
+    const int pairs = (int)(N / 64);
+    const int per_sm = 2;
+    auto smem_of = [&](int splits) {
+        return (size_t)kSmallWarps * 2048 + (size_t)(M + 1) * (size_t)(K / splits) * 2 + (size_t)kSmallWarps * nt * 64 * sizeof(float) +
+               (splits > 1 ? (size_t)2 * kSmallMaxSplits * nt * 64 * sizeof(float) : 0);
+    };
+    int splits = 1;
+    // split K while the pairs alone leave SMs without a block, every warp keeps a tile, and the cluster stays small
+    while (pairs * splits < kNumSMs * per_sm && tpr % (splits * 2) == 0 && tpr / (splits * 2) >= kSmallWarps / 2 && splits < 4) splits *= 2;
+    // ... and, whatever the grid, until the activations of the block's K range fit in shared memory
+    while (smem_of(splits) > 200 * 1024 && tpr % (splits * 2) == 0 && splits < kSmallMaxSplits) splits *= 2;
+    SmallPlan p;
+    p.splits = splits;
+    p.smem = smem_of(splits);
+    const int items = pairs * splits;
+    const int cap = kNumSMs * per_sm / splits * splits;
+    p.grid = items < cap ? items : cap;
+    return p;
+}
+
+template <int FMT, int NG>
+static qmm_status launch_small_t(const SmallPlan& p, const void* packed, int64_t N, int64_t K, const uint16_t* X, int64_t ldx,
+                                 uint16_t* Y, int64_t ldy, int64_t M, cudaStream_t st)
+{
+    auto kern = gemm_small_kernel<FMT, NG>;
+    if (p.smem > 227 * 1024) return fail(QMM_ERR_UNSUPPORTED, "qmm_gemm: K=%lld is too large for the few-token kernel", (long long)K);
+    if (p.smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem);
+        if (e != cudaSuccess) return check_cuda(e, "qmm_gemm few-token kernel shared memory size");
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)p.grid);
+    cfg.blockDim = dim3(kSmallWarps * 32);
+    cfg.dynamicSmemBytes = p.smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = (unsigned)p.splits;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = p.splits > 1 ? 2 : 1;
+    const int tpr = (int)(K / Fmt<FMT>::tile_k);
+    const int items = (int)(N / 64) * p.splits;
+    return check_cuda(cudaLaunchKernelEx(&cfg, kern, (const uint8_t*)packed, X, ldx, Y, ldy, (int)M, (int)K, tpr, p.splits, items),
+                      "qmm_gemm few-token kernel launch");
+}
+
+qmm_status launch_gemm_small(int fmt, const void* packed, int64_t N, int64_t K, const uint16_t* X, int64_t ldx,
+                             uint16_t* Y, int64_t ldy, int64_t M, cudaStream_t st)
+{
+    // one token: the single-token kernel (its cluster form needs no workspace)
+    if (M == 1 && gemv_workspace_bytes(fmt, N, K, true) == 0) return launch_gemv(fmt, packed, N, K, X, Y, nullptr, true, st);
+    const SmallPlan p = small_plan(fmt, M, N, K);
+    const int ng = (int)((M + 7) / 8);
+#define QMM_SMALL_CASE(F, G) \
+    if (fmt == F && ng == G) return launch_small_t<F, G>(p, packed, N, K, X, ldx, Y, ldy, M, st);
+    QMM_SMALL_CASE(QMM_Q4, 1)
+    QMM_SMALL_CASE(QMM_Q8, 1)
+    QMM_SMALL_CASE(QMM_Q5, 1)
+    QMM_SMALL_CASE(QMM_Q6, 1)
+#undef QMM_SMALL_CASE
+    return fail(QMM_ERR_UNSUPPORTED, "qmm_gemm: no few-token kernel for format %d, M=%lld", fmt, (long long)M);
+}
+
+}  // namespace qmm

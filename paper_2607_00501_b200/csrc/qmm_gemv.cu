@@ -30,21 +30,6 @@ constexpr int kUnroll = QMM_GEMV_UNROLL;   // tile pairs in flight per warp (4 x
 constexpr int kMaxClusterSplits = 8;                            // portable cluster size (room in shared memory)
 constexpr int kPlanClusterSplits = 4;                           // what the plan asks for: clusters of 8 measured slower to schedule
 
-// Store to the same shared-memory location in the cluster's first block.
-__device__ __forceinline__ void st_cluster_rank0(float* local_ptr, float v)
-{
-    uint32_t local = static_cast<uint32_t>(__cvta_generic_to_shared(local_ptr)), remote;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, 0;" : "=r"(remote) : "r"(local));
-    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(v) : "memory");
-}
-
-// Barrier over all threads of the cluster (hardware barrier; the blocks of a cluster are co-scheduled).
-__device__ __forceinline__ void cluster_sync()
-{
-    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-
 // Codes and scales of kUnroll tile pairs held in registers.
 template <int FMT>
 struct TileRegs {
