@@ -3,8 +3,9 @@
 //
 // At these sizes the product is bound by streaming W once, exactly like the single-token product
 // (Sec. 3.3: decode is memory-bound), so it runs on the decode kernels' inner product rather than on
-// the prefill kernel, whose 128-row tiles and fp16 expansion cost the same whatever M is: codes are
-// streamed into registers, unpacked once, and multiplied by eight tokens per warp-level MMA (see FragRegs).
+// the prefill kernel, whose 128-row tiles and fp16 expansion cost the same whatever M is: the codes are
+// streamed once, unpacked once, and multiplied by all eight tokens in one warp-level MMA per 256
+// weights (see FragRegs).
 //
 // Work item = (pair of row groups, K split): 64 outputs for every token; the block's warps split the
 // item's K range, their sums are added in warp order.  K is split across blocks only when the row
@@ -15,7 +16,6 @@
 
 namespace qmm {
 
-constexpr int kSmallUnroll = 2;             // tile pairs in flight per warp
 constexpr int kSmallWarps = 8;
 constexpr int kSmallMaxSplits = 8;          // portable cluster size
 constexpr int kSmallMaxTokens = 8;          // one group of eight tokens per MMA
@@ -23,20 +23,17 @@ constexpr int kSmallMaxTokens = 8;          // one group of eight tokens per MMA
 // How a warp multiplies a tile pair by up to eight tokens with one MMA per 256 weights.
 //
 // The single-token kernels give every lane one matrix row and pay for it with a sparse B operand.
-// Here the codes are streamed the same way (32 bytes per lane = one row of the tile, the widest loads)
-// but then transposed inside the warp through a 2 KiB patch of shared memory: every lane stores its
-// row, and ldmatrix hands lane l = 4g + t, of each of the four rows 4g .. 4g+3 of both row groups
-// (P, Q), the packed words t and t + 4: one 8-k chunk of each 32-element block (Q8: 4-k chunks of the
-// tile's one block).  For row i of the four, the lane's words are then exactly its share of a 16 x 16
+// Here every lane still moves its own row of the tile (32 contiguous bytes), but into shared memory,
+// transposed on the way: ldmatrix then hands lane l = 4g + t, of each of the four rows 4g .. 4g+3 of
+// both row groups (P, Q), the packed words t and t + 4: one 8-k chunk of each 32-element block (Q8:
+// 4-k chunks of the tile's one block).  For row i of the four, the lane's words are then exactly its share of a 16 x 16
 // A fragment whose MMA row g is matrix row 4g+i of P, MMA row g+8 the same row of Q, and whose 16 k
 // are the chunk t of every lane t -- all inside one quantisation block, so the block's scale still
 // multiplies the fp32 sum afterwards and the integer products stay exact.  B is dense: lane (g, t)
-// supplies token g's activations for chunk t (one 16-byte shared-memory load per block and token group,
-// shared by the four rows).  D[g][2t, 2t+1] / D[g+8][..] are row 4g+i of P / Q for tokens 2t, 2t+1.
+// supplies token g's activations for chunk t (one 16-byte load per block, shared by the four rows).  D[g][2t, 2t+1] / D[g+8][..] are row 4g+i of P / Q for tokens 2t, 2t+1.
 template <int FMT>
-struct SmallSlot {                                              // one tile pair in flight
+struct SmallSlot {                                              // what a lane needs of a tile pair beside the codes
     static constexpr int HW = FMT == QMM_Q5 || FMT == QMM_Q6 ? 2 : 0;
-    u32x8 cp, cq;                                               // the lane's row of P and of Q
     uint32_t hp[4][HW ? HW : 1], hq[4][HW ? HW : 1];            // high-bit words covering words t, t+4 of rows 4g+i (Q5 / Q6)
     uint32_t sp[FMT == QMM_Q8 ? 2 : 4], sq[FMT == QMM_Q8 ? 2 : 4];   // scales of rows 4g .. 4g+3 (fp16; Q8: one per row, else two)
 };
@@ -59,67 +56,13 @@ __device__ __forceinline__ uint4 ld_nc_u32x4(const void* p)
     return r;
 }
 
-// tile_p / tile_q: start of the tile of row group P / Q (not offset by lane).
-template <int FMT>
-__device__ __forceinline__ void load_slot(SmallSlot<FMT>& r, const uint8_t* tile_p, const uint8_t* tile_q, int lane)
-{
-    const int g = lane >> 2, t = lane & 3;
-    r.cp = ld_stream_256(tile_p + 32 * lane);
-    r.cq = ld_stream_256(tile_q + 32 * lane);
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int row = 4 * g + i;
-        if constexpr (FMT == QMM_Q5) {                          // word j is covered by high-bit word j / 4
-            const uint2 a = ld_nc_u32x2(tile_p + kTileCodeBytes + 8 * row), b = ld_nc_u32x2(tile_q + kTileCodeBytes + 8 * row);
-            r.hp[i][0] = a.x, r.hp[i][1] = a.y, r.hq[i][0] = b.x, r.hq[i][1] = b.y;
-        } else if constexpr (FMT == QMM_Q6) {                   // word j is covered by high-bit word j / 2
-            r.hp[i][0] = ld_nc_u32(tile_p + kTileCodeBytes + 16 * row + 4 * (t >> 1));
-            r.hp[i][1] = ld_nc_u32(tile_p + kTileCodeBytes + 16 * row + 4 * (t >> 1) + 8);
-            r.hq[i][0] = ld_nc_u32(tile_q + kTileCodeBytes + 16 * row + 4 * (t >> 1));
-            r.hq[i][1] = ld_nc_u32(tile_q + kTileCodeBytes + 16 * row + 4 * (t >> 1) + 8);
-        }
-    }
-    if constexpr (FMT == QMM_Q8) {
-        const uint2 a = ld_nc_u32x2(tile_p + Fmt<FMT>::scale_off + 8 * g), b = ld_nc_u32x2(tile_q + Fmt<FMT>::scale_off + 8 * g);
-        r.sp[0] = a.x, r.sp[1] = a.y, r.sq[0] = b.x, r.sq[1] = b.y;
-    } else {
-        const uint4 a = ld_nc_u32x4(tile_p + Fmt<FMT>::scale_off + 16 * g), b = ld_nc_u32x4(tile_q + Fmt<FMT>::scale_off + 16 * g);
-        r.sp[0] = a.x, r.sp[1] = a.y, r.sp[2] = a.z, r.sp[3] = a.w;
-        r.sq[0] = b.x, r.sq[1] = b.y, r.sq[2] = b.z, r.sq[3] = b.w;
-    }
-}
-
-// The transposition.  `patch`: the warp's 2 KiB of shared memory as a 32-bit shared address.  Row r of
-// the tile is stored as two 16-byte halves at 128 (r / 4) + 16 (((2 (r % 4) + h)) ^ (r / 4)): the XOR
-// spreads the eight rows that one ldmatrix matrix reads (rows 4g+i, g = 0..7, same i and h) over all
-// banks, and keeps the stores of a quarter-warp apart as well.  Matrix (i, h) of eight 16-byte rows
-// then gives lane (g, t) the 32-bit word t of half h of row 4g+i.
-__device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
-{
-    asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
-}
+// The transposition.  Row r of a tile is stored as two 16-byte halves at
+// 128 (r / 4) + 16 ((2 (r % 4) + h) ^ (r / 4)): the XOR spreads the eight rows that one ldmatrix matrix
+// reads (rows 4g+i, g = 0..7, same i and h) over all banks.  Matrix (i, h) of eight 16-byte rows then
+// gives lane (g, t) the 32-bit word t of half h of row 4g+i.
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& d0, uint32_t& d1, uint32_t& d2, uint32_t& d3)
 {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(d0), "=r"(d1), "=r"(d2), "=r"(d3) : "r"(addr) : "memory");
-}
-
-template <int FMT>
-__device__ __forceinline__ void transpose_slot(const SmallSlot<FMT>& r, FragRegs<FMT>& f, uint32_t patch, int lane)
-{
-    const int wg = lane >> 2, wi = lane & 3;                    // the row this lane stores: 4 wg + wi
-    const uint32_t st0 = patch + 128 * wg + 16 * ((2 * wi) ^ wg), st1 = patch + 128 * wg + 16 * ((2 * wi + 1) ^ wg);
-    const int mg = lane & 7, mj = lane >> 3;                    // ldmatrix: this lane addresses row mg of matrix mj
-    const uint32_t ld0 = patch + 128 * mg + 16 * ((2 * mj) ^ mg), ld1 = patch + 128 * mg + 16 * ((2 * mj + 1) ^ mg);
-    __syncwarp();                                               // the previous tile's reads are done
-    sts128(st0, r.cp.v[0], r.cp.v[1], r.cp.v[2], r.cp.v[3]);
-    sts128(st1, r.cp.v[4], r.cp.v[5], r.cp.v[6], r.cp.v[7]);
-    sts128(st0 + 1024, r.cq.v[0], r.cq.v[1], r.cq.v[2], r.cq.v[3]);
-    sts128(st1 + 1024, r.cq.v[4], r.cq.v[5], r.cq.v[6], r.cq.v[7]);
-    __syncwarp();
-    ldmatrix_x4(ld0, f.wp[0][0], f.wp[1][0], f.wp[2][0], f.wp[3][0]);
-    ldmatrix_x4(ld1, f.wp[0][1], f.wp[1][1], f.wp[2][1], f.wp[3][1]);
-    ldmatrix_x4(ld0 + 1024, f.wq[0][0], f.wq[1][0], f.wq[2][0], f.wq[3][0]);
-    ldmatrix_x4(ld1 + 1024, f.wq[0][1], f.wq[1][1], f.wq[2][1], f.wq[3][1]);
 }
 
 // q56_word_to_h2 for a word whose index within its high-bit word (jq = j & 3 for Q5, j & 1 for Q6) is
@@ -145,11 +88,10 @@ __device__ __forceinline__ void q56_word_to_h2_dyn(uint32_t w, uint32_t H, int j
     q[3] = __hfma2(as_h2(and_or(hi_at(3, 8), m_hi, and_or(w8, k.mask_hi, k.magic))), c16th, c_hi);
 }
 
-// xg[n]: the lane's activation pointer of token group n (token 8n+g, or zeros), in uint4 units;
-// x_off: first chunk of this tile.  acc[n][i][0..1]: row 4g+i of P for tokens 8n+2t, 8n+2t+1;
-// acc[n][i][2..3]: the same row of Q.
+// One tile pair times the lane's activations (xr[b][n]: block b, token group n).
+// acc[n][i][0..1]: row 4g+i of P for tokens 8n+2t, 8n+2t+1; acc[n][i][2..3]: the same row of Q.
 template <int FMT, int NG>
-__device__ __forceinline__ void frag_mma(const SmallSlot<FMT>& r, const FragRegs<FMT>& f, const uint4* const (&xg)[NG], int x_off, int t,
+__device__ __forceinline__ void frag_mma_x(const SmallSlot<FMT>& r, const FragRegs<FMT>& f, const uint4 (&xr)[FMT == QMM_Q8 ? 1 : 2][NG], int t,
                                          float (&acc)[NG][4][4], const Q4Consts& kc)
 {
     constexpr int BLOCKS = FMT == QMM_Q8 ? 1 : 2;
@@ -157,16 +99,7 @@ __device__ __forceinline__ void frag_mma(const SmallSlot<FMT>& r, const FragRegs
     for (int b = 0; b < BLOCKS; ++b) {
         uint4 xv[NG];
 #pragma unroll
-        for (int n = 0; n < NG; ++n) {
-            if constexpr (FMT == QMM_Q8) {
-                // words t and 4 + t of the row are k = 4t .. 4t+3 and 16 + 4t .. 16 + 4t+3 of the tile
-                const uint2* x2 = reinterpret_cast<const uint2*>(xg[n] + x_off);
-                const uint2 lo = x2[t], hi = x2[4 + t];
-                xv[n] = make_uint4(lo.x, lo.y, hi.x, hi.y);
-            } else {
-                xv[n] = xg[n][x_off + 4 * b + t];
-            }
-        }
+        for (int n = 0; n < NG; ++n) xv[n] = xr[b][n];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             __half2 p[4], q[4];
@@ -212,107 +145,194 @@ __device__ __forceinline__ void frag_mma(const SmallSlot<FMT>& r, const FragRegs
     }
 }
 
-// Dynamic shared memory: WARPS * 2 KiB of transposition patches, activations of the block's K range
-// for M tokens, the same number of fp16 zeros once, WARPS * 8*NG * 64 floats for the warps' sums, and
-// (cluster form, used in the first block) 2 * kSmallMaxSplits * 8*NG * 64 floats.
+// ------------------------------------------------------------------ the ring
+//
+// The tile pairs in flight are held in shared memory, not in registers: every warp owns a ring of
+// kRingStages slots and fills them with 16-byte asynchronous copies -- each lane copies the two halves
+// of its row straight to their transposed places, the first lanes the scale (and high-bit) planes as
+// they are -- one commit group per tile pair.  Nothing is held in registers while the copies fly, so
+// the ring is deep and the loop needs no register double buffer; the copies of the block's next work
+// item run under the reduction of the current one.
+constexpr int kRingStages = 4;
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait()
+{
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr)
+{
+    uint4 r;
+    asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(addr));
+    return r;
+}
+__device__ __forceinline__ uint2 lds64(uint32_t addr)
+{
+    uint2 r;
+    asm volatile("ld.shared.v2.b32 {%0,%1}, [%2];" : "=r"(r.x), "=r"(r.y) : "r"(addr));
+    return r;
+}
+__device__ __forceinline__ uint32_t lds32(uint32_t addr)
+{
+    uint32_t r;
+    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(r) : "r"(addr));
+    return r;
+}
+
+// One tile pair -> one slot (2 * tile bytes: P then Q; the first 1024 bytes of each transposed).
+template <int FMT>
+__device__ __forceinline__ void ring_issue(uint32_t slot, const uint8_t* tile_p, const uint8_t* tile_q, int lane)
+{
+    constexpr int TB = Fmt<FMT>::tile_bytes;
+    constexpr int EX = (TB - kTileCodeBytes) / 16;              // 16-byte chunks behind the codes
+    const int wg = lane >> 2, wi = lane & 3;
+    const uint32_t st0 = slot + 128 * wg + 16 * ((2 * wi) ^ wg), st1 = slot + 128 * wg + 16 * ((2 * wi + 1) ^ wg);
+    cp_async16(st0, tile_p + 32 * lane);
+    cp_async16(st1, tile_p + 32 * lane + 16);
+    cp_async16(st0 + TB, tile_q + 32 * lane);
+    cp_async16(st1 + TB, tile_q + 32 * lane + 16);
+#pragma unroll
+    for (int c0 = 0; c0 < EX; c0 += 32) {
+        const int c = c0 + lane;
+        if (c < EX) {
+            cp_async16(slot + kTileCodeBytes + 16 * c, tile_p + kTileCodeBytes + 16 * c);
+            cp_async16(slot + TB + kTileCodeBytes + 16 * c, tile_q + kTileCodeBytes + 16 * c);
+        }
+    }
+}
+
+// Slot -> registers: the lane's share of the A fragments, the scales and high-bit words of its rows.
+template <int FMT>
+__device__ __forceinline__ void ring_read(uint32_t slot, SmallSlot<FMT>& r, FragRegs<FMT>& f, int lane)
+{
+    constexpr int TB = Fmt<FMT>::tile_bytes;
+    const int g = lane >> 2, t = lane & 3;
+    const int mg = lane & 7, mj = lane >> 3;                    // ldmatrix: this lane addresses row mg of matrix mj
+    const uint32_t ld0 = slot + 128 * mg + 16 * ((2 * mj) ^ mg), ld1 = slot + 128 * mg + 16 * ((2 * mj + 1) ^ mg);
+    ldmatrix_x4(ld0, f.wp[0][0], f.wp[1][0], f.wp[2][0], f.wp[3][0]);
+    ldmatrix_x4(ld1, f.wp[0][1], f.wp[1][1], f.wp[2][1], f.wp[3][1]);
+    ldmatrix_x4(ld0 + TB, f.wq[0][0], f.wq[1][0], f.wq[2][0], f.wq[3][0]);
+    ldmatrix_x4(ld1 + TB, f.wq[0][1], f.wq[1][1], f.wq[2][1], f.wq[3][1]);
+    if constexpr (FMT == QMM_Q8) {
+        const uint2 a = lds64(slot + Fmt<FMT>::scale_off + 8 * g), b = lds64(slot + TB + Fmt<FMT>::scale_off + 8 * g);
+        r.sp[0] = a.x, r.sp[1] = a.y, r.sq[0] = b.x, r.sq[1] = b.y;
+    } else {
+        const uint4 a = lds128(slot + Fmt<FMT>::scale_off + 16 * g), b = lds128(slot + TB + Fmt<FMT>::scale_off + 16 * g);
+        r.sp[0] = a.x, r.sp[1] = a.y, r.sp[2] = a.z, r.sp[3] = a.w;
+        r.sq[0] = b.x, r.sq[1] = b.y, r.sq[2] = b.z, r.sq[3] = b.w;
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int row = 4 * g + i;
+        if constexpr (FMT == QMM_Q5) {
+            const uint2 a = lds64(slot + kTileCodeBytes + 8 * row), b = lds64(slot + TB + kTileCodeBytes + 8 * row);
+            r.hp[i][0] = a.x, r.hp[i][1] = a.y, r.hq[i][0] = b.x, r.hq[i][1] = b.y;
+        } else if constexpr (FMT == QMM_Q6) {
+            r.hp[i][0] = lds32(slot + kTileCodeBytes + 16 * row + 4 * (t >> 1));
+            r.hp[i][1] = lds32(slot + kTileCodeBytes + 16 * row + 4 * (t >> 1) + 8);
+            r.hq[i][0] = lds32(slot + TB + kTileCodeBytes + 16 * row + 4 * (t >> 1));
+            r.hq[i][1] = lds32(slot + TB + kTileCodeBytes + 16 * row + 4 * (t >> 1) + 8);
+        }
+    }
+}
+
+// Dynamic shared memory: WARPS * kRingStages slots, WARPS * 8*NG * 64 floats for the warps' sums, and
+// (cluster form, used in the first block) 2 * splits * 8*NG * 64 floats.
 template <int FMT, int NG>
 __global__ void __launch_bounds__(kSmallWarps * 32, 2)
 gemm_small_kernel(const uint8_t* __restrict__ packed, const uint16_t* __restrict__ X, int64_t ldx,
-                  uint16_t* __restrict__ Y, int64_t ldy, int M, int K, int tiles_per_row, int splits, int items)
+                       uint16_t* __restrict__ Y, int64_t ldy, int M, int K, int tiles_per_row, int splits, int items)
 {
     constexpr int WARPS = kSmallWarps, NT = 8 * NG;
     constexpr int TB = Fmt<FMT>::tile_bytes;
-    constexpr int XV = Fmt<FMT>::tile_k / 8;                    // uint4 of activations per tile
-    constexpr int STEP = kSmallUnroll * WARPS;
+    constexpr int SLOT = 2 * TB;
     extern __shared__ uint4 smem[];
     const int tps = tiles_per_row / splits;                     // tiles per item
-    const int kr8 = tps * XV;                                   // uint4 of one token's activations in the block's K range
-    uint4* xs = smem + WARPS * 128;                             // [M][kr8], behind the warps' patches
-    uint4* zs = xs + M * kr8;                                   // [kr8]
-    float* red = reinterpret_cast<float*>(zs + kr8);
+    float* red = reinterpret_cast<float*>(smem + WARPS * kRingStages * SLOT / 16);   // behind the rings
     float* cred = red + WARPS * NT * 64;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, t4 = lane & 3;
     const bool clustered = splits > 1;
     int cluster_round = 0;
+    const uint32_t ring = static_cast<uint32_t>(__cvta_generic_to_shared(smem)) + warp * (kRingStages * SLOT);
 
     const size_t group_bytes = (size_t)tiles_per_row * TB;
-    int item = blockIdx.x;
-    int pair = item / splits;
-    const int s = item - pair * splits;                         // the same for every item of this block (grid = whole clusters)
-    int t = s * tps + warp;
-    const int t_end = (s + 1) * tps;
-    const uint8_t* tiles_p = packed + (size_t)(2 * pair) * group_bytes;
+    const int s = blockIdx.x % splits;                          // the same for every item of this block (grid = whole clusters)
+    const int t_begin = s * tps + warp, t_end = (s + 1) * tps;
+    const bool has_tiles = warp < tps;
 
-    SmallSlot<FMT> r[kSmallUnroll];
-    const uint32_t patch = static_cast<uint32_t>(__cvta_generic_to_shared(smem + warp * 128));
-    auto load_group = [&]() {
-#pragma unroll
-        for (int u = 0; u < kSmallUnroll; ++u) {
-            const int tt = t + u * WARPS;
-            if (tt < t_end) load_slot<FMT>(r[u], tiles_p + (size_t)tt * TB, tiles_p + (size_t)tt * TB + group_bytes, lane);
+    // producer: runs kRingStages tile pairs ahead of the consumer, across work items
+    int p_item = blockIdx.x, p_t = t_begin;
+    auto produce = [&](int stage) {
+        if (has_tiles && p_item < items) {
+            const uint8_t* tp = packed + (size_t)(2 * (p_item / splits)) * group_bytes + (size_t)p_t * TB;
+            ring_issue<FMT>(ring + stage * SLOT, tp, tp + group_bytes, lane);
+            p_t += WARPS;
+            if (p_t >= t_end) {
+                p_item += gridDim.x;
+                p_t = t_begin;
+            }
         }
+        cp_async_commit();                                      // one group per call, empty or not
     };
-    if (item < items) load_group();                             // weights never depend on the previous kernel
+#pragma unroll
+    for (int st = 0; st < kRingStages; ++st) produce(st);       // weights never depend on the previous kernel
 
     pdl_launch_dependents();
     pdl_wait();                                                 // X may come from the previous kernel
-    for (int i = threadIdx.x; i < kr8; i += WARPS * 32) zs[i] = make_uint4(0u, 0u, 0u, 0u);
-    {
-        // all of a thread's loads in flight before the first store (the rows are short: latency, not bandwidth)
-        const int total = M * kr8;
-        const uint4* x0 = reinterpret_cast<const uint4*>(X) + s * kr8;
-        const int64_t ldx8 = ldx / 8;
-        for (int base = threadIdx.x; base < total; base += 4 * WARPS * 32) {
-            uint4 v[4];
+    // activations come straight from global memory (they are few and shared by every warp: L1 / L2 hits):
+    // lane (g, t) reads token g's chunk t of each 32-element block, lanes of tokens that do not exist read nothing
+    const uint16_t* xrow[NG];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int i = base + u * WARPS * 32;
-                if (i < total) {
-                    const int m = i / kr8;
-                    v[u] = x0[m * ldx8 + (i - m * kr8)];
+    for (int n = 0; n < NG; ++n) xrow[n] = 8 * n + g < M ? X + (size_t)(8 * n + g) * ldx : nullptr;
+    auto load_x = [&](int tt, uint4 (&xr)[FMT == QMM_Q8 ? 1 : 2][NG]) {
+#pragma unroll
+        for (int b = 0; b < (FMT == QMM_Q8 ? 1 : 2); ++b)
+#pragma unroll
+            for (int n = 0; n < NG; ++n) {
+                xr[b][n] = make_uint4(0u, 0u, 0u, 0u);
+                if (xrow[n]) {
+                    const uint16_t* xt = xrow[n] + (size_t)tt * Fmt<FMT>::tile_k;
+                    if constexpr (FMT == QMM_Q8) {
+                        // words t and 4 + t of the row are k = 4t .. 4t+3 and 16 + 4t .. 16 + 4t+3 of the tile
+                        const uint2 lo = ld_nc_u32x2(xt + 4 * t4), hi = ld_nc_u32x2(xt + 16 + 4 * t4);
+                        xr[b][n] = make_uint4(lo.x, lo.y, hi.x, hi.y);
+                    } else {
+                        xr[b][n] = ld_nc_u32x4(xt + 32 * b + 8 * t4);
+                    }
                 }
             }
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int i = base + u * WARPS * 32;
-                if (i < total) xs[i] = v[u];
-            }
-        }
-    }
-    __syncthreads();
-    const uint4* xg[NG];
-#pragma unroll
-    for (int n = 0; n < NG; ++n) xg[n] = 8 * n + g < M ? xs + (8 * n + g) * kr8 : zs;
+    };
     Q4Consts kc;
     kc.init();
 
-    while (item < items) {
+    int stage = 0;
+    for (int item = blockIdx.x; item < items; item += gridDim.x) {
+        const int pair = item / splits;
         float acc[NG][4][4];
 #pragma unroll
         for (int n = 0; n < NG; ++n)
 #pragma unroll
             for (int i = 0; i < 4; ++i) acc[n][i][0] = acc[n][i][1] = acc[n][i][2] = acc[n][i][3] = 0.f;
-        while (t < t_end) {
-#pragma unroll
-            for (int u = 0; u < kSmallUnroll; ++u) {
-                const int tt = t + u * WARPS;
-                if (tt < t_end) {                               // (warp-uniform)
-                    FragRegs<FMT> f;
-                    transpose_slot<FMT>(r[u], f, patch, lane);
-                    frag_mma<FMT, NG>(r[u], f, xg, (tt - s * tps) * XV, t4, acc, kc);
-                }
+        if (has_tiles) {
+            for (int tt = t_begin; tt < t_end; tt += WARPS) {
+                uint4 xr[FMT == QMM_Q8 ? 1 : 2][NG];
+                load_x(tt, xr);                                 // in flight while the tile pair lands
+                cp_async_wait<kRingStages - 1>();               // the oldest group -- this tile pair -- has landed
+                __syncwarp();
+                SmallSlot<FMT> r;
+                FragRegs<FMT> f;
+                ring_read<FMT>(ring + stage * SLOT, r, f, lane);
+                __syncwarp();                                   // every lane has read the slot
+                produce(stage);
+                frag_mma_x<FMT, NG>(r, f, xr, t4, acc, kc);
+                stage = stage + 1 == kRingStages ? 0 : stage + 1;
             }
-            t += STEP;
-            if (t < t_end) load_group();
-        }
-        const int done_pair = pair;
-        item += gridDim.x;
-        if (item < items) {                                     // next item's loads fly during the reduction
-            pair = item / splits;
-            t = s * tps + warp;
-            tiles_p = packed + (size_t)(2 * pair) * group_bytes;
-            load_group();
         }
         // red[warp][token][64]: rows 0..31 of P, then of Q
 #pragma unroll
@@ -332,11 +352,10 @@ gemm_small_kernel(const uint8_t* __restrict__ packed, const uint16_t* __restrict
                 float sum = red[i];
 #pragma unroll
                 for (int w = 1; w < WARPS; ++w) sum += red[w * NT * 64 + i];
-                Y[(size_t)(i >> 6) * ldy + done_pair * 64 + (i & 63)] = __half_as_ushort(__float2half_rn(sum));
+                Y[(size_t)(i >> 6) * ldy + pair * 64 + (i & 63)] = __half_as_ushort(__float2half_rn(sum));
             }
         } else {
-            // every block of the cluster runs the same sequence of pairs, one split each
-            float* slot = cred + (cluster_round & 1) * (kSmallMaxSplits * NT * 64);
+            float* slot = cred + (cluster_round & 1) * (splits * NT * 64);
             for (int i = threadIdx.x; i < live; i += WARPS * 32) {
                 float sum = red[i];
 #pragma unroll
@@ -348,13 +367,14 @@ gemm_small_kernel(const uint8_t* __restrict__ packed, const uint16_t* __restrict
                 for (int i = threadIdx.x; i < live; i += WARPS * 32) {
                     float total = slot[i];
                     for (int sp = 1; sp < splits; ++sp) total += slot[sp * NT * 64 + i];
-                    Y[(size_t)(i >> 6) * ldy + done_pair * 64 + (i & 63)] = __half_as_ushort(__float2half_rn(total));
+                    Y[(size_t)(i >> 6) * ldy + pair * 64 + (i & 63)] = __half_as_ushort(__float2half_rn(total));
                 }
             }
-            ++cluster_round;                                    // two slots: the next item's sums do not wait for this read
+            ++cluster_round;
         }
         __syncthreads();
     }
+    cp_async_wait<0>();                                         // (only empty groups can be left)
 }
 
 // ------------------------------------------------------------------ host
@@ -381,8 +401,8 @@ static SmallPlan small_plan(int fmt, int64_t M, int64_t N, int64_t K)
     const int pairs = (int)(N / 64);
     const int per_sm = 2;
     auto smem_of = [&](int splits) {
-        return (size_t)kSmallWarps * 2048 + (size_t)(M + 1) * (size_t)(K / splits) * 2 + (size_t)kSmallWarps * nt * 64 * sizeof(float) +
-               (splits > 1 ? (size_t)2 * kSmallMaxSplits * nt * 64 * sizeof(float) : 0);
+        return (size_t)kSmallWarps * kRingStages * 2 * tile_bytes_of(fmt) + (size_t)kSmallWarps * nt * 64 * sizeof(float) +
+               (splits > 1 ? (size_t)2 * splits * nt * 64 * sizeof(float) : 0);
     };
     int splits = 1;
     // split K while the pairs alone leave SMs without a block, every warp keeps a tile, and the cluster stays small

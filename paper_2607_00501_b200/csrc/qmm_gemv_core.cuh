@@ -172,77 +172,6 @@ __device__ __forceinline__ void tile_pair_mma(const u32x8& cp, const u32x8& cq, 
     else tile_pair_mma_q56<FMT>(cp, cq, hp, hq, sp, sq, xt, acc, kc);
 }
 
-// Several tokens against the same tile pair: the codes are unpacked once, and every pair of tokens
-// takes one more pass of the MMAs.  Token 2m rides in B columns 0..3 as above; token 2m+1 rides in
-// columns 4..7 (column 4+j = its quadruple in slot group j), which the single-token form leaves
-// zero.  So lanes with g == t read token 2m's activations, lanes with g == t + 4 token 2m+1's, the
-// rest zeros (xt[m] is the lane's pointer for token pair m), and every lane receives sums: lanes
-// with t < 2 rows 4g+2t, 4g+2t+1 for token 2m, lanes with t >= 2 rows 4g+2(t-2), +1 for token 2m+1
-// (acc[m][0..1] of row group P, acc[m][2..3] of Q).
-template <int FMT, int MT>
-__device__ __forceinline__ void tile_pair_mma_multi(const u32x8& cp, const u32x8& cq, const typename HiRegs<FMT>::type& hp,
-                                                    const typename HiRegs<FMT>::type& hq, typename ScaleRegs<FMT>::type sp,
-                                                    typename ScaleRegs<FMT>::type sq, const uint4* const (&xt)[MT], int x_off,
-                                                    float (&acc)[MT][4], const Q4Consts& kc)
-{
-    constexpr int BLOCKS = FMT == QMM_Q8 ? 1 : 2;
-#pragma unroll
-    for (int b = 0; b < BLOCKS; ++b) {
-        float c[MT][4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int j = b * 4 + i;                             // 8-k chunk of the tile
-            __half2 p[4], q[4];
-            if constexpr (FMT == QMM_Q8) {
-                __half2 a[2];
-                q8_word_to_h2(cp.v[2 * j], a);
-                p[0] = a[0], p[1] = a[1];
-                q8_word_to_h2(cp.v[2 * j + 1], a);
-                p[2] = a[0], p[3] = a[1];
-                q8_word_to_h2(cq.v[2 * j], a);
-                q[0] = a[0], q[1] = a[1];
-                q8_word_to_h2(cq.v[2 * j + 1], a);
-                q[2] = a[0], q[3] = a[1];
-            } else if constexpr (FMT == QMM_Q4) {
-                q4_word_to_h2(cp.v[j], p, kc);
-                q4_word_to_h2(cq.v[j], q, kc);
-            } else {
-                const uint32_t* hpw = reinterpret_cast<const uint32_t*>(&hp);
-                const uint32_t* hqw = reinterpret_cast<const uint32_t*>(&hq);
-                const int hw = FMT == QMM_Q5 ? j / 4 : j / 2;
-                q56_word_to_h2<FMT>(cp.v[j], hpw[hw], j, p, kc);
-                q56_word_to_h2<FMT>(cq.v[j], hqw[hw], j, q, kc);
-            }
-#pragma unroll
-            for (int m = 0; m < MT; ++m) {
-                const uint4 xv = xt[m][x_off + j];
-                if (i == 0)
-                    mma16816_zero(c[m], as_u32(p[0]), as_u32(q[0]), as_u32(p[1]), as_u32(q[1]), xv.x, xv.y);
-                else
-                    mma16816(c[m], as_u32(p[0]), as_u32(q[0]), as_u32(p[1]), as_u32(q[1]), xv.x, xv.y);
-                mma16816(c[m], as_u32(p[2]), as_u32(q[2]), as_u32(p[3]), as_u32(q[3]), xv.z, xv.w);
-            }
-        }
-        float dp0, dp1, dq0, dq1;
-        if constexpr (FMT == QMM_Q8) {
-            dp0 = __half2float(__low2half(as_h2(sp))), dp1 = __half2float(__high2half(as_h2(sp)));
-            dq0 = __half2float(__low2half(as_h2(sq))), dq1 = __half2float(__high2half(as_h2(sq)));
-        } else {
-            dp0 = __half2float(b ? __high2half(as_h2(sp.x)) : __low2half(as_h2(sp.x)));
-            dp1 = __half2float(b ? __high2half(as_h2(sp.y)) : __low2half(as_h2(sp.y)));
-            dq0 = __half2float(b ? __high2half(as_h2(sq.x)) : __low2half(as_h2(sq.x)));
-            dq1 = __half2float(b ? __high2half(as_h2(sq.y)) : __low2half(as_h2(sq.y)));
-        }
-#pragma unroll
-        for (int m = 0; m < MT; ++m) {
-            acc[m][0] = fmaf(dp0, c[m][0], acc[m][0]);
-            acc[m][1] = fmaf(dp1, c[m][1], acc[m][1]);
-            acc[m][2] = fmaf(dq0, c[m][2], acc[m][2]);
-            acc[m][3] = fmaf(dq1, c[m][3], acc[m][3]);
-        }
-    }
-}
-
 // Scales of rows 4g+2(t&1) and the next row of one tile (the rows whose sums this lane receives).
 template <int FMT>
 __device__ __forceinline__ typename ScaleRegs<FMT>::type load_scales(const uint8_t* tile, int lane)
