@@ -64,9 +64,10 @@
  * product satisfies |y - y_ref| <= 2e-3 * sum_k |w_k x_k| + 1e-5.  The GEMVs
  * (qmm_gemv*, decode-sized qmm_moe) multiply integer codes by activations
  * exactly and apply the scale in fp32, so this holds for every finite scale.
- * The tensor-core products (qmm_gemm, qmm_moe with more than 32 token-expert
- * rows) feed each weight to the tensor core as fp16(float(d) * q), which adds
- * two limits:
+ * So does qmm_gemm for M <= 8 (its few-token kernel works the same way).
+ * The tensor-core products (qmm_gemm for M > 8, qmm_moe with more than 32
+ * token-expert rows) feed each weight to the tensor core as fp16(float(d) * q),
+ * which adds two limits:
  *   - |d| * max|q| must stay below 65504 (|d| < 8188 for Q4, < 511.75 for Q8),
  *     else the weight becomes inf; qmm_packed_check reports such scales;
  *   - a weight with |d * q| < 2^-14 is a subnormal fp16 and carries an absolute
@@ -290,6 +291,11 @@ qmm_status qmm_chain_run(const qmm_chain_info* info, void* stream);
 /* Prefill matrix-matrix product (Sec. 3.3 "GEMM (prefill, M>1)", Sec. 3.4):
  *   Y[m,n] = fp16( sum_k w[n,k] * X[m,k] ), fp32 accumulation on the tensor
  * cores; weights enter the contraction as fp16(float(d) * q).
+ * For M <= 8 (a decode step of a small batch, the tail of a prefill chunk) the
+ * product is bound by streaming W once, like decode (Sec. 3.3), and runs on a
+ * kernel of the decode family instead: integer codes times activations on the
+ * warp-level tensor path, scales applied in fp32, no workspace use; row m of Y
+ * is then the same bits whatever M (<= 8) is and whatever the other rows hold.
  *   X_fp16  device, [M, ldx] fp16 row-major, ldx >= K, ldx % 8 == 0
  *   Y_fp16  device, [M, ldy] fp16 row-major, ldy >= N, ldy % 8 == 0, written
  *   ws      device, at least qmm_gemm_workspace_bytes(...) bytes: the status
