@@ -947,6 +947,20 @@ def run_case(args):
         y = torch.empty(N, dtype=torch.float16, device="cuda")
         for i in range(8):
             qmm.gemv(f, many[i * 8], N, K, x, y=y)
+    elif name.startswith("gemm_few_q") and "_M" in name:
+        # gemm_few_q4_M8: the few-token kernel (M <= 8) on a [28672, 4096] matrix; three distinct copies
+        # (198 MB in Q4, 374 MB in Q8) taken in turn, so that every launch streams from HBM
+        f = synth.Q4 if name.startswith("gemm_few_q4") else synth.Q8
+        M = int(name.split("_M")[1])
+        N, K = 28672, 4096
+        one = qmm.pack(f, dev(synth.quantize(f, synth.weights(9, 9, N, K))), N, K)
+        copies = [one, one.clone(), one.clone()]
+        X = dev(synth.activations(9, 10 + M, M, K))
+        Y = torch.empty((M, N), dtype=torch.float16, device="cuda")
+        ws = torch.zeros(max(qmm.gemm_workspace_bytes(f, M, N, K), 256), dtype=torch.uint8, device="cuda")
+        for i in range(6):
+            qmm.gemm(f, copies[i % 3], N, K, X, Y=Y, ws=ws)
+        qmm.status_check(ws)
     elif name.startswith("gemm_q") and "_M" in name:
         # gemm_q4_M2048 (gate/up shape), gemm_q8_M1024, gemm_q4_down_M512 ...
         c = synth.CFG3
@@ -977,7 +991,7 @@ def run_case(args):
             qmm.moe(a, ws)
         qmm.status_check(ws)
     else:
-        raise SystemExit("unknown --case %r (gemv_batch_q4|q8, gemv_lm_head_q8, gemv_kv_q4|q8, gemm_q4|q8[_down]_M<M>, "
+        raise SystemExit("unknown --case %r (gemv_batch_q4|q8, gemv_lm_head_q8, gemv_kv_q4|q8, gemm_q4|q8[_down]_M<M>, gemm_few_q4|q8_M<M>, "
                          "moe_q4|q8_T<T>, chain_q4|q8_dependent|independent)" % name)
     torch.cuda.synchronize()
     print("case %s: %d launches done" % (name, reps), file=sys.stderr)
