@@ -640,6 +640,25 @@ def extra_sections(args, qmm, torch, pk, ops, fmts, batch, gpu_index=0):
                                                            "ms_tensor_core_kernel": round(med8t, 4)}, **hbm_fracs(b, med8, pk))
         del g8, g8t, ops8
 
+    # the whole decode stack for a batch of 8 sequences as ONE launch per format (qmm_gemm_batch: the 112
+    # matrices as independent problems, X [8, K] each): the weights are streamed once for all eight tokens,
+    # so the algorithmic bytes are those of the single-token step
+    for f in (fmts if on("batch8") else ()):
+        probs8 = []
+        for w, N, K, x, y in batch[f]._keep:
+            probs8.append((w, N, K, x.reshape(1, K).repeat(8, 1).contiguous(), torch.empty((8, N), dtype=torch.float16, device="cuda")))
+        arr8 = qmm.gemm_batch_problems(probs8)
+        g = torch.cuda.CUDAGraph()
+        s = torch.cuda.Stream()
+        with torch.cuda.stream(s):
+            qmm.gemm_batch(f, arr8)
+            torch.cuda.synchronize()
+            with torch.cuda.graph(g, stream=s):
+                qmm.gemm_batch(f, arr8)
+            m = measure(torch, g.replay, flush)
+        out["decode_stack_q%d_batch8_one_launch" % f] = dict(m, tokens=8, problems=len(probs8), **hbm_fracs(stack_bytes(f), m["ms"], pk))
+        del g, arr8, probs8
+
     # cfg0: one small Q4 GEMV (1.77 MB of weights: 0.27 us of HBM traffic, far below a launch).  Steady
     # state = 300 distinct packed copies (531 MB, larger than L2) so that every product streams from HBM:
     # as 300 chained launches in one graph, and as qmm_gemv_batch launches over the same 300 problems.
@@ -1042,7 +1061,7 @@ def main():
     ap.add_argument("--streams", type=int, default=8, help="streams for --mode streams")
     ap.add_argument("--no-sections", action="store_true", help="skip the LM-head / GEMM / MoE sections")
     ap.add_argument("--sections", default=None,
-                    help="comma list of the sections to run (chain,chained,cfg0,lm_head,ffn,gemm,formats,moe); default: all")
+                    help="comma list of the sections to run (chain,chained,batch8,cfg0,lm_head,ffn,gemm,formats,moe); default: all")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--case", default=None, help="profiling aid: run a few launches of one kernel and exit (see run_case)")

@@ -54,7 +54,7 @@
  *     2 (i % 4), 2 (i % 4) + 1 of qh[i / 4] = u_i >> 4.
  *   (The paper's kernel library spans 2-bit to 16-bit formats, Sec. 3.3 and
  *   Sec. 4.1; Q5 and Q6 are built for qmm_pack, qmm_dequant, qmm_packed_check,
- *   qmm_gemv, qmm_gemv_static, qmm_gemv_batch and qmm_gemm -- every other call returns
+ *   qmm_gemv, qmm_gemv_static, qmm_gemv_batch, qmm_gemm and qmm_gemm_batch -- every other call returns
  *   QMM_ERR_UNSUPPORTED for them.)
  *   Row n of W holds K/32 consecutive blocks; rows are consecutive; block b of
  *   row n covers k in [32 b, 32 b + 32).  Weight value: float(d) * q (exact in
@@ -310,6 +310,26 @@ qmm_status qmm_gemm(qmm_format fmt, const void* packed, int64_t N, int64_t K,
                     const uint16_t* X_fp16, int64_t ldx,
                     uint16_t* Y_fp16, int64_t ldy, int64_t M,
                     void* ws, size_t ws_bytes, void* stream);
+
+/* Many independent few-token products in one launch: problem i computes
+ *   Y_i[m,n] = fp16( sum_k w_i[n,k] * X_i[m,k] ),  m < M,  1 <= M <= 8 for all,
+ * i.e. every matrix of a decode step for a batch of up to eight sequences (the
+ * paper's decode gains come from fewer, fused dispatches, Sec. 3.3; decode is
+ * bound by streaming the weights, which this launch does once for all M
+ * tokens).  The products must be independent, as for qmm_gemv_batch.  Integer
+ * codes times activations, scales applied in fp32 (the accuracy of the GEMVs);
+ * row m of Y_i does not depend on M or on the other rows.  No workspace.
+ *   problems  HOST array of `count` descriptors (read during the call only);
+ *             pointers inside are device pointers: packed 32-byte aligned,
+ *             X [M, ldx] and Y [M, ldy] fp16 row-major, 16-byte aligned,
+ *             ldx >= K, ldy >= N, both multiples of 8 and below 2^31.         */
+typedef struct {
+    const void* packed;        /* device, from qmm_pack                        */
+    const uint16_t* X_fp16;    /* device, [M, ldx] fp16                        */
+    uint16_t* Y_fp16;          /* device, [M, ldy] fp16, written               */
+    int64_t N, K, ldx, ldy;
+} qmm_gemm_problem;
+qmm_status qmm_gemm_batch(qmm_format fmt, const qmm_gemm_problem* problems, int count, int64_t M, void* stream);
 
 /* Top-k mixture-of-experts feed-forward layer.  The paper names
  * mixture-of-experts models as the case with its largest prefill gains

@@ -42,6 +42,7 @@ qmm_status launch_gemv_gate_up(int fmt, const void* packed_gate, const void* pac
 size_t gemm_workspace_bytes(int fmt, int64_t M, int64_t N, int64_t K);
 qmm_status launch_gemm(int fmt, const void* packed, int64_t N, int64_t K, const uint16_t* X, int64_t ldx,
                        uint16_t* Y, int64_t ldy, int64_t M, void* ws, cudaStream_t st);
+qmm_status launch_gemm_small_batch(int fmt, const qmm_gemm_problem* probs, int count, int64_t M, cudaStream_t st);
 size_t moe_workspace_bytes(const qmm_moe_args* a);
 qmm_status launch_moe(const qmm_moe_args* a, void* ws, bool route_only, cudaStream_t st);
 qmm_status status_check(void* ws, cudaStream_t st);
@@ -62,7 +63,7 @@ static bool fmt_ok(int fmt) { return fmt == QMM_Q4 || fmt == QMM_Q5 || fmt == QM
 static qmm_status check_fmt_everywhere(const char* who, int fmt)
 {
     if (fmt == QMM_Q5 || fmt == QMM_Q6)
-        return fail(QMM_ERR_UNSUPPORTED, "%s: format %d is built for qmm_pack, qmm_dequant, qmm_packed_check, qmm_gemv, qmm_gemv_batch and qmm_gemm only", who, fmt);
+        return fail(QMM_ERR_UNSUPPORTED, "%s: format %d is built for qmm_pack, qmm_dequant, qmm_packed_check, qmm_gemv, qmm_gemv_batch, qmm_gemm and qmm_gemm_batch only", who, fmt);
     return QMM_OK;
 }
 
@@ -234,6 +235,28 @@ qmm_status qmm_gemm(qmm_format fmt, const void* packed, int64_t N, int64_t K,
     if (!aligned(ws, 256)) return fail(QMM_ERR_ALIGNMENT, "qmm_gemm: workspace must be 256-byte aligned");
     if ((s = check_device("qmm_gemm")) != QMM_OK) return s;
     return launch_gemm(fmt, packed, N, K, X_fp16, ldx, Y_fp16, ldy, M, ws, (cudaStream_t)stream);
+}
+
+qmm_status qmm_gemm_batch(qmm_format fmt, const qmm_gemm_problem* problems, int count, int64_t M, void* stream)
+{
+    if (count < 0) return fail(QMM_ERR_INVALID_ARG, "qmm_gemm_batch: count=%d is negative", count);
+    if (M < 0 || M > 8) return fail(M < 0 ? QMM_ERR_INVALID_ARG : QMM_ERR_UNSUPPORTED, "qmm_gemm_batch: M=%lld outside [0, 8]", (long long)M);
+    if (count == 0 || M == 0) return QMM_OK;
+    if (!problems) return fail(QMM_ERR_INVALID_ARG, "qmm_gemm_batch: null problem list");
+    for (int i = 0; i < count; ++i) {
+        const qmm_gemm_problem& q = problems[i];
+        qmm_status s = check_matrix("qmm_gemm_batch", fmt, q.N, q.K);
+        if (s != QMM_OK) return s;
+        if (!q.packed || !q.X_fp16 || !q.Y_fp16) return fail(QMM_ERR_INVALID_ARG, "qmm_gemm_batch: problem %d has a null pointer", i);
+        if (q.ldx < q.K || q.ldy < q.N) return fail(QMM_ERR_SHAPE, "qmm_gemm_batch: problem %d: ldx < K or ldy < N", i);
+        if (q.ldx % 8 || q.ldy % 8 || q.ldx >= (1LL << 31) || q.ldy >= (1LL << 31))
+            return fail(QMM_ERR_ALIGNMENT, "qmm_gemm_batch: problem %d: ldx and ldy must be multiples of 8 elements below 2^31", i);
+        if (!aligned(q.packed, 32) || !aligned(q.X_fp16, 16) || !aligned(q.Y_fp16, 16))
+            return fail(QMM_ERR_ALIGNMENT, "qmm_gemm_batch: problem %d: packed must be 32-byte, X and Y 16-byte aligned", i);
+    }
+    qmm_status s = check_device("qmm_gemm_batch");
+    if (s != QMM_OK) return s;
+    return launch_gemm_small_batch(fmt, problems, count, M, (cudaStream_t)stream);
 }
 
 static qmm_status check_moe(const char* who, const qmm_moe_args* a)

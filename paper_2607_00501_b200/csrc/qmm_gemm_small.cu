@@ -377,6 +377,147 @@ gemm_small_kernel(const uint8_t* __restrict__ packed, const uint16_t* __restrict
     cp_async_wait<0>();                                         // (only empty groups can be left)
 }
 
+// ------------------------------------------------------------------ batch
+//
+// Many independent few-token products in ONE launch -- every matrix of a decode step for a batch of
+// up to eight sequences (the paper's decode gains come from fewer, fused dispatches, Sec. 3.3).
+// As in gemv_batch_kernel: work unit = (problem, pair of row groups), the unit list is cut into
+// gridDim.x contiguous ranges of equal cost (tiles), so blocks finish together although problems
+// differ in K; no K split across blocks, no workspace.  The ring runs on across units and problems.
+constexpr int kSmallMaxBatch = 128;
+
+struct SmallBatchProblem {
+    const uint8_t* packed;
+    const uint16_t* X;        // [M, ldx]
+    uint16_t* Y;              // [M, ldy]
+    int ldx, ldy;
+    int tpr;                  // tiles per row
+    int pairs;                // N / 64
+    int cost_begin;           // tiles of all earlier problems
+};
+
+struct SmallBatchParams {
+    int count, total_cost, M;
+    SmallBatchProblem p[kSmallMaxBatch];
+};
+
+template <int FMT>
+__global__ void __launch_bounds__(kSmallWarps * 32, 2)
+gemm_small_batch_kernel(const __grid_constant__ SmallBatchParams bp)
+{
+    constexpr int WARPS = kSmallWarps;
+    constexpr int TB = Fmt<FMT>::tile_bytes, TK = Fmt<FMT>::tile_k;
+    constexpr int SLOT = 2 * TB;
+    extern __shared__ uint4 smem[];
+    float* red_all = reinterpret_cast<float*>(smem + WARPS * kRingStages * SLOT / 16);   // [2][WARPS][8][64], behind the rings
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, t4 = lane & 3;
+    const uint32_t ring = static_cast<uint32_t>(__cvta_generic_to_shared(smem)) + warp * (kRingStages * SLOT);
+    const int M = bp.M;
+
+    // this block's range of the unit list, by cost; a unit belongs to the block whose range holds its first tile
+    const int c0 = (int)(((long long)bp.total_cost * blockIdx.x) / gridDim.x);
+    const int c1 = (int)(((long long)bp.total_cost * (blockIdx.x + 1)) / gridDim.x);
+    int pi0 = 0;
+    while (pi0 < bp.count && bp.p[pi0].cost_begin + bp.p[pi0].pairs * bp.p[pi0].tpr <= c0) ++pi0;
+    int unit0 = 0;
+    if (pi0 < bp.count) {
+        const int rel = c0 - bp.p[pi0].cost_begin;
+        unit0 = rel <= 0 ? 0 : (rel + bp.p[pi0].tpr - 1) / bp.p[pi0].tpr;
+        if (unit0 >= bp.p[pi0].pairs) {
+            ++pi0;
+            unit0 = 0;
+        }
+    }
+    auto valid = [&](int p, int u) { return p < bp.count && bp.p[p].cost_begin + u * bp.p[p].tpr < c1; };
+
+    // producer: runs kRingStages tile pairs ahead of the consumer, across units and problems
+    int p_pi = pi0, p_unit = unit0, p_t = warp;
+    auto produce = [&](int stage) {
+        while (valid(p_pi, p_unit) && p_t >= bp.p[p_pi].tpr) {  // this warp has no (more) tiles in the unit
+            if (++p_unit >= bp.p[p_pi].pairs) {
+                ++p_pi;
+                p_unit = 0;
+            }
+            p_t = warp;
+        }
+        if (valid(p_pi, p_unit)) {
+            const size_t group_bytes = (size_t)bp.p[p_pi].tpr * TB;
+            const uint8_t* tp = bp.p[p_pi].packed + (size_t)(2 * p_unit) * group_bytes + (size_t)p_t * TB;
+            ring_issue<FMT>(ring + stage * SLOT, tp, tp + group_bytes, lane);
+            p_t += WARPS;
+        }
+        cp_async_commit();                                      // one group per call, empty or not
+    };
+#pragma unroll
+    for (int st = 0; st < kRingStages; ++st) produce(st);       // weights never depend on the previous kernel
+
+    pdl_launch_dependents();
+    pdl_wait();                                                 // activations may come from the previous kernel
+    Q4Consts kc;
+    kc.init();
+
+    int stage = 0, round = 0;
+    int pi = pi0, unit = unit0;
+    while (valid(pi, unit)) {
+        float* red = red_all + (round & 1) * (WARPS * 8 * 64);
+        const int tpr = bp.p[pi].tpr;
+        const uint16_t* xrow = g < M ? bp.p[pi].X + (size_t)g * bp.p[pi].ldx : nullptr;
+        float acc[1][4][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[0][i][0] = acc[0][i][1] = acc[0][i][2] = acc[0][i][3] = 0.f;
+        for (int tt = warp; tt < tpr; tt += WARPS) {
+            uint4 xr[FMT == QMM_Q8 ? 1 : 2][1];
+#pragma unroll
+            for (int b = 0; b < (FMT == QMM_Q8 ? 1 : 2); ++b) {
+                xr[b][0] = make_uint4(0u, 0u, 0u, 0u);
+                if (xrow) {
+                    const uint16_t* xt = xrow + (size_t)tt * TK;
+                    if constexpr (FMT == QMM_Q8) {
+                        const uint2 lo = ld_nc_u32x2(xt + 4 * t4), hi = ld_nc_u32x2(xt + 16 + 4 * t4);
+                        xr[b][0] = make_uint4(lo.x, lo.y, hi.x, hi.y);
+                    } else {
+                        xr[b][0] = ld_nc_u32x4(xt + 32 * b + 8 * t4);
+                    }
+                }
+            }
+            cp_async_wait<kRingStages - 1>();                   // the oldest group -- this tile pair -- has landed
+            __syncwarp();
+            SmallSlot<FMT> r;
+            FragRegs<FMT> f;
+            ring_read<FMT>(ring + stage * SLOT, r, f, lane);
+            __syncwarp();                                       // every lane has read the slot
+            produce(stage);
+            frag_mma_x<FMT, 1>(r, f, xr, t4, acc, kc);
+            stage = stage + 1 == kRingStages ? 0 : stage + 1;
+        }
+        // red[warp][token][64]: rows 0..31 of P, then of Q
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float* w = red + (warp * 8 + 2 * t4) * 64 + 4 * g + i;
+            w[0] = acc[0][i][0];
+            w[64] = acc[0][i][1];
+            w[32] = acc[0][i][2];
+            w[64 + 32] = acc[0][i][3];
+        }
+        // one barrier per unit: this buffer is rewritten two units on, after every thread has passed the
+        // next unit's barrier, i.e. has finished reading it
+        __syncthreads();
+        const int nw = tpr < WARPS ? tpr : WARPS;               // warps that had tiles (the others hold zeros)
+        for (int i = threadIdx.x; i < M * 64; i += WARPS * 32) {
+            float sum = red[i];
+            for (int w = 1; w < nw; ++w) sum += red[w * 8 * 64 + i];
+            bp.p[pi].Y[(size_t)(i >> 6) * bp.p[pi].ldy + unit * 64 + (i & 63)] = __half_as_ushort(__float2half_rn(sum));
+        }
+        ++round;
+        if (++unit >= bp.p[pi].pairs) {
+            ++pi;
+            unit = 0;
+        }
+    }
+    cp_async_wait<0>();                                         // (only empty groups can be left)
+}
+
 // ------------------------------------------------------------------ host
 
 bool gemm_small_supported(int fmt, int64_t M)
@@ -463,6 +604,57 @@ qmm_status launch_gemm_small(int fmt, const void* packed, int64_t N, int64_t K, 
     QMM_SMALL_CASE(QMM_Q6, 1)
 #undef QMM_SMALL_CASE
     return fail(QMM_ERR_UNSUPPORTED, "qmm_gemm: no few-token kernel for format %d, M=%lld", fmt, (long long)M);
+}
+
+// Host side of qmm_gemm_batch: up to kSmallMaxBatch problems per launch.
+qmm_status launch_gemm_small_batch(int fmt, const qmm_gemm_problem* probs, int count, int64_t M, cudaStream_t st)
+{
+    for (int first = 0; first < count; first += kSmallMaxBatch) {
+        const int n = count - first < kSmallMaxBatch ? count - first : kSmallMaxBatch;
+        SmallBatchParams bp = {};
+        bp.count = n;
+        bp.M = (int)M;
+        long long cost = 0;
+        int units = 0;
+        for (int i = 0; i < n; ++i) {
+            const qmm_gemm_problem& q = probs[first + i];
+            SmallBatchProblem& b = bp.p[i];
+            b.packed = (const uint8_t*)q.packed;
+            b.X = q.X_fp16;
+            b.Y = q.Y_fp16;
+            b.ldx = (int)q.ldx;
+            b.ldy = (int)q.ldy;
+            b.tpr = (int)(q.K / tile_k_of(fmt));
+            b.pairs = (int)(q.N / 64);
+            b.cost_begin = (int)cost;
+            cost += (long long)b.pairs * b.tpr;
+            units += b.pairs;
+            if (cost > 0x7FFFFFFFLL) return fail(QMM_ERR_UNSUPPORTED, "qmm_gemm_batch: batch too large for one launch");
+        }
+        bp.total_cost = (int)cost;
+        const size_t smem = (size_t)kSmallWarps * kRingStages * 2 * tile_bytes_of(fmt) + (size_t)2 * kSmallWarps * 8 * 64 * sizeof(float);
+        int grid = 2 * kNumSMs;
+        if (units < grid) grid = units;
+        void (*kern)(SmallBatchParams) = fmt == QMM_Q4   ? gemm_small_batch_kernel<QMM_Q4>
+                                         : fmt == QMM_Q5 ? gemm_small_batch_kernel<QMM_Q5>
+                                         : fmt == QMM_Q6 ? gemm_small_batch_kernel<QMM_Q6>
+                                                         : gemm_small_batch_kernel<QMM_Q8>;
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return check_cuda(e, "qmm_gemm_batch shared memory size");
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)grid);
+        cfg.blockDim = dim3(kSmallWarps * 32);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        e = cudaLaunchKernelEx(&cfg, kern, bp);
+        if (e != cudaSuccess) return check_cuda(e, "qmm_gemm_batch launch");
+    }
+    return QMM_OK;
 }
 
 }  // namespace qmm

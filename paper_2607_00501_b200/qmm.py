@@ -33,7 +33,7 @@ STATUS_NAMES = {
 EXPORTS = (
     "qmm_last_error", "qmm_version", "qmm_canonical_bytes", "qmm_packed_bytes", "qmm_pack",
     "qmm_dequant", "qmm_gemv_workspace_bytes", "qmm_gemv", "qmm_gemm_workspace_bytes", "qmm_gemm",
-    "qmm_moe_workspace_bytes", "qmm_moe", "qmm_moe_route", "qmm_status_check", "qmm_gemv_static", "qmm_gemv_batch",
+    "qmm_moe_workspace_bytes", "qmm_moe", "qmm_moe_route", "qmm_status_check", "qmm_gemv_static", "qmm_gemv_batch", "qmm_gemm_batch",
     "qmm_gemv_gate_up", "qmm_packed_check", "qmm_debug_config", "qmm_debug_wait_give_up",
     "qmm_chain_plan_bytes", "qmm_chain_workspace_bytes", "qmm_chain_build", "qmm_chain_run",
 )
@@ -49,6 +49,11 @@ class QmmError(RuntimeError):
 class GemvProblem(ctypes.Structure):
     _fields_ = [("packed", ctypes.c_void_p), ("x_fp16", ctypes.c_void_p), ("y_fp16", ctypes.c_void_p),
                 ("N", ctypes.c_int64), ("K", ctypes.c_int64)]
+
+
+class GemmProblem(ctypes.Structure):
+    _fields_ = [("packed", ctypes.c_void_p), ("X_fp16", ctypes.c_void_p), ("Y_fp16", ctypes.c_void_p),
+                ("N", ctypes.c_int64), ("K", ctypes.c_int64), ("ldx", ctypes.c_int64), ("ldy", ctypes.c_int64)]
 
 
 class ChainStage(ctypes.Structure):
@@ -106,6 +111,7 @@ def lib() -> ctypes.CDLL:
             L.qmm_gemv_static.argtypes = [ci, vp, i64, i64, vp, vp, vp]
             L.qmm_gemv_gate_up.argtypes = [ci, vp, vp, i64, i64, vp, vp, vp]
             L.qmm_gemv_batch.argtypes = [ci, ctypes.POINTER(GemvProblem), ci, vp]
+            L.qmm_gemm_batch.argtypes = [ci, ctypes.POINTER(GemmProblem), ci, i64, vp]
             L.qmm_gemm_workspace_bytes.restype = sz
             L.qmm_gemm_workspace_bytes.argtypes = [ci, i64, i64, i64]
             L.qmm_gemm.argtypes = [ci, vp, i64, i64, vp, i64, vp, i64, i64, vp, sz, vp]
@@ -211,6 +217,28 @@ def gemv_batch(fmt: int, problems) -> None:
     """All products y_i = W_i x_i of the list in one launch.  `problems` is the array made by
     gemv_batch_problems (build it once and reuse it: the call only reads it)."""
     _check(lib().qmm_gemv_batch(fmt, problems, len(problems), _stream()))
+
+
+def gemm_batch_problems(problems):
+    """problems: iterable of (packed, N, K, X [M, K], Y [M, N]) tensors -> ctypes array for gemm_batch (keeps
+    the tensors alive).  Row strides may exceed K / N; every X and Y has the same number of rows."""
+    problems = list(problems)
+    arr = (GemmProblem * len(problems))()
+    for i, (packed, N, K, X, Y) in enumerate(problems):
+        assert X.dtype == torch.float16 and X.dim() == 2 and X.shape[1] == K and X.stride(1) == 1
+        assert Y.dtype == torch.float16 and Y.dim() == 2 and Y.shape == (X.shape[0], N) and Y.stride(1) == 1
+        M = X.shape[0]
+        arr[i] = GemmProblem(packed.data_ptr(), X.data_ptr(), Y.data_ptr(), N, K,
+                             X.stride(0) if M > 1 else max(K, X.stride(0)), Y.stride(0) if M > 1 else max(N, Y.stride(0)))
+    arr._keep = problems
+    arr._M = problems[0][3].shape[0] if problems else 0
+    return arr
+
+
+def gemm_batch(fmt: int, problems) -> None:
+    """All products Y_i = X_i W_i^T (M <= 8 rows each) of the list in one launch.  `problems` is the array
+    made by gemm_batch_problems (build it once and reuse it: the call only reads it)."""
+    _check(lib().qmm_gemm_batch(fmt, problems, len(problems), problems._M, _stream()))
 
 
 GEMV_STATIC_SCRATCH_BYTES = 1 << 20

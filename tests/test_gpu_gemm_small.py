@@ -129,3 +129,110 @@ def test_few_tokens_on_the_full_size_prefill_shapes(qmm, oracle, shape, M):
     Y = util.host_f64(gemm(qmm, c["fmt"], packed, N, K, util.dev(X)))
     Y_ref, B = oracle.gemm(c["fmt"], blocks, N, K, X)
     util.assert_within_tol(Y, Y_ref, B, "cfg3 %s M=%d" % (name, M))
+
+
+# ------------------------------------------------------------------ qmm_gemm_batch
+
+@pytest.mark.parametrize("fmt", FMTS)
+@pytest.mark.parametrize("M", [1, 3, 8])
+def test_gemm_batch_mixed_shapes(qmm, oracle, fmt, M):
+    """One launch over problems that differ in N and K (short K: fewer tiles than warps; long K; many
+    row groups), strided X and Y with guard values; every output against the oracle; repeatable."""
+    shapes = [(128, 256), (384, 1024), (128, 8192), (640, 512), (256, 2048), (128, 256), (2176, 1280)]
+    probs, refs, bufs = [], [], []
+    for i, (N, K) in enumerate(shapes):
+        blocks, _, _ = util.random_blocks(synth, fmt, N, K, seed=97 + 10 * fmt + i, special_scales=True)
+        X = synth.activations(97, 100 + i, M, K)
+        Xbuf = torch.full((M, K + 8 * (i % 3)), 7.0, dtype=torch.float16, device="cuda")
+        Xbuf[:, :K] = util.dev(X)
+        Ybuf = torch.full((M, N + 16), 9.0, dtype=torch.float16, device="cuda")
+        probs.append((qmm.pack(fmt, util.dev(blocks), N, K), N, K, Xbuf[:, :K], Ybuf[:, :N]))
+        refs.append(oracle.gemm(fmt, blocks, N, K, X))
+        bufs.append(Ybuf)
+    arr = qmm.gemm_batch_problems(probs)
+    qmm.gemm_batch(fmt, arr)
+    torch.cuda.synchronize()
+    for (p, N, K, X, Y), (Y_ref, B), Ybuf in zip(probs, refs, bufs):
+        util.assert_within_tol(util.host_f64(Y), Y_ref, B, "batch %dx%d M=%d fmt=%d" % (N, K, M, fmt))
+        assert torch.all(Ybuf[:, N:] == 9.0)
+    first = [b.clone() for b in bufs]
+    qmm.gemm_batch(fmt, arr)
+    for f, b in zip(first, bufs):
+        assert torch.equal(f, b)
+
+
+@pytest.mark.parametrize("fmt", [4, 8])
+def test_gemm_batch_rows_equal_qmm_gemm(qmm, fmt):
+    """Where qmm_gemm does not split K across blocks (many row groups) the two calls add in the same order:
+    the batched launch gives the same bits, and a row does not depend on M."""
+    N, K, M = 19200, 512, 6
+    blocks = synth.quantize(fmt, synth.weights(98, fmt, N, K))
+    packed = qmm.pack(fmt, util.dev(blocks), N, K)
+    X = util.dev(synth.activations(98, 1, M, K))
+    Y1 = gemm(qmm, fmt, packed, N, K, X)
+    Y2 = torch.empty_like(Y1)
+    qmm.gemm_batch(fmt, qmm.gemm_batch_problems([(packed, N, K, X, Y2)]))
+    assert torch.equal(Y1, Y2)
+    Y3 = torch.empty((2, N), dtype=torch.float16, device="cuda")
+    qmm.gemm_batch(fmt, qmm.gemm_batch_problems([(packed, N, K, X[4:6], Y3)]))
+    assert torch.equal(Y3, Y1[4:6])
+
+
+@pytest.mark.parametrize("fmt", [4, 8])
+def test_cfg1_two_layers_full_size_for_a_batch_of_eight(qmm, oracle, fmt):
+    """All 14 matrices of two decoder layers at their real sizes for 8 sequences in one launch."""
+    M = 8
+    probs, refs = [], []
+    for layer in (0, 15):
+        for name, N, K, act, w in synth.cfg1_layer_weights(layer):
+            blocks = synth.quantize(fmt, w)
+            X = synth.activations(99, 16 * layer + len(probs), M, K)
+            Y = torch.empty((M, N), dtype=torch.float16, device="cuda")
+            probs.append((qmm.pack(fmt, util.dev(blocks), N, K), N, K, util.dev(X), Y))
+            refs.append((name, oracle.gemm(fmt, blocks, N, K, X)))
+    qmm.gemm_batch(fmt, qmm.gemm_batch_problems(probs))
+    torch.cuda.synchronize()
+    for (p, N, K, X, Y), (name, (Y_ref, B)) in zip(probs, refs):
+        util.assert_within_tol(util.host_f64(Y), Y_ref, B, "cfg1 batch of 8, %s" % name)
+
+
+def test_gemm_batch_more_problems_than_one_launch_holds(qmm, oracle):
+    fmt, M = 4, 4
+    shapes = [(128, 256), (256, 512), (128, 1024)]
+    probs, refs = [], []
+    for i in range(150):
+        N, K = shapes[i % 3]
+        blocks = synth.quantize(fmt, synth.weights(96, i % 7, N, K))
+        X = synth.activations(96, 300 + i, M, K)
+        probs.append((qmm.pack(fmt, util.dev(blocks), N, K), N, K, util.dev(X), torch.empty((M, N), dtype=torch.float16, device="cuda")))
+        refs.append(oracle.gemm(fmt, blocks, N, K, X))
+    qmm.gemm_batch(fmt, qmm.gemm_batch_problems(probs))
+    torch.cuda.synchronize()
+    for (p, N, K, X, Y), (Y_ref, B) in zip(probs, refs):
+        util.assert_within_tol(util.host_f64(Y), Y_ref, B, "150 problems")
+
+
+def test_gemm_batch_argument_checks(qmm):
+    buf = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
+    Y = torch.zeros((4, 128), dtype=torch.float16, device="cuda")
+    X = torch.zeros((4, 256), dtype=torch.float16, device="cuda")
+    L = qmm.lib()
+    P = qmm.GemmProblem
+    good = qmm.gemm_batch_problems([(buf, 128, 256, X, Y)])
+    assert L.qmm_gemm_batch(4, good, 1, 4, None) == 0
+    assert L.qmm_gemm_batch(4, good, 0, 4, None) == 0 and L.qmm_gemm_batch(4, good, 1, 0, None) == 0
+    assert L.qmm_gemm_batch(4, good, -1, 4, None) == 1 and L.qmm_gemm_batch(4, good, 1, -1, None) == 1
+    assert L.qmm_gemm_batch(4, good, 1, 9, None) == 5                                    # more than eight tokens
+    assert L.qmm_gemm_batch(4, None, 1, 4, None) == 1
+    assert L.qmm_gemm_batch(7, good, 1, 4, None) == 1                                    # unknown format
+    bad = (P * 1)(P(buf.data_ptr() + 8, X.data_ptr(), Y.data_ptr(), 128, 256, 256, 128))
+    assert L.qmm_gemm_batch(4, bad, 1, 4, None) == 3                                     # packed not 32-byte aligned
+    bad = (P * 1)(P(buf.data_ptr(), X.data_ptr(), Y.data_ptr(), 100, 256, 256, 128))
+    assert L.qmm_gemm_batch(4, bad, 1, 4, None) == 5                                     # N not a multiple of 128
+    bad = (P * 1)(P(buf.data_ptr(), X.data_ptr(), Y.data_ptr(), 128, 256, 128, 128))
+    assert L.qmm_gemm_batch(4, bad, 1, 4, None) == 2                                     # ldx < K
+    bad = (P * 1)(P(buf.data_ptr(), X.data_ptr(), Y.data_ptr(), 128, 256, 260, 128))
+    assert L.qmm_gemm_batch(4, bad, 1, 4, None) == 3                                     # ldx not a multiple of 8
+    bad = (P * 1)(P(buf.data_ptr(), 0, Y.data_ptr(), 128, 256, 256, 128))
+    assert L.qmm_gemm_batch(4, bad, 1, 4, None) == 1                                     # null X
+    torch.cuda.synchronize()

@@ -142,6 +142,9 @@ def test_empty_inputs_are_accepted_and_do_nothing(L):
     assert L.qmm_gemm(4, a, 128, 256, a, 256, a, 128, -1, None, 0, None) == 1
     assert L.qmm_gemv_batch(4, None, 0, None) == 0
     assert L.qmm_gemv_batch(4, None, -1, None) == 1
+    assert L.qmm_gemm_batch(4, None, 0, 4, None) == 0 and L.qmm_gemm_batch(4, None, 3, 0, None) == 0
+    assert L.qmm_gemm_batch(4, None, -1, 4, None) == 1 and L.qmm_gemm_batch(4, None, 3, 4, None) == 1
+    assert L.qmm_gemm_batch(4, None, 3, 9, None) == 5
     m = qmm.MoeArgs(0, 2048, 768, 128, 8, 4, a, a, a, a, a, a, None, None, None, None, None, None)
     assert L.qmm_moe(ctypes.byref(m), None, 0, None) == 0
     assert L.qmm_moe_route(ctypes.byref(m), None, 0, None) == 0
