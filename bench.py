@@ -920,6 +920,19 @@ def run_case(args):
         arr = qmm.gemv_batch_problems(probs)
         for _ in range(reps):
             qmm.gemv_batch(f, arr)
+    elif name in ("gemm_batch_q4_M8", "gemm_batch_q8_M8"):
+        # the whole decode stack for a batch of 8 sequences: 112 problems in one qmm_gemm_batch launch
+        f = synth.Q4 if "_q4_" in name else synth.Q8
+        host_blocks, host_acts = build_stack_host(synth.CFG1["layers"], (f,))
+        probs = []
+        for l in range(synth.CFG1["layers"]):
+            for mname, N, K, act in synth.CFG1_LAYER:
+                probs.append((qmm.pack(f, dev(host_blocks[f][l][mname]), N, K), N, K,
+                              dev(host_acts[l][act]).reshape(1, K).repeat(8, 1).contiguous(),
+                              torch.empty((8, N), dtype=torch.float16, device="cuda")))
+        arr = qmm.gemm_batch_problems(probs)
+        for _ in range(reps):
+            qmm.gemm_batch(f, arr)
     elif name in ("chain_q4_dependent", "chain_q4_independent", "chain_q8_dependent", "chain_q8_independent"):
         # four layers of the decode stack (137 / 258 MB of weights) through qmm_chain: as a dependent chain of
         # 16 stages, or as 28 independent products
@@ -1010,7 +1023,7 @@ def run_case(args):
             qmm.moe(a, ws)
         qmm.status_check(ws)
     else:
-        raise SystemExit("unknown --case %r (gemv_batch_q4|q8, gemv_lm_head_q8, gemv_kv_q4|q8, gemm_q4|q8[_down]_M<M>, gemm_few_q4|q8_M<M>, "
+        raise SystemExit("unknown --case %r (gemv_batch_q4|q8, gemm_batch_q4|q8_M8, gemv_lm_head_q8, gemv_kv_q4|q8, gemm_q4|q8[_down]_M<M>, gemm_few_q4|q8_M<M>, "
                          "moe_q4|q8_T<T>, chain_q4|q8_dependent|independent)" % name)
     torch.cuda.synchronize()
     print("case %s: %d launches done" % (name, reps), file=sys.stderr)

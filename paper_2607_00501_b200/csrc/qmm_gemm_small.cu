@@ -148,12 +148,11 @@ __device__ __forceinline__ void frag_mma_x(const SmallSlot<FMT>& r, const FragRe
 // ------------------------------------------------------------------ the ring
 //
 // The tile pairs in flight are held in shared memory, not in registers: every warp owns a ring of
-// kRingStages slots and fills them with 16-byte asynchronous copies -- each lane copies the two halves
+// few slots and fills them with 16-byte asynchronous copies -- each lane copies the two halves
 // of its row straight to their transposed places, the first lanes the scale (and high-bit) planes as
 // they are -- one commit group per tile pair.  Nothing is held in registers while the copies fly, so
 // the ring is deep and the loop needs no register double buffer; the copies of the block's next work
 // item run under the reduction of the current one.
-constexpr int kRingStages = 4;
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src)
 {
@@ -241,32 +240,40 @@ __device__ __forceinline__ void ring_read(uint32_t slot, SmallSlot<FMT>& r, Frag
     }
 }
 
-// Dynamic shared memory: WARPS * kRingStages slots, WARPS * 8*NG * 64 floats for the warps' sums, and
+// Ring depth and resident blocks per SM.  One product at a time (gemm_small_kernel): 4 slots, 2 blocks of
+// 128 registers for every format.  The batched launch: the same for the 4-bit formats, which are bound by
+// instruction issue; Q8, bound by memory latency, runs 3 blocks with 2 slots each (measured both ways;
+// for single products chained on a stream that geometry was slower).
+constexpr int kDenseStages = 4;
+template <int FMT> struct SmallGeom { static constexpr int kStages = 4, kBlocks = 2; };
+template <> struct SmallGeom<QMM_Q8> { static constexpr int kStages = 2, kBlocks = 3; };
+
+// Dynamic shared memory: WARPS * kStages slots, WARPS * 8*NG * 64 floats for the warps' sums, and
 // (cluster form, used in the first block) 2 * splits * 8*NG * 64 floats.
 template <int FMT, int NG>
 __global__ void __launch_bounds__(kSmallWarps * 32, 2)
 gemm_small_kernel(const uint8_t* __restrict__ packed, const uint16_t* __restrict__ X, int64_t ldx,
                        uint16_t* __restrict__ Y, int64_t ldy, int M, int K, int tiles_per_row, int splits, int items)
 {
-    constexpr int WARPS = kSmallWarps, NT = 8 * NG;
+    constexpr int WARPS = kSmallWarps, NT = 8 * NG, kStages = kDenseStages;
     constexpr int TB = Fmt<FMT>::tile_bytes;
     constexpr int SLOT = 2 * TB;
     extern __shared__ uint4 smem[];
     const int tps = tiles_per_row / splits;                     // tiles per item
-    float* red = reinterpret_cast<float*>(smem + WARPS * kRingStages * SLOT / 16);   // behind the rings
+    float* red = reinterpret_cast<float*>(smem + WARPS * kStages * SLOT / 16);   // behind the rings
     float* cred = red + WARPS * NT * 64;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, t4 = lane & 3;
     const bool clustered = splits > 1;
     int cluster_round = 0;
-    const uint32_t ring = static_cast<uint32_t>(__cvta_generic_to_shared(smem)) + warp * (kRingStages * SLOT);
+    const uint32_t ring = static_cast<uint32_t>(__cvta_generic_to_shared(smem)) + warp * (kStages * SLOT);
 
     const size_t group_bytes = (size_t)tiles_per_row * TB;
     const int s = blockIdx.x % splits;                          // the same for every item of this block (grid = whole clusters)
     const int t_begin = s * tps + warp, t_end = (s + 1) * tps;
     const bool has_tiles = warp < tps;
 
-    // producer: runs kRingStages tile pairs ahead of the consumer, across work items
+    // producer: runs kStages tile pairs ahead of the consumer, across work items
     int p_item = blockIdx.x, p_t = t_begin;
     auto produce = [&](int stage) {
         if (has_tiles && p_item < items) {
@@ -281,7 +288,7 @@ gemm_small_kernel(const uint8_t* __restrict__ packed, const uint16_t* __restrict
         cp_async_commit();                                      // one group per call, empty or not
     };
 #pragma unroll
-    for (int st = 0; st < kRingStages; ++st) produce(st);       // weights never depend on the previous kernel
+    for (int st = 0; st < kStages; ++st) produce(st);       // weights never depend on the previous kernel
 
     pdl_launch_dependents();
     pdl_wait();                                                 // X may come from the previous kernel
@@ -323,7 +330,7 @@ gemm_small_kernel(const uint8_t* __restrict__ packed, const uint16_t* __restrict
             for (int tt = t_begin; tt < t_end; tt += WARPS) {
                 uint4 xr[FMT == QMM_Q8 ? 1 : 2][NG];
                 load_x(tt, xr);                                 // in flight while the tile pair lands
-                cp_async_wait<kRingStages - 1>();               // the oldest group -- this tile pair -- has landed
+                cp_async_wait<kStages - 1>();               // the oldest group -- this tile pair -- has landed
                 __syncwarp();
                 SmallSlot<FMT> r;
                 FragRegs<FMT> f;
@@ -331,7 +338,7 @@ gemm_small_kernel(const uint8_t* __restrict__ packed, const uint16_t* __restrict
                 __syncwarp();                                   // every lane has read the slot
                 produce(stage);
                 frag_mma_x<FMT, NG>(r, f, xr, t4, acc, kc);
-                stage = stage + 1 == kRingStages ? 0 : stage + 1;
+                stage = stage + 1 == kStages ? 0 : stage + 1;
             }
         }
         // red[warp][token][64]: rows 0..31 of P, then of Q
@@ -402,17 +409,17 @@ struct SmallBatchParams {
 };
 
 template <int FMT>
-__global__ void __launch_bounds__(kSmallWarps * 32, 2)
+__global__ void __launch_bounds__(kSmallWarps * 32, SmallGeom<FMT>::kBlocks)
 gemm_small_batch_kernel(const __grid_constant__ SmallBatchParams bp)
 {
-    constexpr int WARPS = kSmallWarps;
+    constexpr int WARPS = kSmallWarps, kSBStages = SmallGeom<FMT>::kStages;
     constexpr int TB = Fmt<FMT>::tile_bytes, TK = Fmt<FMT>::tile_k;
     constexpr int SLOT = 2 * TB;
     extern __shared__ uint4 smem[];
-    float* red_all = reinterpret_cast<float*>(smem + WARPS * kRingStages * SLOT / 16);   // [2][WARPS][8][64], behind the rings
+    float* red_all = reinterpret_cast<float*>(smem + WARPS * kSBStages * SLOT / 16);   // [2][WARPS][8][64], behind the rings
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, t4 = lane & 3;
-    const uint32_t ring = static_cast<uint32_t>(__cvta_generic_to_shared(smem)) + warp * (kRingStages * SLOT);
+    const uint32_t ring = static_cast<uint32_t>(__cvta_generic_to_shared(smem)) + warp * (kSBStages * SLOT);
     const int M = bp.M;
 
     // this block's range of the unit list, by cost; a unit belongs to the block whose range holds its first tile
@@ -431,26 +438,43 @@ gemm_small_batch_kernel(const __grid_constant__ SmallBatchParams bp)
     }
     auto valid = [&](int p, int u) { return p < bp.count && bp.p[p].cost_begin + u * bp.p[p].tpr < c1; };
 
-    // producer: runs kRingStages tile pairs ahead of the consumer, across units and problems
-    int p_pi = pi0, p_unit = unit0, p_t = warp;
-    auto produce = [&](int stage) {
-        while (valid(p_pi, p_unit) && p_t >= bp.p[p_pi].tpr) {  // this warp has no (more) tiles in the unit
+    // producer: runs kSBStages tile pairs ahead of the consumer, across units and problems
+    int p_pi = pi0, p_unit = unit0, p_left = 0;                 // p_left: this warp's tiles still to request in the unit
+    const uint8_t* p_tp = nullptr;
+    size_t p_gb = 0;
+    auto p_open = [&]() {                                       // the first unit from (p_pi, p_unit) on in which this warp has tiles
+        while (valid(p_pi, p_unit)) {
+            const int tpr = bp.p[p_pi].tpr;
+            if (warp < tpr) {
+                p_gb = (size_t)tpr * TB;
+                p_tp = bp.p[p_pi].packed + (size_t)(2 * p_unit) * p_gb + (size_t)warp * TB;
+                p_left = (tpr - warp + WARPS - 1) / WARPS;
+                return;
+            }
             if (++p_unit >= bp.p[p_pi].pairs) {
                 ++p_pi;
                 p_unit = 0;
             }
-            p_t = warp;
         }
-        if (valid(p_pi, p_unit)) {
-            const size_t group_bytes = (size_t)bp.p[p_pi].tpr * TB;
-            const uint8_t* tp = bp.p[p_pi].packed + (size_t)(2 * p_unit) * group_bytes + (size_t)p_t * TB;
-            ring_issue<FMT>(ring + stage * SLOT, tp, tp + group_bytes, lane);
-            p_t += WARPS;
+        p_left = 0;
+    };
+    p_open();
+    auto produce = [&](int stage) {
+        if (p_left) {
+            ring_issue<FMT>(ring + stage * SLOT, p_tp, p_tp + p_gb, lane);
+            p_tp += WARPS * TB;
+            if (--p_left == 0) {
+                if (++p_unit >= bp.p[p_pi].pairs) {
+                    ++p_pi;
+                    p_unit = 0;
+                }
+                p_open();
+            }
         }
         cp_async_commit();                                      // one group per call, empty or not
     };
 #pragma unroll
-    for (int st = 0; st < kRingStages; ++st) produce(st);       // weights never depend on the previous kernel
+    for (int st = 0; st < kSBStages; ++st) produce(st);       // weights never depend on the previous kernel
 
     pdl_launch_dependents();
     pdl_wait();                                                 // activations may come from the previous kernel
@@ -481,7 +505,7 @@ gemm_small_batch_kernel(const __grid_constant__ SmallBatchParams bp)
                     }
                 }
             }
-            cp_async_wait<kRingStages - 1>();                   // the oldest group -- this tile pair -- has landed
+            cp_async_wait<kSBStages - 1>();                   // the oldest group -- this tile pair -- has landed
             __syncwarp();
             SmallSlot<FMT> r;
             FragRegs<FMT> f;
@@ -489,7 +513,7 @@ gemm_small_batch_kernel(const __grid_constant__ SmallBatchParams bp)
             __syncwarp();                                       // every lane has read the slot
             produce(stage);
             frag_mma_x<FMT, 1>(r, f, xr, t4, acc, kc);
-            stage = stage + 1 == kRingStages ? 0 : stage + 1;
+            stage = stage + 1 == kSBStages ? 0 : stage + 1;
         }
         // red[warp][token][64]: rows 0..31 of P, then of Q
 #pragma unroll
@@ -540,16 +564,14 @@ static SmallPlan small_plan(int fmt, int64_t M, int64_t N, int64_t K)
     const int ng = (int)((M + 7) / 8), nt = 8 * ng;
     const int tpr = (int)(K / tile_k_of(fmt));
     const int pairs = (int)(N / 64);
-    const int per_sm = 2;
+    const int per_sm = 2, stages = kDenseStages;
     auto smem_of = [&](int splits) {
-        return (size_t)kSmallWarps * kRingStages * 2 * tile_bytes_of(fmt) + (size_t)kSmallWarps * nt * 64 * sizeof(float) +
+        return (size_t)kSmallWarps * stages * 2 * tile_bytes_of(fmt) + (size_t)kSmallWarps * nt * 64 * sizeof(float) +
                (splits > 1 ? (size_t)2 * splits * nt * 64 * sizeof(float) : 0);
     };
     int splits = 1;
     // split K while the pairs alone leave SMs without a block, every warp keeps a tile, and the cluster stays small
     while (pairs * splits < kNumSMs * per_sm && tpr % (splits * 2) == 0 && tpr / (splits * 2) >= kSmallWarps / 2 && splits < 4) splits *= 2;
-    // ... and, whatever the grid, until the activations of the block's K range fit in shared memory
-    while (smem_of(splits) > 200 * 1024 && tpr % (splits * 2) == 0 && splits < kSmallMaxSplits) splits *= 2;
     SmallPlan p;
     p.splits = splits;
     p.smem = smem_of(splits);
@@ -632,8 +654,10 @@ qmm_status launch_gemm_small_batch(int fmt, const qmm_gemm_problem* probs, int c
             if (cost > 0x7FFFFFFFLL) return fail(QMM_ERR_UNSUPPORTED, "qmm_gemm_batch: batch too large for one launch");
         }
         bp.total_cost = (int)cost;
-        const size_t smem = (size_t)kSmallWarps * kRingStages * 2 * tile_bytes_of(fmt) + (size_t)2 * kSmallWarps * 8 * 64 * sizeof(float);
-        int grid = 2 * kNumSMs;
+        const int stages = fmt == QMM_Q8 ? SmallGeom<QMM_Q8>::kStages : SmallGeom<QMM_Q4>::kStages;
+        const int blocks = fmt == QMM_Q8 ? SmallGeom<QMM_Q8>::kBlocks : SmallGeom<QMM_Q4>::kBlocks;
+        const size_t smem = (size_t)kSmallWarps * stages * 2 * tile_bytes_of(fmt) + (size_t)2 * kSmallWarps * 8 * 64 * sizeof(float);
+        int grid = blocks * kNumSMs;
         if (units < grid) grid = units;
         void (*kern)(SmallBatchParams) = fmt == QMM_Q4   ? gemm_small_batch_kernel<QMM_Q4>
                                          : fmt == QMM_Q5 ? gemm_small_batch_kernel<QMM_Q5>

@@ -165,7 +165,7 @@ def test_gemm_batch_mixed_shapes(qmm, oracle, fmt, M):
 def test_gemm_batch_rows_equal_qmm_gemm(qmm, fmt):
     """Where qmm_gemm does not split K across blocks (many row groups) the two calls add in the same order:
     the batched launch gives the same bits, and a row does not depend on M."""
-    N, K, M = 19200, 512, 6
+    N, K, M = 38400, 512, 6
     blocks = synth.quantize(fmt, synth.weights(98, fmt, N, K))
     packed = qmm.pack(fmt, util.dev(blocks), N, K)
     X = util.dev(synth.activations(98, 1, M, K))
