@@ -629,8 +629,32 @@ qmm_status launch_gemm_small(int fmt, const void* packed, int64_t N, int64_t K, 
 }
 
 // Host side of qmm_gemm_batch: up to kSmallMaxBatch problems per launch.
+qmm_status launch_gemv_batch(int fmt, const qmm_gemv_problem* probs, int count, cudaStream_t st, bool out_f32);
+
 qmm_status launch_gemm_small_batch(int fmt, const qmm_gemm_problem* probs, int count, int64_t M, cudaStream_t st)
 {
+    if (M == 1) {
+        // one token: the single-token batched kernel (its activations are staged in shared memory: K <= 32768)
+        bool fits = true;
+        for (int i = 0; i < count; ++i) fits = fits && probs[i].K <= 32768;
+        if (fits) {
+            for (int first = 0; first < count; first += kSmallMaxBatch) {
+                const int n = count - first < kSmallMaxBatch ? count - first : kSmallMaxBatch;
+                qmm_gemv_problem v[kSmallMaxBatch];
+                for (int i = 0; i < n; ++i) {
+                    const qmm_gemm_problem& q = probs[first + i];
+                    v[i].packed = q.packed;
+                    v[i].x_fp16 = q.X_fp16;
+                    v[i].y_fp16 = q.Y_fp16;
+                    v[i].N = q.N;
+                    v[i].K = q.K;
+                }
+                const qmm_status s = launch_gemv_batch(fmt, v, n, st, false);
+                if (s != QMM_OK) return s;
+            }
+            return QMM_OK;
+        }
+    }
     for (int first = 0; first < count; first += kSmallMaxBatch) {
         const int n = count - first < kSmallMaxBatch ? count - first : kSmallMaxBatch;
         SmallBatchParams bp = {};
