@@ -359,7 +359,7 @@ class Chain:
 
 
 def packed_check(fmt: int, packed: torch.Tensor, N: int, K: int, ws: torch.Tensor) -> None:
-    """Enqueue the plausibility check of a packed buffer; status_check(ws) reports the verdict."""
+    """Enqueue the plausibility check of a packed buffer; status_check(ws) reports the outcome."""
     _check(lib().qmm_packed_check(fmt, packed.data_ptr(), N, K, ws.data_ptr(), _stream()))
 
 
