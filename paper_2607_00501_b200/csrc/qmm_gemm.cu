@@ -222,7 +222,8 @@ static RoundCost round_cost(int64_t tiles, int64_t kb, int64_t stage, int64_t ha
 
 // Workspace of qmm_gemm: [0, 4) status word, [4096, 8192) trace samples (tuning aid), then the
 // partial-sum slots.
-constexpr size_t kGemmWsTrace = 4096, kGemmWsHeader = 8192;
+[[maybe_unused]] constexpr size_t kGemmWsTrace = 4096;
+constexpr size_t kGemmWsHeader = 8192;
 
 // Token tile: 256 (the widest MMA, N = 256) once M exceeds one 128-token tile, else the smallest
 // that holds M -- or half / a quarter of that when this yields between 3/4 and one round of whole

@@ -393,7 +393,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
     const int m_tiles = grouped ? *p.num_tiles : (p.M + BN - 1) / BN;
     const int total_tiles = n_tiles * m_tiles;
     const int KB = p.K / kGemmBK;                                         // k-blocks per tile
-    const int U = grouped ? 0 : p.units_per_block;
+    const int U = DENSE && !grouped ? p.units_per_block : 0;           // (a compile-time 0 in the grouped kernels)
 
     // ---- set-up
     if (threadIdx.x == 0) {
@@ -469,8 +469,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             const long long tb = (long long)t * KB;                       // first unit of tile t
             w.kb0 = (int)max(u0 - tb, 0LL);
             w.kb1 = (int)min(u1 - tb, (long long)KB);
-            w.first = (int)(tb / U);
-            w.cn = (int)((tb + KB - 1) / U) - w.first + 1;
+            const int Ud = U > 0 ? U : 1;                                 // (U > 0 here; spelled out for the grouped instantiations)
+            w.first = (int)(tb / Ud);
+            w.cn = (int)((tb + KB - 1) / Ud) - w.first + 1;
             t += t0;
         } else {
             if (grouped && p.tile_counter != nullptr) {
