@@ -61,7 +61,8 @@
  *   fp32).  Scales must be finite.
  *
  * Accuracy.  With y_ref and sum|w x| evaluated exactly, every output of every
- * product satisfies |y - y_ref| <= 2e-3 * sum_k |w_k x_k| + 1e-5.  The GEMVs
+ * product satisfies |y - y_ref| <= 2e-3 * sum_k |w_k x_k| + 1e-5 (outputs are
+ * fp16: an exact result beyond 65504 in magnitude is stored as infinity).  The GEMVs
  * (qmm_gemv*, decode-sized qmm_moe) multiply integer codes by activations
  * exactly and apply the scale in fp32, so this holds for every finite scale.
  * So does qmm_gemm for M <= 8 (its few-token kernel works the same way).
