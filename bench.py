@@ -640,24 +640,26 @@ def extra_sections(args, qmm, torch, pk, ops, fmts, batch, gpu_index=0):
                                                            "ms_tensor_core_kernel": round(med8t, 4)}, **hbm_fracs(b, med8, pk))
         del g8, g8t, ops8
 
-    # the whole decode stack for a batch of 8 sequences as ONE launch per format (qmm_gemm_batch: the 112
-    # matrices as independent problems, X [8, K] each): the weights are streamed once for all eight tokens,
-    # so the algorithmic bytes are those of the single-token step
+    # the whole decode stack for a batch of 2 / 8 sequences as ONE launch per format (qmm_gemm_batch: the 112
+    # matrices as independent problems, X [M, K] each): the weights are streamed once for all tokens, so the
+    # algorithmic bytes are those of the single-token step.  Two sequences ride in the single-token kernel's
+    # MMAs (the half of the B operand it leaves zero); eight run on the few-token ring kernel.
     for f in (fmts if on("batch8") else ()):
-        probs8 = []
-        for w, N, K, x, y in batch[f]._keep:
-            probs8.append((w, N, K, x.reshape(1, K).repeat(8, 1).contiguous(), torch.empty((8, N), dtype=torch.float16, device="cuda")))
-        arr8 = qmm.gemm_batch_problems(probs8)
-        g = torch.cuda.CUDAGraph()
-        s = torch.cuda.Stream()
-        with torch.cuda.stream(s):
-            qmm.gemm_batch(f, arr8)
-            torch.cuda.synchronize()
-            with torch.cuda.graph(g, stream=s):
-                qmm.gemm_batch(f, arr8)
-            m = measure(torch, g.replay, flush)
-        out["decode_stack_q%d_batch8_one_launch" % f] = dict(m, tokens=8, problems=len(probs8), **hbm_fracs(stack_bytes(f), m["ms"], pk))
-        del g, arr8, probs8
+        for Mb in (2, 8):
+            probs_m = []
+            for w, N, K, x, y in batch[f]._keep:
+                probs_m.append((w, N, K, x.reshape(1, K).repeat(Mb, 1).contiguous(), torch.empty((Mb, N), dtype=torch.float16, device="cuda")))
+            arr_m = qmm.gemm_batch_problems(probs_m)
+            g = torch.cuda.CUDAGraph()
+            s = torch.cuda.Stream()
+            with torch.cuda.stream(s):
+                qmm.gemm_batch(f, arr_m)
+                torch.cuda.synchronize()
+                with torch.cuda.graph(g, stream=s):
+                    qmm.gemm_batch(f, arr_m)
+                m = measure(torch, g.replay, flush)
+            out["decode_stack_q%d_batch%d_one_launch" % (f, Mb)] = dict(m, tokens=Mb, problems=len(probs_m), **hbm_fracs(stack_bytes(f), m["ms"], pk))
+            del g, arr_m, probs_m
 
     # cfg0: one small Q4 GEMV (1.77 MB of weights: 0.27 us of HBM traffic, far below a launch).  Steady
     # state = 300 distinct packed copies (531 MB, larger than L2) so that every product streams from HBM:

@@ -296,7 +296,8 @@ qmm_status qmm_chain_run(const qmm_chain_info* info, void* stream);
  * product is bound by streaming W once, like decode (Sec. 3.3), and runs on a
  * kernel of the decode family instead: integer codes times activations on the
  * warp-level tensor path, scales applied in fp32, no workspace use; row m of Y
- * is then the same bits whatever M (<= 8) is and whatever the other rows hold.
+ * is then the same bits whatever the other rows hold and whatever M in 2..8 is
+ * (M = 1 runs on the qmm_gemv kernel, which adds in another order).
  *   X_fp16  device, [M, ldx] fp16 row-major, ldx >= K, ldx % 8 == 0
  *   Y_fp16  device, [M, ldy] fp16 row-major, ldy >= N, ldy % 8 == 0, written
  *   ws      device, at least qmm_gemm_workspace_bytes(...) bytes: the status
@@ -319,7 +320,9 @@ qmm_status qmm_gemm(qmm_format fmt, const void* packed, int64_t N, int64_t K,
  * bound by streaming the weights, which this launch does once for all M
  * tokens).  The products must be independent, as for qmm_gemv_batch.  Integer
  * codes times activations, scales applied in fp32 (the accuracy of the GEMVs);
- * row m of Y_i does not depend on M or on the other rows.  No workspace.
+ * row m of Y_i does not depend on the other rows, nor on M within 3..8 (one and
+ * two tokens run on the single-token batched kernel: two tokens cost what one
+ * costs there).  No workspace.
  *   problems  HOST array of `count` descriptors (read during the call only);
  *             pointers inside are device pointers: packed 32-byte aligned,
  *             X [M, ldx] and Y [M, ldy] fp16 row-major, 16-byte aligned,

@@ -631,8 +631,17 @@ qmm_status launch_gemm_small(int fmt, const void* packed, int64_t N, int64_t K, 
 // Host side of qmm_gemm_batch: up to kSmallMaxBatch problems per launch.
 qmm_status launch_gemv_batch(int fmt, const qmm_gemv_problem* probs, int count, cudaStream_t st, bool out_f32);
 
+qmm_status launch_gemv_batch_two(int fmt, const qmm_gemm_problem* probs, int count, cudaStream_t st);
+
 qmm_status launch_gemm_small_batch(int fmt, const qmm_gemm_problem* probs, int count, int64_t M, cudaStream_t st)
 {
+    if (M == 2) {
+        // two tokens: the single-token batched kernel carries the second token in the idle half of its
+        // MMAs' B operand (activations staged in shared memory: K <= 32768)
+        bool fits = true;
+        for (int i = 0; i < count; ++i) fits = fits && probs[i].K <= 32768;
+        if (fits) return launch_gemv_batch_two(fmt, probs, count, st);
+    }
     if (M == 1) {
         // one token: the single-token batched kernel (its activations are staged in shared memory: K <= 32768)
         bool fits = true;

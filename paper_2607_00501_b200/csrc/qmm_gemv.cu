@@ -205,6 +205,8 @@ struct BatchProblem {
     const uint8_t* packed;
     const uint16_t* x;
     uint16_t* y;
+    const uint16_t* x2;   // TWO form: the second token's activations and outputs
+    uint16_t* y2;
     int K;            // input features
     int tpr;          // tiles per row
     int pairs;        // N / 64
@@ -219,17 +221,22 @@ struct BatchParams {
     BatchProblem p[kMaxBatch];
 };
 
-template <int FMT, int WARPS>
+// TWO: every problem has two activation vectors (two decode sequences).  The one-row-per-lane MMA
+// scheme leaves B columns 4..7 zero; the second token rides there (column 4+j = its quadruple in slot
+// group j: lanes with g == t + 4 read it), so both products cost the MMAs of one, and the lanes with
+// t >= 2, idle otherwise, receive the second token's sums (rows 4g+2(t-2), +1 of both row groups).
+template <int FMT, int WARPS, bool TWO = false>
 #ifndef QMM_BATCH_THREADS_PER_SM
 #define QMM_BATCH_THREADS_PER_SM 768
 #endif
 __global__ void __launch_bounds__(WARPS * 32, QMM_BATCH_THREADS_PER_SM / (WARPS * 32))
 gemv_batch_kernel(const __grid_constant__ BatchParams bp)
 {
+    constexpr int NTOK = TWO ? 2 : 1;
     extern __shared__ uint4 smem[];
-    uint4* xs = smem;
-    uint4* zs = smem + bp.max_k / 8;
-    float* red = reinterpret_cast<float*>(smem + bp.max_k / 4);
+    uint4* xs = smem;                                           // [NTOK][max_k / 8]
+    uint4* zs = smem + NTOK * (bp.max_k / 8);
+    float* red = reinterpret_cast<float*>(zs + bp.max_k / 8);   // [WARPS][NTOK][64]
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     constexpr int TB = Fmt<FMT>::tile_bytes;
     constexpr int XV = Fmt<FMT>::tile_k / 8;
@@ -287,10 +294,15 @@ gemv_batch_kernel(const __grid_constant__ BatchParams bp)
     pdl_launch_dependents();
     pdl_wait();                                                 // activations may come from the previous kernel
     for (int i = threadIdx.x; i < bp.max_k / 8; i += WARPS * 32) zs[i] = make_uint4(0u, 0u, 0u, 0u);
-    if (have)
-        for (int i = threadIdx.x; i < bp.p[pi].K / 8; i += WARPS * 32) xs[i] = reinterpret_cast<const uint4*>(bp.p[pi].x)[i];
+    auto stage_x = [&](int p) {
+        for (int i = threadIdx.x; i < bp.p[p].K / 8; i += WARPS * 32) {
+            xs[i] = reinterpret_cast<const uint4*>(bp.p[p].x)[i];
+            if (TWO) xs[bp.max_k / 8 + i] = reinterpret_cast<const uint4*>(bp.p[p].x2)[i];
+        }
+    };
+    if (have) stage_x(pi);
     __syncthreads();
-    const uint4* xb = ((lane >> 2) == (lane & 3)) ? xs : zs;
+    const uint4* xb = ((lane >> 2) == (lane & 3)) ? xs : (TWO && (lane >> 2) == (lane & 3) + 4) ? xs + bp.max_k / 8 : zs;
     Q4Consts kc;
     kc.init();
 
@@ -315,26 +327,26 @@ gemv_batch_kernel(const __grid_constant__ BatchParams bp)
             open_unit(pi, unit);
             load_group();
         }
-        if ((lane & 3) < 2) {
+        if (TWO || (lane & 3) < 2) {
             const int row = (lane & ~3) + 2 * (lane & 1);
-            float* w = red + warp * 64;
+            float* w = red + (warp * NTOK + (TWO ? (lane & 3) >> 1 : 0)) * 64;
             w[row] = acc[0];
             w[row + 1] = acc[1];
             w[32 + row] = acc[2];
             w[32 + row + 1] = acc[3];
         }
         __syncthreads();                                        // also: every warp is done with xs
-        if (threadIdx.x < 64) {
+        if (threadIdx.x < 64 * NTOK) {
             float sum = red[threadIdx.x];
 #pragma unroll
-            for (int w = 1; w < WARPS; ++w) sum += red[w * 64 + threadIdx.x];
+            for (int w = 1; w < WARPS; ++w) sum += red[w * 64 * NTOK + threadIdx.x];
+            uint16_t* yt = TWO && threadIdx.x >= 64 ? bp.p[done_p].y2 : bp.p[done_p].y;
             if (bp.out_f32)
-                reinterpret_cast<float*>(bp.p[done_p].y)[done_u * 64 + threadIdx.x] = sum;
+                reinterpret_cast<float*>(yt)[done_u * 64 + (threadIdx.x & 63)] = sum;
             else
-                bp.p[done_p].y[done_u * 64 + threadIdx.x] = __half_as_ushort(__float2half_rn(sum));
+                yt[done_u * 64 + (threadIdx.x & 63)] = __half_as_ushort(__float2half_rn(sum));
         }
-        if (have && pi != done_p)                               // next unit reads another activation vector
-            for (int i = threadIdx.x; i < bp.p[pi].K / 8; i += WARPS * 32) xs[i] = reinterpret_cast<const uint4*>(bp.p[pi].x)[i];
+        if (have && pi != done_p) stage_x(pi);                  // next unit reads other activation vectors
         __syncthreads();
     }
 }
@@ -1083,6 +1095,51 @@ qmm_status launch_gemv_batch(int fmt, const qmm_gemv_problem* probs, int count, 
         else QMM_BATCH_CASE(QMM_Q8)
 #undef QMM_BATCH_CASE
         if (e != cudaSuccess) return check_cuda(e, "qmm_gemv_batch launch");
+    }
+    return QMM_OK;
+}
+
+// qmm_gemm_batch for two tokens: the batched kernel's TWO form (both tokens at the cost of one).
+qmm_status launch_gemv_batch_two(int fmt, const qmm_gemm_problem* probs, int count, cudaStream_t st)
+{
+    for (int first = 0; first < count; first += kMaxBatch) {
+        const int n = count - first < kMaxBatch ? count - first : kMaxBatch;
+        BatchParams bp = {};
+        bp.count = n;
+        int cost = 0, max_k = 0;
+        for (int i = 0; i < n; ++i) {
+            const qmm_gemm_problem& q = probs[first + i];
+            BatchProblem& b = bp.p[i];
+            b.packed = (const uint8_t*)q.packed;
+            b.x = q.X_fp16;
+            b.x2 = q.X_fp16 + q.ldx;
+            b.y = q.Y_fp16;
+            b.y2 = q.Y_fp16 + q.ldy;
+            b.K = (int)q.K;
+            b.tpr = (int)(q.K / tile_k_of(fmt));
+            b.pairs = (int)(q.N / (2 * kRowsPerGroup));
+            b.cost_begin = cost;
+            if ((long long)cost + (long long)b.pairs * b.tpr > 0x7FFFFFFFLL)
+                return fail(QMM_ERR_UNSUPPORTED, "qmm_gemm_batch: batch too large for one launch");
+            cost += b.pairs * b.tpr;
+            if (b.K > max_k) max_k = b.K;
+        }
+        bp.total_cost = cost;
+        bp.max_k = max_k;
+        constexpr int WARPS = 8;
+        const size_t smem = (size_t)max_k * 6 + (size_t)WARPS * 128 * sizeof(float);
+        const int units = cost / (max_k / tile_k_of(fmt)) + 1;
+        int grid = kNumSMs * (QMM_BATCH_THREADS_PER_SM / (WARPS * 32));
+        if (units < grid) grid = units;
+        void (*kern)(BatchParams) = fmt == QMM_Q4   ? gemv_batch_kernel<QMM_Q4, WARPS, true>
+                                    : fmt == QMM_Q5 ? gemv_batch_kernel<QMM_Q5, WARPS, true>
+                                    : fmt == QMM_Q6 ? gemv_batch_kernel<QMM_Q6, WARPS, true>
+                                                    : gemv_batch_kernel<QMM_Q8, WARPS, true>;
+        cudaError_t e = cudaSuccess;
+        if (smem > 48 * 1024) e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return check_cuda(e, "qmm_gemm_batch shared memory size");
+        e = launch_pdl(kern, dim3(grid), dim3(WARPS * 32), smem, st, bp);
+        if (e != cudaSuccess) return check_cuda(e, "qmm_gemm_batch launch");
     }
     return QMM_OK;
 }

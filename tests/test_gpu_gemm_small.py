@@ -134,7 +134,7 @@ def test_few_tokens_on_the_full_size_prefill_shapes(qmm, oracle, shape, M):
 # ------------------------------------------------------------------ qmm_gemm_batch
 
 @pytest.mark.parametrize("fmt", FMTS)
-@pytest.mark.parametrize("M", [1, 3, 8])
+@pytest.mark.parametrize("M", [1, 2, 3, 8])
 def test_gemm_batch_mixed_shapes(qmm, oracle, fmt, M):
     """One launch over problems that differ in N and K (short K: fewer tiles than warps; long K; many
     row groups), strided X and Y with guard values; every output against the oracle; repeatable."""
@@ -164,7 +164,8 @@ def test_gemm_batch_mixed_shapes(qmm, oracle, fmt, M):
 @pytest.mark.parametrize("fmt", [4, 8])
 def test_gemm_batch_rows_equal_qmm_gemm(qmm, fmt):
     """Where qmm_gemm does not split K across blocks (many row groups) the two calls add in the same order:
-    the batched launch gives the same bits, and a row does not depend on M."""
+    the batched launch gives the same bits, and a row does not depend on M (3 <= M <= 8: one and two
+    tokens run on the single-token kernels, which add in another order)."""
     N, K, M = 38400, 512, 6
     blocks = synth.quantize(fmt, synth.weights(98, fmt, N, K))
     packed = qmm.pack(fmt, util.dev(blocks), N, K)
@@ -173,15 +174,16 @@ def test_gemm_batch_rows_equal_qmm_gemm(qmm, fmt):
     Y2 = torch.empty_like(Y1)
     qmm.gemm_batch(fmt, qmm.gemm_batch_problems([(packed, N, K, X, Y2)]))
     assert torch.equal(Y1, Y2)
-    Y3 = torch.empty((2, N), dtype=torch.float16, device="cuda")
-    qmm.gemm_batch(fmt, qmm.gemm_batch_problems([(packed, N, K, X[4:6], Y3)]))
-    assert torch.equal(Y3, Y1[4:6])
+    Y3 = torch.empty((3, N), dtype=torch.float16, device="cuda")
+    qmm.gemm_batch(fmt, qmm.gemm_batch_problems([(packed, N, K, X[3:6], Y3)]))
+    assert torch.equal(Y3, Y1[3:6])
 
 
 @pytest.mark.parametrize("fmt", [4, 8])
-def test_cfg1_two_layers_full_size_for_a_batch_of_eight(qmm, oracle, fmt):
-    """All 14 matrices of two decoder layers at their real sizes for 8 sequences in one launch."""
-    M = 8
+@pytest.mark.parametrize("M", [2, 8])
+def test_cfg1_two_layers_full_size_for_a_batch_of_sequences(qmm, oracle, fmt, M):
+    """All 14 matrices of two decoder layers at their real sizes for 2 / 8 sequences in one launch (two
+    sequences ride in the single-token kernel's MMAs, eight run on the few-token ring kernel)."""
     probs, refs = [], []
     for layer in (0, 15):
         for name, N, K, act, w in synth.cfg1_layer_weights(layer):
@@ -193,7 +195,7 @@ def test_cfg1_two_layers_full_size_for_a_batch_of_eight(qmm, oracle, fmt):
     qmm.gemm_batch(fmt, qmm.gemm_batch_problems(probs))
     torch.cuda.synchronize()
     for (p, N, K, X, Y), (name, (Y_ref, B)) in zip(probs, refs):
-        util.assert_within_tol(util.host_f64(Y), Y_ref, B, "cfg1 batch of 8, %s" % name)
+        util.assert_within_tol(util.host_f64(Y), Y_ref, B, "cfg1 batch of %d, %s" % (M, name))
 
 
 def test_gemm_batch_more_problems_than_one_launch_holds(qmm, oracle):
