@@ -922,16 +922,17 @@ def run_case(args):
         arr = qmm.gemv_batch_problems(probs)
         for _ in range(reps):
             qmm.gemv_batch(f, arr)
-    elif name in ("gemm_batch_q4_M8", "gemm_batch_q8_M8"):
-        # the whole decode stack for a batch of 8 sequences: 112 problems in one qmm_gemm_batch launch
+    elif name in ("gemm_batch_q4_M8", "gemm_batch_q8_M8", "gemm_batch_q4_M2", "gemm_batch_q8_M2"):
+        # the whole decode stack for a batch of 8 (or 2) sequences: 112 problems in one qmm_gemm_batch launch
         f = synth.Q4 if "_q4_" in name else synth.Q8
+        Mb = int(name[-1])
         host_blocks, host_acts = build_stack_host(synth.CFG1["layers"], (f,))
         probs = []
         for l in range(synth.CFG1["layers"]):
             for mname, N, K, act in synth.CFG1_LAYER:
                 probs.append((qmm.pack(f, dev(host_blocks[f][l][mname]), N, K), N, K,
-                              dev(host_acts[l][act]).reshape(1, K).repeat(8, 1).contiguous(),
-                              torch.empty((8, N), dtype=torch.float16, device="cuda")))
+                              dev(host_acts[l][act]).reshape(1, K).repeat(Mb, 1).contiguous(),
+                              torch.empty((Mb, N), dtype=torch.float16, device="cuda")))
         arr = qmm.gemm_batch_problems(probs)
         for _ in range(reps):
             qmm.gemm_batch(f, arr)
@@ -1025,7 +1026,7 @@ def run_case(args):
             qmm.moe(a, ws)
         qmm.status_check(ws)
     else:
-        raise SystemExit("unknown --case %r (gemv_batch_q4|q8, gemm_batch_q4|q8_M8, gemv_lm_head_q8, gemv_kv_q4|q8, gemm_q4|q8[_down]_M<M>, gemm_few_q4|q8_M<M>, "
+        raise SystemExit("unknown --case %r (gemv_batch_q4|q8, gemm_batch_q4|q8_M2|M8, gemv_lm_head_q8, gemv_kv_q4|q8, gemm_q4|q8[_down]_M<M>, gemm_few_q4|q8_M<M>, "
                          "moe_q4|q8_T<T>, chain_q4|q8_dependent|independent)" % name)
     torch.cuda.synchronize()
     print("case %s: %d launches done" % (name, reps), file=sys.stderr)
