@@ -607,38 +607,40 @@ def extra_sections(args, qmm, torch, pk, ops, fmts, batch, gpu_index=0):
             med, best = time_op(torch, g.replay, 10)
         b = stack_bytes(f)
         out["decode_stack_q%d_chained" % f] = dict({"ms": round(med, 4), "launches": len(ops[f])}, **hbm_fracs(b, med, pk))
-        # the same chain for a decode batch of 8 tokens: qmm_gemm with M = 8 (few-token kernel) per fused
-        # matrix; the weights are streamed once for all eight tokens, so the bytes are the same
-        g8 = torch.cuda.CUDAGraph()
-        with torch.cuda.stream(s):
-            ops8 = []
-            for N, K, w, x, y, ws in ops[f]:
-                X8 = x.reshape(1, K).repeat(8, 1).contiguous()
-                Y8 = torch.empty((8, N), dtype=torch.float16, device="cuda")
-                ws8 = torch.zeros(max(qmm.gemm_workspace_bytes(f, 8, N, K), 256), dtype=torch.uint8, device="cuda")
-                ops8.append((N, K, w, X8, Y8, ws8))
-            for N, K, w, X8, Y8, ws8 in ops8[:4]:
-                qmm.gemm(f, w, N, K, X8, Y=Y8, ws=ws8)
-            torch.cuda.synchronize()
-            with torch.cuda.graph(g8, stream=s):
-                for N, K, w, X8, Y8, ws8 in ops8:
-                    qmm.gemm(f, w, N, K, X8, Y=Y8, ws=ws8)
-            med8, _ = time_op(torch, g8.replay, 10)
-            # for comparison: the same eight tokens through the tensor-core prefill kernel
-            qmm.debug_config("gemm_no_small", "1")
-            g8t = torch.cuda.CUDAGraph()
-            for N, K, w, X8, Y8, ws8 in ops8[:4]:
-                qmm.gemm(f, w, N, K, X8, Y=Y8, ws=ws8)
-            torch.cuda.synchronize()
-            with torch.cuda.graph(g8t, stream=s):
-                for N, K, w, X8, Y8, ws8 in ops8:
-                    qmm.gemm(f, w, N, K, X8, Y=Y8, ws=ws8)
-            qmm.debug_config("gemm_no_small", "0")
-            med8t, _ = time_op(torch, g8t.replay, 10)
-        out["decode_stack_q%d_chained_batch8" % f] = dict({"ms": round(med8, 4), "launches": len(ops8), "tokens": 8,
-                                                           "ms_over_single_token": round(med8 / med, 3),
-                                                           "ms_tensor_core_kernel": round(med8t, 4)}, **hbm_fracs(b, med8, pk))
-        del g8, g8t, ops8
+        # the same chain for a decode batch of 2 / 8 sequences: qmm_gemm with M = 2 (the single-token kernel
+        # with the second token in the idle half of its MMAs) / M = 8 (few-token kernel) per fused matrix;
+        # the weights are streamed once for all tokens, so the bytes are the same
+        for Mb in (2, 8):
+            gm = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(s):
+                opsm = []
+                for N, K, w, x, y, ws in ops[f]:
+                    Xm = x.reshape(1, K).repeat(Mb, 1).contiguous()
+                    Ym = torch.empty((Mb, N), dtype=torch.float16, device="cuda")
+                    wsm = torch.zeros(max(qmm.gemm_workspace_bytes(f, Mb, N, K), 256), dtype=torch.uint8, device="cuda")
+                    opsm.append((N, K, w, Xm, Ym, wsm))
+                for N, K, w, Xm, Ym, wsm in opsm[:4]:
+                    qmm.gemm(f, w, N, K, Xm, Y=Ym, ws=wsm)
+                torch.cuda.synchronize()
+                with torch.cuda.graph(gm, stream=s):
+                    for N, K, w, Xm, Ym, wsm in opsm:
+                        qmm.gemm(f, w, N, K, Xm, Y=Ym, ws=wsm)
+                medm, _ = time_op(torch, gm.replay, 10)
+                # for comparison: the same tokens through the tensor-core prefill kernel
+                qmm.debug_config("gemm_no_small", "1")
+                gt = torch.cuda.CUDAGraph()
+                for N, K, w, Xm, Ym, wsm in opsm[:4]:
+                    qmm.gemm(f, w, N, K, Xm, Y=Ym, ws=wsm)
+                torch.cuda.synchronize()
+                with torch.cuda.graph(gt, stream=s):
+                    for N, K, w, Xm, Ym, wsm in opsm:
+                        qmm.gemm(f, w, N, K, Xm, Y=Ym, ws=wsm)
+                qmm.debug_config("gemm_no_small", "0")
+                medt, _ = time_op(torch, gt.replay, 10)
+            out["decode_stack_q%d_chained_batch%d" % (f, Mb)] = dict({"ms": round(medm, 4), "launches": len(opsm), "tokens": Mb,
+                                                                      "ms_over_single_token": round(medm / med, 3),
+                                                                      "ms_tensor_core_kernel": round(medt, 4)}, **hbm_fracs(b, medm, pk))
+            del gm, gt, opsm
 
     # the whole decode stack for a batch of 2 / 8 sequences as ONE launch per format (qmm_gemm_batch: the 112
     # matrices as independent problems, X [M, K] each): the weights are streamed once for all tokens, so the

@@ -296,8 +296,9 @@ qmm_status qmm_chain_run(const qmm_chain_info* info, void* stream);
  * product is bound by streaming W once, like decode (Sec. 3.3), and runs on a
  * kernel of the decode family instead: integer codes times activations on the
  * warp-level tensor path, scales applied in fp32, no workspace use; row m of Y
- * is then the same bits whatever the other rows hold and whatever M in 2..8 is
- * (M = 1 runs on the qmm_gemv kernel, which adds in another order).
+ * is then the same bits whatever the other rows hold and whatever M in 3..8 is
+ * (M = 1 and M = 2 run on the qmm_gemv kernel -- two tokens cost what one costs
+ * there -- and give each row the bits of qmm_gemv).
  *   X_fp16  device, [M, ldx] fp16 row-major, ldx >= K, ldx % 8 == 0
  *   Y_fp16  device, [M, ldy] fp16 row-major, ldy >= N, ldy % 8 == 0, written
  *   ws      device, at least qmm_gemm_workspace_bytes(...) bytes: the status

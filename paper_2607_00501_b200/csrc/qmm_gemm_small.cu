@@ -553,6 +553,9 @@ bool gemm_small_supported(int fmt, int64_t M)
 qmm_status launch_gemv(int fmt, const void* packed, int64_t N, int64_t K, const uint16_t* x, uint16_t* y,
                        void* ws, bool allow_cluster, cudaStream_t st);
 size_t gemv_workspace_bytes(int fmt, int64_t N, int64_t K, bool allow_cluster);
+bool gemv_two_supported(int fmt, int64_t N, int64_t K);
+qmm_status launch_gemv_two(int fmt, const void* packed, int64_t N, int64_t K, const uint16_t* X, int64_t ldx, uint16_t* Y,
+                           int64_t ldy, cudaStream_t st);
 
 struct SmallPlan {
     int splits, grid;
@@ -616,6 +619,11 @@ qmm_status launch_gemm_small(int fmt, const void* packed, int64_t N, int64_t K, 
 {
     // one token: the single-token kernel (its cluster form needs no workspace)
     if (M == 1 && gemv_workspace_bytes(fmt, N, K, true) == 0) return launch_gemv(fmt, packed, N, K, X, Y, nullptr, true, st);
+    // two tokens: the same kernel, the second token in the half of the MMAs' B operand it leaves idle
+    if (M == 2 && gemv_two_supported(fmt, N, K)) {
+        const qmm_status s2 = launch_gemv_two(fmt, packed, N, K, X, ldx, Y, ldy, st);
+        if (s2 != QMM_ERR_UNSUPPORTED) return s2;
+    }
     const SmallPlan p = small_plan(fmt, M, N, K);
     const int ng = (int)((M + 7) / 8);
 #define QMM_SMALL_CASE(F, G) \

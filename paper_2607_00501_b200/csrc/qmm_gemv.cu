@@ -55,17 +55,26 @@ struct TileRegs {
 // GATEUP: the row-group pair of an item is (group j of `packed`, group j of `packed_up`) -- the gate
 // rows and the up rows of the same 32 outputs -- and the item writes h = fp16(silu(g) * u) for them
 // (no K split across blocks in this form).
-template <int FMT, int WARPS, bool GATEUP = false>
+//
+// TWO: two activation vectors (x and x + ldx2) against the same matrix, outputs to y and y + ldy2.  The
+// one-row-per-lane MMA scheme leaves B columns 4..7 zero; the second token rides there (column 4+j = its
+// quadruple in slot group j: lanes with g == t + 4 read it), so both products cost the MMAs of one, and
+// the lanes with t >= 2, idle otherwise, receive the second token's sums.  Each token's sums are added
+// exactly as in the single-token form (cluster form or no K split only).
+template <int FMT, int WARPS, bool GATEUP = false, bool TWO = false>
 __global__ void __launch_bounds__(WARPS * 32, 768 / (WARPS * 32))
 gemv_kernel(const uint8_t* __restrict__ packed, const uint16_t* __restrict__ x,
             uint16_t* __restrict__ y, float* __restrict__ partial,
-            int N, int K, int tiles_per_row, int splits, int items, const uint8_t* __restrict__ packed_up)
+            int N, int K, int tiles_per_row, int splits, int items, const uint8_t* __restrict__ packed_up,
+            int64_t ldx2, int64_t ldy2)
 {
+    static_assert(!(GATEUP && TWO), "the fused gate/up form takes one token");
+    constexpr int NTOK = TWO ? 2 : 1;
     extern __shared__ uint4 smem[];
-    uint4* xs = smem;
-    uint4* zs = smem + K / 8;
-    float* red = reinterpret_cast<float*>(smem + K / 4);
-    float* cred = red + WARPS * 64;                             // cluster form: [2][kMaxClusterSplits][64] in the first block
+    uint4* xs = smem;                                           // [NTOK][K / 8]
+    uint4* zs = smem + NTOK * (K / 8);
+    float* red = reinterpret_cast<float*>(zs + K / 8);          // [WARPS][NTOK][64]
+    float* cred = red + WARPS * NTOK * 64;                      // cluster form: [2][kMaxClusterSplits][NTOK * 64] in the first block
     const bool clustered = !GATEUP && splits > 1 && partial == nullptr;
     int cluster_round = 0;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -108,10 +117,11 @@ gemv_kernel(const uint8_t* __restrict__ packed, const uint16_t* __restrict__ x,
     pdl_wait();                                                 // x may come from the previous kernel
     for (int i = threadIdx.x; i < K / 8; i += WARPS * 32) {
         xs[i] = reinterpret_cast<const uint4*>(x)[i];
+        if (TWO) xs[K / 8 + i] = reinterpret_cast<const uint4*>(x + ldx2)[i];
         zs[i] = make_uint4(0u, 0u, 0u, 0u);
     }
     __syncthreads();
-    const uint4* xb = ((lane >> 2) == (lane & 3)) ? xs : zs;
+    const uint4* xb = ((lane >> 2) == (lane & 3)) ? xs : (TWO && (lane >> 2) == (lane & 3) + 4) ? xs + K / 8 : zs;
     Q4Consts kc;
     kc.init();
 
@@ -137,9 +147,9 @@ gemv_kernel(const uint8_t* __restrict__ packed, const uint16_t* __restrict__ x,
             load_group();
         }
         // add the warps' partial sums in warp order
-        if ((lane & 3) < 2) {                                   // lanes that received sums (see above)
+        if (TWO || (lane & 3) < 2) {                            // lanes that received sums (see above)
             const int row = (lane & ~3) + 2 * (lane & 1);
-            float* w = red + warp * 64;
+            float* w = red + (warp * NTOK + (TWO ? (lane & 3) >> 1 : 0)) * 64;
             w[row] = acc[0];
             w[row + 1] = acc[1];
             w[32 + row] = acc[2];
@@ -158,29 +168,30 @@ gemv_kernel(const uint8_t* __restrict__ packed, const uint16_t* __restrict__ x,
             }
         } else if (clustered) {
             // every block of the cluster runs the same sequence of items, one split each
-            float* slot = cred + (cluster_round & 1) * (kMaxClusterSplits * 64);
-            if (threadIdx.x < 64) {
+            float* slot = cred + (cluster_round & 1) * (kMaxClusterSplits * NTOK * 64);
+            if (threadIdx.x < NTOK * 64) {
                 float sum = red[threadIdx.x];
 #pragma unroll
-                for (int w = 1; w < WARPS; ++w) sum += red[w * 64 + threadIdx.x];
-                st_cluster_rank0(slot + done_s * 64 + threadIdx.x, sum);
+                for (int w = 1; w < WARPS; ++w) sum += red[w * NTOK * 64 + threadIdx.x];
+                st_cluster_rank0(slot + done_s * NTOK * 64 + threadIdx.x, sum);
             }
             cluster_sync();
-            if (done_s == 0 && threadIdx.x < 64) {
+            if (done_s == 0 && threadIdx.x < NTOK * 64) {
                 float total = slot[threadIdx.x];
-                for (int sp = 1; sp < splits; ++sp) total += slot[sp * 64 + threadIdx.x];
-                y[done_pair * 64 + threadIdx.x] = __half_as_ushort(__float2half_rn(total));
+                for (int sp = 1; sp < splits; ++sp) total += slot[sp * NTOK * 64 + threadIdx.x];
+                uint16_t* yt = TWO && threadIdx.x >= 64 ? y + ldy2 : y;
+                yt[done_pair * 64 + (threadIdx.x & 63)] = __half_as_ushort(__float2half_rn(total));
             }
             ++cluster_round;                                    // (two slots: the next item's sums do not wait for this read)
-        } else if (threadIdx.x < 64) {
+        } else if (threadIdx.x < NTOK * 64) {
             float sum = red[threadIdx.x];
 #pragma unroll
-            for (int w = 1; w < WARPS; ++w) sum += red[w * 64 + threadIdx.x];
-            const int n = done_pair * 64 + threadIdx.x;
+            for (int w = 1; w < WARPS; ++w) sum += red[w * NTOK * 64 + threadIdx.x];
+            const int n = done_pair * 64 + (threadIdx.x & 63);
             if (splits == 1)
-                y[n] = __half_as_ushort(__float2half_rn(sum));
+                (TWO && threadIdx.x >= 64 ? y + ldy2 : y)[n] = __half_as_ushort(__float2half_rn(sum));
             else
-                partial[(size_t)done_s * N + n] = sum;
+                partial[(size_t)done_s * N + n] = sum;              // (single token only)
         }
         __syncthreads();
     }
@@ -899,11 +910,11 @@ static qmm_status launch_gemv_t(const GemvPlan& p, const void* packed, int64_t N
         cfg.attrs = attr;
         cfg.numAttrs = 2;
         return check_cuda(cudaLaunchKernelEx(&cfg, kern, (const uint8_t*)packed, x, y, (float*)nullptr, (int)N, (int)K, tpr, p.splits,
-                                             items, (const uint8_t*)nullptr),
+                                             items, (const uint8_t*)nullptr, (int64_t)0, (int64_t)0),
                           "qmm_gemv cluster launch");
     }
     cudaError_t e = launch_pdl(kern, dim3(p.grid), dim3(WARPS * 32), smem, st,
-                               (const uint8_t*)packed, x, y, partial, (int)N, (int)K, tpr, p.splits, items, (const uint8_t*)nullptr);
+                               (const uint8_t*)packed, x, y, partial, (int)N, (int)K, tpr, p.splits, items, (const uint8_t*)nullptr, (int64_t)0, (int64_t)0);
     if (e != cudaSuccess) return check_cuda(e, "qmm_gemv launch");
     if (p.splits > 1) {
         e = launch_pdl(gemv_reduce_kernel, dim3((unsigned)((N + 255) / 256)), dim3(256), 0, st,
@@ -928,13 +939,13 @@ qmm_status launch_gemv_gate_up(int fmt, const void* packed_gate, const void* pac
         if (smem > 48 * 1024) e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e == cudaSuccess)
             e = launch_pdl(kern, dim3(grid), dim3(WARPS * 32), smem, st, (const uint8_t*)packed_gate, x, h, (float*)nullptr, (int)N,
-                           (int)K, tpr, 1, items, (const uint8_t*)packed_up);
+                           (int)K, tpr, 1, items, (const uint8_t*)packed_up, (int64_t)0, (int64_t)0);
     } else {
         auto kern = gemv_kernel<QMM_Q8, WARPS, true>;
         if (smem > 48 * 1024) e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e == cudaSuccess)
             e = launch_pdl(kern, dim3(grid), dim3(WARPS * 32), smem, st, (const uint8_t*)packed_gate, x, h, (float*)nullptr, (int)N,
-                           (int)K, tpr, 1, items, (const uint8_t*)packed_up);
+                           (int)K, tpr, 1, items, (const uint8_t*)packed_up, (int64_t)0, (int64_t)0);
     }
     return check_cuda(e, "qmm_gemv_gate_up launch");
 }
@@ -1097,6 +1108,67 @@ qmm_status launch_gemv_batch(int fmt, const qmm_gemv_problem* probs, int count, 
         if (e != cudaSuccess) return check_cuda(e, "qmm_gemv_batch launch");
     }
     return QMM_OK;
+}
+
+// qmm_gemm for two tokens: gemv_kernel's TWO form.  Returns QMM_ERR_UNSUPPORTED without touching the error text
+// when the shape needs the workspace form of the K split or more shared memory than a block has; the caller
+// then takes its other kernel.
+template <int FMT, int WARPS>
+static qmm_status launch_gemv_two_t(const GemvPlan& p, const void* packed, int64_t N, int64_t K, const uint16_t* X, int64_t ldx,
+                                    uint16_t* Y, int64_t ldy, cudaStream_t st)
+{
+    const bool cluster = p.splits > 1;
+    const size_t smem = (size_t)K * 6 + (size_t)WARPS * 128 * sizeof(float) + (cluster ? 2 * kMaxClusterSplits * 128 * sizeof(float) : 0);
+    if (smem > 227 * 1024) return QMM_ERR_UNSUPPORTED;
+    auto kern = gemv_kernel<FMT, WARPS, false, true>;
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return check_cuda(e, "qmm_gemm two-token kernel shared memory size");
+    }
+    const int tpr = (int)(K / Fmt<FMT>::tile_k);
+    const int items = (int)(N / (2 * kRowsPerGroup)) * p.splits;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(cluster ? p.grid / p.splits * p.splits : p.grid));
+    cfg.blockDim = dim3(WARPS * 32);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = (unsigned)p.splits;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = cluster ? 2 : 1;
+    return check_cuda(cudaLaunchKernelEx(&cfg, kern, (const uint8_t*)packed, X, Y, (float*)nullptr, (int)N, (int)K, tpr, p.splits, items,
+                                         (const uint8_t*)nullptr, ldx, ldy),
+                      "qmm_gemm two-token kernel launch");
+}
+
+bool gemv_two_supported(int fmt, int64_t N, int64_t K)
+{
+    if (K > 32768 || g_knobs.gemv_no_cluster) return false;
+    const GemvPlan p = gemv_plan(fmt, N, K, true);
+    return p.splits <= kMaxClusterSplits;
+}
+
+qmm_status launch_gemv_two(int fmt, const void* packed, int64_t N, int64_t K, const uint16_t* X, int64_t ldx, uint16_t* Y,
+                           int64_t ldy, cudaStream_t st)
+{
+    const GemvPlan p = gemv_plan(fmt, N, K, true);
+#define QMM_GEMV2_CASE(F, W) \
+    if (fmt == F && p.warps == W) return launch_gemv_two_t<F, W>(p, packed, N, K, X, ldx, Y, ldy, st);
+    QMM_GEMV2_CASE(QMM_Q4, 8)
+    QMM_GEMV2_CASE(QMM_Q4, 16)
+    QMM_GEMV2_CASE(QMM_Q8, 8)
+    QMM_GEMV2_CASE(QMM_Q8, 16)
+    QMM_GEMV2_CASE(QMM_Q5, 8)
+    QMM_GEMV2_CASE(QMM_Q5, 16)
+    QMM_GEMV2_CASE(QMM_Q6, 8)
+    QMM_GEMV2_CASE(QMM_Q6, 16)
+#undef QMM_GEMV2_CASE
+    return QMM_ERR_UNSUPPORTED;
 }
 
 // qmm_gemm_batch for two tokens: the batched kernel's TWO form (both tokens at the cost of one).

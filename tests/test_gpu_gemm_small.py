@@ -59,19 +59,27 @@ def test_few_tokens_many_items_per_block(qmm, oracle, fmt, N, K):
 
 @pytest.mark.parametrize("fmt", [4, 8])
 def test_a_token_row_does_not_depend_on_the_other_tokens(qmm, fmt):
-    """Row m of Y is the same bits whatever M is (2..8) and whichever slot of the token group it rides in:
-    the order of its fp32 additions is fixed by the shape alone.  A repeated call gives the same bits."""
+    """Row m of Y is the same bits whatever M is (3..8) and whichever slot of the token group it rides in:
+    the order of its fp32 additions is fixed by the shape alone.  A repeated call gives the same bits.
+    One and two tokens run on the single-token kernel: their rows are the bits of qmm_gemv."""
     for N, K in ((256, 2048), (128, 8192), (640, 512)):
         blocks = synth.quantize(fmt, synth.weights(83, fmt, N, K))
         packed = qmm.pack(fmt, util.dev(blocks), N, K)
         X = util.dev(synth.activations(83, N + K, 8, K))
         Y8 = gemm(qmm, fmt, packed, N, K, X)
         assert torch.equal(Y8, gemm(qmm, fmt, packed, N, K, X))
-        for M in (2, 3, 5, 7):
+        for M in (3, 5, 7):
             assert torch.equal(gemm(qmm, fmt, packed, N, K, X[:M]), Y8[:M])
-        # token 5 in the first slot of the group, and in the second slot behind token 0
-        assert torch.equal(gemm(qmm, fmt, packed, N, K, X[5:7])[0], Y8[5])
-        assert torch.equal(gemm(qmm, fmt, packed, N, K, X[[0, 5]].contiguous())[1], Y8[5])
+        # token 5 in the first slot of the group, and in the third slot behind tokens 0 and 1
+        assert torch.equal(gemm(qmm, fmt, packed, N, K, X[5:8])[0], Y8[5])
+        assert torch.equal(gemm(qmm, fmt, packed, N, K, X[[0, 1, 5]].contiguous())[2], Y8[5])
+        # two tokens: each row as qmm_gemv computes it, whichever of the two it is
+        y3, y6 = qmm.gemv(fmt, packed, N, K, X[3].contiguous()), qmm.gemv(fmt, packed, N, K, X[6].contiguous())
+        Y2 = gemm(qmm, fmt, packed, N, K, X[[3, 6]].contiguous())
+        assert torch.equal(Y2[0], y3) and torch.equal(Y2[1], y6)
+        Y2 = gemm(qmm, fmt, packed, N, K, X[[6, 3]].contiguous())
+        assert torch.equal(Y2[0], y6) and torch.equal(Y2[1], y3)
+        assert torch.equal(gemm(qmm, fmt, packed, N, K, X[3:4])[0], y3)
 
 
 @pytest.mark.parametrize("fmt", FMTS)
