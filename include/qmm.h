@@ -297,8 +297,8 @@ qmm_status qmm_chain_run(const qmm_chain_info* info, void* stream);
  * kernel of the decode family instead: integer codes times activations on the
  * warp-level tensor path, scales applied in fp32, no workspace use; row m of Y
  * is then the same bits whatever the other rows hold and whatever M in 3..8 is
- * (M = 1 and M = 2 run on the qmm_gemv kernel -- two tokens cost what one costs
- * there -- and give each row the bits of qmm_gemv).
+ * (M = 1 and M = 2 run on the qmm_gemv kernel -- two tokens cost little more
+ * than one there -- and give each row the bits of qmm_gemv).
  *   X_fp16  device, [M, ldx] fp16 row-major, ldx >= K, ldx % 8 == 0
  *   Y_fp16  device, [M, ldy] fp16 row-major, ldy >= N, ldy % 8 == 0, written
  *   ws      device, at least qmm_gemm_workspace_bytes(...) bytes: the status
@@ -322,8 +322,8 @@ qmm_status qmm_gemm(qmm_format fmt, const void* packed, int64_t N, int64_t K,
  * tokens).  The products must be independent, as for qmm_gemv_batch.  Integer
  * codes times activations, scales applied in fp32 (the accuracy of the GEMVs);
  * row m of Y_i does not depend on the other rows, nor on M within 3..8 (one and
- * two tokens run on the single-token batched kernel: two tokens cost what one
- * costs there).  No workspace.
+ * two tokens run on the single-token batched kernel: two tokens cost little
+ * more than one there).  No workspace.
  *   problems  HOST array of `count` descriptors (read during the call only);
  *             pointers inside are device pointers: packed 32-byte aligned,
  *             X [M, ldx] and Y [M, ldy] fp16 row-major, 16-byte aligned,
